@@ -1,0 +1,159 @@
+"""CPU oracle for the DVM hot path -- TEST INFRASTRUCTURE, not a product path.
+
+What the device-side virtual machine must produce is, by construction of the
+method, the same tensors as evaluating the fused program's basic operators one
+after another on whole tensors: fusion only replaces global-memory round trips
+by local memory (Sec. 5.1, "Pattern-based fusion") and tiling only partitions
+the iteration space (Sec. 4.2, "Shape tiling").  So this oracle is that plain
+definition: it walks the op program in order and materialises every
+intermediate as a whole float64 numpy array.  No tiling, no fusion, no
+bytecode, no blocking.  It shares no code with the encoder or the CUDA
+kernels and imports nothing from the product package.
+
+Arithmetic: every value is float64.  bf16 / fp32 inputs are widened exactly by
+the caller.  A "cast" node in the middle of a program is a semantic rounding
+point (Table 1, Cast) and rounds to the target format (nearest-even) before
+widening again; the device's implicit fp32 working precision is NOT emulated.
+Outputs are returned unrounded in float64.
+
+Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
+  Add/Sub/Mul/Div/Min/Max  elementwise                       (Table 1, binary rows)
+  Adds/Muls                x op scalar                        (Table 1, Adds/Muls)
+  Sqrt/Abs/Log/Exp/Round/Floor                                (Table 1, unary rows)
+  Cast                     (dst_dtype)(x)                     (Table 1, Cast)
+  Sum/Max/Min reduce       [M,size,N] -> [M,1,N], here N = 1  (Table 1, Sum/Max/Min)
+  Broadcast                implicit in numpy-style broadcasting (Table 1, Broadcast)
+Extensions that the benchmark programs need and Table 1 lacks (stated as such
+in the design doc): erf, sigmoid(x) = 1/(1+exp(-x)), rsqrt(x) = 1/sqrt(x),
+recip, neg, tanh, and matmul C[i,j] = sum_k A[i,k] B[k,j] (the paper's cube
+operation, Sec. 4.2, described in prose only).
+
+Pins (tests/test_oracle_pins.py): closed forms (softmax rows sum to 1, causal
+row i is 1/(i+1) for equal scores, RMSNorm unit RMS, LayerNorm zero mean /
+unit variance, GELU/sigmoid identities), torch float64 library routines on the
+special cases they cover, a pure-Python scalar evaluator on tiny inputs, and a
+triple-loop matmul.  NaN propagation in min/max, pow and log of non-positive
+numbers are "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+from scipy import special as _special
+
+__all__ = ["evaluate", "round_to_bf16", "round_to_f32"]
+
+
+def round_to_f32(x: np.ndarray) -> np.ndarray:
+    """Nearest-even rounding of float64 to the fp32 grid, returned as float64."""
+    with np.errstate(over="ignore"):
+        return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest-even rounding of float64 to the bfloat16 grid, returned as float64.
+
+    bf16 is the top 16 bits of an fp32 word.  Rounding goes through fp32; when
+    the fp32 value sits exactly on a bf16 tie although x did not, the tie is
+    broken towards x so that the result is the single correct rounding of x.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        y = x.astype(np.float32)
+    u = y.view(np.uint32).astype(np.uint64)
+    low = u & 0xFFFF
+    base = u & 0xFFFF0000
+    up = base + 0x10000
+    is_tie = low == 0x8000
+    # direction of the discarded part of x relative to the fp32 value y
+    mag_gt = np.abs(x) > np.abs(y.astype(np.float64))
+    mag_lt = np.abs(x) < np.abs(y.astype(np.float64))
+    even_up = ((u >> 16) & 1) == 1
+    round_up = np.where(is_tie, np.where(mag_gt, True, np.where(mag_lt, False, even_up)),
+                        low > 0x8000)
+    r = np.where(round_up, up, base).astype(np.uint32)
+    out = r.view(np.float32).astype(np.float64)
+    # NaN / inf keep their class
+    out = np.where(np.isnan(x), np.nan, out)
+    out = np.where(np.isinf(x), x, out)
+    return out.reshape(x.shape)
+
+
+def _round_to(x, dtype):
+    if dtype == "f32":
+        return round_to_f32(x)
+    if dtype == "bf16":
+        return round_to_bf16(x)
+    raise ValueError(f"unknown dtype {dtype}")
+
+
+_UNARY = {
+    "exp": np.exp,                                   # Table 1, Exp
+    "sqrt": np.sqrt,                                 # Table 1, Sqrt
+    "abs": np.abs,                                   # Table 1, Abs
+    "log": np.log,                                   # Table 1, Log
+    "floor": np.floor,                               # Table 1, Floor
+    "round": np.rint,                                # Table 1, Round (half to even)
+    "rsqrt": lambda x: 1.0 / np.sqrt(x),             # extension
+    "erf": _special.erf,                             # extension
+    "sigmoid": lambda x: 1.0 / (1.0 + np.exp(-x)),   # extension
+    "neg": lambda x: -x,                             # extension
+    "recip": lambda x: 1.0 / x,                      # extension
+    "tanh": np.tanh,                                 # extension
+}
+
+_BINARY = {
+    "add": lambda a, b: a + b,                       # Table 1, Add
+    "sub": lambda a, b: a - b,                       # Table 1, Sub
+    "mul": lambda a, b: a * b,                       # Table 1, Mul
+    "div": lambda a, b: a / b,                       # Table 1, Div
+    "max": lambda a, b: np.where(a > b, a, b),       # Table 1, Max
+    "min": lambda a, b: np.where(a < b, a, b),       # Table 1, Min
+}
+
+_REDUCE = {
+    "sum": lambda x: np.sum(x, axis=-1, keepdims=True),   # Table 1, Sum with N = 1
+    "max": lambda x: np.max(x, axis=-1, keepdims=True),   # Table 1, Max (reduce)
+    "min": lambda x: np.min(x, axis=-1, keepdims=True),   # Table 1, Min (reduce)
+}
+
+
+def evaluate(nodes, inputs, params=()):
+    """Evaluate an op program node by node on whole tensors.
+
+    nodes  : list of node tuples (see the workload module's docstring).
+    inputs : float64 numpy arrays, one per "input" node, in order; shapes may
+             broadcast against each other numpy-style (right-aligned).
+    params : runtime scalar arguments referenced by ("param", k).
+    Returns the list of outputs (float64, unrounded), in "output"-node order.
+    """
+    vals = [None] * len(nodes)
+    outs = []
+    it = iter(inputs)
+    with np.errstate(all="ignore"):
+        for i, n in enumerate(nodes):
+            kind = n[0]
+            if kind == "input":
+                a = np.asarray(next(it), dtype=np.float64)
+                if a.ndim != n[2]:
+                    raise ValueError(f"input node {i}: rank {a.ndim} != declared {n[2]}")
+                vals[i] = a
+            elif kind == "unary":
+                vals[i] = _UNARY[n[1]](vals[n[2]])
+            elif kind == "binary":
+                vals[i] = _BINARY[n[1]](vals[n[2]], vals[n[3]])
+            elif kind == "scalar":
+                s = n[3]
+                # the scalar is an fp32 immediate widened exactly (Table 1, Adds/Muls)
+                s = float(np.float32(params[s[1]] if isinstance(s, tuple) else s))
+                vals[i] = vals[n[2]] + s if n[1] == "adds" else vals[n[2]] * s
+            elif kind == "cast":
+                vals[i] = _round_to(vals[n[1]], n[2])
+            elif kind == "reduce":
+                vals[i] = _REDUCE[n[1]](vals[n[2]])
+            elif kind == "matmul":
+                vals[i] = np.matmul(vals[n[1]], vals[n[2]])
+            elif kind == "output":
+                outs.append(np.array(vals[n[1]], dtype=np.float64))
+            else:
+                raise ValueError(f"unknown node kind {kind}")
+    return outs

@@ -1,0 +1,395 @@
+"""Pins for the CPU oracle: things the paper and the mathematics fix, none of
+which is the oracle's own formula retyped.
+
+ * a scalar, pure-Python evaluator (math module, explicit broadcast indexing)
+   as brute force on tiny inputs;
+ * closed forms of each benchmark program;
+ * torch float64 library routines on the special cases they cover;
+ * hand-computed bf16 rounding cases.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import dvm_workloads as wl
+from oracle import dvm_oracle as orc
+
+RNG = np.random.default_rng(12345)
+
+
+# ---------------------------------------------------------------- brute force
+def _bcast_index(idx, shape, out_rank):
+    """Index into an array of `shape` for output index `idx` (right-aligned)."""
+    pad = out_rank - len(shape)
+    return tuple(0 if shape[d] == 1 else idx[pad + d] for d in range(len(shape)))
+
+
+def brute(nodes, inputs, params=()):
+    """Element-by-element evaluation with Python floats.  Tiny inputs only."""
+    un = {"exp": math.exp, "sqrt": math.sqrt, "abs": abs, "log": math.log,
+          "floor": math.floor, "erf": math.erf, "neg": lambda v: -v,
+          "rsqrt": lambda v: 1.0 / math.sqrt(v), "recip": lambda v: 1.0 / v,
+          "sigmoid": lambda v: 1.0 / (1.0 + math.exp(-v)), "tanh": math.tanh,
+          "round": lambda v: float(round(v))}   # Python round() is half-to-even
+    bi = {"add": lambda a, b: a + b, "sub": lambda a, b: a - b, "mul": lambda a, b: a * b,
+          "div": lambda a, b: a / b, "max": max, "min": min}
+    vals, shapes, outs = {}, {}, []
+    it = iter(inputs)
+    for i, n in enumerate(nodes):
+        k = n[0]
+        if k == "input":
+            a = np.asarray(next(it), dtype=np.float64)
+            shapes[i] = a.shape
+            vals[i] = {idx: float(a[idx]) for idx in np.ndindex(a.shape)}
+        elif k in ("unary", "scalar", "cast"):
+            src = n[2] if k != "cast" else n[1]
+            shapes[i] = shapes[src]
+            if k == "unary":
+                f = un[n[1]]
+            elif k == "scalar":
+                s = n[3]
+                s = float(np.float32(params[s[1]] if isinstance(s, tuple) else s))
+                f = (lambda v, s=s: v + s) if n[1] == "adds" else (lambda v, s=s: v * s)
+            else:
+                tdt = torch.bfloat16 if n[2] == "bf16" else torch.float32
+                f = lambda v, tdt=tdt: float(torch.tensor(v, dtype=torch.float64).to(tdt))
+            vals[i] = {idx: f(v) for idx, v in vals[src].items()}
+        elif k == "binary":
+            sa, sb = shapes[n[2]], shapes[n[3]]
+            r = max(len(sa), len(sb))
+            pa, pb = (1,) * (r - len(sa)) + sa, (1,) * (r - len(sb)) + sb
+            so = tuple(max(x, y) for x, y in zip(pa, pb))
+            shapes[i] = so
+            vals[i] = {idx: bi[n[1]](vals[n[2]][_bcast_index(idx, sa, r)],
+                                     vals[n[3]][_bcast_index(idx, sb, r)])
+                       for idx in np.ndindex(so)}
+        elif k == "reduce":
+            s = shapes[n[2]]
+            so = s[:-1] + (1,)
+            shapes[i] = so
+            red = {"sum": sum, "max": max, "min": min}[n[1]]
+            vals[i] = {idx: red(vals[n[2]][idx[:-1] + (j,)] for j in range(s[-1]))
+                       for idx in np.ndindex(so)}
+        elif k == "matmul":
+            (M, K), (K2, N) = shapes[n[1]], shapes[n[2]]
+            assert K == K2
+            shapes[i] = (M, N)
+            vals[i] = {(r, c): sum(vals[n[1]][(r, kk)] * vals[n[2]][(kk, c)] for kk in range(K))
+                       for r in range(M) for c in range(N)}
+        elif k == "output":
+            o = np.empty(shapes[n[1]])
+            for idx, v in vals[n[1]].items():
+                o[idx] = v
+            outs.append(o)
+    return outs
+
+
+def _tiny_inputs(prog, shapes):
+    ins = []
+    for s in shapes:
+        ins.append(RNG.normal(size=s))
+    return ins
+
+
+TINY = [
+    (wl.program_c1(), [(3, 5)] * 3, ()),
+    (wl.program_add_rmsnorm(hidden=6), [(4, 6), (4, 6), (6,)], ()),
+    (wl.program_masked_softmax(), [(2, 3, 4, 4), (1, 1, 4, 4)], ()),
+    (wl.program_gelu_affine(), [(3, 7), (1, 7), (1, 7)], ()),
+    (wl.program_layernorm(), [(3, 9)], (1.0 / 9,)),
+    (wl.program_sigmoid_mul(), [(2, 5), (2, 5)], ()),
+    (wl.program_mlp_gate(), [(3, 4), (4, 5), (4, 5)], ()),
+    (wl.program_add_sqrt(), [(2, 3), (2, 3)], ()),
+]
+
+
+@pytest.mark.parametrize("prog,shapes,params", TINY, ids=[t[0].name for t in TINY])
+def test_matches_scalar_brute_force(prog, shapes, params):
+    ins = _tiny_inputs(prog, shapes)
+    if prog.name == "add_sqrt":
+        ins = [np.abs(a) for a in ins]
+    got = orc.evaluate(prog.nodes, ins, params)
+    want = brute(prog.nodes, ins, params)
+    assert len(got) == len(want)
+    for g, w in zip(got, want):
+        assert g.shape == w.shape
+        np.testing.assert_allclose(g, w, rtol=1e-13, atol=1e-15)
+
+
+def test_every_primitive_against_brute_force():
+    x = RNG.uniform(0.1, 3.0, size=(2, 5))
+    y = RNG.uniform(0.1, 3.0, size=(1, 5))
+    for op in wl.UNARY_OPS:
+        p = wl.OpProgram()
+        a = p.input("f32", 2)
+        p.output(p.unary(op, a), "f32")
+        xx = x - 1.5 if op in ("abs", "floor", "round", "neg", "erf", "tanh", "sigmoid", "exp") else x
+        np.testing.assert_allclose(orc.evaluate(p.nodes, [xx])[0], brute(p.nodes, [xx])[0], rtol=1e-14)
+    for op in wl.BINARY_OPS:
+        p = wl.OpProgram()
+        a, b = p.input("f32", 2), p.input("f32", 2)
+        p.output(p.binary(op, a, b), "f32")
+        np.testing.assert_allclose(orc.evaluate(p.nodes, [x - 1, y - 1])[0],
+                                   brute(p.nodes, [x - 1, y - 1])[0], rtol=1e-14)
+    for op in wl.REDUCE_OPS:
+        p = wl.OpProgram()
+        a = p.input("f32", 2)
+        p.output(p.reduce(op, a), "f32")
+        np.testing.assert_allclose(orc.evaluate(p.nodes, [x])[0], brute(p.nodes, [x])[0], rtol=1e-14)
+
+
+# ---------------------------------------------------------------- primitives: exact identities
+def test_primitive_identities():
+    def run1(kind, op, x, *extra):
+        p = wl.OpProgram()
+        a = p.input("f32", 1)
+        v = getattr(p, kind)(op, a, *extra)
+        p.output(v, "f32")
+        return orc.evaluate(p.nodes, [np.asarray(x, dtype=np.float64)])[0]
+
+    assert run1("unary", "exp", [0.0])[0] == 1.0
+    assert run1("unary", "sqrt", [4.0])[0] == 2.0
+    assert run1("unary", "log", [1.0])[0] == 0.0
+    assert run1("unary", "abs", [-3.5])[0] == 3.5
+    assert run1("unary", "rsqrt", [0.25])[0] == 2.0
+    assert run1("unary", "recip", [8.0])[0] == 0.125
+    assert run1("unary", "sigmoid", [0.0])[0] == 0.5
+    assert run1("unary", "erf", [0.0])[0] == 0.0
+    assert list(run1("unary", "floor", [-1.5, 1.5])) == [-2.0, 1.0]
+    assert list(run1("unary", "round", [0.5, 1.5, 2.5, -0.5])) == [0.0, 2.0, 2.0, -0.0]
+    assert run1("scalar", "adds", [1.0], 0.5)[0] == 1.5
+    assert run1("scalar", "muls", [3.0], 0.5)[0] == 1.5
+    # Adds/Muls equal Add/Mul with a broadcast scalar tensor
+    x = RNG.normal(size=(4, 3))
+    p = wl.OpProgram(); a = p.input("f32", 2); p.output(p.scalar("muls", a, 0.375), "f32")
+    q = wl.OpProgram(); a = q.input("f32", 2); s = q.input("f32", 2); q.output(q.binary("mul", a, s), "f32")
+    np.testing.assert_array_equal(orc.evaluate(p.nodes, [x])[0],
+                                  orc.evaluate(q.nodes, [x, np.full((1, 1), 0.375)])[0])
+
+
+def test_scalar_immediate_is_fp32():
+    p = wl.OpProgram(); a = p.input("f32", 1); p.output(p.scalar("muls", a, 0.1), "f32")
+    got = orc.evaluate(p.nodes, [np.array([1.0])])[0][0]
+    assert got == float(np.float32(0.1)) and got != 0.1
+
+
+def test_sub_div_operand_order():
+    p = wl.OpProgram(); a = p.input("f32", 1); b = p.input("f32", 1)
+    p.output(p.binary("sub", a, b), "f32"); p.output(p.binary("div", a, b), "f32")
+    s, d = orc.evaluate(p.nodes, [np.array([6.0]), np.array([2.0])])
+    assert s[0] == 4.0 and d[0] == 3.0
+
+
+# ---------------------------------------------------------------- rounding
+def test_bf16_rounding_hand_cases():
+    e = 2.0 ** -8          # half of the bf16 spacing at 1.0 (2^-7)
+    cases = {
+        1.0: 1.0,
+        1.0 + e: 1.0,                          # tie -> even (mantissa 0)
+        1.0 + 3 * e: 1.0 + 4 * e,              # tie -> even (mantissa 2)
+        1.0 + e + 2.0 ** -40: 1.0 + 2 * e,     # above the tie only in float64: double rounding trap
+        1.0 + e - 2.0 ** -40: 1.0,
+        -(1.0 + e + 2.0 ** -40): -(1.0 + 2 * e),
+        3.140625: 3.140625,                    # exactly representable
+        0.0: 0.0,
+    }
+    got = orc.round_to_bf16(np.array(list(cases.keys())))
+    np.testing.assert_array_equal(got, np.array(list(cases.values())))
+    assert np.isnan(orc.round_to_bf16(np.array([np.nan])))[0]
+    assert orc.round_to_bf16(np.array([-np.inf]))[0] == -np.inf
+
+
+def test_bf16_rounding_matches_torch_on_fp32_values():
+    x32 = torch.randn(20000, generator=torch.Generator().manual_seed(5)) * 37.0
+    want = x32.to(torch.bfloat16).to(torch.float64).numpy()
+    got = orc.round_to_bf16(x32.to(torch.float64).numpy())
+    np.testing.assert_array_equal(got, want)
+
+
+def test_cast_node_rounds():
+    p = wl.OpProgram(); a = p.input("f32", 1)
+    p.output(p.cast(a, "bf16"), "f32"); p.output(p.cast(a, "f32"), "f32")
+    x = np.array([1.0 + 2.0 ** -8 + 2.0 ** -40, 1.0 + 2.0 ** -30])
+    b, f = orc.evaluate(p.nodes, [x])
+    assert list(b) == [1.0 + 2.0 ** -7, 1.0]
+    assert list(f) == [float(np.float32(x[0])), 1.0]
+
+
+# ---------------------------------------------------------------- broadcasting
+def test_broadcast_equals_materialised():
+    p = wl.program_gelu_affine()
+    x, w, b = RNG.normal(size=(5, 8)), RNG.normal(size=(1, 8)), RNG.normal(size=(1, 8))
+    a = orc.evaluate(p.nodes, [x, w, b])[0]
+    c = orc.evaluate(p.nodes, [x, np.repeat(w, 5, 0), np.repeat(b, 5, 0)])[0]
+    np.testing.assert_array_equal(a, c)
+    # w = 1, b = 0 reduces the affine part to x: GELU(x) against torch
+    g = orc.evaluate(p.nodes, [x, np.ones((1, 8)), np.zeros((1, 8))])[0]
+    want = torch.nn.functional.gelu(torch.tensor(x, dtype=torch.float64)).numpy()
+    # 1/sqrt(2) enters as an fp32 immediate: relative error of the argument 3e-8
+    np.testing.assert_allclose(g, want, rtol=1e-6, atol=1e-8)
+
+    q = wl.program_masked_softmax()
+    s = RNG.normal(size=(2, 3, 6, 6))
+    m = wl.to_f64(wl.causal_mask(6))
+    a = orc.evaluate(q.nodes, [s, m])[0]
+    c = orc.evaluate(q.nodes, [s, np.broadcast_to(m, s.shape).copy()])[0]
+    np.testing.assert_array_equal(a, c)
+
+
+# ---------------------------------------------------------------- C1
+def test_c1_closed_forms():
+    p = wl.program_c1()
+    a, b, c = (wl.to_f64(t) for t in wl.inputs_c1())
+    out = orc.evaluate(p.nodes, [a, b, c])[0]
+    np.testing.assert_allclose(out, np.exp(a * b + c) - a, rtol=1e-15)
+    z = np.zeros_like(a)
+    np.testing.assert_array_equal(orc.evaluate(p.nodes, [a, z, z])[0], 1.0 - a)
+    np.testing.assert_array_equal(orc.evaluate(p.nodes, [z, b, c])[0], np.exp(c))
+
+
+# ---------------------------------------------------------------- softmax
+def test_softmax_closed_forms():
+    p = wl.program_masked_softmax()
+    B, H, S = 2, 3, 19
+    s, m = (wl.to_f64(t) for t in wl.inputs_masked_softmax(B, H, S, 11))
+    out = orc.evaluate(p.nodes, [s, m])[0]
+    assert out.shape == (B, H, S, S)
+    np.testing.assert_allclose(out.sum(-1), 1.0, rtol=0, atol=1e-14)       # rows sum to 1
+    assert np.all(out[..., 0, 0] == 1.0) and np.all(out[..., 0, 1:] == 0)    # causal row 0
+    iu = np.triu_indices(S, 1)
+    assert np.all(out[..., iu[0], iu[1]] == 0.0)                             # masked exactly +0
+    assert not np.any(np.signbit(out))
+    # equal scores: row i is 1/(i+1) on j <= i
+    eq = orc.evaluate(p.nodes, [np.full((1, 1, S, S), 0.75), m])[0][0, 0]
+    for i in range(S):
+        np.testing.assert_allclose(eq[i, :i + 1], 1.0 / (i + 1), rtol=1e-15)
+    # shift invariance
+    sh = orc.evaluate(p.nodes, [s + 3.0, m])[0]
+    np.testing.assert_allclose(sh, out, rtol=1e-12, atol=1e-18)
+    # library routine
+    scale = float(np.float32(1.0 / math.sqrt(128)))
+    want = torch.softmax((torch.tensor(s) + torch.tensor(m)) * scale, dim=-1).numpy()
+    np.testing.assert_allclose(out, want, rtol=1e-13, atol=1e-18)
+    # mask-then-scale equals scale-then-mask for a 0/-inf mask
+    alt = torch.softmax(torch.tensor(s) * scale + torch.tensor(m), dim=-1).numpy()
+    np.testing.assert_allclose(out, alt, rtol=1e-13, atol=1e-18)
+
+
+# ---------------------------------------------------------------- RMSNorm
+def test_rmsnorm_closed_forms():
+    Hd = 64
+    p = wl.program_add_rmsnorm(hidden=Hd, eps=1e-6)
+    x, res, w = (wl.to_f64(t) for t in wl.inputs_add_rmsnorm(9, Hd, 3))
+    y, h = orc.evaluate(p.nodes, [x, res, w])
+    np.testing.assert_array_equal(h, x + res)                         # residual stream is exact
+    ones = np.ones(Hd)
+    y1, _ = orc.evaluate(p.nodes, [x, res, ones])
+    ms = np.mean((x + res) ** 2, axis=-1)
+    np.testing.assert_allclose(np.sqrt(np.mean(y1 ** 2, -1)), np.sqrt(ms / (ms + 1e-6)), rtol=1e-9)
+    np.testing.assert_allclose(np.sqrt(np.mean(y1 ** 2, -1)), 1.0, atol=5e-6)   # unit RMS
+    np.testing.assert_allclose(y, y1 * w, rtol=1e-15)                 # weight applies elementwise
+    # constant row c -> c / sqrt(c^2 + eps)
+    c = 0.5
+    yc, _ = orc.evaluate(p.nodes, [np.full((1, Hd), c), np.zeros((1, Hd)), ones])
+    np.testing.assert_allclose(yc, c / math.sqrt(c * c + float(np.float32(1e-6))), rtol=1e-9)
+    # positive scale invariance up to eps
+    y4, _ = orc.evaluate(p.nodes, [4 * x, 4 * res, ones])
+    np.testing.assert_allclose(y4, y1, rtol=1e-5)
+    # library routine
+    want = torch.nn.functional.rms_norm(torch.tensor(x + res), (Hd,), torch.tensor(w),
+                                        eps=float(np.float32(1e-6))).numpy()
+    np.testing.assert_allclose(y, want, rtol=1e-9)
+
+
+# ---------------------------------------------------------------- LayerNorm
+def test_layernorm_closed_forms():
+    p = wl.program_layernorm()
+    cols = 37
+    x = RNG.normal(size=(6, cols)) * 3 + 1
+    (o,) = orc.evaluate(p.nodes, [x], (1.0 / cols,))
+    v = x.var(-1)
+    np.testing.assert_allclose(o.mean(-1), 0.0, atol=1e-7)   # 1/37 is an fp32 immediate
+    np.testing.assert_allclose(o.var(-1), v / (v + 1e-5), rtol=1e-6)
+    want = torch.nn.functional.layer_norm(torch.tensor(x), (cols,), eps=1e-5).numpy()
+    np.testing.assert_allclose(o, want, rtol=1e-6, atol=1e-7)   # 1/cols is an fp32 immediate
+    # exact-in-fp32 reciprocal: cols = 32
+    x32 = RNG.normal(size=(4, 32))
+    (o32,) = orc.evaluate(p.nodes, [x32], (1.0 / 32,))
+    want = torch.nn.functional.layer_norm(torch.tensor(x32), (32,), eps=float(np.float32(1e-5))).numpy()
+    np.testing.assert_allclose(o32, want, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(o32.mean(-1), 0.0, atol=1e-15)
+    (oc,) = orc.evaluate(p.nodes, [np.full((1, 32), 2.5)], (1.0 / 32,))
+    assert np.all(oc == 0.0)                                         # constant row -> 0
+    alt = np.tile([1.0, -1.0], 16)[None]
+    (oa,) = orc.evaluate(p.nodes, [alt], (1.0 / 32,))
+    np.testing.assert_allclose(oa, alt / math.sqrt(1 + float(np.float32(1e-5))), rtol=1e-14)
+
+
+# ---------------------------------------------------------------- GELU / sigmoid / SiLU
+def test_gelu_sigmoid_identities():
+    p = wl.program_gelu_affine()
+    t = RNG.normal(size=(3, 10)) * 2
+    one, zero = np.ones((1, 10)), np.zeros((1, 10))
+    g_pos = orc.evaluate(p.nodes, [t, one, zero])[0]
+    g_neg = orc.evaluate(p.nodes, [-t, one, zero])[0]
+    np.testing.assert_allclose(g_pos - g_neg, t, rtol=1e-6, atol=1e-7)   # 1/sqrt(2) is fp32
+    assert orc.evaluate(p.nodes, [np.zeros((1, 10)), one, zero])[0].max() == 0.0
+
+    q = wl.program_sigmoid_mul()
+    x, y = RNG.normal(size=(4, 6)) * 4, RNG.normal(size=(4, 6))
+    o = orc.evaluate(q.nodes, [x, y])[0]
+    on = orc.evaluate(q.nodes, [-x, y])[0]
+    np.testing.assert_allclose(o + on, y, rtol=1e-13)                    # s(x) + s(-x) = 1
+    np.testing.assert_array_equal(orc.evaluate(q.nodes, [np.zeros((4, 6)), y])[0], y / 2)
+    np.testing.assert_allclose(o, (torch.sigmoid(torch.tensor(x)) * torch.tensor(y)).numpy(), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- matmul + epilogue
+def test_mlp_gate_closed_forms():
+    p = wl.program_mlp_gate()
+    K, N = 8, 5
+    wg, wu = RNG.normal(size=(K, N)), RNG.normal(size=(K, N))
+    # X = I picks out the weight rows
+    o = orc.evaluate(p.nodes, [np.eye(K), wg, wu])[0]
+    np.testing.assert_allclose(o, wg / (1 + np.exp(-wg)) * wu, rtol=1e-14)
+    # W_gate = 0 -> 0
+    x = RNG.normal(size=(3, K))
+    assert np.all(orc.evaluate(p.nodes, [x, np.zeros((K, N)), wu])[0] == 0)
+    # all ones -> K * sigmoid(K) * K
+    o1 = orc.evaluate(p.nodes, [np.ones((2, K)), np.ones((K, N)), np.ones((K, N))])[0]
+    np.testing.assert_allclose(o1, K / (1 + math.exp(-K)) * K, rtol=1e-14)
+    # non-square, transposition-sensitive: triple loop
+    M = 4
+    g = np.zeros((M, N)); u = np.zeros((M, N))
+    xx = RNG.normal(size=(M, K))
+    for i in range(M):
+        for j in range(N):
+            for k in range(K):
+                g[i, j] += xx[i, k] * wg[k, j]
+                u[i, j] += xx[i, k] * wu[k, j]
+    want = torch.nn.functional.silu(torch.tensor(g)).numpy() * u
+    np.testing.assert_allclose(orc.evaluate(p.nodes, [xx, wg, wu])[0], want, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- fusion equivalence (Sec. 5.1)
+def test_fused_equals_chain_of_single_ops():
+    a, b = np.abs(RNG.normal(size=(3, 4))), np.abs(RNG.normal(size=(3, 4)))
+    fused = orc.evaluate(wl.program_add_sqrt().nodes, [a, b])[0]
+    p1 = wl.OpProgram(); i0 = p1.input("f32", 2); i1 = p1.input("f32", 2); p1.output(p1.binary("add", i0, i1), "f32")
+    p2 = wl.OpProgram(); i0 = p2.input("f32", 2); p2.output(p2.unary("sqrt", i0), "f32")
+    c = orc.evaluate(p1.nodes, [a, b])[0]
+    np.testing.assert_array_equal(fused, orc.evaluate(p2.nodes, [c])[0])
+
+
+def test_oracle_does_not_import_product():
+    import ast, os
+    src = open(os.path.join(os.path.dirname(orc.__file__), "dvm_oracle.py")).read()
+    mods = set()
+    for node in ast.walk(ast.parse(src)):
+        if isinstance(node, ast.Import):
+            mods |= {a.name.split(".")[0] for a in node.names}
+        elif isinstance(node, ast.ImportFrom):
+            mods.add((node.module or "").split(".")[0])
+    assert mods <= {"__future__", "numpy", "scipy"}, mods
