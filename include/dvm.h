@@ -1,0 +1,197 @@
+/* libdvm -- C ABI of the B200-native bytecode virtual machine for fused dynamic
+ * tensor operators.
+ *
+ * The calls follow the paper's statement of the problem (Sec. 3 "Operator
+ * Compiler", Sec. 4): given a computation graph of basic operators to fuse and
+ * the concrete input shapes of one instance, the host encodes a bytecode
+ * program (dvm_encode); the program is sent to the device, where a virtual
+ * machine decodes it into tile-level virtual instructions and executes them
+ * over the tiles of the runtime shape (dvm_launch); several independent
+ * meta-kernels may be stacked into one kernel (dvm_launch_stacked, Sec. 5.1
+ * "Stacking-based fusion").  Nothing is cached between instances.
+ *
+ * Conventions
+ *  - Every call returns an int status: DVM_OK (0) or a negative DVM_ERR_*.
+ *    No exception crosses the boundary, nothing traps.
+ *  - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global
+ *    memory of the current device.  The library never allocates, frees or
+ *    copies tensor memory and never synchronises a stream (dvm_run_host and
+ *    dvm_last_device_status are the documented exceptions).
+ *  - Tensors are dense row-major.  A dimension of size 1 broadcasts
+ *    numpy-style (right-aligned) against the other operands.
+ *  - Bytecode refers to tensor *slots* (inputs in declaration order, then
+ *    outputs in declaration order); device addresses are supplied at launch, so
+ *    one encoded program can be launched on any buffers of the encoded shapes.
+ */
+#ifndef DVM_H_
+#define DVM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DVM_MAX_RANK 6
+
+enum {
+  DVM_OK = 0,
+  DVM_ERR_INVALID_ARG = -1,      /* NULL pointer, bad id / enum, bad rank, misaligned element pointer */
+  DVM_ERR_SHAPE_MISMATCH = -2,   /* operands do not broadcast, matmul inner dims differ */
+  DVM_ERR_UNSUPPORTED = -3,      /* valid program the VM cannot run (row longer than the register
+                                    budget, too many live values, more than 3 non-mergeable outer dims) */
+  DVM_ERR_BUFFER_TOO_SMALL = -4, /* code buffer too small; *code_size receives the need */
+  DVM_ERR_BAD_CODE = -5,         /* bytecode failed verification */
+  DVM_ERR_CUDA = -6,             /* a CUDA runtime call failed; see dvm_last_cuda_error */
+  DVM_ERR_DEVICE_TIMEOUT = -7,   /* a bounded device-side wait ran out (status word) */
+  DVM_ERR_DEVICE_BAD_CODE = -8,  /* the interpreter met an instruction it cannot decode (status word) */
+  DVM_ERR_NOT_FINALIZED = -9,
+  DVM_ERR_TOO_LARGE = -10        /* program / stack exceeds a fixed library limit */
+};
+
+enum { DVM_F32 = 0, DVM_BF16 = 1 };
+
+/* Unary operators.  EXP SQRT ABS LOG FLOOR ROUND are Table 1's; the others are
+ * extensions the LLM programs need (Table 1 has no erf / sigmoid / rsqrt). */
+enum {
+  DVM_EXP = 0, DVM_SQRT = 1, DVM_RSQRT = 2, DVM_ABS = 3, DVM_LOG = 4, DVM_ERF = 5,
+  DVM_SIGMOID = 6, DVM_NEG = 7, DVM_RECIP = 8, DVM_FLOOR = 9, DVM_ROUND = 10, DVM_TANH = 11
+};
+/* Binary operators (Table 1: Add Sub Mul Div Min Max). */
+enum { DVM_ADD = 0, DVM_SUB = 1, DVM_MUL = 2, DVM_DIV = 3, DVM_MIN = 4, DVM_MAX = 5 };
+/* Tensor-scalar operators (Table 1: Adds, Muls). */
+enum { DVM_ADDS = 0, DVM_MULS = 1 };
+/* Row reductions over the last axis, keepdim (Table 1: Sum / Max / Min with N = 1). */
+enum { DVM_SUM = 0, DVM_RMAX = 1, DVM_RMIN = 2 };
+
+typedef struct dvm_program dvm_program; /* opaque; owned by the library */
+
+typedef struct {
+  int32_t rank;                /* 0 <= rank <= DVM_MAX_RANK */
+  int64_t dims[DVM_MAX_RANK];  /* row-major, dense */
+} dvm_shape;
+
+/* ------------------------------------------------------------------------
+ * Program description: the shape-agnostic "computation graph of basic
+ * operators to fuse" (Sec. 3).  Built once, immutable after finalize, shared
+ * by every instance.  Each builder call appends one node and returns its
+ * value id in *value_id; operands must be earlier value ids.
+ * All pointers are host pointers.
+ * ---------------------------------------------------------------------- */
+int dvm_program_create(dvm_program** out);
+void dvm_program_destroy(dvm_program* p); /* NULL is allowed */
+
+/* A global-memory input of the given element type and rank. */
+int dvm_program_input(dvm_program* p, int dtype, int rank, int* value_id);
+/* Table 1 unary rows (Sqrt Abs Log Exp Round Floor) + extensions. */
+int dvm_program_unary(dvm_program* p, int op, int x, int* value_id);
+/* Table 1 binary rows; operands broadcast (Table 1, Broadcast). */
+int dvm_program_binary(dvm_program* p, int op, int x, int y, int* value_id);
+/* Table 1 Adds / Muls with an fp32 immediate. */
+int dvm_program_scalar(dvm_program* p, int op, int x, float s, int* value_id);
+/* Same, the scalar being runtime argument `param` of dvm_encode (e.g. 1/cols). */
+int dvm_program_scalar_param(dvm_program* p, int op, int x, int param, int* value_id);
+/* Table 1 Cast: rounds the value to `dtype` (nearest even); values stay fp32 in registers. */
+int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
+/* Table 1 Sum / Max / Min over the last axis (axis must be -1), size-1 axis kept. */
+int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id);
+/* The cube operation (Sec. 4.2, matrix operations): a [M,K] x b [K,N], bf16 inputs, fp32 value.
+ * Both operands must be program inputs; every matmul of a program shares `a`. */
+int dvm_program_matmul(dvm_program* p, int a, int b, int* value_id);
+/* Marks value x as an output stored with element type `dtype` (cast on store). */
+int dvm_program_output(dvm_program* p, int x, int dtype);
+/* Validates the graph.  Required before dvm_encode. */
+int dvm_program_finalize(dvm_program* p);
+int dvm_program_num_inputs(const dvm_program* p);
+int dvm_program_num_outputs(const dvm_program* p);
+
+/* ------------------------------------------------------------------------
+ * Per-instance encode (Sec. 4.2: shape tiling, then bytecode encoding).
+ * Pure CPU, no CUDA call, no heap allocation; thread-safe on a finalized
+ * program.
+ *   in_shapes[n_in]    concrete input shapes, in input order
+ *   scalars[n_scalars] runtime scalar arguments (may be NULL when n_scalars = 0)
+ *   code               caller-owned host buffer of code_capacity bytes, 8-byte aligned
+ *   *code_size         receives the encoded size in bytes (also on BUFFER_TOO_SMALL)
+ *   out_shapes[n_out]  receives the inferred output shapes (may be NULL)
+ * ---------------------------------------------------------------------- */
+int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
+               const float* scalars, int n_scalars,
+               void* code, size_t code_capacity, size_t* code_size,
+               dvm_shape* out_shapes, int n_out);
+/* Upper bound of the encoded size, in bytes, for any shape. */
+size_t dvm_code_max_size(const dvm_program* p);
+
+/* Number of parallel units N the tiling cost model balances for (Sec. 4.2: cost
+ * = ceil(#tiles / N) * (tile + overhead)).  Default 148 SMs x 3 resident CTAs.
+ * n <= 0 restores the default.  Process-wide; not thread-safe against encode. */
+void dvm_set_num_cores(int n);
+int dvm_get_num_cores(void);
+
+/* The paper's tile-size rule for a flat vector operator (Sec. 4.2,
+ * hardware_align_div): among tile sizes t in [1, min(total, t_max)] take the
+ * one minimising ceil(ceil(total / t) / n_cores) * (t + overhead) (ties: the
+ * larger t), then round it up to a multiple of `align` elements without
+ * exceeding t_max.  Outputs (each may be NULL): the min-cost tile, the rounded
+ * tile, the tile count and tail size for the min-cost tile.  Host only. */
+int dvm_hardware_align_div(int64_t total, int n_cores, int64_t align, int64_t t_max,
+                           int64_t overhead, int64_t* min_cost_tile, int64_t* rounded_tile,
+                           int64_t* n_tiles, int64_t* tail);
+
+/* Algorithm 2's tile range of core `id`: m = ceil(M / N), [m*id, min(M, m*(id+1))). */
+int dvm_vm_tile_range(int64_t n_tiles, int n_cores, int id, int64_t* begin, int64_t* end);
+
+/* ------------------------------------------------------------------------
+ * Launch (Sec. 4.3, Algorithm 2).  Asynchronous on `cuda_stream` (a
+ * cudaStream_t passed as void*; NULL = default stream).  `code` is a host
+ * pointer; it is copied into the launch, so the caller may reuse it when the
+ * call returns.  tensors[n_tensors] are DEVICE pointers, inputs then outputs,
+ * caller-owned, element-aligned; they must stay valid until the stream has run
+ * the kernel.  Zero-size instances launch nothing.
+ * ---------------------------------------------------------------------- */
+int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_tensors,
+               void* cuda_stream);
+
+/* Stacking-based fusion (Sec. 5.1): n_programs independent vector meta-kernels
+ * run as ONE kernel; their tiles are claimed from one work queue, spread over
+ * SMs (spatial) and run back to back on each SM (temporal).
+ * codes[i] / code_sizes[i] / tensors[i] / n_tensors[i] as for dvm_launch. */
+int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
+                       void* const* const* tensors, const int* n_tensors, void* cuda_stream);
+
+/* End-to-end convenience for HOST tensors: copies the inputs to device staging
+ * memory the caller provides (`staging`, device pointer, staging_bytes >= sum of
+ * all tensor sizes rounded up to 256 B each), launches, copies the outputs back
+ * and synchronises the stream.  host_tensors[i] has tensor_bytes[i] bytes;
+ * pinned host memory makes the copies asynchronous. */
+int dvm_run_host(const void* code, size_t code_size, void* const* host_tensors,
+                 const size_t* tensor_bytes, int n_tensors, void* staging, size_t staging_bytes,
+                 void* cuda_stream);
+
+/* ------------------------------------------------------------------------
+ * Support
+ * ---------------------------------------------------------------------- */
+/* Host-side validation of a bytecode program (every instruction id, length,
+ * register, operand and slot index, table sizes).  dvm_launch runs it too. */
+int dvm_verify(const void* code, size_t code_size);
+/* Readable dump (the paper's Fig. 5 prints one: tile count, per-core tiles,
+ * kernel type, one line per operation).  Returns DVM_ERR_BUFFER_TOO_SMALL if
+ * `cap` is too small; the text is always NUL-terminated when cap > 0. */
+int dvm_disassemble(const void* code, size_t code_size, char* buf, size_t cap);
+/* Header fields of an encoded program (each output may be NULL). */
+int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t* n_tiles,
+                  int* code_body_bytes, int* threads_per_row, int* vector_width, int* n_tile_regs);
+/* Synchronises `cuda_stream`, then reads and clears the device status word of
+ * the current device: *status is DVM_OK or a DVM_ERR_DEVICE_* code. */
+int dvm_last_device_status(void* cuda_stream, int* status);
+/* The cudaError_t (as int) of the last failed CUDA call on this thread. */
+int dvm_last_cuda_error(void);
+/* Number of kernels this library has launched in this process. */
+int64_t dvm_launch_count(void);
+const char* dvm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DVM_H_ */

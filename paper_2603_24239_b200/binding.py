@@ -1,0 +1,318 @@
+"""ctypes binding of libdvm.so: argument marshalling only.
+
+Every step of the hot path (shape tiling, bytecode encoding, the virtual
+machine) runs inside the library.  If the library is missing the import fails
+loudly -- there is no other implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Iterable, List, Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdvm.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is not built. Run `python -m paper_2603_24239_b200.build` "
+        "(or __graft_entry__.build()); the library has no CPU fallback.")
+lib = C.CDLL(LIB_PATH)
+
+DVM_MAX_RANK = 6
+F32, BF16 = 0, 1
+DTYPES = {"f32": F32, "bf16": BF16}
+UNARY = {"exp": 0, "sqrt": 1, "rsqrt": 2, "abs": 3, "log": 4, "erf": 5, "sigmoid": 6, "neg": 7,
+         "recip": 8, "floor": 9, "round": 10, "tanh": 11}
+BINARY = {"add": 0, "sub": 1, "mul": 2, "div": 3, "min": 4, "max": 5}
+SCALAR = {"adds": 0, "muls": 1}
+REDUCE = {"sum": 0, "max": 1, "min": 2}
+
+
+class Shape(C.Structure):
+    _fields_ = [("rank", C.c_int32), ("dims", C.c_int64 * DVM_MAX_RANK)]
+
+
+class DvmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib.dvm_strerror(status).decode()
+        if status == -6:
+            msg += f" (cudaError {lib.dvm_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+
+
+_vp, _i, _sz = C.c_void_p, C.c_int, C.c_size_t
+_pi = C.POINTER(C.c_int)
+_p64 = C.POINTER(C.c_int64)
+_sig = {
+    "dvm_program_create": ([C.POINTER(_vp)], _i),
+    "dvm_program_destroy": ([_vp], None),
+    "dvm_program_input": ([_vp, _i, _i, _pi], _i),
+    "dvm_program_unary": ([_vp, _i, _i, _pi], _i),
+    "dvm_program_binary": ([_vp, _i, _i, _i, _pi], _i),
+    "dvm_program_scalar": ([_vp, _i, _i, C.c_float, _pi], _i),
+    "dvm_program_scalar_param": ([_vp, _i, _i, _i, _pi], _i),
+    "dvm_program_cast": ([_vp, _i, _i, _pi], _i),
+    "dvm_program_reduce": ([_vp, _i, _i, _i, _pi], _i),
+    "dvm_program_matmul": ([_vp, _i, _i, _pi], _i),
+    "dvm_program_output": ([_vp, _i, _i], _i),
+    "dvm_program_finalize": ([_vp], _i),
+    "dvm_program_num_inputs": ([_vp], _i),
+    "dvm_program_num_outputs": ([_vp], _i),
+    "dvm_encode": ([_vp, C.POINTER(Shape), _i, C.POINTER(C.c_float), _i, _vp, _sz, C.POINTER(_sz),
+                    C.POINTER(Shape), _i], _i),
+    "dvm_code_max_size": ([_vp], _sz),
+    "dvm_set_num_cores": ([_i], None),
+    "dvm_get_num_cores": ([], _i),
+    "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
+    "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
+    "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
+    "dvm_launch_stacked": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _vp], _i),
+    "dvm_run_host": ([_vp, _sz, C.POINTER(_vp), C.POINTER(_sz), _i, _vp, _sz, _vp], _i),
+    "dvm_verify": ([_vp, _sz], _i),
+    "dvm_disassemble": ([_vp, _sz, C.c_char_p, _sz], _i),
+    "dvm_code_info": ([_vp, _sz, _pi, _p64, _pi, _pi, _pi, _pi], _i),
+    "dvm_last_device_status": ([_vp, _pi], _i),
+    "dvm_last_cuda_error": ([], _i),
+    "dvm_launch_count": ([], C.c_int64),
+    "dvm_strerror": ([_i], C.c_char_p),
+}
+for _name, (_args, _res) in _sig.items():
+    _f = getattr(lib, _name)
+    _f.argtypes = _args
+    _f.restype = _res
+EXPORTS = tuple(_sig)
+
+
+def _check(st: int, where: str):
+    if st != 0:
+        raise DvmError(st, where)
+
+
+class Program:
+    """A shape-agnostic fused operator program (dvm_program)."""
+
+    def __init__(self):
+        self._h = _vp()
+        _check(lib.dvm_program_create(C.byref(self._h)), "dvm_program_create")
+        self._max_code = 0
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            lib.dvm_program_destroy(h)
+
+    def _node(self, fn, *args) -> int:
+        out = C.c_int(-1)
+        _check(fn(self._h, *args, C.byref(out)), fn.__name__)
+        return out.value
+
+    def input(self, dtype, rank):
+        return self._node(lib.dvm_program_input, DTYPES.get(dtype, dtype), rank)
+
+    def unary(self, op, x):
+        return self._node(lib.dvm_program_unary, UNARY.get(op, op), x)
+
+    def binary(self, op, x, y):
+        return self._node(lib.dvm_program_binary, BINARY.get(op, op), x, y)
+
+    def scalar(self, op, x, s):
+        return self._node(lib.dvm_program_scalar, SCALAR.get(op, op), x, float(s))
+
+    def scalar_param(self, op, x, k):
+        return self._node(lib.dvm_program_scalar_param, SCALAR.get(op, op), x, int(k))
+
+    def cast(self, x, dtype):
+        return self._node(lib.dvm_program_cast, x, DTYPES.get(dtype, dtype))
+
+    def reduce(self, op, x, axis=-1):
+        return self._node(lib.dvm_program_reduce, REDUCE.get(op, op), x, axis)
+
+    def matmul(self, a, b):
+        return self._node(lib.dvm_program_matmul, a, b)
+
+    def output(self, x, dtype):
+        _check(lib.dvm_program_output(self._h, x, DTYPES.get(dtype, dtype)), "dvm_program_output")
+
+    def finalize(self):
+        _check(lib.dvm_program_finalize(self._h), "dvm_program_finalize")
+        self._max_code = lib.dvm_code_max_size(self._h)
+        return self
+
+    @property
+    def n_inputs(self):
+        return lib.dvm_program_num_inputs(self._h)
+
+    @property
+    def n_outputs(self):
+        return lib.dvm_program_num_outputs(self._h)
+
+
+def program_from_nodes(nodes: Iterable[tuple]) -> Program:
+    """Builds a Program from the plain-data node list of the workload module."""
+    p = Program()
+    ids = {}
+    for i, n in enumerate(nodes):
+        k = n[0]
+        if k == "input":
+            ids[i] = p.input(n[1], n[2])
+        elif k == "unary":
+            ids[i] = p.unary(n[1], ids[n[2]])
+        elif k == "binary":
+            ids[i] = p.binary(n[1], ids[n[2]], ids[n[3]])
+        elif k == "scalar":
+            if isinstance(n[3], tuple):
+                ids[i] = p.scalar_param(n[1], ids[n[2]], n[3][1])
+            else:
+                ids[i] = p.scalar(n[1], ids[n[2]], n[3])
+        elif k == "cast":
+            ids[i] = p.cast(ids[n[1]], n[2])
+        elif k == "reduce":
+            ids[i] = p.reduce(n[1], ids[n[2]])
+        elif k == "matmul":
+            ids[i] = p.matmul(ids[n[1]], ids[n[2]])
+        elif k == "output":
+            p.output(ids[n[1]], n[2])
+        else:
+            raise ValueError(f"unknown node kind {k}")
+    return p.finalize()
+
+
+class Code:
+    """An encoded bytecode program in host memory plus the inferred output shapes."""
+    __slots__ = ("buf", "size", "out_shapes")
+
+    def __init__(self, buf, size, out_shapes):
+        self.buf, self.size, self.out_shapes = buf, size, out_shapes
+
+    def bytes(self) -> bytes:
+        return bytes(self.buf)[: self.size]
+
+
+class Encoder:
+    """Reusable argument block for dvm_encode (no Python allocation per call)."""
+
+    def __init__(self, program: Program):
+        self.program = program
+        self.n_in, self.n_out = program.n_inputs, program.n_outputs
+        self.shapes = (Shape * self.n_in)()
+        self.out_shapes = (Shape * max(self.n_out, 1))()
+        self.cap = program._max_code
+        self.buf = (C.c_uint64 * ((self.cap + 7) // 8))()
+        self.size = _sz(0)
+        self.scalars = (C.c_float * 16)()
+
+    def encode(self, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = ()) -> int:
+        for s, shp in zip(self.shapes, shapes):
+            s.rank = len(shp)
+            for k, d in enumerate(shp):
+                s.dims[k] = d
+        for k, v in enumerate(scalars):
+            self.scalars[k] = v
+        st = lib.dvm_encode(self.program._h, self.shapes, self.n_in, self.scalars, len(scalars),
+                            self.buf, self.cap, C.byref(self.size), self.out_shapes, self.n_out)
+        if st != 0:
+            raise DvmError(st, "dvm_encode")
+        return self.size.value
+
+    def output_shapes(self) -> List[tuple]:
+        return [tuple(self.out_shapes[o].dims[k] for k in range(self.out_shapes[o].rank))
+                for o in range(self.n_out)]
+
+
+def encode(program: Program, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = ()) -> Code:
+    """dvm_encode: one dynamic-shape instance -> bytecode."""
+    enc = Encoder(program)
+    size = enc.encode(shapes, scalars)
+    return Code(enc.buf, size, enc.output_shapes())
+
+
+def _ptr(t) -> int:
+    return t if isinstance(t, int) else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def launch(code: Code, tensors: Sequence, stream=None):
+    """dvm_launch: tensors are device tensors (or raw device addresses), inputs then outputs."""
+    arr = (_vp * len(tensors))(*[_ptr(t) for t in tensors])
+    _check(lib.dvm_launch(code.buf, code.size, arr, len(tensors), _stream(stream)), "dvm_launch")
+
+
+def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None):
+    """dvm_launch_stacked: many independent programs in one kernel launch."""
+    n = len(codes)
+    cptr = (_vp * n)(*[C.addressof(c.buf) for c in codes])
+    csz = (_sz * n)(*[c.size for c in codes])
+    keep = [(_vp * len(tl))(*[_ptr(t) for t in tl]) for tl in tensor_lists]
+    tptr = (C.POINTER(_vp) * n)(*[C.cast(k, C.POINTER(_vp)) for k in keep])
+    nt = (_i * n)(*[len(tl) for tl in tensor_lists])
+    _check(lib.dvm_launch_stacked(n, cptr, csz, tptr, nt, _stream(stream)), "dvm_launch_stacked")
+
+
+def run_host(code: Code, host_tensors: Sequence, staging, stream=None):
+    """dvm_run_host: host tensors in, host tensors out; copies are inside the call."""
+    n = len(host_tensors)
+    arr = (_vp * n)(*[_ptr(t) for t in host_tensors])
+    nbytes = (_sz * n)(*[t.numel() * t.element_size() for t in host_tensors])
+    _check(lib.dvm_run_host(code.buf, code.size, arr, nbytes, n, _ptr(staging),
+                            staging.numel() * staging.element_size(), _stream(stream)), "dvm_run_host")
+
+
+def verify(code) -> int:
+    if isinstance(code, Code):
+        return lib.dvm_verify(code.buf, code.size)
+    raw = bytes(code)
+    buf = (C.c_uint64 * ((len(raw) + 7) // 8 + 1))()
+    C.memmove(buf, raw, len(raw))
+    return lib.dvm_verify(buf, len(raw))
+
+
+def disassemble(code: Code) -> str:
+    out = C.create_string_buffer(1 << 16)
+    _check(lib.dvm_disassemble(code.buf, code.size, out, len(out)), "dvm_disassemble")
+    return out.value.decode()
+
+
+def code_info(code: Code) -> dict:
+    kt, bb, tpr, vw, nr = C.c_int(), C.c_int(), C.c_int(), C.c_int(), C.c_int()
+    nt = C.c_int64()
+    _check(lib.dvm_code_info(code.buf, code.size, C.byref(kt), C.byref(nt), C.byref(bb), C.byref(tpr),
+                             C.byref(vw), C.byref(nr)), "dvm_code_info")
+    return {"kernel_type": kt.value, "n_tiles": nt.value, "code_body_bytes": bb.value,
+            "threads_per_row": tpr.value, "vector_width": vw.value, "n_tile_regs": nr.value}
+
+
+def last_device_status(stream=None) -> int:
+    st = C.c_int(0)
+    _check(lib.dvm_last_device_status(_stream(stream), C.byref(st)), "dvm_last_device_status")
+    return st.value
+
+
+def launch_count() -> int:
+    return lib.dvm_launch_count()
+
+
+def hardware_align_div(total, n_cores, align, t_max, overhead=2):
+    a, b, c, d = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64()
+    _check(lib.dvm_hardware_align_div(total, n_cores, align, t_max, overhead, C.byref(a), C.byref(b),
+                                      C.byref(c), C.byref(d)), "dvm_hardware_align_div")
+    return {"min_cost_tile": a.value, "rounded_tile": b.value, "n_tiles": c.value, "tail": d.value}
+
+
+def vm_tile_range(n_tiles, n_cores, core_id):
+    b, e = C.c_int64(), C.c_int64()
+    _check(lib.dvm_vm_tile_range(n_tiles, n_cores, core_id, C.byref(b), C.byref(e)), "dvm_vm_tile_range")
+    return b.value, e.value
+
+
+def set_num_cores(n: int):
+    lib.dvm_set_num_cores(n)
+
+
+def get_num_cores() -> int:
+    return lib.dvm_get_num_cores()

@@ -1,0 +1,128 @@
+// Bytecode program format of the device-side virtual machine (host + device).
+//
+// The paper fixes only the parts list (Sec. 4.2 "Bytecode encoding"): a code
+// header {KernelType, CodeSize, total number of tiles} and a code body with one
+// bytecode per operation {instruction id, bytecode length, source / destination
+// tile operands, compute size, extras}.  Field widths and ids are this
+// library's own.  Everything is 32-bit little-endian words.
+//
+//   [ header : DVM_HDR_WORDS words ]
+//   [ tensor table : 2 words per tensor slot (device pointer, patched at launch) ]
+//   [ operand table : DVM_OPD_WORDS words per global-memory operand ]
+//   [ code body : CodeSize words, instructions of 1..3 words ]
+//
+// Unlike the paper's bytecode, a memory instruction does not carry an address:
+// it names an operand descriptor, which names a tensor slot; the launch call
+// supplies the pointers.  The tile id an instruction needs (Algorithm 2) is the
+// interpreter's loop variable.
+#pragma once
+#include <stdint.h>
+
+#define DVM_MAGIC 0x314D5644u /* "DVM1" */
+
+enum {
+  DVM_KERNEL_VEC = 1,     // meta-kernel of vector operations
+  DVM_KERNEL_MATMUL = 2,  // meta-kernel: matmul instruction + fused epilogue
+  DVM_KERNEL_STACKED = 3  // several meta-kernels in one launch (built at launch time)
+};
+
+// ---- header word indices ----
+enum {
+  DVM_H_MAGIC = 0,
+  DVM_H_KERNEL_TYPE = 1,
+  DVM_H_CODE_WORDS = 2,   // CodeSize: body length in words
+  DVM_H_N_TILES = 3,      // total number of tiles
+  DVM_H_TOTAL_WORDS = 4,  // header + tables + body
+  DVM_H_COUNTS = 5,       // n_tensors | n_inputs << 8 | n_operands << 16 | n_outputs << 24
+  DVM_H_GEOM = 6,         // log2G | W << 8 | nreg << 16 | flags << 24
+  DVM_H_COLS = 7,         // C: columns of the dominant (collapsed) shape
+  DVM_H_ROWS_LO = 8,      // R: rows of the dominant shape (64 bit)
+  DVM_H_ROWS_HI = 9,
+  DVM_H_COL_BLOCKS = 10,  // number of column blocks per row group
+  DVM_H_COL_TILE = 11,    // columns per column block
+  DVM_H_OUTER0 = 12,      // sizes of the (up to 3) collapsed outer dims, innermost first
+  DVM_H_OUTER1 = 13,
+  DVM_H_OUTER2 = 14,
+  DVM_H_LAST_ROW_COLS = 15,  // valid columns of the last row (flat programs), else C
+  DVM_H_PRIMARY = 16,        // operand whose row starts define the vector alignment, or 0xffffffff
+  DVM_HDR_WORDS = 20         // 17..19 reserved (zero)
+};
+
+// flags in DVM_H_GEOM bits 24..31
+enum {
+  DVM_F_ALIGNED = 1,    // every row segment of the primary operand starts on a W-element
+                        // boundary provided its base pointer is 16-byte aligned
+  DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
+  DVM_F_FLAT = 4        // pure elementwise program laid out as a flat range
+};
+
+// ---- operand descriptor ----
+enum {
+  DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24
+  DVM_OPD_RSVD = 1,
+  DVM_OPD_STRIDE0 = 2,   // int64 element stride of outer dim 0 (lo, hi)
+  DVM_OPD_STRIDE1 = 4,
+  DVM_OPD_STRIDE2 = 6,
+  DVM_OPD_WORDS = 8
+};
+
+enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
+
+// ---- limits ----
+#define DVM_VM_THREADS 256       // threads per CTA of the interpreter
+#define DVM_VM_V 16              // elements of a tile register held by one thread
+#define DVM_MAX_TREGS 8          // tile registers (R0 is the accumulator)
+#define DVM_MAX_SREGS 8          // per-row scalar registers
+#define DVM_MAX_TENSORS 16
+#define DVM_MAX_OPERANDS 24
+#define DVM_MAX_NODES 96
+#define DVM_MAX_STACK 256        // programs per stacked launch
+
+// ---- instruction word 0:  op | len << 8 | a << 16 | b << 24 ----
+#define DVM_INSN(op, len, a, b) \
+  ((uint32_t)(op) | ((uint32_t)(len) << 8) | ((uint32_t)(a) << 16) | ((uint32_t)(b) << 24))
+#define DVM_INSN_OP(w) ((w) & 0xffu)
+#define DVM_INSN_LEN(w) (((w) >> 8) & 0xffu)
+#define DVM_INSN_A(w) (((w) >> 16) & 0xffu)
+#define DVM_INSN_B(w) (((w) >> 24) & 0xffu)
+
+// Arithmetic sub-operations (shared numbering for tile and scalar forms).
+enum {
+  DVM_A_ADD = 0, DVM_A_SUB = 1, DVM_A_RSUB = 2, DVM_A_MUL = 3,
+  DVM_A_DIV = 4, DVM_A_RDIV = 5, DVM_A_MIN = 6, DVM_A_MAX = 7,
+  DVM_A_NBIN = 8
+};
+enum {
+  DVM_U_EXP = 0, DVM_U_SQRT = 1, DVM_U_RSQRT = 2, DVM_U_ABS = 3, DVM_U_LOG = 4,
+  DVM_U_ERF = 5, DVM_U_SIGMOID = 6, DVM_U_NEG = 7, DVM_U_RECIP = 8, DVM_U_FLOOR = 9,
+  DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12, DVM_U_NUN = 13
+};
+enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_NRED = 3 };
+
+// Instruction ids.  R0 is the accumulator: arithmetic reads and writes R0.
+enum {
+  DVM_OP_NOP = 0x00,
+  DVM_OP_LDG = 0x01,   // a = tile reg, b = operand      : issue the tile load (raw element bits)
+  DVM_OP_CVT = 0x02,   // a = tile reg, b = dtype        : widen raw bits to fp32 in place
+  DVM_OP_STG = 0x03,   // a = 0,        b = operand      : narrow R0 and store the tile
+  DVM_OP_LDS = 0x04,   // a = scalar reg, b = operand    : load one value per row
+  DVM_OP_STS = 0x05,   // a = scalar reg, b = operand    : store one value per row
+  DVM_OP_MOV = 0x06,   // a = dst tile reg, b = src tile reg
+  DVM_OP_BCS = 0x07,   // a = scalar reg                 : R0 = broadcast(S[a])   (Table 1, Broadcast)
+  DVM_OP_BINI = 0x10,  // 0x10 + arith; len 2, word1 = fp32 immediate : R0 = R0 op imm  (Adds/Muls)
+  DVM_OP_BIN = 0x20,   // 0x20 + arith * 8 + reg                      : R0 = R0 op R[reg]
+  DVM_OP_BINS = 0x60,  // 0x60 + arith; a = scalar reg                : R0 = R0 op S[a] (row broadcast)
+  DVM_OP_UN = 0x70,    // 0x70 + unary                                : R0 = f(R0)
+  DVM_OP_RED = 0x80,   // 0x80 + reduce; a = dst scalar reg           : S[a] = reduce(R0) over the row
+  DVM_OP_SOP = 0x90,   // per-row scalar arithmetic; a = dst scalar reg, b = kind;
+                       // len 2: word1 = sub_op | src1 << 8 | src2 << 16 ; len 3: word2 = fp32 immediate
+  DVM_OP_LAST = 0x91
+};
+enum { DVM_SK_BIN = 0, DVM_SK_BINI = 1, DVM_SK_UN = 2 };
+
+// ---- matmul meta-kernel: extra header words follow the common header ----
+// (see dvm_matmul.cu)
+enum {
+  DVM_MM_M = 0, DVM_MM_N = 1, DVM_MM_K = 2, DVM_MM_NB = 3,  // NB: number of B matrices (1 or 2)
+  DVM_MM_WORDS = 4
+};

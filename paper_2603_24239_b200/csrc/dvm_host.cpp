@@ -1,0 +1,1132 @@
+// Host half of the operator compiler: program description, per-instance shape
+// inference, shape tiling, bytecode encoding, verification and the readable dump.
+// No CUDA here; dvm_encode performs no heap allocation.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/dvm.h"
+#include "dvm_format.h"
+#include "dvm_internal.h"
+
+// ---------------------------------------------------------------------------
+// Program description
+// ---------------------------------------------------------------------------
+enum NodeKind : uint8_t { NK_INPUT, NK_UNARY, NK_BINARY, NK_SCALAR, NK_CAST, NK_REDUCE, NK_MATMUL };
+
+struct Node {
+  uint8_t kind;
+  uint8_t op;
+  uint8_t dtype;
+  int8_t rank;
+  int16_t x, y;
+  int16_t param;  // >= 0: scalar comes from the runtime argument list
+  float imm;
+};
+
+struct OutputRef {
+  int16_t value;
+  uint8_t dtype;
+};
+
+struct dvm_program {
+  Node nodes[DVM_MAX_NODES];
+  int n_nodes;
+  int16_t inputs[DVM_MAX_TENSORS];
+  int n_inputs;
+  OutputRef outputs[DVM_MAX_TENSORS];
+  int n_outputs;
+  int n_params;
+  int n_matmul;
+  bool finalized;
+};
+
+static int g_num_cores = 0;
+static const int kDefaultCores = 148 * 3;
+
+extern "C" void dvm_set_num_cores(int n) { g_num_cores = n > 0 ? n : 0; }
+extern "C" int dvm_get_num_cores(void) { return g_num_cores > 0 ? g_num_cores : kDefaultCores; }
+
+extern "C" int dvm_program_create(dvm_program** out) {
+  if (!out) return DVM_ERR_INVALID_ARG;
+  dvm_program* p = (dvm_program*)calloc(1, sizeof(dvm_program));
+  if (!p) return DVM_ERR_INVALID_ARG;
+  *out = p;
+  return DVM_OK;
+}
+
+extern "C" void dvm_program_destroy(dvm_program* p) { free(p); }
+
+static int push_node(dvm_program* p, const Node& n, int* value_id) {
+  if (!p || !value_id) return DVM_ERR_INVALID_ARG;
+  if (p->finalized) return DVM_ERR_INVALID_ARG;
+  if (p->n_nodes >= DVM_MAX_NODES) return DVM_ERR_TOO_LARGE;
+  p->nodes[p->n_nodes] = n;
+  *value_id = p->n_nodes++;
+  return DVM_OK;
+}
+
+static bool valid_value(const dvm_program* p, int v) { return p && v >= 0 && v < p->n_nodes; }
+
+extern "C" int dvm_program_input(dvm_program* p, int dtype, int rank, int* value_id) {
+  if (!p) return DVM_ERR_INVALID_ARG;
+  if (dtype != DVM_F32 && dtype != DVM_BF16) return DVM_ERR_INVALID_ARG;
+  if (rank < 0 || rank > DVM_MAX_RANK) return DVM_ERR_INVALID_ARG;
+  if (p->n_inputs >= DVM_MAX_TENSORS) return DVM_ERR_TOO_LARGE;
+  Node n = {};
+  n.kind = NK_INPUT;
+  n.dtype = (uint8_t)dtype;
+  n.rank = (int8_t)rank;
+  n.x = n.y = n.param = -1;
+  int st = push_node(p, n, value_id);
+  if (st == DVM_OK) p->inputs[p->n_inputs++] = (int16_t)*value_id;
+  return st;
+}
+
+extern "C" int dvm_program_unary(dvm_program* p, int op, int x, int* value_id) {
+  if (!valid_value(p, x) || op < 0 || op > DVM_TANH) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_UNARY;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = n.param = -1;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_binary(dvm_program* p, int op, int x, int y, int* value_id) {
+  if (!valid_value(p, x) || !valid_value(p, y) || op < 0 || op > DVM_MAX) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_BINARY;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = (int16_t)y;
+  n.param = -1;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_scalar(dvm_program* p, int op, int x, float s, int* value_id) {
+  if (!valid_value(p, x) || op < 0 || op > DVM_MULS) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_SCALAR;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = n.param = -1;
+  n.imm = s;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_scalar_param(dvm_program* p, int op, int x, int param, int* value_id) {
+  if (!valid_value(p, x) || op < 0 || op > DVM_MULS || param < 0 || param >= 64)
+    return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_SCALAR;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = -1;
+  n.param = (int16_t)param;
+  int st = push_node(p, n, value_id);
+  if (st == DVM_OK && param + 1 > p->n_params) p->n_params = param + 1;
+  return st;
+}
+
+extern "C" int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id) {
+  if (!valid_value(p, x) || (dtype != DVM_F32 && dtype != DVM_BF16)) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_CAST;
+  n.dtype = (uint8_t)dtype;
+  n.x = (int16_t)x;
+  n.y = n.param = -1;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id) {
+  if (!valid_value(p, x) || op < 0 || op > DVM_RMIN) return DVM_ERR_INVALID_ARG;
+  if (axis != -1) return DVM_ERR_UNSUPPORTED;
+  Node n = {};
+  n.kind = NK_REDUCE;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = n.param = -1;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_matmul(dvm_program* p, int a, int b, int* value_id) {
+  if (!valid_value(p, a) || !valid_value(p, b)) return DVM_ERR_INVALID_ARG;
+  if (p->nodes[a].kind != NK_INPUT || p->nodes[b].kind != NK_INPUT) return DVM_ERR_UNSUPPORTED;
+  Node n = {};
+  n.kind = NK_MATMUL;
+  n.x = (int16_t)a;
+  n.y = (int16_t)b;
+  n.param = -1;
+  int st = push_node(p, n, value_id);
+  if (st == DVM_OK) p->n_matmul++;
+  return st;
+}
+
+extern "C" int dvm_program_output(dvm_program* p, int x, int dtype) {
+  if (!valid_value(p, x) || (dtype != DVM_F32 && dtype != DVM_BF16)) return DVM_ERR_INVALID_ARG;
+  if (p->finalized) return DVM_ERR_INVALID_ARG;
+  if (p->n_outputs >= DVM_MAX_TENSORS) return DVM_ERR_TOO_LARGE;
+  p->outputs[p->n_outputs].value = (int16_t)x;
+  p->outputs[p->n_outputs].dtype = (uint8_t)dtype;
+  p->n_outputs++;
+  return DVM_OK;
+}
+
+extern "C" int dvm_program_finalize(dvm_program* p) {
+  if (!p) return DVM_ERR_INVALID_ARG;
+  if (p->n_outputs == 0 || p->n_inputs == 0) return DVM_ERR_INVALID_ARG;
+  if (p->n_inputs + p->n_outputs > DVM_MAX_TENSORS) return DVM_ERR_TOO_LARGE;
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind != NK_INPUT && (n.x < 0 || n.x >= i)) return DVM_ERR_INVALID_ARG;
+    if ((n.kind == NK_BINARY || n.kind == NK_MATMUL) && (n.y < 0 || n.y >= i)) return DVM_ERR_INVALID_ARG;
+  }
+  if (p->n_matmul > 0) {
+    if (p->n_matmul > 2) return DVM_ERR_UNSUPPORTED;
+    int a = -1;
+    for (int i = 0; i < p->n_nodes; ++i) {
+      const Node& n = p->nodes[i];
+      if (n.kind == NK_MATMUL) {
+        if (a >= 0 && n.x != a) return DVM_ERR_UNSUPPORTED;
+        a = n.x;
+        if (p->nodes[n.x].dtype != DVM_BF16 || p->nodes[n.y].dtype != DVM_BF16) return DVM_ERR_UNSUPPORTED;
+      }
+      if (n.kind == NK_REDUCE) return DVM_ERR_UNSUPPORTED;  // cube-vector fusion: elementwise epilogue only
+    }
+  }
+  p->finalized = true;
+  return DVM_OK;
+}
+
+extern "C" int dvm_program_num_inputs(const dvm_program* p) { return p ? p->n_inputs : DVM_ERR_INVALID_ARG; }
+extern "C" int dvm_program_num_outputs(const dvm_program* p) { return p ? p->n_outputs : DVM_ERR_INVALID_ARG; }
+
+extern "C" size_t dvm_code_max_size(const dvm_program* p) {
+  if (!p) return 0;
+  // header + matmul extension + tensor table + operand table + 6 words per node (loads, converts,
+  // spills, the operation with immediate) + stores
+  size_t words = DVM_HDR_WORDS + DVM_MM_WORDS + 2 * DVM_MAX_TENSORS + DVM_OPD_WORDS * DVM_MAX_OPERANDS +
+                 8 * (size_t)p->n_nodes + 4 * (size_t)p->n_outputs + 16;
+  return words * 4;
+}
+
+// ---------------------------------------------------------------------------
+// The paper's tile-size rule and Algorithm 2's tile range (exported for tests)
+// ---------------------------------------------------------------------------
+static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+extern "C" int dvm_hardware_align_div(int64_t total, int n_cores, int64_t align, int64_t t_max,
+                                      int64_t overhead, int64_t* min_cost_tile, int64_t* rounded_tile,
+                                      int64_t* n_tiles, int64_t* tail) {
+  if (total <= 0 || n_cores <= 0 || align <= 0 || t_max <= 0 || overhead < 0) return DVM_ERR_INVALID_ARG;
+  int64_t hi = total < t_max ? total : t_max;
+  int64_t best_t = 1, best_cost = -1;
+  for (int64_t t = 1; t <= hi; ++t) {
+    int64_t cost = cdiv(cdiv(total, t), n_cores) * (t + overhead);
+    if (best_cost < 0 || cost <= best_cost) {  // ties: the larger tile
+      best_cost = cost;
+      best_t = t;
+    }
+  }
+  int64_t r = cdiv(best_t, align) * align;
+  if (r > t_max) r = best_t;  // rounding must respect the tile size limit
+  int64_t nt = cdiv(total, best_t);
+  if (min_cost_tile) *min_cost_tile = best_t;
+  if (rounded_tile) *rounded_tile = r;
+  if (n_tiles) *n_tiles = nt;
+  if (tail) *tail = total - (nt - 1) * best_t;
+  return DVM_OK;
+}
+
+extern "C" int dvm_vm_tile_range(int64_t n_tiles, int n_cores, int id, int64_t* begin, int64_t* end) {
+  if (n_tiles < 0 || n_cores <= 0 || id < 0 || id >= n_cores || !begin || !end) return DVM_ERR_INVALID_ARG;
+  int64_t m = cdiv(n_tiles, n_cores);
+  int64_t b = m * id, e = m * (id + 1);
+  if (b > n_tiles) b = n_tiles;
+  if (e > n_tiles) e = n_tiles;
+  *begin = b;
+  *end = e;
+  return DVM_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Encode
+// ---------------------------------------------------------------------------
+namespace {
+
+enum { CLS_TILE = 0, CLS_SCAL = 1 };
+
+struct Operand {       // one global-memory access
+  int slot;            // tensor slot
+  int dtype;
+  int col_stride;      // 1 or 0
+  int64_t stride[DVM_MAX_RANK];  // element strides over the dominant dims (before merging)
+  int64_t ostride[3];            // after merging: outer dims, innermost first
+  bool primary;
+};
+
+struct Enc {
+  const dvm_program* p;
+  int D;                          // rank of the dominant shape
+  int64_t Sd[DVM_MAX_RANK];       // dominant shape
+  int64_t dims[DVM_MAX_NODES][DVM_MAX_RANK];  // right-aligned per value
+  int8_t cls[DVM_MAX_NODES];
+  int16_t alias[DVM_MAX_NODES];   // identity nodes resolve to another value
+  bool reduce_identity_axis;
+  // code generation state
+  uint32_t body[8 * DVM_MAX_NODES + 64];
+  int n_body;
+  Operand opd[DVM_MAX_OPERANDS];
+  int n_opd;
+  int16_t uses[DVM_MAX_NODES];
+  int8_t reg_of[DVM_MAX_NODES];   // tile register >= 1 holding the value, or -1
+  int8_t sreg_of[DVM_MAX_NODES];
+  int16_t treg_val[DVM_MAX_TREGS];
+  bool needs_cvt[DVM_MAX_TREGS];
+  int16_t sreg_val[DVM_MAX_SREGS];
+  int16_t acc;                    // value in R0 or -1
+  int nreg_limit;
+  int max_treg;
+  int8_t in_operand[DVM_MAX_NODES];   // operand index of an input value
+  bool stored[DVM_MAX_TENSORS];       // output already stored
+  int8_t out_operand[DVM_MAX_TENSORS];
+  const float* scalars;
+  int n_scalars;
+  bool fail;
+};
+
+static inline int root(const Enc& e, int v) {
+  while (e.alias[v] >= 0) v = e.alias[v];
+  return v;
+}
+
+static inline void emit(Enc& e, uint32_t w) { e.body[e.n_body++] = w; }
+
+static inline uint32_t f2u(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return u;
+}
+
+static int alloc_treg(Enc& e) {
+  for (int k = 1; k < e.nreg_limit; ++k)
+    if (e.treg_val[k] < 0) {
+      if (k > e.max_treg) e.max_treg = k;
+      return k;
+    }
+  e.fail = true;
+  return -1;
+}
+
+static int alloc_sreg(Enc& e) {
+  for (int k = 0; k < DVM_MAX_SREGS; ++k)
+    if (e.sreg_val[k] < 0) return k;
+  e.fail = true;
+  return -1;
+}
+
+static void cvt_if_needed(Enc& e, int k) {
+  if (e.needs_cvt[k]) {
+    emit(e, DVM_INSN(DVM_OP_CVT, 1, k, DVM_DT_BF16));
+    e.needs_cvt[k] = false;
+  }
+}
+
+static void release(Enc& e, int v) {  // free the registers of a dead value
+  if (e.uses[v] > 0) return;
+  if (e.cls[v] == CLS_TILE) {
+    if (e.reg_of[v] >= 1) {
+      e.treg_val[e.reg_of[v]] = -1;
+      e.needs_cvt[e.reg_of[v]] = false;
+      e.reg_of[v] = -1;
+    }
+  } else if (e.sreg_of[v] >= 0) {
+    e.sreg_val[e.sreg_of[v]] = -1;
+    e.sreg_of[v] = -1;
+  }
+}
+
+static void load_input_to(Enc& e, int v, int k) {  // issue the tile load of input value v into Rk
+  int od = e.in_operand[v];
+  emit(e, DVM_INSN(DVM_OP_LDG, 1, k, od));
+  e.needs_cvt[k] = e.opd[od].dtype == DVM_DT_BF16;
+  if (k == 0) {
+    e.acc = (int16_t)v;
+  } else {
+    e.reg_of[v] = (int8_t)k;
+    e.treg_val[k] = (int16_t)v;
+  }
+}
+
+static void spill_acc_if_live(Enc& e) {
+  int a = e.acc;
+  if (a >= 0 && e.uses[a] > 0 && e.reg_of[a] < 0) {
+    int k = alloc_treg(e);
+    if (k < 0) return;
+    cvt_if_needed(e, 0);
+    emit(e, DVM_INSN(DVM_OP_MOV, 1, k, 0));
+    e.reg_of[a] = (int8_t)k;
+    e.treg_val[k] = (int16_t)a;
+  }
+}
+
+static void ensure_acc(Enc& e, int v) {
+  if (e.acc == v) {
+    cvt_if_needed(e, 0);
+    return;
+  }
+  spill_acc_if_live(e);
+  if (e.fail) return;
+  if (e.reg_of[v] >= 1) {
+    cvt_if_needed(e, e.reg_of[v]);
+    emit(e, DVM_INSN(DVM_OP_MOV, 1, 0, e.reg_of[v]));
+    e.acc = (int16_t)v;
+  } else if (e.p->nodes[v].kind == NK_INPUT) {
+    load_input_to(e, v, 0);
+    cvt_if_needed(e, 0);
+  } else {
+    e.fail = true;  // value was dropped: cannot happen with correct use counts
+  }
+}
+
+static int ensure_reg(Enc& e, int v) {  // a tile value as the non-accumulator operand
+  if (e.acc == v && e.reg_of[v] < 0) return 0;
+  if (e.reg_of[v] >= 1) {
+    cvt_if_needed(e, e.reg_of[v]);
+    return e.reg_of[v];
+  }
+  if (e.p->nodes[v].kind == NK_INPUT) {
+    int k = alloc_treg(e);
+    if (k < 0) return -1;
+    load_input_to(e, v, k);
+    cvt_if_needed(e, k);
+    return k;
+  }
+  e.fail = true;
+  return -1;
+}
+
+static int ensure_sreg(Enc& e, int v) {
+  if (e.sreg_of[v] >= 0) return e.sreg_of[v];
+  if (e.p->nodes[v].kind == NK_INPUT) {
+    int k = alloc_sreg(e);
+    if (k < 0) return -1;
+    emit(e, DVM_INSN(DVM_OP_LDS, 1, k, e.in_operand[v]));
+    e.sreg_of[v] = (int8_t)k;
+    e.sreg_val[k] = (int16_t)v;
+    return k;
+  }
+  e.fail = true;
+  return -1;
+}
+
+static void store_outputs_of(Enc& e, int v) {  // value v is live in R0 (tile) or a scalar register
+  for (int o = 0; o < e.p->n_outputs; ++o) {
+    if (e.stored[o] || root(e, e.p->outputs[o].value) != v) continue;
+    if (e.cls[v] == CLS_TILE) {
+      ensure_acc(e, v);
+      if (e.fail) return;
+      emit(e, DVM_INSN(DVM_OP_STG, 1, 0, e.out_operand[o]));
+    } else {
+      int s = ensure_sreg(e, v);
+      if (s < 0) return;
+      emit(e, DVM_INSN(DVM_OP_STS, 1, s, e.out_operand[o]));
+    }
+    e.stored[o] = true;
+    e.uses[v]--;
+  }
+}
+
+static const uint8_t kBinMap[6] = {DVM_A_ADD, DVM_A_SUB, DVM_A_MUL, DVM_A_DIV, DVM_A_MIN, DVM_A_MAX};
+static inline uint8_t reversed(uint8_t a) {
+  if (a == DVM_A_SUB) return DVM_A_RSUB;
+  if (a == DVM_A_DIV) return DVM_A_RDIV;
+  return a;
+}
+static const uint8_t kUnMap[12] = {DVM_U_EXP, DVM_U_SQRT, DVM_U_RSQRT, DVM_U_ABS, DVM_U_LOG, DVM_U_ERF,
+                                   DVM_U_SIGMOID, DVM_U_NEG, DVM_U_RECIP, DVM_U_FLOOR, DVM_U_ROUND, DVM_U_TANH};
+
+// Generates the code body.  hoist: issue every tile load at the top of the body so that all
+// of a tile's global loads are in flight before the first use.
+static bool gen_body(Enc& e, bool hoist, int nreg_limit) {
+  const dvm_program* p = e.p;
+  e.n_body = 0;
+  e.fail = false;
+  e.acc = -1;
+  e.nreg_limit = nreg_limit;
+  e.max_treg = 0;
+  for (int k = 0; k < DVM_MAX_TREGS; ++k) { e.treg_val[k] = -1; e.needs_cvt[k] = false; }
+  for (int k = 0; k < DVM_MAX_SREGS; ++k) e.sreg_val[k] = -1;
+  for (int o = 0; o < p->n_outputs; ++o) e.stored[o] = false;
+  for (int i = 0; i < p->n_nodes; ++i) { e.uses[i] = 0; e.reg_of[i] = -1; e.sreg_of[i] = -1; }
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
+    e.uses[root(e, n.x)]++;
+    if (n.kind == NK_BINARY) e.uses[root(e, n.y)]++;
+  }
+  for (int o = 0; o < p->n_outputs; ++o) e.uses[root(e, p->outputs[o].value)]++;
+
+  if (hoist) {
+    // the first tile-class operation decides which input is loaded straight into R0
+    int first_acc = -1;
+    for (int i = 0; i < p->n_nodes && first_acc < 0; ++i) {
+      const Node& n = p->nodes[i];
+      if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
+      int x = root(e, n.x);
+      int y = n.kind == NK_BINARY ? root(e, n.y) : -1;
+      if (e.cls[x] == CLS_TILE && p->nodes[x].kind == NK_INPUT) first_acc = x;
+      else if (y >= 0 && e.cls[y] == CLS_TILE && p->nodes[y].kind == NK_INPUT) first_acc = y;
+      else if (e.cls[x] == CLS_TILE || (y >= 0 && e.cls[y] == CLS_TILE)) break;
+    }
+    if (first_acc < 0) {
+      for (int o = 0; o < p->n_outputs && first_acc < 0; ++o) {
+        int v = root(e, p->outputs[o].value);
+        if (e.cls[v] == CLS_TILE && p->nodes[v].kind == NK_INPUT) first_acc = v;
+      }
+    }
+    // loads in order of first use
+    bool seen[DVM_MAX_NODES] = {};
+    auto hoist_one = [&](int v) {
+      if (v < 0 || seen[v] || p->nodes[v].kind != NK_INPUT || e.uses[v] == 0) return;
+      seen[v] = true;
+      if (e.cls[v] == CLS_SCAL) { ensure_sreg(e, v); return; }
+      if (v == first_acc) { load_input_to(e, v, 0); return; }
+      int k = alloc_treg(e);
+      if (k >= 0) load_input_to(e, v, k);
+    };
+    hoist_one(first_acc);
+    for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
+      const Node& n = p->nodes[i];
+      if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
+      hoist_one(root(e, n.x));
+      if (n.kind == NK_BINARY) hoist_one(root(e, n.y));
+    }
+    for (int o = 0; o < p->n_outputs && !e.fail; ++o) hoist_one(root(e, p->outputs[o].value));
+    if (e.fail) return false;
+  }
+
+  for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
+    int x = root(e, n.x);
+    if (e.cls[i] == CLS_SCAL && n.kind != NK_REDUCE) {
+      // ---- per-row scalar arithmetic ----
+      int sx = ensure_sreg(e, x);
+      int sy = -1;
+      int y = -1;
+      if (n.kind == NK_BINARY) { y = root(e, n.y); sy = ensure_sreg(e, y); }
+      if (e.fail) break;
+      e.uses[x]--;
+      if (y >= 0) e.uses[y]--;
+      release(e, x);
+      if (y >= 0 && y != x) release(e, y);
+      int d = alloc_sreg(e);
+      if (d < 0) break;
+      if (n.kind == NK_BINARY) {
+        emit(e, DVM_INSN(DVM_OP_SOP, 2, d, DVM_SK_BIN));
+        emit(e, (uint32_t)kBinMap[n.op] | ((uint32_t)sx << 8) | ((uint32_t)sy << 16));
+      } else if (n.kind == NK_SCALAR) {
+        float s = n.param >= 0 ? e.scalars[n.param] : n.imm;
+        emit(e, DVM_INSN(DVM_OP_SOP, 3, d, DVM_SK_BINI));
+        emit(e, (uint32_t)(n.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL) | ((uint32_t)sx << 8));
+        emit(e, f2u(s));
+      } else {  // unary or rounding cast
+        uint32_t u = n.kind == NK_CAST ? (uint32_t)DVM_U_RND_BF16 : (uint32_t)kUnMap[n.op];
+        emit(e, DVM_INSN(DVM_OP_SOP, 2, d, DVM_SK_UN));
+        emit(e, u | ((uint32_t)sx << 8));
+      }
+      e.sreg_of[i] = (int8_t)d;
+      e.sreg_val[d] = (int16_t)i;
+      store_outputs_of(e, i);
+      release(e, i);
+      continue;
+    }
+    if (n.kind == NK_REDUCE) {
+      ensure_acc(e, x);
+      if (e.fail) break;
+      e.uses[x]--;
+      int d = alloc_sreg(e);
+      if (d < 0) break;
+      emit(e, DVM_INSN(DVM_OP_RED + (n.op == DVM_SUM ? DVM_R_SUM : n.op == DVM_RMAX ? DVM_R_MAX : DVM_R_MIN),
+                       1, d, 0));
+      e.sreg_of[i] = (int8_t)d;
+      e.sreg_val[d] = (int16_t)i;
+      if (e.uses[x] == 0) { release(e, x); }
+      store_outputs_of(e, i);
+      release(e, i);
+      continue;
+    }
+    // ---- tile-class result in the accumulator ----
+    if (n.kind == NK_BINARY) {
+      int y = root(e, n.y);
+      uint8_t ar = kBinMap[n.op];
+      int a = x, b = y;  // a: accumulator operand, b: the other
+      bool swap = false;
+      if (e.cls[x] == CLS_SCAL) swap = true;                                   // scalar (op) tile
+      else if (e.cls[y] == CLS_TILE && e.acc == y && e.acc != x) swap = true;   // right operand already in R0
+      if (swap) { a = y; b = x; ar = reversed(ar); }
+      ensure_acc(e, a);
+      if (e.fail) break;
+      int bk = -1;
+      if (e.cls[b] == CLS_TILE) bk = (b == a) ? 0 : ensure_reg(e, b);
+      else bk = ensure_sreg(e, b);
+      if (e.fail || bk < 0) { e.fail = true; break; }
+      e.uses[a]--;
+      e.uses[b]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      if (e.cls[b] == CLS_TILE) emit(e, DVM_INSN(DVM_OP_BIN + ar * 8 + bk, 1, 0, 0));
+      else emit(e, DVM_INSN(DVM_OP_BINS + ar, 1, bk, 0));
+      e.acc = (int16_t)i;
+      release(e, a);
+      if (b != a) release(e, b);
+    } else {
+      ensure_acc(e, x);
+      if (e.fail) break;
+      e.uses[x]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      if (n.kind == NK_UNARY) {
+        emit(e, DVM_INSN(DVM_OP_UN + kUnMap[n.op], 1, 0, 0));
+      } else if (n.kind == NK_SCALAR) {
+        float s = n.param >= 0 ? e.scalars[n.param] : n.imm;
+        emit(e, DVM_INSN(DVM_OP_BINI + (n.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL), 2, 0, 0));
+        emit(e, f2u(s));
+      } else {  // NK_CAST to bf16 (casts to f32 are aliases)
+        emit(e, DVM_INSN(DVM_OP_UN + DVM_U_RND_BF16, 1, 0, 0));
+      }
+      e.acc = (int16_t)i;
+      release(e, x);
+    }
+    store_outputs_of(e, i);
+    if (e.acc == i && e.uses[i] == 0) e.acc = -1;
+  }
+  if (e.fail) return false;
+  // outputs that are inputs (or aliases of inputs)
+  for (int o = 0; o < p->n_outputs && !e.fail; ++o)
+    if (!e.stored[o]) store_outputs_of(e, root(e, p->outputs[o].value));
+  return !e.fail;
+}
+
+}  // namespace
+
+int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in, const float* scalars,
+                      int n_scalars, void* code, size_t code_capacity, size_t* code_size,
+                      dvm_shape* out_shapes, int n_out);
+
+extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
+                          const float* scalars, int n_scalars, void* code, size_t code_capacity,
+                          size_t* code_size, dvm_shape* out_shapes, int n_out) {
+  if (!p || !in_shapes || !code_size) return DVM_ERR_INVALID_ARG;
+  if (!p->finalized) return DVM_ERR_NOT_FINALIZED;
+  if (n_in != p->n_inputs) return DVM_ERR_INVALID_ARG;
+  if (n_scalars < p->n_params || (p->n_params > 0 && !scalars)) return DVM_ERR_INVALID_ARG;
+  if (out_shapes && n_out < p->n_outputs) return DVM_ERR_INVALID_ARG;
+  if (((uintptr_t)code & 7) != 0) return DVM_ERR_INVALID_ARG;
+  if (p->n_matmul > 0)
+    return dvm_encode_matmul(p, in_shapes, n_in, scalars, n_scalars, code, code_capacity, code_size,
+                             out_shapes, n_out);
+
+  Enc e;
+  e.p = p;
+  e.scalars = scalars;
+  e.n_scalars = n_scalars;
+  const int NN = p->n_nodes;
+
+  // ---- 1. shape inference (numpy-style right-aligned broadcasting) ----
+  int D = 1;
+  for (int i = 0; i < n_in; ++i) {
+    if (in_shapes[i].rank != p->nodes[p->inputs[i]].rank) return DVM_ERR_INVALID_ARG;
+    if (in_shapes[i].rank > D) D = in_shapes[i].rank;
+  }
+  {
+    int ii = 0;
+    for (int i = 0; i < NN; ++i) {
+      const Node& n = p->nodes[i];
+      int64_t* d = e.dims[i];
+      e.alias[i] = -1;
+      if (n.kind == NK_INPUT) {
+        const dvm_shape& s = in_shapes[ii++];
+        for (int k = 0; k < D; ++k) d[k] = 1;
+        for (int k = 0; k < s.rank; ++k) {
+          if (s.dims[k] < 0) return DVM_ERR_INVALID_ARG;
+          d[D - s.rank + k] = s.dims[k];
+        }
+      } else if (n.kind == NK_BINARY) {
+        const int64_t* a = e.dims[n.x];
+        const int64_t* b = e.dims[n.y];
+        for (int k = 0; k < D; ++k) {
+          if (a[k] == b[k]) d[k] = a[k];
+          else if (a[k] == 1) d[k] = b[k];
+          else if (b[k] == 1) d[k] = a[k];
+          else return DVM_ERR_SHAPE_MISMATCH;
+        }
+      } else {
+        for (int k = 0; k < D; ++k) d[k] = e.dims[n.x][k];
+        if (n.kind == NK_REDUCE) d[D - 1] = 1;
+      }
+    }
+  }
+  for (int k = 0; k < D; ++k) {
+    int64_t m = 1;
+    bool zero = false;
+    for (int i = 0; i < NN; ++i) {
+      if (e.dims[i][k] == 0) zero = true;
+      if (e.dims[i][k] > m) m = e.dims[i][k];
+    }
+    e.Sd[k] = zero ? 0 : m;
+  }
+  for (int i = 0; i < NN; ++i)
+    for (int k = 0; k < D; ++k)
+      if (e.dims[i][k] != 1 && e.dims[i][k] != e.Sd[k]) return DVM_ERR_SHAPE_MISMATCH;
+  if (out_shapes) {
+    for (int o = 0; o < p->n_outputs; ++o) {
+      // the rank of an output is the rank the dominant shape has (leading 1s kept)
+      out_shapes[o].rank = D;
+      for (int k = 0; k < DVM_MAX_RANK; ++k) out_shapes[o].dims[k] = k < D ? e.dims[p->outputs[o].value][k] : 0;
+    }
+  }
+  bool empty = false;
+  for (int k = 0; k < D; ++k) if (e.Sd[k] == 0) empty = true;
+
+  // ---- 2. classes: a value whose last dim is 1 while the dominant last dim is not is a per-row scalar ----
+  int Dt = D;  // trailing size-1 dominant dims carry no extent: drop them
+  while (Dt > 1 && e.Sd[Dt - 1] == 1) --Dt;
+  const int64_t Ccols = empty ? 1 : e.Sd[Dt - 1];
+  bool has_reduce = false;
+  for (int i = 0; i < NN; ++i) {
+    const Node& n = p->nodes[i];
+    int64_t last = e.dims[i][Dt - 1];
+    e.cls[i] = (last == 1 && Ccols > 1) ? CLS_SCAL : CLS_TILE;
+    if (n.kind == NK_REDUCE) {
+      if (Dt < D || e.dims[n.x][Dt - 1] == 1) e.alias[i] = n.x;  // reducing a size-1 axis: identity
+      else has_reduce = true;
+    }
+    if (n.kind == NK_CAST && n.dtype == DVM_F32) e.alias[i] = n.x;  // registers are fp32 already
+  }
+
+  // ---- 3. operands: inputs and outputs with their strides over the dominant dims ----
+  e.n_opd = 0;
+  int W = 4;
+  for (int i = 0; i < n_in + p->n_outputs; ++i) {
+    Operand& od = e.opd[e.n_opd];
+    int v = i < n_in ? p->inputs[i] : p->outputs[i - n_in].value;
+    od.slot = i;
+    od.dtype = i < n_in ? p->nodes[v].dtype : p->outputs[i - n_in].dtype;
+    od.primary = false;
+    int64_t st = 1;
+    for (int k = D - 1; k >= 0; --k) {
+      int64_t dk = e.dims[v][k];
+      od.stride[k] = (dk == 1 && e.Sd[k] != 1) ? 0 : st;
+      st *= dk;
+    }
+    od.col_stride = (e.dims[v][Dt - 1] == 1 && Ccols > 1) ? 0 : 1;
+    if (i >= n_in) {
+      // an output must cover the dominant shape (or be one value per row); otherwise several
+      // tiles would write the same element
+      for (int k = 0; k < Dt - 1; ++k)
+        if (e.dims[v][k] != e.Sd[k]) return DVM_ERR_UNSUPPORTED;
+      e.out_operand[i - n_in] = (int8_t)e.n_opd;
+    } else {
+      e.in_operand[v] = (int8_t)e.n_opd;
+    }
+    if (od.col_stride == 1 && od.dtype == DVM_DT_BF16) W = 8;
+    e.n_opd++;
+  }
+
+  // ---- 4. merge adjacent dims that are dense in every operand (dims of size 1 vanish) ----
+  // groups are collected innermost first; group 0 is the column dim.
+  int64_t gsize[DVM_MAX_RANK];
+  int64_t gstride[DVM_MAX_OPERANDS][DVM_MAX_RANK];
+  int ng = 0;
+  for (int k = Dt - 1; k >= 0; --k) {
+    if (e.Sd[k] == 1 && k != Dt - 1) continue;
+    bool merged = ng > 0 && !(ng == 1 && has_reduce);  // a reduced row never merges with outer dims
+    if (merged) {
+      for (int o = 0; o < e.n_opd; ++o)
+        if (e.opd[o].stride[k] != gstride[o][ng - 1] * gsize[ng - 1]) { merged = false; break; }
+    }
+    if (merged) {
+      gsize[ng - 1] *= e.Sd[k];
+    } else {
+      gsize[ng] = e.Sd[k];
+      for (int o = 0; o < e.n_opd; ++o) gstride[o][ng] = (k == Dt - 1) ? e.opd[o].col_stride : e.opd[o].stride[k];
+      ng++;
+    }
+  }
+  if (ng > 4) return DVM_ERR_UNSUPPORTED;
+  int64_t C = gsize[0];
+  int64_t outer[3] = {1, 1, 1};
+  for (int g = 1; g < ng; ++g) outer[g - 1] = gsize[g];
+  for (int o = 0; o < e.n_opd; ++o)
+    for (int g = 0; g < 3; ++g) e.opd[o].ostride[g] = (g + 1 < ng) ? gstride[o][g + 1] : 0;
+  int64_t R = outer[0] * outer[1] * outer[2];
+  if (empty) { R = 0; C = 1; }
+  const bool flat = (ng == 1) && !has_reduce;
+
+  // primary operand: the first tile-class access that spans the whole dominant shape
+  int primary = -1;
+  for (int o = 0; o < e.n_opd && primary < 0; ++o) {
+    const Operand& od = e.opd[o];
+    if (od.col_stride != 1) continue;
+    bool full = true;
+    for (int g = 0; g < 3; ++g) if (outer[g] > 1 && od.ostride[g] == 0) full = false;
+    if (full) primary = o;
+  }
+  if (primary < 0) {
+    for (int o = 0; o < e.n_opd && primary < 0; ++o) if (e.opd[o].col_stride == 1) primary = o;
+  }
+  if (primary >= 0) e.opd[primary].primary = true;
+
+  // ---- 5. shape tiling: threads per row G, column tile, tile count (cost model of Sec. 4.2) ----
+  const int V = DVM_VM_V, T = DVM_VM_THREADS;
+  const int64_t N = dvm_get_num_cores();
+  const int64_t beta = 4;  // per-tile decode overhead in element units (the paper's "+2")
+  int log2G = 8;
+  int64_t Ctile = C, CB = 1, rowsR = R, lastRowCols = C;
+  uint32_t flags = 0;
+  int64_t n_tiles = 0;
+  if (flat) {
+    int64_t total = empty ? 0 : C;  // everything merged into one dim
+    int64_t best_cost = -1, best_chunk = (int64_t)T * W;
+    for (int k = 1; k <= V / W; ++k) {
+      int64_t chunk = (int64_t)T * W * k;
+      int64_t cost = cdiv(cdiv(total, chunk), N) * (W * k + beta);
+      if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_chunk = chunk; }
+    }
+    Ctile = best_chunk;
+    rowsR = cdiv(total, Ctile);
+    lastRowCols = rowsR > 0 ? total - (rowsR - 1) * Ctile : Ctile;
+    C = Ctile;
+    CB = 1;
+    log2G = 8;
+    n_tiles = rowsR;
+    flags |= DVM_F_FLAT | DVM_F_ALIGNED;
+    for (int o = 0; o < e.n_opd; ++o) {
+      e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile : 0;
+      e.opd[o].ostride[1] = e.opd[o].ostride[2] = 0;
+    }
+    outer[0] = rowsR; outer[1] = outer[2] = 1;
+  } else {
+    // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
+    bool aligned = primary >= 0;
+    if (primary >= 0)
+      for (int g = 0; g < 3; ++g)
+        if (outer[g] > 1 && (e.opd[primary].ostride[g] % W) != 0) aligned = false;
+    int64_t best_cost = -1;
+    int bestW = W;
+    for (int pass = 0; pass < 2 && best_cost < 0; ++pass) {
+      const int w = pass == 0 ? W : 1;  // second pass: element-wise mapping, which needs no padding
+      const bool al = pass == 0 ? aligned : true;
+      const int64_t pad = al ? 0 : w - 1;
+      for (int lg = 0; lg <= 8; ++lg) {
+        int64_t G = 1 << lg, cap = G * V;
+        int64_t ct;
+        if (has_reduce) {
+          if (cap < C + pad) continue;
+          ct = C;
+        } else {
+          ct = ((cap - pad) / w) * w;
+          if (ct <= 0) continue;
+          if (ct > C) ct = C;
+        }
+        int64_t cb = cdiv(C, ct);
+        int64_t tiles = cdiv(R, T / G) * cb;
+        int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
+        int64_t cost = cdiv(tiles, N) * (u + beta);
+        if (best_cost < 0 || cost < best_cost) {
+          best_cost = cost; log2G = lg; Ctile = ct; CB = cb; n_tiles = tiles; bestW = w;
+          flags = al ? DVM_F_ALIGNED : 0;
+        }
+      }
+    }
+    if (best_cost < 0) return DVM_ERR_UNSUPPORTED;  // a reduced row does not fit the register budget
+    W = bestW;
+    if (outer[1] > 1 || outer[2] > 1) flags |= DVM_F_OUTER_DIMS;
+    lastRowCols = C;
+    if (empty) n_tiles = 0;
+  }
+  if (n_tiles > 0xffffffffll) return DVM_ERR_TOO_LARGE;
+
+  // ---- 6. code body ----
+  int nreg = 4;
+  bool ok = gen_body(e, true, 4);
+  if (!ok) ok = gen_body(e, false, 4);
+  if (!ok) { nreg = 8; ok = gen_body(e, true, 8); }
+  if (!ok) ok = gen_body(e, false, 8);
+  if (!ok) return DVM_ERR_UNSUPPORTED;  // more live tile values than tile registers
+  if (e.max_treg >= 4) nreg = 8;
+
+  // ---- 7. assemble ----
+  const int n_tensors = n_in + p->n_outputs;
+  size_t words = DVM_HDR_WORDS + 2 * (size_t)n_tensors + (size_t)DVM_OPD_WORDS * e.n_opd + e.n_body;
+  *code_size = words * 4;
+  if (!code || code_capacity < words * 4) return DVM_ERR_BUFFER_TOO_SMALL;
+  uint32_t* w = (uint32_t*)code;
+  memset(w, 0, words * 4);
+  w[DVM_H_MAGIC] = DVM_MAGIC;
+  w[DVM_H_KERNEL_TYPE] = DVM_KERNEL_VEC;
+  w[DVM_H_CODE_WORDS] = (uint32_t)e.n_body;
+  w[DVM_H_N_TILES] = (uint32_t)n_tiles;
+  w[DVM_H_TOTAL_WORDS] = (uint32_t)words;
+  w[DVM_H_COUNTS] = (uint32_t)n_tensors | ((uint32_t)n_in << 8) | ((uint32_t)e.n_opd << 16) |
+                    ((uint32_t)p->n_outputs << 24);
+  w[DVM_H_GEOM] = (uint32_t)log2G | ((uint32_t)W << 8) | ((uint32_t)nreg << 16) | (flags << 24);
+  w[DVM_H_COLS] = (uint32_t)C;
+  w[DVM_H_ROWS_LO] = (uint32_t)(flat ? rowsR : R);
+  w[DVM_H_ROWS_HI] = (uint32_t)((uint64_t)(flat ? rowsR : R) >> 32);
+  w[DVM_H_COL_BLOCKS] = (uint32_t)CB;
+  w[DVM_H_COL_TILE] = (uint32_t)Ctile;
+  w[DVM_H_OUTER0] = (uint32_t)outer[0];
+  w[DVM_H_OUTER1] = (uint32_t)outer[1];
+  w[DVM_H_OUTER2] = (uint32_t)outer[2];
+  w[DVM_H_LAST_ROW_COLS] = (uint32_t)lastRowCols;
+  w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
+  uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    uint32_t* d = ot + o * DVM_OPD_WORDS;
+    d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
+                      ((uint32_t)(od.primary ? 1 : 0) << 24);
+    for (int g = 0; g < 3; ++g) {
+      d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
+      d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
+    }
+  }
+  memcpy(ot + e.n_opd * DVM_OPD_WORDS, e.body, (size_t)e.n_body * 4);
+  if (C > 0xffffffffll || outer[0] > 0xffffffffll || outer[1] > 0xffffffffll || outer[2] > 0xffffffffll)
+    return DVM_ERR_TOO_LARGE;
+  return DVM_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Verification and the readable dump
+// ---------------------------------------------------------------------------
+static int insn_expected_len(uint32_t op, uint32_t w0) {
+  if (op == DVM_OP_NOP || op == DVM_OP_LDG || op == DVM_OP_CVT || op == DVM_OP_STG || op == DVM_OP_LDS ||
+      op == DVM_OP_STS || op == DVM_OP_MOV || op == DVM_OP_BCS)
+    return 1;
+  if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) return 2;
+  if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8 * DVM_A_NBIN) return 1;
+  if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) return 1;
+  if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) return 1;
+  if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) return 1;
+  if (op == DVM_OP_SOP) return DVM_INSN_B(w0) == DVM_SK_BINI ? 3 : 2;
+  return -1;
+}
+
+int dvm_verify_matmul(const uint32_t* w, size_t n_words);
+
+extern "C" int dvm_verify(const void* code, size_t code_size) {
+  if (!code) return DVM_ERR_INVALID_ARG;
+  if (code_size < DVM_HDR_WORDS * 4 || (code_size & 3) || ((uintptr_t)code & 3)) return DVM_ERR_BAD_CODE;
+  const uint32_t* w = (const uint32_t*)code;
+  if (w[DVM_H_MAGIC] != DVM_MAGIC) return DVM_ERR_BAD_CODE;
+  if (w[DVM_H_TOTAL_WORDS] * 4ull != code_size) return DVM_ERR_BAD_CODE;
+  if (w[DVM_H_KERNEL_TYPE] == DVM_KERNEL_MATMUL) return dvm_verify_matmul(w, code_size / 4);
+  if (w[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_BAD_CODE;
+  uint32_t counts = w[DVM_H_COUNTS];
+  uint32_t n_tensors = counts & 0xff, n_in = (counts >> 8) & 0xff, n_opd = (counts >> 16) & 0xff,
+           n_out = counts >> 24;
+  if (n_tensors > DVM_MAX_TENSORS || n_opd > DVM_MAX_OPERANDS || n_in + n_out != n_tensors) return DVM_ERR_BAD_CODE;
+  uint32_t body = w[DVM_H_CODE_WORDS];
+  if ((uint64_t)DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd + body != w[DVM_H_TOTAL_WORDS])
+    return DVM_ERR_BAD_CODE;
+  uint32_t geom = w[DVM_H_GEOM];
+  uint32_t lg = geom & 0xff, W = (geom >> 8) & 0xff, nreg = (geom >> 16) & 0xff;
+  if (lg > 8 || !(W == 1 || W == 4 || W == 8) || !(nreg == 4 || nreg == 8)) return DVM_ERR_BAD_CODE;
+  uint64_t G = 1ull << lg;
+  uint64_t ctile = w[DVM_H_COL_TILE], cb = w[DVM_H_COL_BLOCKS], C = w[DVM_H_COLS];
+  uint64_t R = (uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32);
+  uint32_t flags = geom >> 24;
+  uint64_t pad = (flags & DVM_F_ALIGNED) ? 0 : W - 1;
+  if (w[DVM_H_N_TILES] > 0) {
+    if (ctile == 0 || cb == 0 || ctile + pad > G * DVM_VM_V) return DVM_ERR_BAD_CODE;
+    if (cb * ctile < C || (cb - 1) * ctile >= C) return DVM_ERR_BAD_CODE;
+    uint64_t rpt = DVM_VM_THREADS / G;
+    if ((uint64_t)w[DVM_H_N_TILES] != ((R + rpt - 1) / rpt) * cb) return DVM_ERR_BAD_CODE;
+    if (w[DVM_H_LAST_ROW_COLS] == 0 || w[DVM_H_LAST_ROW_COLS] > C) return DVM_ERR_BAD_CODE;
+    if ((uint64_t)w[DVM_H_OUTER0] * w[DVM_H_OUTER1] * w[DVM_H_OUTER2] != R) return DVM_ERR_BAD_CODE;
+  }
+  const uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
+  int n_primary = 0;
+  for (uint32_t o = 0; o < n_opd; ++o) {
+    uint32_t info = ot[o * DVM_OPD_WORDS + DVM_OPD_INFO];
+    if ((info & 0xff) >= n_tensors) return DVM_ERR_BAD_CODE;
+    if (((info >> 8) & 0xff) > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
+    if (((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
+    n_primary += (info >> 24) & 1;
+  }
+  if (n_primary > 1) return DVM_ERR_BAD_CODE;
+  if (w[DVM_H_PRIMARY] != 0xffffffffu) {
+    if (w[DVM_H_PRIMARY] >= n_opd || !((ot[w[DVM_H_PRIMARY] * DVM_OPD_WORDS] >> 24) & 1)) return DVM_ERR_BAD_CODE;
+  } else if (n_primary != 0) {
+    return DVM_ERR_BAD_CODE;
+  }
+  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS;
+  uint32_t pc = 0;
+  while (pc < body) {
+    uint32_t w0 = b[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), bb = DVM_INSN_B(w0);
+    int el = insn_expected_len(op, w0);
+    if (el < 0 || (uint32_t)el != len || pc + len > body) return DVM_ERR_BAD_CODE;
+    if (op == DVM_OP_LDG || op == DVM_OP_STG) {
+      if (a >= nreg || bb >= n_opd) return DVM_ERR_BAD_CODE;
+      if (op == DVM_OP_STG && a != 0) return DVM_ERR_BAD_CODE;
+      uint32_t info = ot[bb * DVM_OPD_WORDS];
+      bool is_out = (info & 0xff) >= n_in;
+      if ((op == DVM_OP_STG) != is_out) return DVM_ERR_BAD_CODE;  // never store to an input, never load an output
+      if (((info >> 16) & 0xff) != 1) return DVM_ERR_BAD_CODE;
+    } else if (op == DVM_OP_LDS || op == DVM_OP_STS) {
+      if (a >= DVM_MAX_SREGS || bb >= n_opd) return DVM_ERR_BAD_CODE;
+      uint32_t info = ot[bb * DVM_OPD_WORDS];
+      bool is_out = (info & 0xff) >= n_in;
+      if ((op == DVM_OP_STS) != is_out) return DVM_ERR_BAD_CODE;
+      if (((info >> 16) & 0xff) != 0) return DVM_ERR_BAD_CODE;
+    } else if (op == DVM_OP_CVT) {
+      if (a >= nreg || bb > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
+    } else if (op == DVM_OP_MOV) {
+      if (a >= nreg || bb >= nreg || ((a == 0) == (bb == 0))) return DVM_ERR_BAD_CODE;  // to or from R0 only
+    } else if (op == DVM_OP_BCS) {
+      if (a >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
+    } else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8 * DVM_A_NBIN) {
+      if (((op - DVM_OP_BIN) & 7) >= nreg) return DVM_ERR_BAD_CODE;
+    } else if ((op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) ||
+               (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED)) {
+      if (a >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
+    } else if (op == DVM_OP_SOP) {
+      uint32_t w1 = b[pc + 1], sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
+      if (a >= DVM_MAX_SREGS || s1 >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
+      if (bb == DVM_SK_BIN) { if (sub >= DVM_A_NBIN || s2 >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE; }
+      else if (bb == DVM_SK_BINI) { if (sub >= DVM_A_NBIN) return DVM_ERR_BAD_CODE; }
+      else if (bb == DVM_SK_UN) { if (sub >= DVM_U_NUN) return DVM_ERR_BAD_CODE; }
+      else return DVM_ERR_BAD_CODE;
+    }
+    pc += len;
+  }
+  return pc == body ? DVM_OK : DVM_ERR_BAD_CODE;
+}
+
+namespace {
+struct Out {
+  char* buf;
+  size_t cap, len;
+  bool overflow;
+};
+static void outf(Out& o, const char* fmt, ...) {
+  char tmp[256];
+  va_list ap;
+  va_start(ap, fmt);
+  int n = vsnprintf(tmp, sizeof tmp, fmt, ap);
+  va_end(ap);
+  if (n < 0) return;
+  if ((size_t)n >= sizeof tmp) n = sizeof tmp - 1;
+  if (o.len + (size_t)n + 1 > o.cap) { o.overflow = true; return; }
+  memcpy(o.buf + o.len, tmp, (size_t)n);
+  o.len += (size_t)n;
+  o.buf[o.len] = 0;
+}
+static const char* kArith[8] = {"add", "sub", "rsub", "mul", "div", "rdiv", "min", "max"};
+static const char* kUn[DVM_U_NUN] = {"exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
+                                     "recip", "floor", "round", "tanh", "rnd_bf16"};
+static const char* kRed[3] = {"sum", "max", "min"};
+}  // namespace
+
+int dvm_disassemble_matmul(const uint32_t* w, size_t n_words, char* buf, size_t cap);
+
+extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, size_t cap) {
+  if (!buf || cap == 0) return DVM_ERR_INVALID_ARG;
+  buf[0] = 0;
+  int st = dvm_verify(code, code_size);
+  if (st != DVM_OK) return st;
+  const uint32_t* w = (const uint32_t*)code;
+  if (w[DVM_H_KERNEL_TYPE] == DVM_KERNEL_MATMUL) return dvm_disassemble_matmul(w, code_size / 4, buf, cap);
+  Out o = {buf, cap, 0, false};
+  uint32_t counts = w[DVM_H_COUNTS];
+  uint32_t n_tensors = counts & 0xff, n_in = (counts >> 8) & 0xff, n_opd = (counts >> 16) & 0xff;
+  uint32_t geom = w[DVM_H_GEOM];
+  int64_t n_tiles = w[DVM_H_N_TILES];
+  int cores = dvm_get_num_cores();
+  outf(o, "kernel vmain.vec  block_dim=%lld  body_tile=%lld  code_size=%u\n", (long long)n_tiles,
+       (long long)((n_tiles + cores - 1) / cores), w[DVM_H_CODE_WORDS] * 4);
+  outf(o, "  rows=%llu cols=%u col_tile=%u col_blocks=%u threads_per_row=%u vec=%u tile_regs=%u flags=%s%s%s\n",
+       (unsigned long long)((uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32)), w[DVM_H_COLS],
+       w[DVM_H_COL_TILE], w[DVM_H_COL_BLOCKS], 1u << (geom & 0xff), (geom >> 8) & 0xff, (geom >> 16) & 0xff,
+       ((geom >> 24) & DVM_F_ALIGNED) ? "A" : "-", ((geom >> 24) & DVM_F_OUTER_DIMS) ? "O" : "-",
+       ((geom >> 24) & DVM_F_FLAT) ? "F" : "-");
+  const uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
+  for (uint32_t k = 0; k < n_opd; ++k) {
+    const uint32_t* d = ot + k * DVM_OPD_WORDS;
+    uint32_t info = d[0];
+    outf(o, "  operand m%u: %s%u %s col_stride=%u strides=[%lld,%lld,%lld]%s\n", k,
+         (info & 0xff) < n_in ? "in" : "out", (info & 0xff) < n_in ? (info & 0xff) : (info & 0xff) - n_in,
+         ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", (info >> 16) & 0xff,
+         (long long)((uint64_t)d[2] | ((uint64_t)d[3] << 32)), (long long)((uint64_t)d[4] | ((uint64_t)d[5] << 32)),
+         (long long)((uint64_t)d[6] | ((uint64_t)d[7] << 32)), (info >> 24) & 1 ? " primary" : "");
+  }
+  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS;
+  uint32_t body = w[DVM_H_CODE_WORDS], pc = 0;
+  while (pc < body) {
+    uint32_t w0 = b[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), bb = DVM_INSN_B(w0);
+    outf(o, "  %04x: ", pc * 4);
+    float imm = 0.f;
+    if (len >= 2) memcpy(&imm, &b[pc + len - 1], 4);
+    if (op == DVM_OP_NOP) outf(o, "nop\n");
+    else if (op == DVM_OP_LDG) outf(o, "load      r%u, m%u\n", a, bb);
+    else if (op == DVM_OP_CVT) outf(o, "widen     r%u, %s\n", a, bb == DVM_DT_BF16 ? "bf16" : "f32");
+    else if (op == DVM_OP_STG) outf(o, "store     m%u, r%u\n", bb, a);
+    else if (op == DVM_OP_LDS) outf(o, "load.row  s%u, m%u\n", a, bb);
+    else if (op == DVM_OP_STS) outf(o, "store.row m%u, s%u\n", bb, a);
+    else if (op == DVM_OP_MOV) outf(o, "copy      r%u, r%u\n", a, bb);
+    else if (op == DVM_OP_BCS) outf(o, "broadcast r0, s%u\n", a);
+    else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + 8) outf(o, "%ss      r0, %.9g\n", kArith[op - DVM_OP_BINI], imm);
+    else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 64)
+      outf(o, "%-9s r0, r0, r%u\n", kArith[(op - DVM_OP_BIN) >> 3], (op - DVM_OP_BIN) & 7);
+    else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + 8) outf(o, "%-9s r0, r0, s%u\n", kArith[op - DVM_OP_BINS], a);
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) outf(o, "%-9s r0, r0\n", kUn[op - DVM_OP_UN]);
+    else if (op >= DVM_OP_RED && op < DVM_OP_RED + 3) outf(o, "row%-6s s%u, r0\n", kRed[op - DVM_OP_RED], a);
+    else if (op == DVM_OP_SOP) {
+      uint32_t w1 = b[pc + 1], sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
+      if (bb == DVM_SK_BIN) outf(o, "s.%-7s s%u, s%u, s%u\n", kArith[sub], a, s1, s2);
+      else if (bb == DVM_SK_BINI) outf(o, "s.%ss    s%u, s%u, %.9g\n", kArith[sub], a, s1, imm);
+      else outf(o, "s.%-7s s%u, s%u\n", kUn[sub], a, s1);
+    }
+    pc += len;
+  }
+  return o.overflow ? DVM_ERR_BUFFER_TOO_SMALL : DVM_OK;
+}
+
+extern "C" int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t* n_tiles,
+                             int* code_body_bytes, int* threads_per_row, int* vector_width, int* n_tile_regs) {
+  int st = dvm_verify(code, code_size);
+  if (st != DVM_OK) return st;
+  const uint32_t* w = (const uint32_t*)code;
+  if (kernel_type) *kernel_type = (int)w[DVM_H_KERNEL_TYPE];
+  if (n_tiles) *n_tiles = w[DVM_H_N_TILES];
+  if (code_body_bytes) *code_body_bytes = (int)w[DVM_H_CODE_WORDS] * 4;
+  uint32_t geom = w[DVM_H_GEOM];
+  if (threads_per_row) *threads_per_row = 1 << (geom & 0xff);
+  if (vector_width) *vector_width = (geom >> 8) & 0xff;
+  if (n_tile_regs) *n_tile_regs = (geom >> 16) & 0xff;
+  return DVM_OK;
+}
+
+extern "C" const char* dvm_strerror(int status) {
+  switch (status) {
+    case DVM_OK: return "ok";
+    case DVM_ERR_INVALID_ARG: return "invalid argument";
+    case DVM_ERR_SHAPE_MISMATCH: return "shapes do not broadcast";
+    case DVM_ERR_UNSUPPORTED: return "program not supported by the virtual machine";
+    case DVM_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case DVM_ERR_BAD_CODE: return "bytecode failed verification";
+    case DVM_ERR_CUDA: return "CUDA runtime error";
+    case DVM_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case DVM_ERR_DEVICE_BAD_CODE: return "device met an undecodable instruction";
+    case DVM_ERR_NOT_FINALIZED: return "program not finalized";
+    case DVM_ERR_TOO_LARGE: return "program exceeds a library limit";
+    default: return "unknown status";
+  }
+}

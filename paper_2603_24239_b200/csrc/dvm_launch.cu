@@ -1,0 +1,250 @@
+// Launch side of libdvm: sends a bytecode program to the device (as the kernel-parameter block)
+// and starts the virtual machine on a persistent grid.
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/dvm.h"
+#include "dvm_format.h"
+#include "dvm_internal.h"
+#include "dvm_launch.h"
+#include "dvm_vm.cuh"
+
+namespace {
+
+constexpr int PW_SMALL = 496;    // words of code in a 2 KB parameter block
+constexpr int PW_LARGE = 8000;   // ... in a 32 KB parameter block (the sm_70+ limit is 32764 bytes)
+constexpr int QUEUE_SLOTS = 504;
+constexpr int MAX_DEVICES = 64;
+
+struct DeviceState {
+  bool ready = false;
+  unsigned int* scratch = nullptr;  // [0] status word, [8 + 2*slot] work-queue counter pairs
+  int sm_count = 0;
+  int occ[2][2] = {{0, 0}, {0, 0}};  // resident CTAs per SM for [nreg8][large]
+  unsigned queue_slot = 0;
+};
+
+DeviceState g_dev[MAX_DEVICES];
+std::mutex g_mu;
+thread_local int t_last_cuda_error = 0;
+long long g_launches = 0;
+
+#define DVM_CUDA(call)                       \
+  do {                                       \
+    cudaError_t e_ = (call);                 \
+    if (e_ != cudaSuccess) {                 \
+      t_last_cuda_error = (int)e_;           \
+      return DVM_ERR_CUDA;                   \
+    }                                        \
+  } while (0)
+
+template <int NREG, int PW>
+int occupancy(int* out, size_t smem) {
+  int n = 0;
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<NREG, PW>, dvm::THREADS, smem));
+  *out = n > 0 ? n : 1;
+  return DVM_OK;
+}
+
+}  // namespace
+
+int dvm_device_state(DvmDeviceInfo* info) {
+  int dev = 0;
+  DVM_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return DVM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceState& d = g_dev[dev];
+  if (!d.ready) {
+    DVM_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    DVM_CUDA(cudaMalloc(&d.scratch, 4096));
+    DVM_CUDA(cudaMemset(d.scratch, 0, 4096));
+    int st;
+    if ((st = occupancy<4, PW_SMALL>(&d.occ[0][0], 2048)) != DVM_OK) return st;
+    if ((st = occupancy<4, PW_LARGE>(&d.occ[0][1], 32768)) != DVM_OK) return st;
+    if ((st = occupancy<8, PW_SMALL>(&d.occ[1][0], 2048)) != DVM_OK) return st;
+    if ((st = occupancy<8, PW_LARGE>(&d.occ[1][1], 32768)) != DVM_OK) return st;
+    d.ready = true;
+  }
+  info->scratch = d.scratch;
+  info->sm_count = d.sm_count;
+  info->queue_slot = d.queue_slot;
+  d.queue_slot = (d.queue_slot + 1) % QUEUE_SLOTS;
+  memcpy(info->occ, d.occ, sizeof d.occ);
+  return DVM_OK;
+}
+
+void dvm_note_cuda_error(int e) { t_last_cuda_error = e; }
+void dvm_count_launch() { __atomic_add_fetch(&g_launches, 1, __ATOMIC_RELAXED); }
+
+extern "C" int dvm_last_cuda_error(void) { return t_last_cuda_error; }
+extern "C" int64_t dvm_launch_count(void) { return (int64_t)__atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
+
+namespace {
+
+// Copies one verified vector program into `dst`, patches its tensor table, and falls back to
+// the element-wise mapping (W = 1) when the program assumed 16-byte aligned rows but the primary
+// operand's base pointer is not.
+int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int n_tensors) {
+  const uint32_t total = code[DVM_H_TOTAL_WORDS];
+  memcpy(dst, code, (size_t)total * 4);
+  const uint32_t counts = code[DVM_H_COUNTS];
+  const uint32_t nt = counts & 0xff, n_opd = (counts >> 16) & 0xff;
+  if ((uint32_t)n_tensors != nt) return DVM_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < nt; ++i) {
+    if (!tensors[i]) return DVM_ERR_INVALID_ARG;
+    unsigned long long a = (unsigned long long)(uintptr_t)tensors[i];
+    dst[DVM_HDR_WORDS + 2 * i] = (uint32_t)a;
+    dst[DVM_HDR_WORDS + 2 * i + 1] = (uint32_t)(a >> 32);
+  }
+  const uint32_t* ot = code + DVM_HDR_WORDS + 2 * nt;
+  for (uint32_t o = 0; o < n_opd; ++o) {
+    uint32_t info = ot[o * DVM_OPD_WORDS];
+    uintptr_t a = (uintptr_t)tensors[info & 0xff];
+    uintptr_t es = ((info >> 8) & 0xff) == DVM_DT_BF16 ? 2 : 4;
+    if (a % es) return DVM_ERR_INVALID_ARG;
+  }
+  uint32_t geom = code[DVM_H_GEOM];
+  uint32_t W = (geom >> 8) & 0xff, flags = geom >> 24;
+  if ((flags & DVM_F_ALIGNED) && W > 1 && code[DVM_H_PRIMARY] != 0xffffffffu) {
+    uint32_t info = ot[code[DVM_H_PRIMARY] * DVM_OPD_WORDS];
+    if (((uintptr_t)tensors[info & 0xff]) & 15) dst[DVM_H_GEOM] = (geom & ~0xff00u) | (1u << 8);
+  }
+  return DVM_OK;
+}
+
+template <int NREG, int PW>
+int launch_variant(const dvm::VMParams<PW>& prm, int grid, cudaStream_t stream) {
+  size_t smem = (size_t)prm.n_words * 4;
+  dvm::dvm_vm_kernel<NREG, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  DVM_CUDA(cudaGetLastError());
+  dvm_count_launch();
+  return DVM_OK;
+}
+
+thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
+
+int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
+               bool use_queue, cudaStream_t stream) {
+  // directory: [program word offsets (n)][tile prefix sums (n+1)]
+  uint32_t dir = 2 * (uint32_t)n_programs + 1;
+  uint64_t need = dir;
+  uint64_t total_tiles = 0;
+  uint32_t nreg = 4;
+  for (int i = 0; i < n_programs; ++i) {
+    const uint32_t* c = (const uint32_t*)codes[i];
+    need += c[DVM_H_TOTAL_WORDS];
+    total_tiles += c[DVM_H_N_TILES];
+    if (((c[DVM_H_GEOM] >> 16) & 0xff) > nreg) nreg = 8;
+  }
+  if (need > PW_LARGE || total_tiles > 0xffffffffull) return DVM_ERR_TOO_LARGE;
+  if (total_tiles == 0) return DVM_OK;
+
+  DvmDeviceInfo dev;
+  int st = dvm_device_state(&dev);
+  if (st != DVM_OK) return st;
+
+  dvm::VMParams<PW_LARGE>& P = t_large;
+  uint32_t pos = dir, tb = 0;
+  for (int i = 0; i < n_programs; ++i) {
+    const uint32_t* c = (const uint32_t*)codes[i];
+    P.words[i] = pos;
+    P.words[n_programs + i] = tb;
+    st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
+    if (st != DVM_OK) return st;
+    pos += c[DVM_H_TOTAL_WORDS];
+    tb += c[DVM_H_N_TILES];
+  }
+  P.words[2 * n_programs] = tb;
+  P.n_programs = (uint32_t)n_programs;
+  P.total_tiles = (uint32_t)total_tiles;
+  P.n_words = pos;
+  P.use_queue = use_queue ? 1u : 0u;
+  P.status = dev.scratch;
+  P.queue = dev.scratch + 8 + 2 * dev.queue_slot;
+
+  const bool large = pos > PW_SMALL;
+  const int occ = dev.occ[nreg == 8][large];
+  uint64_t slots = (uint64_t)dev.sm_count * occ;
+  int grid = (int)(total_tiles < slots ? total_tiles : slots);
+  if (!large) {
+    dvm::VMParams<PW_SMALL> S;
+    memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
+    return nreg == 8 ? launch_variant<8, PW_SMALL>(S, grid, stream) : launch_variant<4, PW_SMALL>(S, grid, stream);
+  }
+  return nreg == 8 ? launch_variant<8, PW_LARGE>(P, grid, stream) : launch_variant<4, PW_LARGE>(P, grid, stream);
+}
+
+}  // namespace
+
+extern "C" int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_tensors,
+                          void* cuda_stream) {
+  if (!code || !tensors) return DVM_ERR_INVALID_ARG;
+  int st = dvm_verify(code, code_size);
+  if (st != DVM_OK) return st;
+  const uint32_t* w = (const uint32_t*)code;
+  if (w[DVM_H_KERNEL_TYPE] == DVM_KERNEL_MATMUL)
+    return dvm_launch_matmul(w, code_size / 4, tensors, n_tensors, (cudaStream_t)cuda_stream);
+  const void* codes[1] = {code};
+  void* const* tl[1] = {tensors};
+  return launch_vec(1, codes, tl, &n_tensors, false, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
+                                  void* const* const* tensors, const int* n_tensors, void* cuda_stream) {
+  if (n_programs < 0 || (n_programs > 0 && (!codes || !code_sizes || !tensors || !n_tensors)))
+    return DVM_ERR_INVALID_ARG;
+  if (n_programs == 0) return DVM_OK;
+  if (n_programs > DVM_MAX_STACK) return DVM_ERR_TOO_LARGE;
+  for (int i = 0; i < n_programs; ++i) {
+    if (!codes[i] || !tensors[i]) return DVM_ERR_INVALID_ARG;
+    int st = dvm_verify(codes[i], code_sizes[i]);
+    if (st != DVM_OK) return st;
+    // only vector meta-kernels stack (Sec. 5.1: stacking of meta-kernels on the Vector units)
+    if (((const uint32_t*)codes[i])[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_UNSUPPORTED;
+  }
+  return launch_vec(n_programs, codes, tensors, n_tensors, true, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int dvm_run_host(const void* code, size_t code_size, void* const* host_tensors,
+                            const size_t* tensor_bytes, int n_tensors, void* staging, size_t staging_bytes,
+                            void* cuda_stream) {
+  if (!code || !host_tensors || !tensor_bytes || !staging) return DVM_ERR_INVALID_ARG;
+  int st = dvm_verify(code, code_size);
+  if (st != DVM_OK) return st;
+  const uint32_t* w = (const uint32_t*)code;
+  const uint32_t counts = w[DVM_H_COUNTS];
+  const int nt = counts & 0xff, n_in = (counts >> 8) & 0xff;
+  if (n_tensors != nt || nt > DVM_MAX_TENSORS) return DVM_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  void* dev[DVM_MAX_TENSORS];
+  size_t off = 0;
+  for (int i = 0; i < nt; ++i) {
+    dev[i] = (char*)staging + off;
+    off += (tensor_bytes[i] + 255) & ~(size_t)255;
+  }
+  if (off > staging_bytes) return DVM_ERR_BUFFER_TOO_SMALL;
+  for (int i = 0; i < n_in; ++i)
+    if (tensor_bytes[i]) DVM_CUDA(cudaMemcpyAsync(dev[i], host_tensors[i], tensor_bytes[i], cudaMemcpyHostToDevice, stream));
+  st = dvm_launch(code, code_size, dev, nt, cuda_stream);
+  if (st != DVM_OK) return st;
+  for (int i = n_in; i < nt; ++i)
+    if (tensor_bytes[i]) DVM_CUDA(cudaMemcpyAsync(host_tensors[i], dev[i], tensor_bytes[i], cudaMemcpyDeviceToHost, stream));
+  DVM_CUDA(cudaStreamSynchronize(stream));
+  return DVM_OK;
+}
+
+extern "C" int dvm_last_device_status(void* cuda_stream, int* status) {
+  if (!status) return DVM_ERR_INVALID_ARG;
+  DVM_CUDA(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+  DvmDeviceInfo dev;
+  int st = dvm_device_state(&dev);
+  if (st != DVM_OK) return st;
+  unsigned int v = 0;
+  DVM_CUDA(cudaMemcpy(&v, dev.scratch, 4, cudaMemcpyDeviceToHost));
+  if (v) DVM_CUDA(cudaMemset(dev.scratch, 0, 4));
+  *status = v == dvm::ST_OK ? DVM_OK : (v == dvm::ST_TIMEOUT ? DVM_ERR_DEVICE_TIMEOUT : DVM_ERR_DEVICE_BAD_CODE);
+  return DVM_OK;
+}

@@ -1,0 +1,81 @@
+"""Helpers shared by the parity tests: run a program through the C-ABI on the GPU,
+evaluate the same inputs with the CPU oracle, and apply the tolerance gates.
+
+Gates (derivation in DESIGN.md, "Tolerances"):
+  G1  |g - o| <= R * max(|o|, max_j |o_row_j|)   every program, every element
+  G2  |g - o| <= R * |o|                          programs without subtractive cancellation
+  G3  exact                                       structural zeros / integer outputs
+with R = 1e-5 for fp32 programs and 2e-2 for bf16 programs.  Non-finite oracle
+values must be matched in class and sign.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from oracle import dvm_oracle as orc
+
+TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+R_TOL = {"f32": 1e-5, "bf16": 2e-2}
+
+
+def program_dtype(prog: wl.OpProgram) -> str:
+    """bf16 if any tensor of the program is bf16 (the looser tolerance applies), else f32."""
+    kinds = [n[1] for n in prog.nodes if n[0] == "input"] + [n[2] for n in prog.nodes if n[0] == "output"]
+    return "bf16" if "bf16" in kinds else "f32"
+
+
+def gpu_run(prog: wl.OpProgram, inputs, params=(), stream=None, poison=True):
+    """Encode for the inputs' shapes, launch once, return (outputs, code)."""
+    p = dvm.program_from_nodes(prog.nodes)
+    dev_in = [t.cuda() for t in inputs]
+    code = dvm.encode(p, [tuple(t.shape) for t in dev_in], params)
+    outs = []
+    for shp, node in zip(code.out_shapes, prog.output_nodes):
+        o = torch.empty(shp, dtype=TORCH_DT[node[2]], device="cuda")
+        if poison:
+            o.fill_(float("nan"))
+        outs.append(o)
+    torch.cuda.synchronize()
+    dvm.launch(code, dev_in + outs, stream)
+    assert dvm.last_device_status(stream) == 0
+    return outs, code
+
+
+def oracle_run(prog: wl.OpProgram, inputs, params=()):
+    return orc.evaluate(prog.nodes, [wl.to_f64(t) for t in inputs], params)
+
+
+def gate_errors(got: np.ndarray, want: np.ndarray):
+    """Returns (g1_err, g2_err): max over elements of |g-o| / scale for both denominators."""
+    got = np.asarray(got, dtype=np.float64)
+    assert got.shape == want.shape, (got.shape, want.shape)
+    fin = np.isfinite(want)
+    # non-finite values: same class and sign
+    assert np.array_equal(np.isnan(got), np.isnan(want)), "NaN pattern differs"
+    inf = np.isinf(want)
+    assert np.array_equal(got[inf], want[inf]), "infinities differ"
+    if want.size == 0:
+        return 0.0, 0.0
+    diff = np.where(fin, np.abs(got - np.where(fin, want, 0.0)), 0.0)
+    absw = np.where(fin, np.abs(want), 0.0)
+    rowmax = np.max(absw, axis=-1, keepdims=True) if want.ndim else absw
+    den1 = np.maximum(absw, rowmax)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        g1 = np.where(diff == 0, 0.0, diff / den1)
+        g2 = np.where(diff == 0, 0.0, diff / absw)
+    return float(np.max(g1)), float(np.max(g2))
+
+
+def check(prog, got_list, want_list, strict=False, tol=None):
+    r = tol if tol is not None else R_TOL[program_dtype(prog)]
+    worst = (0.0, 0.0)
+    for g, w in zip(got_list, want_list):
+        g1, g2 = gate_errors(wl.to_f64(g) if isinstance(g, torch.Tensor) else g, w)
+        assert g1 <= r, f"{prog.name}: G1 error {g1:.3e} > {r:.1e}"
+        if strict:
+            assert g2 <= r, f"{prog.name}: G2 (strict) error {g2:.3e} > {r:.1e}"
+        worst = (max(worst[0], g1), max(worst[1], g2))
+    return worst
