@@ -128,6 +128,12 @@ size_t dvm_code_max_size(const dvm_program* p);
  * n <= 0 restores the default.  Process-wide; not thread-safe against encode. */
 void dvm_set_num_cores(int n);
 int dvm_get_num_cores(void);
+/* Elements of a tile register that one thread holds (the analogue of the paper's tile size
+ * limit T_max = M / n_max): 16 or 32.  0 (default) lets the cost model choose per instance.
+ * Programs stacked into one launch must all use the same value, so callers of
+ * dvm_launch_stacked fix it before encoding.  Process-wide; not thread-safe against encode. */
+void dvm_set_elems_per_thread(int v);
+int dvm_get_elems_per_thread(void);
 
 /* The paper's tile-size rule for a flat vector operator (Sec. 4.2,
  * hardware_align_div): among tile sizes t in [1, min(total, t_max)] take the
@@ -156,7 +162,8 @@ int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_t
 /* Stacking-based fusion (Sec. 5.1): n_programs independent vector meta-kernels
  * run as ONE kernel; their tiles are claimed from one work queue, spread over
  * SMs (spatial) and run back to back on each SM (temporal).
- * codes[i] / code_sizes[i] / tensors[i] / n_tensors[i] as for dvm_launch. */
+ * codes[i] / code_sizes[i] / tensors[i] / n_tensors[i] as for dvm_launch.  All programs must have
+ * been encoded with the same elements-per-thread setting (DVM_ERR_INVALID_ARG otherwise). */
 int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
                        void* const* const* tensors, const int* n_tensors, void* cuda_stream);
 

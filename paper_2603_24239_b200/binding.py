@@ -64,6 +64,8 @@ _sig = {
     "dvm_code_max_size": ([_vp], _sz),
     "dvm_set_num_cores": ([_i], None),
     "dvm_get_num_cores": ([], _i),
+    "dvm_set_elems_per_thread": ([_i], None),
+    "dvm_get_elems_per_thread": ([], _i),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -99,7 +101,7 @@ class Program:
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
+        if h and lib is not None:
             lib.dvm_program_destroy(h)
 
     def _node(self, fn, *args) -> int:
@@ -316,3 +318,7 @@ def set_num_cores(n: int):
 
 def get_num_cores() -> int:
     return lib.dvm_get_num_cores()
+
+
+def set_elems_per_thread(v: int):
+    lib.dvm_set_elems_per_thread(v)

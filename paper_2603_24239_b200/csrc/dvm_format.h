@@ -9,6 +9,7 @@
 //   [ header : DVM_HDR_WORDS words ]
 //   [ tensor table : 2 words per tensor slot (device pointer, patched at launch) ]
 //   [ operand table : DVM_OPD_WORDS words per global-memory operand ]
+//   [ local register table : one word per local register: unit offset of buffer 0 | buffer 1 << 16 ]
 //   [ code body : CodeSize words, instructions of 1..3 words ]
 //
 // Unlike the paper's bytecode, a memory instruction does not carry an address:
@@ -34,7 +35,7 @@ enum {
   DVM_H_N_TILES = 3,      // total number of tiles
   DVM_H_TOTAL_WORDS = 4,  // header + tables + body
   DVM_H_COUNTS = 5,       // n_tensors | n_inputs << 8 | n_operands << 16 | n_outputs << 24
-  DVM_H_GEOM = 6,         // log2G | W << 8 | nreg << 16 | flags << 24
+  DVM_H_GEOM = 6,         // log2G | W << 8 | local registers << 16 | flags << 24
   DVM_H_COLS = 7,         // C: columns of the dominant (collapsed) shape
   DVM_H_ROWS_LO = 8,      // R: rows of the dominant shape (64 bit)
   DVM_H_ROWS_HI = 9,
@@ -45,7 +46,11 @@ enum {
   DVM_H_OUTER2 = 14,
   DVM_H_LAST_ROW_COLS = 15,  // valid columns of the last row (flat programs), else C
   DVM_H_PRIMARY = 16,        // operand whose row starts define the vector alignment, or 0xffffffff
-  DVM_HDR_WORDS = 20         // 17..19 reserved (zero)
+  DVM_H_LOCAL = 17,          // n_in_regs | n_tmp_regs << 8 | n_scalar_slots << 16 | V << 24 (elements per thread: 16 or 32)
+  DVM_H_LOAD_WORDS = 18,     // length of the load section (words) at the start of the code body
+  DVM_H_LOCAL2 = 19,         // staging unit offset (buffer 0) | scalar-slot unit offset << 8 | total units << 16 |
+                             // staging unit offset (buffer 1) << 24
+  DVM_HDR_WORDS = 20
 };
 
 // flags in DVM_H_GEOM bits 24..31
@@ -70,8 +75,11 @@ enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
 
 // ---- limits ----
 #define DVM_VM_THREADS 256       // threads per CTA of the interpreter
-#define DVM_VM_V 16              // elements of a tile register held by one thread
-#define DVM_MAX_TREGS 8          // tile registers (R0 is the accumulator)
+#define DVM_VM_VMAX 32           // most elements of a tile register one thread holds (V is 16 or 32)
+#define DVM_MAX_LREGS 10         // local tile registers of a program (inputs + temporaries)
+#define DVM_MAX_SSLOTS 8         // per-row scalar inputs of a program
+#define DVM_LOCAL_UNIT 8192      // bytes of one local-memory unit: 32 B per thread (16 bf16 or 8 fp32 words)
+#define DVM_MAX_LOCAL_UNITS 27   // units a CTA can hold (2 x inputs + temporaries + staging + scalars), 216 KB
 #define DVM_MAX_SREGS 8          // per-row scalar registers
 #define DVM_MAX_TENSORS 16
 #define DVM_MAX_OPERANDS 24
@@ -97,28 +105,38 @@ enum {
   DVM_U_ERF = 5, DVM_U_SIGMOID = 6, DVM_U_NEG = 7, DVM_U_RECIP = 8, DVM_U_FLOOR = 9,
   DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12, DVM_U_NUN = 13
 };
-enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_NRED = 3 };
+// SUMSQ (sum of squares of R0, R0 kept) is what the encoder emits for reduce_sum(x * x).
+enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_SUMSQ = 3, DVM_R_NRED = 4 };
 
-// Instruction ids.  R0 is the accumulator: arithmetic reads and writes R0.
+// Instruction ids.  The code body is [load section][compute section].
+// ACC is the register-resident accumulator tile; L[k] are tile registers in local (shared) memory,
+// thread-private, k < n_in: input registers (double buffered, filled by the load section of the
+// next tile while the current one is computed), k >= n_in: temporaries; S[k] are per-row scalars.
 enum {
   DVM_OP_NOP = 0x00,
-  DVM_OP_LDG = 0x01,   // a = tile reg, b = operand      : issue the tile load (raw element bits)
-  DVM_OP_CVT = 0x02,   // a = tile reg, b = dtype        : widen raw bits to fp32 in place
-  DVM_OP_STG = 0x03,   // a = 0,        b = operand      : narrow R0 and store the tile
-  DVM_OP_LDS = 0x04,   // a = scalar reg, b = operand    : load one value per row
-  DVM_OP_STS = 0x05,   // a = scalar reg, b = operand    : store one value per row
-  DVM_OP_MOV = 0x06,   // a = dst tile reg, b = src tile reg
-  DVM_OP_BCS = 0x07,   // a = scalar reg                 : R0 = broadcast(S[a])   (Table 1, Broadcast)
-  DVM_OP_BINI = 0x10,  // 0x10 + arith; len 2, word1 = fp32 immediate : R0 = R0 op imm  (Adds/Muls)
-  DVM_OP_BIN = 0x20,   // 0x20 + arith * 8 + reg                      : R0 = R0 op R[reg]
-  DVM_OP_BINS = 0x60,  // 0x60 + arith; a = scalar reg                : R0 = R0 op S[a] (row broadcast)
-  DVM_OP_UN = 0x70,    // 0x70 + unary                                : R0 = f(R0)
-  DVM_OP_RED = 0x80,   // 0x80 + reduce; a = dst scalar reg           : S[a] = reduce(R0) over the row
-  DVM_OP_SOP = 0x90,   // per-row scalar arithmetic; a = dst scalar reg, b = kind;
+  DVM_OP_LDG = 0x01,   // [load] a = local register (| 0x80: tile-invariant, loaded once per CTA and program),
+                       //        b = operand : async tile load (raw element bits)
+  DVM_OP_LDS = 0x02,   // [load] a = scalar slot,    b = operand : async load of one value per row
+  DVM_OP_LDA = 0x03,   // a = local register, b = dtype of its content : ACC = widen(L[a])
+  DVM_OP_STA = 0x04,   // a = local register                           : L[a] = ACC (fp32)   (Table 1, Copy)
+  DVM_OP_LSS = 0x05,   // a = scalar register, b = scalar slot          : S[a] = loaded per-row value
+  DVM_OP_STG = 0x06,   // b = operand                                  : narrow ACC and store the tile
+  DVM_OP_STS = 0x07,   // a = scalar register, b = operand             : store one value per row
+  DVM_OP_BCS = 0x08,   // a = scalar register                          : ACC = broadcast(S[a]) (Table 1, Broadcast)
+  DVM_OP_SOP = 0x09,   // per-row scalar arithmetic; a = dst scalar register, b = kind;
                        // len 2: word1 = sub_op | src1 << 8 | src2 << 16 ; len 3: word2 = fp32 immediate
-  DVM_OP_LAST = 0x91
+  DVM_OP_BINI = 0x10,  // 0x10 + arith; len 2, word1 = fp32 immediate  : ACC = ACC op imm     (Adds / Muls)
+  DVM_OP_BIN = 0x18,   // 0x18 + arith; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC op L[a]
+  DVM_OP_BINS = 0x20,  // 0x20 + arith; a = scalar register            : ACC = ACC op S[a]    (row broadcast)
+  DVM_OP_UN = 0x28,    // 0x28 + unary (13)                            : ACC = f(ACC)
+  DVM_OP_RED = 0x38,   // 0x38 + reduce (4); a = dst scalar register   : S[a] = reduce(ACC) over the row
+  DVM_OP_LD2 = 0x40,   // 0x40 + arith; a = local register x, b = local register y | dtype(x) << 6 | dtype(y) << 7
+                       //                                             : ACC = L[x] op L[y]   (fused copy + arithmetic)
+  DVM_OP_LAST = 0x48   // every arithmetic class starts at a multiple of 8: the low 3 bits are the operation
 };
-enum { DVM_SK_BIN = 0, DVM_SK_BINI = 1, DVM_SK_UN = 2 };
+#define DVM_REG_ACC 0xff
+// DVM_SK_FMAU: S[a] = unary(S[src] * imm0 + imm1); len 4: word1 = unary (0xff: none) | src << 8, word2 = imm0, word3 = imm1
+enum { DVM_SK_BIN = 0, DVM_SK_BINI = 1, DVM_SK_UN = 2, DVM_SK_FMAU = 3 };
 
 // ---- matmul meta-kernel: extra header words follow the common header ----
 // (see dvm_matmul.cu)

@@ -46,6 +46,9 @@ struct dvm_program {
 static int g_num_cores = 0;
 static const int kDefaultCores = 148 * 3;
 
+static int g_elems_per_thread = 0;
+extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 32) ? v : 0; }
+extern "C" int dvm_get_elems_per_thread(void) { return g_elems_per_thread; }
 extern "C" void dvm_set_num_cores(int n) { g_num_cores = n > 0 ? n : 0; }
 extern "C" int dvm_get_num_cores(void) { return g_num_cores > 0 ? g_num_cores : kDefaultCores; }
 
@@ -270,28 +273,33 @@ struct Operand {       // one global-memory access
 
 struct Enc {
   const dvm_program* p;
-  int D;                          // rank of the dominant shape
   int64_t Sd[DVM_MAX_RANK];       // dominant shape
   int64_t dims[DVM_MAX_NODES][DVM_MAX_RANK];  // right-aligned per value
   int8_t cls[DVM_MAX_NODES];
   int16_t alias[DVM_MAX_NODES];   // identity nodes resolve to another value
-  bool reduce_identity_axis;
   // code generation state
-  uint32_t body[8 * DVM_MAX_NODES + 64];
+  uint32_t loads[4 * DVM_MAX_TENSORS];          // load section
+  int n_loads;
+  uint32_t body[8 * DVM_MAX_NODES + 64];        // compute section
   int n_body;
   Operand opd[DVM_MAX_OPERANDS];
   int n_opd;
   int16_t uses[DVM_MAX_NODES];
-  int8_t reg_of[DVM_MAX_NODES];   // tile register >= 1 holding the value, or -1
+  int8_t lreg_of[DVM_MAX_NODES];  // local (shared-memory) register holding the value, or -1
+  int8_t ldt_of[DVM_MAX_NODES];   // element type of that register's content
   int8_t sreg_of[DVM_MAX_NODES];
-  int16_t treg_val[DVM_MAX_TREGS];
-  bool needs_cvt[DVM_MAX_TREGS];
+  int8_t sslot_of[DVM_MAX_NODES]; // local scalar slot of a per-row scalar input
+  int16_t tmp_val[DVM_MAX_LREGS]; // temporaries: value held or -1
   int16_t sreg_val[DVM_MAX_SREGS];
-  int16_t acc;                    // value in R0 or -1
-  int nreg_limit;
-  int max_treg;
-  int8_t in_operand[DVM_MAX_NODES];   // operand index of an input value
-  bool stored[DVM_MAX_TENSORS];       // output already stored
+  int16_t acc;                    // value in the accumulator or -1
+  int n_in_regs, n_tmp_regs, n_sslots;
+  bool fused_sq[DVM_MAX_NODES];   // x*x whose only consumer is a row sum: folded into that reduction
+  bool fused_sc[DVM_MAX_NODES];   // per-row scalar muls/adds folded into a later multiply-add(-unary) instruction
+  int16_t n_cons[DVM_MAX_NODES];  // number of consuming nodes / outputs of a value
+  int16_t one_cons[DVM_MAX_NODES];// the consuming node when there is exactly one (and it is a node)
+  int lda_pos;                    // body position of the LDA just emitted by ensure_acc, or -1
+  int8_t in_operand[DVM_MAX_NODES];
+  bool stored[DVM_MAX_TENSORS];
   int8_t out_operand[DVM_MAX_TENSORS];
   const float* scalars;
   int n_scalars;
@@ -311,11 +319,11 @@ static inline uint32_t f2u(float f) {
   return u;
 }
 
-static int alloc_treg(Enc& e) {
-  for (int k = 1; k < e.nreg_limit; ++k)
-    if (e.treg_val[k] < 0) {
-      if (k > e.max_treg) e.max_treg = k;
-      return k;
+static int alloc_tmp(Enc& e) {  // a temporary local register (numbered after the input registers)
+  for (int k = 0; k < DVM_MAX_LREGS - e.n_in_regs; ++k)
+    if (e.tmp_val[k] < 0) {
+      if (k + 1 > e.n_tmp_regs) e.n_tmp_regs = k + 1;
+      return e.n_in_regs + k;
     }
   e.fail = true;
   return -1;
@@ -328,20 +336,12 @@ static int alloc_sreg(Enc& e) {
   return -1;
 }
 
-static void cvt_if_needed(Enc& e, int k) {
-  if (e.needs_cvt[k]) {
-    emit(e, DVM_INSN(DVM_OP_CVT, 1, k, DVM_DT_BF16));
-    e.needs_cvt[k] = false;
-  }
-}
-
 static void release(Enc& e, int v) {  // free the registers of a dead value
   if (e.uses[v] > 0) return;
   if (e.cls[v] == CLS_TILE) {
-    if (e.reg_of[v] >= 1) {
-      e.treg_val[e.reg_of[v]] = -1;
-      e.needs_cvt[e.reg_of[v]] = false;
-      e.reg_of[v] = -1;
+    if (e.lreg_of[v] >= e.n_in_regs) {  // input registers stay bound to their input for the whole tile
+      e.tmp_val[e.lreg_of[v] - e.n_in_regs] = -1;
+      e.lreg_of[v] = -1;
     }
   } else if (e.sreg_of[v] >= 0) {
     e.sreg_val[e.sreg_of[v]] = -1;
@@ -349,72 +349,37 @@ static void release(Enc& e, int v) {  // free the registers of a dead value
   }
 }
 
-static void load_input_to(Enc& e, int v, int k) {  // issue the tile load of input value v into Rk
-  int od = e.in_operand[v];
-  emit(e, DVM_INSN(DVM_OP_LDG, 1, k, od));
-  e.needs_cvt[k] = e.opd[od].dtype == DVM_DT_BF16;
-  if (k == 0) {
-    e.acc = (int16_t)v;
-  } else {
-    e.reg_of[v] = (int8_t)k;
-    e.treg_val[k] = (int16_t)v;
-  }
-}
-
 static void spill_acc_if_live(Enc& e) {
   int a = e.acc;
-  if (a >= 0 && e.uses[a] > 0 && e.reg_of[a] < 0) {
-    int k = alloc_treg(e);
+  if (a >= 0 && e.uses[a] > 0 && e.lreg_of[a] < 0) {
+    int k = alloc_tmp(e);
     if (k < 0) return;
-    cvt_if_needed(e, 0);
-    emit(e, DVM_INSN(DVM_OP_MOV, 1, k, 0));
-    e.reg_of[a] = (int8_t)k;
-    e.treg_val[k] = (int16_t)a;
+    emit(e, DVM_INSN(DVM_OP_STA, 1, k, 0));
+    e.lreg_of[a] = (int8_t)k;
+    e.ldt_of[a] = DVM_DT_F32;
+    e.tmp_val[k - e.n_in_regs] = (int16_t)a;
   }
 }
 
 static void ensure_acc(Enc& e, int v) {
-  if (e.acc == v) {
-    cvt_if_needed(e, 0);
-    return;
-  }
+  if (e.acc == v) return;
   spill_acc_if_live(e);
   if (e.fail) return;
-  if (e.reg_of[v] >= 1) {
-    cvt_if_needed(e, e.reg_of[v]);
-    emit(e, DVM_INSN(DVM_OP_MOV, 1, 0, e.reg_of[v]));
+  if (e.lreg_of[v] >= 0) {
+    e.lda_pos = e.n_body;
+    emit(e, DVM_INSN(DVM_OP_LDA, 1, e.lreg_of[v], e.ldt_of[v]));
     e.acc = (int16_t)v;
-  } else if (e.p->nodes[v].kind == NK_INPUT) {
-    load_input_to(e, v, 0);
-    cvt_if_needed(e, 0);
   } else {
     e.fail = true;  // value was dropped: cannot happen with correct use counts
   }
 }
 
-static int ensure_reg(Enc& e, int v) {  // a tile value as the non-accumulator operand
-  if (e.acc == v && e.reg_of[v] < 0) return 0;
-  if (e.reg_of[v] >= 1) {
-    cvt_if_needed(e, e.reg_of[v]);
-    return e.reg_of[v];
-  }
-  if (e.p->nodes[v].kind == NK_INPUT) {
-    int k = alloc_treg(e);
-    if (k < 0) return -1;
-    load_input_to(e, v, k);
-    cvt_if_needed(e, k);
-    return k;
-  }
-  e.fail = true;
-  return -1;
-}
-
 static int ensure_sreg(Enc& e, int v) {
   if (e.sreg_of[v] >= 0) return e.sreg_of[v];
-  if (e.p->nodes[v].kind == NK_INPUT) {
+  if (e.sslot_of[v] >= 0) {
     int k = alloc_sreg(e);
     if (k < 0) return -1;
-    emit(e, DVM_INSN(DVM_OP_LDS, 1, k, e.in_operand[v]));
+    emit(e, DVM_INSN(DVM_OP_LSS, 1, k, e.sslot_of[v]));
     e.sreg_of[v] = (int8_t)k;
     e.sreg_val[k] = (int16_t)v;
     return k;
@@ -423,7 +388,7 @@ static int ensure_sreg(Enc& e, int v) {
   return -1;
 }
 
-static void store_outputs_of(Enc& e, int v) {  // value v is live in R0 (tile) or a scalar register
+static void store_outputs_of(Enc& e, int v) {  // value v is live in the accumulator (tile) or a scalar register
   for (int o = 0; o < e.p->n_outputs; ++o) {
     if (e.stored[o] || root(e, e.p->outputs[o].value) != v) continue;
     if (e.cls[v] == CLS_TILE) {
@@ -449,19 +414,22 @@ static inline uint8_t reversed(uint8_t a) {
 static const uint8_t kUnMap[12] = {DVM_U_EXP, DVM_U_SQRT, DVM_U_RSQRT, DVM_U_ABS, DVM_U_LOG, DVM_U_ERF,
                                    DVM_U_SIGMOID, DVM_U_NEG, DVM_U_RECIP, DVM_U_FLOOR, DVM_U_ROUND, DVM_U_TANH};
 
-// Generates the code body.  hoist: issue every tile load at the top of the body so that all
-// of a tile's global loads are in flight before the first use.
-static bool gen_body(Enc& e, bool hoist, int nreg_limit) {
+// Generates the load section (every global load of a tile, issued asynchronously into local
+// registers before the tile is computed) and the compute section (accumulator code).
+static bool gen_body(Enc& e) {
   const dvm_program* p = e.p;
-  e.n_body = 0;
+  e.n_body = e.n_loads = 0;
+  e.lda_pos = -1;
   e.fail = false;
   e.acc = -1;
-  e.nreg_limit = nreg_limit;
-  e.max_treg = 0;
-  for (int k = 0; k < DVM_MAX_TREGS; ++k) { e.treg_val[k] = -1; e.needs_cvt[k] = false; }
+  e.n_in_regs = e.n_tmp_regs = e.n_sslots = 0;
+  for (int k = 0; k < DVM_MAX_LREGS; ++k) e.tmp_val[k] = -1;
   for (int k = 0; k < DVM_MAX_SREGS; ++k) e.sreg_val[k] = -1;
   for (int o = 0; o < p->n_outputs; ++o) e.stored[o] = false;
-  for (int i = 0; i < p->n_nodes; ++i) { e.uses[i] = 0; e.reg_of[i] = -1; e.sreg_of[i] = -1; }
+  for (int i = 0; i < p->n_nodes; ++i) {
+    e.uses[i] = 0; e.lreg_of[i] = -1; e.sreg_of[i] = -1; e.sslot_of[i] = -1; e.ldt_of[i] = DVM_DT_F32;
+    e.fused_sq[i] = false;
+  }
   for (int i = 0; i < p->n_nodes; ++i) {
     const Node& n = p->nodes[i];
     if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
@@ -469,52 +437,106 @@ static bool gen_body(Enc& e, bool hoist, int nreg_limit) {
     if (n.kind == NK_BINARY) e.uses[root(e, n.y)]++;
   }
   for (int o = 0; o < p->n_outputs; ++o) e.uses[root(e, p->outputs[o].value)]++;
-
-  if (hoist) {
-    // the first tile-class operation decides which input is loaded straight into R0
-    int first_acc = -1;
-    for (int i = 0; i < p->n_nodes && first_acc < 0; ++i) {
-      const Node& n = p->nodes[i];
-      if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
-      int x = root(e, n.x);
-      int y = n.kind == NK_BINARY ? root(e, n.y) : -1;
-      if (e.cls[x] == CLS_TILE && p->nodes[x].kind == NK_INPUT) first_acc = x;
-      else if (y >= 0 && e.cls[y] == CLS_TILE && p->nodes[y].kind == NK_INPUT) first_acc = y;
-      else if (e.cls[x] == CLS_TILE || (y >= 0 && e.cls[y] == CLS_TILE)) break;
+  // reduce_sum(x * x) with no other consumer of the square becomes one sum-of-squares reduction
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind != NK_REDUCE || n.op != DVM_SUM || e.alias[i] >= 0) continue;
+    const int m = root(e, n.x);
+    const Node& mn = p->nodes[m];
+    if (mn.kind == NK_BINARY && mn.op == DVM_MUL && root(e, mn.x) == root(e, mn.y) && e.uses[m] == 1 &&
+        e.cls[m] == CLS_TILE) {
+      e.fused_sq[m] = true;
+      e.uses[root(e, mn.x)] -= 1;  // the square consumed x twice, the fused reduction consumes it once
+      e.uses[m] = 0;
     }
-    if (first_acc < 0) {
-      for (int o = 0; o < p->n_outputs && first_acc < 0; ++o) {
-        int v = root(e, p->outputs[o].value);
-        if (e.cls[v] == CLS_TILE && p->nodes[v].kind == NK_INPUT) first_acc = v;
-      }
-    }
-    // loads in order of first use
-    bool seen[DVM_MAX_NODES] = {};
-    auto hoist_one = [&](int v) {
-      if (v < 0 || seen[v] || p->nodes[v].kind != NK_INPUT || e.uses[v] == 0) return;
-      seen[v] = true;
-      if (e.cls[v] == CLS_SCAL) { ensure_sreg(e, v); return; }
-      if (v == first_acc) { load_input_to(e, v, 0); return; }
-      int k = alloc_treg(e);
-      if (k >= 0) load_input_to(e, v, k);
-    };
-    hoist_one(first_acc);
-    for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
-      const Node& n = p->nodes[i];
-      if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
-      hoist_one(root(e, n.x));
-      if (n.kind == NK_BINARY) hoist_one(root(e, n.y));
-    }
-    for (int o = 0; o < p->n_outputs && !e.fail; ++o) hoist_one(root(e, p->outputs[o].value));
-    if (e.fail) return false;
   }
 
+  // consumers of every value (for the scalar multiply-add fusion below)
+  for (int i = 0; i < p->n_nodes; ++i) { e.n_cons[i] = 0; e.one_cons[i] = -1; e.fused_sc[i] = false; }
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i]) continue;
+    int x = root(e, n.x);
+    if (n.kind == NK_REDUCE && e.fused_sq[x]) x = root(e, p->nodes[x].x);
+    e.n_cons[x]++; e.one_cons[x] = (int16_t)i;
+    if (n.kind == NK_BINARY) { int y = root(e, n.y); e.n_cons[y]++; e.one_cons[y] = (int16_t)i; }
+  }
+  for (int o = 0; o < p->n_outputs; ++o) { int v = root(e, p->outputs[o].value); e.n_cons[v] += 2; }
+
+  // ---- load section: one instruction per used input ----
+  for (int ii = 0; ii < p->n_inputs; ++ii) {
+    const int v = p->inputs[ii];
+    if (e.uses[v] == 0) continue;
+    const int od = e.in_operand[v];
+    if (e.cls[v] == CLS_TILE) {
+      if (e.n_in_regs >= DVM_MAX_LREGS - 1) return false;
+      const int k = e.n_in_regs++;
+      e.loads[e.n_loads++] = DVM_INSN(DVM_OP_LDG, 1, k, od);
+      e.lreg_of[v] = (int8_t)k;
+      e.ldt_of[v] = (int8_t)e.opd[od].dtype;
+    } else {
+      if (e.n_sslots >= DVM_MAX_SSLOTS) return false;
+      const int k = e.n_sslots++;
+      e.loads[e.n_loads++] = DVM_INSN(DVM_OP_LDS, 1, k, od);
+      e.sslot_of[v] = (int8_t)k;
+    }
+  }
+
+  // ---- compute section ----
   for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
     const Node& n = p->nodes[i];
-    if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
+    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i]) continue;
     int x = root(e, n.x);
     if (e.cls[i] == CLS_SCAL && n.kind != NK_REDUCE) {
       // ---- per-row scalar arithmetic ----
+      if (e.fused_sc[i]) continue;  // folded into the multiply-add instruction of a later node
+      // s * m + a followed by a unary (the rstd of a norm, a mean) is ONE instruction: walk the chain of
+      // single-consumer muls -> adds -> unary nodes that starts here
+      if (n.kind == NK_SCALAR) {
+        auto imm_of = [&](const Node& c) { return c.param >= 0 ? e.scalars[c.param] : c.imm; };
+        int chain[3] = {i, -1, -1};
+        int len = 1, un = 0xff;
+        bool have_add = n.op == DVM_ADDS;
+        float m = have_add ? 1.0f : imm_of(n), a = have_add ? imm_of(n) : 0.0f;
+        int cur = i;
+        while (len < 3) {
+          const int nx = e.n_cons[cur] == 1 ? e.one_cons[cur] : -1;
+          if (nx < 0 || e.cls[nx] != CLS_SCAL || root(e, p->nodes[nx].x) != cur) break;
+          const Node& nn = p->nodes[nx];
+          if (nn.kind == NK_SCALAR && nn.op == DVM_ADDS && !have_add) {
+            a = imm_of(nn);
+            have_add = true;
+            chain[len++] = nx;
+            cur = nx;
+          } else if (nn.kind == NK_UNARY) {
+            un = kUnMap[nn.op];
+            chain[len++] = nx;
+            break;
+          } else {
+            break;
+          }
+        }
+        if (len >= 2) {
+          const int last = chain[len - 1];
+          int sx = ensure_sreg(e, x);
+          if (e.fail) break;
+          e.uses[x]--;
+          release(e, x);
+          int d = alloc_sreg(e);
+          if (d < 0) break;
+          emit(e, DVM_INSN(DVM_OP_SOP, 4, d, DVM_SK_FMAU));
+          emit(e, (uint32_t)un | ((uint32_t)sx << 8));
+          emit(e, f2u(m));
+          emit(e, f2u(a));
+          for (int q = 0; q < len; ++q) e.fused_sc[chain[q]] = true;   // later chain nodes are skipped
+          for (int q = 0; q + 1 < len; ++q) e.uses[chain[q]] = 0;       // intermediates never materialise
+          e.sreg_of[last] = (int8_t)d;
+          e.sreg_val[d] = (int16_t)last;
+          store_outputs_of(e, last);
+          release(e, last);
+          continue;
+        }
+      }
       int sx = ensure_sreg(e, x);
       int sy = -1;
       int y = -1;
@@ -546,16 +568,18 @@ static bool gen_body(Enc& e, bool hoist, int nreg_limit) {
       continue;
     }
     if (n.kind == NK_REDUCE) {
+      const bool sq = e.fused_sq[x];
+      if (sq) x = root(e, p->nodes[x].x);
       ensure_acc(e, x);
       if (e.fail) break;
       e.uses[x]--;
       int d = alloc_sreg(e);
       if (d < 0) break;
-      emit(e, DVM_INSN(DVM_OP_RED + (n.op == DVM_SUM ? DVM_R_SUM : n.op == DVM_RMAX ? DVM_R_MAX : DVM_R_MIN),
+      emit(e, DVM_INSN(DVM_OP_RED + (sq ? DVM_R_SUMSQ : n.op == DVM_SUM ? DVM_R_SUM : n.op == DVM_RMAX ? DVM_R_MAX : DVM_R_MIN),
                        1, d, 0));
       e.sreg_of[i] = (int8_t)d;
       e.sreg_val[d] = (int16_t)i;
-      if (e.uses[x] == 0) { release(e, x); }
+      release(e, x);
       store_outputs_of(e, i);
       release(e, i);
       continue;
@@ -567,20 +591,36 @@ static bool gen_body(Enc& e, bool hoist, int nreg_limit) {
       int a = x, b = y;  // a: accumulator operand, b: the other
       bool swap = false;
       if (e.cls[x] == CLS_SCAL) swap = true;                                   // scalar (op) tile
-      else if (e.cls[y] == CLS_TILE && e.acc == y && e.acc != x) swap = true;   // right operand already in R0
+      else if (e.cls[y] == CLS_TILE && e.acc == y && e.acc != x) swap = true;   // right operand already in the accumulator
       if (swap) { a = y; b = x; ar = reversed(ar); }
       ensure_acc(e, a);
       if (e.fail) break;
       int bk = -1;
-      if (e.cls[b] == CLS_TILE) bk = (b == a) ? 0 : ensure_reg(e, b);
-      else bk = ensure_sreg(e, b);
+      if (e.cls[b] == CLS_TILE) {
+        if (b == a) bk = 0xff;
+        else if (e.lreg_of[b] >= 0) bk = e.lreg_of[b];
+        else e.fail = true;
+      } else {
+        bk = ensure_sreg(e, b);
+      }
       if (e.fail || bk < 0) { e.fail = true; break; }
       e.uses[a]--;
       e.uses[b]--;
       spill_acc_if_live(e);
       if (e.fail) break;
-      if (e.cls[b] == CLS_TILE) emit(e, DVM_INSN(DVM_OP_BIN + ar * 8 + bk, 1, 0, 0));
-      else emit(e, DVM_INSN(DVM_OP_BINS + ar, 1, bk, 0));
+      if (e.cls[b] == CLS_TILE) {
+        if (b != a && e.lda_pos == e.n_body - 1) {
+          // the accumulator was loaded just for this operation: one fused instruction ACC = L[x] op L[y]
+          const uint32_t lda = e.body[e.lda_pos];
+          e.body[e.lda_pos] = DVM_INSN(DVM_OP_LD2 + ar, 1, DVM_INSN_A(lda),
+                                       (uint32_t)bk | (DVM_INSN_B(lda) << 6) | ((uint32_t)e.ldt_of[b] << 7));
+          e.lda_pos = -1;
+        } else {
+          emit(e, DVM_INSN(DVM_OP_BIN + ar, 1, bk, b == a ? DVM_DT_F32 : e.ldt_of[b]));
+        }
+      } else {
+        emit(e, DVM_INSN(DVM_OP_BINS + ar, 1, bk, 0));
+      }
       e.acc = (int16_t)i;
       release(e, a);
       if (b != a) release(e, b);
@@ -782,103 +822,197 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   }
   if (primary >= 0) e.opd[primary].primary = true;
 
-  // ---- 5. shape tiling: threads per row G, column tile, tile count (cost model of Sec. 4.2) ----
-  const int V = DVM_VM_V, T = DVM_VM_THREADS;
-  const int64_t N = dvm_get_num_cores();
-  const int64_t beta = 4;  // per-tile decode overhead in element units (the paper's "+2")
-  int log2G = 8;
-  int64_t Ctile = C, CB = 1, rowsR = R, lastRowCols = C;
-  uint32_t flags = 0;
-  int64_t n_tiles = 0;
-  if (flat) {
-    int64_t total = empty ? 0 : C;  // everything merged into one dim
-    int64_t best_cost = -1, best_chunk = (int64_t)T * W;
-    for (int k = 1; k <= V / W; ++k) {
-      int64_t chunk = (int64_t)T * W * k;
-      int64_t cost = cdiv(cdiv(total, chunk), N) * (W * k + beta);
-      if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_chunk = chunk; }
+  // ---- 5. code: load section + compute section (independent of the tile geometry) ----
+  if (!gen_body(e)) return DVM_ERR_UNSUPPORTED;  // more live tile values than local registers
+  const int nreg = e.n_in_regs + e.n_tmp_regs;
+  int in_dtype[DVM_MAX_LREGS], in_opd[DVM_MAX_LREGS];
+  for (int k = 0; k < e.n_in_regs; ++k) {
+    in_dtype[k] = DVM_DT_F32;
+    in_opd[k] = 0;
+    for (int q = 0; q < e.n_loads; ++q)
+      if (DVM_INSN_OP(e.loads[q]) == DVM_OP_LDG && (int)DVM_INSN_A(e.loads[q]) == k) {
+        in_opd[k] = (int)DVM_INSN_B(e.loads[q]);
+        in_dtype[k] = e.opd[in_opd[k]].dtype;
+      }
+  }
+  int out_es = 2;
+  for (int o = 0; o < p->n_outputs; ++o)
+    if (p->outputs[o].dtype == DVM_F32 && e.cls[root(e, p->outputs[o].value)] == CLS_TILE) out_es = 4;
+
+  // ---- 6. shape tiling (Sec. 4.2): elements per thread V, threads per row G, column tile, tile count.
+  // Candidates are compared with the paper's cost  ceil(#tiles / N) * (tile + overhead)  in per-thread
+  // element units; N is the number of CTAs resident at once, which the local-memory need decides.
+  const int T = DVM_VM_THREADS;
+  const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
+  struct Geo {
+    int V, log2G, W, units, staging_unit[2], scalar_unit;
+    int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
+    uint32_t flags, inv_mask;
+    uint32_t lreg_table[DVM_MAX_LREGS];
+  } best;
+  best.cost = -1;
+  const int W0 = W;
+  // local registers that no instruction touches after the first tile store: the store's staging line may
+  // reuse one of them
+  uint32_t dead_at_store = 0;
+  {
+    int first_stg = -1;
+    uint32_t used_after = 0;
+    for (int pc = 0; pc < e.n_body; pc += (int)DVM_INSN_LEN(e.body[pc])) {
+      const uint32_t w0 = e.body[pc], op = DVM_INSN_OP(w0), ra = DVM_INSN_A(w0), rb = DVM_INSN_B(w0);
+      if (op == DVM_OP_STG && first_stg < 0) first_stg = pc;
+      if (first_stg < 0) continue;
+      if (op == DVM_OP_LDA || op == DVM_OP_STA) used_after |= 1u << ra;
+      else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) { if (ra != DVM_REG_ACC) used_after |= 1u << ra; }
+      else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) used_after |= (1u << ra) | (1u << (rb & 0x3f));
     }
-    Ctile = best_chunk;
-    rowsR = cdiv(total, Ctile);
-    lastRowCols = rowsR > 0 ? total - (rowsR - 1) * Ctile : Ctile;
+    if (first_stg >= 0) dead_at_store = ~used_after & ((1u << nreg) - 1);
+  }
+  for (int vi = 0; vi < 2; ++vi) {
+    Geo g;
+    g.V = vi == 0 ? 32 : 16;
+    if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
+    int ctas_guess = 2;
+    bool ok = false;
+    for (int attempt = 0; attempt < 3 && !ok; ++attempt) {
+      const int64_t N = (int64_t)dvm_get_num_cores() * ctas_guess / 3;  // the core count is quoted at 3 CTAs per SM
+      g.cost = -1;
+      g.W = W0;
+      if (flat) {
+        int64_t total = empty ? 0 : C;  // everything merged into one dim
+        int64_t best_chunk = (int64_t)T * W0;
+        for (int k = 1; k <= g.V / W0; ++k) {
+          int64_t chunk = (int64_t)T * W0 * k;
+          int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
+          if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
+        }
+        g.Ctile = best_chunk;
+        g.rowsR = cdiv(total, g.Ctile);
+        g.lastRowCols = g.rowsR > 0 ? total - (g.rowsR - 1) * g.Ctile : g.Ctile;
+        g.CB = 1;
+        g.log2G = 8;
+        g.n_tiles = g.rowsR;
+        g.flags = DVM_F_FLAT | DVM_F_ALIGNED;
+      } else {
+        // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
+        bool aligned = primary >= 0;
+        if (primary >= 0)
+          for (int q = 0; q < 3; ++q)
+            if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
+        for (int pass = 0; pass < 2 && g.cost < 0; ++pass) {
+          const int w = pass == 0 ? W0 : 1;  // second pass: element-wise mapping, which needs no padding
+          const bool al = pass == 0 ? aligned : true;
+          const int64_t pad = al ? 0 : w - 1;
+          for (int lg = 0; lg <= 8; ++lg) {
+            int64_t G = 1 << lg, cap = G * g.V;
+            int64_t ct;
+            if (has_reduce) {
+              if (cap < C + pad) continue;
+              ct = C;
+            } else {
+              ct = ((cap - pad) / w) * w;
+              if (ct <= 0) continue;
+              if (ct > C) ct = C;
+            }
+            int64_t cb = cdiv(C, ct);
+            int64_t tiles = cdiv(R, T / G) * cb;
+            int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
+            int64_t cost = cdiv(tiles, N) * (u + beta);
+            if (g.cost < 0 || cost < g.cost) {
+              g.cost = cost; g.log2G = lg; g.Ctile = ct; g.CB = cb; g.n_tiles = tiles; g.W = w;
+              g.flags = al ? DVM_F_ALIGNED : 0;
+            }
+          }
+        }
+        if (g.cost < 0) break;  // a reduced row does not fit V elements per thread
+        if (outer[1] > 1 || outer[2] > 1) g.flags |= DVM_F_OUTER_DIMS;
+        g.rowsR = R;
+        g.lastRowCols = C;
+        if (empty) g.n_tiles = 0;
+      }
+      // local-memory layout in 8 KB units (32 bytes per thread): input registers twice (double buffering;
+      // a row-vector input of an aligned program is the same for every tile of a thread: once),
+      // temporaries, the staging line of the scalar store path, per-row scalar slots
+      g.inv_mask = 0;
+      int in_units = 0, inv_units = 0, off[DVM_MAX_LREGS], usz[DVM_MAX_LREGS];
+      for (int k = 0; k < e.n_in_regs; ++k) {
+        usz[k] = g.V * (in_dtype[k] == DVM_DT_BF16 ? 2 : 4) / 32;
+        const Operand& od = e.opd[in_opd[k]];
+        const bool inv = !flat && (g.flags & DVM_F_ALIGNED) && g.W > 1 && g.CB == 1 && od.ostride[0] == 0 &&
+                         od.ostride[1] == 0 && od.ostride[2] == 0;
+        if (inv) g.inv_mask |= 1u << k;
+        else { off[k] = in_units; in_units += usz[k]; }
+      }
+      for (int k = 0; k < e.n_in_regs; ++k)
+        if ((g.inv_mask >> k) & 1) { off[k] = 2 * in_units + inv_units; inv_units += usz[k]; }
+      for (int k = 0; k < e.n_in_regs; ++k)
+        g.lreg_table[k] = ((g.inv_mask >> k) & 1) ? ((uint32_t)off[k] | ((uint32_t)off[k] << 16))
+                                                   : ((uint32_t)off[k] | ((uint32_t)(off[k] + in_units) << 16));
+      g.units = 2 * in_units + inv_units;
+      for (int k = e.n_in_regs; k < nreg; ++k) {
+        usz[k] = g.V * 4 / 32;
+        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)g.units << 16);
+        g.units += usz[k];
+      }
+      const int need = g.V * out_es / 32;
+      int alias = -1;
+      for (int k = 0; k < nreg && alias < 0; ++k)
+        if (((dead_at_store >> k) & 1) && !((g.inv_mask >> k) & 1) && usz[k] >= need) alias = k;
+      if (alias >= 0) {
+        g.staging_unit[0] = (int)(g.lreg_table[alias] & 0xffff);
+        g.staging_unit[1] = (int)(g.lreg_table[alias] >> 16);
+      } else {
+        g.staging_unit[0] = g.staging_unit[1] = g.units;
+        g.units += need;
+      }
+      g.scalar_unit = g.units;
+      if (e.n_sslots > 0) g.units += 2;
+      if (g.units > DVM_MAX_LOCAL_UNITS) break;
+      int ctas = 233472 / (g.units * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
+      if (ctas > 2) ctas = 2;  // the interpreter is compiled for two resident CTAs per SM
+      if (ctas < 1) break;
+      if (ctas == ctas_guess) ok = true;
+      else ctas_guess = ctas;
+    }
+    if (!ok) continue;
+    if (best.cost < 0 || g.cost < best.cost) best = g;
+  }
+  if (best.cost < 0) return DVM_ERR_UNSUPPORTED;  // row longer than the register budget, or too much local memory
+  const int log2G = best.log2G;
+  W = best.W;
+  const int64_t Ctile = best.Ctile, CB = best.CB, rowsR = best.rowsR, lastRowCols = best.lastRowCols, n_tiles = best.n_tiles;
+  const uint32_t flags = best.flags;
+  const int units = best.units, scalar_unit = best.scalar_unit;
+  const uint32_t* lreg_table = best.lreg_table;
+  if (flat) {
     C = Ctile;
-    CB = 1;
-    log2G = 8;
-    n_tiles = rowsR;
-    flags |= DVM_F_FLAT | DVM_F_ALIGNED;
     for (int o = 0; o < e.n_opd; ++o) {
       e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile : 0;
       e.opd[o].ostride[1] = e.opd[o].ostride[2] = 0;
     }
     outer[0] = rowsR; outer[1] = outer[2] = 1;
-  } else {
-    // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
-    bool aligned = primary >= 0;
-    if (primary >= 0)
-      for (int g = 0; g < 3; ++g)
-        if (outer[g] > 1 && (e.opd[primary].ostride[g] % W) != 0) aligned = false;
-    int64_t best_cost = -1;
-    int bestW = W;
-    for (int pass = 0; pass < 2 && best_cost < 0; ++pass) {
-      const int w = pass == 0 ? W : 1;  // second pass: element-wise mapping, which needs no padding
-      const bool al = pass == 0 ? aligned : true;
-      const int64_t pad = al ? 0 : w - 1;
-      for (int lg = 0; lg <= 8; ++lg) {
-        int64_t G = 1 << lg, cap = G * V;
-        int64_t ct;
-        if (has_reduce) {
-          if (cap < C + pad) continue;
-          ct = C;
-        } else {
-          ct = ((cap - pad) / w) * w;
-          if (ct <= 0) continue;
-          if (ct > C) ct = C;
-        }
-        int64_t cb = cdiv(C, ct);
-        int64_t tiles = cdiv(R, T / G) * cb;
-        int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
-        int64_t cost = cdiv(tiles, N) * (u + beta);
-        if (best_cost < 0 || cost < best_cost) {
-          best_cost = cost; log2G = lg; Ctile = ct; CB = cb; n_tiles = tiles; bestW = w;
-          flags = al ? DVM_F_ALIGNED : 0;
-        }
-      }
-    }
-    if (best_cost < 0) return DVM_ERR_UNSUPPORTED;  // a reduced row does not fit the register budget
-    W = bestW;
-    if (outer[1] > 1 || outer[2] > 1) flags |= DVM_F_OUTER_DIMS;
-    lastRowCols = C;
-    if (empty) n_tiles = 0;
   }
-  if (n_tiles > 0xffffffffll) return DVM_ERR_TOO_LARGE;
-
-  // ---- 6. code body ----
-  int nreg = 4;
-  bool ok = gen_body(e, true, 4);
-  if (!ok) ok = gen_body(e, false, 4);
-  if (!ok) { nreg = 8; ok = gen_body(e, true, 8); }
-  if (!ok) ok = gen_body(e, false, 8);
-  if (!ok) return DVM_ERR_UNSUPPORTED;  // more live tile values than tile registers
-  if (e.max_treg >= 4) nreg = 8;
+  if (n_tiles > 0xffffffffll || rowsR > 0xffffffffll) return DVM_ERR_TOO_LARGE;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
-  size_t words = DVM_HDR_WORDS + 2 * (size_t)n_tensors + (size_t)DVM_OPD_WORDS * e.n_opd + e.n_body;
+  const int code_words = e.n_loads + e.n_body;
+  size_t words = DVM_HDR_WORDS + 2 * (size_t)n_tensors + (size_t)DVM_OPD_WORDS * e.n_opd + nreg + code_words;
   *code_size = words * 4;
   if (!code || code_capacity < words * 4) return DVM_ERR_BUFFER_TOO_SMALL;
   uint32_t* w = (uint32_t*)code;
   memset(w, 0, words * 4);
   w[DVM_H_MAGIC] = DVM_MAGIC;
   w[DVM_H_KERNEL_TYPE] = DVM_KERNEL_VEC;
-  w[DVM_H_CODE_WORDS] = (uint32_t)e.n_body;
+  w[DVM_H_CODE_WORDS] = (uint32_t)code_words;
   w[DVM_H_N_TILES] = (uint32_t)n_tiles;
   w[DVM_H_TOTAL_WORDS] = (uint32_t)words;
   w[DVM_H_COUNTS] = (uint32_t)n_tensors | ((uint32_t)n_in << 8) | ((uint32_t)e.n_opd << 16) |
                     ((uint32_t)p->n_outputs << 24);
   w[DVM_H_GEOM] = (uint32_t)log2G | ((uint32_t)W << 8) | ((uint32_t)nreg << 16) | (flags << 24);
   w[DVM_H_COLS] = (uint32_t)C;
-  w[DVM_H_ROWS_LO] = (uint32_t)(flat ? rowsR : R);
-  w[DVM_H_ROWS_HI] = (uint32_t)((uint64_t)(flat ? rowsR : R) >> 32);
+  w[DVM_H_ROWS_LO] = (uint32_t)rowsR;
+  w[DVM_H_ROWS_HI] = (uint32_t)((uint64_t)rowsR >> 32);
   w[DVM_H_COL_BLOCKS] = (uint32_t)CB;
   w[DVM_H_COL_TILE] = (uint32_t)Ctile;
   w[DVM_H_OUTER0] = (uint32_t)outer[0];
@@ -886,6 +1020,10 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   w[DVM_H_OUTER2] = (uint32_t)outer[2];
   w[DVM_H_LAST_ROW_COLS] = (uint32_t)lastRowCols;
   w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
+  w[DVM_H_LOCAL] = (uint32_t)e.n_in_regs | ((uint32_t)e.n_tmp_regs << 8) | ((uint32_t)e.n_sslots << 16) | ((uint32_t)best.V << 24);
+  w[DVM_H_LOAD_WORDS] = (uint32_t)e.n_loads;
+  w[DVM_H_LOCAL2] = (uint32_t)best.staging_unit[0] | ((uint32_t)scalar_unit << 8) | ((uint32_t)units << 16) |
+                    ((uint32_t)best.staging_unit[1] << 24);
   uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
   for (int o = 0; o < e.n_opd; ++o) {
     const Operand& od = e.opd[o];
@@ -897,7 +1035,12 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
       d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
     }
   }
-  memcpy(ot + e.n_opd * DVM_OPD_WORDS, e.body, (size_t)e.n_body * 4);
+  uint32_t* lt = ot + e.n_opd * DVM_OPD_WORDS;
+  memcpy(lt, lreg_table, (size_t)nreg * 4);
+  for (int q = 0; q < e.n_loads; ++q)
+    if (DVM_INSN_OP(e.loads[q]) == DVM_OP_LDG && ((best.inv_mask >> DVM_INSN_A(e.loads[q])) & 1)) e.loads[q] |= 0x80u << 16;
+  memcpy(lt + nreg, e.loads, (size_t)e.n_loads * 4);
+  memcpy(lt + nreg + e.n_loads, e.body, (size_t)e.n_body * 4);
   if (C > 0xffffffffll || outer[0] > 0xffffffffll || outer[1] > 0xffffffffll || outer[2] > 0xffffffffll)
     return DVM_ERR_TOO_LARGE;
   return DVM_OK;
@@ -907,11 +1050,11 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
 // Verification and the readable dump
 // ---------------------------------------------------------------------------
 static int insn_expected_len(uint32_t op, uint32_t w0) {
-  if (op == DVM_OP_NOP || op == DVM_OP_LDG || op == DVM_OP_CVT || op == DVM_OP_STG || op == DVM_OP_LDS ||
-      op == DVM_OP_STS || op == DVM_OP_MOV || op == DVM_OP_BCS)
-    return 1;
+  if (op <= DVM_OP_BCS) return 1;
+  if (op == DVM_OP_SOP) return DVM_INSN_B(w0) == DVM_SK_BINI ? 3 : (DVM_INSN_B(w0) == DVM_SK_FMAU ? 4 : 2);
+  if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) return 2;
-  if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8 * DVM_A_NBIN) return 1;
+  if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) return 1;
   if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) return 1;
@@ -934,18 +1077,35 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
            n_out = counts >> 24;
   if (n_tensors > DVM_MAX_TENSORS || n_opd > DVM_MAX_OPERANDS || n_in + n_out != n_tensors) return DVM_ERR_BAD_CODE;
   uint32_t body = w[DVM_H_CODE_WORDS];
-  if ((uint64_t)DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd + body != w[DVM_H_TOTAL_WORDS])
+  const uint32_t n_lregs = (w[DVM_H_GEOM] >> 16) & 0xff;
+  if ((uint64_t)DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd + n_lregs + body != w[DVM_H_TOTAL_WORDS])
     return DVM_ERR_BAD_CODE;
   uint32_t geom = w[DVM_H_GEOM];
   uint32_t lg = geom & 0xff, W = (geom >> 8) & 0xff, nreg = (geom >> 16) & 0xff;
-  if (lg > 8 || !(W == 1 || W == 4 || W == 8) || !(nreg == 4 || nreg == 8)) return DVM_ERR_BAD_CODE;
+  const uint32_t local = w[DVM_H_LOCAL];
+  const uint32_t n_inr = local & 0xff, n_tmpr = (local >> 8) & 0xff, n_ss = (local >> 16) & 0xff, Vv = local >> 24;
+  if (Vv != 16 && Vv != 32) return DVM_ERR_BAD_CODE;
+  const uint32_t u_bf16 = Vv * 2 / 32, u_f32 = Vv * 4 / 32;  // local-memory units of one tile register
+  if (lg > 8 || !(W == 1 || W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
+  const uint32_t local2 = w[DVM_H_LOCAL2];
+  const uint32_t units = (local2 >> 16) & 0xff, scalar_unit = (local2 >> 8) & 0xff;
+  const uint32_t staging_unit = (local2 & 0xff) > (local2 >> 24) ? (local2 & 0xff) : (local2 >> 24);  // the larger offset bounds both
+  if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || units > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
+  if (staging_unit + u_bf16 > units || (n_ss && scalar_unit + 2 > units)) return DVM_ERR_BAD_CODE;
+  const uint32_t* lt = w + DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd;
+  // a local register access of `need` units (bf16: 1, fp32: 2) must stay inside the CTA's local memory
+  auto lreg_ok = [&](uint32_t k, uint32_t need) {
+    return k < nreg && (lt[k] & 0xffff) + need <= units && (lt[k] >> 16) + need <= units;
+  };
+  const uint32_t load_words = w[DVM_H_LOAD_WORDS];
+  if (load_words > body) return DVM_ERR_BAD_CODE;
   uint64_t G = 1ull << lg;
   uint64_t ctile = w[DVM_H_COL_TILE], cb = w[DVM_H_COL_BLOCKS], C = w[DVM_H_COLS];
   uint64_t R = (uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32);
   uint32_t flags = geom >> 24;
   uint64_t pad = (flags & DVM_F_ALIGNED) ? 0 : W - 1;
   if (w[DVM_H_N_TILES] > 0) {
-    if (ctile == 0 || cb == 0 || ctile + pad > G * DVM_VM_V) return DVM_ERR_BAD_CODE;
+    if (ctile == 0 || cb == 0 || ctile + pad > G * Vv) return DVM_ERR_BAD_CODE;
     if (cb * ctile < C || (cb - 1) * ctile >= C) return DVM_ERR_BAD_CODE;
     uint64_t rpt = DVM_VM_THREADS / G;
     if ((uint64_t)w[DVM_H_N_TILES] != ((R + rpt - 1) / rpt) * cb) return DVM_ERR_BAD_CODE;
@@ -967,33 +1127,39 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   } else if (n_primary != 0) {
     return DVM_ERR_BAD_CODE;
   }
-  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS;
+  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS + n_lregs;
   uint32_t pc = 0;
   while (pc < body) {
     uint32_t w0 = b[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), bb = DVM_INSN_B(w0);
     int el = insn_expected_len(op, w0);
     if (el < 0 || (uint32_t)el != len || pc + len > body) return DVM_ERR_BAD_CODE;
+    const bool in_load = pc < load_words;
+    if ((op == DVM_OP_LDG || op == DVM_OP_LDS) != in_load) return DVM_ERR_BAD_CODE;  // loads live in the load section only
     if (op == DVM_OP_LDG || op == DVM_OP_STG) {
-      if (a >= nreg || bb >= n_opd) return DVM_ERR_BAD_CODE;
-      if (op == DVM_OP_STG && a != 0) return DVM_ERR_BAD_CODE;
+      if (bb >= n_opd) return DVM_ERR_BAD_CODE;
       uint32_t info = ot[bb * DVM_OPD_WORDS];
+      if (op == DVM_OP_LDG && ((a & 0x7f) >= n_inr || !lreg_ok(a & 0x7f, ((info >> 8) & 0xff) == DVM_DT_BF16 ? u_bf16 : u_f32))) return DVM_ERR_BAD_CODE;
       bool is_out = (info & 0xff) >= n_in;
       if ((op == DVM_OP_STG) != is_out) return DVM_ERR_BAD_CODE;  // never store to an input, never load an output
+      if (op == DVM_OP_STG && staging_unit + (((info >> 8) & 0xff) == DVM_DT_BF16 ? u_bf16 : u_f32) > units) return DVM_ERR_BAD_CODE;
       if (((info >> 16) & 0xff) != 1) return DVM_ERR_BAD_CODE;
     } else if (op == DVM_OP_LDS || op == DVM_OP_STS) {
-      if (a >= DVM_MAX_SREGS || bb >= n_opd) return DVM_ERR_BAD_CODE;
+      if (bb >= n_opd) return DVM_ERR_BAD_CODE;
+      if (op == DVM_OP_LDS ? a >= n_ss : a >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
       uint32_t info = ot[bb * DVM_OPD_WORDS];
       bool is_out = (info & 0xff) >= n_in;
       if ((op == DVM_OP_STS) != is_out) return DVM_ERR_BAD_CODE;
       if (((info >> 16) & 0xff) != 0) return DVM_ERR_BAD_CODE;
-    } else if (op == DVM_OP_CVT) {
-      if (a >= nreg || bb > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
-    } else if (op == DVM_OP_MOV) {
-      if (a >= nreg || bb >= nreg || ((a == 0) == (bb == 0))) return DVM_ERR_BAD_CODE;  // to or from R0 only
+    } else if (op == DVM_OP_LDA) {
+      if (bb > DVM_DT_BF16 || !lreg_ok(a, bb == DVM_DT_BF16 ? u_bf16 : u_f32)) return DVM_ERR_BAD_CODE;
+    } else if (op == DVM_OP_STA) {
+      if (a < n_inr || !lreg_ok(a, u_f32)) return DVM_ERR_BAD_CODE;  // input registers are read-only
+    } else if (op == DVM_OP_LSS) {
+      if (a >= DVM_MAX_SREGS || bb >= n_ss) return DVM_ERR_BAD_CODE;
     } else if (op == DVM_OP_BCS) {
       if (a >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
-    } else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8 * DVM_A_NBIN) {
-      if (((op - DVM_OP_BIN) & 7) >= nreg) return DVM_ERR_BAD_CODE;
+    } else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) {
+      if (bb > DVM_DT_BF16 || (a != DVM_REG_ACC && !lreg_ok(a, bb == DVM_DT_BF16 ? u_bf16 : u_f32))) return DVM_ERR_BAD_CODE;
     } else if ((op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) ||
                (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED)) {
       if (a >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE;
@@ -1003,7 +1169,10 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       if (bb == DVM_SK_BIN) { if (sub >= DVM_A_NBIN || s2 >= DVM_MAX_SREGS) return DVM_ERR_BAD_CODE; }
       else if (bb == DVM_SK_BINI) { if (sub >= DVM_A_NBIN) return DVM_ERR_BAD_CODE; }
       else if (bb == DVM_SK_UN) { if (sub >= DVM_U_NUN) return DVM_ERR_BAD_CODE; }
+      else if (bb == DVM_SK_FMAU) { if (sub >= DVM_U_NUN && sub != 0xff) return DVM_ERR_BAD_CODE; }
       else return DVM_ERR_BAD_CODE;
+    } else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) {
+      if (!lreg_ok(a, ((bb >> 6) & 1) ? u_bf16 : u_f32) || !lreg_ok(bb & 0x3f, (bb >> 7) ? u_bf16 : u_f32)) return DVM_ERR_BAD_CODE;
     }
     pc += len;
   }
@@ -1032,7 +1201,7 @@ static void outf(Out& o, const char* fmt, ...) {
 static const char* kArith[8] = {"add", "sub", "rsub", "mul", "div", "rdiv", "min", "max"};
 static const char* kUn[DVM_U_NUN] = {"exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
                                      "recip", "floor", "round", "tanh", "rnd_bf16"};
-static const char* kRed[3] = {"sum", "max", "min"};
+static const char* kRed[DVM_R_NRED] = {"sum", "max", "min", "sumsq"};
 }  // namespace
 
 int dvm_disassemble_matmul(const uint32_t* w, size_t n_words, char* buf, size_t cap);
@@ -1052,7 +1221,8 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
   int cores = dvm_get_num_cores();
   outf(o, "kernel vmain.vec  block_dim=%lld  body_tile=%lld  code_size=%u\n", (long long)n_tiles,
        (long long)((n_tiles + cores - 1) / cores), w[DVM_H_CODE_WORDS] * 4);
-  outf(o, "  rows=%llu cols=%u col_tile=%u col_blocks=%u threads_per_row=%u vec=%u tile_regs=%u flags=%s%s%s\n",
+  outf(o, "  elems_per_thread=%u local_units=%u\n", w[DVM_H_LOCAL] >> 24, (w[DVM_H_LOCAL2] >> 16) & 0xff);
+  outf(o, "  rows=%llu cols=%u col_tile=%u col_blocks=%u threads_per_row=%u vec=%u local_regs=%u flags=%s%s%s\n",
        (unsigned long long)((uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32)), w[DVM_H_COLS],
        w[DVM_H_COL_TILE], w[DVM_H_COL_BLOCKS], 1u << (geom & 0xff), (geom >> 8) & 0xff, (geom >> 16) & 0xff,
        ((geom >> 24) & DVM_F_ALIGNED) ? "A" : "-", ((geom >> 24) & DVM_F_OUTER_DIMS) ? "O" : "-",
@@ -1067,30 +1237,42 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
          (long long)((uint64_t)d[2] | ((uint64_t)d[3] << 32)), (long long)((uint64_t)d[4] | ((uint64_t)d[5] << 32)),
          (long long)((uint64_t)d[6] | ((uint64_t)d[7] << 32)), (info >> 24) & 1 ? " primary" : "");
   }
-  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS;
+  const uint32_t* b = ot + n_opd * DVM_OPD_WORDS + ((geom >> 16) & 0xff);
   uint32_t body = w[DVM_H_CODE_WORDS], pc = 0;
   while (pc < body) {
     uint32_t w0 = b[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), bb = DVM_INSN_B(w0);
+    if (pc == w[DVM_H_LOAD_WORDS]) outf(o, "  ---- compute ----\n");
     outf(o, "  %04x: ", pc * 4);
     float imm = 0.f;
     if (len >= 2) memcpy(&imm, &b[pc + len - 1], 4);
+    const char* dts = bb == DVM_DT_BF16 ? ".bf16" : "";
     if (op == DVM_OP_NOP) outf(o, "nop\n");
-    else if (op == DVM_OP_LDG) outf(o, "load      r%u, m%u\n", a, bb);
-    else if (op == DVM_OP_CVT) outf(o, "widen     r%u, %s\n", a, bb == DVM_DT_BF16 ? "bf16" : "f32");
-    else if (op == DVM_OP_STG) outf(o, "store     m%u, r%u\n", bb, a);
-    else if (op == DVM_OP_LDS) outf(o, "load.row  s%u, m%u\n", a, bb);
+    else if (op == DVM_OP_LDG) outf(o, "load%s l%u, m%u\n", (a & 0x80) ? ".once" : "     ", a & 0x7f, bb);
+    else if (op == DVM_OP_LDS) outf(o, "load.row  x%u, m%u\n", a, bb);
+    else if (op == DVM_OP_LDA) outf(o, "copy      acc, l%u%s\n", a, dts);
+    else if (op == DVM_OP_STA) outf(o, "copy      l%u, acc\n", a);
+    else if (op == DVM_OP_LSS) outf(o, "copy      s%u, x%u\n", a, bb);
+    else if (op == DVM_OP_STG) outf(o, "store     m%u, acc\n", bb);
     else if (op == DVM_OP_STS) outf(o, "store.row m%u, s%u\n", bb, a);
-    else if (op == DVM_OP_MOV) outf(o, "copy      r%u, r%u\n", a, bb);
-    else if (op == DVM_OP_BCS) outf(o, "broadcast r0, s%u\n", a);
-    else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + 8) outf(o, "%ss      r0, %.9g\n", kArith[op - DVM_OP_BINI], imm);
-    else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 64)
-      outf(o, "%-9s r0, r0, r%u\n", kArith[(op - DVM_OP_BIN) >> 3], (op - DVM_OP_BIN) & 7);
-    else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + 8) outf(o, "%-9s r0, r0, s%u\n", kArith[op - DVM_OP_BINS], a);
-    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) outf(o, "%-9s r0, r0\n", kUn[op - DVM_OP_UN]);
-    else if (op >= DVM_OP_RED && op < DVM_OP_RED + 3) outf(o, "row%-6s s%u, r0\n", kRed[op - DVM_OP_RED], a);
+    else if (op == DVM_OP_BCS) outf(o, "broadcast acc, s%u\n", a);
+    else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + 8) outf(o, "%ss      acc, %.9g\n", kArith[op - DVM_OP_BINI], imm);
+    else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8) {
+      if (a == DVM_REG_ACC) outf(o, "%-9s acc, acc, acc\n", kArith[op - DVM_OP_BIN]);
+      else outf(o, "%-9s acc, acc, l%u%s\n", kArith[op - DVM_OP_BIN], a, dts);
+    }
+    else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + 8) outf(o, "%-9s acc, acc, s%u\n", kArith[op - DVM_OP_BINS], a);
+    else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + 8)
+      outf(o, "%-9s acc, l%u%s, l%u%s\n", kArith[op - DVM_OP_LD2], a, ((bb >> 6) & 1) ? ".bf16" : "", bb & 0x3f, (bb >> 7) ? ".bf16" : "");
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) outf(o, "%-9s acc, acc\n", kUn[op - DVM_OP_UN]);
+    else if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) outf(o, "row%-6s s%u, acc\n", kRed[op - DVM_OP_RED], a);
     else if (op == DVM_OP_SOP) {
       uint32_t w1 = b[pc + 1], sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
-      if (bb == DVM_SK_BIN) outf(o, "s.%-7s s%u, s%u, s%u\n", kArith[sub], a, s1, s2);
+      if (bb == DVM_SK_FMAU) {
+        float m2, a2;
+        memcpy(&m2, &b[pc + 2], 4); memcpy(&a2, &b[pc + 3], 4);
+        outf(o, "s.fma%-5s s%u, s%u * %.9g + %.9g\n", sub == 0xff ? "" : kUn[sub], a, s1, m2, a2);
+      }
+      else if (bb == DVM_SK_BIN) outf(o, "s.%-7s s%u, s%u, s%u\n", kArith[sub], a, s1, s2);
       else if (bb == DVM_SK_BINI) outf(o, "s.%ss    s%u, s%u, %.9g\n", kArith[sub], a, s1, imm);
       else outf(o, "s.%-7s s%u, s%u\n", kUn[sub], a, s1);
     }

@@ -18,12 +18,13 @@ constexpr int PW_SMALL = 496;    // words of code in a 2 KB parameter block
 constexpr int PW_LARGE = 8000;   // ... in a 32 KB parameter block (the sm_70+ limit is 32764 bytes)
 constexpr int QUEUE_SLOTS = 504;
 constexpr int MAX_DEVICES = 64;
+constexpr size_t kMaxDynSmem = 227 * 1024 - 256;  // dynamic shared memory a CTA may ask for (static part excluded)
 
 struct DeviceState {
   bool ready = false;
   unsigned int* scratch = nullptr;  // [0] status word, [8 + 2*slot] work-queue counter pairs
   int sm_count = 0;
-  int occ[2][2] = {{0, 0}, {0, 0}};  // resident CTAs per SM for [nreg8][large]
+  int occ[2][2][DVM_MAX_LOCAL_UNITS + 1];  // resident CTAs per SM for [V == 32][large parameter block][local units], 0 = not yet asked
   unsigned queue_slot = 0;
 };
 
@@ -41,10 +42,11 @@ long long g_launches = 0;
     }                                        \
   } while (0)
 
-template <int NREG, int PW>
+template <int V, int PW>
 int occupancy(int* out, size_t smem) {
   int n = 0;
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<NREG, PW>, dvm::THREADS, smem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW>, dvm::THREADS, smem));
   *out = n > 0 ? n : 1;
   return DVM_OK;
 }
@@ -61,18 +63,29 @@ int dvm_device_state(DvmDeviceInfo* info) {
     DVM_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
     DVM_CUDA(cudaMalloc(&d.scratch, 4096));
     DVM_CUDA(cudaMemset(d.scratch, 0, 4096));
-    int st;
-    if ((st = occupancy<4, PW_SMALL>(&d.occ[0][0], 2048)) != DVM_OK) return st;
-    if ((st = occupancy<4, PW_LARGE>(&d.occ[0][1], 32768)) != DVM_OK) return st;
-    if ((st = occupancy<8, PW_SMALL>(&d.occ[1][0], 2048)) != DVM_OK) return st;
-    if ((st = occupancy<8, PW_LARGE>(&d.occ[1][1], 32768)) != DVM_OK) return st;
+    memset(d.occ, 0, sizeof d.occ);
     d.ready = true;
   }
   info->scratch = d.scratch;
   info->sm_count = d.sm_count;
   info->queue_slot = d.queue_slot;
   d.queue_slot = (d.queue_slot + 1) % QUEUE_SLOTS;
-  memcpy(info->occ, d.occ, sizeof d.occ);
+  return DVM_OK;
+}
+
+// Resident CTAs per SM of the interpreter for a launch with `units` local-memory units (cached per device).
+static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out) {
+  int dev = 0;
+  DVM_CUDA(cudaGetDevice(&dev));
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceState& d = g_dev[dev];
+  int& slot = d.occ[V == 32][large ? 1 : 0][units];
+  if (slot == 0) {
+    int st = V == 32 ? (large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem))
+                     : (large ? occupancy<16, PW_LARGE>(&slot, smem) : occupancy<16, PW_SMALL>(&slot, smem));
+    if (st != DVM_OK) return st;
+  }
+  *out = slot;
   return DVM_OK;
 }
 
@@ -115,10 +128,10 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   return DVM_OK;
 }
 
-template <int NREG, int PW>
-int launch_variant(const dvm::VMParams<PW>& prm, int grid, cudaStream_t stream) {
-  size_t smem = (size_t)prm.n_words * 4;
-  dvm::dvm_vm_kernel<NREG, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
+template <int PW>
+int launch_variant(int V, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+  if (V == 32) dvm::dvm_vm_kernel<32, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  else dvm::dvm_vm_kernel<16, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;
@@ -132,12 +145,16 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   uint32_t dir = 2 * (uint32_t)n_programs + 1;
   uint64_t need = dir;
   uint64_t total_tiles = 0;
-  uint32_t nreg = 4;
+  uint32_t units = 0;
+  int V = 0;
   for (int i = 0; i < n_programs; ++i) {
     const uint32_t* c = (const uint32_t*)codes[i];
     need += c[DVM_H_TOTAL_WORDS];
     total_tiles += c[DVM_H_N_TILES];
-    if (((c[DVM_H_GEOM] >> 16) & 0xff) > nreg) nreg = 8;
+    if (((c[DVM_H_LOCAL2] >> 16) & 0xff) > units) units = (c[DVM_H_LOCAL2] >> 16) & 0xff;
+    const int v = (int)(c[DVM_H_LOCAL] >> 24);
+    if (V && v != V) return DVM_ERR_INVALID_ARG;  // one kernel variant per launch: same elements per thread
+    V = v;
   }
   if (need > PW_LARGE || total_tiles > 0xffffffffull) return DVM_ERR_TOO_LARGE;
   if (total_tiles == 0) return DVM_OK;
@@ -166,15 +183,19 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.queue = dev.scratch + 8 + 2 * dev.queue_slot;
 
   const bool large = pos > PW_SMALL;
-  const int occ = dev.occ[nreg == 8][large];
+  const size_t smem = (size_t)units * DVM_LOCAL_UNIT;
+  if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
+  int occ = 0;
+  st = dvm_occupancy(V, large, (int)units, smem, &occ);
+  if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
   int grid = (int)(total_tiles < slots ? total_tiles : slots);
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
-    return nreg == 8 ? launch_variant<8, PW_SMALL>(S, grid, stream) : launch_variant<4, PW_SMALL>(S, grid, stream);
+    return launch_variant<PW_SMALL>(V, S, grid, smem, stream);
   }
-  return nreg == 8 ? launch_variant<8, PW_LARGE>(P, grid, stream) : launch_variant<4, PW_LARGE>(P, grid, stream);
+  return launch_variant<PW_LARGE>(V, P, grid, smem, stream);
 }
 
 }  // namespace

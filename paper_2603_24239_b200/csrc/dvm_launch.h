@@ -8,7 +8,6 @@ struct DvmDeviceInfo {
   unsigned int* scratch;  // library-owned device words: [0] status, then work-queue counter pairs
   int sm_count;
   unsigned queue_slot;    // work-queue slot reserved for this launch
-  int occ[2][2];
 };
 
 // Per-device lazy set-up (scratch allocation, occupancy) for the current device.

@@ -1,22 +1,36 @@
 // Device half of the operator compiler: the virtual machine (Sec. 4.3, Algorithm 2)
 // as a persistent sm_100a kernel.
 //
-// One CTA of 256 threads is one "core" of Algorithm 2.  It copies the bytecode
-// program(s) from the kernel-parameter block into shared memory once, then loops
-// over its tiles; per tile every warp walks the code body, decoding one
-// instruction word at a time (a warp-uniform shared-memory read and a uniform
-// branch) and executing the tile-level virtual instruction on register-resident
-// tile registers.
+// One CTA of 256 threads is one "core" of Algorithm 2.  The bytecode program(s)
+// arrive as the kernel-parameter block; every warp fetches instruction words
+// from that block through the constant bank (a warp-uniform load, so decode and
+// dispatch run on uniform registers and uniform branches) and loops over the
+// CTA's tiles.  A code body is [load section][compute section]:
+//   * the load section of tile i+1 is executed while tile i is computed: every
+//     global tile load is an asynchronous 16-byte global->shared copy
+//     (cp.async) into a thread-private "local register" in shared memory -- the
+//     paper's local memory -- so the next tile's HBM traffic is in flight with
+//     no register cost (double-buffered input registers);
+//   * the compute section is accumulator code: ACC is one register-resident tile
+//     (V = 16 or 32 fp32 per thread, as float2 pairs so that add / mul / fma
+//     issue as packed f32x2 instructions); other operands are read from local
+//     registers with 128-bit shared loads (bf16 operands widened on the fly) or
+//     are per-row scalars S0..S7.
 //
 // Tile geometry (chosen per instance by the host's shape tiling):
 //   G = 2^lgG threads share one row; a CTA holds 256/G rows per tile.
-//   Every thread owns V = 16 element slots of each tile register; slot s maps to
+//   Every thread owns V element slots of a tile register; slot s maps to
 //   column  (t + G*(s / W)) * W + (s % W) - shift  of the tile's column block,
 //   t = thread index inside the row group, W = vector width in elements,
 //   shift = misalignment of the row segment start, so that a thread's W-slot
 //   chunk is a 16-byte aligned vector of the primary operand.
-// Tile registers R0..R{NREG-1} hold fp32 values (R0 is the accumulator); S0..S7
-// hold one fp32 value per row (reduction results, per-row inputs).
+// Chunks that are not whole, aligned 16-byte vectors (row heads and tails, the
+// element-wise W = 1 mapping, operands whose alignment differs from the primary
+// operand's) take a scalar path through the same local registers.
+//
+// Local memory layout: units of 8 KB (32 bytes per thread); 16-byte vector q of a
+// register at unit offset U lives at  U*8192 + (q * 256 + tid) * 16,
+// i.e. consecutive threads touch consecutive vectors (no bank conflicts).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -26,8 +40,10 @@
 
 namespace dvm {
 
-constexpr int V = DVM_VM_V;
 constexpr int THREADS = DVM_VM_THREADS;
+#ifndef DVM_VM_MIN_CTAS
+#define DVM_VM_MIN_CTAS 2
+#endif
 
 // Device status word values (read back by dvm_last_device_status).
 enum { ST_OK = 0, ST_BAD_CODE = 1, ST_TIMEOUT = 2 };
@@ -44,36 +60,18 @@ struct VMParams {
 };
 
 struct TileCtx {
-  int t;        // thread index within the row group
-  int lgG;
-  int W, lgW;
+  uint32_t prog;     // word offset of the tile's program in the parameter block
+  int t;             // thread index within the row group
+  int lgG, lgW;
   int shift;
-  int ncols;    // valid columns of this thread's row inside the column block (0: nothing to do)
-  uint32_t vmask;  // bit s set: slot s holds a valid element
-  long long i0, i1, i2;  // row coordinates over the collapsed outer dims
-  long long col0;
-  bool outer;
+  int ncols;         // valid columns of this thread's row inside the column block (0: nothing to do)
+  uint32_t vmask;    // bit s: slot s holds a valid element
+  uint32_t fullmask; // bit j: chunk j lies entirely inside the row segment
+  uint32_t partmask; // bit j: chunk j straddles the segment boundary (W == 1: the slot is valid)
+  uint32_t i0, i1, i2;  // row coordinates over the collapsed outer dims
+  uint32_t col0;
+  uint32_t flags;
 };
-
-template <int NREG, class F>
-__device__ __forceinline__ void with_reg(float (&R)[NREG][V], int k, F&& f) {
-  switch (k) {
-    case 0: f(R[0]); break;
-    case 1: f(R[1]); break;
-    case 2: f(R[2]); break;
-    case 3: f(R[3]); break;
-    default:
-      if constexpr (NREG > 4) {
-        switch (k) {
-          case 4: f(R[4]); break;
-          case 5: f(R[5]); break;
-          case 6: f(R[6]); break;
-          default: f(R[7]); break;
-        }
-      }
-      break;
-  }
-}
 
 __device__ __forceinline__ float sget(const float (&S)[DVM_MAX_SREGS], int k) {
   float v = S[0];
@@ -86,7 +84,9 @@ __device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) 
   for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = (k == i) ? v : S[i];
 }
 
-__device__ __forceinline__ float arith(int op, float a, float b) {
+__device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+__device__ __forceinline__ float scalar_arith(int op, float a, float b) {
   switch (op) {
     case DVM_A_ADD: return a + b;
     case DVM_A_SUB: return a - b;
@@ -99,9 +99,7 @@ __device__ __forceinline__ float arith(int op, float a, float b) {
   }
 }
 
-__device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
-
-__device__ __forceinline__ float unary(int op, float x) {
+__device__ __forceinline__ float scalar_unary(int op, float x) {
   switch (op) {
     case DVM_U_EXP: return expf(x);
     case DVM_U_SQRT: return sqrtf(x);
@@ -119,359 +117,346 @@ __device__ __forceinline__ float unary(int op, float x) {
   }
 }
 
-// Column (relative to the column block) of the first slot of chunk j.
-__device__ __forceinline__ int chunk_col(const TileCtx& c, int j) {
-  return ((c.t + (j << c.lgG)) << c.lgW) - c.shift;
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Column (relative to the column block) of slot s.
+__device__ __forceinline__ int slot_col(const TileCtx& c, int s) {
+  return ((c.t + ((s >> c.lgW) << c.lgG)) << c.lgW) + (s & ((1 << c.lgW) - 1)) - c.shift;
 }
 
-// ---- tile load: vector path straight into the destination register ---------------------------
-// Raw element bits are written: fp32 as is, bf16 packed two per word (slots 2i, 2i+1 in word i);
-// a later CVT instruction widens bf16 in place.  Chunks that straddle the row boundary or are not
-// 16-byte aligned are flagged in slow_mask and fetched element-wise by ldg_slow.
-template <int W, bool BF16>
-__device__ __forceinline__ void ldg_fast(float (&r)[V], const char* p, const TileCtx& c, uint32_t& slow_mask) {
-  constexpr int ES = BF16 ? 2 : 4;
-#pragma unroll
-  for (int i = 0; i < V; ++i) r[i] = 0.f;
-  if constexpr (W == 1) {
-#pragma unroll
-    for (int s = 0; s < V; ++s) {
-      int col = c.t + (s << c.lgG);
-      if (col < c.ncols) {
-        if constexpr (BF16) {
-          uint32_t h = *reinterpret_cast<const unsigned short*>(p + (long long)col * ES);
-          uint32_t w = __float_as_uint(r[s >> 1]) | (h << (16 * (s & 1)));
-          r[s >> 1] = __uint_as_float(w);
-        } else {
-          r[s] = *reinterpret_cast<const float*>(p + (long long)col * ES);
-        }
-      }
-    }
-  } else {
-    constexpr int NCH = V / W;
-#pragma unroll
-    for (int j = 0; j < NCH; ++j) {
-      int c0 = chunk_col(c, j);
-      const char* q = p + (long long)c0 * ES;
-      bool full = (c0 >= 0) && (c0 + W <= c.ncols);
-      bool al = (reinterpret_cast<uintptr_t>(q) & 15) == 0;
-      if (full && al) {
-        if constexpr (BF16) {  // W == 8: one 16-byte vector
-          uint4 v = *reinterpret_cast<const uint4*>(q);
-          r[4 * j + 0] = __uint_as_float(v.x);
-          r[4 * j + 1] = __uint_as_float(v.y);
-          r[4 * j + 2] = __uint_as_float(v.z);
-          r[4 * j + 3] = __uint_as_float(v.w);
-        } else {
-#pragma unroll
-          for (int h = 0; h < W / 4; ++h) {
-            float4 v = *reinterpret_cast<const float4*>(q + 16 * h);
-            r[W * j + 4 * h + 0] = v.x;
-            r[W * j + 4 * h + 1] = v.y;
-            r[W * j + 4 * h + 2] = v.z;
-            r[W * j + 4 * h + 3] = v.w;
-          }
-        }
-      } else if (c0 + W > 0 && c0 < c.ncols) {
-        slow_mask |= 1u << j;
-      }
-    }
-  }
-}
-
-// Element-wise fetch of the chunks flagged in slow_mask into tmp (same raw layout).
-template <int W, bool BF16>
-__device__ __noinline__ void ldg_slow(float (&tmp)[V], const char* p, const TileCtx& c, uint32_t slow_mask) {
-  constexpr int ES = BF16 ? 2 : 4;
-  constexpr int NCH = V / W;
-#pragma unroll
-  for (int i = 0; i < V; ++i) tmp[i] = 0.f;
-#pragma unroll
-  for (int j = 0; j < NCH; ++j) {
-    if (!((slow_mask >> j) & 1)) continue;
-    int c0 = chunk_col(c, j);
-#pragma unroll
-    for (int e = 0; e < W; ++e) {
-      int col = c0 + e;
-      int s = W * j + e;
-      if (col >= 0 && col < c.ncols) {
-        if constexpr (BF16) {
-          uint32_t h = *reinterpret_cast<const unsigned short*>(p + (long long)col * ES);
-          uint32_t w = __float_as_uint(tmp[s >> 1]) | (h << (16 * (s & 1)));
-          tmp[s >> 1] = __uint_as_float(w);
-        } else {
-          tmp[s] = *reinterpret_cast<const float*>(p + (long long)col * ES);
-        }
-      }
-    }
-  }
-}
-
-template <int W, bool BF16>
-__device__ __forceinline__ void merge_slow(float (&r)[V], const float (&tmp)[V], uint32_t slow_mask) {
-  constexpr int NCH = V / W;
-  constexpr int WPC = BF16 ? W / 2 : W;  // raw words per chunk
-#pragma unroll
-  for (int j = 0; j < NCH; ++j) {
-    bool take = (slow_mask >> j) & 1;
-#pragma unroll
-    for (int i = 0; i < WPC; ++i) r[WPC * j + i] = take ? tmp[WPC * j + i] : r[WPC * j + i];
-  }
-}
-
-// ---- tile store from the accumulator -------------------------------------------------------------
-template <int W, bool BF16>
-__device__ __forceinline__ void stg_tile(const float (&a)[V], char* p, const TileCtx& c) {
-  constexpr int ES = BF16 ? 2 : 4;
-  if constexpr (W == 1) {
-#pragma unroll
-    for (int s = 0; s < V; ++s) {
-      int col = c.t + (s << c.lgG);
-      if (col < c.ncols) {
-        if constexpr (BF16) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * ES) = __float2bfloat16_rn(a[s]);
-        else *reinterpret_cast<float*>(p + (long long)col * ES) = a[s];
-      }
-    }
-  } else {
-    constexpr int NCH = V / W;
-#pragma unroll
-    for (int j = 0; j < NCH; ++j) {
-      int c0 = chunk_col(c, j);
-      char* q = p + (long long)c0 * ES;
-      bool full = (c0 >= 0) && (c0 + W <= c.ncols);
-      bool al = (reinterpret_cast<uintptr_t>(q) & 15) == 0;
-      if (full && al) {
-        if constexpr (BF16) {
-          uint4 v;
-          __nv_bfloat162 b0 = __floats2bfloat162_rn(a[8 * j + 0], a[8 * j + 1]);
-          __nv_bfloat162 b1 = __floats2bfloat162_rn(a[8 * j + 2], a[8 * j + 3]);
-          __nv_bfloat162 b2 = __floats2bfloat162_rn(a[8 * j + 4], a[8 * j + 5]);
-          __nv_bfloat162 b3 = __floats2bfloat162_rn(a[8 * j + 6], a[8 * j + 7]);
-          v.x = *reinterpret_cast<uint32_t*>(&b0);
-          v.y = *reinterpret_cast<uint32_t*>(&b1);
-          v.z = *reinterpret_cast<uint32_t*>(&b2);
-          v.w = *reinterpret_cast<uint32_t*>(&b3);
-          *reinterpret_cast<uint4*>(q) = v;
-        } else {
-#pragma unroll
-          for (int h = 0; h < W / 4; ++h)
-            *reinterpret_cast<float4*>(q + 16 * h) =
-                make_float4(a[W * j + 4 * h], a[W * j + 4 * h + 1], a[W * j + 4 * h + 2], a[W * j + 4 * h + 3]);
-        }
-      } else if (c0 + W > 0 && c0 < c.ncols) {
-#pragma unroll
-        for (int e = 0; e < W; ++e) {
-          int col = c0 + e;
-          if (col >= 0 && col < c.ncols) {
-            if constexpr (BF16)
-              *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * ES) = __float2bfloat16_rn(a[W * j + e]);
-            else
-              *reinterpret_cast<float*>(p + (long long)col * ES) = a[W * j + e];
-          }
-        }
-      }
-    }
-  }
-}
-
-// bf16 raw words -> fp32 values, in place (descending so that no raw word is overwritten early).
-__device__ __forceinline__ void widen_bf16(float (&r)[V]) {
-#pragma unroll
-  for (int i = V / 2 - 1; i >= 0; --i) {
-    uint32_t w = __float_as_uint(r[i]);
-    r[2 * i + 1] = __uint_as_float(w & 0xffff0000u);
-    r[2 * i] = __uint_as_float(w << 16);
-  }
-}
-
-struct OperandAddr {
-  char* ptr;    // address of element (row, col0) -- or of the row's single value for col_stride 0
-  int dtype;
-};
-
-__device__ __forceinline__ OperandAddr operand_addr(const uint32_t* prog, const uint32_t* opd_table, int b,
-                                                    const TileCtx& c) {
-  const uint32_t* d = opd_table + b * DVM_OPD_WORDS;
-  uint32_t info = d[DVM_OPD_INFO];
-  int slot = info & 0xff;
-  int dt = (info >> 8) & 0xff;
-  int cs = (info >> 16) & 0xff;
-  const uint32_t* tp = prog + DVM_HDR_WORDS + 2 * slot;
-  unsigned long long base = (unsigned long long)tp[0] | ((unsigned long long)tp[1] << 32);
-  long long s0 = (long long)((unsigned long long)d[DVM_OPD_STRIDE0] | ((unsigned long long)d[DVM_OPD_STRIDE0 + 1] << 32));
-  long long off = c.i0 * s0;
-  if (c.outer) {
-    long long s1 = (long long)((unsigned long long)d[DVM_OPD_STRIDE1] | ((unsigned long long)d[DVM_OPD_STRIDE1 + 1] << 32));
-    long long s2 = (long long)((unsigned long long)d[DVM_OPD_STRIDE2] | ((unsigned long long)d[DVM_OPD_STRIDE2 + 1] << 32));
-    off += c.i1 * s1 + c.i2 * s2;
-  }
-  if (cs) off += c.col0;
-  OperandAddr a;
-  a.ptr = reinterpret_cast<char*>(base) + off * (dt == DVM_DT_BF16 ? 2 : 4);
-  a.dtype = dt;
-  return a;
-}
-
-template <int NREG, int PW>
-__global__ void __launch_bounds__(THREADS, (NREG <= 4 ? 2 : 1))
-dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
-  extern __shared__ __align__(16) uint32_t s_code[];
+template <int V, int PW>
+__global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
+  constexpr int VP = V / 2;  // float2 pairs per tile register
+  extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ float s_red[2][THREADS / 32];
   __shared__ uint32_t s_next[2];
 
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
-  for (uint32_t i = tid; i < prm.n_words; i += THREADS) s_code[i] = prm.words[i];
-  __syncthreads();
-
+  const uint32_t local_base = static_cast<uint32_t>(__cvta_generic_to_shared(s_dyn)) + (uint32_t)tid * 16;
   const uint32_t n_prog = prm.n_programs;
-  const uint32_t* tile_base = s_code + n_prog;
-  float R[NREG][V];
+#define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
+
+  // shared-memory address of 16-byte vector q of the register at unit offset U (this thread's part)
+  auto lvec = [&](uint32_t unit, int q) -> uint32_t { return local_base + unit * DVM_LOCAL_UNIT + (uint32_t)q * (THREADS * 16); };
+
+  // word offsets of a program's tables
+  auto opd_base = [&](uint32_t prog) -> uint32_t { return prog + DVM_HDR_WORDS + 2 * (CW(prog + DVM_H_COUNTS) & 0xff); };
+  auto lreg_base = [&](uint32_t prog) -> uint32_t { return opd_base(prog) + ((CW(prog + DVM_H_COUNTS) >> 16) & 0xff) * DVM_OPD_WORDS; };
+  auto body_base = [&](uint32_t prog) -> uint32_t { return lreg_base(prog) + ((CW(prog + DVM_H_GEOM) >> 16) & 0xff); };
+
+  // Address of element (row, col0) of operand b -- or of the row's single value when col_stride = 0.
+  auto operand_addr = [&](uint32_t prog, uint32_t opd0, int b, const TileCtx& c, int& dtype) -> char* {
+    const uint32_t d = opd0 + b * DVM_OPD_WORDS;
+    const uint32_t info = CW(d + DVM_OPD_INFO);
+    const uint32_t tp = prog + DVM_HDR_WORDS + 2 * (info & 0xff);
+    const unsigned long long base = (unsigned long long)CW(tp) | ((unsigned long long)CW(tp + 1) << 32);
+    dtype = (info >> 8) & 0xff;
+    unsigned long long off =
+        (unsigned long long)c.i0 * ((unsigned long long)CW(d + DVM_OPD_STRIDE0) | ((unsigned long long)CW(d + DVM_OPD_STRIDE0 + 1) << 32));
+    if (c.flags & DVM_F_OUTER_DIMS) {
+      off += (unsigned long long)c.i1 * ((unsigned long long)CW(d + DVM_OPD_STRIDE1) | ((unsigned long long)CW(d + DVM_OPD_STRIDE1 + 1) << 32));
+      off += (unsigned long long)c.i2 * ((unsigned long long)CW(d + DVM_OPD_STRIDE2) | ((unsigned long long)CW(d + DVM_OPD_STRIDE2 + 1) << 32));
+    }
+    if ((info >> 16) & 0xff) off += c.col0;
+    return reinterpret_cast<char*>(base + (off << (dtype == DVM_DT_BF16 ? 1 : 2)));
+  };
+
+  // Tile id -> geometry of this thread's part of the tile.
+  auto make_ctx = [&](TileCtx& c, uint32_t prog, uint32_t local_tile) {
+    c.prog = prog;
+    const uint32_t geom = CW(prog + DVM_H_GEOM);
+    c.lgG = geom & 0xff;
+    const int W = (geom >> 8) & 0xff;
+    c.lgW = W == 8 ? 3 : (W == 4 ? 2 : 0);
+    c.flags = geom >> 24;
+    const int G = 1 << c.lgG;
+    c.t = tid & (G - 1);
+    const uint32_t CB = CW(prog + DVM_H_COL_BLOCKS);
+    uint32_t rb = local_tile, cb = 0;
+    if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
+    const uint32_t rows = CW(prog + DVM_H_ROWS_LO);  // the host rejects more than 2^32 - 1 rows per program
+    const uint32_t row = rb * (uint32_t)(THREADS >> c.lgG) + (uint32_t)(tid >> c.lgG);
+    const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
+    c.col0 = cb * ctile;
+    const uint32_t cend = (row == rows - 1) ? CW(prog + DVM_H_LAST_ROW_COLS) : CW(prog + DVM_H_COLS);
+    int nc = 0;
+    if (row < rows && cend > c.col0) nc = (int)min(cend - c.col0, ctile);
+    c.ncols = nc;
+    c.i0 = row < rows ? row : 0;
+    c.i1 = c.i2 = 0;
+    if (c.flags & DVM_F_OUTER_DIMS) {
+      const uint32_t n0 = CW(prog + DVM_H_OUTER0), n1 = CW(prog + DVM_H_OUTER1);
+      const uint32_t q = c.i0 / n0;
+      c.i0 -= q * n0;
+      c.i2 = q / n1;
+      c.i1 = q - c.i2 * n1;
+    }
+    c.shift = 0;
+    if (!(c.flags & DVM_F_ALIGNED) && W > 1) {
+      const uint32_t pr = CW(prog + DVM_H_PRIMARY);
+      if (pr != 0xffffffffu) {
+        int dt;
+        const unsigned long long a = reinterpret_cast<unsigned long long>(operand_addr(prog, opd_base(prog), (int)pr, c, dt));
+        c.shift = (int)((a >> (dt == DVM_DT_BF16 ? 1 : 2)) & (unsigned long long)(W - 1));
+      }
+    }
+    // chunk j of this thread covers columns [c0 + j*G*W, +W)
+    uint32_t full = 0, part = 0, vm = 0;
+    if (W > 1 && c.shift == 0) {
+      // aligned row segment: the first nf chunks are whole, chunk nf may be cut by the segment end
+      const int nch = V >> c.lgW;
+      const int avail = (c.ncols >> c.lgW) - c.t;               // whole chunks of the row at or after chunk t
+      int nf = avail > 0 ? ((avail + G - 1) >> c.lgG) : 0;       // those that belong to this thread
+      nf = nf < nch ? nf : nch;
+      full = (1u << nf) - 1u;
+      vm = nf >= (32 >> c.lgW) ? 0xffffffffu : ((1u << (nf << c.lgW)) - 1u);
+      if (nf < nch) {
+        const int rem = c.ncols - ((c.t + (nf << c.lgG)) << c.lgW);  // valid columns of the next chunk
+        if (rem > 0) { part = 1u << nf; vm |= ((1u << rem) - 1u) << (nf << c.lgW); }
+      }
+    } else if (W > 1) {
+      const int nch = V >> c.lgW;
+      const int c0 = (c.t << c.lgW) - c.shift;
+      const int step = G << c.lgW;
+#pragma unroll 1
+      for (int j = 0; j < nch; ++j) {
+        const int cj = c0 + j * step;
+        if (cj >= 0 && cj + W <= c.ncols) { full |= 1u << j; vm |= ((1u << W) - 1) << (j * W); }
+        else if (cj + W > 0 && cj < c.ncols) part |= 1u << j;
+      }
+      if (part) {
+#pragma unroll 1
+        for (int s = 0; s < V; ++s) {
+          const int col = slot_col(c, s);
+          if (((part >> (s >> c.lgW)) & 1) && col >= 0 && col < c.ncols) vm |= 1u << s;
+        }
+      }
+    } else {
+#pragma unroll 1
+      for (int s = 0; s < V; ++s)
+        if (c.t + s * G < c.ncols) vm |= 1u << s;
+      part = vm;  // element-wise mapping: every valid slot takes the scalar path
+    }
+    c.vmask = vm;
+    c.fullmask = full;
+    c.partmask = part;
+  };
+
+  // ---- load section of one tile: asynchronous copies into the input registers of buffer `buf` ----
+  auto issue_loads = [&](const TileCtx& c, int buf, bool first_of_program) {
+    const uint32_t prog = c.prog;
+    const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
+    const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
+    const int W = 1 << c.lgW;
+    const int G = 1 << c.lgG;
+    for (uint32_t pc = 0; pc < load_words; ++pc) {
+      const uint32_t w0 = CW(body0 + pc);
+      const int ia = DVM_INSN_A(w0) & 0x7f, ib = DVM_INSN_B(w0);
+      if ((DVM_INSN_A(w0) & 0x80) && !first_of_program) continue;  // tile-invariant operand: already in local memory
+      int dt;
+      const char* p = operand_addr(prog, opd0, ib, c, dt);
+      if (DVM_INSN_OP(w0) == DVM_OP_LDG) {
+        const uint32_t lt = CW(lreg0 + ia);
+        const uint32_t unit = buf ? (lt >> 16) : (lt & 0xffff);
+        const int es = dt == DVM_DT_BF16 ? 2 : 4;
+        const char* q0 = p + (long long)((c.t << c.lgW) - c.shift) * es;
+        const long long qstep = (long long)(G << c.lgW) * es;
+        const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
+        const uint32_t fast = (al && W > 1) ? c.fullmask : 0u;
+        const uint32_t slow = c.partmask | (c.fullmask & ~fast);
+        const int vpc = (W * es) >> 4;  // 16-byte vectors per chunk (1 or 2); W = 1 never takes this path
+        if (fast) {
+#pragma unroll
+          for (int j = 0; j < V / 4; ++j) {
+            if ((fast >> j) & 1) {
+              cp_async16(lvec(unit, j * vpc), q0 + j * qstep);
+              if (vpc == 2) cp_async16(lvec(unit, j * vpc + 1), q0 + j * qstep + 16);
+            }
+          }
+        }
+        if (slow) {
+          // scalar path: element by element into the same local register (raw element bits)
+#pragma unroll 1
+          for (int s = 0; s < V; ++s) {
+            if (!((slow >> (s >> c.lgW)) & 1) || !((c.vmask >> s) & 1)) continue;
+            const int col = slot_col(c, s);
+            const uint32_t b = (uint32_t)s * es;
+            const uint32_t dst = lvec(unit, b >> 4) + (b & 15);
+            if (dt == DVM_DT_BF16) {
+              const unsigned short hv = *reinterpret_cast<const unsigned short*>(p + (long long)col * 2);
+              asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst), "h"(hv) : "memory");
+            } else {
+              cp_async4(dst, p + (long long)col * 4);
+            }
+          }
+        }
+      } else {  // DVM_OP_LDS: one value per row into scalar slot ia of this buffer
+        const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
+        const uint32_t w = (uint32_t)buf * DVM_MAX_SSLOTS + (uint32_t)ia;
+        const uint32_t dst = lvec(unit, w >> 2) + (w & 3) * 4;
+        if (c.ncols > 0) {
+          if (dt == DVM_DT_BF16) {
+            const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(p));
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(v) : "memory");
+          } else {
+            cp_async4(dst, p);
+          }
+        }
+      }
+    }
+  };
+
+  float2 A[VP];
   float S[DVM_MAX_SREGS];
 #pragma unroll
   for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = 0.f;
 #pragma unroll
-  for (int k = 0; k < NREG; ++k)
+  for (int i = 0; i < VP; ++i) A[i] = make_float2(0.f, 0.f);
+
+#define DVM_EACH_PAIR _Pragma("unroll") for (int i = 0; i < VP; ++i)
+
+  // reads local register `unit` (element type dt) into o[] as fp32 pairs
+  auto read_lreg = [&](float2 (&o)[VP], uint32_t unit, int dt) {
+    const uint32_t a0 = lvec(unit, 0);
+    if (dt == DVM_DT_BF16) {
 #pragma unroll
-    for (int i = 0; i < V; ++i) R[k][i] = 0.f;
+      for (int q = 0; q < V / 8; ++q) {
+        uint4 v;
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a0 + q * (THREADS * 16)));
+        o[4 * q + 0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+        o[4 * q + 1] = make_float2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+        o[4 * q + 2] = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
+        o[4 * q + 3] = make_float2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < V / 4; ++q) {
+        float4 v;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a0 + q * (THREADS * 16)));
+        o[2 * q] = make_float2(v.x, v.y);
+        o[2 * q + 1] = make_float2(v.z, v.w);
+      }
+    }
+  };
 
   uint32_t prog_idx = 0;
   uint32_t tile = blockIdx.x;
   uint32_t iter = 0;
   int red_par = 0;
+  int buf = 0;
   unsigned err = 0;
 
+  TileCtx c;
+  if (tile < prm.total_tiles) {
+    while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
+    make_ctx(c, CW(prog_idx), tile - CW(n_prog + prog_idx));
+    issue_loads(c, buf, true);
+    cp_async_commit();
+  }
+
   while (tile < prm.total_tiles) {
-    if (prm.use_queue && tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
+    // ---- Algorithm 2, outer loop: next tile of this core; its loads start now when it runs the same program ----
+    uint32_t next;
+    if (prm.use_queue) {
+      if (tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
+      __syncthreads();
+      next = s_next[iter & 1];
+    } else {
+      next = tile + gridDim.x;
+    }
+    ++iter;
+    TileCtx cn = c;
+    const bool have_next = next < prm.total_tiles;
+    bool early = false;
+    uint32_t next_prog_idx = prog_idx;
+    if (have_next) {
+      while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
+      early = next_prog_idx == prog_idx;  // another program has another local-memory layout: load it after this tile
+      make_ctx(cn, CW(next_prog_idx), next - CW(n_prog + next_prog_idx));
+      if (early) {
+        issue_loads(cn, buf ^ 1, false);
+        cp_async_commit();
+      }
+    }
+    if (early) cp_async_wait<1>(); else cp_async_wait<0>();
 
-    // ---- locate the program of this tile (stacked launches); tiles are claimed in increasing order ----
-    while (prog_idx + 1 < n_prog && tile >= tile_base[prog_idx + 1]) ++prog_idx;
-    const uint32_t* prog = s_code + s_code[prog_idx];
-    const uint32_t counts = prog[DVM_H_COUNTS];
-    const uint32_t n_tensors = counts & 0xff, n_opd = (counts >> 16) & 0xff;
-    const uint32_t* opd_table = prog + DVM_HDR_WORDS + 2 * n_tensors;
-    const uint32_t* body = opd_table + n_opd * DVM_OPD_WORDS;
-    const uint32_t body_words = prog[DVM_H_CODE_WORDS];
-    const uint32_t geom = prog[DVM_H_GEOM];
-
-    TileCtx c;
-    c.lgG = geom & 0xff;
-    c.W = (geom >> 8) & 0xff;
-    c.lgW = c.W == 8 ? 3 : (c.W == 4 ? 2 : 0);
-    const uint32_t flags = geom >> 24;
-    c.outer = (flags & DVM_F_OUTER_DIMS) != 0;
+    const uint32_t prog = c.prog;
+    const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
+    const uint32_t body_words = CW(prog + DVM_H_CODE_WORDS);
+    const int W = 1 << c.lgW;
     const int G = 1 << c.lgG;
-    c.t = tid & (G - 1);
-    const int g = tid >> c.lgG;
-    const uint32_t local_tile = tile - tile_base[prog_idx];
-    const uint32_t CB = prog[DVM_H_COL_BLOCKS];
-    uint32_t rb = local_tile, cb = 0;
-    if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
-    const long long rows = (long long)((unsigned long long)prog[DVM_H_ROWS_LO] | ((unsigned long long)prog[DVM_H_ROWS_HI] << 32));
-    const long long row = (long long)rb * (THREADS >> c.lgG) + g;
-    const uint32_t ctile = prog[DVM_H_COL_TILE];
-    c.col0 = (long long)cb * ctile;
-    {
-      long long cend = (row == rows - 1) ? (long long)prog[DVM_H_LAST_ROW_COLS] : (long long)prog[DVM_H_COLS];
-      long long nc = cend - c.col0;
-      if (nc > (long long)ctile) nc = ctile;
-      if (nc < 0 || row >= rows) nc = 0;
-      c.ncols = (int)nc;
-    }
-    c.i0 = row < rows ? row : 0;
-    c.i1 = c.i2 = 0;
-    if (c.outer) {
-      unsigned long long n0 = prog[DVM_H_OUTER0], n1 = prog[DVM_H_OUTER1];
-      unsigned long long q = (unsigned long long)c.i0 / n0;
-      c.i0 = (long long)((unsigned long long)c.i0 - q * n0);
-      unsigned long long q2 = q / n1;
-      c.i1 = (long long)(q - q2 * n1);
-      c.i2 = (long long)q2;
-    }
-    c.shift = 0;
-    if (!(flags & DVM_F_ALIGNED) && c.W > 1) {
-      const uint32_t pr = prog[DVM_H_PRIMARY];
-      if (pr != 0xffffffffu) {
-        OperandAddr pa = operand_addr(prog, opd_table, (int)pr, c);
-        unsigned long long e = reinterpret_cast<unsigned long long>(pa.ptr) >> (pa.dtype == DVM_DT_BF16 ? 1 : 2);
-        c.shift = (int)(e & (unsigned long long)(c.W - 1));
-      }
-    }
-    {
-      uint32_t m = 0;
-#pragma unroll
-      for (int s = 0; s < V; ++s) {
-        int col = ((c.t + ((s >> c.lgW) << c.lgG)) << c.lgW) + (s & (c.W - 1)) - c.shift;
-        if (col >= 0 && col < c.ncols) m |= 1u << s;
-      }
-      c.vmask = m;
-    }
+    const bool all_valid = __all_sync(0xffffffffu, c.vmask == (V == 32 ? 0xffffffffu : 0xffffu));
+    const uint32_t staging_unit = buf ? (CW(prog + DVM_H_LOCAL2) >> 24) : (CW(prog + DVM_H_LOCAL2) & 0xff);
 
-    // ---- Algorithm 2, inner loop: walk the code body ----
-    float (&A)[V] = R[0];
-    uint32_t pc = 0;
+    // ---- Algorithm 2, inner loop: walk the compute section ----
+    uint32_t pc = CW(prog + DVM_H_LOAD_WORDS);
     while (pc < body_words) {
-      const uint32_t w0 = body[pc];
+      const uint32_t w0 = CW(body0 + pc);
       const uint32_t op = DVM_INSN_OP(w0);
       const int ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
-      const uint32_t len = DVM_INSN_LEN(w0);
-      if (op >= DVM_OP_BIN && op < DVM_OP_BIN + 8 * DVM_A_NBIN) {
-        const int ar = (op - DVM_OP_BIN) >> 3, k = (op - DVM_OP_BIN) & 7;
-        switch (ar) {
-#define DVM_BIN_CASE(AR, EXPR)                                   \
-  case AR:                                                       \
-    with_reg<NREG>(R, k, [&](float (&r)[V]) {                    \
-      _Pragma("unroll") for (int i = 0; i < V; ++i) {            \
-        const float x = A[i], y = r[i];                          \
-        A[i] = (EXPR);                                           \
-      }                                                          \
-    });                                                          \
+      pc += max(DVM_INSN_LEN(w0), 1u);  // Insn_Len (Algorithm 2); the host verifier rejects 0
+
+      if ((op >= DVM_OP_BINI && op < DVM_OP_UN) || op >= DVM_OP_LD2) {
+        // ---- ACC = ACC op o : o an immediate, a local register (or ACC itself), or a per-row scalar;
+        //      LD2 first copies a local register into ACC ----
+        float2 o[VP];
+        if (op >= DVM_OP_LD2) {
+          const uint32_t lx = CW(lreg0 + ia), ly = CW(lreg0 + (ib & 0x3f));
+          read_lreg(A, buf ? (lx >> 16) : (lx & 0xffff), (ib >> 6) & 1);
+          read_lreg(o, buf ? (ly >> 16) : (ly & 0xffff), (ib >> 7) & 1);
+        } else if (op >= DVM_OP_BINS) {
+          const float y = sget(S, ia);
+          DVM_EACH_PAIR o[i] = make_float2(y, y);
+        } else if (op >= DVM_OP_BIN) {
+          if (ia == DVM_REG_ACC) {
+            DVM_EACH_PAIR o[i] = A[i];
+          } else {
+            const uint32_t lt = CW(lreg0 + ia);
+            read_lreg(o, buf ? (lt >> 16) : (lt & 0xffff), ib);
+          }
+        } else {
+          const float y = __uint_as_float(CW(body0 + pc - 1));
+          DVM_EACH_PAIR o[i] = make_float2(y, y);
+        }
+        switch (op & 7) {
+          case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], o[i]); break;
+          case DVM_A_SUB: DVM_EACH_PAIR A[i] = __ffma2_rn(o[i], make_float2(-1.f, -1.f), A[i]); break;
+          case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), o[i]); break;
+          case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], o[i]); break;
+          case DVM_A_DIV:
+            if ((op >= DVM_OP_BIN && op < DVM_OP_BINS) || op >= DVM_OP_LD2) {
+              DVM_EACH_PAIR A[i] = make_float2(A[i].x / o[i].x, A[i].y / o[i].y);
+            } else {
+              // division by a per-row scalar or an immediate: one correctly rounded reciprocal, packed multiplies
+              const float rcp = 1.0f / o[0].x;
+              DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], make_float2(rcp, rcp));
+            }
+            break;
+          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(o[i].x / A[i].x, o[i].y / A[i].y); break;
+          case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < o[i].x ? A[i].x : o[i].x, A[i].y < o[i].y ? A[i].y : o[i].y); break;
+          default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > o[i].x ? A[i].x : o[i].x, A[i].y > o[i].y ? A[i].y : o[i].y); break;
+        }
+        continue;
+      }
+      if (op >= DVM_OP_UN && op < DVM_OP_RED) {
+#define DVM_UN_CASE(U, EXPR)                                                          \
+  case U:                                                                             \
+    DVM_EACH_PAIR {                                                                   \
+      float x = A[i].x; const float vx = (EXPR);                                      \
+      x = A[i].y; const float vy = (EXPR);                                            \
+      A[i] = make_float2(vx, vy);                                                     \
+    }                                                                                 \
     break;
-          DVM_BIN_CASE(DVM_A_ADD, x + y)
-          DVM_BIN_CASE(DVM_A_SUB, x - y)
-          DVM_BIN_CASE(DVM_A_RSUB, y - x)
-          DVM_BIN_CASE(DVM_A_MUL, x * y)
-          DVM_BIN_CASE(DVM_A_DIV, x / y)
-          DVM_BIN_CASE(DVM_A_RDIV, y / x)
-          DVM_BIN_CASE(DVM_A_MIN, x < y ? x : y)
-          DVM_BIN_CASE(DVM_A_MAX, x > y ? x : y)
-#undef DVM_BIN_CASE
-        }
-      } else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) {
-        const float y = sget(S, ia);
-        switch (op - DVM_OP_BINS) {
-#define DVM_BINS_CASE(AR, EXPR)                                                                  \
-  case AR:                                                                                       \
-    _Pragma("unroll") for (int i = 0; i < V; ++i) { const float x = A[i]; A[i] = (EXPR); }       \
-    break;
-          DVM_BINS_CASE(DVM_A_ADD, x + y)
-          DVM_BINS_CASE(DVM_A_SUB, x - y)
-          DVM_BINS_CASE(DVM_A_RSUB, y - x)
-          DVM_BINS_CASE(DVM_A_MUL, x * y)
-          DVM_BINS_CASE(DVM_A_DIV, x / y)
-          DVM_BINS_CASE(DVM_A_RDIV, y / x)
-          DVM_BINS_CASE(DVM_A_MIN, x < y ? x : y)
-          DVM_BINS_CASE(DVM_A_MAX, x > y ? x : y)
-        }
-      } else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) {
-        const float y = __uint_as_float(body[pc + 1]);
-        switch (op - DVM_OP_BINI) {
-          DVM_BINS_CASE(DVM_A_ADD, x + y)
-          DVM_BINS_CASE(DVM_A_SUB, x - y)
-          DVM_BINS_CASE(DVM_A_RSUB, y - x)
-          DVM_BINS_CASE(DVM_A_MUL, x * y)
-          DVM_BINS_CASE(DVM_A_DIV, x / y)
-          DVM_BINS_CASE(DVM_A_RDIV, y / x)
-          DVM_BINS_CASE(DVM_A_MIN, x < y ? x : y)
-          DVM_BINS_CASE(DVM_A_MAX, x > y ? x : y)
-#undef DVM_BINS_CASE
-        }
-      } else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
         switch (op - DVM_OP_UN) {
-#define DVM_UN_CASE(U, EXPR)                                                                     \
-  case U:                                                                                        \
-    _Pragma("unroll") for (int i = 0; i < V; ++i) { const float x = A[i]; A[i] = (EXPR); }       \
-    break;
           DVM_UN_CASE(DVM_U_EXP, expf(x))
           DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
           DVM_UN_CASE(DVM_U_RSQRT, 1.0f / sqrtf(x))
@@ -484,150 +469,200 @@ dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
           DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
           DVM_UN_CASE(DVM_U_ROUND, rintf(x))
           DVM_UN_CASE(DVM_U_TANH, tanhf(x))
-          DVM_UN_CASE(DVM_U_RND_BF16, round_bf16(x))
+          default:
+            DVM_EACH_PAIR A[i] = make_float2(round_bf16(A[i].x), round_bf16(A[i].y));
+            break;
+        }
 #undef DVM_UN_CASE
-        }
-      } else if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) {
-        // row reduction: thread-local over valid slots, shuffles inside the warp, shared memory across
-        // the warps of a row group (Table 1, Sum / Max / Min with N = 1)
+        continue;
+      }
+      if (op >= DVM_OP_RED && op < DVM_OP_LD2) {
+        // ---- row reduction (Table 1, Sum / Max / Min with N = 1): thread-local over valid slots, shuffles
+        // inside the warp, shared memory across the warps of a row group ----
         const int rop = op - DVM_OP_RED;
-        const float ident = rop == DVM_R_SUM ? 0.f : (rop == DVM_R_MAX ? -INFINITY : INFINITY);
-        float v = ident;
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-          const float x = ((c.vmask >> i) & 1) ? A[i] : ident;
-          v = rop == DVM_R_SUM ? v + x : (rop == DVM_R_MAX ? (x > v ? x : v) : (x < v ? x : v));
-        }
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          if (o < G) {
-            const float x = __shfl_xor_sync(0xffffffffu, v, o);
-            v = rop == DVM_R_SUM ? v + x : (rop == DVM_R_MAX ? (x > v ? x : v) : (x < v ? x : v));
+        float v;
+        if (rop == DVM_R_SUM || rop == DVM_R_SUMSQ) {
+          float2 acc = make_float2(0.f, 0.f);
+          if (all_valid) {
+            if (rop == DVM_R_SUM) { DVM_EACH_PAIR acc = __fadd2_rn(acc, A[i]); }
+            else { DVM_EACH_PAIR acc = __ffma2_rn(A[i], A[i], acc); }
+          } else {
+            DVM_EACH_PAIR {
+              const float2 x = make_float2(((c.vmask >> (2 * i)) & 1) ? A[i].x : 0.f, ((c.vmask >> (2 * i + 1)) & 1) ? A[i].y : 0.f);
+              acc = rop == DVM_R_SUM ? __fadd2_rn(acc, x) : __ffma2_rn(x, x, acc);
+            }
           }
+          v = acc.x + acc.y;
+#pragma unroll
+          for (int sh = 1; sh < 32; sh <<= 1)
+            if (sh < G) v += __shfl_xor_sync(0xffffffffu, v, sh);
+        } else {
+          const bool mx = rop == DVM_R_MAX;
+          const float ident = mx ? -INFINITY : INFINITY;
+          v = ident;
+          DVM_EACH_PAIR {
+            const float x0 = ((c.vmask >> (2 * i)) & 1) ? A[i].x : ident;
+            const float x1 = ((c.vmask >> (2 * i + 1)) & 1) ? A[i].y : ident;
+            v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
+          }
+#pragma unroll
+          for (int sh = 1; sh < 32; sh <<= 1)
+            if (sh < G) {
+              const float x = __shfl_xor_sync(0xffffffffu, v, sh);
+              v = mx ? fmaxf(v, x) : fminf(v, x);
+            }
         }
         if (G > 32) {
           if (lane == 0) s_red[red_par][warp] = v;
           __syncthreads();
-          const int wpg = G >> 5;          // warps per row group
-          const int w0i = (warp / wpg) * wpg;
-          float acc = ident;
-          for (int i = 0; i < wpg; ++i) {
+          const int wpg = G >> 5;  // warps per row group
+          const int w0i = warp & ~(wpg - 1);
+          float acc = s_red[red_par][w0i];
+          for (int i = 1; i < wpg; ++i) {
             const float x = s_red[red_par][w0i + i];
-            acc = rop == DVM_R_SUM ? acc + x : (rop == DVM_R_MAX ? (x > acc ? x : acc) : (x < acc ? x : acc));
+            acc = rop == DVM_R_MAX ? fmaxf(acc, x) : (rop == DVM_R_MIN ? fminf(acc, x) : acc + x);
           }
           v = acc;
           red_par ^= 1;
         }
         sset(S, ia, v);
-      } else {
-        switch (op) {
-          case DVM_OP_NOP: break;
-          case DVM_OP_LDG: {
-            const OperandAddr oa = operand_addr(prog, opd_table, ib, c);
-            uint32_t slow = 0;
-            const int variant = (oa.dtype == DVM_DT_BF16 ? 1 : 0) | (c.W == 8 ? 2 : (c.W == 4 ? 4 : 0));
-            with_reg<NREG>(R, ia, [&](float (&r)[V]) {
-              switch (variant) {
-                case 0: ldg_fast<1, false>(r, oa.ptr, c, slow); break;
-                case 1: ldg_fast<1, true>(r, oa.ptr, c, slow); break;
-                case 2: ldg_fast<8, false>(r, oa.ptr, c, slow); break;
-                case 3: ldg_fast<8, true>(r, oa.ptr, c, slow); break;
-                case 4: ldg_fast<4, false>(r, oa.ptr, c, slow); break;
-                default: err = ST_BAD_CODE; break;
-              }
-            });
-            if (slow) {
-              float tmp[V];
-              switch (variant) {
-                case 2: ldg_slow<8, false>(tmp, oa.ptr, c, slow); break;
-                case 3: ldg_slow<8, true>(tmp, oa.ptr, c, slow); break;
-                default: ldg_slow<4, false>(tmp, oa.ptr, c, slow); break;
-              }
-              with_reg<NREG>(R, ia, [&](float (&r)[V]) {
-                switch (variant) {
-                  case 2: merge_slow<8, false>(r, tmp, slow); break;
-                  case 3: merge_slow<8, true>(r, tmp, slow); break;
-                  default: merge_slow<4, false>(r, tmp, slow); break;
-                }
-              });
-            }
-          } break;
-          case DVM_OP_CVT:
-            if (ib == DVM_DT_BF16) with_reg<NREG>(R, ia, [&](float (&r)[V]) { widen_bf16(r); });
-            break;
-          case DVM_OP_STG: {
-            const OperandAddr oa = operand_addr(prog, opd_table, ib, c);
-            const int variant = (oa.dtype == DVM_DT_BF16 ? 1 : 0) | (c.W == 8 ? 2 : (c.W == 4 ? 4 : 0));
-            switch (variant) {
-              case 0: stg_tile<1, false>(A, oa.ptr, c); break;
-              case 1: stg_tile<1, true>(A, oa.ptr, c); break;
-              case 2: stg_tile<8, false>(A, oa.ptr, c); break;
-              case 3: stg_tile<8, true>(A, oa.ptr, c); break;
-              case 4: stg_tile<4, false>(A, oa.ptr, c); break;
-              default: err = ST_BAD_CODE; break;
-            }
-          } break;
-          case DVM_OP_LDS: {
-            const OperandAddr oa = operand_addr(prog, opd_table, ib, c);
-            float v = 0.f;
-            if (c.ncols > 0) {
-              if (oa.dtype == DVM_DT_BF16) v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(oa.ptr));
-              else v = *reinterpret_cast<const float*>(oa.ptr);
-            }
-            sset(S, ia, v);
-          } break;
-          case DVM_OP_STS: {
-            const OperandAddr oa = operand_addr(prog, opd_table, ib, c);
-            const float v = sget(S, ia);
-            if (c.ncols > 0 && c.t == 0 && c.col0 == 0) {
-              if (oa.dtype == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(oa.ptr) = __float2bfloat16_rn(v);
-              else *reinterpret_cast<float*>(oa.ptr) = v;
-            }
-          } break;
-          case DVM_OP_MOV:
-            if (ia == 0) {
-              with_reg<NREG>(R, ib, [&](float (&r)[V]) {
-#pragma unroll
-                for (int i = 0; i < V; ++i) A[i] = r[i];
-              });
-            } else {
-              with_reg<NREG>(R, ia, [&](float (&r)[V]) {
-#pragma unroll
-                for (int i = 0; i < V; ++i) r[i] = A[i];
-              });
-            }
-            break;
-          case DVM_OP_BCS: {
-            const float v = sget(S, ia);
-#pragma unroll
-            for (int i = 0; i < V; ++i) A[i] = v;
-          } break;
-          case DVM_OP_SOP: {
-            const uint32_t w1 = body[pc + 1];
-            const int sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
-            const float x = sget(S, s1);
-            float rv;
-            if (ib == DVM_SK_BIN) rv = arith(sub, x, sget(S, s2));
-            else if (ib == DVM_SK_BINI) rv = arith(sub, x, __uint_as_float(body[pc + 2]));
-            else rv = unary(sub, x);
-            sset(S, ia, rv);
-          } break;
-          default:
-            err = ST_BAD_CODE;
-            break;
-        }
+        continue;
       }
-      pc += len ? len : 1;  // Insn_Len; the host verifier rejects len == 0, this only bounds the walk
+
+      switch (op) {
+        case DVM_OP_NOP: break;
+        case DVM_OP_LDA: {
+          const uint32_t lt = CW(lreg0 + ia);
+          read_lreg(A, buf ? (lt >> 16) : (lt & 0xffff), ib);
+        } break;
+        case DVM_OP_STA: {
+          const uint32_t a0 = lvec(CW(lreg0 + ia) & 0xffff, 0);
+#pragma unroll
+          for (int q = 0; q < V / 4; ++q)
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * (THREADS * 16)), "f"(A[2 * q].x), "f"(A[2 * q].y),
+                         "f"(A[2 * q + 1].x), "f"(A[2 * q + 1].y)
+                         : "memory");
+        } break;
+        case DVM_OP_LSS: {
+          const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
+          const uint32_t w = (uint32_t)buf * DVM_MAX_SSLOTS + (uint32_t)ib;
+          float v;
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lvec(unit, w >> 2) + (w & 3) * 4));
+          sset(S, ia, c.ncols > 0 ? v : 0.f);
+        } break;
+        case DVM_OP_STG: {
+          int dt;
+          char* p = operand_addr(prog, opd0, ib, c, dt);
+          const int es = dt == DVM_DT_BF16 ? 2 : 4;
+          char* q0 = p + (long long)((c.t << c.lgW) - c.shift) * es;
+          const long long qstep = (long long)(G << c.lgW) * es;
+          const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
+          const uint32_t fast = (al && W > 1) ? c.fullmask : 0u;
+          const uint32_t slow = c.partmask | (c.fullmask & ~fast);
+          const uint32_t st0 = lvec(staging_unit, 0);
+          if (dt == DVM_DT_BF16) {
+            uint32_t pk[VP];
+            DVM_EACH_PAIR {
+              const __nv_bfloat162 b = __floats2bfloat162_rn(A[i].x, A[i].y);
+              pk[i] = *reinterpret_cast<const uint32_t*>(&b);
+            }
+#pragma unroll
+            for (int j = 0; j < V / 8; ++j)
+              if ((fast >> j) & 1)
+                *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+            if (slow) {
+#pragma unroll
+              for (int q = 0; q < V / 8; ++q)
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(st0 + q * (THREADS * 16)), "r"(pk[4 * q]), "r"(pk[4 * q + 1]),
+                             "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3])
+                             : "memory");
+            }
+          } else {
+            if (W == 8) {
+#pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1) {
+                  *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y);
+                  *reinterpret_cast<float4*>(q0 + j * qstep + 16) = make_float4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y);
+                }
+            } else {
+#pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
+            }
+            if (slow) {
+#pragma unroll
+              for (int q = 0; q < V / 4; ++q)
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(st0 + q * (THREADS * 16)), "f"(A[2 * q].x), "f"(A[2 * q].y),
+                             "f"(A[2 * q + 1].x), "f"(A[2 * q + 1].y)
+                             : "memory");
+            }
+          }
+          if (slow) {
+            // scalar path: the narrowed tile sits in this thread's staging line
+#pragma unroll 1
+            for (int s = 0; s < V; ++s) {
+              if (!((slow >> (s >> c.lgW)) & 1) || !((c.vmask >> s) & 1)) continue;
+              const int col = slot_col(c, s);
+              const uint32_t b = (uint32_t)s * es;
+              const uint32_t src = lvec(staging_unit, b >> 4) + (b & 15);
+              if (dt == DVM_DT_BF16) {
+                unsigned short hv;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(hv) : "r"(src));
+                *reinterpret_cast<unsigned short*>(p + (long long)col * 2) = hv;
+              } else {
+                uint32_t wv;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(wv) : "r"(src));
+                *reinterpret_cast<uint32_t*>(p + (long long)col * 4) = wv;
+              }
+            }
+          }
+        } break;
+        case DVM_OP_STS: {
+          int dt;
+          char* p = operand_addr(prog, opd0, ib, c, dt);
+          const float v = sget(S, ia);
+          if (c.ncols > 0 && c.t == 0 && c.col0 == 0) {
+            if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
+            else *reinterpret_cast<float*>(p) = v;
+          }
+        } break;
+        case DVM_OP_BCS: {
+          const float v = sget(S, ia);
+          DVM_EACH_PAIR A[i] = make_float2(v, v);
+        } break;
+        case DVM_OP_SOP: {
+          const uint32_t w1 = CW(body0 + pc - (ib == DVM_SK_BINI ? 2 : (ib == DVM_SK_FMAU ? 3 : 1)));
+          const int sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
+          const float x = sget(S, s1);
+          float rv;
+          if (ib == DVM_SK_FMAU) {
+            // unary(x * m + a): multiply and add round separately, exactly like the unfused instructions
+            rv = __fadd_rn(__fmul_rn(x, __uint_as_float(CW(body0 + pc - 2))), __uint_as_float(CW(body0 + pc - 1)));
+            if (sub != 0xff) rv = scalar_unary(sub, rv);
+          } else if (ib == DVM_SK_UN) rv = scalar_unary(sub, x);
+          else rv = scalar_arith(sub, x, ib == DVM_SK_BIN ? sget(S, s2) : __uint_as_float(CW(body0 + pc - 1)));
+          sset(S, ia, rv);
+        } break;
+        default:
+          err = ST_BAD_CODE;
+          pc = body_words;  // stop walking code that cannot be decoded
+          break;
+      }
     }
 
-    ++iter;
-    if (prm.use_queue) {
-      __syncthreads();
-      tile = s_next[(iter - 1) & 1];
-    } else {
-      tile += gridDim.x;
+    // ---- advance to the next tile ----
+    if (have_next && !early) {
+      issue_loads(cn, buf ^ 1, true);
+      cp_async_commit();
     }
+    c = cn;
+    prog_idx = next_prog_idx;
+    tile = next;
+    buf ^= 1;
   }
+  cp_async_wait<0>();
 
   if (err && tid == 0) atomicMax(prm.status, err);
   if (prm.use_queue) {
@@ -643,6 +678,8 @@ dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
       }
     }
   }
+#undef DVM_EACH_PAIR
+#undef CW
 }
 
 }  // namespace dvm

@@ -1,0 +1,101 @@
+"""GPU parity of stacking-based fusion: many independent programs in one launch (config 4)."""
+import pytest
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from tests.parity_util import check, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True, params=[16, 32])
+def elems_per_thread(request):
+    """Programs of one stacked launch share the elements-per-thread setting; both settings are covered."""
+    dvm.set_elems_per_thread(request.param)
+    yield request.param
+    dvm.set_elems_per_thread(0)
+
+
+def _stack(items, seed0):
+    progs = {k: wl.stack_program(k) for k in wl.STACK_KINDS}
+    ps = {k: dvm.program_from_nodes(p.nodes) for k, p in progs.items()}
+    codes, tls, meta = [], [], []
+    for j, (kind, r, c) in enumerate(items):
+        ins, params = wl.inputs_stack(kind, r, c, seed0 + 4 * j)
+        dev = [t.cuda() for t in ins]
+        out = torch.full((r, c), float("nan"), dtype=torch.float32, device="cuda")
+        codes.append(dvm.encode(ps[kind], [tuple(t.shape) for t in ins], params))
+        tls.append(dev + [out])
+        meta.append((progs[kind], ins, params, out, kind))
+    return codes, tls, meta
+
+
+def _check_all(meta):
+    for prog, ins, params, out, kind in meta:
+        check(prog, [out], oracle_run(prog, ins, params), strict=(kind == "sigmoid_mul"))
+
+
+def test_stacked_small_mix():
+    items = [("gelu_affine", 3, 65), ("layernorm", 17, 100), ("sigmoid_mul", 1, 64), ("layernorm", 1, 4096),
+             ("gelu_affine", 200, 333), ("sigmoid_mul", 511, 4095), ("layernorm", 512, 64)]
+    codes, tls, meta = _stack(items, 100)
+    dvm.launch_stacked(codes, tls)
+    assert dvm.last_device_status() == 0
+    _check_all(meta)
+
+
+def test_stacked_config4_first_launch():
+    """The first seeded launch of config 4: 64 programs, one kernel."""
+    items = wl.shapes_c4(1)[0]
+    assert len(items) == 64
+    codes, tls, meta = _stack(items, wl.data_seed("c4", 0))
+    n0 = dvm.launch_count()
+    dvm.launch_stacked(codes, tls)
+    assert dvm.last_device_status() == 0
+    assert dvm.launch_count() - n0 == 1
+    _check_all(meta)
+
+
+def test_stacked_repeated_launches_reuse_queue():
+    """The work queue returns to its resting state after every launch."""
+    items = wl.shapes_c4(2)[1][:16]
+    codes, tls, meta = _stack(items, 999)
+    for _ in range(5):
+        for t in tls:
+            t[-1].fill_(float("nan"))
+        dvm.launch_stacked(codes, tls)
+        assert dvm.last_device_status() == 0
+        _check_all(meta)
+
+
+def test_stacked_rejects_mixed_settings():
+    dvm.set_elems_per_thread(16)
+    c1, t1, _ = _stack([("sigmoid_mul", 5, 70)], 5)
+    dvm.set_elems_per_thread(32)
+    c2, t2, _ = _stack([("sigmoid_mul", 5, 70)], 6)
+    with pytest.raises(dvm.DvmError) as e:
+        dvm.launch_stacked(c1 + c2, t1 + t2)
+    assert e.value.status == -1
+
+
+def test_stacked_one_and_empty():
+    codes, tls, meta = _stack([("sigmoid_mul", 5, 70)], 5)
+    dvm.launch_stacked(codes, tls)
+    assert dvm.last_device_status() == 0
+    _check_all(meta)
+    dvm.launch_stacked([], [])
+
+
+def test_stacked_equals_separate_launches():
+    items = wl.shapes_c4(3)[2][:12]
+    codes, tls, meta = _stack(items, 31337)
+    dvm.launch_stacked(codes, tls)
+    torch.cuda.synchronize()
+    stacked = [t[-1].clone() for t in tls]
+    for c, t in zip(codes, tls):
+        t[-1].fill_(float("nan"))
+        dvm.launch(c, t)
+    torch.cuda.synchronize()
+    for a, t in zip(stacked, tls):
+        assert torch.equal(a, t[-1])

@@ -1,0 +1,180 @@
+"""Host logic on CPU: the C-ABI library loads and exports every declared symbol, the paper's
+tiling example and tile partition, encoder geometry, verifier and dump."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from paper_2603_24239_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "dvm.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(dvm_[a-z0-9_]+)\s*\(", hdr))
+    assert len(declared) >= 25
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"libdvm.so does not export {name}"
+    assert declared == set(binding.EXPORTS), declared ^ set(binding.EXPORTS)
+
+
+def test_paper_tiling_example():
+    """Sec. 4.2 worked example: fp16 [32,1024] add, 40 cores, 32-byte instruction width."""
+    row = [l for l in open(os.path.join(ROOT, "tests", "golden", "paper_tiling_example.txt"))
+           if not l.startswith("#")][0].split()
+    total, cores, align_b, esize, want_t, want_n, want_tail, want_r = map(int, row)
+    r = dvm.hardware_align_div(total, cores, align_b // esize, 1 << 20, 2)
+    assert r == {"min_cost_tile": want_t, "rounded_tile": want_r, "n_tiles": want_n, "tail": want_tail}
+    # the minimum is unique: brute force over every tile size
+    costs = {t: -(-(-(-total // t)) // cores) * (t + 2) for t in range(1, total + 1)}
+    best = min(costs.values())
+    assert [t for t, c in costs.items() if c == best] == [want_t]
+    # rounding never exceeds the tile size limit
+    r = dvm.hardware_align_div(total, cores, 16, 825, 2)
+    assert r["rounded_tile"] <= 825
+
+
+@pytest.mark.parametrize("M,N", [(41, 40), (40, 40), (1, 40), (0, 7), (1000, 148), (7, 444)])
+def test_vm_tile_partition_is_exact_cover(M, N):
+    """Algorithm 2: core id runs [m*id, min(M, m*(id+1))), m = ceil(M/N)."""
+    seen = []
+    busy = 0
+    for i in range(N):
+        b, e = dvm.vm_tile_range(M, N, i)
+        seen += list(range(b, e))
+        busy += e > b
+    assert seen == list(range(M))
+    if (M, N) == (41, 40):
+        assert busy == 21 and dvm.vm_tile_range(M, N, 20) == (40, 41)
+
+
+def _enc(prog, shapes, params=()):
+    return dvm.encode(dvm.program_from_nodes(prog.nodes), shapes, params)
+
+
+def test_encode_geometry_and_shapes():
+    c = _enc(wl.program_add_rmsnorm(), [(1000, 4096), (1000, 4096), (4096,)])
+    assert c.out_shapes == [(1000, 4096), (1000, 4096)]
+    info = dvm.code_info(c)
+    # 4096 columns: 128 threads x 32 elements (two rows per tile) or 256 x 16 (one row per tile)
+    assert info["threads_per_row"] in (128, 256) and info["vector_width"] == 8
+    assert info["n_tiles"] == 1000 * info["threads_per_row"] // 256
+    assert info["kernel_type"] == 1 and info["n_tile_regs"] == 3   # three inputs in local registers, no temporaries
+    c = _enc(wl.program_masked_softmax(), [(2, 32, 100, 100), (1, 1, 100, 100)])
+    assert c.out_shapes == [(2, 32, 100, 100)]
+    info = dvm.code_info(c)
+    assert info["threads_per_row"] * 32 >= 100                # rows of 100 bf16 start on 8-byte boundaries only
+    assert info["n_tiles"] == -(-6400 // (256 // info["threads_per_row"]))
+    # pure elementwise program collapses to a flat range
+    c = _enc(wl.program_c1(), [(7, 1531)] * 3)
+    d = dvm.disassemble(c)
+    assert "flags=A-F" in d and "exp" in d and "block_dim=" in d and "body_tile=" in d
+    # zero-size instance
+    c = _enc(wl.program_c1(), [(0, 5)] * 3)
+    assert dvm.code_info(c)["n_tiles"] == 0 and c.out_shapes == [(0, 5)]
+
+
+def test_encode_is_shape_dependent_and_deterministic():
+    p = dvm.program_from_nodes(wl.program_layernorm().nodes)
+    a = dvm.encode(p, [(10, 100)], (0.01,)).bytes()
+    b = dvm.encode(p, [(10, 100)], (0.01,)).bytes()
+    c = dvm.encode(p, [(11, 100)], (0.01,)).bytes()
+    assert a == b and a != c
+
+
+def test_encode_errors():
+    p = dvm.program_from_nodes(wl.program_c1().nodes)
+    with pytest.raises(dvm.DvmError) as e:
+        dvm.encode(p, [(7, 5), (7, 6), (7, 5)])
+    assert e.value.status == -2
+    with pytest.raises(dvm.DvmError) as e:
+        dvm.encode(p, [(7, 5), (7, 5)])
+    assert e.value.status == -1
+    # a reduced row longer than the register budget
+    q = dvm.program_from_nodes(wl.program_layernorm().nodes)
+    with pytest.raises(dvm.DvmError) as e:
+        dvm.encode(q, [(4, 9000)], (1 / 9000,))
+    assert e.value.status == -3
+    # missing runtime scalar
+    with pytest.raises(dvm.DvmError):
+        dvm.encode(q, [(4, 50)], ())
+    # unfinalized program
+    r = dvm.Program(); r.input("f32", 1)
+    with pytest.raises(dvm.DvmError):
+        dvm.encode(r, [(4,)])
+
+
+def test_buffer_too_small_reports_need():
+    import ctypes as C
+    p = dvm.program_from_nodes(wl.program_c1().nodes)
+    enc = binding.Encoder(p)
+    need = enc.encode([(7, 1531)] * 3)
+    small = (C.c_uint64 * 4)()
+    size = C.c_size_t(0)
+    st = binding.lib.dvm_encode(p._h, enc.shapes, 3, enc.scalars, 0, small, 32, C.byref(size), None, 0)
+    assert st == -4 and size.value == need
+
+
+def test_verify_rejects_malformed_code():
+    c = _enc(wl.program_masked_softmax(), [(1, 2, 40, 40), (1, 1, 40, 40)])
+    good = bytearray(c.bytes())
+    assert dvm.verify(bytes(good)) == 0
+    import random
+    rnd = random.Random(7)
+    rejected = 0
+    for _ in range(400):
+        bad = bytearray(good)
+        k = rnd.randrange(len(bad))
+        bad[k] ^= 1 << rnd.randrange(8)
+        st = dvm.verify(bytes(bad))
+        assert st in (0, -5)
+        rejected += st == -5
+    assert rejected > 100           # most single-bit flips are caught; the rest are value changes
+    assert dvm.verify(bytes(good[:-4])) == -5
+    assert dvm.verify(b"\0" * 80) == -5
+    bad = bytearray(good); bad[-4] = 0xEE     # unknown instruction id in the last word
+    assert dvm.verify(bytes(bad)) == -5
+
+
+def test_local_register_pressure():
+    p = wl.OpProgram("wide")
+    ins = [p.input("f32", 2) for _ in range(6)]
+    acc = p.binary("mul", ins[0], ins[1])
+    for i in range(2, 6):
+        acc = p.binary("add", acc, ins[i])
+    for i in range(6):                     # every input is used again at the end
+        acc = p.binary("mul", acc, ins[i])
+    p.output(acc, "f32")
+    c = _enc(p, [(3, 50)] * 6)
+    assert dvm.code_info(c)["n_tile_regs"] == 6          # inputs stay in their local registers, no spill
+    q = wl.OpProgram("too_wide")
+    ins = [q.input("f32", 2) for _ in range(10)]
+    acc = q.binary("mul", ins[0], ins[1])
+    for i in range(2, 10):
+        acc = q.binary("add", acc, ins[i])
+    for i in range(10):
+        acc = q.binary("mul", acc, ins[i])
+    q.output(acc, "f32")
+    with pytest.raises(dvm.DvmError) as e:
+        _enc(q, [(3, 50)] * 10)
+    assert e.value.status == -3
+
+
+def test_encode_latency_budget():
+    """Host encode stays far below the 50 us budget even on this CPU machine (median over many calls)."""
+    import time
+    p = dvm.program_from_nodes(wl.program_add_rmsnorm().nodes)
+    enc = binding.Encoder(p)
+    ts = []
+    for i in range(2000):
+        t0 = time.perf_counter_ns()
+        enc.encode(((1000 + i, 4096), (1000 + i, 4096), (4096,)))
+        ts.append(time.perf_counter_ns() - t0)
+    ts.sort()
+    assert ts[len(ts) // 2] < 50_000
