@@ -299,7 +299,7 @@ class C4Workload:
 
     def __init__(self, dvm, n_launches=50, device="cuda"):
         self.dvm = dvm
-        dvm.set_elems_per_thread(32)   # programs of one stacked launch share the setting
+        dvm.set_elems_per_thread(16)   # programs of one stacked launch share the setting; 16 fits every program
         self.launches = wl.shapes_c4(n_launches)
         self.progs = {k: wl.stack_program(k) for k in wl.STACK_KINDS}
         self.ps = {k: dvm.program_from_nodes(p.nodes) for k, p in self.progs.items()}

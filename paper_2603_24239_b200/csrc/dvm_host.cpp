@@ -902,7 +902,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
         for (int pass = 0; pass < 2 && g.cost < 0; ++pass) {
           const int w = pass == 0 ? W0 : 1;  // second pass: element-wise mapping, which needs no padding
           const bool al = pass == 0 ? aligned : true;
-          const int64_t pad = al ? 0 : w - 1;
+          const int64_t pad = 0;  // a misaligned row wraps its last columns into the unused head slots: no padding
           for (int lg = 0; lg <= 8; ++lg) {
             int64_t G = 1 << lg, cap = G * g.V;
             int64_t ct;
@@ -1043,6 +1043,9 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   memcpy(lt + nreg + e.n_loads, e.body, (size_t)e.n_body * 4);
   if (C > 0xffffffffll || outer[0] > 0xffffffffll || outer[1] > 0xffffffffll || outer[2] > 0xffffffffll)
     return DVM_ERR_TOO_LARGE;
+  for (int o = 0; o < e.n_opd; ++o)
+    for (int q = 0; q < 3; ++q)
+      if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
   return DVM_OK;
 }
 
@@ -1103,7 +1106,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   uint64_t ctile = w[DVM_H_COL_TILE], cb = w[DVM_H_COL_BLOCKS], C = w[DVM_H_COLS];
   uint64_t R = (uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32);
   uint32_t flags = geom >> 24;
-  uint64_t pad = (flags & DVM_F_ALIGNED) ? 0 : W - 1;
+  uint64_t pad = 0;
   if (w[DVM_H_N_TILES] > 0) {
     if (ctile == 0 || cb == 0 || ctile + pad > G * Vv) return DVM_ERR_BAD_CODE;
     if (cb * ctile < C || (cb - 1) * ctile >= C) return DVM_ERR_BAD_CODE;
@@ -1119,6 +1122,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if ((info & 0xff) >= n_tensors) return DVM_ERR_BAD_CODE;
     if (((info >> 8) & 0xff) > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
     if (((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
+    if (ot[o * DVM_OPD_WORDS + 3] | ot[o * DVM_OPD_WORDS + 5] | ot[o * DVM_OPD_WORDS + 7]) return DVM_ERR_BAD_CODE;  // 32-bit strides
     n_primary += (info >> 24) & 1;
   }
   if (n_primary > 1) return DVM_ERR_BAD_CODE;

@@ -86,6 +86,29 @@ __device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) 
 
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
+// exp(x) = 2^(x * log2 e) with the product carried in two fp32 pieces (t exact to 2^-24 |t|, plus the
+// rounding residual of the multiply and the low part of log2 e), the power of two from the SFU
+// (ex2.approx, relative error <= 2^-22) and a first-order correction: about 3e-7 relative error over the
+// whole finite range, in 6 instructions instead of expf's ~12.
+__device__ __forceinline__ float fast_exp(float x) {
+  const float L2E_HI = 1.44269502162933349609375f, L2E_LO = 1.925963033500011e-8f;
+  const float t = x * L2E_HI;
+  float r = __fmaf_rn(x, L2E_HI, -t);
+  r = __fmaf_rn(x, L2E_LO, r);
+  float p;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(t));
+  // outside the finite range (t = +-inf from a masked score, overflow, NaN) the SFU value stands alone:
+  // exp(-inf) must be exactly +0
+  return fabsf(t) < 126.0f ? __fmaf_rn(p * r, 0.693147182464599609375f, p) : p;
+}
+// reciprocal and quotient from the SFU (rcp.approx, 1 ulp) : 2 ulp quotients
+__device__ __forceinline__ float fast_rcp(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float fast_div(float a, float b) { return __fdividef(a, b); }
+
 __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
   switch (op) {
     case DVM_A_ADD: return a + b;
@@ -120,6 +143,10 @@ __device__ __forceinline__ float scalar_unary(int op, float x) {
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+// 16-byte copy when `on`, otherwise nothing is read (source size 0) and the destination is zero-filled
+__device__ __forceinline__ void cp_async16_if(uint32_t dst, const void* src, bool on) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(on ? 16 : 0) : "memory");
+}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -127,9 +154,13 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Column (relative to the column block) of slot s.
-__device__ __forceinline__ int slot_col(const TileCtx& c, int s) {
-  return ((c.t + ((s >> c.lgW) << c.lgG)) << c.lgW) + (s & ((1 << c.lgW) - 1)) - c.shift;
+// Column (relative to the column block) of slot s of a V-slot register.  With a misaligned row segment
+// (shift > 0) the first `shift` slots of the row group's first chunk would fall before the segment; they
+// hold the segment's last columns instead (wrap-around by the row group's capacity G*V), so a row needs
+// no more slots than it has columns.
+__device__ __forceinline__ int slot_col(const TileCtx& c, int s, int V) {
+  const int col = ((c.t + ((s >> c.lgW) << c.lgG)) << c.lgW) + (s & ((1 << c.lgW) - 1)) - c.shift;
+  return col < 0 ? col + (V << c.lgG) : col;
 }
 
 template <int V, int PW>
@@ -160,11 +191,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t tp = prog + DVM_HDR_WORDS + 2 * (info & 0xff);
     const unsigned long long base = (unsigned long long)CW(tp) | ((unsigned long long)CW(tp + 1) << 32);
     dtype = (info >> 8) & 0xff;
-    unsigned long long off =
-        (unsigned long long)c.i0 * ((unsigned long long)CW(d + DVM_OPD_STRIDE0) | ((unsigned long long)CW(d + DVM_OPD_STRIDE0 + 1) << 32));
+    // strides are below 2^32 elements (the host rejects larger ones): 32 x 32 -> 64-bit products
+    unsigned long long off = (unsigned long long)c.i0 * CW(d + DVM_OPD_STRIDE0);
     if (c.flags & DVM_F_OUTER_DIMS) {
-      off += (unsigned long long)c.i1 * ((unsigned long long)CW(d + DVM_OPD_STRIDE1) | ((unsigned long long)CW(d + DVM_OPD_STRIDE1 + 1) << 32));
-      off += (unsigned long long)c.i2 * ((unsigned long long)CW(d + DVM_OPD_STRIDE2) | ((unsigned long long)CW(d + DVM_OPD_STRIDE2 + 1) << 32));
+      off += (unsigned long long)c.i1 * CW(d + DVM_OPD_STRIDE1);
+      off += (unsigned long long)c.i2 * CW(d + DVM_OPD_STRIDE2);
     }
     if ((info >> 16) & 0xff) off += c.col0;
     return reinterpret_cast<char*>(base + (off << (dtype == DVM_DT_BF16 ? 1 : 2)));
@@ -236,8 +267,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       if (part) {
 #pragma unroll 1
         for (int s = 0; s < V; ++s) {
-          const int col = slot_col(c, s);
-          if (((part >> (s >> c.lgW)) & 1) && col >= 0 && col < c.ncols) vm |= 1u << s;
+          const int col = slot_col(c, s, V);
+          if (((part >> (s >> c.lgW)) & 1) && col < c.ncols) vm |= 1u << s;
         }
       }
     } else {
@@ -270,32 +301,106 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         const int es = dt == DVM_DT_BF16 ? 2 : 4;
         const char* q0 = p + (long long)((c.t << c.lgW) - c.shift) * es;
         const long long qstep = (long long)(G << c.lgW) * es;
-        const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
-        const uint32_t fast = (al && W > 1) ? c.fullmask : 0u;
-        const uint32_t slow = c.partmask | (c.fullmask & ~fast);
-        const int vpc = (W * es) >> 4;  // 16-byte vectors per chunk (1 or 2); W = 1 never takes this path
-        if (fast) {
-#pragma unroll
-          for (int j = 0; j < V / 4; ++j) {
-            if ((fast >> j) & 1) {
-              cp_async16(lvec(unit, j * vpc), q0 + j * qstep);
-              if (vpc == 2) cp_async16(lvec(unit, j * vpc + 1), q0 + j * qstep + 16);
-            }
-          }
-        }
-        if (slow) {
-          // scalar path: element by element into the same local register (raw element bits)
+        const uint32_t d0 = lvec(unit, 0);
+        if (W == 1) {
+          // element-wise mapping: every valid slot is one scalar copy
 #pragma unroll 1
-          for (int s = 0; s < V; ++s) {
-            if (!((slow >> (s >> c.lgW)) & 1) || !((c.vmask >> s) & 1)) continue;
-            const int col = slot_col(c, s);
-            const uint32_t b = (uint32_t)s * es;
-            const uint32_t dst = lvec(unit, b >> 4) + (b & 15);
+          for (int sl = 0; sl < V; ++sl) {
+            if (!((c.vmask >> sl) & 1)) continue;
+            const int col = c.t + (sl << c.lgG);
+            const uint32_t b = (uint32_t)sl * es;
+            const uint32_t dst = d0 + (b >> 4) * (THREADS * 16) + (b & 15);
             if (dt == DVM_DT_BF16) {
               const unsigned short hv = *reinterpret_cast<const unsigned short*>(p + (long long)col * 2);
               asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst), "h"(hv) : "memory");
             } else {
               cp_async4(dst, p + (long long)col * 4);
+            }
+          }
+          continue;
+        }
+        const uint32_t mis = (uint32_t)(reinterpret_cast<uintptr_t>(q0) & 15);
+        const uint32_t fast = mis ? 0u : c.fullmask;
+        const uint32_t rea = mis ? c.fullmask : 0u;  // whole chunks at a misaligned address
+        const int vpc = (W * es) >> 4;               // 16-byte vectors per chunk (1 or 2)
+        if (fast && !c.partmask) {
+          // every chunk of this thread is whole and aligned, or empty: one (bf16, fp32 W = 4) or two (fp32 W = 8)
+          // 16-byte copies per chunk, switched off through the copy's source size (an empty chunk is zero-filled),
+          // so that the chunk loop has no branches
+          if (es == 2) {
+#pragma unroll
+            for (int j = 0; j < V / 8; ++j) cp_async16_if(d0 + j * (THREADS * 16), q0 + j * qstep, (fast >> j) & 1);
+          } else if (W == 8) {
+#pragma unroll
+            for (int j = 0; j < V / 8; ++j) {
+              cp_async16_if(d0 + (2 * j) * (THREADS * 16), q0 + j * qstep, (fast >> j) & 1);
+              cp_async16_if(d0 + (2 * j + 1) * (THREADS * 16), q0 + j * qstep + 16, (fast >> j) & 1);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < V / 4; ++j) cp_async16_if(d0 + j * (THREADS * 16), q0 + j * qstep, (fast >> j) & 1);
+          }
+        } else if (fast) {
+          // a chunk of this thread takes the scalar path below: copy only the whole ones (no zero fill may race with it)
+#pragma unroll 1
+          for (uint32_t m = fast; m; m &= m - 1) {
+            const int j = __ffs(m) - 1;
+            cp_async16(d0 + (j * vpc) * (THREADS * 16), q0 + j * qstep);
+            if (vpc == 2) cp_async16(d0 + (j * vpc + 1) * (THREADS * 16), q0 + j * qstep + 16);
+          }
+        }
+        if (rea) {
+          // the operand's rows are aligned differently from the tile mapping: fetch the two aligned 16-byte
+          // words that cover each vector and realign them in registers (word select + byte permute)
+          const char* qa = q0 - mis;
+          const uint32_t woff = mis >> 2, sel = (mis & 2) ? 0x5432u : 0x3210u;
+#pragma unroll 1
+          for (uint32_t m = rea; m; m &= m - 1) {
+            const int j = __ffs(m) - 1;
+            for (int v = 0; v < vpc; ++v) {
+              const uint4 a = *reinterpret_cast<const uint4*>(qa + j * qstep + 16 * v);
+              const uint4 bq = *reinterpret_cast<const uint4*>(qa + j * qstep + 16 * v + 16);
+              uint32_t t0 = a.x, t1 = a.y, t2 = a.z, t3 = a.w, t4 = bq.x, t5 = bq.y;
+              if (woff & 2) { t0 = a.z; t1 = a.w; t2 = bq.x; t3 = bq.y; t4 = bq.z; t5 = bq.w; }
+              if (woff & 1) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = t5; }
+              const uint32_t o0 = __byte_perm(t0, t1, sel), o1 = __byte_perm(t1, t2, sel), o2 = __byte_perm(t2, t3, sel),
+                             o3 = __byte_perm(t3, t4, sel);
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + (j * vpc + v) * (THREADS * 16)), "r"(o0), "r"(o1),
+                           "r"(o2), "r"(o3)
+                           : "memory");
+            }
+          }
+        }
+        if (c.partmask) {
+          // chunks cut by the row segment's head or tail: predicated element loads, one vector store
+#pragma unroll 1
+          for (uint32_t m = c.partmask; m; m &= m - 1) {
+            const int j = __ffs(m) - 1;
+            const int cc = ((c.t + (j << c.lgG)) << c.lgW) - c.shift;
+            if (es == 2) {
+              uint32_t h[8];
+#pragma unroll
+              for (int el = 0; el < 8; ++el) {
+                int col = cc + el;
+                col = col < 0 ? col + (V << c.lgG) : col;
+                h[el] = col < c.ncols ? (uint32_t)*reinterpret_cast<const unsigned short*>(p + (long long)col * 2) : 0u;
+              }
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + j * (THREADS * 16)), "r"(h[0] | (h[1] << 16)),
+                           "r"(h[2] | (h[3] << 16)), "r"(h[4] | (h[5] << 16)), "r"(h[6] | (h[7] << 16))
+                           : "memory");
+            } else {
+              for (int v = 0; v < vpc; ++v) {
+                uint32_t h[4];
+#pragma unroll
+                for (int el = 0; el < 4; ++el) {
+                  int col = cc + 4 * v + el;
+                  col = col < 0 ? col + (V << c.lgG) : col;
+                  h[el] = col < c.ncols ? *reinterpret_cast<const uint32_t*>(p + (long long)col * 4) : 0u;
+                }
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + (j * vpc + v) * (THREADS * 16)), "r"(h[0]), "r"(h[1]),
+                             "r"(h[2]), "r"(h[3])
+                             : "memory");
+              }
             }
           }
         }
@@ -434,14 +539,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], o[i]); break;
           case DVM_A_DIV:
             if ((op >= DVM_OP_BIN && op < DVM_OP_BINS) || op >= DVM_OP_LD2) {
-              DVM_EACH_PAIR A[i] = make_float2(A[i].x / o[i].x, A[i].y / o[i].y);
+              DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, o[i].x), fast_div(A[i].y, o[i].y));
             } else {
               // division by a per-row scalar or an immediate: one correctly rounded reciprocal, packed multiplies
               const float rcp = 1.0f / o[0].x;
               DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], make_float2(rcp, rcp));
             }
             break;
-          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(o[i].x / A[i].x, o[i].y / A[i].y); break;
+          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(o[i].x, A[i].x), fast_div(o[i].y, A[i].y)); break;
           case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < o[i].x ? A[i].x : o[i].x, A[i].y < o[i].y ? A[i].y : o[i].y); break;
           default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > o[i].x ? A[i].x : o[i].x, A[i].y > o[i].y ? A[i].y : o[i].y); break;
         }
@@ -457,15 +562,15 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     }                                                                                 \
     break;
         switch (op - DVM_OP_UN) {
-          DVM_UN_CASE(DVM_U_EXP, expf(x))
+          DVM_UN_CASE(DVM_U_EXP, fast_exp(x))
           DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
-          DVM_UN_CASE(DVM_U_RSQRT, 1.0f / sqrtf(x))
+          DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
           DVM_UN_CASE(DVM_U_ABS, fabsf(x))
           DVM_UN_CASE(DVM_U_LOG, logf(x))
           DVM_UN_CASE(DVM_U_ERF, erff(x))
-          DVM_UN_CASE(DVM_U_SIGMOID, 1.0f / (1.0f + expf(-x)))
+          DVM_UN_CASE(DVM_U_SIGMOID, fast_rcp(1.0f + fast_exp(-x)))
           DVM_UN_CASE(DVM_U_NEG, -x)
-          DVM_UN_CASE(DVM_U_RECIP, 1.0f / x)
+          DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
           DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
           DVM_UN_CASE(DVM_U_ROUND, rintf(x))
           DVM_UN_CASE(DVM_U_TANH, tanhf(x))
@@ -500,10 +605,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           const bool mx = rop == DVM_R_MAX;
           const float ident = mx ? -INFINITY : INFINITY;
           v = ident;
-          DVM_EACH_PAIR {
-            const float x0 = ((c.vmask >> (2 * i)) & 1) ? A[i].x : ident;
-            const float x1 = ((c.vmask >> (2 * i + 1)) & 1) ? A[i].y : ident;
-            v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
+          if (all_valid) {
+            DVM_EACH_PAIR v = mx ? fmaxf(v, fmaxf(A[i].x, A[i].y)) : fminf(v, fminf(A[i].x, A[i].y));
+          } else {
+            DVM_EACH_PAIR {
+              const float x0 = ((c.vmask >> (2 * i)) & 1) ? A[i].x : ident;
+              const float x1 = ((c.vmask >> (2 * i + 1)) & 1) ? A[i].y : ident;
+              v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
+            }
           }
 #pragma unroll
           for (int sh = 1; sh < 32; sh <<= 1)
@@ -604,7 +713,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 #pragma unroll 1
             for (int s = 0; s < V; ++s) {
               if (!((slow >> (s >> c.lgW)) & 1) || !((c.vmask >> s) & 1)) continue;
-              const int col = slot_col(c, s);
+              const int col = slot_col(c, s, V);
               const uint32_t b = (uint32_t)s * es;
               const uint32_t src = lvec(staging_unit, b >> 4) + (b & 15);
               if (dt == DVM_DT_BF16) {
