@@ -45,8 +45,9 @@ long long g_launches = 0;
 template <int V, int PW>
 int occupancy(int* out, size_t smem) {
   int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW>, dvm::THREADS, smem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false>, dvm::THREADS, smem));
   *out = n > 0 ? n : 1;
   return DVM_OK;
 }
@@ -130,8 +131,14 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
 
 template <int PW>
 int launch_variant(int V, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
-  if (V == 32) dvm::dvm_vm_kernel<32, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
-  else dvm::dvm_vm_kernel<16, PW><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  const bool single = prm.n_programs == 1 && !prm.use_queue;
+  if (V == 32) {
+    if (single) dvm::dvm_vm_kernel<32, PW, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<32, PW, false><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  } else {
+    if (single) dvm::dvm_vm_kernel<16, PW, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<16, PW, false><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  }
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;

@@ -86,6 +86,7 @@ __device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) 
 
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
+
 // exp(x) = 2^(x * log2 e) with the product carried in two fp32 pieces (t exact to 2^-24 |t|, plus the
 // rounding residual of the multiply and the low part of log2 e), the power of two from the SFU
 // (ex2.approx, relative error <= 2^-22) and a first-order correction: about 3e-7 relative error over the
@@ -115,8 +116,8 @@ __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
     case DVM_A_SUB: return a - b;
     case DVM_A_RSUB: return b - a;
     case DVM_A_MUL: return a * b;
-    case DVM_A_DIV: return a / b;
-    case DVM_A_RDIV: return b / a;
+    case DVM_A_DIV: return fast_div(a, b);
+    case DVM_A_RDIV: return fast_div(b, a);
     case DVM_A_MIN: return a < b ? a : b;
     default: return a > b ? a : b;
   }
@@ -124,15 +125,15 @@ __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
 
 __device__ __forceinline__ float scalar_unary(int op, float x) {
   switch (op) {
-    case DVM_U_EXP: return expf(x);
+    case DVM_U_EXP: return fast_exp(x);
     case DVM_U_SQRT: return sqrtf(x);
-    case DVM_U_RSQRT: return 1.0f / sqrtf(x);
+    case DVM_U_RSQRT: return rsqrtf(x);
     case DVM_U_ABS: return fabsf(x);
     case DVM_U_LOG: return logf(x);
     case DVM_U_ERF: return erff(x);
-    case DVM_U_SIGMOID: return 1.0f / (1.0f + expf(-x));
+    case DVM_U_SIGMOID: return fast_rcp(1.0f + fast_exp(-x));
     case DVM_U_NEG: return -x;
-    case DVM_U_RECIP: return 1.0f / x;
+    case DVM_U_RECIP: return fast_rcp(x);
     case DVM_U_FLOOR: return floorf(x);
     case DVM_U_ROUND: return rintf(x);
     case DVM_U_TANH: return tanhf(x);
@@ -163,8 +164,11 @@ __device__ __forceinline__ int slot_col(const TileCtx& c, int s, int V) {
   return col < 0 ? col + (V << c.lgG) : col;
 }
 
-template <int V, int PW>
+// SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
+// constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
+template <int V, int PW, bool SINGLE>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
+  constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;  // float2 pairs per tile register
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ float s_red[2][THREADS / 32];
@@ -173,7 +177,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const uint32_t local_base = static_cast<uint32_t>(__cvta_generic_to_shared(s_dyn)) + (uint32_t)tid * 16;
-  const uint32_t n_prog = prm.n_programs;
+  const uint32_t n_prog = SINGLE ? 1u : prm.n_programs;
+  const bool use_queue = SINGLE ? false : prm.use_queue != 0;
 #define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
 
   // shared-memory address of 16-byte vector q of the register at unit offset U (this thread's part)
@@ -284,7 +289,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
   // ---- load section of one tile: asynchronous copies into the input registers of buffer `buf` ----
   auto issue_loads = [&](const TileCtx& c, int buf, bool first_of_program) {
-    const uint32_t prog = c.prog;
+    const uint32_t prog = SINGLE ? kSingleProg : c.prog;
     const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
     const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
     const int W = 1 << c.lgW;
@@ -462,8 +467,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
   TileCtx c;
   if (tile < prm.total_tiles) {
-    while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
-    make_ctx(c, CW(prog_idx), tile - CW(n_prog + prog_idx));
+    if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
+    make_ctx(c, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
     issue_loads(c, buf, true);
     cp_async_commit();
   }
@@ -471,7 +476,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   while (tile < prm.total_tiles) {
     // ---- Algorithm 2, outer loop: next tile of this core; its loads start now when it runs the same program ----
     uint32_t next;
-    if (prm.use_queue) {
+    if (use_queue) {
       if (tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
       __syncthreads();
       next = s_next[iter & 1];
@@ -484,9 +489,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     bool early = false;
     uint32_t next_prog_idx = prog_idx;
     if (have_next) {
-      while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
+      if (!SINGLE) while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
       early = next_prog_idx == prog_idx;  // another program has another local-memory layout: load it after this tile
-      make_ctx(cn, CW(next_prog_idx), next - CW(n_prog + next_prog_idx));
+      make_ctx(cn, SINGLE ? kSingleProg : CW(next_prog_idx), SINGLE ? next : next - CW(n_prog + next_prog_idx));
       if (early) {
         issue_loads(cn, buf ^ 1, false);
         cp_async_commit();
@@ -494,7 +499,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     }
     if (early) cp_async_wait<1>(); else cp_async_wait<0>();
 
-    const uint32_t prog = c.prog;
+    const uint32_t prog = SINGLE ? kSingleProg : c.prog;
     const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
     const uint32_t body_words = CW(prog + DVM_H_CODE_WORDS);
     const int W = 1 << c.lgW;
@@ -541,8 +546,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             if ((op >= DVM_OP_BIN && op < DVM_OP_BINS) || op >= DVM_OP_LD2) {
               DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, o[i].x), fast_div(A[i].y, o[i].y));
             } else {
-              // division by a per-row scalar or an immediate: one correctly rounded reciprocal, packed multiplies
-              const float rcp = 1.0f / o[0].x;
+              // division by a per-row scalar or an immediate: one SFU reciprocal (1 ulp), packed multiplies
+              const float rcp = fast_rcp(o[0].x);
               DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], make_float2(rcp, rcp));
             }
             break;
@@ -774,7 +779,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   cp_async_wait<0>();
 
   if (err && tid == 0) atomicMax(prm.status, err);
-  if (prm.use_queue) {
+  if (use_queue) {
     // the last CTA to finish returns the queue to its resting state (both counters zero)
     __syncthreads();
     if (tid == 0) {
