@@ -299,7 +299,8 @@ class C4Workload:
 
     def __init__(self, dvm, n_launches=50, device="cuda"):
         self.dvm = dvm
-        dvm.set_elems_per_thread(16)   # programs of one stacked launch share the setting; 16 fits every program
+        if not dvm.binding.lib.dvm_get_elems_per_thread():
+            dvm.set_elems_per_thread(16)   # programs of one stacked launch share the setting; 16 fits every program
         self.launches = wl.shapes_c4(n_launches)
         self.progs = {k: wl.stack_program(k) for k in wl.STACK_KINDS}
         self.ps = {k: dvm.program_from_nodes(p.nodes) for k, p in self.progs.items()}
@@ -440,6 +441,7 @@ def main():
     ap.add_argument("--impl", default="dvm", choices=["dvm", "reference"])
     ap.add_argument("--instances", type=int, default=0, help="override the number of instances (debug)")
     ap.add_argument("--max-rows", type=int, default=0, help="cap rows per instance (small profiling case)")
+    ap.add_argument("--elems-per-thread", type=int, default=0, help="fix the encoder's elements per thread (16/32/64; 0 = cost model)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--detail", default="", help="write per-instance timings to this JSON file")
@@ -464,6 +466,8 @@ def main():
     dvm.binding = binding
 
     kw = {}
+    if args.elems_per_thread:
+        dvm.set_elems_per_thread(args.elems_per_thread)
     if args.instances:
         kw = {"n_launches": args.instances} if args.workload == "c4" else {"n_instances": args.instances}
     if args.max_rows and args.workload == "c2":

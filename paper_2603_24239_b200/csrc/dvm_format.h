@@ -48,8 +48,7 @@ enum {
   DVM_H_PRIMARY = 16,        // operand whose row starts define the vector alignment, or 0xffffffff
   DVM_H_LOCAL = 17,          // n_in_regs | n_tmp_regs << 8 | n_scalar_slots << 16 | V << 24 (elements per thread: 16 or 32)
   DVM_H_LOAD_WORDS = 18,     // length of the load section (words) at the start of the code body
-  DVM_H_LOCAL2 = 19,         // staging unit offset (buffer 0) | scalar-slot unit offset << 8 | total units << 16 |
-                             // staging unit offset (buffer 1) << 24
+  DVM_H_LOCAL2 = 19,         // scalar-slot unit offset << 8 | total units << 16
   DVM_HDR_WORDS = 20
 };
 
@@ -63,7 +62,8 @@ enum {
 
 // ---- operand descriptor ----
 enum {
-  DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24
+  DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24 | dense << 25
+                         // (dense: element (row, col) sits at flat offset row * C + col)
   DVM_OPD_RSVD = 1,
   DVM_OPD_STRIDE0 = 2,   // int64 element stride of outer dim 0 (lo, hi)
   DVM_OPD_STRIDE1 = 4,
@@ -110,8 +110,10 @@ enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_SUMSQ = 3, DVM_R_NRED 
 
 // Instruction ids.  The code body is [load section][compute section].
 // ACC is the register-resident accumulator tile; L[k] are tile registers in local (shared) memory,
-// thread-private, k < n_in: input registers (double buffered, filled by the load section of the
-// next tile while the current one is computed), k >= n_in: temporaries; S[k] are per-row scalars.
+// thread-private, k < n_in: input registers, k >= n_in: temporaries; S[k] are per-row scalars.
+// The next tile's loads overlap the current tile's compute: input registers are double-buffered and the
+// load section of tile i+1 runs when tile i starts; a row-vector input of an aligned program is the same
+// for every tile of a thread and is loaded once.
 enum {
   DVM_OP_NOP = 0x00,
   DVM_OP_LDG = 0x01,   // [load] a = local register (| 0x80: tile-invariant, loaded once per CTA and program),

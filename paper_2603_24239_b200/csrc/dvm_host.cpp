@@ -844,33 +844,18 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   // element units; N is the number of CTAs resident at once, which the local-memory need decides.
   const int T = DVM_VM_THREADS;
   const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
+  const uint32_t single_mask = 0;  // every tile input is double-buffered (a tile-invariant one is loaded once)
   struct Geo {
-    int V, log2G, W, units, staging_unit[2], scalar_unit;
+    int V, log2G, W, units, scalar_unit;
     int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
     uint32_t flags, inv_mask;
     uint32_t lreg_table[DVM_MAX_LREGS];
   } best;
   best.cost = -1;
   const int W0 = W;
-  // local registers that no instruction touches after the first tile store: the store's staging line may
-  // reuse one of them
-  uint32_t dead_at_store = 0;
-  {
-    int first_stg = -1;
-    uint32_t used_after = 0;
-    for (int pc = 0; pc < e.n_body; pc += (int)DVM_INSN_LEN(e.body[pc])) {
-      const uint32_t w0 = e.body[pc], op = DVM_INSN_OP(w0), ra = DVM_INSN_A(w0), rb = DVM_INSN_B(w0);
-      if (op == DVM_OP_STG && first_stg < 0) first_stg = pc;
-      if (first_stg < 0) continue;
-      if (op == DVM_OP_LDA || op == DVM_OP_STA) used_after |= 1u << ra;
-      else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) { if (ra != DVM_REG_ACC) used_after |= 1u << ra; }
-      else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) used_after |= (1u << ra) | (1u << (rb & 0x3f));
-    }
-    if (first_stg >= 0) dead_at_store = ~used_after & ((1u << nreg) - 1);
-  }
   for (int vi = 0; vi < 2; ++vi) {
     Geo g;
-    g.V = vi == 0 ? 32 : 16;
+    g.V = 32 >> vi;
     if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
     int ctas_guess = 2;
     bool ok = false;
@@ -934,36 +919,25 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
       // a row-vector input of an aligned program is the same for every tile of a thread: once),
       // temporaries, the staging line of the scalar store path, per-row scalar slots
       g.inv_mask = 0;
-      int in_units = 0, inv_units = 0, off[DVM_MAX_LREGS], usz[DVM_MAX_LREGS];
+      g.units = 0;
+      int usz[DVM_MAX_LREGS];
       for (int k = 0; k < e.n_in_regs; ++k) {
         usz[k] = g.V * (in_dtype[k] == DVM_DT_BF16 ? 2 : 4) / 32;
         const Operand& od = e.opd[in_opd[k]];
         const bool inv = !flat && (g.flags & DVM_F_ALIGNED) && g.W > 1 && g.CB == 1 && od.ostride[0] == 0 &&
                          od.ostride[1] == 0 && od.ostride[2] == 0;
         if (inv) g.inv_mask |= 1u << k;
-        else { off[k] = in_units; in_units += usz[k]; }
-      }
-      for (int k = 0; k < e.n_in_regs; ++k)
-        if ((g.inv_mask >> k) & 1) { off[k] = 2 * in_units + inv_units; inv_units += usz[k]; }
-      for (int k = 0; k < e.n_in_regs; ++k)
-        g.lreg_table[k] = ((g.inv_mask >> k) & 1) ? ((uint32_t)off[k] | ((uint32_t)off[k] << 16))
-                                                   : ((uint32_t)off[k] | ((uint32_t)(off[k] + in_units) << 16));
-      g.units = 2 * in_units + inv_units;
-      for (int k = e.n_in_regs; k < nreg; ++k) {
-        usz[k] = g.V * 4 / 32;
         g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)g.units << 16);
         g.units += usz[k];
       }
-      const int need = g.V * out_es / 32;
-      int alias = -1;
-      for (int k = 0; k < nreg && alias < 0; ++k)
-        if (((dead_at_store >> k) & 1) && !((g.inv_mask >> k) & 1) && usz[k] >= need) alias = k;
-      if (alias >= 0) {
-        g.staging_unit[0] = (int)(g.lreg_table[alias] & 0xffff);
-        g.staging_unit[1] = (int)(g.lreg_table[alias] >> 16);
-      } else {
-        g.staging_unit[0] = g.staging_unit[1] = g.units;
-        g.units += need;
+      for (int k = 0; k < e.n_in_regs; ++k) {
+        if (((g.inv_mask | single_mask) >> k) & 1) continue;   // one copy is enough
+        g.lreg_table[k] = (g.lreg_table[k] & 0xffff) | ((uint32_t)g.units << 16);
+        g.units += usz[k];
+      }
+      for (int k = e.n_in_regs; k < nreg; ++k) {
+        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)g.units << 16);
+        g.units += g.V * 4 / 32;
       }
       g.scalar_unit = g.units;
       if (e.n_sslots > 0) g.units += 2;
@@ -1022,14 +996,17 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
   w[DVM_H_LOCAL] = (uint32_t)e.n_in_regs | ((uint32_t)e.n_tmp_regs << 8) | ((uint32_t)e.n_sslots << 16) | ((uint32_t)best.V << 24);
   w[DVM_H_LOAD_WORDS] = (uint32_t)e.n_loads;
-  w[DVM_H_LOCAL2] = (uint32_t)best.staging_unit[0] | ((uint32_t)scalar_unit << 8) | ((uint32_t)units << 16) |
-                    ((uint32_t)best.staging_unit[1] << 24);
+  w[DVM_H_LOCAL2] = ((uint32_t)scalar_unit << 8) | ((uint32_t)units << 16);
   uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
   for (int o = 0; o < e.n_opd; ++o) {
     const Operand& od = e.opd[o];
     uint32_t* d = ot + o * DVM_OPD_WORDS;
+    // dense: the rows of a tile are one contiguous byte range (flat offset = row * C + col)
+    bool dense = od.col_stride == 1 && od.ostride[0] == C;
+    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
     d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
-                      ((uint32_t)(od.primary ? 1 : 0) << 24);
+                      ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25);
     for (int g = 0; g < 3; ++g) {
       d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
       d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
@@ -1092,9 +1069,8 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   if (lg > 8 || !(W == 1 || W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
   const uint32_t local2 = w[DVM_H_LOCAL2];
   const uint32_t units = (local2 >> 16) & 0xff, scalar_unit = (local2 >> 8) & 0xff;
-  const uint32_t staging_unit = (local2 & 0xff) > (local2 >> 24) ? (local2 & 0xff) : (local2 >> 24);  // the larger offset bounds both
   if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || units > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
-  if (staging_unit + u_bf16 > units || (n_ss && scalar_unit + 2 > units)) return DVM_ERR_BAD_CODE;
+  if (n_ss && scalar_unit + 2 > units) return DVM_ERR_BAD_CODE;
   const uint32_t* lt = w + DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd;
   // a local register access of `need` units (bf16: 1, fp32: 2) must stay inside the CTA's local memory
   auto lreg_ok = [&](uint32_t k, uint32_t need) {
@@ -1124,6 +1100,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if (((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
     if (ot[o * DVM_OPD_WORDS + 3] | ot[o * DVM_OPD_WORDS + 5] | ot[o * DVM_OPD_WORDS + 7]) return DVM_ERR_BAD_CODE;  // 32-bit strides
     n_primary += (info >> 24) & 1;
+    if (info >> 26) return DVM_ERR_BAD_CODE;
   }
   if (n_primary > 1) return DVM_ERR_BAD_CODE;
   if (w[DVM_H_PRIMARY] != 0xffffffffu) {
@@ -1145,7 +1122,6 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       if (op == DVM_OP_LDG && ((a & 0x7f) >= n_inr || !lreg_ok(a & 0x7f, ((info >> 8) & 0xff) == DVM_DT_BF16 ? u_bf16 : u_f32))) return DVM_ERR_BAD_CODE;
       bool is_out = (info & 0xff) >= n_in;
       if ((op == DVM_OP_STG) != is_out) return DVM_ERR_BAD_CODE;  // never store to an input, never load an output
-      if (op == DVM_OP_STG && staging_unit + (((info >> 8) & 0xff) == DVM_DT_BF16 ? u_bf16 : u_f32) > units) return DVM_ERR_BAD_CODE;
       if (((info >> 16) & 0xff) != 1) return DVM_ERR_BAD_CODE;
     } else if (op == DVM_OP_LDS || op == DVM_OP_STS) {
       if (bb >= n_opd) return DVM_ERR_BAD_CODE;

@@ -80,10 +80,11 @@ static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out) {
   DVM_CUDA(cudaGetDevice(&dev));
   std::lock_guard<std::mutex> lk(g_mu);
   DeviceState& d = g_dev[dev];
-  int& slot = d.occ[V == 32][large ? 1 : 0][units];
+  int& slot = d.occ[V == 32 ? 1 : 0][large ? 1 : 0][units];
   if (slot == 0) {
-    int st = V == 32 ? (large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem))
-                     : (large ? occupancy<16, PW_LARGE>(&slot, smem) : occupancy<16, PW_SMALL>(&slot, smem));
+    int st;
+    if (V == 32) st = large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem);
+    else st = large ? occupancy<16, PW_LARGE>(&slot, smem) : occupancy<16, PW_SMALL>(&slot, smem);
     if (st != DVM_OK) return st;
   }
   *out = slot;

@@ -62,14 +62,14 @@ def test_encode_geometry_and_shapes():
     c = _enc(wl.program_add_rmsnorm(), [(1000, 4096), (1000, 4096), (4096,)])
     assert c.out_shapes == [(1000, 4096), (1000, 4096)]
     info = dvm.code_info(c)
-    # 4096 columns: 128 threads x 32 elements (two rows per tile) or 256 x 16 (one row per tile)
-    assert info["threads_per_row"] in (128, 256) and info["vector_width"] == 8
+    # 4096 columns: 64 threads x 64 elements (four rows per tile), 128 x 32 or 256 x 16
+    assert info["threads_per_row"] in (64, 128, 256) and info["vector_width"] == 8
     assert info["n_tiles"] == 1000 * info["threads_per_row"] // 256
     assert info["kernel_type"] == 1 and info["n_tile_regs"] == 3   # three inputs in local registers, no temporaries
     c = _enc(wl.program_masked_softmax(), [(2, 32, 100, 100), (1, 1, 100, 100)])
     assert c.out_shapes == [(2, 32, 100, 100)]
     info = dvm.code_info(c)
-    assert info["threads_per_row"] * 32 >= 100                # rows of 100 bf16 start on 8-byte boundaries only
+    assert info["threads_per_row"] * 64 >= 100                # rows of 100 bf16 start on 8-byte boundaries only
     assert info["n_tiles"] == -(-6400 // (256 // info["threads_per_row"]))
     # pure elementwise program collapses to a flat range
     c = _enc(wl.program_c1(), [(7, 1531)] * 3)
@@ -99,7 +99,7 @@ def test_encode_errors():
     # a reduced row longer than the register budget
     q = dvm.program_from_nodes(wl.program_layernorm().nodes)
     with pytest.raises(dvm.DvmError) as e:
-        dvm.encode(q, [(4, 9000)], (1 / 9000,))
+        dvm.encode(q, [(4, 17000)], (1 / 17000,))
     assert e.value.status == -3
     # missing runtime scalar
     with pytest.raises(dvm.DvmError):
