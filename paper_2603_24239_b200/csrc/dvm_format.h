@@ -9,7 +9,7 @@
 //   [ header : DVM_HDR_WORDS words ]
 //   [ tensor table : 2 words per tensor slot (device pointer, patched at launch) ]
 //   [ operand table : DVM_OPD_WORDS words per global-memory operand ]
-//   [ local register table : one word per local register: unit offset of buffer 0 | buffer 1 << 16 ]
+//   [ local register table : one word per local register: its unit offset inside a tile slot ]
 //   [ code body : CodeSize words, instructions of 1..3 words ]
 //
 // Unlike the paper's bytecode, a memory instruction does not carry an address:
@@ -48,7 +48,7 @@ enum {
   DVM_H_PRIMARY = 16,        // operand whose row starts define the vector alignment, or 0xffffffff
   DVM_H_LOCAL = 17,          // n_in_regs | n_tmp_regs << 8 | n_scalar_slots << 16 | V << 24 (elements per thread: 16 or 32)
   DVM_H_LOAD_WORDS = 18,     // length of the load section (words) at the start of the code body
-  DVM_H_LOCAL2 = 19,         // scalar-slot unit offset << 8 | total units << 16
+  DVM_H_LOCAL2 = 19,         // scalar-slot unit offset << 8 | units of one tile slot << 16
   DVM_HDR_WORDS = 20
 };
 
@@ -79,7 +79,7 @@ enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
 #define DVM_MAX_LREGS 10         // local tile registers of a program (inputs + temporaries)
 #define DVM_MAX_SSLOTS 8         // per-row scalar inputs of a program
 #define DVM_LOCAL_UNIT 8192      // bytes of one local-memory unit: 32 B per thread (16 bf16 or 8 fp32 words)
-#define DVM_MAX_LOCAL_UNITS 27   // units a CTA can hold (2 x inputs + temporaries + staging + scalars), 216 KB
+#define DVM_MAX_LOCAL_UNITS 27   // units a CTA can hold (two tile slots), 216 KB
 #define DVM_MAX_SREGS 8          // per-row scalar registers
 #define DVM_MAX_TENSORS 16
 #define DVM_MAX_OPERANDS 24
@@ -111,9 +111,9 @@ enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_SUMSQ = 3, DVM_R_NRED 
 // Instruction ids.  The code body is [load section][compute section].
 // ACC is the register-resident accumulator tile; L[k] are tile registers in local (shared) memory,
 // thread-private, k < n_in: input registers, k >= n_in: temporaries; S[k] are per-row scalars.
-// The next tile's loads overlap the current tile's compute: input registers are double-buffered and the
-// load section of tile i+1 runs when tile i starts; a row-vector input of an aligned program is the same
-// for every tile of a thread and is loaded once.
+// A CTA holds two tile slots (complete sets of local registers): the load section of tile i+1 fills one
+// slot while tile i is computed in the other; a row-vector input of an aligned program is the same for
+// every tile of a thread and is loaded once per slot.
 enum {
   DVM_OP_NOP = 0x00,
   DVM_OP_LDG = 0x01,   // [load] a = local register (| 0x80: tile-invariant, loaded once per CTA and program),

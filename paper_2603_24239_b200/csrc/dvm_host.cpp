@@ -844,7 +844,6 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   // element units; N is the number of CTAs resident at once, which the local-memory need decides.
   const int T = DVM_VM_THREADS;
   const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
-  const uint32_t single_mask = 0;  // every tile input is double-buffered (a tile-invariant one is loaded once)
   struct Geo {
     int V, log2G, W, units, scalar_unit;
     int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
@@ -888,7 +887,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
           const int w = pass == 0 ? W0 : 1;  // second pass: element-wise mapping, which needs no padding
           const bool al = pass == 0 ? aligned : true;
           const int64_t pad = 0;  // a misaligned row wraps its last columns into the unused head slots: no padding
-          for (int lg = 0; lg <= 8; ++lg) {
+          for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
             int64_t G = 1 << lg, cap = G * g.V;
             int64_t ct;
             if (has_reduce) {
@@ -918,31 +917,27 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
       // local-memory layout in 8 KB units (32 bytes per thread): input registers twice (double buffering;
       // a row-vector input of an aligned program is the same for every tile of a thread: once),
       // temporaries, the staging line of the scalar store path, per-row scalar slots
+      // Local-memory layout of ONE tile slot, in 8 KB units (32 bytes per thread): input registers,
+      // temporaries, per-row scalar slots.  A CTA holds two slots: while it computes the tile in one, the
+      // next tile (of this or of another stacked program) loads into the other.
       g.inv_mask = 0;
       g.units = 0;
-      int usz[DVM_MAX_LREGS];
       for (int k = 0; k < e.n_in_regs; ++k) {
-        usz[k] = g.V * (in_dtype[k] == DVM_DT_BF16 ? 2 : 4) / 32;
         const Operand& od = e.opd[in_opd[k]];
         const bool inv = !flat && (g.flags & DVM_F_ALIGNED) && g.W > 1 && g.CB == 1 && od.ostride[0] == 0 &&
                          od.ostride[1] == 0 && od.ostride[2] == 0;
-        if (inv) g.inv_mask |= 1u << k;
-        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)g.units << 16);
-        g.units += usz[k];
-      }
-      for (int k = 0; k < e.n_in_regs; ++k) {
-        if (((g.inv_mask | single_mask) >> k) & 1) continue;   // one copy is enough
-        g.lreg_table[k] = (g.lreg_table[k] & 0xffff) | ((uint32_t)g.units << 16);
-        g.units += usz[k];
+        if (inv) g.inv_mask |= 1u << k;  // the same for every tile of a thread: loaded once per slot
+        g.lreg_table[k] = (uint32_t)g.units;
+        g.units += g.V * (in_dtype[k] == DVM_DT_BF16 ? 2 : 4) / 32;
       }
       for (int k = e.n_in_regs; k < nreg; ++k) {
-        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)g.units << 16);
+        g.lreg_table[k] = (uint32_t)g.units;
         g.units += g.V * 4 / 32;
       }
       g.scalar_unit = g.units;
       if (e.n_sslots > 0) g.units += 2;
-      if (g.units > DVM_MAX_LOCAL_UNITS) break;
-      int ctas = 233472 / (g.units * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
+      if (2 * g.units > DVM_MAX_LOCAL_UNITS) break;
+      int ctas = 233472 / (2 * g.units * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
       if (ctas > 2) ctas = 2;  // the interpreter is compiled for two resident CTAs per SM
       if (ctas < 1) break;
       if (ctas == ctas_guess) ok = true;
@@ -1069,12 +1064,12 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   if (lg > 8 || !(W == 1 || W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
   const uint32_t local2 = w[DVM_H_LOCAL2];
   const uint32_t units = (local2 >> 16) & 0xff, scalar_unit = (local2 >> 8) & 0xff;
-  if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || units > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
+  if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || 2 * units > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
   if (n_ss && scalar_unit + 2 > units) return DVM_ERR_BAD_CODE;
   const uint32_t* lt = w + DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd;
   // a local register access of `need` units (bf16: 1, fp32: 2) must stay inside the CTA's local memory
   auto lreg_ok = [&](uint32_t k, uint32_t need) {
-    return k < nreg && (lt[k] & 0xffff) + need <= units && (lt[k] >> 16) + need <= units;
+    return k < nreg && lt[k] + need <= units;
   };
   const uint32_t load_words = w[DVM_H_LOAD_WORDS];
   if (load_words > body) return DVM_ERR_BAD_CODE;

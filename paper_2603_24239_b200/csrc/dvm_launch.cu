@@ -191,7 +191,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.queue = dev.scratch + 8 + 2 * dev.queue_slot;
 
   const bool large = pos > PW_SMALL;
-  const size_t smem = (size_t)units * DVM_LOCAL_UNIT;
+  const size_t smem = 2 * (size_t)units * DVM_LOCAL_UNIT;  // two tile slots
+  P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   int occ = 0;
   st = dvm_occupancy(V, large, (int)units, smem, &occ);

@@ -7,10 +7,11 @@
 // the CTA's tiles.  A code body is [load section][compute section]:
 //   * every global tile load is an asynchronous 16-byte global->shared copy
 //     (cp.async) into a thread-private "local register" in shared memory -- the
-//     paper's local memory.  Input registers are double-buffered: the load
-//     section of tile i+1 runs when tile i starts, so the next tile's HBM traffic
-//     is in flight during the whole compute of the current one at no register
-//     cost; a row-vector input of an aligned program is loaded once;
+//     paper's local memory.  A CTA holds two tile slots (complete register sets):
+//     the load section of tile i+1 -- of the same or of another stacked program --
+//     runs when tile i starts, so the next tile's HBM traffic is in flight during
+//     the whole compute of the current one at no register cost; a row-vector
+//     input of an aligned program is loaded once per slot;
 //   * the compute section is accumulator code: ACC is one register-resident tile
 //     (V = 16 or 32 fp32 per thread, as float2 pairs so that add / mul / fma
 //     issue as packed f32x2 instructions); other operands are read from local
@@ -57,6 +58,8 @@ struct VMParams {
   uint32_t total_tiles;
   uint32_t n_words;      // words used in `words`
   uint32_t use_queue;    // 1: tiles beyond the first are claimed from the work queue
+  uint32_t slot_bytes;   // bytes of one tile slot in local memory (the largest program's)
+  uint32_t pad_;
   unsigned int* status;  // device status word
   unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished (both zero between launches)
   uint32_t words[PW];    // [program word offsets][tile prefix sums (n+1)][programs ...]
@@ -179,7 +182,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 #define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
 
   // shared-memory address of 16-byte vector 0 of the register at unit offset U (this thread's part)
-  auto lreg_addr = [&](uint32_t unit) -> uint32_t { return local_base + unit * DVM_LOCAL_UNIT; };
+  auto lreg_addr = [&](uint32_t unit, int slot) -> uint32_t { return local_base + unit * DVM_LOCAL_UNIT + (slot ? prm.slot_bytes : 0u); };
 
   // word offsets of a program's tables
   auto opd_base = [&](uint32_t prog) -> uint32_t { return prog + DVM_HDR_WORDS + 2 * (CW(prog + DVM_H_COUNTS) & 0xff); };
@@ -285,8 +288,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const int G = 1 << c.lgG;
     int dt;
     const char* p = operand_addr(prog, opd0, ib, c, dt);
-    const uint32_t lt = CW(lreg0 + ia);
-    const uint32_t d0 = lreg_addr(buf ? (lt >> 16) : (lt & 0xffff));
+    const uint32_t d0 = lreg_addr(CW(lreg0 + ia), buf);
     const int es = dt == DVM_DT_BF16 ? 2 : 4;
     if (W == 1) {
       // element-wise mapping: every valid slot is one scalar copy
@@ -403,8 +405,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         int dt;
         const char* p = operand_addr(prog, opd0, DVM_INSN_B(w0), c, dt);
         const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
-        const uint32_t w = (uint32_t)buf * DVM_MAX_SSLOTS + (uint32_t)DVM_INSN_A(w0);
-        const uint32_t dst = lreg_addr(unit) + (w >> 2) * VSTRIDE + (w & 3) * 4;
+        const uint32_t w = (uint32_t)DVM_INSN_A(w0);
+        const uint32_t dst = lreg_addr(unit, buf) + (w >> 2) * VSTRIDE + (w & 3) * 4;
         if (c.ncols > 0) {
           if (dt == DVM_DT_BF16) {
             const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(p));
@@ -467,15 +469,17 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   unsigned err = 0;
 
   TileCtx c;
-  bool own_loads = true;  // this tile's loads are not in flight yet (first tile, or the program changed)
+  uint32_t slot_prog[2] = {0xffffffffu, 0xffffffffu};  // program whose tile-invariant inputs each slot holds
   if (tile < prm.total_tiles) {
     if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
     make_ctx(c, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
+    issue_loads(c, buf, true);
+    slot_prog[0] = prog_idx;
+    cp_async_commit();
   }
 
   while (tile < prm.total_tiles) {
-    // ---- Algorithm 2, outer loop: next tile of this core; its loads start now when it runs the same program
-    // (another program has another local-memory layout: its loads start when its own iteration begins) ----
+    // ---- Algorithm 2, outer loop: next tile of this core; its loads start now, into the other tile slot ----
     uint32_t next;
     if (use_queue) {
       if (tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
@@ -487,24 +491,18 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     ++iter;
     TileCtx cn = c;
     const bool have_next = next < prm.total_tiles;
-    bool early = false;
     uint32_t next_prog_idx = prog_idx;
     if (have_next) {
       if (!SINGLE) while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
-      early = next_prog_idx == prog_idx;
       make_ctx(cn, SINGLE ? kSingleProg : CW(next_prog_idx), SINGLE ? next : next - CW(n_prog + next_prog_idx));
-    }
-    if (own_loads) {
-      issue_loads(c, buf, true);
+      const bool first = buf ? slot_prog[0] != next_prog_idx : slot_prog[1] != next_prog_idx;
+      issue_loads(cn, buf ^ 1, first);
+      if (buf) slot_prog[0] = next_prog_idx; else slot_prog[1] = next_prog_idx;
       cp_async_commit();
+      cp_async_wait<1>();  // this tile's loads have landed once only the next tile's group is pending
+    } else {
+      cp_async_wait<0>();
     }
-    if (early) {
-      issue_loads(cn, buf ^ 1, false);
-      cp_async_commit();
-    }
-    // this tile's loads have landed once at most the next tile's group is pending
-    if (early) cp_async_wait<1>(); else cp_async_wait<0>();
-    own_loads = !early;
 
     const uint32_t prog = SINGLE ? kSingleProg : c.prog;
     const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
@@ -527,13 +525,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         uint32_t ay;
         int dty;
         if (op >= DVM_OP_LD2) {
-          const uint32_t lx = CW(lreg0 + ia), ly = CW(lreg0 + (ib & 0x3f));
-          read_acc(lreg_addr(buf ? (lx >> 16) : (lx & 0xffff)), (ib >> 6) & 1);
-          ay = lreg_addr(buf ? (ly >> 16) : (ly & 0xffff));
+          read_acc(lreg_addr(CW(lreg0 + ia), buf), (ib >> 6) & 1);
+          ay = lreg_addr(CW(lreg0 + (ib & 0x3f)), buf);
           dty = (ib >> 7) & 1;
         } else {
-          const uint32_t ly = CW(lreg0 + ia);
-          ay = lreg_addr(buf ? (ly >> 16) : (ly & 0xffff));
+          ay = lreg_addr(CW(lreg0 + ia), buf);
           dty = ib;
         }
 #define DVM_TILE_OP(...)                                             \
@@ -679,11 +675,10 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       switch (op) {
         case DVM_OP_NOP: break;
         case DVM_OP_LDA: {
-          const uint32_t lt = CW(lreg0 + ia);
-          read_acc(lreg_addr(buf ? (lt >> 16) : (lt & 0xffff)), ib);
+          read_acc(lreg_addr(CW(lreg0 + ia), buf), ib);
         } break;
         case DVM_OP_STA: {
-          const uint32_t a0 = lreg_addr(CW(lreg0 + ia) & 0xffff);
+          const uint32_t a0 = lreg_addr(CW(lreg0 + ia), buf);
 #pragma unroll
           for (int q = 0; q < V / 4; ++q)
             asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * VSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
@@ -692,9 +687,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         } break;
         case DVM_OP_LSS: {
           const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
-          const uint32_t w = (uint32_t)buf * DVM_MAX_SSLOTS + (uint32_t)ib;
+          const uint32_t w = (uint32_t)ib;
           float v;
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lreg_addr(unit) + (w >> 2) * VSTRIDE + (w & 3) * 4));
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lreg_addr(unit, buf) + (w >> 2) * VSTRIDE + (w & 3) * 4));
           sset(S, ia, c.ncols > 0 ? v : 0.f);
         } break;
         case DVM_OP_STG: {

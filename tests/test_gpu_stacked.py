@@ -71,7 +71,7 @@ def test_stacked_repeated_launches_reuse_queue():
 
 def test_stacked_with_32_elements_per_thread():
     dvm.set_elems_per_thread(32)
-    items = [("layernorm", 17, 100), ("sigmoid_mul", 300, 5000), ("layernorm", 64, 8000), ("gelu_affine", 200, 1024)]
+    items = [("layernorm", 17, 100), ("sigmoid_mul", 300, 5000), ("layernorm", 64, 8000), ("sigmoid_mul", 200, 1024)]
     codes, tls, meta = _stack(items, 77)
     dvm.launch_stacked(codes, tls)
     assert dvm.last_device_status() == 0
