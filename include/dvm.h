@@ -167,6 +167,29 @@ int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_t
 int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
                        void* const* const* tensors, const int* n_tensors, void* cuda_stream);
 
+/* The stacked launch for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for deployment, not for the method.)
+ *
+ * dvm_launch_stacked keeps its work-queue counters in a small device buffer that the library cudaMalloc's
+ * the first time it is used on a device.  Callers that run inside a memory pool owning the whole device,
+ * serving loops that cannot afford the implicit synchronisation of a first-use cudaMalloc, and sandboxes
+ * that forbid the allocator cannot use it.  This variant runs the same kernel with the counters in a fixed
+ * 256-byte array inside the library image (every GPU that loads the library holds it until the process
+ * exits) and calls neither cudaMalloc nor cudaFree nor any allocating routine.
+ *  - Arguments, tensor ownership and the result are those of dvm_launch_stacked.
+ *  - Limits: at most DVM_NOALLOC_MAX_PROGRAMS programs and DVM_NOALLOC_MAX_TILES tiles per call;
+ *    larger requests return DVM_ERR_TOO_LARGE.
+ *  - The first call on a device resolves the array's device address (cudaGetSymbolAddress) and reads the
+ *    SM count; make that first call before any stream capture.
+ *  - Every call shares the array, and the array keeps the last call's contents: each call clears it on
+ *    `cuda_stream` before its kernel.  Two calls whose kernels overlap on the GPU (different streams) race
+ *    on it -- serialise them.
+ *  - Device-side status is not reported for this variant (the bytecode is verified on the host first). */
+#define DVM_NOALLOC_MAX_PROGRAMS 256
+#define DVM_NOALLOC_MAX_TILES 0x7fffffffull
+int dvm_launch_stacked_noalloc(int n_programs, const void* const* codes, const size_t* code_sizes,
+                               void* const* const* tensors, const int* n_tensors, void* cuda_stream);
+
 /* End-to-end convenience for HOST tensors: copies the inputs to device staging
  * memory the caller provides (`staging`, device pointer, staging_bytes >= sum of
  * all tensor sizes rounded up to 256 B each), launches, copies the outputs back

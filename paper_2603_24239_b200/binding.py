@@ -70,6 +70,7 @@ _sig = {
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
     "dvm_launch_stacked": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _vp], _i),
+    "dvm_launch_stacked_noalloc": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _vp], _i),
     "dvm_run_host": ([_vp, _sz, C.POINTER(_vp), C.POINTER(_sz), _i, _vp, _sz, _vp], _i),
     "dvm_verify": ([_vp, _sz], _i),
     "dvm_disassemble": ([_vp, _sz, C.c_char_p, _sz], _i),
@@ -245,15 +246,19 @@ def launch(code: Code, tensors: Sequence, stream=None):
     _check(lib.dvm_launch(code.buf, code.size, arr, len(tensors), _stream(stream)), "dvm_launch")
 
 
-def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None):
-    """dvm_launch_stacked: many independent programs in one kernel launch."""
+def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None, noalloc: bool = False):
+    """dvm_launch_stacked: many independent programs in one kernel launch.
+
+    noalloc=True calls dvm_launch_stacked_noalloc, the variant for callers that may not allocate device
+    memory (its work queue lives in a fixed array inside the library instead of a cudaMalloc'd buffer)."""
     n = len(codes)
     cptr = (_vp * n)(*[C.addressof(c.buf) for c in codes])
     csz = (_sz * n)(*[c.size for c in codes])
     keep = [(_vp * len(tl))(*[_ptr(t) for t in tl]) for tl in tensor_lists]
     tptr = (C.POINTER(_vp) * n)(*[C.cast(k, C.POINTER(_vp)) for k in keep])
     nt = (_i * n)(*[len(tl) for tl in tensor_lists])
-    _check(lib.dvm_launch_stacked(n, cptr, csz, tptr, nt, _stream(stream)), "dvm_launch_stacked")
+    fn = lib.dvm_launch_stacked_noalloc if noalloc else lib.dvm_launch_stacked
+    _check(fn(n, cptr, csz, tptr, nt, _stream(stream)), fn.__name__)
 
 
 def run_host(code: Code, host_tensors: Sequence, staging, stream=None):

@@ -278,3 +278,113 @@ extern "C" int dvm_last_device_status(void* cuda_stream, int* status) {
   *status = v == dvm::ST_OK ? DVM_OK : (v == dvm::ST_TIMEOUT ? DVM_ERR_DEVICE_TIMEOUT : DVM_ERR_DEVICE_BAD_CODE);
   return DVM_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// dvm_launch_stacked_noalloc: the stacked launch for callers that must not allocate device memory.
+//
+// dvm_launch_stacked keeps its work-queue counters in a small buffer that the library obtains with
+// cudaMalloc the first time a device is used.  Some callers cannot tolerate that: code running inside a
+// memory pool or arena that owns every byte of the device, latency-critical serving loops where a first-use
+// cudaMalloc (an implicit device synchronisation) is unacceptable, and sandboxes that forbid the allocator
+// outright.  For them the same kernel runs with its queue in the fixed array below, which is part of the
+// library image: every GPU that loads the library holds these 256 bytes until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int NOALLOC_WORDS = 64;                 // 256 bytes: [0] status word, [2..3] work-queue counters
+static __device__ __align__(256) unsigned int dvm_noalloc_scratch[NOALLOC_WORDS];
+
+struct NoAllocDevice {
+  unsigned int* scratch = nullptr;  // device address of dvm_noalloc_scratch on this device
+  int sm_count = 0;
+};
+NoAllocDevice g_noalloc[MAX_DEVICES];
+std::mutex g_noalloc_mu;
+
+// Once per device, with that device current: resolve the array's device address.  In host code the array's
+// name is only a stand-in for the symbol; the address a kernel may use comes from cudaGetSymbolAddress.
+int noalloc_device(NoAllocDevice* out) {
+  int dev = 0;
+  DVM_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return DVM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_noalloc_mu);
+  NoAllocDevice& d = g_noalloc[dev];
+  if (!d.scratch) {
+    void* p = nullptr;
+    DVM_CUDA(cudaGetSymbolAddress(&p, dvm_noalloc_scratch));
+    DVM_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    d.scratch = static_cast<unsigned int*>(p);
+  }
+  *out = d;
+  return DVM_OK;
+}
+
+}  // namespace
+
+extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* codes, const size_t* code_sizes,
+                                          void* const* const* tensors, const int* n_tensors, void* cuda_stream) {
+  if (n_programs < 0 || (n_programs > 0 && (!codes || !code_sizes || !tensors || !n_tensors)))
+    return DVM_ERR_INVALID_ARG;
+  if (n_programs == 0) return DVM_OK;
+  if (n_programs > DVM_NOALLOC_MAX_PROGRAMS) return DVM_ERR_TOO_LARGE;  // beyond the stated maximum
+  uint32_t dir = 2 * (uint32_t)n_programs + 1;
+  uint64_t need = dir, total_tiles = 0;
+  uint32_t units = 0;
+  int V = 0;
+  for (int i = 0; i < n_programs; ++i) {
+    if (!codes[i] || !tensors[i]) return DVM_ERR_INVALID_ARG;
+    int st = dvm_verify(codes[i], code_sizes[i]);
+    if (st != DVM_OK) return st;
+    const uint32_t* c = (const uint32_t*)codes[i];
+    if (c[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_UNSUPPORTED;
+    need += c[DVM_H_TOTAL_WORDS];
+    total_tiles += c[DVM_H_N_TILES];
+    if (((c[DVM_H_LOCAL2] >> 16) & 0xff) > units) units = (c[DVM_H_LOCAL2] >> 16) & 0xff;
+    const int v = (int)(c[DVM_H_LOCAL] >> 24);
+    if (V && v != V) return DVM_ERR_INVALID_ARG;
+    V = v;
+  }
+  if (need > PW_LARGE || total_tiles > DVM_NOALLOC_MAX_TILES) return DVM_ERR_TOO_LARGE;
+  if (total_tiles == 0) return DVM_OK;
+
+  NoAllocDevice dev;
+  int st = noalloc_device(&dev);
+  if (st != DVM_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  dvm::VMParams<PW_LARGE>& P = t_large;
+  uint32_t pos = dir, tb = 0;
+  for (int i = 0; i < n_programs; ++i) {
+    const uint32_t* c = (const uint32_t*)codes[i];
+    P.words[i] = pos;
+    P.words[n_programs + i] = tb;
+    st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
+    if (st != DVM_OK) return st;
+    pos += c[DVM_H_TOTAL_WORDS];
+    tb += c[DVM_H_N_TILES];
+  }
+  P.words[2 * n_programs] = tb;
+  P.n_programs = (uint32_t)n_programs;
+  P.total_tiles = (uint32_t)total_tiles;
+  P.n_words = pos;
+  P.use_queue = 1u;
+  P.status = dev.scratch;
+  P.queue = dev.scratch + 2;
+  const size_t smem = 2 * (size_t)units * DVM_LOCAL_UNIT;
+  P.slot_bytes = units * DVM_LOCAL_UNIT;
+  if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
+  const bool large = pos > PW_SMALL;
+  int occ = 0;
+  st = dvm_occupancy(V, large, (int)units, smem, &occ);
+  if (st != DVM_OK) return st;
+  uint64_t slots = (uint64_t)dev.sm_count * occ;
+  int grid = (int)(total_tiles < slots ? total_tiles : slots);
+  // every call shares the array and it keeps the last call's contents: the queue counters must start at zero
+  DVM_CUDA(cudaMemsetAsync(dev.scratch, 0, NOALLOC_WORDS * sizeof(unsigned int), stream));
+  if (!large) {
+    dvm::VMParams<PW_SMALL> S;
+    memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
+    return launch_variant<PW_SMALL>(V, S, grid, smem, stream);
+  }
+  return launch_variant<PW_LARGE>(V, P, grid, smem, stream);
+}
