@@ -140,9 +140,27 @@ enum {
 // DVM_SK_FMAU: S[a] = unary(S[src] * imm0 + imm1); len 4: word1 = unary (0xff: none) | src << 8, word2 = imm0, word3 = imm1
 enum { DVM_SK_BIN = 0, DVM_SK_BINI = 1, DVM_SK_UN = 2, DVM_SK_FMAU = 3 };
 
-// ---- matmul meta-kernel: extra header words follow the common header ----
-// (see dvm_matmul.cu)
+// ---- matmul meta-kernel (DVM_KERNEL_MATMUL): matmul instruction + interpreted epilogue ----
+//   [ header ][ tensor table ][ matmul extension : DVM_MM_WORDS ][ operand table ][ epilogue code ]
+// Header fields reused: N_TILES = row blocks x column blocks of the output, COLS = N, ROWS_LO = M.
+// The epilogue is accumulator code over one chunk of DVM_MM_CHUNK output columns of one output row
+// per thread.  Register operands of LDA / BIN / STA name
+//   r <  NB            : the fp32 result of matmul r (tensor memory),
+//   NB <= r < NB + n_tmp : a temporary (shared memory),
+//   0x80 | k           : global operand k of the operand table (an extra [M,N] / [1,N] / [M,1] input),
+//   0xff               : the accumulator itself.
+// STG names an operand of the operand table (an output, row-major [M,N]).
 enum {
-  DVM_MM_M = 0, DVM_MM_N = 1, DVM_MM_K = 2, DVM_MM_NB = 3,  // NB: number of B matrices (1 or 2)
-  DVM_MM_WORDS = 4
+  DVM_MM_M = 0, DVM_MM_N = 1, DVM_MM_K = 2,
+  DVM_MM_NB = 3,        // number of B matrices sharing A (1 or 2)
+  DVM_MM_TILE_N = 4,    // output columns per tile: 128 (NB = 2) or 256 (NB = 1)
+  DVM_MM_SLOTS = 5,     // tensor slot of A | slot of B0 << 8 | slot of B1 << 16
+  DVM_MM_NTMP = 6,      // epilogue temporaries
+  DVM_MM_MBLOCKS = 7, DVM_MM_NBLOCKS = 8, DVM_MM_KBLOCKS = 9,
+  DVM_MM_WORDS = 10
 };
+#define DVM_MM_BLOCK_M 128   // output rows per tile (one UMMA M)
+#define DVM_MM_BLOCK_K 64    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+#define DVM_MM_CHUNK 32      // output columns an epilogue thread holds at a time
+#define DVM_MM_MAX_TMP 2
+#define DVM_MM_MAX_WORDS 320 // whole matmul program (header, tables, code) in the kernel-parameter block

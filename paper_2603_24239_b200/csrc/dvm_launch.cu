@@ -33,14 +33,6 @@ std::mutex g_mu;
 thread_local int t_last_cuda_error = 0;
 long long g_launches = 0;
 
-#define DVM_CUDA(call)                       \
-  do {                                       \
-    cudaError_t e_ = (call);                 \
-    if (e_ != cudaSuccess) {                 \
-      t_last_cuda_error = (int)e_;           \
-      return DVM_ERR_CUDA;                   \
-    }                                        \
-  } while (0)
 
 template <int V, int PW>
 int occupancy(int* out, size_t smem) {

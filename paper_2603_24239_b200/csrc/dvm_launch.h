@@ -4,6 +4,21 @@
 #include <stddef.h>
 #include <stdint.h>
 
+// Device status word values (read back by dvm_last_device_status).
+namespace dvm {
+enum { ST_OK = 0, ST_BAD_CODE = 1, ST_TIMEOUT = 2 };
+}
+
+// Records a failed CUDA runtime call (dvm_last_cuda_error) and returns DVM_ERR_CUDA from the caller.
+#define DVM_CUDA(call)                \
+  do {                                \
+    cudaError_t e_ = (call);          \
+    if (e_ != cudaSuccess) {          \
+      dvm_note_cuda_error((int)e_);   \
+      return DVM_ERR_CUDA;            \
+    }                                 \
+  } while (0)
+
 struct DvmDeviceInfo {
   unsigned int* scratch;  // library-owned device words: [0] status, then work-queue counter pairs
   int sm_count;

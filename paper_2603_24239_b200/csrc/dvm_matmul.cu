@@ -1,13 +1,1020 @@
-// Matmul meta-kernel (placeholder until the tcgen05 path lands): reports "unsupported".
+// Matmul meta-kernel (Sec. 4.2 "matrix operations", Sec. 5.1 cube-vector fusion): the matmul
+// instruction on the sm_100a tensor cores with the fused elementwise epilogue interpreted from bytecode.
+//
+//   out[M,N] = epilogue( A[M,K] x B_0[K,N] , A x B_1 , extra inputs )      bf16 operands, fp32 accumulate
+//
+// Host half: dvm_encode_matmul (shape check, output tiling, epilogue accumulator code), verifier, dump.
+// Device half: one persistent CTA per SM, warp-specialised:
+//   warp 0      one thread issues the TMA tile loads of a 4-stage shared-memory ring
+//               (A: 128 x 64 K-major, B: 64 x 256 as four 64 x 64 boxes, 128-byte swizzle);
+//   warp 1      one thread issues tcgen05.mma (M = 128, N = 256, K = 16 per instruction) into one of two
+//               256-column accumulator stages of tensor memory and commits stage / tile completion to
+//               mbarriers; with two B matrices the accumulator columns are [B_0 tile | B_1 tile], so the
+//               gate and up products of one output tile sit side by side (the cube-vector constraint:
+//               the epilogue needs matching tiles of both);
+//   warps 2..5  the epilogue interpreter: every thread owns one output row of the tile, pulls
+//               32-column chunks of the accumulators out of tensor memory (tcgen05.ld), runs the
+//               epilogue code on them in registers and stores the narrowed result; it overlaps the
+//               next tile's MMAs (the other accumulator stage).
+// Every wait on an mbarrier is bounded (time and iteration limit): when one runs out the CTA raises its
+// abort flag, every role leaves its loop, copies and MMAs in flight are awaited (bounded again), tensor
+// memory is released and the status word reports DVM_ERR_DEVICE_TIMEOUT.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
 #include "../../include/dvm.h"
 #include "dvm_format.h"
 #include "dvm_internal.h"
 #include "dvm_launch.h"
+#include "dvm_math.cuh"
+#include "dvm_program.h"
 
-int dvm_encode_matmul(const dvm_program*, const dvm_shape*, int, const float*, int, void*, size_t, size_t*,
-                      dvm_shape*, int) {
-  return DVM_ERR_UNSUPPORTED;
+// =================================================================================================
+// Host: encode
+// =================================================================================================
+namespace {
+
+constexpr int MM_MAX_BODY = 6 * DVM_MAX_NODES + 4 * DVM_MAX_TENSORS;
+
+struct MmOperand {
+  int slot, dtype, col_stride;
+  int64_t row_stride;
+};
+
+struct MmEnc {
+  const dvm_program* p;
+  int16_t alias[DVM_MAX_NODES];
+  int16_t uses[DVM_MAX_NODES];
+  int16_t loc[DVM_MAX_NODES];  // register operand byte naming where the value lives, or -1
+  int16_t tmp_val[DVM_MM_MAX_TMP];
+  int n_tmp, nb;
+  int16_t acc;
+  uint32_t body[MM_MAX_BODY];
+  int n_body;
+  MmOperand opd[DVM_MAX_OPERANDS];
+  int n_opd;
+  bool stored[DVM_MAX_TENSORS];
+  int8_t out_operand[DVM_MAX_TENSORS];
+  const float* scalars;
+  bool fail;
+};
+
+inline int mroot(const MmEnc& e, int v) {
+  while (e.alias[v] >= 0) v = e.alias[v];
+  return v;
 }
-int dvm_verify_matmul(const uint32_t*, size_t) { return DVM_ERR_BAD_CODE; }
-int dvm_disassemble_matmul(const uint32_t*, size_t, char*, size_t) { return DVM_ERR_BAD_CODE; }
-int dvm_launch_matmul(const uint32_t*, size_t, void* const*, int, cudaStream_t) { return DVM_ERR_UNSUPPORTED; }
+inline void memit(MmEnc& e, uint32_t w) {
+  if (e.n_body < MM_MAX_BODY) e.body[e.n_body++] = w;
+  else e.fail = true;
+}
+inline uint32_t mf2u(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return u;
+}
+
+void mm_spill_acc_if_live(MmEnc& e) {
+  const int a = e.acc;
+  if (a < 0 || e.uses[a] <= 0 || e.loc[a] >= 0) return;
+  for (int k = 0; k < DVM_MM_MAX_TMP; ++k)
+    if (e.tmp_val[k] < 0) {
+      if (k + 1 > e.n_tmp) e.n_tmp = k + 1;
+      memit(e, DVM_INSN(DVM_OP_STA, 1, e.nb + k, 0));
+      e.tmp_val[k] = (int16_t)a;
+      e.loc[a] = (int16_t)(e.nb + k);
+      return;
+    }
+  e.fail = true;  // more live epilogue values than temporaries
+}
+
+void mm_ensure_acc(MmEnc& e, int v) {
+  if (e.acc == v) return;
+  mm_spill_acc_if_live(e);
+  if (e.fail) return;
+  if (e.loc[v] < 0) {
+    e.fail = true;
+    return;
+  }
+  memit(e, DVM_INSN(DVM_OP_LDA, 1, e.loc[v], 0));
+  e.acc = (int16_t)v;
+}
+
+// One consumer of value v (held in a temporary) is done: free the temporary of a dead value.
+void mm_release(MmEnc& e, int v) {
+  if (e.uses[v] > 0) return;
+  const int l = e.loc[v];
+  if (l >= e.nb && l < e.nb + DVM_MM_MAX_TMP) {
+    e.tmp_val[l - e.nb] = -1;
+    e.loc[v] = -1;
+  }
+}
+
+void mm_store_outputs_of(MmEnc& e, int v) {
+  for (int o = 0; o < e.p->n_outputs; ++o) {
+    if (e.stored[o] || mroot(e, e.p->outputs[o].value) != v) continue;
+    mm_ensure_acc(e, v);
+    if (e.fail) return;
+    memit(e, DVM_INSN(DVM_OP_STG, 1, 0, e.out_operand[o]));
+    e.stored[o] = true;
+    e.uses[v]--;
+  }
+}
+
+const uint8_t kMmBin[6] = {DVM_A_ADD, DVM_A_SUB, DVM_A_MUL, DVM_A_DIV, DVM_A_MIN, DVM_A_MAX};
+inline uint8_t mm_reversed(uint8_t a) { return a == DVM_A_SUB ? DVM_A_RSUB : a == DVM_A_DIV ? DVM_A_RDIV : a; }
+
+// Accumulator code of the elementwise epilogue (every value has the shape of the output tile).
+bool mm_gen_epilogue(MmEnc& e) {
+  const dvm_program* p = e.p;
+  e.n_body = 0;
+  e.n_tmp = 0;
+  e.acc = -1;
+  e.fail = false;
+  for (int k = 0; k < DVM_MM_MAX_TMP; ++k) e.tmp_val[k] = -1;
+  for (int o = 0; o < p->n_outputs; ++o) e.stored[o] = false;
+  for (int i = 0; i < p->n_nodes; ++i) e.uses[i] = 0;
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || n.kind == NK_MATMUL || e.alias[i] >= 0) continue;
+    e.uses[mroot(e, n.x)]++;
+    if (n.kind == NK_BINARY) e.uses[mroot(e, n.y)]++;
+  }
+  for (int o = 0; o < p->n_outputs; ++o) e.uses[mroot(e, p->outputs[o].value)]++;
+
+  for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || n.kind == NK_MATMUL || e.alias[i] >= 0) continue;
+    if (e.uses[i] == 0) continue;  // dead value
+    const int x = mroot(e, n.x);
+    switch (n.kind) {
+      case NK_UNARY:
+      case NK_SCALAR:
+      case NK_CAST: {
+        mm_ensure_acc(e, x);
+        if (e.fail) break;
+        e.uses[x]--;
+        mm_spill_acc_if_live(e);
+        mm_release(e, x);
+        if (n.kind == NK_UNARY) memit(e, DVM_INSN(DVM_OP_UN + n.op, 1, 0, 0));
+        else if (n.kind == NK_CAST) memit(e, DVM_INSN(DVM_OP_UN + DVM_U_RND_BF16, 1, 0, 0));
+        else {
+          const float s = n.param >= 0 ? e.scalars[n.param] : n.imm;
+          memit(e, DVM_INSN(DVM_OP_BINI + (n.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL), 2, 0, 0));
+          memit(e, mf2u(s));
+        }
+        e.acc = (int16_t)i;
+        break;
+      }
+      case NK_BINARY: {
+        const int y = mroot(e, n.y);
+        uint8_t op = kMmBin[n.op];
+        int other;  // the operand that is not in the accumulator
+        if (e.acc == x) other = y;
+        else if (e.acc == y) { other = x; op = mm_reversed(op); }
+        else { mm_ensure_acc(e, x); other = y; }
+        if (e.fail) break;
+        const int held = e.acc;
+        e.uses[x]--;
+        e.uses[y]--;
+        mm_spill_acc_if_live(e);
+        if (e.fail) break;
+        int operand;
+        if (other == held) operand = DVM_REG_ACC;
+        else if (e.loc[other] >= 0) operand = e.loc[other];
+        else { e.fail = true; break; }
+        memit(e, DVM_INSN(DVM_OP_BIN + op, 1, operand, 0));
+        mm_release(e, x);
+        if (y != x) mm_release(e, y);
+        e.acc = (int16_t)i;
+        break;
+      }
+      default:
+        e.fail = true;
+    }
+    if (!e.fail) mm_store_outputs_of(e, i);
+  }
+  for (int o = 0; o < p->n_outputs && !e.fail; ++o)
+    if (!e.stored[o]) mm_store_outputs_of(e, mroot(e, p->outputs[o].value));
+  return !e.fail;
+}
+
+}  // namespace
+
+int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in, const float* scalars,
+                      int n_scalars, void* code, size_t code_capacity, size_t* code_size,
+                      dvm_shape* out_shapes, int n_out) {
+  (void)n_scalars;
+  (void)n_out;
+  MmEnc e;
+  e.p = p;
+  e.scalars = scalars;
+  const int NN = p->n_nodes;
+
+  // ---- the matmul instructions: one shared A [M,K], one or two B [K,N] ----
+  int a_val = -1, b_val[2] = {-1, -1}, nb = 0;
+  for (int i = 0; i < NN; ++i) {
+    const Node& n = p->nodes[i];
+    e.alias[i] = -1;
+    e.loc[i] = -1;
+    if (n.kind == NK_MATMUL) {
+      if (nb >= 2) return DVM_ERR_UNSUPPORTED;
+      a_val = n.x;
+      b_val[nb] = n.y;
+      e.loc[i] = (int16_t)nb;  // register nb: the accumulator of this matmul
+      nb++;
+    } else if (n.kind == NK_CAST && n.dtype == DVM_F32) {
+      e.alias[i] = n.x;  // values are fp32 already
+    } else if (n.kind == NK_REDUCE) {
+      return DVM_ERR_UNSUPPORTED;
+    }
+  }
+  if (nb == 0) return DVM_ERR_INVALID_ARG;
+  if (nb == 2 && b_val[0] == b_val[1]) return DVM_ERR_UNSUPPORTED;
+  e.nb = nb;
+  int slot_of[DVM_MAX_NODES];
+  for (int i = 0; i < NN; ++i) slot_of[i] = -1;
+  for (int i = 0; i < n_in; ++i) slot_of[p->inputs[i]] = i;
+  const dvm_shape& sa = in_shapes[slot_of[a_val]];
+  if (sa.rank != 2) return DVM_ERR_UNSUPPORTED;
+  const int64_t M = sa.dims[0], K = sa.dims[1];
+  int64_t N = -1;
+  for (int j = 0; j < nb; ++j) {
+    const dvm_shape& sb = in_shapes[slot_of[b_val[j]]];
+    if (sb.rank != 2) return DVM_ERR_UNSUPPORTED;
+    if (sb.dims[0] != K) return DVM_ERR_SHAPE_MISMATCH;
+    if (N >= 0 && sb.dims[1] != N) return DVM_ERR_SHAPE_MISMATCH;
+    N = sb.dims[1];
+  }
+  if (M < 0 || N < 0 || K < 0) return DVM_ERR_INVALID_ARG;
+  // the tile loads want 16-byte row pitches; an empty inner dimension has no tensor-core form
+  if (K <= 0 || (K % 8) != 0 || (N % 8) != 0) return DVM_ERR_UNSUPPORTED;
+  if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return DVM_ERR_UNSUPPORTED;
+
+  // ---- matmul operands feed only the matmul instructions; other inputs are epilogue operands ----
+  e.n_opd = 0;
+  for (int i = 0; i < NN; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_INPUT || n.kind == NK_MATMUL) continue;
+    const int xs[2] = {n.x, n.kind == NK_BINARY ? n.y : -1};
+    for (int k = 0; k < 2; ++k)
+      if (xs[k] >= 0 && (xs[k] == a_val || xs[k] == b_val[0] || xs[k] == b_val[1])) return DVM_ERR_UNSUPPORTED;
+  }
+  for (int o = 0; o < p->n_outputs; ++o) {
+    const int v = p->outputs[o].value;
+    if (v == a_val || v == b_val[0] || v == b_val[1]) return DVM_ERR_UNSUPPORTED;
+  }
+  for (int i = 0; i < n_in; ++i) {
+    const int v = p->inputs[i];
+    if (v == a_val || v == b_val[0] || v == b_val[1]) continue;
+    const dvm_shape& s = in_shapes[i];
+    if (s.rank != p->nodes[v].rank) return DVM_ERR_INVALID_ARG;
+    if (s.rank > 2) return DVM_ERR_UNSUPPORTED;
+    int64_t r = 1, c = 1;
+    if (s.rank >= 1) c = s.dims[s.rank - 1];
+    if (s.rank == 2) r = s.dims[0];
+    if ((r != 1 && r != M) || (c != 1 && c != N)) return DVM_ERR_SHAPE_MISMATCH;
+    if (e.n_opd >= DVM_MAX_OPERANDS) return DVM_ERR_TOO_LARGE;
+    MmOperand& od = e.opd[e.n_opd];
+    od.slot = i;
+    od.dtype = p->nodes[v].dtype == DVM_BF16 ? DVM_DT_BF16 : DVM_DT_F32;
+    od.col_stride = c == 1 ? 0 : 1;
+    od.row_stride = r == 1 ? 0 : c;
+    e.loc[v] = (int16_t)(0x80 | e.n_opd);
+    e.n_opd++;
+  }
+  for (int o = 0; o < p->n_outputs; ++o) {
+    if (e.n_opd >= DVM_MAX_OPERANDS) return DVM_ERR_TOO_LARGE;
+    MmOperand& od = e.opd[e.n_opd];
+    od.slot = n_in + o;
+    od.dtype = p->outputs[o].dtype == DVM_BF16 ? DVM_DT_BF16 : DVM_DT_F32;
+    od.col_stride = 1;
+    od.row_stride = N;
+    e.out_operand[o] = (int8_t)e.n_opd++;
+    if (out_shapes) {
+      out_shapes[o].rank = 2;
+      out_shapes[o].dims[0] = M;
+      out_shapes[o].dims[1] = N;
+    }
+  }
+
+  if (!mm_gen_epilogue(e)) return DVM_ERR_UNSUPPORTED;
+
+  // ---- output tiling: 128-row blocks x (128 | 256)-column blocks; one tile = one accumulator stage ----
+  const int tile_n = nb == 2 ? 128 : 256;
+  const int64_t mb = (M + DVM_MM_BLOCK_M - 1) / DVM_MM_BLOCK_M, nbk = (N + tile_n - 1) / tile_n;
+  const int64_t kb = (K + DVM_MM_BLOCK_K - 1) / DVM_MM_BLOCK_K;
+  if (mb * nbk >= (1ll << 31)) return DVM_ERR_UNSUPPORTED;
+
+  const int nt = n_in + p->n_outputs;
+  const size_t total = DVM_HDR_WORDS + 2 * (size_t)nt + DVM_MM_WORDS + (size_t)DVM_OPD_WORDS * e.n_opd + e.n_body;
+  if (total > DVM_MM_MAX_WORDS) return DVM_ERR_TOO_LARGE;
+  *code_size = total * 4;
+  if (!code || code_capacity < total * 4) return DVM_ERR_BUFFER_TOO_SMALL;
+  uint32_t* w = (uint32_t*)code;
+  memset(w, 0, total * 4);
+  w[DVM_H_MAGIC] = DVM_MAGIC;
+  w[DVM_H_KERNEL_TYPE] = DVM_KERNEL_MATMUL;
+  w[DVM_H_CODE_WORDS] = (uint32_t)e.n_body;
+  w[DVM_H_N_TILES] = (uint32_t)(mb * nbk);
+  w[DVM_H_TOTAL_WORDS] = (uint32_t)total;
+  w[DVM_H_COUNTS] = (uint32_t)nt | ((uint32_t)n_in << 8) | ((uint32_t)e.n_opd << 16) | ((uint32_t)p->n_outputs << 24);
+  w[DVM_H_COLS] = (uint32_t)N;
+  w[DVM_H_ROWS_LO] = (uint32_t)M;
+  w[DVM_H_PRIMARY] = 0xffffffffu;
+  uint32_t* x = w + DVM_HDR_WORDS + 2 * nt;
+  x[DVM_MM_M] = (uint32_t)M;
+  x[DVM_MM_N] = (uint32_t)N;
+  x[DVM_MM_K] = (uint32_t)K;
+  x[DVM_MM_NB] = (uint32_t)nb;
+  x[DVM_MM_TILE_N] = (uint32_t)tile_n;
+  x[DVM_MM_SLOTS] = (uint32_t)slot_of[a_val] | ((uint32_t)slot_of[b_val[0]] << 8) |
+                    ((uint32_t)slot_of[b_val[nb - 1]] << 16);
+  x[DVM_MM_NTMP] = (uint32_t)e.n_tmp;
+  x[DVM_MM_MBLOCKS] = (uint32_t)mb;
+  x[DVM_MM_NBLOCKS] = (uint32_t)nbk;
+  x[DVM_MM_KBLOCKS] = (uint32_t)kb;
+  uint32_t* ot = x + DVM_MM_WORDS;
+  for (int k = 0; k < e.n_opd; ++k) {
+    uint32_t* d = ot + k * DVM_OPD_WORDS;
+    d[DVM_OPD_INFO] = (uint32_t)e.opd[k].slot | ((uint32_t)e.opd[k].dtype << 8) | ((uint32_t)e.opd[k].col_stride << 16);
+    d[DVM_OPD_STRIDE0] = (uint32_t)e.opd[k].row_stride;
+    d[DVM_OPD_STRIDE0 + 1] = (uint32_t)((uint64_t)e.opd[k].row_stride >> 32);
+  }
+  memcpy(ot + e.n_opd * DVM_OPD_WORDS, e.body, (size_t)e.n_body * 4);
+  return DVM_OK;
+}
+
+// =================================================================================================
+// Host: verifier and readable dump
+// =================================================================================================
+namespace {
+struct MmView {
+  uint32_t nt, n_in, n_opd, n_out, nb, ntmp;
+  const uint32_t *x, *ot, *body;
+  uint32_t n_body;
+};
+
+bool mm_view(const uint32_t* w, size_t n_words, MmView* v) {
+  if (n_words < DVM_HDR_WORDS || w[DVM_H_MAGIC] != DVM_MAGIC || w[DVM_H_KERNEL_TYPE] != DVM_KERNEL_MATMUL) return false;
+  const uint32_t c = w[DVM_H_COUNTS];
+  v->nt = c & 0xff; v->n_in = (c >> 8) & 0xff; v->n_opd = (c >> 16) & 0xff; v->n_out = c >> 24;
+  if (v->nt > DVM_MAX_TENSORS || v->n_opd > DVM_MAX_OPERANDS || v->n_in + v->n_out != v->nt) return false;
+  const size_t fixed = DVM_HDR_WORDS + 2 * (size_t)v->nt + DVM_MM_WORDS + (size_t)DVM_OPD_WORDS * v->n_opd;
+  v->n_body = w[DVM_H_CODE_WORDS];
+  if (w[DVM_H_TOTAL_WORDS] != n_words || fixed + v->n_body != n_words || n_words > DVM_MM_MAX_WORDS) return false;
+  v->x = w + DVM_HDR_WORDS + 2 * v->nt;
+  v->ot = v->x + DVM_MM_WORDS;
+  v->body = v->ot + v->n_opd * DVM_OPD_WORDS;
+  v->nb = v->x[DVM_MM_NB];
+  v->ntmp = v->x[DVM_MM_NTMP];
+  return true;
+}
+
+bool mm_reg_ok(const MmView& v, uint32_t r, bool allow_acc, bool temps_only) {
+  if (temps_only) return r >= v.nb && r < v.nb + v.ntmp;
+  if (r == DVM_REG_ACC) return allow_acc;
+  if (r & 0x80) {
+    const uint32_t k = r & 0x7f;
+    return k < v.n_opd && (v.ot[k * DVM_OPD_WORDS] & 0xff) < v.n_in;
+  }
+  return r < v.nb + v.ntmp;
+}
+}  // namespace
+
+int dvm_verify_matmul(const uint32_t* w, size_t n_words) {
+  MmView v;
+  if (!mm_view(w, n_words, &v)) return DVM_ERR_BAD_CODE;
+  const uint32_t* x = v.x;
+  const uint64_t M = x[DVM_MM_M], N = x[DVM_MM_N], K = x[DVM_MM_K];
+  if (v.nb < 1 || v.nb > 2 || v.ntmp > DVM_MM_MAX_TMP) return DVM_ERR_BAD_CODE;
+  if (x[DVM_MM_TILE_N] != (v.nb == 2 ? 128u : 256u)) return DVM_ERR_BAD_CODE;
+  if (K == 0 || (K % 8) || (N % 8) || (M >> 31) || (N >> 31) || (K >> 31)) return DVM_ERR_BAD_CODE;
+  const uint64_t mb = (M + DVM_MM_BLOCK_M - 1) / DVM_MM_BLOCK_M, nbk = (N + x[DVM_MM_TILE_N] - 1) / x[DVM_MM_TILE_N];
+  if (x[DVM_MM_MBLOCKS] != mb || x[DVM_MM_NBLOCKS] != nbk || w[DVM_H_N_TILES] != mb * nbk) return DVM_ERR_BAD_CODE;
+  if (x[DVM_MM_KBLOCKS] != (K + DVM_MM_BLOCK_K - 1) / DVM_MM_BLOCK_K) return DVM_ERR_BAD_CODE;
+  if (w[DVM_H_COLS] != N || w[DVM_H_ROWS_LO] != M) return DVM_ERR_BAD_CODE;
+  const uint32_t sl = x[DVM_MM_SLOTS];
+  if ((sl & 0xff) >= v.n_in || ((sl >> 8) & 0xff) >= v.n_in || ((sl >> 16) & 0xff) >= v.n_in) return DVM_ERR_BAD_CODE;
+  for (uint32_t k = 0; k < v.n_opd; ++k) {
+    const uint32_t* d = v.ot + k * DVM_OPD_WORDS;
+    const uint32_t info = d[DVM_OPD_INFO];
+    if ((info & 0xff) >= v.nt || ((info >> 8) & 0xff) > DVM_DT_BF16 || ((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
+    const uint64_t rs = d[DVM_OPD_STRIDE0] | ((uint64_t)d[DVM_OPD_STRIDE0 + 1] << 32);
+    if (rs != 0 && rs != N && rs != 1) return DVM_ERR_BAD_CODE;
+    if ((info & 0xff) >= v.n_in && (rs != N || ((info >> 16) & 0xff) != 1)) return DVM_ERR_BAD_CODE;  // outputs are dense
+  }
+  uint32_t pc = 0, stores = 0;
+  while (pc < v.n_body) {
+    const uint32_t iw = v.body[pc], op = DVM_INSN_OP(iw), len = DVM_INSN_LEN(iw), a = DVM_INSN_A(iw), b = DVM_INSN_B(iw);
+    if (len == 0 || pc + len > v.n_body) return DVM_ERR_BAD_CODE;
+    uint32_t want = 1;
+    if (op == DVM_OP_LDA) { if (!mm_reg_ok(v, a, false, false)) return DVM_ERR_BAD_CODE; }
+    else if (op == DVM_OP_STA) { if (!mm_reg_ok(v, a, false, true)) return DVM_ERR_BAD_CODE; }
+    else if (op == DVM_OP_STG) {
+      if (b >= v.n_opd || (v.ot[b * DVM_OPD_WORDS] & 0xff) < v.n_in) return DVM_ERR_BAD_CODE;
+      stores++;
+    }
+    else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) want = 2;
+    else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) { if (!mm_reg_ok(v, a, true, false)) return DVM_ERR_BAD_CODE; }
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {}
+    else return DVM_ERR_BAD_CODE;
+    if (len != want) return DVM_ERR_BAD_CODE;
+    pc += len;
+  }
+  if (stores == 0) return DVM_ERR_BAD_CODE;
+  return DVM_OK;
+}
+
+namespace {
+struct MmOut {
+  char* buf;
+  size_t cap, n;
+};
+void mm_printf(MmOut& o, const char* fmt, ...) {
+  char tmp[256];
+  va_list ap;
+  va_start(ap, fmt);
+  int k = vsnprintf(tmp, sizeof tmp, fmt, ap);
+  va_end(ap);
+  if (k < 0) return;
+  for (int i = 0; i < k && i < (int)sizeof tmp - 1; ++i) {
+    if (o.buf && o.n + 1 < o.cap) o.buf[o.n] = tmp[i];
+    o.n++;
+  }
+}
+const char* kMmArith[8] = {"add", "sub", "rsub", "mul", "div", "rdiv", "min", "max"};
+const char* kMmUn[13] = {"exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg", "recip", "floor", "round", "tanh", "rnd_bf16"};
+void mm_reg_name(const MmView& v, uint32_t r, char* out, size_t cap) {
+  if (r == DVM_REG_ACC) snprintf(out, cap, "ACC");
+  else if (r & 0x80) snprintf(out, cap, "G[%u]", r & 0x7f);
+  else if (r < v.nb) snprintf(out, cap, "MM%u", r);
+  else snprintf(out, cap, "T%u", r - v.nb);
+}
+}  // namespace
+
+int dvm_disassemble_matmul(const uint32_t* w, size_t n_words, char* buf, size_t cap) {
+  MmView v;
+  if (!mm_view(w, n_words, &v)) return DVM_ERR_BAD_CODE;
+  MmOut o = {buf, cap, 0};
+  const uint32_t* x = v.x;
+  mm_printf(o, "kernel matmul  code %u words  tiles %u (%u x %u, %u k-blocks)\n", v.n_body, w[DVM_H_N_TILES],
+            x[DVM_MM_MBLOCKS], x[DVM_MM_NBLOCKS], x[DVM_MM_KBLOCKS]);
+  mm_printf(o, "  M %u  N %u  K %u  B matrices %u  tile 128 x %u  temporaries %u\n", x[DVM_MM_M], x[DVM_MM_N],
+            x[DVM_MM_K], v.nb, x[DVM_MM_TILE_N], v.ntmp);
+  const uint32_t sl = x[DVM_MM_SLOTS];
+  for (uint32_t j = 0; j < v.nb; ++j)
+    mm_printf(o, "  MATMUL MM%u = slot%u x slot%u\n", j, sl & 0xff, (sl >> (8 + 8 * j)) & 0xff);
+  for (uint32_t k = 0; k < v.n_opd; ++k) {
+    const uint32_t* d = v.ot + k * DVM_OPD_WORDS;
+    const uint32_t info = d[DVM_OPD_INFO];
+    mm_printf(o, "  operand %u: slot%u %s row_stride %u col_stride %u\n", k, info & 0xff,
+              ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", d[DVM_OPD_STRIDE0], (info >> 16) & 0xff);
+  }
+  uint32_t pc = 0;
+  char r[16];
+  while (pc < v.n_body) {
+    const uint32_t iw = v.body[pc], op = DVM_INSN_OP(iw), len = DVM_INSN_LEN(iw), a = DVM_INSN_A(iw), b = DVM_INSN_B(iw);
+    if (len == 0 || pc + len > v.n_body) return DVM_ERR_BAD_CODE;
+    mm_reg_name(v, a, r, sizeof r);
+    if (op == DVM_OP_LDA) mm_printf(o, "  %3u: LDA   ACC = %s\n", pc, r);
+    else if (op == DVM_OP_STA) mm_printf(o, "  %3u: STA   %s = ACC\n", pc, r);
+    else if (op == DVM_OP_STG) mm_printf(o, "  %3u: STG   operand %u = ACC\n", pc, b);
+    else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) {
+      float f;
+      memcpy(&f, &v.body[pc + 1], 4);
+      mm_printf(o, "  %3u: BINI  ACC = ACC %s %g\n", pc, kMmArith[op & 7], f);
+    } else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) mm_printf(o, "  %3u: BIN   ACC = ACC %s %s\n", pc, kMmArith[op & 7], r);
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) mm_printf(o, "  %3u: UN    ACC = %s(ACC)\n", pc, kMmUn[op - DVM_OP_UN]);
+    else return DVM_ERR_BAD_CODE;
+    pc += len;
+  }
+  if (buf && cap) buf[o.n < cap ? o.n : cap - 1] = 0;
+  return o.n < cap ? DVM_OK : DVM_ERR_BUFFER_TOO_SMALL;
+}
+
+// =================================================================================================
+// Device
+// =================================================================================================
+namespace dvm {
+namespace mm {
+
+constexpr int BLOCK_M = DVM_MM_BLOCK_M, BLOCK_K = DVM_MM_BLOCK_K, CHUNK = DVM_MM_CHUNK;
+constexpr int ACC_COLS = 256;                       // accumulator columns of one tile (one UMMA N)
+constexpr uint32_t STAGE_A = BLOCK_M * BLOCK_K * 2; // 16 KB: 128 rows of 128 bytes
+constexpr uint32_t BOX_B = 64 * BLOCK_K * 2;        // 8 KB: 64 k-rows of 64 columns
+constexpr uint32_t STAGE_BYTES = STAGE_A + 4 * BOX_B;  // 48 KB
+constexpr int MAX_STAGES = 4;
+constexpr uint32_t TMP_BYTES = 128 * CHUNK * 4;     // one epilogue temporary: 16 KB
+constexpr int THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_NS = 2000000000ull;   // limit of one wait: 2 s
+constexpr unsigned long long DRAIN_NS = 200000000ull;   // limit of a wait for work in flight after an abort
+constexpr uint32_t WAIT_SPINS = 1u << 27;
+
+struct MMParams {
+  unsigned int* status;
+  uint32_t n_words;
+  uint32_t n_stages;
+  uint32_t words[DVM_MM_MAX_WORDS];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long gtimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after limit_ns (or WAIT_SPINS polls), raising the CTA's abort flag; with
+// heed_abort it also gives up as soon as another role has raised the flag.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            unsigned long long limit_ns, bool heed_abort) {
+  const unsigned long long t0 = gtimer();
+  for (uint32_t spin = 0; spin < WAIT_SPINS; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if (heed_abort && *abort_flag) return false;
+    if (gtimer() - t0 > limit_ns) break;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, WAIT_NS, true);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrive once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive accumulator columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[CHUNK]) {
+  uint32_t r[CHUNK];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < CHUNK; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptors (128-byte swizzle, sm_100 descriptor version 1).
+// A tile, K-major: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3fff) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// B tile, N-major: 64-column boxes 8192 bytes apart (leading offset), 8-deep k groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_n_major(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3fff) | ((uint64_t)(BOX_B >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = 256
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                           ((uint32_t)(ACC_COLS >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+
+__device__ __forceinline__ float mm_arith(int op, float a, float b) { return scalar_arith(op, a, b); }
+
+__global__ void __launch_bounds__(THREADS, 1)
+dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+              const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ MMParams prm) {
+#define MW(i) (prm.words[(i)])
+  extern __shared__ uint8_t mm_smem_raw[];
+  const uint32_t raw = smem_u32(mm_smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
+  uint8_t* const sm = mm_smem_raw + (base - raw);
+
+  const uint32_t nt = MW(DVM_H_COUNTS) & 0xff, n_opd = (MW(DVM_H_COUNTS) >> 16) & 0xff;
+  const uint32_t XO = DVM_HDR_WORDS + 2 * nt;       // matmul extension
+  const uint32_t OT = XO + DVM_MM_WORDS;            // operand table
+  const uint32_t CODE = OT + n_opd * DVM_OPD_WORDS; // epilogue code
+  const uint32_t code_end = CODE + MW(DVM_H_CODE_WORDS);
+  const int M = (int)MW(XO + DVM_MM_M), N = (int)MW(XO + DVM_MM_N);
+  const int nb = (int)MW(XO + DVM_MM_NB), tile_n = (int)MW(XO + DVM_MM_TILE_N);
+  const int ntmp = (int)MW(XO + DVM_MM_NTMP);
+  const uint32_t m_blocks = MW(XO + DVM_MM_MBLOCKS), k_blocks = MW(XO + DVM_MM_KBLOCKS);
+  const uint32_t n_tiles = MW(DVM_H_N_TILES);
+  const uint32_t n_stages = prm.n_stages;
+
+  const uint32_t tmp_base = n_stages * STAGE_BYTES;                 // byte offsets from `base`
+  const uint32_t bar_base = base + tmp_base + (uint32_t)ntmp * TMP_BYTES;
+  // barriers: full[4] empty[4] tmem_full[2] tmem_empty[2] drain
+  const uint32_t bar_full = bar_base, bar_empty = bar_base + 32, bar_tfull = bar_base + 64, bar_tempty = bar_base + 80,
+                 bar_drain = bar_base + 96;
+  uint32_t* const tmem_slot = (uint32_t*)(sm + tmp_base + (uint32_t)ntmp * TMP_BYTES + 112);
+  volatile uint32_t* const abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < MAX_STAGES; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (uint32_t a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8 * a, 1);
+      mbar_init(bar_tempty + 8 * a, 128);
+    }
+    mbar_init(bar_drain, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // tensor memory: both accumulator stages
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)tmem_slot;
+
+  uint32_t issued = 0, p_stage = 0, p_phase = 0;  // producer state, kept for the abort path
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
+        for (uint32_t kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(bar_empty + 8 * p_stage, p_phase ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t full = bar_full + 8 * p_stage;
+          const uint32_t sa = base + p_stage * STAGE_BYTES;
+          mbar_expect_tx(full, STAGE_BYTES);
+          const int k0 = (int)kb * BLOCK_K;
+          tma_load_2d(sa, &tmA, full, k0, m0);
+          if (nb == 2) {
+            tma_load_2d(sa + STAGE_A, &tmB0, full, n0, k0);
+            tma_load_2d(sa + STAGE_A + BOX_B, &tmB0, full, n0 + 64, k0);
+            tma_load_2d(sa + STAGE_A + 2 * BOX_B, &tmB1, full, n0, k0);
+            tma_load_2d(sa + STAGE_A + 3 * BOX_B, &tmB1, full, n0 + 64, k0);
+          } else {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) tma_load_2d(sa + STAGE_A + b * BOX_B, &tmB0, full, n0 + 64 * b, k0);
+          }
+          ++issued;
+          if (++p_stage == n_stages) { p_stage = 0; p_phase ^= 1; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, it = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+        const uint32_t as = it & 1, aph = (it >> 1) & 1;
+        if (!mbar_wait(bar_tempty + 8 * as, aph ^ 1, abort_flag)) break;  // the epilogue has drained this stage
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * ACC_COLS;
+        for (uint32_t kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint64_t adesc = desc_k_major(sa), bdesc = desc_n_major(sa + STAGE_A);
+#pragma unroll
+          for (uint32_t j = 0; j < BLOCK_K / 16; ++j)  // K = 16 per instruction: 32 bytes along A's rows, two k groups of B
+            umma_bf16(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC, (kb | j) != 0);
+          umma_commit(bar_empty + 8 * stage);  // the stage is free once these MMAs have read it
+          if (++stage == n_stages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(bar_tfull + 8 * as);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue interpreter ----------------
+    const int q = warp & 3;                 // tensor-memory lane quadrant this warp may read
+    const int erow = q * 32 + lane;         // row of the tile
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    float* const tmp_mine = (float*)(sm + tmp_base) + erow * 4;
+    uint32_t it = 0;
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+      const uint32_t as = it & 1, aph = (it >> 1) & 1;
+      const bool got = mbar_wait(bar_tfull + 8 * as, aph, abort_flag);
+      if (!__all_sync(0xffffffffu, got)) break;
+      tc_fence_after();
+      const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
+      const int row = m0 + erow;
+      const bool row_ok = row < M;
+      const int n_chunks = tile_n / CHUNK;
+      for (int c = 0; c < n_chunks; ++c) {
+        const int col0 = n0 + c * CHUNK;
+        if (col0 >= N) break;
+        const uint32_t acc_addr = lane_addr + as * ACC_COLS + (uint32_t)(c * CHUNK);
+        float acc[CHUNK];
+#pragma unroll
+        for (int i = 0; i < CHUNK; ++i) acc[i] = 0.0f;
+
+        // operand `a` of LDA / BIN as CHUNK fp32 values
+        auto fetch = [&](uint32_t a, float (&v)[CHUNK]) {
+          if (a < (uint32_t)nb) {
+            tmem_ld32(acc_addr + a * 128u, v);
+          } else if (a < 0x80u) {
+            const float4* src = (const float4*)(tmp_mine + (a - nb) * (TMP_BYTES / 4));
+#pragma unroll
+            for (int j = 0; j < CHUNK / 4; ++j) {
+              const float4 f = src[j * 128];
+              v[4 * j] = f.x; v[4 * j + 1] = f.y; v[4 * j + 2] = f.z; v[4 * j + 3] = f.w;
+            }
+          } else {
+            const uint32_t od = OT + (a & 0x7fu) * DVM_OPD_WORDS;
+            const uint32_t info = MW(od + DVM_OPD_INFO);
+            const uint32_t slot = info & 0xff;
+            const char* ptr = (const char*)(((unsigned long long)MW(DVM_HDR_WORDS + 2 * slot + 1) << 32) | MW(DVM_HDR_WORDS + 2 * slot));
+            const long long rs = (long long)(((unsigned long long)MW(od + DVM_OPD_STRIDE0 + 1) << 32) | MW(od + DVM_OPD_STRIDE0));
+            const int cs = (info >> 16) & 0xff;
+            const bool bf = ((info >> 8) & 0xff) == DVM_DT_BF16;
+            const long long off = (long long)row * rs + (long long)col0 * cs;
+#pragma unroll
+            for (int i = 0; i < CHUNK; ++i) {
+              float x = 0.0f;
+              if (row_ok && col0 + i < N) {
+                const long long e = off + (long long)i * cs;
+                x = bf ? __bfloat162float(((const __nv_bfloat16*)ptr)[e]) : ((const float*)ptr)[e];
+              }
+              v[i] = x;
+            }
+          }
+        };
+
+        for (uint32_t pc = CODE; pc < code_end;) {
+          const uint32_t iw = MW(pc);
+          const uint32_t op = DVM_INSN_OP(iw), a = DVM_INSN_A(iw);
+          if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) {
+            const int sub = op & 7;
+            if (a == DVM_REG_ACC) {
+#pragma unroll
+              for (int i = 0; i < CHUNK; ++i) acc[i] = mm_arith(sub, acc[i], acc[i]);
+            } else {
+              float v[CHUNK];
+              fetch(a, v);
+              switch (sub) {
+                case DVM_A_ADD:
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i) acc[i] = acc[i] + v[i];
+                  break;
+                case DVM_A_MUL:
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i) acc[i] = acc[i] * v[i];
+                  break;
+                default:
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i) acc[i] = mm_arith(sub, acc[i], v[i]);
+              }
+            }
+          } else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
+            const int u = op - DVM_OP_UN;
+            if (u == DVM_U_SIGMOID) {
+#pragma unroll
+              for (int i = 0; i < CHUNK; ++i) acc[i] = fast_rcp(1.0f + fast_exp(-acc[i]));
+            } else {
+#pragma unroll 4
+              for (int i = 0; i < CHUNK; ++i) acc[i] = scalar_unary(u, acc[i]);
+            }
+          } else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) {
+            const float imm = __uint_as_float(MW(pc + 1));
+            const int sub = op & 7;
+#pragma unroll
+            for (int i = 0; i < CHUNK; ++i) acc[i] = mm_arith(sub, acc[i], imm);
+          } else if (op == DVM_OP_LDA) {
+            fetch(a, acc);
+          } else if (op == DVM_OP_STA) {
+            float4* dst = (float4*)(tmp_mine + (a - nb) * (TMP_BYTES / 4));
+#pragma unroll
+            for (int j = 0; j < CHUNK / 4; ++j) dst[j * 128] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+          } else if (op == DVM_OP_STG) {
+            const uint32_t od = OT + DVM_INSN_B(iw) * DVM_OPD_WORDS;
+            const uint32_t info = MW(od + DVM_OPD_INFO);
+            const uint32_t slot = info & 0xff;
+            char* ptr = (char*)(((unsigned long long)MW(DVM_HDR_WORDS + 2 * slot + 1) << 32) | MW(DVM_HDR_WORDS + 2 * slot));
+            const bool bf = ((info >> 8) & 0xff) == DVM_DT_BF16;
+            const bool vec = (((unsigned long long)ptr) & 15) == 0;  // N is a multiple of 8, col0 of 32
+            if (row_ok) {
+              const long long e0 = (long long)row * N + col0;
+              if (bf) {
+                __nv_bfloat16* o = (__nv_bfloat16*)ptr + e0;
+                if (vec) {
+#pragma unroll
+                  for (int g = 0; g < CHUNK / 8; ++g) {
+                    if (col0 + 8 * g < N) {
+                      uint4 pk;
+                      __nv_bfloat162 h;
+                      h = __floats2bfloat162_rn(acc[8 * g], acc[8 * g + 1]);     pk.x = *(uint32_t*)&h;
+                      h = __floats2bfloat162_rn(acc[8 * g + 2], acc[8 * g + 3]); pk.y = *(uint32_t*)&h;
+                      h = __floats2bfloat162_rn(acc[8 * g + 4], acc[8 * g + 5]); pk.z = *(uint32_t*)&h;
+                      h = __floats2bfloat162_rn(acc[8 * g + 6], acc[8 * g + 7]); pk.w = *(uint32_t*)&h;
+                      *(uint4*)(o + 8 * g) = pk;
+                    }
+                  }
+                } else {
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i)
+                    if (col0 + i < N) o[i] = __float2bfloat16_rn(acc[i]);
+                }
+              } else {
+                float* o = (float*)ptr + e0;
+                if (vec) {
+#pragma unroll
+                  for (int g = 0; g < CHUNK / 4; ++g)
+                    if (col0 + 4 * g < N) *(float4*)(o + 4 * g) = make_float4(acc[4 * g], acc[4 * g + 1], acc[4 * g + 2], acc[4 * g + 3]);
+                } else {
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i)
+                    if (col0 + i < N) o[i] = acc[i];
+                }
+              }
+            }
+          }
+          pc += DVM_INSN_LEN(iw);
+        }
+      }
+      // this accumulator stage may be overwritten by the tile after next
+      tc_fence_before();
+      mbar_arrive(bar_tempty + 8 * as);
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (warp == 0 && lane == 0) {
+      // wait (bounded) for the tile loads still in flight: the latest fill of every stage
+      uint32_t s = p_stage, ph = p_phase;
+      const uint32_t n = issued < n_stages ? issued : n_stages;
+      for (uint32_t i = 0; i < n; ++i) {
+        if (s == 0) { s = n_stages - 1; ph ^= 1; } else --s;
+        if (!mbar_try(bar_full + 8 * s, ph)) mbar_wait_slow(bar_full + 8 * s, ph, abort_flag, DRAIN_NS, false);
+      }
+    }
+    if (warp == 1 && lane == 0) {
+      // wait (bounded) for every MMA issued so far
+      umma_commit(bar_drain);
+      if (!mbar_try(bar_drain, 0)) mbar_wait_slow(bar_drain, 0, abort_flag, DRAIN_NS, false);
+    }
+    if (threadIdx.x == 0) atomicMax(prm.status, (unsigned int)ST_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+#undef MW
+}
+
+}  // namespace mm
+}  // namespace dvm
+
+// =================================================================================================
+// Host: launch
+// =================================================================================================
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_mm_mu;
+EncodeTiledFn g_encode_tiled = nullptr;
+bool g_attr_set[64] = {};
+
+int mm_encode_fn(EncodeTiledFn* out) {
+  std::lock_guard<std::mutex> lk(g_mm_mu);
+  if (!g_encode_tiled) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+      dvm_note_cuda_error(e != cudaSuccess ? (int)e : (int)cudaErrorNotSupported);
+      return DVM_ERR_CUDA;
+    }
+    g_encode_tiled = (EncodeTiledFn)fn;
+  }
+  *out = g_encode_tiled;
+  return DVM_OK;
+}
+
+// A row-major bf16 matrix [rows, cols] as a 2-D tensor map with a (box_cols x box_rows) box, 128-byte swizzle.
+int mm_make_map(EncodeTiledFn fn, CUtensorMap* map, void* ptr, uint64_t rows, uint64_t cols, uint32_t box_cols,
+                uint32_t box_rows) {
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {cols * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    dvm_note_cuda_error((int)cudaErrorInvalidValue);
+    return DVM_ERR_CUDA;
+  }
+  return DVM_OK;
+}
+
+}  // namespace
+
+int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors, int n_tensors, cudaStream_t stream) {
+  MmView v;
+  if (!mm_view(code, n_words, &v)) return DVM_ERR_BAD_CODE;
+  if ((uint32_t)n_tensors != v.nt) return DVM_ERR_INVALID_ARG;
+  if (code[DVM_H_N_TILES] == 0) return DVM_OK;  // an empty output launches nothing
+  for (int i = 0; i < n_tensors; ++i)
+    if (!tensors[i]) return DVM_ERR_INVALID_ARG;
+  const uint32_t* x = v.x;
+  const uint64_t M = x[DVM_MM_M], N = x[DVM_MM_N], K = x[DVM_MM_K];
+
+  DvmDeviceInfo dev;
+  int st = dvm_device_state(&dev);
+  if (st != DVM_OK) return st;
+
+  static thread_local dvm::mm::MMParams P;
+  memcpy(P.words, code, n_words * 4);
+  for (uint32_t i = 0; i < v.nt; ++i) {
+    const unsigned long long a = (unsigned long long)(uintptr_t)tensors[i];
+    P.words[DVM_HDR_WORDS + 2 * i] = (uint32_t)a;
+    P.words[DVM_HDR_WORDS + 2 * i + 1] = (uint32_t)(a >> 32);
+  }
+  for (uint32_t k = 0; k < v.n_opd; ++k) {
+    const uint32_t info = v.ot[k * DVM_OPD_WORDS];
+    const uintptr_t es = ((info >> 8) & 0xff) == DVM_DT_BF16 ? 2 : 4;
+    if ((uintptr_t)tensors[info & 0xff] % es) return DVM_ERR_INVALID_ARG;
+  }
+  const uint32_t sl = x[DVM_MM_SLOTS];
+  void* pa = tensors[sl & 0xff];
+  void* pb0 = tensors[(sl >> 8) & 0xff];
+  void* pb1 = tensors[(sl >> 16) & 0xff];
+  // the tile loads need 16-byte aligned matrices
+  if (((uintptr_t)pa | (uintptr_t)pb0 | (uintptr_t)pb1) & 15) return DVM_ERR_INVALID_ARG;
+
+  EncodeTiledFn fn;
+  st = mm_encode_fn(&fn);
+  if (st != DVM_OK) return st;
+  CUtensorMap ma, mb0, mb1;
+  if ((st = mm_make_map(fn, &ma, pa, M, K, DVM_MM_BLOCK_K, DVM_MM_BLOCK_M)) != DVM_OK) return st;
+  if ((st = mm_make_map(fn, &mb0, pb0, K, N, 64, DVM_MM_BLOCK_K)) != DVM_OK) return st;
+  if ((st = mm_make_map(fn, &mb1, pb1, K, N, 64, DVM_MM_BLOCK_K)) != DVM_OK) return st;
+
+  const uint32_t n_stages = dvm::mm::MAX_STAGES;
+  const size_t smem = 1024 + (size_t)n_stages * dvm::mm::STAGE_BYTES + (size_t)v.ntmp * dvm::mm::TMP_BYTES + 128;
+  int devid = 0;
+  DVM_CUDA(cudaGetDevice(&devid));
+  {
+    std::lock_guard<std::mutex> lk(g_mm_mu);
+    if (devid >= 0 && devid < 64 && !g_attr_set[devid]) {
+      DVM_CUDA(cudaFuncSetAttribute(dvm::mm::dvm_mm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024));
+      g_attr_set[devid] = true;
+    }
+  }
+  P.status = dev.scratch;
+  P.n_words = (uint32_t)n_words;
+  P.n_stages = n_stages;
+  const uint32_t tiles = code[DVM_H_N_TILES];
+  const int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
+  dvm::mm::dvm_mm_kernel<<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);
+  DVM_CUDA(cudaGetLastError());
+  dvm_count_launch();
+  return DVM_OK;
+}

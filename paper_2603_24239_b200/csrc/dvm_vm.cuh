@@ -41,6 +41,8 @@
 #include <stdint.h>
 
 #include "dvm_format.h"
+#include "dvm_launch.h"
+#include "dvm_math.cuh"
 
 namespace dvm {
 
@@ -49,8 +51,6 @@ constexpr int THREADS = DVM_VM_THREADS;
 #define DVM_VM_MIN_CTAS 2
 #endif
 
-// Device status word values (read back by dvm_last_device_status).
-enum { ST_OK = 0, ST_BAD_CODE = 1, ST_TIMEOUT = 2 };
 
 template <int PW>
 struct VMParams {
@@ -89,62 +89,6 @@ __device__ __forceinline__ float sget(const float (&S)[DVM_MAX_SREGS], int k) {
 __device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) {
 #pragma unroll
   for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = (k == i) ? v : S[i];
-}
-
-__device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
-
-// exp(x) = 2^(x * log2 e) with the product carried in two fp32 pieces (t exact to 2^-24 |t|, plus the
-// rounding residual of the multiply and the low part of log2 e), the power of two from the SFU
-// (ex2.approx, relative error <= 2^-22) and a first-order correction: about 3e-7 relative error over the
-// whole finite range, in 7 instructions instead of expf's ~12.
-__device__ __forceinline__ float fast_exp(float x) {
-  const float L2E_HI = 1.44269502162933349609375f, L2E_LO = 1.925963033500011e-8f;
-  const float t = x * L2E_HI;
-  float r = __fmaf_rn(x, L2E_HI, -t);
-  r = __fmaf_rn(x, L2E_LO, r);
-  float p;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(t));
-  // outside the finite range (t = +-inf from a masked score, overflow, NaN) the SFU value stands alone:
-  // exp(-inf) must be exactly +0
-  return fabsf(t) < 126.0f ? __fmaf_rn(p * r, 0.693147182464599609375f, p) : p;
-}
-// reciprocal and quotient from the SFU (rcp.approx, 1 ulp): 2 ulp quotients
-__device__ __forceinline__ float fast_rcp(float x) {
-  float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ float fast_div(float a, float b) { return __fdividef(a, b); }
-
-__device__ __forceinline__ float scalar_arith(int op, float a, float b) {
-  switch (op) {
-    case DVM_A_ADD: return a + b;
-    case DVM_A_SUB: return a - b;
-    case DVM_A_RSUB: return b - a;
-    case DVM_A_MUL: return a * b;
-    case DVM_A_DIV: return fast_div(a, b);
-    case DVM_A_RDIV: return fast_div(b, a);
-    case DVM_A_MIN: return a < b ? a : b;
-    default: return a > b ? a : b;
-  }
-}
-
-__device__ __forceinline__ float scalar_unary(int op, float x) {
-  switch (op) {
-    case DVM_U_EXP: return fast_exp(x);
-    case DVM_U_SQRT: return sqrtf(x);
-    case DVM_U_RSQRT: return rsqrtf(x);
-    case DVM_U_ABS: return fabsf(x);
-    case DVM_U_LOG: return logf(x);
-    case DVM_U_ERF: return erff(x);
-    case DVM_U_SIGMOID: return fast_rcp(1.0f + fast_exp(-x));
-    case DVM_U_NEG: return -x;
-    case DVM_U_RECIP: return fast_rcp(x);
-    case DVM_U_FLOOR: return floorf(x);
-    case DVM_U_ROUND: return rintf(x);
-    case DVM_U_TANH: return tanhf(x);
-    default: return round_bf16(x);
-  }
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {

@@ -1,0 +1,161 @@
+"""GPU parity of the matmul meta-kernel (tcgen05 matmul instruction + interpreted epilogue) against the
+CPU oracle: every output element at small sizes (ragged M, N and K tails, several tiles), sampled rows at
+the full size of config 5, special cases with exact answers, and epilogues with extra operands."""
+import numpy as np
+import pytest
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from tests.parity_util import check, gate_errors, gpu_run, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+R_BF16 = 2e-2  # bf16 programs, fp32 accumulation
+
+
+def _mlp_inputs(M, K, N, seed):
+    x = wl.randn((M, K), torch.bfloat16, seed)
+    wg = wl.randn((K, N), torch.bfloat16, seed + 1, std=0.02)
+    wu = wl.randn((K, N), torch.bfloat16, seed + 2, std=0.02)
+    return [x, wg, wu]
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 64, 128), (7, 64, 128), (128, 64, 128), (129, 128, 256), (77, 200, 264),
+                                   (300, 1024, 392), (257, 4096, 512), (128, 72, 8), (5, 8, 8)])
+def test_mlp_gate_small(M, K, N):
+    """out = SiLU(X Wg) * (X Wu): every element, row-scaled gate at 2e-2."""
+    ins = _mlp_inputs(M, K, N, seed=M + N)
+    outs, code = gpu_run(wl.program_mlp_gate(), ins)
+    want = oracle_run(wl.program_mlp_gate(), ins)
+    g1, _ = check(wl.program_mlp_gate(), outs, want)
+    assert not torch.isnan(outs[0].float()).any()  # every element of the poisoned output was written
+
+
+def test_mlp_gate_config_shape_rows():
+    """Config 5 geometry (K = 4096, N = 11008) at a token count the oracle finishes in seconds."""
+    M, K, N = 200, 4096, 11008
+    w = wl.mlp_weights(K, N)
+    ins = wl.inputs_mlp_gate(M, K, N, seed=wl.data_seed("c5", 0), weights=w)
+    outs, _ = gpu_run(wl.program_mlp_gate(), ins)
+    want = oracle_run(wl.program_mlp_gate(), ins)
+    check(wl.program_mlp_gate(), outs, want)
+
+
+def test_mlp_gate_full_size_sampled_rows():
+    """M = 4096 (the largest instance of config 5, the launch the bench times): 48 sampled rows, one by one."""
+    M, K, N = 4096, 4096, 11008
+    w = wl.mlp_weights(K, N)
+    ins = wl.inputs_mlp_gate(M, K, N, seed=wl.data_seed("c5", 1), weights=w)
+    outs, _ = gpu_run(wl.program_mlp_gate(), ins)
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 127, 128, 4095], rng.integers(0, M, 44)]))
+    sub = [ins[0][rows], ins[1], ins[2]]
+    want = oracle_run(wl.program_mlp_gate(), sub)
+    got = wl.to_f64(outs[0])[rows]
+    g1, _ = gate_errors(got, want[0])
+    assert g1 <= R_BF16, g1
+    assert not torch.isnan(outs[0].float()).any()
+
+
+def _plain_matmul(out_dtype="bf16"):
+    p = wl.OpProgram("matmul")
+    a, b = p.input("bf16", 2), p.input("bf16", 2)
+    p.output(p.matmul(a, b), out_dtype)
+    return p
+
+
+@pytest.mark.parametrize("M,K,N", [(64, 64, 256), (130, 136, 520), (1, 4096, 264)])
+def test_plain_matmul_f32_out(M, K, N):
+    """One B matrix (256-column tiles), fp32 output: products of bf16 are exact in fp32, so only the
+    accumulation order differs from the oracle: 1e-5 row-scaled."""
+    a = wl.randn((M, K), torch.bfloat16, 11)
+    b = wl.randn((K, N), torch.bfloat16, 12)
+    prog = _plain_matmul("f32")
+    outs, _ = gpu_run(prog, [a, b])
+    want = oracle_run(prog, [a, b])
+    g1, _ = gate_errors(wl.to_f64(outs[0]), want[0])
+    assert g1 <= 1e-5, g1
+
+
+def test_identity_picks_out_b():
+    """X = I (K = 128) returns B exactly, element by element (each product has a single non-zero term)."""
+    K, N = 128, 384
+    b = wl.randn((K, N), torch.bfloat16, 3)
+    a = torch.eye(K, dtype=torch.bfloat16)
+    outs, _ = gpu_run(_plain_matmul("bf16"), [a, b])
+    assert torch.equal(outs[0].cpu(), b)
+
+
+def test_permutation_rows():
+    """A row permutation matrix as X permutes the rows of B exactly (catches a transposed or swizzled operand)."""
+    K, N = 192, 264
+    perm = torch.randperm(K, generator=torch.Generator().manual_seed(4))
+    a = torch.zeros((K, K), dtype=torch.bfloat16)
+    a[torch.arange(K), perm] = 1
+    b = wl.randn((K, N), torch.bfloat16, 5)
+    outs, _ = gpu_run(_plain_matmul("bf16"), [a, b])
+    assert torch.equal(outs[0].cpu(), b[perm])
+
+
+def test_zero_gate_gives_zero():
+    M, K, N = 100, 256, 256
+    x = wl.randn((M, K), torch.bfloat16, 1)
+    wu = wl.randn((K, N), torch.bfloat16, 2)
+    outs, _ = gpu_run(wl.program_mlp_gate(), [x, torch.zeros((K, N), dtype=torch.bfloat16), wu])
+    assert torch.all(outs[0] == 0)
+
+
+def test_all_ones_closed_form():
+    """All-ones operands: g = u = K, out = K * sigmoid(K) * K."""
+    M, K, N = 130, 64, 136
+    one = lambda *s: torch.ones(s, dtype=torch.bfloat16)
+    outs, _ = gpu_run(wl.program_mlp_gate(), [one(M, K), one(K, N), one(K, N)])
+    want = torch.tensor(K * K / (1 + np.exp(-K)), dtype=torch.float64).to(torch.bfloat16)
+    assert torch.all(outs[0].cpu() == want)
+
+
+def test_epilogue_with_extra_operands_and_temporaries():
+    """addmm-like epilogue: bias row vector, residual matrix, a column vector, two outputs, a spilled value."""
+    M, K, N = 150, 192, 392
+    p = wl.OpProgram("addmm_chain")
+    x, w = p.input("bf16", 2), p.input("bf16", 2)
+    bias, res, colv = p.input("f32", 1), p.input("bf16", 2), p.input("f32", 2)
+    g = p.matmul(x, w)
+    t = p.binary("add", g, bias)
+    u = p.binary("sub", res, p.unary("tanh", t))
+    v = p.binary("mul", p.binary("mul", u, t), colv)
+    p.output(p.scalar("muls", v, 0.5), "f32")
+    p.output(t, "bf16")
+    ins = [wl.randn((M, K), torch.bfloat16, 1), wl.randn((K, N), torch.bfloat16, 2, std=0.05),
+           wl.randn((N,), torch.float32, 3), wl.randn((M, N), torch.bfloat16, 4), wl.randn((M, 1), torch.float32, 5)]
+    outs, code = gpu_run(p, ins)
+    want = oracle_run(p, ins)
+    check(p, outs, want)
+
+
+def test_two_launches_same_code_other_buffers():
+    """Bytecode holds tensor slots, not addresses: one encoded program runs on other buffers."""
+    M, K, N = 140, 128, 256
+    prog = wl.program_mlp_gate()
+    p = dvm.program_from_nodes(prog.nodes)
+    code = dvm.encode(p, [(M, K), (K, N), (K, N)])
+    for seed in (1, 2):
+        ins = _mlp_inputs(M, K, N, seed)
+        dev = [t.cuda() for t in ins]
+        out = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        dvm.launch(code, dev + [out])
+        assert dvm.last_device_status() == 0
+        check(prog, [out], oracle_run(prog, ins))
+
+
+def test_empty_m_launches_nothing():
+    prog = wl.program_mlp_gate()
+    p = dvm.program_from_nodes(prog.nodes)
+    code = dvm.encode(p, [(0, 64), (64, 128), (64, 128)])
+    x = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((64, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((0, 128), dtype=torch.bfloat16, device="cuda")
+    n0 = dvm.launch_count()
+    dvm.launch(code, [x, w, w.clone(), out])
+    assert dvm.launch_count() == n0
