@@ -7,7 +7,7 @@ dvm_launch_stacked); nothing is cached between instances.  The default
 workload is the fused residual-add + RMSNorm sweep (200 instances, bf16
 [B*S, 4096], B in 1..32, S in 1..8192).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4] [--impl dvm|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl dvm|reference]
 
 Prints one JSON line (rank 0).  `value` is algorithmic GB/s of the whole job
 with inputs resident in HBM; `e2e` is the same metric through dvm_run_host
@@ -193,15 +193,16 @@ class C2Workload:
     def oracle_sample(self, budget_s=12.0):
         from oracle import dvm_oracle as orc
         H = self.hidden
-        rows = 256
-        x = wl.to_f64(self.x[:rows]); r = wl.to_f64(self.res[:rows]); w = wl.to_f64(self.w)
-        t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [x, r, w]); dt = time.perf_counter() - t0
-        rows = int(min(self.pool_rows, max(256, rows * budget_s / max(dt, 1e-4))))
-        rows = min(rows, 32768)
-        x = wl.to_f64(self.x[:rows]); r = wl.to_f64(self.res[:rows])
-        t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [x, r, w]); dt = time.perf_counter() - t0
-        nbytes = rows * H * 8 + H * 2
-        return nbytes / dt / 1e9, dt, f"first {rows} rows x {H} of the c2 pools (one instance), numpy float64"
+        w = wl.to_f64(self.w)
+        rows, t_all, done, off = min(8192, self.pool_rows), 0.0, 0, 0
+        while t_all < budget_s:
+            if off + rows > self.pool_rows:
+                off = 0
+            x = wl.to_f64(self.x[off:off + rows]); r = wl.to_f64(self.res[off:off + rows])
+            t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [x, r, w]); t_all += time.perf_counter() - t0
+            done += rows; off += rows
+        nbytes = done * H * 8 + H * 2
+        return nbytes / t_all / 1e9, t_all, f"{done} rows x {H} of the c2 pools in windows of {rows} rows, numpy float64"
 
 
 class C3Workload:
@@ -281,16 +282,17 @@ class C3Workload:
 
     def oracle_sample(self, budget_s=12.0):
         from oracle import dvm_oracle as orc
-        S, B, Hh = 512, 1, 4
+        S, B, Hh = 512, 1, 8
         n = B * Hh * S * S
-        sc = wl.to_f64(self.scores[:n]).reshape(B, Hh, S, S)
         m = wl.to_f64(wl.causal_mask(S))
-        t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [sc, m]); dt = time.perf_counter() - t0
-        Hh = int(max(4, min(64, Hh * budget_s / max(dt, 1e-4))))
-        n = B * Hh * S * S
-        sc = wl.to_f64(self.scores[:n]).reshape(B, Hh, S, S)
-        t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [sc, m]); dt = time.perf_counter() - t0
-        return (n * 4 + 2 * S * S) / dt / 1e9, dt, f"scores [1,{Hh},{S},{S}] from the c3 pool, numpy float64"
+        t_all, done, off = 0.0, 0, 0
+        while t_all < budget_s:
+            if off + n > self.pool:
+                off = 0
+            sc = wl.to_f64(self.scores[off:off + n]).reshape(B, Hh, S, S)
+            t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [sc, m]); t_all += time.perf_counter() - t0
+            done += 1; off += n
+        return done * (n * 4 + 2 * S * S) / t_all / 1e9, t_all, f"{done} instances of scores [1,{Hh},{S},{S}] from the c3 pool, numpy float64"
 
 
 class C4Workload:
@@ -371,16 +373,118 @@ class C4Workload:
         from oracle import dvm_oracle as orc
         t0 = time.perf_counter()
         nbytes, k = 0, 0
-        for (kind, r, c, ins, params, out, per) in self.items[0]:
-            orc.evaluate(self.progs[kind].nodes, [wl.to_f64(t) for t in ins], params)
-            nbytes += per; k += 1
+        for row in self.items:
+            for (kind, r, c, ins, params, out, per) in row:
+                orc.evaluate(self.progs[kind].nodes, [wl.to_f64(t) for t in ins], params)
+                nbytes += per; k += 1
+                if time.perf_counter() - t0 > budget_s:
+                    break
             if time.perf_counter() - t0 > budget_s:
                 break
         dt = time.perf_counter() - t0
-        return nbytes / dt / 1e9, dt, f"first {k} programs of launch 0, numpy float64"
+        return nbytes / dt / 1e9, dt, f"first {k} programs of the sweep (launch 0 onwards), numpy float64, input widening included"
 
 
-WORKLOADS = {"c2": C2Workload, "c3": C3Workload, "c4": C4Workload}
+class C5Workload:
+    """LLM MLP gate SiLU(X Wg) * (X Wu), bf16 X [M,4096], W [4096,11008] x2, fp32 accumulate, bf16 out (config 5)."""
+    name = "c5"
+    K, N = 4096, 11008
+    metric, unit, scale, bound, kernel, peak_key = "tflops_dynamic_shape_sweep", "TFLOP/s", 1e12, "tensor", "dvm_mm_kernel", "bf16_tflops_sustained"
+
+    def __init__(self, dvm, n_instances=64, device="cuda", max_rows=0):
+        self.dvm = dvm
+        self.prog = wl.program_mlp_gate()
+        self.p = dvm.program_from_nodes(self.prog.nodes)
+        self.enc = dvm.binding.Encoder(self.p)
+        self.Ms = wl.shapes_c5(n_instances)
+        if max_rows:
+            self.Ms = [min(m, max_rows) for m in self.Ms]
+        K, N = self.K, self.N
+        self.wg, self.wu = wl.mlp_weights(K, N, device)      # generated once, reused by every instance
+        self.pool_rows = max(self.Ms)
+        self.x = wl.randn((self.pool_rows, K), torch.bfloat16, wl.data_seed("c5", 0), device)
+        self.out = torch.empty((self.pool_rows, N), dtype=torch.bfloat16, device=device)
+        self.work_per_instance = [4 * m * K * N for m in self.Ms]          # two matmuls, 2 flops per multiply-add
+        self.bytes_per_instance = [2 * K * N * 2 + m * K * 2 + m * N * 2 for m in self.Ms]
+        self.total_work = sum(self.work_per_instance)
+        self.total_bytes = sum(self.bytes_per_instance)
+        self.description = ("c5: MLP gate SiLU(X Wg) * (X Wu), bf16 X [M,4096] x W [4096,11008] x2 (row-major), fp32 "
+                            f"accumulate, bf16 out, {n_instances} dynamic instances (M 1..4096), each re-encoded per launch")
+        self.l2_policy = "every instance streams both weight matrices (180 MB > L2) plus its own X / out windows"
+
+    def run_step(self, stream, events=None, enc_ns=None):
+        import ctypes as C
+        lib_launch = self.dvm.binding.lib.dvm_launch
+        K, N = self.K, self.N
+        for m in self.Ms:
+            t0 = time.perf_counter_ns()
+            size = self.enc.encode(((m, K), (K, N), (K, N)))
+            t1 = time.perf_counter_ns()
+            if enc_ns is not None:
+                enc_ns.append(t1 - t0)
+            arr = (C.c_void_p * 4)(self.x.data_ptr(), self.wg.data_ptr(), self.wu.data_ptr(), self.out.data_ptr())
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st = lib_launch(self.enc.buf, size, arr, 4, stream.cuda_stream)
+            if st != 0:
+                raise self.dvm.DvmError(st, "dvm_launch")
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+        return len(self.Ms)
+
+    def setup_e2e(self):
+        K, N = self.K, self.N
+        self.hx = self.x.cpu().pin_memory()
+        self.hwg = self.wg.cpu().pin_memory()
+        self.hwu = self.wu.cpu().pin_memory()
+        self.hout = torch.empty((self.pool_rows, N), dtype=torch.bfloat16).pin_memory()
+        self.staging = torch.empty(2 * K * N * 2 + self.pool_rows * (K + N) * 2 + 4 * 256, dtype=torch.uint8, device="cuda")
+
+    def run_step_e2e(self, stream):
+        K, N = self.K, self.N
+        h2d = d2h = 0
+        for m in self.Ms:
+            self.enc.encode(((m, K), (K, N), (K, N)))
+            code = self.dvm.Code(self.enc.buf, self.enc.size.value, None)
+            self.dvm.run_host(code, [self.hx[:m], self.hwg, self.hwu, self.hout[:m]], self.staging, stream)
+            h2d += 2 * K * N * 2 + m * K * 2
+            d2h += m * N * 2
+        return h2d, d2h
+
+    def oracle_sample(self, budget_s=12.0):
+        from oracle import dvm_oracle as orc
+        K, N = self.K, self.N
+        wg, wu = wl.to_f64(self.wg), wl.to_f64(self.wu)
+        t_all, flops, rows_done, off, m = 0.0, 0, 0, 0, min(256, self.pool_rows)
+        while t_all < budget_s:
+            if off + m > self.pool_rows:
+                off = 0
+            x = wl.to_f64(self.x[off:off + m])
+            t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [x, wg, wu]); t_all += time.perf_counter() - t0
+            flops += 4 * m * K * N
+            rows_done += m; off += m
+        return flops / t_all / 1e12, t_all, f"{rows_done} rows of X in windows of {m} rows against both full weight matrices, numpy float64"
+
+
+WORKLOADS = {"c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
+for _W in (C2Workload, C3Workload, C4Workload):   # the memory-bound sweeps: work = algorithmic bytes
+    _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
+    _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
+
+
+def oracle_threads(workload: str) -> int:
+    """Threads the numpy oracle actually uses: elementwise programs run on one core; the matmul of c5 goes
+    through numpy's BLAS, which uses its own pool."""
+    if workload != "c5":
+        return 1
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
 
 
 # ----------------------------------------------------------------------------- reference arm
@@ -390,7 +494,6 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import dvm_oracle as orc
-    torch.set_num_threads(1)
     if args.workload == "c2":
         prog = wl.program_add_rmsnorm(4096)
         rows = 4096
@@ -407,6 +510,14 @@ def run_reference(args):
         sample = "scores [1,8,512,512] per step, numpy float64"
         desc = C3Workload.__doc__
         params = ()
+    elif args.workload == "c5":
+        prog = wl.program_mlp_gate()
+        M = 64
+        ins = [wl.to_f64(t) for t in wl.inputs_mlp_gate(M, 4096, 11008, wl.data_seed("c5", 0))]
+        nbytes = 4 * M * 4096 * 11008   # flops
+        sample = f"X [{M},4096] against both weight matrices per step, numpy float64"
+        desc = C5Workload.__doc__
+        params = ()
     else:
         prog = wl.program_sigmoid_mul()
         ins = [wl.to_f64(t) for t in wl.inputs_stack("sigmoid_mul", 512, 4096, 1)[0]]
@@ -420,13 +531,16 @@ def run_reference(args):
     for _ in range(args.steps):
         orc.evaluate(prog.nodes, ins, params)
     dt = time.perf_counter() - t0
-    val = nbytes * args.steps / dt / 1e9
-    line = {"impl": "reference", "metric": "hbm_gbs_dynamic_shape_sweep", "value": val, "unit": "GB/s",
+    tensor = args.workload == "c5"
+    val = nbytes * args.steps / dt / (1e12 if tensor else 1e9)
+    unit = "TFLOP/s" if tensor else "GB/s"
+    line = {"impl": "reference", "metric": "tflops_dynamic_shape_sweep" if tensor else "hbm_gbs_dynamic_shape_sweep",
+            "value": val, "unit": unit,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": desc, "sample": sample},
-            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
-            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "cpu_baseline": {"value": val, "unit": unit, "cores": oracle_threads(args.workload), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
@@ -470,7 +584,7 @@ def main():
         dvm.set_elems_per_thread(args.elems_per_thread)
     if args.instances:
         kw = {"n_launches": args.instances} if args.workload == "c4" else {"n_instances": args.instances}
-    if args.max_rows and args.workload == "c2":
+    if args.max_rows and args.workload in ("c2", "c5"):
         kw["max_rows"] = args.max_rows
     W = WORKLOADS[args.workload](dvm, **kw)
     stream = torch.cuda.current_stream()
@@ -511,16 +625,27 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
-    value = W.total_bytes * world / (ms_per_step * 1e-3) / 1e9
+    work_each = getattr(W, "work_per_instance", W.bytes_per_instance)
+    total_work = sum(work_each)
+    value = total_work * world / (ms_per_step * 1e-3) / W.scale
 
     # dominant kernel: algorithmic bytes per launch over its CUDA-event time
     kern_ms = [a.elapsed_time(b) for a, b in events]
     per_launch_bytes = W.bytes_per_instance * args.steps
+    per_launch_work = work_each * args.steps
     kernel_total_ms = sum(kern_ms)
-    achieved = sum(per_launch_bytes) / (kernel_total_ms * 1e-3) / 1e9
-    big = [(b, m) for b, m in zip(per_launch_bytes, kern_ms) if b >= 256e6]
-    large_gbs = (sum(b for b, _ in big) / (sum(m for _, m in big) * 1e-3) / 1e9) if big else None
-    gbs_each = sorted(b / (m * 1e-3) / 1e9 for b, m in zip(per_launch_bytes, kern_ms))
+    achieved = sum(per_launch_work) / (kernel_total_ms * 1e-3) / W.scale
+    peak = peaks[W.peak_key]
+    if W.bound == "hbm":   # "large shapes": instances moving >= 256 MB
+        big = [(b, m) for b, m in zip(per_launch_work, kern_ms) if b >= 256e6]
+    else:                  # instances that are tensor-bound by a wide margin (M >= 1024)
+        big = [(b, m) for b, m in zip(per_launch_work, kern_ms) if b >= 4 * 1024 * 4096 * 11008]
+    large_gbs = (sum(b for b, _ in big) / (sum(m for _, m in big) * 1e-3) / W.scale) if big else None
+    gbs_each = sorted(b / (m * 1e-3) / W.scale for b, m in zip(per_launch_work, kern_ms))
+    # per-launch roofline time: the slower of (flops / tensor peak) and (bytes / HBM peak)
+    roof_ms = [max((w / (peak * 1e12) if W.bound == "tensor" else 0.0), b / (peaks["hbm_gbs"] * 1e9)) * 1e3
+               for w, b in zip(per_launch_work, per_launch_bytes)]
+    roofline_time_frac = sum(roof_ms) / kernel_total_ms
     enc_us = sorted(x / 1e3 for x in enc_ns)
 
     def pct(v, q):
@@ -535,19 +660,25 @@ def main():
         traffic = tj["dram_bytes_per_algorithmic_byte"] * sum(per_launch_bytes) / len(per_launch_bytes)
 
     line = {
-        "metric": "hbm_gbs_dynamic_shape_sweep", "value": value, "unit": "GB/s", "n_gpus": world,
+        "metric": W.metric, "value": value, "unit": W.unit, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 x bf16 -> f32" if W.bound == "tensor" else "f32", "data": "synthetic",
         "config": {"workload": W.description, "l2": W.l2_policy, "instances_per_step": n_inst,
-                   "algorithmic_bytes_per_step": W.total_bytes, "multi_gpu": "replicas only (no collective)"},
-        "pct_of_nominal_8TBs": value / world / 8000.0,
+                   "algorithmic_bytes_per_step": W.total_bytes,
+                   "algorithmic_flops_per_step": total_work if W.bound == "tensor" else None,
+                   "multi_gpu": "replicas only (no collective)"},
+        "pct_of_nominal": {"value": value / world / (2250.0 if W.bound == "tensor" else 8000.0),
+                           "nominal": "2.25 PFLOP/s dense bf16" if W.bound == "tensor" else "8 TB/s"},
         "encode_us": {"mean": sum(enc_us) / len(enc_us), "p50": pct(enc_us, 0.5), "p99": pct(enc_us, 0.99),
                       "max": enc_us[-1], "n": len(enc_us), "note": "perf_counter around the ctypes call to dvm_encode"},
-        "roofline": {"bound": "hbm", "kernel": "dvm_vm_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
-                     "traffic": traffic, "large_instances_gbs": large_gbs,
-                     "per_launch_gbs": {"min": gbs_each[0], "p10": pct(gbs_each, 0.1), "p50": pct(gbs_each, 0.5),
-                                        "max": gbs_each[-1]},
+        "roofline": {"bound": W.bound, "kernel": W.kernel, "achieved": achieved, "peak": peak,
+                     "unit": W.unit, "frac": achieved / peak, "peak_kind": f"of {peak_kind} ({W.peak_key})",
+                     "traffic": traffic, "large_instances": large_gbs,
+                     "large_instances_frac": (large_gbs / peak) if large_gbs else None,
+                     "roofline_time_frac": roofline_time_frac,
+                     "per_launch": {"min": gbs_each[0], "p10": pct(gbs_each, 0.1), "p50": pct(gbs_each, 0.5),
+                                    "max": gbs_each[-1]},
                      "launches_timed": len(kern_ms), "kernel_ms_per_step": kernel_total_ms / args.steps},
         "gpu_launches": launches,
         "clocks": clocks,
@@ -569,15 +700,15 @@ def main():
             tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
             if dist is not None:
                 dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e = {"value": W.total_bytes * world / float(tt.item()) / 1e9, "unit": "GB/s",
+            e2e = {"value": total_work * world / float(tt.item()) / W.scale, "unit": W.unit,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": 1,
                    "note": "dvm_run_host per instance: pinned host -> device, launch, device -> pinned host, sync"}
     line["e2e"] = e2e
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, dt, sample = W.oracle_sample()
-        line["cpu_baseline"] = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
-                                "seconds": dt, "host_cores_available": os.cpu_count()}
+        line["cpu_baseline"] = {"value": v, "unit": W.unit, "cores": oracle_threads(W.name), "kind": "oracle",
+                                "sample": sample, "seconds": dt, "host_cores_available": os.cpu_count()}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
