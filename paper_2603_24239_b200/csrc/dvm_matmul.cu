@@ -812,8 +812,19 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
               for (int i = 0; i < CHUNK; ++i) acc[i] = fast_rcp(1.0f + fast_exp(-acc[i]));
             } else {
-#pragma unroll 4
-              for (int i = 0; i < CHUNK; ++i) acc[i] = scalar_unary(u, acc[i]);
+#define DVM_MM_UN(U)                                                     \
+  case U:                                                                \
+    _Pragma("unroll") for (int i = 0; i < CHUNK; ++i) acc[i] = scalar_unary(U, acc[i]); \
+    break;
+              switch (u) {
+                DVM_MM_UN(DVM_U_EXP) DVM_MM_UN(DVM_U_SQRT) DVM_MM_UN(DVM_U_RSQRT) DVM_MM_UN(DVM_U_ABS)
+                DVM_MM_UN(DVM_U_LOG) DVM_MM_UN(DVM_U_ERF) DVM_MM_UN(DVM_U_NEG) DVM_MM_UN(DVM_U_RECIP)
+                DVM_MM_UN(DVM_U_FLOOR) DVM_MM_UN(DVM_U_ROUND) DVM_MM_UN(DVM_U_TANH)
+                default:
+#pragma unroll
+                  for (int i = 0; i < CHUNK; ++i) acc[i] = round_bf16(acc[i]);
+              }
+#undef DVM_MM_UN
             }
           } else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) {
             const float imm = __uint_as_float(MW(pc + 1));
