@@ -545,6 +545,20 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- multi-rank aggregation
+def reduce_max_over_ranks(x: float, dist, device) -> float:
+    """The slowest rank's time: all-reduce MAX over the process group (identity without one)."""
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(work_per_rank: float, world: int, ms_per_step: float, scale: float) -> float:
+    """Replicas only: every rank processes the same sweep, the job's work is world x one rank's."""
+    return work_per_rank * world / (ms_per_step * 1e-3) / scale
+
+
 # ----------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -620,14 +634,11 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     assert dvm.last_device_status() == 0
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = reduce_max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
     work_each = getattr(W, "work_per_instance", W.bytes_per_instance)
     total_work = sum(work_each)
-    value = total_work * world / (ms_per_step * 1e-3) / W.scale
+    value = whole_job_value(total_work, world, ms_per_step, W.scale)
 
     # dominant kernel: algorithmic bytes per launch over its CUDA-event time
     kern_ms = [a.elapsed_time(b) for a, b in events]
@@ -697,10 +708,8 @@ def main():
             h2d, d2h = W.run_step_e2e(stream)
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
-            tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
-            if dist is not None:
-                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e = {"value": total_work * world / float(tt.item()) / W.scale, "unit": W.unit,
+            dt = reduce_max_over_ranks(dt, dist, "cuda")
+            e2e = {"value": whole_job_value(total_work, world, dt * 1e3, W.scale), "unit": W.unit,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": 1,
                    "note": "dvm_run_host per instance: pinned host -> device, launch, device -> pinned host, sync"}
     line["e2e"] = e2e

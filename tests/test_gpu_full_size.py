@@ -1,0 +1,68 @@
+"""Parity at the full sizes of the sweeps, in the launch configuration bench.py times: the largest
+instances are too big for the oracle as a whole, but their rows are independent, so sampled rows are
+evaluated by the oracle one by one and compared element by element."""
+import numpy as np
+import pytest
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from oracle import dvm_oracle as orc
+from tests.parity_util import gate_errors
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_rows(n, k, seed, extra=()):
+    rng = np.random.default_rng(seed)
+    return np.unique(np.concatenate([[0, n - 1], np.asarray(extra, dtype=np.int64), rng.integers(0, n, k)]))
+
+
+@pytest.mark.parametrize("rows", [262144, 32 * 8192 - 4097])
+def test_add_rmsnorm_max_rows_sampled(rows):
+    """Config 2 at its largest instance (B = 32, S = 8192: 2 GiB per tensor) and a ragged neighbour."""
+    H = 4096
+    x = wl.randn((rows, H), torch.bfloat16, 11, "cuda")
+    res = wl.randn((rows, H), torch.bfloat16, 12, "cuda")
+    w = wl.randn((H,), torch.bfloat16, 13, "cuda", mean=1.0, std=0.02)
+    y = torch.full((rows, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    h = torch.full((rows, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    prog = wl.program_add_rmsnorm(H)
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [(rows, H), (rows, H), (H,)])
+    dvm.launch(code, [x, res, w, y, h])
+    assert dvm.last_device_status() == 0
+    idx = _sample_rows(rows, 60, 1, extra=[255, 256, rows // 2])
+    ti = torch.from_numpy(idx).cuda()
+    want = orc.evaluate(prog.nodes, [wl.to_f64(x[ti]), wl.to_f64(res[ti]), wl.to_f64(w)])
+    for got, ref in zip((y, h), want):
+        g1, g2 = gate_errors(wl.to_f64(got[ti]), ref)
+        assert g2 <= 2e-2, (g1, g2)
+    # every row was written: no poison left anywhere
+    assert not torch.isnan(y.view(torch.int16).bitwise_and(0x7fff).float().max()) and not torch.isnan(y.float().sum())
+
+
+@pytest.mark.parametrize("B,S", [(8, 2048), (8, 2047), (3, 1531)])
+def test_masked_softmax_max_size_sampled(B, S):
+    """Config 3 at its largest instance (B = 8, S = 2048: 2^30 scores) and unaligned neighbours."""
+    Hh = 32
+    scores = wl.randn((B, Hh, S, S), torch.bfloat16, 21, "cuda")
+    mask = wl.causal_mask(S, "cuda")
+    out = torch.full((B, Hh, S, S), float("nan"), dtype=torch.bfloat16, device="cuda")
+    prog = wl.program_masked_softmax(128)
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [(B, Hh, S, S), (1, 1, S, S)])
+    dvm.launch(code, [scores, mask, out])
+    assert dvm.last_device_status() == 0
+    n_rows = B * Hh * S
+    idx = _sample_rows(n_rows, 60, 2, extra=[S - 1, S, n_rows // 2])
+    flat_s, flat_o = scores.view(n_rows, S), out.view(n_rows, S)
+    ti = torch.from_numpy(idx).cuda()
+    sc = wl.to_f64(flat_s[ti])                       # [k, S]
+    mk = wl.to_f64(mask.view(S, S)[ti % S])          # the mask row of each sampled query position
+    got = wl.to_f64(flat_o[ti])
+    for r in range(len(idx)):                        # the oracle, one sampled row at a time
+        ref = orc.evaluate(prog.nodes, [sc[r].reshape(1, 1, 1, S), mk[r].reshape(1, 1, 1, S)])[0].reshape(S)
+        g1, g2 = gate_errors(got[r], ref)
+        assert g2 <= 2e-2, (idx[r], g1, g2)
+        q = int(idx[r] % S)
+        assert np.all(got[r][q + 1:] == 0)           # masked entries exactly zero
+    assert not torch.isnan(out.float().sum())
