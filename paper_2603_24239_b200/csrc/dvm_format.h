@@ -48,7 +48,7 @@ enum {
   DVM_H_PRIMARY = 16,        // operand whose row starts define the vector alignment, or 0xffffffff
   DVM_H_LOCAL = 17,          // n_in_regs | n_tmp_regs << 8 | n_scalar_slots << 16 | V << 24 (elements per thread: 16 or 32)
   DVM_H_LOAD_WORDS = 18,     // length of the load section (words) at the start of the code body
-  DVM_H_LOCAL2 = 19,         // scalar-slot unit offset << 8 | units of one tile slot << 16
+  DVM_H_LOCAL2 = 19,         // unit offset of the per-row scalar slots | units of one tile slot << 16
   DVM_HDR_WORDS = 20
 };
 
@@ -57,8 +57,19 @@ enum {
   DVM_F_ALIGNED = 1,    // every row segment of the primary operand starts on a W-element
                         // boundary provided its base pointer is 16-byte aligned
   DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
-  DVM_F_FLAT = 4        // pure elementwise program laid out as a flat range
+  DVM_F_FLAT = 4,       // pure elementwise program laid out as a flat range
+  DVM_F_PRIMARY_DENSE = 8  // the primary operand is dense: row r starts at element r * C of its tensor
 };
+
+// ---- local register table: one word per local register: unit offset inside a tile slot | mode << 16 ----
+enum {
+  DVM_LM_PRIVATE = 0,  // temporary: thread-private fp32 vectors, vector q of thread tid at (q * 256 + tid) * 16
+  DVM_LM_BLOCK = 1,    // input whose tile is one contiguous byte range of global memory: one bulk copy per tile
+  DVM_LM_ROWS = 2,     // input copied row by row (one bulk copy per row): row images DVM_ROW_PITCH(...) apart
+  DVM_LM_BCAST = 3     // row-vector input, the same for every row and tile: one row image per slot
+};
+// bytes between the row images of a ROWS register (room for the 16-byte alignment slack on both sides)
+#define DVM_ROW_PITCH(G, V, es) ((uint32_t)(G) * (uint32_t)(V) * (uint32_t)(es) + 32u)
 
 // ---- operand descriptor ----
 enum {
@@ -78,8 +89,8 @@ enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
 #define DVM_VM_VMAX 32           // most elements of a tile register one thread holds (V is 16 or 32)
 #define DVM_MAX_LREGS 10         // local tile registers of a program (inputs + temporaries)
 #define DVM_MAX_SSLOTS 8         // per-row scalar inputs of a program
-#define DVM_LOCAL_UNIT 8192      // bytes of one local-memory unit: 32 B per thread (16 bf16 or 8 fp32 words)
-#define DVM_MAX_LOCAL_UNITS 27   // units a CTA can hold (two tile slots), 216 KB
+#define DVM_LOCAL_UNIT 256       // bytes of one local-memory unit (layout granule)
+#define DVM_MAX_LOCAL_UNITS 896  // units a CTA can hold (two tile slots), 224 KB
 #define DVM_MAX_SREGS 8          // per-row scalar registers
 #define DVM_MAX_TENSORS 16
 #define DVM_MAX_OPERANDS 24

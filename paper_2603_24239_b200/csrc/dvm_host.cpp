@@ -855,15 +855,18 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
         if (primary >= 0)
           for (int q = 0; q < 3; ++q)
             if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
-        for (int pass = 0; pass < 2 && g.cost < 0; ++pass) {
-          const int w = pass == 0 ? W0 : 1;  // second pass: element-wise mapping, which needs no padding
-          const bool al = pass == 0 ? aligned : true;
-          const int64_t pad = 0;  // a misaligned row wraps its last columns into the unused head slots: no padding
+        {
+          const int w = W0;
+          const bool al = aligned;
+          // a misaligned row segment starts up to w - 1 slots into its first chunk: keep that much spare capacity
+          const int64_t pad = al ? 0 : w - 1;
           for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
             int64_t G = 1 << lg, cap = G * g.V;
             int64_t ct;
             if (has_reduce) {
-              if (cap < C + pad) continue;
+              // a whole row per thread group; at the widest group a row may use the full capacity: its last
+              // columns then wrap around into the head slots of a misaligned row
+              if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
               ct = C;
             } else {
               ct = ((cap - pad) / w) * w;
@@ -886,33 +889,44 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
         g.lastRowCols = C;
         if (empty) g.n_tiles = 0;
       }
-      // local-memory layout in 8 KB units (32 bytes per thread): input registers twice (double buffering;
-      // a row-vector input of an aligned program is the same for every tile of a thread: once),
-      // temporaries, the staging line of the scalar store path, per-row scalar slots
-      // Local-memory layout of ONE tile slot, in 8 KB units (32 bytes per thread): input registers,
-      // temporaries, per-row scalar slots.  A CTA holds two slots: while it computes the tile in one, the
-      // next tile (of this or of another stacked program) loads into the other.
+      // Local-memory layout of ONE tile slot, in 256-byte units.  An input register is an image of the
+      // tile's rows as they lie in global memory (a dense operand: one contiguous range; otherwise one
+      // image per row, DVM_ROW_PITCH apart; a row vector shared by every row: one row image); a
+      // temporary is thread-private (V fp32 per thread); per-row scalar slots are thread-private.
+      // A CTA holds two slots: while it computes the tile in one, the next tile (of this or of another
+      // stacked program) loads into the other.
       g.inv_mask = 0;
       g.units = 0;
+      const int64_t Gthreads = 1ll << g.log2G;
       for (int k = 0; k < e.n_in_regs; ++k) {
         const Operand& od = e.opd[in_opd[k]];
-        const bool inv = !flat && (g.flags & DVM_F_ALIGNED) && g.W > 1 && g.CB == 1 && od.ostride[0] == 0 &&
-                         od.ostride[1] == 0 && od.ostride[2] == 0;
-        if (inv) g.inv_mask |= 1u << k;  // the same for every tile of a thread: loaded once per slot
-        g.lreg_table[k] = (uint32_t)g.units;
-        g.units += g.V * (in_dtype[k] == DVM_DT_BF16 ? 2 : 4) / 32;
+        const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
+        const bool inv = !flat && g.CB == 1 && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
+        bool dense = od.col_stride == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
+        if (!flat) {
+          if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+          if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+        }
+        const int mode = inv ? DVM_LM_BCAST : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
+        if (inv) g.inv_mask |= 1u << k;  // the same for every tile: loaded once per slot
+        const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
+        const int64_t bytes = inv ? pitch : pitch * (T / Gthreads);
+        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
+        g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
       }
       for (int k = e.n_in_regs; k < nreg; ++k) {
-        g.lreg_table[k] = (uint32_t)g.units;
-        g.units += g.V * 4 / 32;
+        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)DVM_LM_PRIVATE << 16);
+        g.units += g.V * 4 * T / DVM_LOCAL_UNIT;
       }
       g.scalar_unit = g.units;
-      if (e.n_sslots > 0) g.units += 2;
-      if (2 * g.units > DVM_MAX_LOCAL_UNITS) break;
-      int ctas = 233472 / (2 * g.units * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
+      if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
+      if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) break;
+      int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
       if (ctas > 2) ctas = 2;  // the interpreter is compiled for two resident CTAs per SM
       if (ctas < 1) break;
-      if (ctas == ctas_guess) ok = true;
+      // the geometry was costed for ctas_guess resident CTAs per SM: at least that many must fit
+      // (more is harmless; fewer: cost it again for the smaller number)
+      if (ctas >= ctas_guess) ok = true;
       else ctas_guess = ctas;
     }
     if (!ok) continue;
@@ -922,7 +936,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   const int log2G = best.log2G;
   W = best.W;
   const int64_t Ctile = best.Ctile, CB = best.CB, rowsR = best.rowsR, lastRowCols = best.lastRowCols, n_tiles = best.n_tiles;
-  const uint32_t flags = best.flags;
+  uint32_t flags = best.flags;
   const int units = best.units, scalar_unit = best.scalar_unit;
   const uint32_t* lreg_table = best.lreg_table;
   if (flat) {
@@ -934,6 +948,18 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
     outer[0] = rowsR; outer[1] = outer[2] = 1;
   }
   if (n_tiles > 0xffffffffll || rowsR > 0xffffffffll) return DVM_ERR_TOO_LARGE;
+
+  // dense operands: the rows of a tile are one contiguous range (flat offset = row * C + col)
+  bool dense_of[DVM_MAX_OPERANDS];
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    bool dense = od.col_stride == 1 && od.ostride[0] == C;
+    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+    dense_of[o] = dense;
+  }
+  if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
+  if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
@@ -963,15 +989,12 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
   w[DVM_H_LOCAL] = (uint32_t)e.n_in_regs | ((uint32_t)e.n_tmp_regs << 8) | ((uint32_t)e.n_sslots << 16) | ((uint32_t)best.V << 24);
   w[DVM_H_LOAD_WORDS] = (uint32_t)e.n_loads;
-  w[DVM_H_LOCAL2] = ((uint32_t)scalar_unit << 8) | ((uint32_t)units << 16);
+  w[DVM_H_LOCAL2] = (uint32_t)scalar_unit | ((uint32_t)units << 16);
   uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
   for (int o = 0; o < e.n_opd; ++o) {
     const Operand& od = e.opd[o];
     uint32_t* d = ot + o * DVM_OPD_WORDS;
-    // dense: the rows of a tile are one contiguous byte range (flat offset = row * C + col)
-    bool dense = od.col_stride == 1 && od.ostride[0] == C;
-    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
-    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+    const bool dense = dense_of[o];
     d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
                       ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25);
     for (int g = 0; g < 3; ++g) {
@@ -1032,16 +1055,31 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   const uint32_t local = w[DVM_H_LOCAL];
   const uint32_t n_inr = local & 0xff, n_tmpr = (local >> 8) & 0xff, n_ss = (local >> 16) & 0xff, Vv = local >> 24;
   if (Vv != 16 && Vv != 32) return DVM_ERR_BAD_CODE;
-  const uint32_t u_bf16 = Vv * 2 / 32, u_f32 = Vv * 4 / 32;  // local-memory units of one tile register
-  if (lg > 8 || !(W == 1 || W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
+  const uint32_t u_bf16 = DVM_DT_BF16, u_f32 = DVM_DT_F32;  // element type an instruction expects in a register
+  if (lg > 8 || !(W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
   const uint32_t local2 = w[DVM_H_LOCAL2];
-  const uint32_t units = (local2 >> 16) & 0xff, scalar_unit = (local2 >> 8) & 0xff;
-  if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || 2 * units > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
-  if (n_ss && scalar_unit + 2 > units) return DVM_ERR_BAD_CODE;
+  const uint32_t units = local2 >> 16, scalar_unit = local2 & 0xffffu;
+  if (n_inr + n_tmpr > DVM_MAX_LREGS || n_ss > DVM_MAX_SSLOTS || 2 * units + 1 > DVM_MAX_LOCAL_UNITS) return DVM_ERR_BAD_CODE;
+  if (n_ss && scalar_unit + 2 * 16 * DVM_VM_THREADS / DVM_LOCAL_UNIT > units) return DVM_ERR_BAD_CODE;
   const uint32_t* lt = w + DVM_HDR_WORDS + 2 * n_tensors + DVM_OPD_WORDS * n_opd;
-  // a local register access of `need` units (bf16: 1, fp32: 2) must stay inside the CTA's local memory
-  auto lreg_ok = [&](uint32_t k, uint32_t need) {
-    return k < nreg && lt[k] + need <= units;
+  const uint32_t* otab = w + DVM_HDR_WORDS + 2 * n_tensors;
+  // a local register must lie inside the tile slot, in the layout its kind implies, and hold the element
+  // type the instruction expects
+  auto lreg_ok = [&](uint32_t k, uint32_t dt) {
+    if (k >= nreg) return false;
+    const uint32_t lw = lt[k], unit = lw & 0xffffu, mode = (lw >> 16) & 0xff, od = lw >> 24;
+    uint64_t need;
+    if (k >= n_inr) {
+      if (mode != DVM_LM_PRIVATE || dt != DVM_DT_F32) return false;
+      need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
+    } else {
+      if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST || od >= n_opd) return false;
+      if (((otab[od * DVM_OPD_WORDS] >> 8) & 0xff) != dt) return false;
+      const uint64_t pitch = DVM_ROW_PITCH(1u << lg, Vv, dt == DVM_DT_BF16 ? 2 : 4);
+      const uint64_t bytes = mode == DVM_LM_BCAST ? pitch : pitch * (DVM_VM_THREADS >> lg);
+      need = (bytes + DVM_LOCAL_UNIT - 1) / DVM_LOCAL_UNIT;
+    }
+    return unit + need <= units;
   };
   const uint32_t load_words = w[DVM_H_LOAD_WORDS];
   if (load_words > body) return DVM_ERR_BAD_CODE;
@@ -1049,7 +1087,8 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   uint64_t ctile = w[DVM_H_COL_TILE], cb = w[DVM_H_COL_BLOCKS], C = w[DVM_H_COLS];
   uint64_t R = (uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32);
   uint32_t flags = geom >> 24;
-  uint64_t pad = 0;
+  const uint64_t pad = 0;  // a misaligned row that fills the whole capacity wraps its last columns into the head slots
+  if (!(flags & DVM_F_ALIGNED) && w[DVM_H_PRIMARY] == 0xffffffffu) return DVM_ERR_BAD_CODE;
   if (w[DVM_H_N_TILES] > 0) {
     if (ctile == 0 || cb == 0 || ctile + pad > G * Vv) return DVM_ERR_BAD_CODE;
     if (cb * ctile < C || (cb - 1) * ctile >= C) return DVM_ERR_BAD_CODE;
@@ -1168,7 +1207,7 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
   int cores = dvm_get_num_cores();
   outf(o, "kernel vmain.vec  block_dim=%lld  body_tile=%lld  code_size=%u\n", (long long)n_tiles,
        (long long)((n_tiles + cores - 1) / cores), w[DVM_H_CODE_WORDS] * 4);
-  outf(o, "  elems_per_thread=%u local_units=%u\n", w[DVM_H_LOCAL] >> 24, (w[DVM_H_LOCAL2] >> 16) & 0xff);
+  outf(o, "  elems_per_thread=%u local_units=%u\n", w[DVM_H_LOCAL] >> 24, w[DVM_H_LOCAL2] >> 16);
   outf(o, "  rows=%llu cols=%u col_tile=%u col_blocks=%u threads_per_row=%u vec=%u local_regs=%u flags=%s%s%s\n",
        (unsigned long long)((uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32)), w[DVM_H_COLS],
        w[DVM_H_COL_TILE], w[DVM_H_COL_BLOCKS], 1u << (geom & 0xff), (geom >> 8) & 0xff, (geom >> 16) & 0xff,

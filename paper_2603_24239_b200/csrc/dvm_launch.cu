@@ -113,11 +113,14 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
     uintptr_t es = ((info >> 8) & 0xff) == DVM_DT_BF16 ? 2 : 4;
     if (a % es) return DVM_ERR_INVALID_ARG;
   }
-  uint32_t geom = code[DVM_H_GEOM];
-  uint32_t W = (geom >> 8) & 0xff, flags = geom >> 24;
-  if ((flags & DVM_F_ALIGNED) && W > 1 && code[DVM_H_PRIMARY] != 0xffffffffu) {
-    uint32_t info = ot[code[DVM_H_PRIMARY] * DVM_OPD_WORDS];
-    if (((uintptr_t)tensors[info & 0xff]) & 15) dst[DVM_H_GEOM] = (geom & ~0xff00u) | (1u << 8);
+  // A program encoded for aligned rows relies on a 16-byte aligned primary tensor; on any other base address
+  // the interpreter derives the row shift from the actual address instead (the rows' last columns then
+  // wrap around into the head slots when a row fills its whole capacity).
+  const uint32_t geom = code[DVM_H_GEOM];
+  const uint32_t flags = geom >> 24;
+  if ((flags & DVM_F_ALIGNED) && code[DVM_H_PRIMARY] != 0xffffffffu) {
+    const uint32_t info = ot[code[DVM_H_PRIMARY] * DVM_OPD_WORDS];
+    if (((uintptr_t)tensors[info & 0xff]) & 15) dst[DVM_H_GEOM] = geom & ~((uint32_t)DVM_F_ALIGNED << 24);
   }
   return DVM_OK;
 }
@@ -151,7 +154,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     const uint32_t* c = (const uint32_t*)codes[i];
     need += c[DVM_H_TOTAL_WORDS];
     total_tiles += c[DVM_H_N_TILES];
-    if (((c[DVM_H_LOCAL2] >> 16) & 0xff) > units) units = (c[DVM_H_LOCAL2] >> 16) & 0xff;
+    if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
     if (V && v != V) return DVM_ERR_INVALID_ARG;  // one kernel variant per launch: same elements per thread
     V = v;
@@ -183,7 +186,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.queue = dev.scratch + 8 + 2 * dev.queue_slot;
 
   const bool large = pos > PW_SMALL;
-  const size_t smem = 2 * (size_t)units * DVM_LOCAL_UNIT;  // two tile slots
+  const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;  // one spare unit, two tile slots
   P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   int occ = 0;
@@ -331,7 +334,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     if (c[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_UNSUPPORTED;
     need += c[DVM_H_TOTAL_WORDS];
     total_tiles += c[DVM_H_N_TILES];
-    if (((c[DVM_H_LOCAL2] >> 16) & 0xff) > units) units = (c[DVM_H_LOCAL2] >> 16) & 0xff;
+    if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
     if (V && v != V) return DVM_ERR_INVALID_ARG;
     V = v;
@@ -362,7 +365,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.use_queue = 1u;
   P.status = dev.scratch;
   P.queue = dev.scratch + 2;
-  const size_t smem = 2 * (size_t)units * DVM_LOCAL_UNIT;
+  const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;
   P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool large = pos > PW_SMALL;

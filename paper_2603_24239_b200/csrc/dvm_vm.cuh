@@ -5,18 +5,23 @@
 // arrive as the kernel-parameter block; every warp fetches instruction words
 // from that block through the constant bank (warp-uniform loads) and loops over
 // the CTA's tiles.  A code body is [load section][compute section]:
-//   * every global tile load is an asynchronous 16-byte global->shared copy
-//     (cp.async) into a thread-private "local register" in shared memory -- the
-//     paper's local memory.  A CTA holds two tile slots (complete register sets):
-//     the load section of tile i+1 -- of the same or of another stacked program --
-//     runs when tile i starts, so the next tile's HBM traffic is in flight during
-//     the whole compute of the current one at no register cost; a row-vector
-//     input of an aligned program is loaded once per slot;
+//   * every global tile load is a TMA bulk copy (cp.async.bulk, global ->
+//     shared, completion on an mbarrier) that lands the tile's bytes in local
+//     memory exactly as they lie in global memory: an "image" of the tile's
+//     rows.  A dense operand's tile is one contiguous byte range: one copy,
+//     issued by one thread; other operands are copied row by row (the first
+//     thread of each row issues its row); a row vector shared by all rows is
+//     copied once per slot.  Copies start and end on 16-byte boundaries (the
+//     enclosing aligned range is fetched), so any row alignment works.
+//     A CTA holds two tile slots: the copies of tile i+1 -- of the same or of
+//     another stacked program -- are issued when tile i starts, so the next
+//     tile's HBM traffic is in flight during the whole compute of the current
+//     one and costs the compute threads no instructions;
 //   * the compute section is accumulator code: ACC is one register-resident tile
 //     (V = 16 or 32 fp32 per thread, as float2 pairs so that add / mul / fma
-//     issue as packed f32x2 instructions); other operands are read from local
-//     registers with 128-bit shared loads (bf16 operands widened on the fly), or
-//     are per-row scalars S0..S7.
+//     issue as packed f32x2 instructions); other operands are read from the
+//     images (or from thread-private temporaries) with 128-bit shared loads,
+//     bf16 widened on the fly, or are per-row scalars S0..S7.
 //
 // Tile geometry (chosen per instance by the host's shape tiling):
 //   G = 2^lgG threads share one row; a CTA holds 256/G rows per tile.
@@ -24,17 +29,14 @@
 //   column  (t + G*(s / W)) * W + (s % W) - shift  of the tile's column block,
 //   t = thread index inside the row group, W = vector width in elements,
 //   shift = misalignment of the row segment start, so that a thread's W-slot
-//   chunk is a 16-byte aligned vector of the primary operand.  The `shift` slots
-//   in front of the segment hold the segment's last columns (wrap-around), so a
-//   row never needs more slots than it has columns.
-// Whole chunks of an operand whose rows are aligned like the primary operand's
-// are copied with cp.async; whole chunks at another alignment are fetched as the
-// two covering aligned 16-byte words and realigned in registers; chunks cut by
-// the segment's head or tail are assembled from predicated element loads.
+//   chunk is a 16-byte aligned vector of the primary operand -- in global
+//   memory and therefore in its image.  An operand whose rows are aligned
+//   differently is read as the two covering aligned vectors and realigned in
+//   registers.  Slots outside the row segment hold whatever the enclosing
+//   vectors contain; reductions and stores mask them.
 //
-// Local memory layout: units of 8 KB (32 bytes per thread); 16-byte vector q of a
-// register at unit offset U lives at  U*8192 + (q * 256 + tid) * 16,
-// i.e. consecutive threads touch consecutive vectors (no bank conflicts).
+// Every wait on an mbarrier is bounded; a wait that runs out sets the status
+// word to ST_TIMEOUT and the CTA leaves its tile loop.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -51,7 +53,6 @@ constexpr int THREADS = DVM_VM_THREADS;
 #define DVM_VM_MIN_CTAS 2
 #endif
 
-
 template <int PW>
 struct VMParams {
   uint32_t n_programs;
@@ -67,14 +68,17 @@ struct VMParams {
 
 struct TileCtx {
   uint32_t prog;     // word offset of the tile's program in the parameter block
-  int t;             // thread index within the row group
   int lgG, lgW;
-  int shift;
+  int shift;         // elements between the thread-0 chunk start and the row segment start
+  int cbase;         // (t << lgW) - shift: column of this thread's slot 0
+  int ov;            // thread 0 of a row only: its first `ov` slots hold the row's last columns (wrap-around, see make_ctx)
   int ncols;         // valid columns of this thread's row inside the column block (0: nothing to do)
   int nvalid;        // slots s >= 8 are valid iff s < nvalid (the valid slots of a thread form a prefix,
   uint32_t hm;       //   except in the first chunk of a misaligned row: bit s of hm covers slots 0..7)
   uint32_t fullmask; // bit j: chunk j lies entirely inside the row segment
   uint32_t partmask; // bit j: chunk j is cut by the segment's head or tail
+  uint32_t row;      // row of the dominant (collapsed) shape
+  uint32_t row0;     // first row of the tile
   uint32_t i0, i1, i2;  // row coordinates over the collapsed outer dims
   uint32_t col0;
   uint32_t flags;
@@ -91,19 +95,53 @@ __device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) 
   for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = (k == i) ? v : S[i];
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-// 16-byte copy when `on`, otherwise nothing is read (source size 0) and the destination is zero-filled
-__device__ __forceinline__ void cp_async16_if(uint32_t dst, const void* src, bool on) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(on ? 16 : 0) : "memory");
-}
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// ---- mbarrier + bulk copy ----
+__device__ __forceinline__ void vm_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void vm_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void vm_mbar_arrive_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool vm_mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait (2 s of %globaltimer, and a poll cap): false when it ran out.
+__device__ __noinline__ bool vm_mbar_wait_slow(uint32_t bar, uint32_t parity) {
+  unsigned long long t0, t1;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (uint32_t spin = 0; spin < (1u << 27); ++spin) {
+    if (vm_mbar_try(bar, parity)) return true;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    if (t1 - t0 > 2000000000ull) break;
+  }
+  return false;
+}
+__device__ __forceinline__ bool vm_mbar_wait(uint32_t bar, uint32_t parity) {
+  if (vm_mbar_try(bar, parity)) return true;
+  return vm_mbar_wait_slow(bar, parity);
+}
+// global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned), completion on `bar`
+__device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+               "r"(bytes), "r"(bar)
+               : "memory");
+}
 
 // SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
@@ -113,71 +151,79 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   constexpr int VP = V / 2;            // float2 pairs per tile register
   constexpr int NST = V / 16;          // 16-element steps of a local-register operand
   constexpr int GRP = V >= 32 ? 2 : 1; // steps whose shared loads are issued together, ahead of their arithmetic
-  constexpr uint32_t VSTRIDE = THREADS * 16;  // bytes between consecutive 16-byte vectors of a local register
+  constexpr uint32_t PSTRIDE = THREADS * 16;  // bytes between consecutive vectors of a thread-private register
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ float s_red[2][THREADS / 32];
   __shared__ uint32_t s_next[2];
+  __shared__ __align__(8) unsigned long long s_bar[2];  // "tile landed" barrier of each tile slot
+  __shared__ volatile uint32_t s_abort;
 
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
-  const uint32_t local_base = static_cast<uint32_t>(__cvta_generic_to_shared(s_dyn)) + (uint32_t)tid * 16;
+  // one spare unit in front of the slots: a realigned read may touch the 16 bytes below an image
+  const uint32_t local_base = static_cast<uint32_t>(__cvta_generic_to_shared(s_dyn)) + DVM_LOCAL_UNIT;
+  const uint32_t bar0 = static_cast<uint32_t>(__cvta_generic_to_shared(s_bar));
   const uint32_t n_prog = SINGLE ? 1u : prm.n_programs;
   const bool use_queue = SINGLE ? false : prm.use_queue != 0;
 #define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
 
-  // shared-memory address of 16-byte vector 0 of the register at unit offset U (this thread's part)
-  auto lreg_addr = [&](uint32_t unit, int slot) -> uint32_t { return local_base + unit * DVM_LOCAL_UNIT + (slot ? prm.slot_bytes : 0u); };
+  if (tid == 0) {
+    s_abort = 0;
+    vm_mbar_init(bar0, THREADS);
+    vm_mbar_init(bar0 + 8, THREADS);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  auto slot_base = [&](int slot) -> uint32_t { return local_base + (slot ? prm.slot_bytes : 0u); };
 
   // word offsets of a program's tables
   auto opd_base = [&](uint32_t prog) -> uint32_t { return prog + DVM_HDR_WORDS + 2 * (CW(prog + DVM_H_COUNTS) & 0xff); };
   auto lreg_base = [&](uint32_t prog) -> uint32_t { return opd_base(prog) + ((CW(prog + DVM_H_COUNTS) >> 16) & 0xff) * DVM_OPD_WORDS; };
   auto body_base = [&](uint32_t prog) -> uint32_t { return lreg_base(prog) + ((CW(prog + DVM_H_GEOM) >> 16) & 0xff); };
 
-  // Address of element (row, col0) of operand b -- or of the row's single value when col_stride = 0.
-  auto operand_addr = [&](uint32_t prog, uint32_t opd0, int b, const TileCtx& c, int& dtype) -> char* {
-    const uint32_t d = opd0 + b * DVM_OPD_WORDS;
-    const uint32_t info = CW(d + DVM_OPD_INFO);
-    const uint32_t tp = prog + DVM_HDR_WORDS + 2 * (info & 0xff);
-    const unsigned long long base = (unsigned long long)CW(tp) | ((unsigned long long)CW(tp + 1) << 32);
-    dtype = (info >> 8) & 0xff;
-    // strides are below 2^32 elements (the host rejects larger ones): 32 x 32 -> 64-bit products
+  // device address of the tensor an operand descriptor (word offset d) names
+  auto tensor_ptr = [&](uint32_t prog, uint32_t d) -> unsigned long long {
+    const uint32_t tp = prog + DVM_HDR_WORDS + 2 * (CW(d + DVM_OPD_INFO) & 0xff);
+    return (unsigned long long)CW(tp) | ((unsigned long long)CW(tp + 1) << 32);
+  };
+  // element offset of this thread's row (plus the column block start) inside operand d
+  // (strides are below 2^32 elements -- the host rejects larger ones: 32 x 32 -> 64-bit products)
+  auto row_offset = [&](uint32_t d, const TileCtx& c) -> unsigned long long {
     unsigned long long off = (unsigned long long)c.i0 * CW(d + DVM_OPD_STRIDE0);
     if (c.flags & DVM_F_OUTER_DIMS) {
       off += (unsigned long long)c.i1 * CW(d + DVM_OPD_STRIDE1);
       off += (unsigned long long)c.i2 * CW(d + DVM_OPD_STRIDE2);
     }
-    if ((info >> 16) & 0xff) off += c.col0;
-    return reinterpret_cast<char*>(base + (off << (dtype == DVM_DT_BF16 ? 1 : 2)));
+    if ((CW(d + DVM_OPD_INFO) >> 16) & 0xff) off += c.col0;
+    return off;
   };
 
-  // Column (relative to the column block) of element e of chunk j, with the wrap-around of the head slots.
-  auto chunk_col = [&](const TileCtx& c, int j, int e) -> int {
-    const int col = ((c.t + (j << c.lgG)) << c.lgW) + e - c.shift;
-    return col < 0 ? col + (V << c.lgG) : col;
-  };
-
-  // Tile id -> geometry of this thread's part of the tile (closed forms, no loops).
+  // Tile id -> geometry of this thread's part of the tile (closed forms, no loops).  `c` holds the previous
+  // tile's geometry on entry: the slot masks are kept when the row segment has the same length and shift.
   auto make_ctx = [&](TileCtx& c, uint32_t prog, uint32_t local_tile) {
+    const bool same_prog = c.prog == prog;
     c.prog = prog;
     const uint32_t geom = CW(prog + DVM_H_GEOM);
     c.lgG = geom & 0xff;
     const int W = (geom >> 8) & 0xff;
-    c.lgW = W == 8 ? 3 : (W == 4 ? 2 : 0);
+    c.lgW = W == 8 ? 3 : 2;
     c.flags = geom >> 24;
     const int G = 1 << c.lgG;
-    c.t = tid & (G - 1);
+    const int t = tid & (G - 1);
     const uint32_t CB = CW(prog + DVM_H_COL_BLOCKS);
     uint32_t rb = local_tile, cb = 0;
     if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
     const uint32_t rows = CW(prog + DVM_H_ROWS_LO);  // the host rejects more than 2^32 - 1 rows per program
-    const uint32_t row = rb * (uint32_t)(THREADS >> c.lgG) + (uint32_t)(tid >> c.lgG);
+    c.row0 = rb * (uint32_t)(THREADS >> c.lgG);
+    const uint32_t row = c.row0 + (uint32_t)(tid >> c.lgG);
     const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
     c.col0 = cb * ctile;
     const uint32_t cend = (row == rows - 1) ? CW(prog + DVM_H_LAST_ROW_COLS) : CW(prog + DVM_H_COLS);
     int nc = 0;
     if (row < rows && cend > c.col0) nc = (int)min(cend - c.col0, ctile);
-    c.ncols = nc;
-    c.i0 = row < rows ? row : 0;
+    c.row = row < rows ? row : 0;
+    c.i0 = c.row;
     c.i1 = c.i2 = 0;
     if (c.flags & DVM_F_OUTER_DIMS) {
       const uint32_t n0 = CW(prog + DVM_H_OUTER0), n1 = CW(prog + DVM_H_OUTER1);
@@ -186,38 +232,47 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       c.i2 = q / n1;
       c.i1 = q - c.i2 * n1;
     }
-    c.shift = 0;
-    if (!(c.flags & DVM_F_ALIGNED) && W > 1) {
-      const uint32_t pr = CW(prog + DVM_H_PRIMARY);
-      if (pr != 0xffffffffu) {
-        int dt;
-        const unsigned long long a = reinterpret_cast<unsigned long long>(operand_addr(prog, opd_base(prog), (int)pr, c, dt));
-        c.shift = (int)((a >> (dt == DVM_DT_BF16 ? 1 : 2)) & (unsigned long long)(W - 1));
-      }
+    int shift = 0;
+    if (!(c.flags & DVM_F_ALIGNED)) {
+      // misalignment (in elements) of the row segment start of the primary operand
+      const uint32_t d = opd_base(prog) + CW(prog + DVM_H_PRIMARY) * DVM_OPD_WORDS;
+      const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
+      const uint32_t base_el = (uint32_t)tensor_ptr(prog, d) >> lg_es;
+      uint32_t off;
+      if (c.flags & DVM_F_PRIMARY_DENSE) off = c.row * CW(prog + DVM_H_COLS) + c.col0;  // low bits are all that matter
+      else off = (uint32_t)row_offset(d, c);
+      shift = (int)((base_el + off) & (uint32_t)(W - 1));
     }
+    c.cbase = (t << c.lgW) - shift;
+    if (same_prog && nc == c.ncols && shift == c.shift) return;  // same masks as the previous tile
+    c.ncols = nc;
+    c.shift = shift;
     // In mapping coordinates the segment is [shift, shift + ncols); this thread owns chunks t, t+G, ...
     // The first nf of them are whole, the next one may be cut by the segment's end: a prefix of P slots.
     const int nch = V >> c.lgW;
-    const int n2 = nc > 0 ? nc + c.shift : 0;
-    const int avail = (n2 >> c.lgW) - c.t;                      // whole chunks of the row at or after chunk t
+    const int n2 = nc > 0 ? nc + shift : 0;
+    const int avail = (n2 >> c.lgW) - t;                         // whole chunks of the row at or after chunk t
     int nf = avail > 0 ? ((avail + G - 1) >> c.lgG) : 0;         // those that belong to this thread
     nf = nf < nch ? nf : nch;
-    int rem = nf < nch ? n2 - ((c.t + (nf << c.lgG)) << c.lgW) : 0;
+    int rem = nf < nch ? n2 - ((t + (nf << c.lgG)) << c.lgW) : 0;
     rem = rem > 0 ? (rem < W ? rem : W) : 0;
     const int P = (nf << c.lgW) + rem;
     uint32_t full = (nf >= 32) ? 0xffffffffu : ((1u << nf) - 1u);
     uint32_t part = rem > 0 ? (1u << nf) : 0u;
     uint32_t hm = P >= 8 ? 0xffu : ((1u << P) - 1u);
-    if (c.shift > 0 && c.t == 0 && nc > 0) {
-      // head chunk of a misaligned row: slots [0, shift) lie before the segment and hold its last
-      // columns when the row fills the whole capacity (wrap-around)
-      const int ov = nc + c.shift - (V << c.lgG);
-      hm &= ~((1u << c.shift) - 1u);
-      if (ov > 0) hm |= (1u << ov) - 1u;
+    int ov = 0;
+    if (shift > 0 && t == 0 && nc > 0) {
+      // head chunk of a misaligned row: slots [0, shift) lie before the segment.  A program encoded for
+      // aligned rows that is run on a misaligned tensor may fill its whole capacity: the row's last
+      // `ov` columns then have no slot of their own and wrap around into these head slots.
+      ov = nc + shift - (V << c.lgG);
+      ov = ov > 0 ? ov : 0;
+      hm &= ~((1u << shift) - 1u);
+      hm |= (1u << ov) - 1u;
       full &= ~1u;
       part |= 1u;
     }
-    if (W == 1) { full = 0; part = 0; }  // element-wise mapping: the load / store paths count slots
+    c.ov = ov;
     c.hm = hm;
     c.nvalid = P;
     c.fullmask = full;
@@ -225,132 +280,60 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   };
   auto slot_valid = [&](const TileCtx& c, int s) -> bool { return s < 8 ? ((c.hm >> s) & 1u) != 0 : s < c.nvalid; };
 
-  // ---- one tile load (LDG instruction word w0) into buffer `buf` of its local register ----
-  auto load_tile = [&](const TileCtx& c, uint32_t prog, uint32_t opd0, uint32_t lreg0, uint32_t w0, int buf) {
-    const int ia = DVM_INSN_A(w0) & 0x7f, ib = DVM_INSN_B(w0);
-    const int W = 1 << c.lgW;
-    const int G = 1 << c.lgG;
-    int dt;
-    const char* p = operand_addr(prog, opd0, ib, c, dt);
-    const uint32_t d0 = lreg_addr(CW(lreg0 + ia), buf);
-    const int es = dt == DVM_DT_BF16 ? 2 : 4;
-    if (W == 1) {
-      // element-wise mapping: every valid slot is one scalar copy
-#pragma unroll 1
-      for (int sl = 0; sl < c.nvalid; ++sl) {
-        const int col = c.t + (sl << c.lgG);
-        const uint32_t b = (uint32_t)sl * es;
-        const uint32_t dst = d0 + (b >> 4) * VSTRIDE + (b & 15);
-        if (dt == DVM_DT_BF16) {
-          const unsigned short hv = *reinterpret_cast<const unsigned short*>(p + (long long)col * 2);
-          asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst), "h"(hv) : "memory");
-        } else {
-          cp_async4(dst, p + (long long)col * 4);
-        }
-      }
-      return;
-    }
-    const char* q0 = p + (long long)((c.t << c.lgW) - c.shift) * es;
-    const long long qstep = (long long)(G << c.lgW) * es;
-    const uint32_t mis = (uint32_t)(reinterpret_cast<uintptr_t>(q0) & 15);
-    const uint32_t fast = mis ? 0u : c.fullmask;
-    const uint32_t rea = mis ? c.fullmask : 0u;  // whole chunks at a misaligned address
-    const int vpc = (W * es) >> 4;               // 16-byte vectors per chunk (1 or 2)
-    if (fast && !c.partmask) {
-      // every chunk of this thread is whole and aligned, or empty: one (bf16, fp32 W = 4) or two (fp32 W = 8)
-      // 16-byte copies per chunk, switched off through the copy's source size (an empty chunk is zero-filled),
-      // so that the chunk loop has no branches
-      if (es == 2) {
-#pragma unroll
-        for (int j = 0; j < V / 8; ++j) cp_async16_if(d0 + j * VSTRIDE, q0 + j * qstep, (fast >> j) & 1);
-      } else if (W == 8) {
-#pragma unroll
-        for (int j = 0; j < V / 8; ++j) {
-          cp_async16_if(d0 + (2 * j) * VSTRIDE, q0 + j * qstep, (fast >> j) & 1);
-          cp_async16_if(d0 + (2 * j + 1) * VSTRIDE, q0 + j * qstep + 16, (fast >> j) & 1);
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < V / 4; ++j) cp_async16_if(d0 + j * VSTRIDE, q0 + j * qstep, (fast >> j) & 1);
-      }
-    } else if (fast) {
-      // a chunk of this thread takes the element path below: copy only the whole ones (no zero fill may race with it)
-#pragma unroll 1
-      for (uint32_t m = fast; m; m &= m - 1) {
-        const int j = __ffs(m) - 1;
-        cp_async16(d0 + (j * vpc) * VSTRIDE, q0 + j * qstep);
-        if (vpc == 2) cp_async16(d0 + (j * vpc + 1) * VSTRIDE, q0 + j * qstep + 16);
-      }
-    }
-    if (rea) {
-      // the operand's rows are aligned differently from the tile mapping: fetch the two aligned 16-byte
-      // words that cover each vector and realign them in registers (word select + byte permute)
-      const char* qa = q0 - mis;
-      const uint32_t woff = mis >> 2, sel = (mis & 2) ? 0x5432u : 0x3210u;
-#pragma unroll 1
-      for (uint32_t m = rea; m; m &= m - 1) {
-        const int j = __ffs(m) - 1;
-        for (int v = 0; v < vpc; ++v) {
-          const uint4 a = *reinterpret_cast<const uint4*>(qa + j * qstep + 16 * v);
-          const uint4 bq = *reinterpret_cast<const uint4*>(qa + j * qstep + 16 * v + 16);
-          uint32_t t0 = a.x, t1 = a.y, t2 = a.z, t3 = a.w, t4 = bq.x, t5 = bq.y;
-          if (woff & 2) { t0 = a.z; t1 = a.w; t2 = bq.x; t3 = bq.y; t4 = bq.z; t5 = bq.w; }
-          if (woff & 1) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = t5; }
-          const uint32_t o0 = __byte_perm(t0, t1, sel), o1 = __byte_perm(t1, t2, sel), o2 = __byte_perm(t2, t3, sel),
-                         o3 = __byte_perm(t3, t4, sel);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + (j * vpc + v) * VSTRIDE), "r"(o0), "r"(o1), "r"(o2), "r"(o3)
-                       : "memory");
-        }
-      }
-    }
-    if (c.partmask) {
-      // chunks cut by the row segment's head or tail: predicated element loads, one vector store
-#pragma unroll 1
-      for (uint32_t m = c.partmask; m; m &= m - 1) {
-        const int j = __ffs(m) - 1;
-        if (es == 2) {
-          uint32_t h[8];
-#pragma unroll
-          for (int el = 0; el < 8; ++el) {
-            const int col = chunk_col(c, j, el);
-            h[el] = col < c.ncols ? (uint32_t)*reinterpret_cast<const unsigned short*>(p + (long long)col * 2) : 0u;
-          }
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + j * VSTRIDE), "r"(h[0] | (h[1] << 16)),
-                       "r"(h[2] | (h[3] << 16)), "r"(h[4] | (h[5] << 16)), "r"(h[6] | (h[7] << 16))
-                       : "memory");
-        } else {
-          for (int v = 0; v < vpc; ++v) {
-            uint32_t h[4];
-#pragma unroll
-            for (int el = 0; el < 4; ++el) {
-              const int col = chunk_col(c, j, 4 * v + el);
-              h[el] = col < c.ncols ? *reinterpret_cast<const uint32_t*>(p + (long long)col * 4) : 0u;
-            }
-            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d0 + (j * vpc + v) * VSTRIDE), "r"(h[0]), "r"(h[1]), "r"(h[2]),
-                         "r"(h[3])
-                         : "memory");
-          }
-        }
-      }
-    }
-  };
-
-  // ---- load section of a tile (the first tile of a program on this CTA also loads the tile-invariant inputs) ----
-  auto issue_loads = [&](const TileCtx& c, int buf, bool first_of_program) {
+  // ---- load section of a tile: bulk copies into the images of slot `slot`, one arrival per thread ----
+  auto issue_loads = [&](const TileCtx& c, int slot, bool first_of_program) {
     const uint32_t prog = SINGLE ? kSingleProg : c.prog;
     const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
     const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
+    const uint32_t bar = bar0 + 8 * slot;
+    const uint32_t sb = slot_base(slot);
+    const int t = tid & ((1 << c.lgG) - 1);
     for (uint32_t pc = 0; pc < load_words; ++pc) {
       const uint32_t w0 = CW(body0 + pc);
+      const uint32_t d = opd0 + DVM_INSN_B(w0) * DVM_OPD_WORDS;
       if (DVM_INSN_OP(w0) == DVM_OP_LDG) {
-        if ((DVM_INSN_A(w0) & 0x80) && !first_of_program) continue;  // tile-invariant operand: already in local memory
-        load_tile(c, prog, opd0, lreg0, w0, buf);
-      } else {  // DVM_OP_LDS: one value per row into scalar slot ia of this buffer
-        int dt;
-        const char* p = operand_addr(prog, opd0, DVM_INSN_B(w0), c, dt);
-        const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
+        const uint32_t lw = CW(lreg0 + (DVM_INSN_A(w0) & 0x7f));
+        const uint32_t mode = (lw >> 16) & 0xff;
+        uint32_t dst = sb + (lw & 0xffffu) * DVM_LOCAL_UNIT;
+        const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
+        unsigned long long a = 0, n_el = 0;
+        bool mine = false;
+        if (mode == DVM_LM_BLOCK) {
+          if (tid == 0) {  // thread 0's row is the tile's first row: the whole tile is one byte range from there
+            mine = true;
+            const uint32_t rows = CW(prog + DVM_H_ROWS_LO), C = CW(prog + DVM_H_COLS);
+            const uint32_t R = (uint32_t)(THREADS >> c.lgG);
+            const uint32_t rv = min(R, rows - c.row0);
+            const uint32_t last = (c.row0 + rv == rows) ? CW(prog + DVM_H_LAST_ROW_COLS) : C;
+            a = (unsigned long long)c.row0 * C;
+            n_el = (unsigned long long)(rv - 1) * C + last;
+          }
+        } else if (mode == DVM_LM_ROWS) {
+          if (t == 0 && c.ncols > 0) {
+            mine = true;
+            a = row_offset(d, c);
+            n_el = (unsigned long long)c.ncols;
+            dst += (uint32_t)(tid >> c.lgG) * DVM_ROW_PITCH(1 << c.lgG, V, 1u << lg_es);
+          }
+        } else {  // DVM_LM_BCAST: the same row for every tile of the program
+          if (first_of_program && tid == 0) {
+            mine = true;
+            a = c.col0;
+            n_el = min(CW(prog + DVM_H_COLS) - c.col0, CW(prog + DVM_H_COL_TILE));
+          }
+        }
+        if (mine) {
+          const unsigned long long g0 = tensor_ptr(prog, d) + (a << lg_es);
+          const unsigned long long gs = g0 & ~15ull, ge = (g0 + (n_el << lg_es) + 15ull) & ~15ull;
+          const uint32_t bytes = (uint32_t)(ge - gs);
+          asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+          vm_bulk_load(dst, reinterpret_cast<const void*>(gs), bytes, bar);
+        }
+      } else {  // DVM_OP_LDS: one value per row into scalar slot ia of this tile slot (thread-private)
+        const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+        const char* p = reinterpret_cast<const char*>(tensor_ptr(prog, d) + (row_offset(d, c) << (dt == DVM_DT_BF16 ? 1 : 2)));
         const uint32_t w = (uint32_t)DVM_INSN_A(w0);
-        const uint32_t dst = lreg_addr(unit, buf) + (w >> 2) * VSTRIDE + (w & 3) * 4;
+        const uint32_t dst = sb + (CW(prog + DVM_H_LOCAL2) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16 + (w >> 2) * PSTRIDE + (w & 3) * 4;
         if (c.ncols > 0) {
           if (dt == DVM_DT_BF16) {
             const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(p));
@@ -361,6 +344,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         }
       }
     }
+    vm_mbar_arrive(bar);
   };
 
   float2 A[VP];
@@ -372,36 +356,117 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
 #define DVM_EACH_PAIR _Pragma("unroll") for (int i = 0; i < VP; ++i)
 
-  // reads 16 elements (step h) of the local register at address a0 (element type dt) into o[0..7] as fp32 pairs
-  auto read_step = [&](float2 (&o)[8], uint32_t a0, int dt, int h) {
+  // Where this thread's part of local register k (element type dt) lies in tile slot `buf`:
+  // 16-byte vector u is at  (u & 1 ? a1 : a) + (u >> 1) * vA ;  mis != 0: the vectors are not 16-byte aligned.
+  struct RegView { uint32_t a, a1, vA, mis; bool image; };
+  auto reg_view = [&](const TileCtx& c, uint32_t prog, uint32_t opd0, uint32_t lreg0, int k, int dt, int buf) -> RegView {
+    RegView r;
+    const uint32_t lw = CW(lreg0 + k);
+    const uint32_t mode = (lw >> 16) & 0xff;
+    uint32_t a = slot_base(buf) + (lw & 0xffffu) * DVM_LOCAL_UNIT;
+    if (mode == DVM_LM_PRIVATE) {
+      r.a = a + (uint32_t)tid * 16;
+      r.a1 = r.a + PSTRIDE;
+      r.vA = 2 * PSTRIDE;
+      r.mis = 0;
+      r.image = false;
+      return r;
+    }
+    const uint32_t d = opd0 + (lw >> 24) * DVM_OPD_WORDS;
+    const uint32_t lg_es = dt == DVM_DT_BF16 ? 1 : 2;
+    const uint32_t base_lo = CW(prog + DVM_HDR_WORDS + 2 * (CW(d + DVM_OPD_INFO) & 0xff));
+    const uint32_t rr = (uint32_t)(tid >> c.lgG);
+    uint32_t off;  // element offset (low bits suffice) of the image's first element inside the tensor
+    if (mode == DVM_LM_BLOCK) {
+      const uint32_t C = CW(prog + DVM_H_COLS);
+      off = c.row0 * C;
+      a += (rr * C) << lg_es;
+    } else if (mode == DVM_LM_ROWS) {
+      off = (uint32_t)row_offset(d, c);
+      a += rr * (((uint32_t)V << (c.lgG + lg_es)) + 32u);
+    } else {
+      off = c.col0;
+    }
+    a += ((base_lo + (off << lg_es)) & 15u) + ((uint32_t)c.cbase << lg_es);
+    const uint32_t vstr = (1u << (c.lgG + c.lgW)) << lg_es;  // bytes from one chunk of the thread to its next
+    const bool half = lg_es == 2 && c.lgW == 3;              // an fp32 chunk of 8 elements is two vectors
+    r.a = a;
+    r.a1 = a + (half ? 16u : vstr);
+    r.vA = half ? vstr : 2 * vstr;
+    r.mis = a & 15u;
+    r.image = true;
+    return r;
+  };
+  auto lds128 = [&](uint32_t addr) -> uint4 {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+  };
+  // one 16-byte vector that starts `mis` bytes into an aligned word: the two covering words, realigned
+  auto lds128_realign = [&](uint32_t addr, uint32_t mis) -> uint4 {
+    const uint32_t b = addr - mis;
+    const uint4 x = lds128(b), y = lds128(b + 16);
+    const uint32_t woff = mis >> 2, sel = (mis & 2) ? 0x5432u : 0x3210u;
+    uint32_t t0 = x.x, t1 = x.y, t2 = x.z, t3 = x.w, t4 = y.x, t5 = y.y;
+    if (woff & 2) { t0 = x.z; t1 = x.w; t2 = y.x; t3 = y.y; t4 = y.z; t5 = y.w; }
+    if (woff & 1) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = t5; }
+    return make_uint4(__byte_perm(t0, t1, sel), __byte_perm(t1, t2, sel), __byte_perm(t2, t3, sel), __byte_perm(t3, t4, sel));
+  };
+  auto widen_bf16 = [&](const uint4& v, float2* o) {
+    o[0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+    o[1] = make_float2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+    o[2] = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
+    o[3] = make_float2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+  };
+  // D = L[k] widened to fp32: the whole tile register of this thread.  One warp-uniform branch picks the
+  // variant (element type; aligned vectors or realigned ones); each variant is straight-line code.
+  auto load_reg = [&](float2 (&D)[VP], const TileCtx& c, const RegView& r, int dt) {
+    const bool slow = __any_sync(0xffffffffu, r.mis != 0 || (c.ov > 0 && r.image));
     if (dt == DVM_DT_BF16) {
+      if (!slow) {
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        uint4 v;
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a0 + (2 * h + q) * VSTRIDE));
-        o[4 * q + 0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
-        o[4 * q + 1] = make_float2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
-        o[4 * q + 2] = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
-        o[4 * q + 3] = make_float2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+        for (int u = 0; u < V / 8; ++u) widen_bf16(lds128(((u & 1) ? r.a1 : r.a) + (uint32_t)(u >> 1) * r.vA), &D[4 * u]);
+      } else {
+#pragma unroll
+        for (int u = 0; u < V / 8; ++u)
+          widen_bf16(lds128_realign(((u & 1) ? r.a1 : r.a) + (uint32_t)(u >> 1) * r.vA, r.mis), &D[4 * u]);
       }
     } else {
+      if (!slow) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float4 v;
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a0 + (4 * h + q) * VSTRIDE));
-        o[2 * q] = make_float2(v.x, v.y);
-        o[2 * q + 1] = make_float2(v.z, v.w);
+        for (int u = 0; u < V / 4; ++u) {
+          const uint4 v = lds128(((u & 1) ? r.a1 : r.a) + (uint32_t)(u >> 1) * r.vA);
+          D[2 * u] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+          D[2 * u + 1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < V / 4; ++u) {
+          const uint4 v = lds128_realign(((u & 1) ? r.a1 : r.a) + (uint32_t)(u >> 1) * r.vA, r.mis);
+          D[2 * u] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+          D[2 * u + 1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+        }
       }
     }
-  };
-  // ACC = L[unit]
-  auto read_acc = [&](uint32_t a0, int dt) {
+    if (slow && c.ov > 0 && r.image) {
+      // wrap-around: the first `ov` slots are the columns one chunk past this thread's last chunk
+      float2 e[4];
+      const uint32_t wa = r.a + (uint32_t)(V >> (dt == DVM_DT_BF16 ? 4 : 3)) * r.vA;  // vector index V * es / 16
+      const uint4 v0 = lds128_realign(wa, r.mis);
+      if (dt == DVM_DT_BF16) {
+        widen_bf16(v0, e);
+      } else {
+        const uint4 v1 = lds128_realign(wa + (r.a1 - r.a), r.mis);  // second half of an 8-element chunk (unused when W = 4)
+        e[0] = make_float2(__uint_as_float(v0.x), __uint_as_float(v0.y));
+        e[1] = make_float2(__uint_as_float(v0.z), __uint_as_float(v0.w));
+        e[2] = make_float2(__uint_as_float(v1.x), __uint_as_float(v1.y));
+        e[3] = make_float2(__uint_as_float(v1.z), __uint_as_float(v1.w));
+      }
 #pragma unroll
-    for (int h = 0; h < NST; ++h) {
-      float2 o[8];
-      read_step(o, a0, dt, h);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) A[8 * h + i] = o[i];
+      for (int s2 = 0; s2 < 4; ++s2) {
+        if (2 * s2 < c.ov) D[s2].x = e[s2].x;
+        if (2 * s2 + 1 < c.ov) D[s2].y = e[s2].y;
+      }
     }
   };
 
@@ -413,7 +478,13 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   unsigned err = 0;
 
   TileCtx c;
-  uint32_t slot_prog[2] = {0xffffffffu, 0xffffffffu};  // program whose tile-invariant inputs each slot holds
+  c.prog = 0xffffffffu;
+  c.ncols = -1;
+  c.shift = 0;
+  c.hm = c.fullmask = c.partmask = 0;
+  c.nvalid = 0;
+  c.ov = 0;
+  uint32_t slot_prog[2] = {0xffffffffu, 0xffffffffu};  // program whose row-vector inputs each slot holds
   if (tile < prm.total_tiles) {
     if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
     make_ctx(c, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
@@ -423,15 +494,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   }
 
   while (tile < prm.total_tiles) {
-    // ---- Algorithm 2, outer loop: next tile of this core; its loads start now, into the other tile slot ----
-    uint32_t next;
-    if (use_queue) {
-      if (tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
-      __syncthreads();
-      next = s_next[iter & 1];
-    } else {
-      next = tile + gridDim.x;
-    }
+    // ---- Algorithm 2, outer loop.  Every thread must be done with the previous tile before the other slot
+    // is overwritten with the next tile's loads, which start now, ahead of the wait for this tile's bytes. ----
+    if (use_queue && tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
+    __syncthreads();
+    if (s_abort) break;  // a wait ran out in some thread during the previous tile
+    const uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
     ++iter;
     TileCtx cn = c;
     const bool have_next = next < prm.total_tiles;
@@ -443,9 +511,15 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       issue_loads(cn, buf ^ 1, first);
       if (buf) slot_prog[0] = next_prog_idx; else slot_prog[1] = next_prog_idx;
       cp_async_commit();
-      cp_async_wait<1>();  // this tile's loads have landed once only the next tile's group is pending
+      cp_async_wait<1>();  // this tile's per-row scalars have landed once only the next tile's group is pending
     } else {
       cp_async_wait<0>();
+    }
+    if (!vm_mbar_wait(bar0 + 8 * buf, ((iter - 1) >> 1) & 1)) {
+      // this tile's bytes did not land in time: report it, and leave the loop with everybody at the next
+      // barrier; until then this thread keeps in step (the code it walks has the same barriers for all)
+      err = ST_TIMEOUT;
+      s_abort = 1;
     }
 
     const uint32_t prog = SINGLE ? kSingleProg : c.prog;
@@ -461,43 +535,29 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       const uint32_t w0 = CW(body0 + pc);
       const uint32_t op = DVM_INSN_OP(w0);
       const int ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
-      pc += max(DVM_INSN_LEN(w0), 1u);  // Insn_Len (Algorithm 2); the host verifier rejects 0
+      pc += DVM_INSN_LEN(w0);  // Insn_Len (Algorithm 2); the host verifier rejects 0
 
       if ((op >= DVM_OP_BIN && op < DVM_OP_BINS && ia != DVM_REG_ACC) || op >= DVM_OP_LD2) {
-        // ---- ACC = ACC op L[y]   (LD2: ACC = L[x] first) -- the operand streams from local memory 16 elements
-        // at a time ----
-        uint32_t ay;
-        int dty;
+        // ---- ACC = ACC op L[y]   (LD2: ACC = L[x] first) ----
+        int ky = ia, dty = ib;
         if (op >= DVM_OP_LD2) {
-          read_acc(lreg_addr(CW(lreg0 + ia), buf), (ib >> 6) & 1);
-          ay = lreg_addr(CW(lreg0 + (ib & 0x3f)), buf);
+          const int dtx = (ib >> 6) & 1;
+          load_reg(A, c, reg_view(c, prog, opd0, lreg0, ia, dtx, buf), dtx);
+          ky = ib & 0x3f;
           dty = (ib >> 7) & 1;
-        } else {
-          ay = lreg_addr(CW(lreg0 + ia), buf);
-          dty = ib;
         }
-#define DVM_TILE_OP(...)                                             \
-  _Pragma("unroll") for (int g2 = 0; g2 < NST; g2 += GRP) {          \
-    float2 o[GRP][8];                                                \
-    _Pragma("unroll") for (int h = 0; h < GRP; ++h) read_step(o[h], ay, dty, g2 + h); \
-    _Pragma("unroll") for (int h = 0; h < GRP; ++h)                  \
-      _Pragma("unroll") for (int i = 0; i < 8; ++i) {                \
-        float2& a = A[8 * (g2 + h) + i];                             \
-        const float2 y = o[h][i];                                    \
-        __VA_ARGS__                                                  \
-      }                                                              \
-  }
+        float2 Y[VP];
+        load_reg(Y, c, reg_view(c, prog, opd0, lreg0, ky, dty, buf), dty);
         switch (op & 7) {
-          case DVM_A_ADD: DVM_TILE_OP(a = __fadd2_rn(a, y);) break;
-          case DVM_A_SUB: DVM_TILE_OP(a = __ffma2_rn(y, make_float2(-1.f, -1.f), a);) break;
-          case DVM_A_RSUB: DVM_TILE_OP(a = __ffma2_rn(a, make_float2(-1.f, -1.f), y);) break;
-          case DVM_A_MUL: DVM_TILE_OP(a = __fmul2_rn(a, y);) break;
-          case DVM_A_DIV: DVM_TILE_OP(a = make_float2(fast_div(a.x, y.x), fast_div(a.y, y.y));) break;
-          case DVM_A_RDIV: DVM_TILE_OP(a = make_float2(fast_div(y.x, a.x), fast_div(y.y, a.y));) break;
-          case DVM_A_MIN: DVM_TILE_OP(a = make_float2(a.x < y.x ? a.x : y.x, a.y < y.y ? a.y : y.y);) break;
-          default: DVM_TILE_OP(a = make_float2(a.x > y.x ? a.x : y.x, a.y > y.y ? a.y : y.y);) break;
+          case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], Y[i]); break;
+          case DVM_A_SUB: DVM_EACH_PAIR A[i] = __ffma2_rn(Y[i], make_float2(-1.f, -1.f), A[i]); break;
+          case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), Y[i]); break;
+          case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], Y[i]); break;
+          case DVM_A_DIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, Y[i].x), fast_div(A[i].y, Y[i].y)); break;
+          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(Y[i].x, A[i].x), fast_div(Y[i].y, A[i].y)); break;
+          case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < Y[i].x ? A[i].x : Y[i].x, A[i].y < Y[i].y ? A[i].y : Y[i].y); break;
+          default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > Y[i].x ? A[i].x : Y[i].x, A[i].y > Y[i].y ? A[i].y : Y[i].y); break;
         }
-#undef DVM_TILE_OP
         continue;
       }
       if (op >= DVM_OP_BINI && op < DVM_OP_UN) {
@@ -619,46 +679,50 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       switch (op) {
         case DVM_OP_NOP: break;
         case DVM_OP_LDA: {
-          read_acc(lreg_addr(CW(lreg0 + ia), buf), ib);
+          load_reg(A, c, reg_view(c, prog, opd0, lreg0, ia, ib, buf), ib);
         } break;
         case DVM_OP_STA: {
-          const uint32_t a0 = lreg_addr(CW(lreg0 + ia), buf);
+          const uint32_t a0 = slot_base(buf) + (CW(lreg0 + ia) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16;
 #pragma unroll
           for (int q = 0; q < V / 4; ++q)
-            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * VSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * PSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
                          "f"(A[2 * q + 1].x), "f"(A[2 * q + 1].y)
                          : "memory");
         } break;
         case DVM_OP_LSS: {
-          const uint32_t unit = (CW(prog + DVM_H_LOCAL2) >> 8) & 0xff;
           const uint32_t w = (uint32_t)ib;
           float v;
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lreg_addr(unit, buf) + (w >> 2) * VSTRIDE + (w & 3) * 4));
+          asm volatile("ld.shared.f32 %0, [%1];"
+                       : "=f"(v)
+                       : "r"(slot_base(buf) + (CW(prog + DVM_H_LOCAL2) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16 +
+                             (w >> 2) * PSTRIDE + (w & 3) * 4));
           sset(S, ia, c.ncols > 0 ? v : 0.f);
         } break;
         case DVM_OP_STG: {
-          int dt;
-          char* p = operand_addr(prog, opd0, ib, c, dt);
-          const int es = dt == DVM_DT_BF16 ? 2 : 4;
-          if (W == 1) {
-            // element-wise mapping: one predicated scalar store per slot
-#pragma unroll
-            for (int sl = 0; sl < V; ++sl) {
-              if (sl < c.nvalid) {
-                const long long col = c.t + (sl << c.lgG);
-                const float val = (sl & 1) ? A[sl >> 1].y : A[sl >> 1].x;
-                if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + col * 2) = __float2bfloat16_rn(val);
-                else *reinterpret_cast<float*>(p + col * 4) = val;
-              }
-            }
-            break;
-          }
-          char* q0 = p + (long long)((c.t << c.lgW) - c.shift) * es;
-          const long long qstep = (long long)(G << c.lgW) * es;
+          // an output covers the dominant shape: element (row, col) lies at row * C + col
+          const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
+          const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+          const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
+          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) +
+                                            (((unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0) << lg_es));
+          char* q0 = p + ((long long)c.cbase << lg_es);
+          const long long qstep = (long long)((G << c.lgW) << lg_es);
           const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
           const uint32_t fast = al ? c.fullmask : 0u;
           const uint32_t slow = c.partmask | (c.fullmask & ~fast);
-          if (dt == DVM_DT_BF16) {  // W == 8
+          constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
+          if (dt == DVM_DT_BF16 && fast == ALL8) {  // every chunk whole and aligned: straight-line stores
+#pragma unroll
+            for (int j = 0; j < V / 8; ++j) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn(A[4 * j + q].x, A[4 * j + q].y);
+                pk[q] = *reinterpret_cast<const uint32_t*>(&b);
+              }
+              *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          } else if (dt == DVM_DT_BF16) {  // W == 8
 #pragma unroll
             for (int j = 0; j < V / 8; ++j) {
               if ((fast >> j) & 1) {
@@ -703,9 +767,10 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 #pragma unroll
               for (int el = 0; el < 8; ++el) {
                 if (el < W) {
-                  const int col = chunk_col(c, j, el);
+                  int col = c.cbase + (j << (c.lgG + c.lgW)) + el;
+                  if (col < 0 && c.ov > 0) col += V << c.lgG;  // wrap-around slots of the row's first thread
                   const float val = (el & 1) ? tp[el >> 1].y : tp[el >> 1].x;
-                  if (col < c.ncols) {
+                  if (col >= 0 && col < c.ncols) {
                     if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
                     else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
                   }
@@ -715,10 +780,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           }
         } break;
         case DVM_OP_STS: {
-          int dt;
-          char* p = operand_addr(prog, opd0, ib, c, dt);
+          const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
+          const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << (dt == DVM_DT_BF16 ? 1 : 2)));
           const float v = sget(S, ia);
-          if (c.ncols > 0 && c.t == 0 && c.col0 == 0) {
+          if (c.ncols > 0 && (tid & (G - 1)) == 0 && c.col0 == 0) {
             if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
             else *reinterpret_cast<float*>(p) = v;
           }

@@ -38,7 +38,7 @@ def test_add_rmsnorm_max_rows_sampled(rows):
         g1, g2 = gate_errors(wl.to_f64(got[ti]), ref)
         assert g2 <= 2e-2, (g1, g2)
     # every row was written: no poison left anywhere
-    assert not torch.isnan(y.view(torch.int16).bitwise_and(0x7fff).float().max()) and not torch.isnan(y.float().sum())
+    assert not torch.isnan(y.float().sum()) and not torch.isnan(h.float().sum())
 
 
 @pytest.mark.parametrize("B,S", [(8, 2048), (8, 2047), (3, 1531)])

@@ -5,6 +5,7 @@ import pytest
 import torch
 
 import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
 from tests.parity_util import check, gpu_run, oracle_run
 
 pytestmark = pytest.mark.gpu
@@ -98,6 +99,43 @@ def test_unaligned_base_pointers():
     ins = [xs[1:].view(9, 256), full[1].cuda(), full[2].cuda()]
     outs, _ = gpu_run(prog, ins)
     check(prog, outs, oracle_run(prog, ins), strict=True)
+
+
+def _shifted(t: torch.Tensor, k: int) -> torch.Tensor:
+    """A device copy of t that starts k elements into its allocation."""
+    buf = torch.empty(t.numel() + k, dtype=t.dtype, device="cuda")
+    buf[k:] = t.flatten().cuda()
+    return buf[k:].view(t.shape)
+
+
+@pytest.mark.parametrize("kx,kres,kw,ky", [(1, 0, 0, 0), (3, 3, 0, 0), (5, 2, 7, 0), (0, 1, 0, 3), (7, 7, 7, 7)])
+def test_full_capacity_rows_on_misaligned_tensors(kx, kres, kw, ky):
+    """Rows of 4096 bf16 fill the whole tile capacity; on a misaligned primary tensor the rows' last columns
+    wrap around into the head slots, other operands are realigned, misaligned outputs take the element path."""
+    prog = wl.program_add_rmsnorm(4096)
+    full = wl.inputs_add_rmsnorm(37, 4096, 5)
+    ins = [_shifted(full[0], kx), _shifted(full[1], kres), _shifted(full[2], kw)]
+    p = dvm.program_from_nodes(prog.nodes)
+    code = dvm.encode(p, [tuple(t.shape) for t in ins])
+    outs = [_shifted(torch.full((37, 4096), float("nan"), dtype=torch.bfloat16), ky),
+            _shifted(torch.full((37, 4096), float("nan"), dtype=torch.bfloat16), 0)]
+    dvm.launch(code, ins + outs)
+    assert dvm.last_device_status() == 0
+    check(prog, outs, oracle_run(prog, full), strict=True)
+
+
+@pytest.mark.parametrize("cols,k", [(4096, 1), (4095, 0), (4093, 2), (2048, 3), (100, 1)])
+def test_layernorm_misaligned_fp32(cols, k):
+    """fp32 rows at and next to the full capacity, tensor shifted by k elements."""
+    prog = wl.program_layernorm()
+    x = wl.randn((19, cols), torch.float32, cols + k)
+    xs = _shifted(x, k)
+    p = dvm.program_from_nodes(prog.nodes)
+    code = dvm.encode(p, [(19, cols)], [1.0 / cols])
+    out = torch.full((19, cols), float("nan"), dtype=torch.float32, device="cuda")
+    dvm.launch(code, [xs, out])
+    assert dvm.last_device_status() == 0
+    check(prog, [out], oracle_run(prog, [x], [1.0 / cols]))
 
 
 def test_every_unary_and_binary_op():
