@@ -58,7 +58,9 @@ enum {
                         // boundary provided its base pointer is 16-byte aligned
   DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
   DVM_F_FLAT = 4,       // pure elementwise program laid out as a flat range
-  DVM_F_PRIMARY_DENSE = 8  // the primary operand is dense: row r starts at element r * C of its tensor
+  DVM_F_PRIMARY_DENSE = 8, // the primary operand is dense: row r starts at element r * C of its tensor
+  DVM_F_LOADS_BY_ROW = 16  // some load is issued per row (row-by-row images, per-row scalars); otherwise
+                           // thread 0 alone issues every copy of a tile
 };
 
 // ---- local register table: one word per local register: unit offset inside a tile slot | mode << 16 ----
@@ -90,7 +92,7 @@ enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
 #define DVM_MAX_LREGS 10         // local tile registers of a program (inputs + temporaries)
 #define DVM_MAX_SSLOTS 8         // per-row scalar inputs of a program
 #define DVM_LOCAL_UNIT 256       // bytes of one local-memory unit (layout granule)
-#define DVM_MAX_LOCAL_UNITS 896  // units a CTA can hold (two tile slots), 224 KB
+#define DVM_MAX_LOCAL_UNITS 864  // units a CTA can hold (two tile slots + the spare unit), 216 KB
 #define DVM_MAX_SREGS 8          // per-row scalar registers
 #define DVM_MAX_TENSORS 16
 #define DVM_MAX_OPERANDS 24

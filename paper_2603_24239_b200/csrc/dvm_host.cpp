@@ -921,7 +921,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
       g.scalar_unit = g.units;
       if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
       if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) break;
-      int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 1280);  // 228 KB per SM, 1 KB reserved per CTA + static
+      int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
       if (ctas > 2) ctas = 2;  // the interpreter is compiled for two resident CTAs per SM
       if (ctas < 1) break;
       // the geometry was costed for ctas_guess resident CTAs per SM: at least that many must fit
@@ -960,6 +960,9 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   }
   if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
   if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
+  if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
+  for (int k = 0; k < e.n_in_regs; ++k)
+    if (((best.lreg_table[k] >> 16) & 0xff) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;

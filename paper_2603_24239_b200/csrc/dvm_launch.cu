@@ -18,7 +18,7 @@ constexpr int PW_SMALL = 496;    // words of code in a 2 KB parameter block
 constexpr int PW_LARGE = 8000;   // ... in a 32 KB parameter block (the sm_70+ limit is 32764 bytes)
 constexpr int QUEUE_SLOTS = 504;
 constexpr int MAX_DEVICES = 64;
-constexpr size_t kMaxDynSmem = 227 * 1024 - 256;  // dynamic shared memory a CTA may ask for (static part excluded)
+constexpr size_t kMaxDynSmem = 227 * 1024 - 9 * 1024;  // dynamic shared memory a CTA may ask for (8.3 KB static part excluded)
 
 struct DeviceState {
   bool ready = false;

@@ -84,17 +84,6 @@ struct TileCtx {
   uint32_t flags;
 };
 
-__device__ __forceinline__ float sget(const float (&S)[DVM_MAX_SREGS], int k) {
-  float v = S[0];
-#pragma unroll
-  for (int i = 1; i < DVM_MAX_SREGS; ++i) v = (k == i) ? S[i] : v;
-  return v;
-}
-__device__ __forceinline__ void sset(float (&S)[DVM_MAX_SREGS], int k, float v) {
-#pragma unroll
-  for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = (k == i) ? v : S[i];
-}
-
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -155,6 +144,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ float s_red[2][THREADS / 32];
   __shared__ uint32_t s_next[2];
+  __shared__ float s_S[DVM_MAX_SREGS][THREADS];  // per-row scalar registers S0..S7 of every thread
   __shared__ __align__(8) unsigned long long s_bar[2];  // "tile landed" barrier of each tile slot
   __shared__ volatile uint32_t s_abort;
 
@@ -286,6 +276,10 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
     const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
     const uint32_t bar = bar0 + 8 * slot;
+    if (!(c.flags & DVM_F_LOADS_BY_ROW) && warp != 0) {  // thread 0 issues every copy of this program's tiles
+      vm_mbar_arrive(bar);
+      return;
+    }
     const uint32_t sb = slot_base(slot);
     const int t = tid & ((1 << c.lgG) - 1);
     for (uint32_t pc = 0; pc < load_words; ++pc) {
@@ -348,9 +342,6 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   };
 
   float2 A[VP];
-  float S[DVM_MAX_SREGS];
-#pragma unroll
-  for (int i = 0; i < DVM_MAX_SREGS; ++i) S[i] = 0.f;
 #pragma unroll
   for (int i = 0; i < VP; ++i) A[i] = make_float2(0.f, 0.f);
 
@@ -529,68 +520,76 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const int G = 1 << c.lgG;
     const bool all_valid = __all_sync(0xffffffffu, c.nvalid == V && c.hm == 0xffu);
 
-    // ---- Algorithm 2, inner loop: walk the compute section ----
-    uint32_t pc = CW(prog + DVM_H_LOAD_WORDS);
-    while (pc < body_words) {
-      const uint32_t w0 = CW(body0 + pc);
+    // ---- Algorithm 2, inner loop: walk the compute section.  Two-level dispatch: the instruction class
+    // (op >> 3) picks the handler through one jump table, the handler decodes only the fields it uses. ----
+    uint32_t pc = body0 + CW(prog + DVM_H_LOAD_WORDS);
+    const uint32_t pc_end = body0 + body_words;
+    while (pc < pc_end) {
+      const uint32_t w0 = CW(pc);
       const uint32_t op = DVM_INSN_OP(w0);
-      const int ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
-      pc += DVM_INSN_LEN(w0);  // Insn_Len (Algorithm 2); the host verifier rejects 0
-
-      if ((op >= DVM_OP_BIN && op < DVM_OP_BINS && ia != DVM_REG_ACC) || op >= DVM_OP_LD2) {
-        // ---- ACC = ACC op L[y]   (LD2: ACC = L[x] first) ----
-        int ky = ia, dty = ib;
-        if (op >= DVM_OP_LD2) {
-          const int dtx = (ib >> 6) & 1;
-          load_reg(A, c, reg_view(c, prog, opd0, lreg0, ia, dtx, buf), dtx);
-          ky = ib & 0x3f;
-          dty = (ib >> 7) & 1;
-        }
-        float2 Y[VP];
-        load_reg(Y, c, reg_view(c, prog, opd0, lreg0, ky, dty, buf), dty);
-        switch (op & 7) {
-          case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], Y[i]); break;
-          case DVM_A_SUB: DVM_EACH_PAIR A[i] = __ffma2_rn(Y[i], make_float2(-1.f, -1.f), A[i]); break;
-          case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), Y[i]); break;
-          case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], Y[i]); break;
-          case DVM_A_DIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, Y[i].x), fast_div(A[i].y, Y[i].y)); break;
-          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(Y[i].x, A[i].x), fast_div(Y[i].y, A[i].y)); break;
-          case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < Y[i].x ? A[i].x : Y[i].x, A[i].y < Y[i].y ? A[i].y : Y[i].y); break;
-          default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > Y[i].x ? A[i].x : Y[i].x, A[i].y > Y[i].y ? A[i].y : Y[i].y); break;
-        }
-        continue;
-      }
-      if (op >= DVM_OP_BINI && op < DVM_OP_UN) {
-        // ---- ACC = ACC op y : y an immediate, a per-row scalar, or ACC itself ----
-        if (op >= DVM_OP_BIN && op < DVM_OP_BINS) {  // ACC op ACC
-          switch (op & 7) {
-            case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], A[i]); break;
-            case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], A[i]); break;
-            case DVM_A_SUB: case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), A[i]); break;
-            case DVM_A_DIV: case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, A[i].x), fast_div(A[i].y, A[i].y)); break;
-            default: break;  // min / max of a value with itself
+      switch (op >> 3) {
+        case DVM_OP_BIN >> 3:
+          if (DVM_INSN_A(w0) == DVM_REG_ACC) {  // ACC = ACC op ACC
+            pc += 1;
+            switch (op & 7) {
+              case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], A[i]); break;
+              case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], A[i]); break;
+              case DVM_A_SUB: case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), A[i]); break;
+              case DVM_A_DIV: case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, A[i].x), fast_div(A[i].y, A[i].y)); break;
+              default: break;  // min / max of a value with itself
+            }
+            break;
           }
-          continue;
-        }
-        const float y = op >= DVM_OP_BINS ? sget(S, ia) : __uint_as_float(CW(body0 + pc - 1));
-        const float2 y2 = make_float2(y, y);
-        switch (op & 7) {
-          case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], y2); break;
-          case DVM_A_SUB: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], make_float2(-y, -y)); break;
-          case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), y2); break;
-          case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], y2); break;
-          case DVM_A_DIV: {
-            // division by a per-row scalar or an immediate: one SFU reciprocal (1 ulp), packed multiplies
-            const float rcp = fast_rcp(y);
-            DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], make_float2(rcp, rcp));
-          } break;
-          case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(y, A[i].x), fast_div(y, A[i].y)); break;
-          case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < y ? A[i].x : y, A[i].y < y ? A[i].y : y); break;
-          default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > y ? A[i].x : y, A[i].y > y ? A[i].y : y); break;
-        }
-        continue;
-      }
-      if (op >= DVM_OP_UN && op < DVM_OP_RED) {
+          // fall through: ACC = ACC op L[y]
+        case DVM_OP_LD2 >> 3: {
+          // ---- ACC = ACC op L[y]   (LD2: ACC = L[x] first) ----
+          pc += 1;
+          int ky = DVM_INSN_A(w0), dty = DVM_INSN_B(w0);
+          if (op >= DVM_OP_LD2) {
+            const int ib = DVM_INSN_B(w0);
+            const int dtx = (ib >> 6) & 1;
+            load_reg(A, c, reg_view(c, prog, opd0, lreg0, ky, dtx, buf), dtx);
+            ky = ib & 0x3f;
+            dty = (ib >> 7) & 1;
+          }
+          float2 Y[VP];
+          load_reg(Y, c, reg_view(c, prog, opd0, lreg0, ky, dty, buf), dty);
+          switch (op & 7) {
+            case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], Y[i]); break;
+            case DVM_A_SUB: DVM_EACH_PAIR A[i] = __ffma2_rn(Y[i], make_float2(-1.f, -1.f), A[i]); break;
+            case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), Y[i]); break;
+            case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], Y[i]); break;
+            case DVM_A_DIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(A[i].x, Y[i].x), fast_div(A[i].y, Y[i].y)); break;
+            case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(Y[i].x, A[i].x), fast_div(Y[i].y, A[i].y)); break;
+            case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < Y[i].x ? A[i].x : Y[i].x, A[i].y < Y[i].y ? A[i].y : Y[i].y); break;
+            default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > Y[i].x ? A[i].x : Y[i].x, A[i].y > Y[i].y ? A[i].y : Y[i].y); break;
+          }
+        } break;
+        case DVM_OP_BINI >> 3:
+        case DVM_OP_BINS >> 3: {
+          // ---- ACC = ACC op y : y an immediate (word 1) or a per-row scalar ----
+          float y;
+          if (op >= DVM_OP_BINS) { y = s_S[DVM_INSN_A(w0)][tid]; pc += 1; }
+          else { y = __uint_as_float(CW(pc + 1)); pc += 2; }
+          const float2 y2 = make_float2(y, y);
+          switch (op & 7) {
+            case DVM_A_ADD: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], y2); break;
+            case DVM_A_SUB: DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], make_float2(-y, -y)); break;
+            case DVM_A_RSUB: DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(-1.f, -1.f), y2); break;
+            case DVM_A_MUL: DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], y2); break;
+            case DVM_A_DIV: {
+              // division by a per-row scalar or an immediate: one SFU reciprocal (1 ulp), packed multiplies
+              const float rcp = fast_rcp(y);
+              DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], make_float2(rcp, rcp));
+            } break;
+            case DVM_A_RDIV: DVM_EACH_PAIR A[i] = make_float2(fast_div(y, A[i].x), fast_div(y, A[i].y)); break;
+            case DVM_A_MIN: DVM_EACH_PAIR A[i] = make_float2(A[i].x < y ? A[i].x : y, A[i].y < y ? A[i].y : y); break;
+            default: DVM_EACH_PAIR A[i] = make_float2(A[i].x > y ? A[i].x : y, A[i].y > y ? A[i].y : y); break;
+          }
+        } break;
+        case DVM_OP_UN >> 3:
+        case (DVM_OP_UN >> 3) + 1: {
+          pc += 1;
 #define DVM_UN_CASE(U, EXPR)                                                          \
   case U:                                                                             \
     DVM_EACH_PAIR {                                                                   \
@@ -599,216 +598,226 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       A[i] = make_float2(vx, vy);                                                     \
     }                                                                                 \
     break;
-        switch (op - DVM_OP_UN) {
-          DVM_UN_CASE(DVM_U_EXP, fast_exp(x))
-          DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
-          DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
-          DVM_UN_CASE(DVM_U_ABS, fabsf(x))
-          DVM_UN_CASE(DVM_U_LOG, logf(x))
-          DVM_UN_CASE(DVM_U_ERF, erff(x))
-          DVM_UN_CASE(DVM_U_SIGMOID, fast_rcp(1.0f + fast_exp(-x)))
-          DVM_UN_CASE(DVM_U_NEG, -x)
-          DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
-          DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
-          DVM_UN_CASE(DVM_U_ROUND, rintf(x))
-          DVM_UN_CASE(DVM_U_TANH, tanhf(x))
-          default:
-            DVM_EACH_PAIR A[i] = make_float2(round_bf16(A[i].x), round_bf16(A[i].y));
-            break;
-        }
+          switch (op - DVM_OP_UN) {
+            DVM_UN_CASE(DVM_U_EXP, fast_exp(x))
+            DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
+            DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
+            DVM_UN_CASE(DVM_U_ABS, fabsf(x))
+            DVM_UN_CASE(DVM_U_LOG, logf(x))
+            DVM_UN_CASE(DVM_U_ERF, erff(x))
+            DVM_UN_CASE(DVM_U_SIGMOID, fast_rcp(1.0f + fast_exp(-x)))
+            DVM_UN_CASE(DVM_U_NEG, -x)
+            DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
+            DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
+            DVM_UN_CASE(DVM_U_ROUND, rintf(x))
+            DVM_UN_CASE(DVM_U_TANH, tanhf(x))
+            default:
+              DVM_EACH_PAIR A[i] = make_float2(round_bf16(A[i].x), round_bf16(A[i].y));
+              break;
+          }
 #undef DVM_UN_CASE
-        continue;
-      }
-      if (op >= DVM_OP_RED && op < DVM_OP_LD2) {
-        // ---- row reduction (Table 1, Sum / Max / Min with N = 1): thread-local over valid slots, shuffles
-        // inside the warp, shared memory across the warps of a row group ----
-        const int rop = op - DVM_OP_RED;
-        float v;
-        if (rop == DVM_R_SUM || rop == DVM_R_SUMSQ) {
-          float2 acc = make_float2(0.f, 0.f);
-          if (all_valid) {
-            if (rop == DVM_R_SUM) { DVM_EACH_PAIR acc = __fadd2_rn(acc, A[i]); }
-            else { DVM_EACH_PAIR acc = __ffma2_rn(A[i], A[i], acc); }
-          } else {
-            DVM_EACH_PAIR {
-              const float2 x = make_float2(slot_valid(c, 2 * i) ? A[i].x : 0.f, slot_valid(c, 2 * i + 1) ? A[i].y : 0.f);
-              acc = rop == DVM_R_SUM ? __fadd2_rn(acc, x) : __ffma2_rn(x, x, acc);
-            }
-          }
-          v = acc.x + acc.y;
-#pragma unroll
-          for (int sh = 1; sh < 32; sh <<= 1)
-            if (sh < G) v += __shfl_xor_sync(0xffffffffu, v, sh);
-        } else {
-          const bool mx = rop == DVM_R_MAX;
-          const float ident = mx ? -INFINITY : INFINITY;
-          v = ident;
-          if (all_valid) {
-            DVM_EACH_PAIR v = mx ? fmaxf(v, fmaxf(A[i].x, A[i].y)) : fminf(v, fminf(A[i].x, A[i].y));
-          } else {
-            DVM_EACH_PAIR {
-              const float x0 = slot_valid(c, 2 * i) ? A[i].x : ident;
-              const float x1 = slot_valid(c, 2 * i + 1) ? A[i].y : ident;
-              v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
-            }
-          }
-#pragma unroll
-          for (int sh = 1; sh < 32; sh <<= 1)
-            if (sh < G) {
-              const float x = __shfl_xor_sync(0xffffffffu, v, sh);
-              v = mx ? fmaxf(v, x) : fminf(v, x);
-            }
-        }
-        if (G > 32) {
-          if (lane == 0) s_red[red_par][warp] = v;
-          __syncthreads();
-          const int wpg = G >> 5;  // warps per row group
-          const int w0i = warp & ~(wpg - 1);
-          float acc = s_red[red_par][w0i];
-          for (int i = 1; i < wpg; ++i) {
-            const float x = s_red[red_par][w0i + i];
-            acc = rop == DVM_R_MAX ? fmaxf(acc, x) : (rop == DVM_R_MIN ? fminf(acc, x) : acc + x);
-          }
-          v = acc;
-          red_par ^= 1;
-        }
-        sset(S, ia, v);
-        continue;
-      }
-
-      switch (op) {
-        case DVM_OP_NOP: break;
-        case DVM_OP_LDA: {
-          load_reg(A, c, reg_view(c, prog, opd0, lreg0, ia, ib, buf), ib);
         } break;
-        case DVM_OP_STA: {
-          const uint32_t a0 = slot_base(buf) + (CW(lreg0 + ia) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16;
-#pragma unroll
-          for (int q = 0; q < V / 4; ++q)
-            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * PSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
-                         "f"(A[2 * q + 1].x), "f"(A[2 * q + 1].y)
-                         : "memory");
-        } break;
-        case DVM_OP_LSS: {
-          const uint32_t w = (uint32_t)ib;
+        case DVM_OP_RED >> 3: {
+          // ---- row reduction (Table 1, Sum / Max / Min with N = 1): thread-local over valid slots, shuffles
+          // inside the warp, shared memory across the warps of a row group ----
+          pc += 1;
+          const int rop = op & 7;
           float v;
-          asm volatile("ld.shared.f32 %0, [%1];"
-                       : "=f"(v)
-                       : "r"(slot_base(buf) + (CW(prog + DVM_H_LOCAL2) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16 +
-                             (w >> 2) * PSTRIDE + (w & 3) * 4));
-          sset(S, ia, c.ncols > 0 ? v : 0.f);
-        } break;
-        case DVM_OP_STG: {
-          // an output covers the dominant shape: element (row, col) lies at row * C + col
-          const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
-          const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
-          const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
-          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) +
-                                            (((unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0) << lg_es));
-          char* q0 = p + ((long long)c.cbase << lg_es);
-          const long long qstep = (long long)((G << c.lgW) << lg_es);
-          const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
-          const uint32_t fast = al ? c.fullmask : 0u;
-          const uint32_t slow = c.partmask | (c.fullmask & ~fast);
-          constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
-          if (dt == DVM_DT_BF16 && fast == ALL8) {  // every chunk whole and aligned: straight-line stores
-#pragma unroll
-            for (int j = 0; j < V / 8; ++j) {
-              uint32_t pk[4];
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const __nv_bfloat162 b = __floats2bfloat162_rn(A[4 * j + q].x, A[4 * j + q].y);
-                pk[q] = *reinterpret_cast<const uint32_t*>(&b);
+          if (rop == DVM_R_SUM || rop == DVM_R_SUMSQ) {
+            float2 acc = make_float2(0.f, 0.f);
+            if (all_valid) {
+              if (rop == DVM_R_SUM) { DVM_EACH_PAIR acc = __fadd2_rn(acc, A[i]); }
+              else { DVM_EACH_PAIR acc = __ffma2_rn(A[i], A[i], acc); }
+            } else {
+              DVM_EACH_PAIR {
+                const float2 x = make_float2(slot_valid(c, 2 * i) ? A[i].x : 0.f, slot_valid(c, 2 * i + 1) ? A[i].y : 0.f);
+                acc = rop == DVM_R_SUM ? __fadd2_rn(acc, x) : __ffma2_rn(x, x, acc);
               }
-              *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
-          } else if (dt == DVM_DT_BF16) {  // W == 8
+            v = acc.x + acc.y;
 #pragma unroll
-            for (int j = 0; j < V / 8; ++j) {
-              if ((fast >> j) & 1) {
+            for (int sh = 1; sh < 32; sh <<= 1)
+              if (sh < G) v += __shfl_xor_sync(0xffffffffu, v, sh);
+          } else {
+            const bool mx = rop == DVM_R_MAX;
+            const float ident = mx ? -INFINITY : INFINITY;
+            v = ident;
+            if (all_valid) {
+              DVM_EACH_PAIR v = mx ? fmaxf(v, fmaxf(A[i].x, A[i].y)) : fminf(v, fminf(A[i].x, A[i].y));
+            } else {
+              DVM_EACH_PAIR {
+                const float x0 = slot_valid(c, 2 * i) ? A[i].x : ident;
+                const float x1 = slot_valid(c, 2 * i + 1) ? A[i].y : ident;
+                v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
+              }
+            }
+#pragma unroll
+            for (int sh = 1; sh < 32; sh <<= 1)
+              if (sh < G) {
+                const float x = __shfl_xor_sync(0xffffffffu, v, sh);
+                v = mx ? fmaxf(v, x) : fminf(v, x);
+              }
+          }
+          if (G > 32) {
+            if (lane == 0) s_red[red_par][warp] = v;
+            __syncthreads();
+            const int wpg = G >> 5;  // warps per row group: 2, 4 or 8
+            const float* pr = &s_red[red_par][warp & ~(wpg - 1)];
+            float x[8];
+            x[0] = pr[0]; x[1] = pr[1];
+            const float id2 = rop == DVM_R_MAX ? -INFINITY : (rop == DVM_R_MIN ? INFINITY : 0.f);
+#pragma unroll
+            for (int i = 2; i < 8; ++i) x[i] = id2;
+            if (wpg > 2) { x[2] = pr[2]; x[3] = pr[3]; }
+            if (wpg > 4) { x[4] = pr[4]; x[5] = pr[5]; x[6] = pr[6]; x[7] = pr[7]; }
+            if (rop == DVM_R_MAX) v = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+            else if (rop == DVM_R_MIN) v = fminf(fminf(fminf(x[0], x[1]), fminf(x[2], x[3])), fminf(fminf(x[4], x[5]), fminf(x[6], x[7])));
+            else v = ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
+            red_par ^= 1;
+          }
+          s_S[DVM_INSN_A(w0)][tid] = v;
+        } break;
+        case 0: {  // NOP LDG LDS LDA STA LSS STG STS
+          pc += 1;
+          const int ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
+          if (op == DVM_OP_LDA) {
+            load_reg(A, c, reg_view(c, prog, opd0, lreg0, ia, ib, buf), ib);
+          } else if (op == DVM_OP_STA) {
+            const uint32_t a0 = slot_base(buf) + (CW(lreg0 + ia) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16;
+#pragma unroll
+            for (int q = 0; q < V / 4; ++q)
+              asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * PSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
+                           "f"(A[2 * q + 1].x), "f"(A[2 * q + 1].y)
+                           : "memory");
+          } else if (op == DVM_OP_LSS) {
+            const uint32_t w = (uint32_t)ib;
+            float v;
+            asm volatile("ld.shared.f32 %0, [%1];"
+                         : "=f"(v)
+                         : "r"(slot_base(buf) + (CW(prog + DVM_H_LOCAL2) & 0xffffu) * DVM_LOCAL_UNIT + (uint32_t)tid * 16 +
+                               (w >> 2) * PSTRIDE + (w & 3) * 4));
+            s_S[ia][tid] = c.ncols > 0 ? v : 0.f;
+          } else if (op == DVM_OP_STG) {
+            // an output covers the dominant shape: element (row, col) lies at row * C + col
+            const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
+            const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+            const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
+            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) +
+                                              (((unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0) << lg_es));
+            char* q0 = p + ((long long)c.cbase << lg_es);
+            const long long qstep = (long long)((G << c.lgW) << lg_es);
+            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
+            const uint32_t fast = al ? c.fullmask : 0u;
+            const uint32_t slow = c.partmask | (c.fullmask & ~fast);
+            constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
+            if (dt == DVM_DT_BF16 && fast == ALL8) {  // every chunk whole and aligned: straight-line stores
+  #pragma unroll
+              for (int j = 0; j < V / 8; ++j) {
                 uint32_t pk[4];
-#pragma unroll
+  #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                   const __nv_bfloat162 b = __floats2bfloat162_rn(A[4 * j + q].x, A[4 * j + q].y);
                   pk[q] = *reinterpret_cast<const uint32_t*>(&b);
                 }
                 *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
               }
+            } else if (dt == DVM_DT_BF16) {  // W == 8
+  #pragma unroll
+              for (int j = 0; j < V / 8; ++j) {
+                if ((fast >> j) & 1) {
+                  uint32_t pk[4];
+  #pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(A[4 * j + q].x, A[4 * j + q].y);
+                    pk[q] = *reinterpret_cast<const uint32_t*>(&b);
+                  }
+                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+              }
+            } else if (W == 8) {
+  #pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1) {
+                  *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y);
+                  *reinterpret_cast<float4*>(q0 + j * qstep + 16) = make_float4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y);
+                }
+            } else {
+  #pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
             }
-          } else if (W == 8) {
-#pragma unroll
-            for (int j = 0; j < V / 8; ++j)
-              if ((fast >> j) & 1) {
-                *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y);
-                *reinterpret_cast<float4*>(q0 + j * qstep + 16) = make_float4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y);
-              }
-          } else {
-#pragma unroll
-            for (int j = 0; j < V / 4; ++j)
-              if ((fast >> j) & 1)
-                *reinterpret_cast<float4*>(q0 + j * qstep) = make_float4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
-          }
-          if (slow) {
-            // chunks cut by the segment's head or tail (or stored at another alignment than the mapping's):
-            // pick the chunk's pairs out of ACC, then predicated element stores
-#pragma unroll 1
-            for (uint32_t m = slow; m; m &= m - 1) {
-              const int j = __ffs(m) - 1;
-              float2 tp[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-              if (W == 8) {
-#pragma unroll
-                for (int jj = 0; jj < V / 8; ++jj)
-                  if (jj == j) { tp[0] = A[4 * jj]; tp[1] = A[4 * jj + 1]; tp[2] = A[4 * jj + 2]; tp[3] = A[4 * jj + 3]; }
-              } else {
-#pragma unroll
-                for (int jj = 0; jj < V / 4; ++jj)
-                  if (jj == j) { tp[0] = A[2 * jj]; tp[1] = A[2 * jj + 1]; }
-              }
-#pragma unroll
-              for (int el = 0; el < 8; ++el) {
-                if (el < W) {
-                  int col = c.cbase + (j << (c.lgG + c.lgW)) + el;
-                  if (col < 0 && c.ov > 0) col += V << c.lgG;  // wrap-around slots of the row's first thread
-                  const float val = (el & 1) ? tp[el >> 1].y : tp[el >> 1].x;
-                  if (col >= 0 && col < c.ncols) {
-                    if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
-                    else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
+            if (slow) {
+              // chunks cut by the segment's head or tail (or stored at another alignment than the mapping's):
+              // pick the chunk's pairs out of ACC, then predicated element stores
+  #pragma unroll 1
+              for (uint32_t m = slow; m; m &= m - 1) {
+                const int j = __ffs(m) - 1;
+                float2 tp[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                if (W == 8) {
+  #pragma unroll
+                  for (int jj = 0; jj < V / 8; ++jj)
+                    if (jj == j) { tp[0] = A[4 * jj]; tp[1] = A[4 * jj + 1]; tp[2] = A[4 * jj + 2]; tp[3] = A[4 * jj + 3]; }
+                } else {
+  #pragma unroll
+                  for (int jj = 0; jj < V / 4; ++jj)
+                    if (jj == j) { tp[0] = A[2 * jj]; tp[1] = A[2 * jj + 1]; }
+                }
+  #pragma unroll
+                for (int el = 0; el < 8; ++el) {
+                  if (el < W) {
+                    int col = c.cbase + (j << (c.lgG + c.lgW)) + el;
+                    if (col < 0 && c.ov > 0) col += V << c.lgG;  // wrap-around slots of the row's first thread
+                    const float val = (el & 1) ? tp[el >> 1].y : tp[el >> 1].x;
+                    if (col >= 0 && col < c.ncols) {
+                      if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
+                      else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
+                    }
                   }
                 }
               }
             }
+          } else if (op == DVM_OP_STS) {
+            const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
+            const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << (dt == DVM_DT_BF16 ? 1 : 2)));
+            const float v = s_S[ia][tid];
+            if (c.ncols > 0 && (tid & (G - 1)) == 0 && c.col0 == 0) {
+              if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
+              else *reinterpret_cast<float*>(p) = v;
+            }
+          } else if (op != DVM_OP_NOP) {
+            err = ST_BAD_CODE;
+            pc = pc_end;
           }
         } break;
-        case DVM_OP_STS: {
-          const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
-          const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
-          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << (dt == DVM_DT_BF16 ? 1 : 2)));
-          const float v = sget(S, ia);
-          if (c.ncols > 0 && (tid & (G - 1)) == 0 && c.col0 == 0) {
-            if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
-            else *reinterpret_cast<float*>(p) = v;
+        case 1: {  // BCS, SOP
+          const int ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
+          if (op == DVM_OP_BCS) {
+            pc += 1;
+            const float v = s_S[ia][tid];
+            DVM_EACH_PAIR A[i] = make_float2(v, v);
+          } else if (op == DVM_OP_SOP) {
+            const uint32_t w1 = CW(pc + 1);
+            const int sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
+            const float x = s_S[s1][tid];
+            float rv;
+            if (ib == DVM_SK_FMAU) {
+              // unary(x * m + a): multiply and add round separately, exactly like the unfused instructions
+              rv = __fadd_rn(__fmul_rn(x, __uint_as_float(CW(pc + 2))), __uint_as_float(CW(pc + 3)));
+              if (sub != 0xff) rv = scalar_unary(sub, rv);
+            } else if (ib == DVM_SK_UN) rv = scalar_unary(sub, x);
+            else rv = scalar_arith(sub, x, ib == DVM_SK_BIN ? s_S[s2][tid] : __uint_as_float(CW(pc + 2)));
+            s_S[ia][tid] = rv;
+            pc += DVM_INSN_LEN(w0);
+          } else {
+            err = ST_BAD_CODE;
+            pc = pc_end;
           }
-        } break;
-        case DVM_OP_BCS: {
-          const float v = sget(S, ia);
-          DVM_EACH_PAIR A[i] = make_float2(v, v);
-        } break;
-        case DVM_OP_SOP: {
-          const uint32_t w1 = CW(body0 + pc - (ib == DVM_SK_BINI ? 2 : (ib == DVM_SK_FMAU ? 3 : 1)));
-          const int sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
-          const float x = sget(S, s1);
-          float rv;
-          if (ib == DVM_SK_FMAU) {
-            // unary(x * m + a): multiply and add round separately, exactly like the unfused instructions
-            rv = __fadd_rn(__fmul_rn(x, __uint_as_float(CW(body0 + pc - 2))), __uint_as_float(CW(body0 + pc - 1)));
-            if (sub != 0xff) rv = scalar_unary(sub, rv);
-          } else if (ib == DVM_SK_UN) rv = scalar_unary(sub, x);
-          else rv = scalar_arith(sub, x, ib == DVM_SK_BIN ? sget(S, s2) : __uint_as_float(CW(body0 + pc - 1)));
-          sset(S, ia, rv);
         } break;
         default:
           err = ST_BAD_CODE;
-          pc = body_words;  // stop walking code that cannot be decoded
+          pc = pc_end;  // stop walking code that cannot be decoded
           break;
       }
     }
