@@ -189,18 +189,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     return off;
   };
 
-  // Tile id -> geometry of this thread's part of the tile (closed forms, no loops).  `c` holds the previous
-  // tile's geometry on entry: the slot masks are kept when the row segment has the same length and shift.
-  auto make_ctx = [&](TileCtx& c, uint32_t prog, uint32_t local_tile) {
-    const bool same_prog = c.prog == prog;
+  // Tile id -> this thread's row of the tile (closed forms, no loops): all the load section needs.
+  auto ctx_rows = [&](TileCtx& c, uint32_t prog, uint32_t local_tile) {
     c.prog = prog;
     const uint32_t geom = CW(prog + DVM_H_GEOM);
     c.lgG = geom & 0xff;
     const int W = (geom >> 8) & 0xff;
     c.lgW = W == 8 ? 3 : 2;
     c.flags = geom >> 24;
-    const int G = 1 << c.lgG;
-    const int t = tid & (G - 1);
     const uint32_t CB = CW(prog + DVM_H_COL_BLOCKS);
     uint32_t rb = local_tile, cb = 0;
     if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
@@ -212,6 +208,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t cend = (row == rows - 1) ? CW(prog + DVM_H_LAST_ROW_COLS) : CW(prog + DVM_H_COLS);
     int nc = 0;
     if (row < rows && cend > c.col0) nc = (int)min(cend - c.col0, ctile);
+    c.ncols = nc;
     c.row = row < rows ? row : 0;
     c.i0 = c.row;
     c.i1 = c.i2 = 0;
@@ -222,6 +219,15 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       c.i2 = q / n1;
       c.i1 = q - c.i2 * n1;
     }
+  };
+  // The rest of the geometry: the row's shift and this thread's slot masks.  `c` still holds the previous
+  // tile's masks on entry (prev_*: its program, segment length and shift): they are kept when nothing changed.
+  auto ctx_masks = [&](TileCtx& c, uint32_t prev_prog, int prev_ncols, int prev_shift) {
+    const uint32_t prog = c.prog;
+    const int W = 1 << c.lgW;
+    const int G = 1 << c.lgG;
+    const int t = tid & (G - 1);
+    const int nc = c.ncols;
     int shift = 0;
     if (!(c.flags & DVM_F_ALIGNED)) {
       // misalignment (in elements) of the row segment start of the primary operand
@@ -234,9 +240,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       shift = (int)((base_el + off) & (uint32_t)(W - 1));
     }
     c.cbase = (t << c.lgW) - shift;
-    if (same_prog && nc == c.ncols && shift == c.shift) return;  // same masks as the previous tile
-    c.ncols = nc;
     c.shift = shift;
+    if (prev_prog == prog && nc == prev_ncols && shift == prev_shift) return;  // same masks as the previous tile
     // In mapping coordinates the segment is [shift, shift + ncols); this thread owns chunks t, t+G, ...
     // The first nf of them are whole, the next one may be cut by the segment's end: a prefix of P slots.
     const int nch = V >> c.lgW;
@@ -478,8 +483,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   uint32_t slot_prog[2] = {0xffffffffu, 0xffffffffu};  // program whose row-vector inputs each slot holds
   if (tile < prm.total_tiles) {
     if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
-    make_ctx(c, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
-    issue_loads(c, buf, true);
+    TileCtx cl;
+    ctx_rows(cl, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
+    issue_loads(cl, buf, true);
     slot_prog[0] = prog_idx;
     cp_async_commit();
   }
@@ -492,14 +498,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     if (s_abort) break;  // a wait ran out in some thread during the previous tile
     const uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
     ++iter;
-    TileCtx cn = c;
     const bool have_next = next < prm.total_tiles;
     uint32_t next_prog_idx = prog_idx;
     if (have_next) {
       if (!SINGLE) while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
-      make_ctx(cn, SINGLE ? kSingleProg : CW(next_prog_idx), SINGLE ? next : next - CW(n_prog + next_prog_idx));
+      TileCtx cl;  // rows of the next tile: only the threads that issue its copies keep this alive
+      ctx_rows(cl, SINGLE ? kSingleProg : CW(next_prog_idx), SINGLE ? next : next - CW(n_prog + next_prog_idx));
       const bool first = buf ? slot_prog[0] != next_prog_idx : slot_prog[1] != next_prog_idx;
-      issue_loads(cn, buf ^ 1, first);
+      issue_loads(cl, buf ^ 1, first);
       if (buf) slot_prog[0] = next_prog_idx; else slot_prog[1] = next_prog_idx;
       cp_async_commit();
       cp_async_wait<1>();  // this tile's per-row scalars have landed once only the next tile's group is pending
@@ -511,6 +517,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       // barrier; until then this thread keeps in step (the code it walks has the same barriers for all)
       err = ST_TIMEOUT;
       s_abort = 1;
+    }
+    {
+      const uint32_t prev_prog = c.prog;
+      const int prev_ncols = c.ncols, prev_shift = c.shift;
+      ctx_rows(c, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
+      ctx_masks(c, prev_prog, prev_ncols, prev_shift);
     }
 
     const uint32_t prog = SINGLE ? kSingleProg : c.prog;
@@ -823,7 +835,6 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     }
 
     // ---- advance to the next tile ----
-    c = cn;
     prog_idx = next_prog_idx;
     tile = next;
     buf ^= 1;
