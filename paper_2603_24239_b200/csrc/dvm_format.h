@@ -63,7 +63,8 @@ enum {
                            // thread 0 alone issues every copy of a tile
 };
 
-// ---- local register table: one word per local register: unit offset inside a tile slot | mode << 16 ----
+// ---- local register table: one word per local register:
+//      unit offset inside a tile slot | mode << 16 | (tensor address & 15) << 20 (set at launch) | operand << 24 ----
 enum {
   DVM_LM_PRIVATE = 0,  // temporary: thread-private fp32 vectors, vector q of thread tid at (q * 256 + tid) * 16
   DVM_LM_BLOCK = 1,    // input whose tile is one contiguous byte range of global memory: one bulk copy per tile

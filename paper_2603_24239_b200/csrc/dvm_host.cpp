@@ -962,7 +962,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
   if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
   for (int k = 0; k < e.n_in_regs; ++k)
-    if (((best.lreg_table[k] >> 16) & 0xff) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
@@ -1070,7 +1070,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   // type the instruction expects
   auto lreg_ok = [&](uint32_t k, uint32_t dt) {
     if (k >= nreg) return false;
-    const uint32_t lw = lt[k], unit = lw & 0xffffu, mode = (lw >> 16) & 0xff, od = lw >> 24;
+    const uint32_t lw = lt[k], unit = lw & 0xffffu, mode = (lw >> 16) & 0xff, od = lw >> 24;  // bits 20..23 (address phase) are set at launch only
     uint64_t need;
     if (k >= n_inr) {
       if (mode != DVM_LM_PRIVATE || dt != DVM_DT_F32) return false;

@@ -113,6 +113,15 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
     uintptr_t es = ((info >> 8) & 0xff) == DVM_DT_BF16 ? 2 : 4;
     if (a % es) return DVM_ERR_INVALID_ARG;
   }
+  // every input register learns its tensor's address modulo 16 (the images keep that phase)
+  {
+    const uint32_t n_inr = code[DVM_H_LOCAL] & 0xff;
+    uint32_t* lt = dst + DVM_HDR_WORDS + 2 * nt + n_opd * DVM_OPD_WORDS;
+    for (uint32_t k = 0; k < n_inr; ++k) {
+      const uint32_t info = ot[(lt[k] >> 24) * DVM_OPD_WORDS];
+      lt[k] = (lt[k] & ~(0xfu << 20)) | (((uint32_t)(uintptr_t)tensors[info & 0xff] & 15u) << 20);
+    }
+  }
   // A program encoded for aligned rows relies on a 16-byte aligned primary tensor; on any other base address
   // the interpreter derives the row shift from the actual address instead (the rows' last columns then
   // wrap around into the head slots when a row fills its whole capacity).

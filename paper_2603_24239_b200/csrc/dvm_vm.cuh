@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       const uint32_t d = opd0 + DVM_INSN_B(w0) * DVM_OPD_WORDS;
       if (DVM_INSN_OP(w0) == DVM_OP_LDG) {
         const uint32_t lw = CW(lreg0 + (DVM_INSN_A(w0) & 0x7f));
-        const uint32_t mode = (lw >> 16) & 0xff;
+        const uint32_t mode = (lw >> 16) & 0xf;
         uint32_t dst = sb + (lw & 0xffffu) * DVM_LOCAL_UNIT;
         const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
         unsigned long long a = 0, n_el = 0;
@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   auto reg_view = [&](const TileCtx& c, uint32_t prog, uint32_t opd0, uint32_t lreg0, int k, int dt, int buf) -> RegView {
     RegView r;
     const uint32_t lw = CW(lreg0 + k);
-    const uint32_t mode = (lw >> 16) & 0xff;
+    const uint32_t mode = (lw >> 16) & 0xf;
     uint32_t a = slot_base(buf) + (lw & 0xffffu) * DVM_LOCAL_UNIT;
     if (mode == DVM_LM_PRIVATE) {
       r.a = a + (uint32_t)tid * 16;
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     }
     const uint32_t d = opd0 + (lw >> 24) * DVM_OPD_WORDS;
     const uint32_t lg_es = dt == DVM_DT_BF16 ? 1 : 2;
-    const uint32_t base_lo = CW(prog + DVM_HDR_WORDS + 2 * (CW(d + DVM_OPD_INFO) & 0xff));
+    const uint32_t base_lo = (lw >> 20) & 0xfu;  // the tensor address modulo 16 (patched in at launch)
     const uint32_t rr = (uint32_t)(tid >> c.lgG);
     uint32_t off;  // element offset (low bits suffice) of the image's first element inside the tensor
     if (mode == DVM_LM_BLOCK) {
@@ -502,10 +502,15 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     uint32_t next_prog_idx = prog_idx;
     if (have_next) {
       if (!SINGLE) while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
-      TileCtx cl;  // rows of the next tile: only the threads that issue its copies keep this alive
-      ctx_rows(cl, SINGLE ? kSingleProg : CW(next_prog_idx), SINGLE ? next : next - CW(n_prog + next_prog_idx));
+      const uint32_t nprog = SINGLE ? kSingleProg : CW(next_prog_idx);
       const bool first = buf ? slot_prog[0] != next_prog_idx : slot_prog[1] != next_prog_idx;
-      issue_loads(cl, buf ^ 1, first);
+      if (((CW(nprog + DVM_H_GEOM) >> 24) & DVM_F_LOADS_BY_ROW) || warp == 0) {
+        TileCtx cl;  // rows of the next tile, for the threads that may issue its copies
+        ctx_rows(cl, nprog, SINGLE ? next : next - CW(n_prog + next_prog_idx));
+        issue_loads(cl, buf ^ 1, first);
+      } else {
+        vm_mbar_arrive(bar0 + 8 * (buf ^ 1));  // thread 0 issues every copy of that program's tiles
+      }
       if (buf) slot_prog[0] = next_prog_idx; else slot_prog[1] = next_prog_idx;
       cp_async_commit();
       cp_async_wait<1>();  // this tile's per-row scalars have landed once only the next tile's group is pending
