@@ -120,11 +120,21 @@ int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
                const float* scalars, int n_scalars,
                void* code, size_t code_capacity, size_t* code_size,
                dvm_shape* out_shapes, int n_out);
+/* dvm_encode for n independent instances in one call -- the stacked-fusion case (Sec. 5.1), where every
+ * program of a launch is re-encoded per launch.  All arrays are host memory of length n, except
+ * in_shapes / scalars, which concatenate the instances' arguments (instance i consumes n_in[i] shapes and
+ * n_scalars[i] scalars).  codes[i] is a caller-owned 8-byte aligned buffer of caps[i] bytes; sizes[i]
+ * receives the encoded size.  Output shapes are not returned (encode the instance alone to get them).
+ * Stops at the first instance that fails and returns its status, *failed (may be NULL) = its index. */
+int dvm_encode_batch(int n, const dvm_program* const* programs, const dvm_shape* in_shapes, const int* n_in,
+                     const float* scalars, const int* n_scalars, void* const* codes, const size_t* caps,
+                     size_t* sizes, int* failed);
 /* Upper bound of the encoded size, in bytes, for any shape. */
 size_t dvm_code_max_size(const dvm_program* p);
 
 /* Number of parallel units N the tiling cost model balances for (Sec. 4.2: cost
- * = ceil(#tiles / N) * (tile + overhead)).  Default 148 SMs x 3 resident CTAs.
+ * = ceil(#tiles / N) * (tile + overhead)).  Default 444 (148 SMs x 3); the encoder scales it to the
+ * CTAs that are actually resident per SM for the instance (at most 2).
  * n <= 0 restores the default.  Process-wide; not thread-safe against encode. */
 void dvm_set_num_cores(int n);
 int dvm_get_num_cores(void);

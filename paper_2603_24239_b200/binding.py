@@ -7,6 +7,8 @@ loudly -- there is no other implementation to fall back to.
 from __future__ import annotations
 
 import ctypes as C
+
+import numpy as np
 import os
 from typing import Iterable, List, Optional, Sequence
 
@@ -61,6 +63,8 @@ _sig = {
     "dvm_program_num_outputs": ([_vp], _i),
     "dvm_encode": ([_vp, C.POINTER(Shape), _i, C.POINTER(C.c_float), _i, _vp, _sz, C.POINTER(_sz),
                     C.POINTER(Shape), _i], _i),
+    "dvm_encode_batch": ([_i, C.POINTER(_vp), C.POINTER(Shape), _pi, C.POINTER(C.c_float), _pi, C.POINTER(_vp),
+                          C.POINTER(_sz), C.POINTER(_sz), _pi], _i),
     "dvm_code_max_size": ([_vp], _sz),
     "dvm_set_num_cores": ([_i], None),
     "dvm_get_num_cores": ([], _i),
@@ -221,6 +225,53 @@ class Encoder:
     def output_shapes(self) -> List[tuple]:
         return [tuple(self.out_shapes[o].dims[k] for k in range(self.out_shapes[o].rank))
                 for o in range(self.n_out)]
+
+
+class BatchEncoder:
+    """Reusable argument block for dvm_encode_batch: the instances of one stacked launch, encoded in one call.
+
+    `programs` fixes the program of every instance; encode() takes this launch's shapes and scalars.
+    The code buffers stay valid until the next encode(); launch_args() hands them to dvm_launch_stacked."""
+
+    def __init__(self, programs: Sequence[Program]):
+        n = self.n = len(programs)
+        self.programs = list(programs)
+        self.handles = (_vp * n)(*[p._h for p in programs])
+        self.n_in = (_i * n)(*[p.n_inputs for p in programs])
+        self.total_in = sum(p.n_inputs for p in programs)
+        self.shapes = (Shape * self.total_in)()
+        # the same memory as a numpy record array: one vectorised copy marshals every shape of the launch
+        self._np_shapes = np.frombuffer(self.shapes, dtype=np.dtype({"names": ["rank", "dims"],
+                                                                      "formats": ["<i4", ("<i8", DVM_MAX_RANK)],
+                                                                      "offsets": [0, 8], "itemsize": C.sizeof(Shape)}))
+        self.n_scalars = (_i * n)()
+        self.scalars = (C.c_float * (16 * n))()
+        caps = [p._max_code for p in programs]
+        self.bufs = [(C.c_uint64 * ((c + 7) // 8))() for c in caps]
+        self.codes = (_vp * n)(*[C.addressof(b) for b in self.bufs])
+        self.caps = (_sz * n)(*caps)
+        self.sizes = (_sz * n)()
+        self.failed = _i(0)
+
+    def encode(self, shapes: Sequence[Sequence[Sequence[int]]], scalars: Sequence[Sequence[float]]):
+        """shapes[i]: the input shapes of instance i; scalars[i]: its runtime scalar arguments."""
+        flat = [s for inst in shapes for s in inst]
+        ranks = np.fromiter((len(s) for s in flat), dtype=np.int32, count=self.total_in)
+        dims = np.zeros((self.total_in, DVM_MAX_RANK), dtype=np.int64)
+        for k, s in enumerate(flat):
+            dims[k, :len(s)] = s
+        self._np_shapes["rank"] = ranks
+        self._np_shapes["dims"] = dims
+        k = 0
+        for i, sc in enumerate(scalars):
+            self.n_scalars[i] = len(sc)
+            for v in sc:
+                self.scalars[k] = v
+                k += 1
+        st = lib.dvm_encode_batch(self.n, self.handles, self.shapes, self.n_in, self.scalars, self.n_scalars,
+                                  self.codes, self.caps, self.sizes, C.byref(self.failed))
+        if st != 0:
+            raise DvmError(st, f"dvm_encode_batch (instance {self.failed.value})")
 
 
 def encode(program: Program, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = ()) -> Code:

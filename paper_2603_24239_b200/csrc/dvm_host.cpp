@@ -1019,6 +1019,29 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   return DVM_OK;
 }
 
+extern "C" int dvm_encode_batch(int n, const dvm_program* const* programs, const dvm_shape* in_shapes, const int* n_in,
+                                const float* scalars, const int* n_scalars, void* const* codes, const size_t* caps,
+                                size_t* sizes, int* failed) {
+  if (n < 0 || (n > 0 && (!programs || !in_shapes || !n_in || !n_scalars || !codes || !caps || !sizes)))
+    return DVM_ERR_INVALID_ARG;
+  size_t si = 0, fi = 0;
+  for (int i = 0; i < n; ++i) {
+    if (n_in[i] < 0 || n_scalars[i] < 0) {
+      if (failed) *failed = i;
+      return DVM_ERR_INVALID_ARG;
+    }
+    const int st = dvm_encode(programs[i], in_shapes + si, n_in[i], n_scalars[i] ? scalars + fi : nullptr, n_scalars[i],
+                              codes[i], caps[i], &sizes[i], nullptr, 0);
+    if (st != DVM_OK) {
+      if (failed) *failed = i;
+      return st;
+    }
+    si += (size_t)n_in[i];
+    fi += (size_t)n_scalars[i];
+  }
+  return DVM_OK;
+}
+
 // ---------------------------------------------------------------------------
 // Verification and the readable dump
 // ---------------------------------------------------------------------------

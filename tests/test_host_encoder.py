@@ -178,3 +178,28 @@ def test_encode_latency_budget():
         ts.append(time.perf_counter_ns() - t0)
     ts.sort()
     assert ts[len(ts) // 2] < 50_000
+
+
+def test_encode_batch_matches_single_encodes():
+    """dvm_encode_batch produces, instance by instance, the bytes dvm_encode produces."""
+    from paper_2603_24239_b200 import binding
+    dvm.set_elems_per_thread(16)
+    try:
+        items = [("gelu_affine", 3, 65), ("layernorm", 17, 100), ("sigmoid_mul", 1, 64), ("layernorm", 512, 4096)]
+        progs = [dvm.program_from_nodes(wl.stack_program(k).nodes) for k, _, _ in items]
+        shapes = [{"gelu_affine": [(r, c), (1, c), (1, c)], "layernorm": [(r, c)], "sigmoid_mul": [(r, c), (r, c)]}[k]
+                  for k, r, c in items]
+        scalars = [[1.0 / c] if k == "layernorm" else [] for k, r, c in items]
+        be = binding.BatchEncoder(progs)
+        be.encode(shapes, scalars)
+        for i, p in enumerate(progs):
+            single = dvm.encode(p, shapes[i], scalars[i])
+            assert bytes(be.bufs[i])[: be.sizes[i]] == single.bytes()
+        # a failing instance is reported with its index
+        bad = [list(s) for s in shapes]
+        bad[2] = [(1, 64), (2, 63)]
+        with pytest.raises(dvm.DvmError) as ei:
+            be.encode(bad, scalars)
+        assert "instance 2" in str(ei.value)
+    finally:
+        dvm.set_elems_per_thread(0)
