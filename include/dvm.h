@@ -222,6 +222,11 @@ int dvm_disassemble(const void* code, size_t code_size, char* buf, size_t cap);
 /* Header fields of an encoded program (each output may be NULL). */
 int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t* n_tiles,
                   int* code_body_bytes, int* threads_per_row, int* vector_width, int* n_tile_regs);
+/* Self-test of the bounded device-side waits (no counterpart in the paper): launches one CTA that waits on
+ * an mbarrier nobody completes, with the very wait routine of the interpreter (which = 0) or of the matmul
+ * kernel (which = 1).  The wait gives up after its limit (about 2 s), the kernel sets the status word and
+ * returns: dvm_last_device_status then reports DVM_ERR_DEVICE_TIMEOUT and the context stays usable. */
+int dvm_selftest_bounded_wait(int which, void* cuda_stream);
 /* Synchronises `cuda_stream`, then reads and clears the device status word of
  * the current device: *status is DVM_OK or a DVM_ERR_DEVICE_* code. */
 int dvm_last_device_status(void* cuda_stream, int* status);

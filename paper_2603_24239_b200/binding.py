@@ -79,6 +79,7 @@ _sig = {
     "dvm_verify": ([_vp, _sz], _i),
     "dvm_disassemble": ([_vp, _sz, C.c_char_p, _sz], _i),
     "dvm_code_info": ([_vp, _sz, _pi, _p64, _pi, _pi, _pi, _pi], _i),
+    "dvm_selftest_bounded_wait": ([_i, _vp], _i),
     "dvm_last_device_status": ([_vp, _pi], _i),
     "dvm_last_cuda_error": ([], _i),
     "dvm_launch_count": ([], C.c_int64),
@@ -349,6 +350,11 @@ def last_device_status(stream=None) -> int:
     st = C.c_int(0)
     _check(lib.dvm_last_device_status(_stream(stream), C.byref(st)), "dvm_last_device_status")
     return st.value
+
+
+def selftest_bounded_wait(which: int, stream=None):
+    """Launches the kernel whose wait must run out (about 2 s); read the outcome with last_device_status()."""
+    _check(lib.dvm_selftest_bounded_wait(which, _stream(stream)), "dvm_selftest_bounded_wait")
 
 
 def launch_count() -> int:

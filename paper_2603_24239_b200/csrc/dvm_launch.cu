@@ -270,6 +270,37 @@ extern "C" int dvm_run_host(const void* code, size_t code_size, void* const* hos
   return DVM_OK;
 }
 
+// ---- self-test of the bounded waits ----
+namespace {
+__global__ void dvm_selftest_vm_wait_kernel(unsigned int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = static_cast<uint32_t>(__cvta_generic_to_shared(&bar));
+  if (threadIdx.x == 0) {
+    dvm::vm_mbar_init(b, 2);  // two arrivals expected, one ever made: the phase never completes
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    dvm::vm_mbar_arrive(b);
+  }
+  __syncthreads();
+  if (!dvm::vm_mbar_wait(b, 0) && threadIdx.x == 0) atomicMax(status, (unsigned int)dvm::ST_TIMEOUT);
+}
+}  // namespace
+
+int dvm_selftest_mm_wait(unsigned int* status, cudaStream_t stream);
+
+extern "C" int dvm_selftest_bounded_wait(int which, void* cuda_stream) {
+  DvmDeviceInfo dev;
+  int st = dvm_device_state(&dev);
+  if (st != DVM_OK) return st;
+  if (which == 0) {
+    dvm_selftest_vm_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(dev.scratch);
+    DVM_CUDA(cudaGetLastError());
+    dvm_count_launch();
+    return DVM_OK;
+  }
+  if (which == 1) return dvm_selftest_mm_wait(dev.scratch, (cudaStream_t)cuda_stream);
+  return DVM_ERR_INVALID_ARG;
+}
+
 extern "C" int dvm_last_device_status(void* cuda_stream, int* status) {
   if (!status) return DVM_ERR_INVALID_ARG;
   DVM_CUDA(cudaStreamSynchronize((cudaStream_t)cuda_stream));

@@ -1029,3 +1029,31 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   dvm_count_launch();
   return DVM_OK;
 }
+
+// ---- self-test of the matmul kernel's bounded wait (see dvm_selftest_bounded_wait) ----
+namespace dvm {
+namespace mm {
+__global__ void dvm_selftest_mm_wait_kernel(unsigned int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ uint32_t abort_word;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(b, 2);  // two arrivals expected, one ever made: the phase never completes
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_arrive(b);
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(b, 0, &abort_word);
+  __syncthreads();
+  if (!ok && abort_word && threadIdx.x == 0) atomicMax(status, (unsigned int)ST_TIMEOUT);
+}
+}  // namespace mm
+}  // namespace dvm
+
+int dvm_selftest_mm_wait(unsigned int* status, cudaStream_t stream) {
+  dvm::mm::dvm_selftest_mm_wait_kernel<<<1, 32, 0, stream>>>(status);
+  DVM_CUDA(cudaGetLastError());
+  dvm_count_launch();
+  return DVM_OK;
+}
