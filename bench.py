@@ -7,7 +7,7 @@ dvm_launch_stacked); nothing is cached between instances.  The default
 workload is the fused residual-add + RMSNorm sweep (200 instances, bf16
 [B*S, 4096], B in 1..32, S in 1..8192).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl dvm|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5] [--impl dvm|reference]
 
 Prints one JSON line (rank 0).  `value` is algorithmic GB/s of the whole job
 with inputs resident in HBM; `e2e` is the same metric through dvm_run_host
@@ -98,6 +98,70 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- workloads
+class C1Workload:
+    """Single fused elementwise program out = exp(a*b + c) - a, fp32 [7,1531], seed 0 (config 1): launch-latency bound."""
+    name = "c1"
+
+    def __init__(self, dvm, n_instances=1, device="cuda"):
+        self.dvm = dvm
+        self.prog = wl.program_c1()
+        self.p = dvm.program_from_nodes(self.prog.nodes)
+        self.enc = dvm.binding.Encoder(self.p)
+        self.ins = wl.inputs_c1(device)
+        self.out = torch.empty((7, 1531), dtype=torch.float32, device=device)
+        self.n = max(1, n_instances)
+        self.bytes_per_instance = [16 * 7 * 1531] * self.n
+        self.total_bytes = sum(self.bytes_per_instance)
+        self.description = ("c1: out = exp(a*b + c) - a, fp32 [7,1531] U(-1,1) seed 0, encoded and launched once per step "
+                            "(171 KB: launch-latency bound; the figure of merit is microseconds per launch)")
+        self.l2_policy = "171 KB working set: L2-resident by nature; no roofline claim"
+
+    def run_step(self, stream, events=None, enc_ns=None):
+        import ctypes as C
+        lib_launch = self.dvm.binding.lib.dvm_launch
+        for _ in range(self.n):
+            t0 = time.perf_counter_ns()
+            size = self.enc.encode(((7, 1531),) * 3)
+            t1 = time.perf_counter_ns()
+            if enc_ns is not None:
+                enc_ns.append(t1 - t0)
+            arr = (C.c_void_p * 4)(*[t.data_ptr() for t in self.ins], self.out.data_ptr())
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st = lib_launch(self.enc.buf, size, arr, 4, stream.cuda_stream)
+            if st != 0:
+                raise self.dvm.DvmError(st, "dvm_launch")
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+        return self.n
+
+    def setup_e2e(self):
+        self.h_in = [t.cpu().pin_memory() for t in self.ins]
+        self.h_out = torch.empty((7, 1531), dtype=torch.float32).pin_memory()
+        self.staging = torch.empty(4 * 7 * 1531 * 4 + 4 * 256, dtype=torch.uint8, device="cuda")
+
+    def run_step_e2e(self, stream):
+        self.enc.encode(((7, 1531),) * 3)
+        code = self.dvm.Code(self.enc.buf, self.enc.size.value, None)
+        h2d = d2h = 0
+        for _ in range(self.n):
+            self.dvm.run_host(code, self.h_in + [self.h_out], self.staging, stream)
+            h2d += 3 * 7 * 1531 * 4
+            d2h += 7 * 1531 * 4
+        return h2d, d2h
+
+    def oracle_sample(self, budget_s=12.0):
+        from oracle import dvm_oracle as orc
+        ins = [wl.to_f64(t) for t in self.ins]
+        t0 = time.perf_counter(); k = 0
+        while time.perf_counter() - t0 < budget_s:
+            orc.evaluate(self.prog.nodes, ins); k += 1
+        dt = time.perf_counter() - t0
+        return k * 16 * 7 * 1531 / dt / 1e9, dt, f"{k} evaluations of the [7,1531] instance, numpy float64"
+
+
 class C2Workload:
     """Fused residual-add + RMSNorm, bf16 [B*S, 4096], 200 dynamic instances (config 2)."""
     name = "c2"
@@ -491,8 +555,8 @@ class C5Workload:
         return flops / t_all / 1e12, t_all, f"{rows_done} rows of X in windows of {m} rows against both full weight matrices, numpy float64"
 
 
-WORKLOADS = {"c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
-for _W in (C2Workload, C3Workload, C4Workload):   # the memory-bound sweeps: work = algorithmic bytes
+WORKLOADS = {"c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
+for _W in (C1Workload, C2Workload, C3Workload, C4Workload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
 
@@ -525,6 +589,13 @@ def run_reference(args):
         nbytes = rows * 4096 * 8 + 8192
         sample = f"{rows} rows x 4096 (one c2 instance) per step, numpy float64"
         desc = C2Workload.__doc__
+        params = ()
+    elif args.workload == "c1":
+        prog = wl.program_c1()
+        ins = [wl.to_f64(t) for t in wl.inputs_c1()]
+        nbytes = 16 * 7 * 1531
+        sample = "the [7,1531] instance per step, numpy float64"
+        desc = C1Workload.__doc__
         params = ()
     elif args.workload == "c3":
         prog = wl.program_masked_softmax(128)
@@ -568,6 +639,25 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def encode_latency(W, reps):
+    """Host encode latency over `reps` repeats of each of (up to) 20 instances of the sweep: pure dvm_encode calls."""
+    if W.name == "c1":
+        shapes = [((7, 1531),) * 3]
+    elif W.name == "c2":
+        shapes = [((t, 4096), (t, 4096), (4096,)) for t in W.rows[:20]]
+    elif W.name == "c3":
+        shapes = [((b, 32, s_, s_), (1, 1, s_, s_)) for b, s_ in W.shapes[:20]]
+    else:
+        shapes = [((m, 4096), (4096, 11008), (4096, 11008)) for m in W.Ms[:20]]
+    ns = []
+    for shp in shapes:
+        for _ in range(reps):
+            t0 = time.perf_counter_ns(); W.enc.encode(shp); ns.append(time.perf_counter_ns() - t0)
+    us = sorted(x / 1e3 for x in ns)
+    return {"mean": sum(us) / len(us), "p50": us[len(us) // 2], "p99": us[int(0.99 * len(us))], "max": us[-1],
+            "n": len(us), "note": f"{reps} repeats of each of {len(shapes)} instances, perf_counter around the ctypes call"}
+
+
 # ----------------------------------------------------------------------------- multi-rank aggregation
 def reduce_max_over_ranks(x: float, dist, device) -> float:
     """The slowest rank's time: all-reduce MAX over the process group (identity without one)."""
@@ -593,6 +683,7 @@ def main():
     ap.add_argument("--instances", type=int, default=0, help="override the number of instances (debug)")
     ap.add_argument("--max-rows", type=int, default=0, help="cap rows per instance (small profiling case)")
     ap.add_argument("--elems-per-thread", type=int, default=0, help="fix the encoder's elements per thread (16/32/64; 0 = cost model)")
+    ap.add_argument("--encode-reps", type=int, default=1000, help="repeats per instance of the host-encode latency measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--detail", default="", help="write per-instance timings to this JSON file")
@@ -718,6 +809,17 @@ def main():
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    if rank == 0 and W.name == "c1":
+        # the figure of merit of the latency-bound config: host wall time of encode + launch + sync, and the
+        # device time between events around the launch
+        wall = []
+        for _ in range(300):
+            t0 = time.perf_counter_ns(); W.run_step(stream); stream.synchronize(); wall.append((time.perf_counter_ns() - t0) / 1e3)
+        wall.sort()
+        line["latency_us"] = {"encode_launch_sync_wall_p50": wall[len(wall) // 2], "wall_p99": wall[int(0.99 * len(wall))],
+                              "kernel_event_mean": 1e3 * kernel_total_ms / max(len(kern_ms), 1)}
+    if rank == 0 and hasattr(W, "enc") and args.encode_reps > 0:
+        line["encode_us_repeated"] = encode_latency(W, args.encode_reps)
     if args.detail and rank == 0:
         with open(args.detail, "w") as f:
             json.dump({"bytes": per_launch_bytes, "ms": kern_ms, "enc_us": [x / 1e3 for x in enc_ns]}, f)
