@@ -91,9 +91,9 @@ extern "C" int64_t dvm_launch_count(void) { return (int64_t)__atomic_load_n(&g_l
 
 namespace {
 
-// Copies one verified vector program into `dst`, patches its tensor table, and falls back to
-// the element-wise mapping (W = 1) when the program assumed 16-byte aligned rows but the primary
-// operand's base pointer is not.
+// Copies one verified vector program into `dst` and patches in what only the launch knows: the tensor
+// addresses, each input register's address phase (address modulo 16), and -- when the program assumed
+// 16-byte aligned rows but the primary operand's base pointer is not -- the switch to address-derived shifts.
 int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int n_tensors) {
   const uint32_t total = code[DVM_H_TOTAL_WORDS];
   memcpy(dst, code, (size_t)total * 4);
