@@ -173,7 +173,10 @@ int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_t
  * run as ONE kernel; their tiles are claimed from one work queue, spread over
  * SMs (spatial) and run back to back on each SM (temporal).
  * codes[i] / code_sizes[i] / tensors[i] / n_tensors[i] as for dvm_launch.  All programs must have
- * been encoded with the same elements-per-thread setting (DVM_ERR_INVALID_ARG otherwise). */
+ * been encoded with the same elements-per-thread setting (DVM_ERR_INVALID_ARG otherwise).
+ * Limits (DVM_ERR_TOO_LARGE beyond): 256 programs, and the programs travel together in the 32 KB
+ * kernel-parameter block: the sum of their code sizes plus 8 bytes per program must stay within 32000 bytes
+ * (about 130 programs of three tensors each). */
 int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
                        void* const* const* tensors, const int* n_tensors, void* cuda_stream);
 
