@@ -77,9 +77,7 @@ struct TileCtx {
   uint32_t hm;       //   except in the first chunk of a misaligned row: bit s of hm covers slots 0..7)
   uint32_t fullmask; // bit j: chunk j lies entirely inside the row segment
   uint32_t partmask; // bit j: chunk j is cut by the segment's head or tail
-  uint32_t row;      // row of the dominant (collapsed) shape
-  uint32_t row0;     // first row of the tile
-  uint32_t i0, i1, i2;  // row coordinates over the collapsed outer dims
+  uint32_t row;      // row of the dominant (collapsed) shape (not clamped: rows past the end have ncols = 0)
   uint32_t col0;
   uint32_t flags;
 };
@@ -180,11 +178,16 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   // element offset of this thread's row (plus the column block start) inside operand d
   // (strides are below 2^32 elements -- the host rejects larger ones: 32 x 32 -> 64-bit products)
   auto row_offset = [&](uint32_t d, const TileCtx& c) -> unsigned long long {
-    unsigned long long off = (unsigned long long)c.i0 * CW(d + DVM_OPD_STRIDE0);
-    if (c.flags & DVM_F_OUTER_DIMS) {
-      off += (unsigned long long)c.i1 * CW(d + DVM_OPD_STRIDE1);
-      off += (unsigned long long)c.i2 * CW(d + DVM_OPD_STRIDE2);
+    uint32_t i0 = c.row;
+    unsigned long long off = 0;
+    if (c.flags & DVM_F_OUTER_DIMS) {  // row -> coordinates over the collapsed outer dims
+      const uint32_t n0 = CW(c.prog + DVM_H_OUTER0), n1 = CW(c.prog + DVM_H_OUTER1);
+      const uint32_t q = i0 / n0;
+      i0 -= q * n0;
+      const uint32_t i2 = q / n1;
+      off = (unsigned long long)(q - i2 * n1) * CW(d + DVM_OPD_STRIDE1) + (unsigned long long)i2 * CW(d + DVM_OPD_STRIDE2);
     }
+    off += (unsigned long long)i0 * CW(d + DVM_OPD_STRIDE0);
     if ((CW(d + DVM_OPD_INFO) >> 16) & 0xff) off += c.col0;
     return off;
   };
@@ -201,24 +204,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     uint32_t rb = local_tile, cb = 0;
     if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
     const uint32_t rows = CW(prog + DVM_H_ROWS_LO);  // the host rejects more than 2^32 - 1 rows per program
-    c.row0 = rb * (uint32_t)(THREADS >> c.lgG);
-    const uint32_t row = c.row0 + (uint32_t)(tid >> c.lgG);
+    const uint32_t row = rb * (uint32_t)(THREADS >> c.lgG) + (uint32_t)(tid >> c.lgG);
     const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
     c.col0 = cb * ctile;
     const uint32_t cend = (row == rows - 1) ? CW(prog + DVM_H_LAST_ROW_COLS) : CW(prog + DVM_H_COLS);
     int nc = 0;
     if (row < rows && cend > c.col0) nc = (int)min(cend - c.col0, ctile);
     c.ncols = nc;
-    c.row = row < rows ? row : 0;
-    c.i0 = c.row;
-    c.i1 = c.i2 = 0;
-    if (c.flags & DVM_F_OUTER_DIMS) {
-      const uint32_t n0 = CW(prog + DVM_H_OUTER0), n1 = CW(prog + DVM_H_OUTER1);
-      const uint32_t q = c.i0 / n0;
-      c.i0 -= q * n0;
-      c.i2 = q / n1;
-      c.i1 = q - c.i2 * n1;
-    }
+    c.row = row;
   };
   // The rest of the geometry: the row's shift and this thread's slot masks.  `c` still holds the previous
   // tile's masks on entry (prev_*: its program, segment length and shift): they are kept when nothing changed.
@@ -302,9 +295,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             mine = true;
             const uint32_t rows = CW(prog + DVM_H_ROWS_LO), C = CW(prog + DVM_H_COLS);
             const uint32_t R = (uint32_t)(THREADS >> c.lgG);
-            const uint32_t rv = min(R, rows - c.row0);
-            const uint32_t last = (c.row0 + rv == rows) ? CW(prog + DVM_H_LAST_ROW_COLS) : C;
-            a = (unsigned long long)c.row0 * C;
+            const uint32_t rv = min(R, rows - c.row);
+            const uint32_t last = (c.row + rv == rows) ? CW(prog + DVM_H_LAST_ROW_COLS) : C;
+            a = (unsigned long long)c.row * C;
             n_el = (unsigned long long)(rv - 1) * C + last;
           }
         } else if (mode == DVM_LM_ROWS) {
@@ -375,7 +368,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     uint32_t off;  // element offset (low bits suffice) of the image's first element inside the tensor
     if (mode == DVM_LM_BLOCK) {
       const uint32_t C = CW(prog + DVM_H_COLS);
-      off = c.row0 * C;
+      off = (c.row - rr) * C;  // the tile's first row
       a += (rr * C) << lg_es;
     } else if (mode == DVM_LM_ROWS) {
       off = (uint32_t)row_offset(d, c);
