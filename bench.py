@@ -7,7 +7,7 @@ dvm_launch_stacked); nothing is cached between instances.  The default
 workload is the fused residual-add + RMSNorm sweep (200 instances, bf16
 [B*S, 4096], B in 1..32, S in 1..8192).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5] [--impl dvm|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5|addmm] [--impl dvm|reference]
 
 Prints one JSON line (rank 0).  `value` is algorithmic GB/s of the whole job
 with inputs resident in HBM; `e2e` is the same metric through dvm_run_host
@@ -555,7 +555,79 @@ class C5Workload:
         return flops / t_all / 1e12, t_all, f"{rows_done} rows of X in windows of {m} rows against both full weight matrices, numpy float64"
 
 
-WORKLOADS = {"c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
+class AddmmWorkload:
+    """addmm over the paper's LLM (n,k) pairs (Table 2): out = A[m,k] @ B[k,n] + C[m,n], bf16, fp32 accumulate."""
+    name = "addmm"
+    metric, unit, scale, bound, kernel, peak_key = "tflops_dynamic_shape_sweep", "TFLOP/s", 1e12, "tensor", "dvm_mm_kernel", "bf16_tflops_sustained"
+
+    def __init__(self, dvm, n_instances=36, device="cuda", max_rows=0):
+        self.dvm = dvm
+        self.prog = wl.program_addmm()
+        self.p = dvm.program_from_nodes(self.prog.nodes)
+        self.enc = dvm.binding.Encoder(self.p)
+        self.shapes = wl.shapes_addmm(n_instances)
+        if max_rows:
+            self.shapes = [(min(m, max_rows), n, k) for m, n, k in self.shapes]
+        seed = wl.data_seed("addmm", 0)
+        self.B = {nk: wl.randn((nk[1], nk[0]), torch.bfloat16, seed + 10 + i, device, std=0.02)
+                  for i, nk in enumerate(sorted({(n, k) for _, n, k in self.shapes}))}   # weights: once per (n, k)
+        mmax = max(m for m, _, _ in self.shapes)
+        kmax = max(k for _, _, k in self.shapes); nmax = max(n for _, n, _ in self.shapes)
+        self.a_pool = wl.randn((mmax * kmax,), torch.bfloat16, seed, device)
+        self.c_pool = wl.randn((mmax * nmax,), torch.bfloat16, seed + 1, device)
+        self.o_pool = torch.empty((mmax * nmax,), dtype=torch.bfloat16, device=device)
+        self.work_per_instance = [2 * m * n * k for m, n, k in self.shapes]
+        self.bytes_per_instance = [2 * (m * k + k * n + 2 * m * n) for m, n, k in self.shapes]
+        self.total_work = sum(self.work_per_instance)
+        self.total_bytes = sum(self.bytes_per_instance)
+        self.description = (f"addmm: A[m,k] @ B[k,n] + C[m,n], bf16, fp32 accumulate, bf16 out; {n_instances} dynamic instances, "
+                            "m 1..8192, (n,k) cycling through the nine LLM pairs of the paper's Table 2, each re-encoded per launch")
+        self.l2_policy = "every instance streams its weight matrix (33..470 MB) and its own A / C / out windows"
+
+    def _args(self, i):
+        import ctypes as C
+        m, n, k = self.shapes[i]
+        return (C.c_void_p * 4)(self.a_pool.data_ptr(), self.B[(n, k)].data_ptr(), self.c_pool.data_ptr(), self.o_pool.data_ptr())
+
+    def run_step(self, stream, events=None, enc_ns=None):
+        lib_launch = self.dvm.binding.lib.dvm_launch
+        for i, (m, n, k) in enumerate(self.shapes):
+            t0 = time.perf_counter_ns()
+            size = self.enc.encode(((m, k), (k, n), (m, n)))
+            t1 = time.perf_counter_ns()
+            if enc_ns is not None:
+                enc_ns.append(t1 - t0)
+            arr = self._args(i)
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st = lib_launch(self.enc.buf, size, arr, 4, stream.cuda_stream)
+            if st != 0:
+                raise self.dvm.DvmError(st, "dvm_launch")
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+        return len(self.shapes)
+
+    def setup_e2e(self):
+        self.staging = None   # the weights alone are 1.6 GB per sweep over PCIe: no end-to-end leg for this workload
+
+    def run_step_e2e(self, stream):
+        return None
+
+    def oracle_sample(self, budget_s=12.0):
+        from oracle import dvm_oracle as orc
+        n, k = 4096, 4096
+        b = wl.to_f64(self.B[(n, k)]) if (n, k) in self.B else wl.to_f64(wl.randn((k, n), torch.bfloat16, 1, std=0.02))
+        t_all, flops, m = 0.0, 0, 256
+        while t_all < budget_s:
+            a = wl.to_f64(self.a_pool[:m * k]).reshape(m, k); c = wl.to_f64(self.c_pool[:m * n]).reshape(m, n)
+            t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, [a, b, c]); t_all += time.perf_counter() - t0
+            flops += 2 * m * n * k
+        return flops / t_all / 1e12, t_all, f"[256,4096] @ [4096,4096] + [256,4096] repeated for {t_all:.0f} s, numpy float64"
+
+
+WORKLOADS = {"addmm": AddmmWorkload, "c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
 for _W in (C1Workload, C2Workload, C3Workload, C4Workload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
@@ -564,7 +636,7 @@ for _W in (C1Workload, C2Workload, C3Workload, C4Workload):   # the memory-bound
 def oracle_threads(workload: str) -> int:
     """Threads the numpy oracle actually uses: elementwise programs run on one core; the matmul of c5 goes
     through numpy's BLAS, which uses its own pool."""
-    if workload != "c5":
+    if workload not in ("c5", "addmm"):
         return 1
     try:
         from threadpoolctl import threadpool_info
@@ -589,6 +661,15 @@ def run_reference(args):
         nbytes = rows * 4096 * 8 + 8192
         sample = f"{rows} rows x 4096 (one c2 instance) per step, numpy float64"
         desc = C2Workload.__doc__
+        params = ()
+    elif args.workload == "addmm":
+        prog = wl.program_addmm()
+        M = 128
+        ins = [wl.to_f64(wl.randn((M, 4096), torch.bfloat16, 1)), wl.to_f64(wl.randn((4096, 4096), torch.bfloat16, 2, std=0.02)),
+               wl.to_f64(wl.randn((M, 4096), torch.bfloat16, 3))]
+        nbytes = 2 * M * 4096 * 4096   # flops
+        sample = f"[{M},4096] @ [4096,4096] + [{M},4096] per step, numpy float64"
+        desc = AddmmWorkload.__doc__
         params = ()
     elif args.workload == "c1":
         prog = wl.program_c1()
@@ -625,7 +706,7 @@ def run_reference(args):
     for _ in range(args.steps):
         orc.evaluate(prog.nodes, ins, params)
     dt = time.perf_counter() - t0
-    tensor = args.workload == "c5"
+    tensor = args.workload in ("c5", "addmm")
     val = nbytes * args.steps / dt / (1e12 if tensor else 1e9)
     unit = "TFLOP/s" if tensor else "GB/s"
     line = {"impl": "reference", "metric": "tflops_dynamic_shape_sweep" if tensor else "hbm_gbs_dynamic_shape_sweep",
@@ -641,7 +722,9 @@ def run_reference(args):
 
 def encode_latency(W, reps):
     """Host encode latency over `reps` repeats of each of (up to) 20 instances of the sweep: pure dvm_encode calls."""
-    if W.name == "c1":
+    if W.name == "addmm":
+        shapes = [((m, k), (k, n), (m, n)) for m, n, k in W.shapes[:20]]
+    elif W.name == "c1":
         shapes = [((7, 1531),) * 3]
     elif W.name == "c2":
         shapes = [((t, 4096), (t, 4096), (4096,)) for t in W.rows[:20]]
@@ -712,7 +795,7 @@ def main():
         dvm.set_elems_per_thread(args.elems_per_thread)
     if args.instances:
         kw = {"n_launches": args.instances} if args.workload == "c4" else {"n_instances": args.instances}
-    if args.max_rows and args.workload in ("c2", "c5"):
+    if args.max_rows and args.workload in ("c2", "c5", "addmm"):
         kw["max_rows"] = args.max_rows
     W = WORKLOADS[args.workload](dvm, **kw)
     stream = torch.cuda.current_stream()
@@ -764,7 +847,7 @@ def main():
     if W.bound == "hbm":   # "large shapes": instances moving >= 256 MB
         big = [(b, m) for b, m in zip(per_launch_work, kern_ms) if b >= 256e6]
     else:                  # instances that are tensor-bound by a wide margin (M >= 1024)
-        big = [(b, m) for b, m in zip(per_launch_work, kern_ms) if b >= 4 * 1024 * 4096 * 11008]
+        big = [(b, m) for b, m in zip(per_launch_work, kern_ms) if b >= 4 * 1024 * 4096 * 11008 / (2 if W.name == "addmm" else 1)]
     large_gbs = (sum(b for b, _ in big) / (sum(m for _, m in big) * 1e-3) / W.scale) if big else None
     gbs_each = sorted(b / (m * 1e-3) / W.scale for b, m in zip(per_launch_work, kern_ms))
     # per-launch roofline time: the slower of (flops / tensor peak) and (bytes / HBM peak)

@@ -188,6 +188,23 @@ def program_mlp_gate() -> OpProgram:
     return p
 
 
+def program_matmul() -> OpProgram:
+    """out = A @ B, bf16 in, fp32 accumulate, bf16 out (Table 2, matmul)."""
+    p = OpProgram("matmul")
+    a, b = p.input("bf16", 2), p.input("bf16", 2)
+    p.output(p.matmul(a, b), "bf16")
+    return p
+
+
+def program_addmm() -> OpProgram:
+    """out = A @ B + C with C [m,n]: the paper decomposes addmm into matmul and add (Sec. 3); the add is the
+    fused epilogue (cube-vector fusion, Sec. 5.1).  bf16 in, fp32 accumulate, bf16 out."""
+    p = OpProgram("addmm")
+    a, b, c = p.input("bf16", 2), p.input("bf16", 2), p.input("bf16", 2)
+    p.output(p.binary("add", p.matmul(a, b), c), "bf16")
+    return p
+
+
 def program_add_sqrt() -> OpProgram:
     """c = sqrt(a + b): the paper's vector-vector fusion example (Sec. 5.1)."""
     p = OpProgram("add_sqrt")
@@ -208,7 +225,11 @@ def stack_program(kind: str) -> OpProgram:
 # --------------------------------------------------------------------------
 # Seeds, shape samplers
 # --------------------------------------------------------------------------
-CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "addmm": 5}
+
+# (n, k) pairs "extracted from common LLMs" of the paper's matmul / addmm experiments (Table 2)
+LLM_NK = ((4096, 4096), (11008, 4096), (4096, 11008), (5120, 5120), (13696, 5120), (5120, 13696),
+          (8192, 8192), (28672, 8192), (8192, 28672))
 
 
 def _ints(rng, lo, hi, n):
@@ -242,6 +263,13 @@ def shapes_c4(n_launches: int = 50, n_programs: int = 64):
 def shapes_c5(n: int = 64) -> List[int]:
     rng = np.random.default_rng(CFG_SEED["c5"])
     return _ints(rng, 1, 4096, n)
+
+
+def shapes_addmm(n: int = 36) -> List[Tuple[int, int, int]]:
+    """(m, n, k) per instance: m ~ U{1..8192}, (n, k) cycling through the nine pairs of Table 2."""
+    rng = np.random.default_rng(CFG_SEED["addmm"])
+    ms = _ints(rng, 1, 8192, n)
+    return [(m,) + LLM_NK[i % len(LLM_NK)] for i, m in enumerate(ms)]
 
 
 # --------------------------------------------------------------------------

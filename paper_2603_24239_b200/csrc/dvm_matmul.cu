@@ -769,14 +769,37 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const int cs = (info >> 16) & 0xff;
             const bool bf = ((info >> 8) & 0xff) == DVM_DT_BF16;
             const long long off = (long long)row * rs + (long long)col0 * cs;
+            const char* p0 = ptr + off * (bf ? 2 : 4);
+            if (cs == 1 && col0 + CHUNK <= N && (((unsigned long long)p0) & 15) == 0) {
+              // a whole chunk of a row-contiguous operand at an aligned address: 16-byte loads
+              if (bf) {
 #pragma unroll
-            for (int i = 0; i < CHUNK; ++i) {
-              float x = 0.0f;
-              if (row_ok && col0 + i < N) {
-                const long long e = off + (long long)i * cs;
-                x = bf ? __bfloat162float(((const __nv_bfloat16*)ptr)[e]) : ((const float*)ptr)[e];
+                for (int g = 0; g < CHUNK / 8; ++g) {
+                  uint4 q = make_uint4(0u, 0u, 0u, 0u);
+                  if (row_ok) q = *(const uint4*)(p0 + 16 * g);
+                  v[8 * g + 0] = __uint_as_float(q.x << 16); v[8 * g + 1] = __uint_as_float(q.x & 0xffff0000u);
+                  v[8 * g + 2] = __uint_as_float(q.y << 16); v[8 * g + 3] = __uint_as_float(q.y & 0xffff0000u);
+                  v[8 * g + 4] = __uint_as_float(q.z << 16); v[8 * g + 5] = __uint_as_float(q.z & 0xffff0000u);
+                  v[8 * g + 6] = __uint_as_float(q.w << 16); v[8 * g + 7] = __uint_as_float(q.w & 0xffff0000u);
+                }
+              } else {
+#pragma unroll
+                for (int g = 0; g < CHUNK / 4; ++g) {
+                  float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+                  if (row_ok) q = *(const float4*)(p0 + 16 * g);
+                  v[4 * g] = q.x; v[4 * g + 1] = q.y; v[4 * g + 2] = q.z; v[4 * g + 3] = q.w;
+                }
               }
-              v[i] = x;
+            } else {
+#pragma unroll
+              for (int i = 0; i < CHUNK; ++i) {
+                float x = 0.0f;
+                if (row_ok && col0 + i < N) {
+                  const long long e = off + (long long)i * cs;
+                  x = bf ? __bfloat162float(((const __nv_bfloat16*)ptr)[e]) : ((const float*)ptr)[e];
+                }
+                v[i] = x;
+              }
             }
           }
         };

@@ -159,3 +159,35 @@ def test_empty_m_launches_nothing():
     n0 = dvm.launch_count()
     dvm.launch(code, [x, w, w.clone(), out])
     assert dvm.launch_count() == n0
+
+
+@pytest.mark.parametrize("m,n,k", [(1, 4096, 4096), (200, 11008, 4096), (130, 4096, 11008), (257, 5120, 5120),
+                                   (77, 13696, 5120), (300, 5120, 13696), (129, 8192, 8192)])
+def test_addmm_llm_shapes_small_m(m, n, k):
+    """addmm = matmul + fused add of a [m,n] operand (Table 2 shapes at token counts the oracle finishes in
+    seconds): every element."""
+    prog = wl.program_addmm()
+    ins = [wl.randn((m, k), torch.bfloat16, m), wl.randn((k, n), torch.bfloat16, n, std=0.02),
+           wl.randn((m, n), torch.bfloat16, k)]
+    outs, _ = gpu_run(prog, ins)
+    check(prog, outs, oracle_run(prog, ins))
+    assert not torch.isnan(outs[0].float()).any()
+
+
+@pytest.mark.parametrize("m,n,k", [(8192, 28672, 8192), (6000, 8192, 28672)])
+def test_addmm_largest_shapes_sampled_rows(m, n, k):
+    """The largest (n, k) pairs of Table 2 at large m: sampled rows against the oracle, one by one."""
+    prog = wl.program_addmm()
+    a = wl.randn((m, k), torch.bfloat16, 1, "cuda")
+    b = wl.randn((k, n), torch.bfloat16, 2, "cuda", std=0.02)
+    c = wl.randn((m, n), torch.bfloat16, 3, "cuda")
+    out = torch.full((m, n), float("nan"), dtype=torch.bfloat16, device="cuda")
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [(m, k), (k, n), (m, n)])
+    dvm.launch(code, [a, b, c, out])
+    assert dvm.last_device_status() == 0
+    rows = np.unique(np.concatenate([[0, 127, 128, m - 1], np.random.default_rng(7).integers(0, m, 12)]))
+    ti = torch.from_numpy(rows).cuda()
+    want = oracle_run(prog, [a[ti].cpu(), b.cpu(), c[ti].cpu()])
+    g1, _ = gate_errors(wl.to_f64(out[ti]), want[0])
+    assert g1 <= R_BF16, g1
+    assert not torch.isnan(out.float().sum())
