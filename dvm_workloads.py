@@ -39,6 +39,7 @@ UNARY_OPS = ("exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
 BINARY_OPS = ("add", "sub", "mul", "div", "min", "max")
 SCALAR_OPS = ("adds", "muls")
 REDUCE_OPS = ("sum", "max", "min")
+COMPARE_OPS = ("gt", "ge", "lt", "le", "eq", "ne")
 DTYPES = ("f32", "bf16")
 
 
@@ -82,6 +83,13 @@ class OpProgram:
 
     def matmul(self, a: int, b: int) -> int:
         return self._push(("matmul", a, b))
+
+    def compare(self, op: str, x: int, y: int) -> int:
+        assert op in COMPARE_OPS
+        return self._push(("compare", op, x, y))
+
+    def select(self, cond: int, x: int, y: int) -> int:
+        return self._push(("select", cond, x, y))
 
     def output(self, x: int, dtype: str) -> int:
         assert dtype in DTYPES
@@ -188,6 +196,17 @@ def program_mlp_gate() -> OpProgram:
     return p
 
 
+def program_if_else_add() -> OpProgram:
+    """out = (a > b ? 2x : 4x) + y, fp32: the paper's compound operator with a data-dependent branch
+    (Sec. 6, subgraph-level analysis), as Cmp + Select (Table 1)."""
+    p = OpProgram("if_else_add")
+    a, b, x, y = (p.input("f32", 3) for _ in range(4))
+    c = p.compare("gt", a, b)
+    s = p.select(c, p.scalar("muls", x, 2.0), p.scalar("muls", x, 4.0))
+    p.output(p.binary("add", s, y), "f32")
+    return p
+
+
 def program_matmul() -> OpProgram:
     """out = A @ B, bf16 in, fp32 accumulate, bf16 out (Table 2, matmul)."""
     p = OpProgram("matmul")
@@ -225,7 +244,7 @@ def stack_program(kind: str) -> OpProgram:
 # --------------------------------------------------------------------------
 # Seeds, shape samplers
 # --------------------------------------------------------------------------
-CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "addmm": 5}
+CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "addmm": 5, "ifelse": 6}
 
 # (n, k) pairs "extracted from common LLMs" of the paper's matmul / addmm experiments (Table 2)
 LLM_NK = ((4096, 4096), (11008, 4096), (4096, 11008), (5120, 5120), (13696, 5120), (5120, 13696),
@@ -263,6 +282,18 @@ def shapes_c4(n_launches: int = 50, n_programs: int = 64):
 def shapes_c5(n: int = 64) -> List[int]:
     rng = np.random.default_rng(CFG_SEED["c5"])
     return _ints(rng, 1, 4096, n)
+
+
+def shapes_if_else_add(n: int = 50, max_elems: int = 1 << 27) -> List[Tuple[int, int, int]]:
+    """(b, s, f) per instance: b ~ U{1..256}, s ~ U{1..512}, f ~ U{1..8192} (Table 2), redrawn while the
+    instance exceeds max_elems elements (five fp32 tensors of it must fit the device pools)."""
+    rng = np.random.default_rng(CFG_SEED["ifelse"])
+    out = []
+    while len(out) < n:
+        b, s_, f = int(rng.integers(1, 256, endpoint=True)), int(rng.integers(1, 512, endpoint=True)), int(rng.integers(1, 8192, endpoint=True))
+        if b * s_ * f <= max_elems:
+            out.append((b, s_, f))
+    return out
 
 
 def shapes_addmm(n: int = 36) -> List[Tuple[int, int, int]]:

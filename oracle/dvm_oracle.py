@@ -23,6 +23,8 @@ Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
   Cast                     (dst_dtype)(x)                     (Table 1, Cast)
   Sum/Max/Min reduce       [M,size,N] -> [M,1,N], here N = 1  (Table 1, Sum/Max/Min)
   Broadcast                implicit in numpy-style broadcasting (Table 1, Broadcast)
+  Cmp                      1.0 where the relation holds, else 0.0  (Table 1, Cmp)
+  Select                   cond != 0 ? x : y                       (Table 1, Select)
 Extensions that the benchmark programs need and Table 1 lacks (stated as such
 in DESIGN.md): erf, sigmoid(x) = 1/(1+exp(-x)), rsqrt(x) = 1/sqrt(x),
 recip, neg, tanh, and matmul C[i,j] = sum_k A[i,k] B[k,j] (the paper's cube
@@ -110,6 +112,15 @@ _BINARY = {
     "min": lambda a, b: np.where(a < b, a, b),       # Table 1, Min
 }
 
+_COMPARE = {                                         # Table 1, Cmp: 1 where the relation holds, else 0
+    "gt": lambda a, b: (a > b).astype(np.float64),
+    "ge": lambda a, b: (a >= b).astype(np.float64),
+    "lt": lambda a, b: (a < b).astype(np.float64),
+    "le": lambda a, b: (a <= b).astype(np.float64),
+    "eq": lambda a, b: (a == b).astype(np.float64),
+    "ne": lambda a, b: (a != b).astype(np.float64),
+}
+
 _REDUCE = {
     "sum": lambda x: np.sum(x, axis=-1, keepdims=True),   # Table 1, Sum with N = 1
     "max": lambda x: np.max(x, axis=-1, keepdims=True),   # Table 1, Max (reduce)
@@ -152,6 +163,11 @@ def evaluate(nodes, inputs, params=()):
                 vals[i] = _REDUCE[n[1]](vals[n[2]])
             elif kind == "matmul":
                 vals[i] = np.matmul(vals[n[1]], vals[n[2]])
+            elif kind == "compare":
+                vals[i] = _COMPARE[n[1]](*np.broadcast_arrays(vals[n[2]], vals[n[3]]))
+            elif kind == "select":                   # Table 1, Select: cond ? x : y, cond = (value != 0)
+                c, x, y = np.broadcast_arrays(vals[n[1]], vals[n[2]], vals[n[3]])
+                vals[i] = np.where(c != 0, x, y)
             elif kind == "output":
                 outs.append(np.array(vals[n[1]], dtype=np.float64))
             else:

@@ -393,3 +393,33 @@ def test_oracle_does_not_import_product():
         elif isinstance(node, ast.ImportFrom):
             mods.add((node.module or "").split(".")[0])
     assert mods <= {"__future__", "numpy", "scipy"}, mods
+
+
+# ---------------------------------------------------------------- compare / select
+def test_compare_and_select_definitions():
+    """Cmp gives 1 where the relation holds; Select takes x where cond != 0 (Table 1).  Pinned by hand values,
+    by the complement identities gt + le = 1 / eq + ne = 1, and by max(a, b) = select(a > b, a, b)."""
+    a = np.array([[1.0, 2.0, 3.0, -0.0], [5.0, -1.0, 2.5, 0.0]])
+    b = np.array([[1.0, 3.0, 2.0, 0.0], [4.0, -1.0, 2.5, -7.0]])
+    def run(build):
+        p = wl.OpProgram("t"); x, y = p.input("f32", 2), p.input("f32", 2); p.output(build(p, x, y), "f32")
+        return orc.evaluate(p.nodes, [a, b])[0]
+    assert np.array_equal(run(lambda p, x, y: p.compare("gt", x, y)), [[0, 0, 1, 0], [1, 0, 0, 1]])
+    assert np.array_equal(run(lambda p, x, y: p.compare("eq", x, y)), [[1, 0, 0, 1], [0, 1, 1, 0]])   # -0 == +0
+    for u, v in (("gt", "le"), ("ge", "lt"), ("eq", "ne")):
+        assert np.array_equal(run(lambda p, x, y: p.compare(u, x, y)) + run(lambda p, x, y: p.compare(v, x, y)), np.ones((2, 4)))
+    assert np.array_equal(run(lambda p, x, y: p.select(p.compare("gt", x, y), x, y)), np.maximum(a, b))
+    assert np.array_equal(run(lambda p, x, y: p.select(p.compare("lt", x, y), x, y)), np.minimum(a, b))
+    # a non-0/1 condition value counts as true
+    assert np.array_equal(run(lambda p, x, y: p.select(y, x, y)), np.where(b != 0, a, b))
+
+
+def test_if_else_add_closed_form():
+    """(a > b ? 2x : 4x) + y against the formula written out with numpy; a == b takes the else branch."""
+    rng = np.random.default_rng(3)
+    a, b, x, y = (rng.standard_normal((3, 5, 7)) for _ in range(4))
+    b[0, 0, :3] = a[0, 0, :3]
+    got = orc.evaluate(wl.program_if_else_add().nodes, [a, b, x, y])[0]
+    want = np.where(a > b, 2.0 * x, 4.0 * x) + y
+    assert np.array_equal(got, want)
+    assert np.array_equal(got[0, 0, :3], 4.0 * x[0, 0, :3] + y[0, 0, :3])
