@@ -62,6 +62,8 @@ enum {
 enum { DVM_ADD = 0, DVM_SUB = 1, DVM_MUL = 2, DVM_DIV = 3, DVM_MIN = 4, DVM_MAX = 5 };
 /* Tensor-scalar operators (Table 1: Adds, Muls). */
 enum { DVM_ADDS = 0, DVM_MULS = 1 };
+/* Comparisons (Table 1: Cmp): the value is 1.0 where the relation holds, else 0.0. */
+enum { DVM_CMP_GT = 0, DVM_CMP_GE = 1, DVM_CMP_LT = 2, DVM_CMP_LE = 3, DVM_CMP_EQ = 4, DVM_CMP_NE = 5 };
 /* Row reductions over the last axis, keepdim (Table 1: Sum / Max / Min with N = 1). */
 enum { DVM_SUM = 0, DVM_RMAX = 1, DVM_RMIN = 2 };
 
@@ -92,6 +94,11 @@ int dvm_program_binary(dvm_program* p, int op, int x, int y, int* value_id);
 int dvm_program_scalar(dvm_program* p, int op, int x, float s, int* value_id);
 /* Same, the scalar being runtime argument `param` of dvm_encode (e.g. 1/cols). */
 int dvm_program_scalar_param(dvm_program* p, int op, int x, int param, int* value_id);
+/* Table 1 Cmp: x `op` y elementwise (operands broadcast), 1.0 / 0.0. */
+int dvm_program_compare(dvm_program* p, int op, int x, int y, int* value_id);
+/* Table 1 Select: cond != 0 ? x : y elementwise (operands broadcast).  Cmp and Select take tile operands:
+ * an operand that is one value per row makes dvm_encode return DVM_ERR_UNSUPPORTED. */
+int dvm_program_select(dvm_program* p, int cond, int x, int y, int* value_id);
 /* Table 1 Cast: rounds the value to `dtype` (nearest even); values stay fp32 in registers. */
 int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
 /* Table 1 Sum / Max / Min over the last axis (axis must be -1), size-1 axis kept. */

@@ -28,6 +28,7 @@ UNARY = {"exp": 0, "sqrt": 1, "rsqrt": 2, "abs": 3, "log": 4, "erf": 5, "sigmoid
 BINARY = {"add": 0, "sub": 1, "mul": 2, "div": 3, "min": 4, "max": 5}
 SCALAR = {"adds": 0, "muls": 1}
 REDUCE = {"sum": 0, "max": 1, "min": 2}
+COMPARE = {"gt": 0, "ge": 1, "lt": 2, "le": 3, "eq": 4, "ne": 5}
 
 
 class Shape(C.Structure):
@@ -54,6 +55,8 @@ _sig = {
     "dvm_program_binary": ([_vp, _i, _i, _i, _pi], _i),
     "dvm_program_scalar": ([_vp, _i, _i, C.c_float, _pi], _i),
     "dvm_program_scalar_param": ([_vp, _i, _i, _i, _pi], _i),
+    "dvm_program_compare": ([_vp, _i, _i, _i, _pi], _i),
+    "dvm_program_select": ([_vp, _i, _i, _i, _pi], _i),
     "dvm_program_cast": ([_vp, _i, _i, _pi], _i),
     "dvm_program_reduce": ([_vp, _i, _i, _i, _pi], _i),
     "dvm_program_matmul": ([_vp, _i, _i, _pi], _i),
@@ -139,6 +142,12 @@ class Program:
     def matmul(self, a, b):
         return self._node(lib.dvm_program_matmul, a, b)
 
+    def compare(self, op, x, y):
+        return self._node(lib.dvm_program_compare, COMPARE.get(op, op), x, y)
+
+    def select(self, cond, x, y):
+        return self._node(lib.dvm_program_select, cond, x, y)
+
     def output(self, x, dtype):
         _check(lib.dvm_program_output(self._h, x, DTYPES.get(dtype, dtype)), "dvm_program_output")
 
@@ -179,6 +188,10 @@ def program_from_nodes(nodes: Iterable[tuple]) -> Program:
             ids[i] = p.reduce(n[1], ids[n[2]])
         elif k == "matmul":
             ids[i] = p.matmul(ids[n[1]], ids[n[2]])
+        elif k == "compare":
+            ids[i] = p.compare(n[1], ids[n[2]], ids[n[3]])
+        elif k == "select":
+            ids[i] = p.select(ids[n[1]], ids[n[2]], ids[n[3]])
         elif k == "output":
             p.output(ids[n[1]], n[2])
         else:

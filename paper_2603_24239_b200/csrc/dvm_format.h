@@ -59,6 +59,7 @@ enum {
   DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
   DVM_F_FLAT = 4,       // pure elementwise program laid out as a flat range
   DVM_F_PRIMARY_DENSE = 8, // the primary operand is dense: row r starts at element r * C of its tensor
+  DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select: it needs the extended interpreter variant
   DVM_F_LOADS_BY_ROW = 16  // some load is issued per row (row-by-row images, per-row scalars); otherwise
                            // thread 0 alone issues every copy of a tile
 };
@@ -119,6 +120,7 @@ enum {
   DVM_U_ERF = 5, DVM_U_SIGMOID = 6, DVM_U_NEG = 7, DVM_U_RECIP = 8, DVM_U_FLOOR = 9,
   DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12, DVM_U_NUN = 13
 };
+enum { DVM_C_GT = 0, DVM_C_GE = 1, DVM_C_LT = 2, DVM_C_LE = 3, DVM_C_EQ = 4, DVM_C_NE = 5, DVM_C_NCMP = 6 };
 // SUMSQ (sum of squares of R0, R0 kept) is what the encoder emits for reduce_sum(x * x).
 enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_SUMSQ = 3, DVM_R_NRED = 4 };
 
@@ -148,7 +150,12 @@ enum {
   DVM_OP_RED = 0x38,   // 0x38 + reduce (4); a = dst scalar register   : S[a] = reduce(ACC) over the row
   DVM_OP_LD2 = 0x40,   // 0x40 + arith; a = local register x, b = local register y | dtype(x) << 6 | dtype(y) << 7
                        //                                             : ACC = L[x] op L[y]   (fused copy + arithmetic)
-  DVM_OP_LAST = 0x48   // every arithmetic class starts at a multiple of 8: the low 3 bits are the operation
+  DVM_OP_CMP = 0x50,   // 0x50 + comparison; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC cmp L[a] ? 1 : 0
+  DVM_OP_SEL = 0x58,   // Table 1, Select; a = local register p, b = local register q | dtype(p) << 6 | dtype(q) << 7
+                       //   0x58: ACC = ACC != 0 ? L[p] : L[q]     (the condition is in the accumulator)
+                       //   0x59: ACC = L[p] != 0 ? L[q] : ACC     (the else-value is in the accumulator)
+                       //   0x5a: ACC = L[p] != 0 ? ACC : L[q]     (the then-value is in the accumulator)
+  DVM_OP_LAST = 0x60   // every arithmetic class starts at a multiple of 8: the low 3 bits are the operation
 };
 #define DVM_REG_ACC 0xff
 // DVM_SK_FMAU: S[a] = unary(S[src] * imm0 + imm1); len 4: word1 = unary (0xff: none) | src << 8, word2 = imm0, word3 = imm1

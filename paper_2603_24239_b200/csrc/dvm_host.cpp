@@ -127,6 +127,27 @@ extern "C" int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* 
   return push_node(p, n, value_id);
 }
 
+extern "C" int dvm_program_compare(dvm_program* p, int op, int x, int y, int* value_id) {
+  if (!valid_value(p, x) || !valid_value(p, y) || op < 0 || op > DVM_CMP_NE) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_COMPARE;
+  n.op = (uint8_t)op;
+  n.x = (int16_t)x;
+  n.y = (int16_t)y;
+  n.param = -1;
+  return push_node(p, n, value_id);
+}
+
+extern "C" int dvm_program_select(dvm_program* p, int cond, int x, int y, int* value_id) {
+  if (!valid_value(p, cond) || !valid_value(p, x) || !valid_value(p, y)) return DVM_ERR_INVALID_ARG;
+  Node n = {};
+  n.kind = NK_SELECT;
+  n.x = (int16_t)cond;
+  n.y = (int16_t)x;
+  n.param = (int16_t)y;
+  return push_node(p, n, value_id);
+}
+
 extern "C" int dvm_program_matmul(dvm_program* p, int a, int b, int* value_id) {
   if (!valid_value(p, a) || !valid_value(p, b)) return DVM_ERR_INVALID_ARG;
   if (p->nodes[a].kind != NK_INPUT || p->nodes[b].kind != NK_INPUT) return DVM_ERR_UNSUPPORTED;
@@ -157,7 +178,9 @@ extern "C" int dvm_program_finalize(dvm_program* p) {
   for (int i = 0; i < p->n_nodes; ++i) {
     const Node& n = p->nodes[i];
     if (n.kind != NK_INPUT && (n.x < 0 || n.x >= i)) return DVM_ERR_INVALID_ARG;
-    if ((n.kind == NK_BINARY || n.kind == NK_MATMUL) && (n.y < 0 || n.y >= i)) return DVM_ERR_INVALID_ARG;
+    if ((n.kind == NK_BINARY || n.kind == NK_MATMUL || n.kind == NK_COMPARE || n.kind == NK_SELECT) && (n.y < 0 || n.y >= i))
+      return DVM_ERR_INVALID_ARG;
+    if (n.kind == NK_SELECT && (n.param < 0 || n.param >= i)) return DVM_ERR_INVALID_ARG;
   }
   if (p->n_matmul > 0) {
     if (p->n_matmul > 2) return DVM_ERR_UNSUPPORTED;
@@ -169,7 +192,7 @@ extern "C" int dvm_program_finalize(dvm_program* p) {
         a = n.x;
         if (p->nodes[n.x].dtype != DVM_BF16 || p->nodes[n.y].dtype != DVM_BF16) return DVM_ERR_UNSUPPORTED;
       }
-      if (n.kind == NK_REDUCE) return DVM_ERR_UNSUPPORTED;  // cube-vector fusion: elementwise epilogue only
+      if (n.kind == NK_REDUCE || n.kind == NK_COMPARE || n.kind == NK_SELECT) return DVM_ERR_UNSUPPORTED;  // epilogues: plain elementwise arithmetic only
     }
   }
   p->finalized = true;
@@ -406,7 +429,8 @@ static bool gen_body(Enc& e) {
     const Node& n = p->nodes[i];
     if (n.kind == NK_INPUT || e.alias[i] >= 0) continue;
     e.uses[root(e, n.x)]++;
-    if (n.kind == NK_BINARY) e.uses[root(e, n.y)]++;
+    if (n.kind == NK_BINARY || n.kind == NK_COMPARE || n.kind == NK_SELECT) e.uses[root(e, n.y)]++;
+    if (n.kind == NK_SELECT) e.uses[root(e, n.param)]++;
   }
   for (int o = 0; o < p->n_outputs; ++o) e.uses[root(e, p->outputs[o].value)]++;
   // reduce_sum(x * x) with no other consumer of the square becomes one sum-of-squares reduction
@@ -431,7 +455,8 @@ static bool gen_body(Enc& e) {
     int x = root(e, n.x);
     if (n.kind == NK_REDUCE && e.fused_sq[x]) x = root(e, p->nodes[x].x);
     e.n_cons[x]++; e.one_cons[x] = (int16_t)i;
-    if (n.kind == NK_BINARY) { int y = root(e, n.y); e.n_cons[y]++; e.one_cons[y] = (int16_t)i; }
+    if (n.kind == NK_BINARY || n.kind == NK_COMPARE || n.kind == NK_SELECT) { int y = root(e, n.y); e.n_cons[y]++; e.one_cons[y] = (int16_t)i; }
+    if (n.kind == NK_SELECT) { int z = root(e, n.param); e.n_cons[z]++; e.one_cons[z] = (int16_t)i; }
   }
   for (int o = 0; o < p->n_outputs; ++o) { int v = root(e, p->outputs[o].value); e.n_cons[v] += 2; }
 
@@ -459,6 +484,7 @@ static bool gen_body(Enc& e) {
     const Node& n = p->nodes[i];
     if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i]) continue;
     int x = root(e, n.x);
+    if (e.cls[i] == CLS_SCAL && (n.kind == NK_COMPARE || n.kind == NK_SELECT)) { e.fail = true; break; }
     if (e.cls[i] == CLS_SCAL && n.kind != NK_REDUCE) {
       // ---- per-row scalar arithmetic ----
       if (e.fused_sc[i]) continue;  // folded into the multiply-add instruction of a later node
@@ -557,7 +583,61 @@ static bool gen_body(Enc& e) {
       continue;
     }
     // ---- tile-class result in the accumulator ----
-    if (n.kind == NK_BINARY) {
+    if (n.kind == NK_COMPARE) {
+      // ACC = ACC cmp L[b]; with the right operand in the accumulator the relation is mirrored
+      static const uint8_t kMirror[6] = {DVM_C_LT, DVM_C_LE, DVM_C_GT, DVM_C_GE, DVM_C_EQ, DVM_C_NE};
+      const int y = root(e, n.y);
+      if (e.cls[i] != CLS_TILE || e.cls[x] != CLS_TILE || e.cls[y] != CLS_TILE) { e.fail = true; break; }
+      int a = x, b = y;
+      uint8_t cop = n.op;
+      if (e.acc == y && e.acc != x) { a = y; b = x; cop = kMirror[cop]; }
+      ensure_acc(e, a);
+      if (e.fail) break;
+      const int bk = b == a ? 0xff : e.lreg_of[b];
+      if (bk < 0) { e.fail = true; break; }
+      e.uses[a]--;
+      e.uses[b]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      emit(e, DVM_INSN(DVM_OP_CMP + cop, 1, bk, b == a ? DVM_DT_F32 : e.ldt_of[b]));
+      e.acc = (int16_t)i;
+      release(e, a);
+      if (b != a) release(e, b);
+    } else if (n.kind == NK_SELECT) {
+      // one of {condition, then-value, else-value} stays in (or moves to) the accumulator, the other two are
+      // read from local registers
+      const int xv = root(e, n.y), yv = root(e, n.param);
+      if (e.cls[i] != CLS_TILE || e.cls[x] != CLS_TILE || e.cls[xv] != CLS_TILE || e.cls[yv] != CLS_TILE) { e.fail = true; break; }
+      int form = 0, in_acc = x, p1 = xv, p2 = yv;             // 0x58: condition in ACC, L[then], L[else]
+      if (e.acc == yv && yv != x) { form = 1; in_acc = yv; p1 = x; p2 = xv; }        // 0x59: L[cond], L[then], else in ACC
+      else if (e.acc == xv && xv != x) { form = 2; in_acc = xv; p1 = x; p2 = yv; }   // 0x5a: L[cond], then in ACC, L[else]
+      ensure_acc(e, in_acc);
+      if (e.fail) break;
+      const int rd[2] = {p1, p2};
+      for (int q = 0; q < 2 && !e.fail; ++q) {
+        const int v = rd[q];
+        if (e.lreg_of[v] >= 0) continue;
+        if (e.acc != v) { e.fail = true; break; }
+        const int k = alloc_tmp(e);  // also the accumulator's value: keep a copy in a local register
+        if (k < 0) break;
+        emit(e, DVM_INSN(DVM_OP_STA, 1, k, 0));
+        e.lreg_of[v] = (int8_t)k;
+        e.ldt_of[v] = DVM_DT_F32;
+        e.tmp_val[k - e.n_in_regs] = (int16_t)v;
+      }
+      if (e.fail) break;
+      e.uses[x]--;
+      e.uses[xv]--;
+      e.uses[yv]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      emit(e, DVM_INSN(DVM_OP_SEL + form, 1, e.lreg_of[p1],
+                       (uint32_t)e.lreg_of[p2] | ((uint32_t)e.ldt_of[p1] << 6) | ((uint32_t)e.ldt_of[p2] << 7)));
+      e.acc = (int16_t)i;
+      release(e, x);
+      if (xv != x) release(e, xv);
+      if (yv != x && yv != xv) release(e, yv);
+    } else if (n.kind == NK_BINARY) {
       int y = root(e, n.y);
       uint8_t ar = kBinMap[n.op];
       int a = x, b = y;  // a: accumulator operand, b: the other
@@ -668,7 +748,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
           if (s.dims[k] < 0) return DVM_ERR_INVALID_ARG;
           d[D - s.rank + k] = s.dims[k];
         }
-      } else if (n.kind == NK_BINARY) {
+      } else if (n.kind == NK_BINARY || n.kind == NK_COMPARE || n.kind == NK_SELECT) {
         const int64_t* a = e.dims[n.x];
         const int64_t* b = e.dims[n.y];
         for (int k = 0; k < D; ++k) {
@@ -676,6 +756,14 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
           else if (a[k] == 1) d[k] = b[k];
           else if (b[k] == 1) d[k] = a[k];
           else return DVM_ERR_SHAPE_MISMATCH;
+        }
+        if (n.kind == NK_SELECT) {
+          const int64_t* c3 = e.dims[n.param];
+          for (int k = 0; k < D; ++k) {
+            if (c3[k] == d[k] || c3[k] == 1) continue;
+            if (d[k] == 1) d[k] = c3[k];
+            else return DVM_ERR_SHAPE_MISMATCH;
+          }
         }
       } else {
         for (int k = 0; k < D; ++k) d[k] = e.dims[n.x][k];
@@ -961,6 +1049,8 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
   if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
   if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
+  for (int i = 0; i < NN; ++i)
+    if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;
   for (int k = 0; k < e.n_in_regs; ++k)
     if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
 
@@ -1049,6 +1139,8 @@ static int insn_expected_len(uint32_t op, uint32_t w0) {
   if (op <= DVM_OP_BCS) return 1;
   if (op == DVM_OP_SOP) return DVM_INSN_B(w0) == DVM_SK_BINI ? 3 : (DVM_INSN_B(w0) == DVM_SK_FMAU ? 4 : 2);
   if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) return 1;
+  if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) return 1;
+  if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) return 1;
   if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) return 2;
   if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) return 1;
@@ -1183,8 +1275,10 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       else if (bb == DVM_SK_UN) { if (sub >= DVM_U_NUN) return DVM_ERR_BAD_CODE; }
       else if (bb == DVM_SK_FMAU) { if (sub >= DVM_U_NUN && sub != 0xff) return DVM_ERR_BAD_CODE; }
       else return DVM_ERR_BAD_CODE;
-    } else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) {
+    } else if ((op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) || (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3)) {
       if (!lreg_ok(a, ((bb >> 6) & 1) ? u_bf16 : u_f32) || !lreg_ok(bb & 0x3f, (bb >> 7) ? u_bf16 : u_f32)) return DVM_ERR_BAD_CODE;
+    } else if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) {
+      if (bb > DVM_DT_BF16 || (a != DVM_REG_ACC && !lreg_ok(a, bb == DVM_DT_BF16 ? u_bf16 : u_f32))) return DVM_ERR_BAD_CODE;
     }
     pc += len;
   }
@@ -1275,6 +1369,18 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + 8) outf(o, "%-9s acc, acc, s%u\n", kArith[op - DVM_OP_BINS], a);
     else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + 8)
       outf(o, "%-9s acc, l%u%s, l%u%s\n", kArith[op - DVM_OP_LD2], a, ((bb >> 6) & 1) ? ".bf16" : "", bb & 0x3f, (bb >> 7) ? ".bf16" : "");
+    else if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) {
+      static const char* kCmp[6] = {"cmp.gt", "cmp.ge", "cmp.lt", "cmp.le", "cmp.eq", "cmp.ne"};
+      if (a == DVM_REG_ACC) outf(o, "%-9s acc, acc, acc\n", kCmp[op - DVM_OP_CMP]);
+      else outf(o, "%-9s acc, acc, l%u%s\n", kCmp[op - DVM_OP_CMP], a, dts);
+    }
+    else if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) {
+      const char* s1 = ((bb >> 6) & 1) ? ".bf16" : "";
+      const char* s2 = (bb >> 7) ? ".bf16" : "";
+      if (op == DVM_OP_SEL) outf(o, "select    acc, acc ? l%u%s : l%u%s\n", a, s1, bb & 0x3f, s2);
+      else if (op == DVM_OP_SEL + 1) outf(o, "select    acc, l%u%s ? l%u%s : acc\n", a, s1, bb & 0x3f, s2);
+      else outf(o, "select    acc, l%u%s ? acc : l%u%s\n", a, s1, bb & 0x3f, s2);
+    }
     else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) outf(o, "%-9s acc, acc\n", kUn[op - DVM_OP_UN]);
     else if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) outf(o, "row%-6s s%u, acc\n", kRed[op - DVM_OP_RED], a);
     else if (op == DVM_OP_SOP) {

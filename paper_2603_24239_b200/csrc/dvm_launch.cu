@@ -37,9 +37,11 @@ long long g_launches = 0;
 template <int V, int PW>
 int occupancy(int* out, size_t smem) {
   int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false>, dvm::THREADS, smem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false, true>, dvm::THREADS, smem));
   *out = n > 0 ? n : 1;
   return DVM_OK;
 }
@@ -134,16 +136,23 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   return DVM_OK;
 }
 
-template <int PW>
-int launch_variant(int V, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
-  const bool single = prm.n_programs == 1 && !prm.use_queue;
+// One kernel variant per (elements per thread, parameter-block size, single program, extended ISA).
+template <int PW, bool EXT>
+void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
   if (V == 32) {
-    if (single) dvm::dvm_vm_kernel<32, PW, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<32, PW, false><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    if (single) dvm::dvm_vm_kernel<32, PW, true, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<32, PW, false, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
   } else {
-    if (single) dvm::dvm_vm_kernel<16, PW, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<16, PW, false><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    if (single) dvm::dvm_vm_kernel<16, PW, true, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<16, PW, false, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
   }
+}
+
+template <int PW>
+int launch_variant(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+  const bool single = prm.n_programs == 1 && !prm.use_queue;
+  if (ext) launch_variant_ext<PW, true>(V, single, prm, grid, smem, stream);
+  else launch_variant_ext<PW, false>(V, single, prm, grid, smem, stream);
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;
@@ -159,12 +168,14 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   uint64_t total_tiles = 0;
   uint32_t units = 0;
   int V = 0;
+  bool ext = false;  // some program uses Cmp / Select: the extended interpreter variant runs the launch
   for (int i = 0; i < n_programs; ++i) {
     const uint32_t* c = (const uint32_t*)codes[i];
     need += c[DVM_H_TOTAL_WORDS];
     total_tiles += c[DVM_H_N_TILES];
     if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) ext = true;
     if (V && v != V) return DVM_ERR_INVALID_ARG;  // one kernel variant per launch: same elements per thread
     V = v;
   }
@@ -206,9 +217,9 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
-    return launch_variant<PW_SMALL>(V, S, grid, smem, stream);
+    return launch_variant<PW_SMALL>(V, ext, S, grid, smem, stream);
   }
-  return launch_variant<PW_LARGE>(V, P, grid, smem, stream);
+  return launch_variant<PW_LARGE>(V, ext, P, grid, smem, stream);
 }
 
 }  // namespace
@@ -366,6 +377,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   uint64_t need = dir, total_tiles = 0;
   uint32_t units = 0;
   int V = 0;
+  bool ext = false;  // some program uses Cmp / Select: the extended interpreter variant runs the launch
   for (int i = 0; i < n_programs; ++i) {
     if (!codes[i] || !tensors[i]) return DVM_ERR_INVALID_ARG;
     int st = dvm_verify(codes[i], code_sizes[i]);
@@ -376,6 +388,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     total_tiles += c[DVM_H_N_TILES];
     if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) ext = true;
     if (V && v != V) return DVM_ERR_INVALID_ARG;
     V = v;
   }
@@ -419,7 +432,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
-    return launch_variant<PW_SMALL>(V, S, grid, smem, stream);
+    return launch_variant<PW_SMALL>(V, ext, S, grid, smem, stream);
   }
-  return launch_variant<PW_LARGE>(V, P, grid, smem, stream);
+  return launch_variant<PW_LARGE>(V, ext, P, grid, smem, stream);
 }

@@ -5,7 +5,7 @@
 #include "../../include/dvm.h"
 #include "dvm_format.h"
 
-enum NodeKind : uint8_t { NK_INPUT, NK_UNARY, NK_BINARY, NK_SCALAR, NK_CAST, NK_REDUCE, NK_MATMUL };
+enum NodeKind : uint8_t { NK_INPUT, NK_UNARY, NK_BINARY, NK_SCALAR, NK_CAST, NK_REDUCE, NK_MATMUL, NK_COMPARE, NK_SELECT };
 
 struct Node {
   uint8_t kind;
@@ -13,7 +13,7 @@ struct Node {
   uint8_t dtype;
   int8_t rank;
   int16_t x, y;
-  int16_t param;  // >= 0: scalar comes from the runtime argument list
+  int16_t param;  // NK_SCALAR: >= 0: the scalar comes from the runtime argument list; NK_SELECT: the third operand
   float imm;
 };
 

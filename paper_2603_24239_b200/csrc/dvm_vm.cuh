@@ -132,7 +132,9 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
 
 // SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
-template <int V, int PW, bool SINGLE>
+// EXT: the variant that also decodes Cmp / Select (launched when a program uses them: DVM_F_EXT_ISA); the
+// basic variant stays as compact as it is without them.
+template <int V, int PW, bool SINGLE, bool EXT>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
@@ -824,6 +826,44 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             err = ST_BAD_CODE;
             pc = pc_end;
           }
+        } break;
+        case DVM_OP_CMP >> 3: if constexpr (!EXT) { err = ST_BAD_CODE; pc = pc_end; } else {
+          // ---- ACC = ACC cmp L[y] ? 1 : 0   (Table 1, Cmp) ----
+          pc += 1;
+          const int ky = DVM_INSN_A(w0);
+          float2 Y[VP];
+          if (ky == DVM_REG_ACC) { DVM_EACH_PAIR Y[i] = A[i]; }
+          else load_reg(Y, c, reg_view(c, prog, opd0, lreg0, ky, DVM_INSN_B(w0), buf), DVM_INSN_B(w0));
+#define DVM_CMP_CASE(K, REL) \
+  case K: DVM_EACH_PAIR A[i] = make_float2(A[i].x REL Y[i].x ? 1.f : 0.f, A[i].y REL Y[i].y ? 1.f : 0.f); break;
+          switch (op & 7) {
+            DVM_CMP_CASE(DVM_C_GT, >)
+            DVM_CMP_CASE(DVM_C_GE, >=)
+            DVM_CMP_CASE(DVM_C_LT, <)
+            DVM_CMP_CASE(DVM_C_LE, <=)
+            DVM_CMP_CASE(DVM_C_EQ, ==)
+            default: DVM_EACH_PAIR A[i] = make_float2(A[i].x != Y[i].x ? 1.f : 0.f, A[i].y != Y[i].y ? 1.f : 0.f); break;
+          }
+#undef DVM_CMP_CASE
+        } break;
+        case DVM_OP_SEL >> 3: if constexpr (!EXT) { err = ST_BAD_CODE; pc = pc_end; } else {
+          // ---- Table 1, Select: the condition shrinks to one bit per slot; the value not in ACC streams in ----
+          pc += 1;
+          const int ib = DVM_INSN_B(w0);
+          const int dt1 = (ib >> 6) & 1, dt2 = (ib >> 7) & 1;
+          const int form = op & 7;
+          float2 Y[VP];
+          unsigned long long m = 0;
+          if (form == 0) {  // ACC = ACC != 0 ? L[p] : L[q]
+            DVM_EACH_PAIR m |= ((unsigned long long)(A[i].x != 0.f) << (2 * i)) | ((unsigned long long)(A[i].y != 0.f) << (2 * i + 1));
+            load_reg(A, c, reg_view(c, prog, opd0, lreg0, DVM_INSN_A(w0), dt1, buf), dt1);
+          } else {          // the condition is L[p]; 1: ACC = cond ? L[q] : ACC, 2: ACC = cond ? ACC : L[q]
+            load_reg(Y, c, reg_view(c, prog, opd0, lreg0, DVM_INSN_A(w0), dt1, buf), dt1);
+            DVM_EACH_PAIR m |= ((unsigned long long)(Y[i].x != 0.f) << (2 * i)) | ((unsigned long long)(Y[i].y != 0.f) << (2 * i + 1));
+            if (form == 1) m = ~m;  // from here on: bit set = keep ACC
+          }
+          load_reg(Y, c, reg_view(c, prog, opd0, lreg0, ib & 0x3f, dt2, buf), dt2);
+          DVM_EACH_PAIR A[i] = make_float2(((m >> (2 * i)) & 1) ? A[i].x : Y[i].x, ((m >> (2 * i + 1)) & 1) ? A[i].y : Y[i].y);
         } break;
         default:
           err = ST_BAD_CODE;

@@ -1,0 +1,66 @@
+"""GPU parity of Cmp / Select (Table 1) and of the paper's if-else-add compound operator
+(a > b ? 2x : 4x) + y.  Comparisons decide a 0/1 value: the device result must equal the oracle's exactly
+(both sides compare the same fp32 inputs)."""
+import numpy as np
+import pytest
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from tests.parity_util import check, gpu_run, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 1000), (2, 7, 1531), (4, 33, 4096), (1, 2, 8192), (5, 1, 37)])
+def test_if_else_add(shape):
+    prog = wl.program_if_else_add()
+    ins = [wl.randn(shape, torch.float32, 10 + i) for i in range(4)]
+    ins[1].view(-1)[::3] = ins[0].view(-1)[::3]          # ties a == b take the else branch
+    outs, _ = gpu_run(prog, ins)
+    want = oracle_run(prog, ins)
+    # 2x, 4x and the add are exact or correctly rounded in fp32: the result is fixed bit for bit
+    ref = (torch.where(ins[0] > ins[1], 2 * ins[2], 4 * ins[2]).double() + ins[3].double()).float()
+    assert torch.equal(outs[0].cpu(), ref)
+    check(prog, outs, want)
+
+
+@pytest.mark.parametrize("op", wl.COMPARE_OPS)
+def test_every_comparison_is_exact(op):
+    p = wl.OpProgram("cmp_" + op)
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.compare(op, a, b), "f32")
+    x = wl.randn((9, 777), torch.float32, 1)
+    y = wl.randn((9, 777), torch.float32, 2)
+    y[:, ::5] = x[:, ::5]
+    x[0, 0], y[0, 0] = 0.0, -0.0
+    outs, _ = gpu_run(p, [x, y])
+    want = oracle_run(p, [x, y])[0]
+    assert np.array_equal(wl.to_f64(outs[0]), want)
+
+
+def test_select_forms_and_mixed_dtypes():
+    """Condition in the accumulator / then-value in the accumulator / else-value in the accumulator, bf16 and
+    fp32 branches, a computed condition that is not 0/1."""
+    p = wl.OpProgram("sel")
+    c, x, y = p.input("f32", 2), p.input("bf16", 2), p.input("f32", 2)
+    s1 = p.select(c, x, y)                                   # condition loaded last: in ACC
+    s2 = p.select(c, p.unary("neg", s1), y)                  # then-value in ACC
+    s3 = p.select(p.compare("lt", x, y), x, p.scalar("adds", s2, 1.0))   # else-value in ACC
+    p.output(s3, "f32")
+    p.output(s1, "bf16")
+    cc = wl.randn((17, 333), torch.float32, 3)
+    cc[cc.abs() < 0.7] = 0.0
+    ins = [cc, wl.randn((17, 333), torch.bfloat16, 4), wl.randn((17, 333), torch.float32, 5)]
+    outs, code = gpu_run(p, ins)
+    check(p, outs, oracle_run(p, ins), strict=True)
+
+
+def test_compare_on_row_scalars_is_rejected():
+    p = wl.OpProgram("cmp_rows")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.compare("gt", a, p.reduce("max", b)), "f32")
+    pp = dvm.program_from_nodes(p.nodes)
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.encode(pp, [(4, 100), (4, 100)])
+    assert ei.value.status == -3
