@@ -7,7 +7,7 @@ dvm_launch_stacked); nothing is cached between instances.  The default
 workload is the fused residual-add + RMSNorm sweep (200 instances, bf16
 [B*S, 4096], B in 1..32, S in 1..8192).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5|addmm] [--impl dvm|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5|addmm|ifelse] [--impl dvm|reference]
 
 Prints one JSON line (rank 0).  `value` is algorithmic GB/s of the whole job
 with inputs resident in HBM; `e2e` is the same metric through dvm_run_host
@@ -627,8 +627,66 @@ class AddmmWorkload:
         return flops / t_all / 1e12, t_all, f"[256,4096] @ [4096,4096] + [256,4096] repeated for {t_all:.0f} s, numpy float64"
 
 
-WORKLOADS = {"addmm": AddmmWorkload, "c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
-for _W in (C1Workload, C2Workload, C3Workload, C4Workload):   # the memory-bound sweeps: work = algorithmic bytes
+class IfElseWorkload:
+    """The paper's if-else-add compound operator (a > b ? 2x : 4x) + y, fp32 [b,s,f] (Table 2), dynamic instances."""
+    name = "ifelse"
+
+    def __init__(self, dvm, n_instances=50, device="cuda"):
+        self.dvm = dvm
+        self.prog = wl.program_if_else_add()
+        self.p = dvm.program_from_nodes(self.prog.nodes)
+        self.enc = dvm.binding.Encoder(self.p)
+        self.shapes = wl.shapes_if_else_add(n_instances)
+        self.elems = [b * s_ * f for b, s_, f in self.shapes]
+        self.pool = max(self.elems)
+        seed = wl.data_seed("ifelse", 0)
+        self.ins = [wl.randn((self.pool,), torch.float32, seed + i, device) for i in range(4)]
+        self.out = torch.empty((self.pool,), dtype=torch.float32, device=device)
+        self.bytes_per_instance = [20 * n for n in self.elems]   # four fp32 reads, one fp32 write per element
+        self.total_bytes = sum(self.bytes_per_instance)
+        self.description = ("ifelse: (a > b ? 2x : 4x) + y, fp32 [b,s,f], b 1..256, s 1..512, f 1..8192 (instances above "
+                            f"2^27 elements redrawn), {n_instances} dynamic instances, each re-encoded per launch")
+        self.l2_policy = "mean instance 0.8 GB over five tensors, far above L2"
+
+    def run_step(self, stream, events=None, enc_ns=None):
+        import ctypes as C
+        lib_launch = self.dvm.binding.lib.dvm_launch
+        arr = (C.c_void_p * 5)(*[t.data_ptr() for t in self.ins], self.out.data_ptr())
+        for shp in self.shapes:
+            t0 = time.perf_counter_ns()
+            size = self.enc.encode((shp,) * 4)
+            t1 = time.perf_counter_ns()
+            if enc_ns is not None:
+                enc_ns.append(t1 - t0)
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st = lib_launch(self.enc.buf, size, arr, 5, stream.cuda_stream)
+            if st != 0:
+                raise self.dvm.DvmError(st, "dvm_launch")
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+        return len(self.shapes)
+
+    def setup_e2e(self):
+        self.staging = None
+
+    def run_step_e2e(self, stream):
+        return None
+
+    def oracle_sample(self, budget_s=12.0):
+        from oracle import dvm_oracle as orc
+        n = 1 << 22
+        ins = [wl.to_f64(t[:n]).reshape(1, 512, 8192) for t in self.ins]
+        t_all, k = 0.0, 0
+        while t_all < budget_s:
+            t0 = time.perf_counter(); orc.evaluate(self.prog.nodes, ins); t_all += time.perf_counter() - t0; k += 1
+        return k * 20 * n / t_all / 1e9, t_all, f"{k} evaluations of a [1,512,8192] instance, numpy float64"
+
+
+WORKLOADS = {"ifelse": IfElseWorkload, "addmm": AddmmWorkload, "c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
+for _W in (C1Workload, C2Workload, C3Workload, C4Workload, IfElseWorkload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
 
@@ -661,6 +719,13 @@ def run_reference(args):
         nbytes = rows * 4096 * 8 + 8192
         sample = f"{rows} rows x 4096 (one c2 instance) per step, numpy float64"
         desc = C2Workload.__doc__
+        params = ()
+    elif args.workload == "ifelse":
+        prog = wl.program_if_else_add()
+        ins = [wl.to_f64(wl.randn((1, 512, 8192), torch.float32, 1 + i)) for i in range(4)]
+        nbytes = 20 * 512 * 8192
+        sample = "one [1,512,8192] instance per step, numpy float64"
+        desc = IfElseWorkload.__doc__
         params = ()
     elif args.workload == "addmm":
         prog = wl.program_addmm()
@@ -722,7 +787,9 @@ def run_reference(args):
 
 def encode_latency(W, reps):
     """Host encode latency over `reps` repeats of each of (up to) 20 instances of the sweep: pure dvm_encode calls."""
-    if W.name == "addmm":
+    if W.name == "ifelse":
+        shapes = [(shp,) * 4 for shp in W.shapes[:20]]
+    elif W.name == "addmm":
         shapes = [((m, k), (k, n), (m, n)) for m, n, k in W.shapes[:20]]
     elif W.name == "c1":
         shapes = [((7, 1531),) * 3]
