@@ -88,6 +88,19 @@ _sig = {
     "dvm_launch_count": ([], C.c_int64),
     "dvm_strerror": ([_i], C.c_char_p),
 }
+_sig.update({
+    "dvm_fuser_create": ([C.POINTER(_vp), _vp], _i),
+    "dvm_fuser_destroy": ([_vp], None),
+    "dvm_fuser_tensor": ([_vp, _i, C.POINTER(Shape), _vp, _pi], _i),
+    "dvm_fuser_unary": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_binary": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_scalar": ([_vp, _i, _i, C.c_float, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_reduce": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_release": ([_vp, _i], _i),
+    "dvm_fuser_flush": ([_vp], _i),
+    "dvm_fuser_pending": ([_vp, _pi, _pi], _i),
+    "dvm_fuser_stats": ([_vp, _p64, _p64, _p64, _p64], _i),
+})
 for _name, (_args, _res) in _sig.items():
     _f = getattr(lib, _name)
     _f.argtypes = _args
@@ -363,6 +376,83 @@ def last_device_status(stream=None) -> int:
     st = C.c_int(0)
     _check(lib.dvm_last_device_status(_stream(stream), C.byref(st)), "dvm_last_device_status")
     return st.value
+
+
+class Fuser:
+    """The streaming runtime operator fuser (dvm_fuser_*): operators arrive one at a time on device tensors,
+    are fused as they arrive and run at flush().  `alloc(shape, dtype)` returns the device tensor for a result
+    (default: torch.empty on cuda); pass alloc=None ... address pairs for CPU-only planning tests."""
+
+    def __init__(self, stream=None, alloc=None):
+        self._h = _vp()
+        _check(lib.dvm_fuser_create(C.byref(self._h), _stream(stream)), "dvm_fuser_create")
+        self._alloc = alloc
+        self.tensors = {}   # value id -> tensor (keeps result buffers alive)
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib.dvm_fuser_destroy(self._h)
+            self._h = None
+
+    def tensor(self, t, dtype=None, shape=None) -> int:
+        """A tensor already in device memory; t is a torch tensor, or a raw address with dtype and shape."""
+        if isinstance(t, int):
+            addr, dt, shp = t, DTYPES[dtype], tuple(shape)
+        else:
+            import torch
+            addr, dt, shp = t.data_ptr(), (DTYPES["bf16"] if t.dtype == torch.bfloat16 else DTYPES["f32"]), tuple(t.shape)
+        s = Shape()
+        s.rank = len(shp)
+        for k, d in enumerate(shp):
+            s.dims[k] = d
+        out = C.c_int(-1)
+        _check(lib.dvm_fuser_tensor(self._h, dt, C.byref(s), addr, C.byref(out)), "dvm_fuser_tensor")
+        self.tensors[out.value] = t
+        return out.value
+
+    def _result(self, shape_guess, dtype):
+        import torch
+        if self._alloc is not None:
+            return self._alloc(shape_guess, dtype)
+        return torch.empty(shape_guess, dtype=torch.bfloat16 if dtype == "bf16" else torch.float32, device="cuda")
+
+    def _op(self, fn, args, out_shape, dtype):
+        buf = self._result(out_shape, dtype)
+        addr = buf if isinstance(buf, int) else buf.data_ptr()
+        s, out = Shape(), C.c_int(-1)
+        _check(fn(self._h, *args, DTYPES[dtype], addr, C.byref(s), C.byref(out)), fn.__name__)
+        got = tuple(s.dims[k] for k in range(s.rank))
+        assert tuple(out_shape) == got, (out_shape, got)
+        self.tensors[out.value] = buf
+        return out.value
+
+    def unary(self, op, x, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_unary, (UNARY.get(op, op), x), out_shape, dtype)
+
+    def binary(self, op, x, y, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_binary, (BINARY.get(op, op), x, y), out_shape, dtype)
+
+    def scalar(self, op, x, s, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_scalar, (SCALAR.get(op, op), x, float(s)), out_shape, dtype)
+
+    def reduce(self, op, x, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_reduce, (REDUCE.get(op, op), x), out_shape, dtype)
+
+    def release(self, value):
+        _check(lib.dvm_fuser_release(self._h, value), "dvm_fuser_release")
+
+    def flush(self):
+        _check(lib.dvm_fuser_flush(self._h), "dvm_fuser_flush")
+
+    def pending(self):
+        a, b = C.c_int(0), C.c_int(0)
+        _check(lib.dvm_fuser_pending(self._h, C.byref(a), C.byref(b)), "dvm_fuser_pending")
+        return a.value, b.value
+
+    def stats(self):
+        v = [C.c_int64(0) for _ in range(4)]
+        _check(lib.dvm_fuser_stats(self._h, *[C.byref(x) for x in v]), "dvm_fuser_stats")
+        return dict(zip(("ops", "groups", "launches", "stores_elided"), (x.value for x in v)))
 
 
 def selftest_bounded_wait(which: int, stream=None):

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdvm.so")
-SOURCES = ["dvm_host.cpp", "dvm_launch.cu", "dvm_matmul.cu"]
-HEADERS = ["dvm_format.h", "dvm_internal.h", "dvm_launch.h", "dvm_vm.cuh", "dvm_math.cuh", "dvm_program.h", os.path.join("..", "..", "include", "dvm.h")]
+SOURCES = ["dvm_host.cpp", "dvm_fuser.cpp", "dvm_launch.cu", "dvm_matmul.cu"]
+HEADERS = ["dvm_format.h", "dvm_internal.h", "dvm_launch.h", "dvm_vm.cuh", "dvm_math.cuh", "dvm_program.h", os.path.join("..", "..", "include", "dvm.h"), os.path.join("..", "..", "include", "dvm_fuser.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -14,7 +14,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def test_library_exports_every_declared_symbol():
-    hdr = open(os.path.join(ROOT, "include", "dvm.h")).read()
+    hdr = open(os.path.join(ROOT, "include", "dvm.h")).read() + open(os.path.join(ROOT, "include", "dvm_fuser.h")).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
     declared = set(re.findall(r"\b(dvm_[a-z0-9_]+)\s*\(", hdr))
     assert len(declared) >= 25
