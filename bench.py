@@ -927,12 +927,13 @@ def main():
         return v[min(len(v) - 1, int(q * len(v)))] if v else None
 
     traffic = None
-    tp = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.json")
+    tp = os.path.join(ROOT, "profiles", f"{W.kernel}_{args.workload}.md")
     if os.path.exists(tp):
-        with open(tp) as f:
-            tj = json.load(f)
-        # measured DRAM bytes per algorithmic byte on an ncu-captured instance, scaled to the mean launch
-        traffic = tj["dram_bytes_per_algorithmic_byte"] * sum(per_launch_bytes) / len(per_launch_bytes)
+        import re
+        mt = re.search(r"dram_bytes_per_algorithmic_byte:\s*([0-9.]+)", open(tp).read())
+        if mt:
+            # measured DRAM bytes per algorithmic byte on an ncu-captured instance, scaled to the mean launch
+            traffic = float(mt.group(1)) * sum(per_launch_bytes) / len(per_launch_bytes)
 
     line = {
         "metric": W.metric, "value": value, "unit": W.unit, "n_gpus": world,
