@@ -187,6 +187,19 @@ int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_t
 int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
                        void* const* const* tensors, const int* n_tensors, void* cuda_stream);
 
+/* Temporal stacking of DEPENDENT meta-kernels (Sec. 5.1: tiles of different operators run one after the
+ * other on the same core, which "does not require operators to be independent").  As dvm_launch_stacked,
+ * plus level[n_programs] (host): a program may read tensors that programs of LOWER levels of the same call
+ * write; programs of one level must be independent of one another.  Levels must be non-decreasing in i
+ * (DVM_ERR_INVALID_ARG otherwise): the work queue hands tiles out in that order.  Inside the kernel a tile
+ * of level L starts its loads only when every tile of the lower levels has been counted complete (stores
+ * fenced device-wide); that wait is bounded (about 2 s), after which the kernel records
+ * DVM_ERR_DEVICE_TIMEOUT for dvm_last_device_status and returns.  The grid never exceeds the number of
+ * CTAs the device keeps resident, so every tile a waiting CTA depends on is held by a running CTA. */
+int dvm_launch_stacked_levels(int n_programs, const void* const* codes, const size_t* code_sizes,
+                              void* const* const* tensors, const int* n_tensors, const int* level,
+                              void* cuda_stream);
+
 /* The stacked launch for callers that must not allocate device memory.  (The paper has no counterpart:
  * this entry point exists for deployment, not for the method.)
  *
@@ -234,7 +247,8 @@ int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t*
                   int* code_body_bytes, int* threads_per_row, int* vector_width, int* n_tile_regs);
 /* Self-test of the bounded device-side waits (no counterpart in the paper): launches one CTA that waits on
  * an mbarrier nobody completes, with the very wait routine of the interpreter (which = 0) or of the matmul
- * kernel (which = 1).  The wait gives up after its limit (about 2 s), the kernel sets the status word and
+ * kernel (which = 1), or on a tile counter nobody advances with the level wait of dvm_launch_stacked_levels
+ * (which = 2).  The wait gives up after its limit (about 2 s), the kernel sets the status word and
  * returns: dvm_last_device_status then reports DVM_ERR_DEVICE_TIMEOUT and the context stays usable. */
 int dvm_selftest_bounded_wait(int which, void* cuda_stream);
 /* Synchronises `cuda_stream`, then reads and clears the device status word of

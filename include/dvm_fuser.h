@@ -7,8 +7,12 @@
  *  - pattern-based, vector-vector: an arriving operator joins the open group that produced its operands
  *    when the iterations merge, i.e. when the group with the operator still encodes as ONE meta-kernel for
  *    the concrete shapes (the test is a trial dvm_encode: a few microseconds);
- *  - stacking-based: groups that do not depend on one another are launched together as one stacked kernel;
- *    a group that consumes another group's result runs in a later launch on the same stream.
+ *  - stacking-based: groups that do not depend on one another are launched together as one stacked kernel
+ *    (spatial stacking); a group that consumes another group's result joins the same kernel one level later
+ *    (temporal stacking of dependent operators, dvm_launch_stacked_levels), so that a flush of short levels
+ *    is ONE launch.  With temporal stacking switched off, when a level has more than 1024 tiles (4 M
+ *    elements: the host is then far ahead of the device and kernel boundaries cost nothing extra), or when
+ *    the groups do not fit one launch, each level is its own launch on the stream.
  * Flush conditions: dvm_fuser_flush (a result has to go back to the host, a synchronisation point), or the
  * operator buffer is full.  A value whose last reference the framework dropped before the flush
  * (dvm_fuser_release) and that no other group reads is never stored to global memory: that store is the
@@ -34,6 +38,9 @@ typedef struct dvm_fuser dvm_fuser; /* opaque; owned by the library */
 /* cuda_stream: the stream every launch of this fuser is issued on (cudaStream_t as void*, NULL = default). */
 int dvm_fuser_create(dvm_fuser** out, void* cuda_stream);
 void dvm_fuser_destroy(dvm_fuser* f); /* pending operators are dropped, not run; NULL is allowed */
+
+/* Temporal stacking of dependent groups in one launch: on (non-zero, the default) or off. */
+int dvm_fuser_set_temporal_stacking(dvm_fuser* f, int enabled);
 
 /* A tensor that already exists in device memory (a graph input, a parameter): *value names it. */
 int dvm_fuser_tensor(dvm_fuser* f, int dtype, const dvm_shape* shape, void* device_ptr, int* value);

@@ -77,6 +77,7 @@ _sig = {
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
     "dvm_launch_stacked": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _vp], _i),
+    "dvm_launch_stacked_levels": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _pi, _vp], _i),
     "dvm_launch_stacked_noalloc": ([_i, C.POINTER(_vp), C.POINTER(_sz), C.POINTER(C.POINTER(_vp)), _pi, _vp], _i),
     "dvm_run_host": ([_vp, _sz, C.POINTER(_vp), C.POINTER(_sz), _i, _vp, _sz, _vp], _i),
     "dvm_verify": ([_vp, _sz], _i),
@@ -91,6 +92,7 @@ _sig = {
 _sig.update({
     "dvm_fuser_create": ([C.POINTER(_vp), _vp], _i),
     "dvm_fuser_destroy": ([_vp], None),
+    "dvm_fuser_set_temporal_stacking": ([_vp, _i], _i),
     "dvm_fuser_tensor": ([_vp, _i, C.POINTER(Shape), _vp, _pi], _i),
     "dvm_fuser_unary": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_binary": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
@@ -324,8 +326,12 @@ def launch(code: Code, tensors: Sequence, stream=None):
     _check(lib.dvm_launch(code.buf, code.size, arr, len(tensors), _stream(stream)), "dvm_launch")
 
 
-def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None, noalloc: bool = False):
+def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None, noalloc: bool = False,
+                   levels: Optional[Sequence[int]] = None):
     """dvm_launch_stacked: many independent programs in one kernel launch.
+
+    levels (non-decreasing, one per program) calls dvm_launch_stacked_levels instead: a program may read what
+    programs of lower levels of the same launch write.
 
     noalloc=True calls dvm_launch_stacked_noalloc, the variant for callers that may not allocate device
     memory (its work queue lives in a fixed array inside the library instead of a cudaMalloc'd buffer)."""
@@ -335,6 +341,10 @@ def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stre
     keep = [(_vp * len(tl))(*[_ptr(t) for t in tl]) for tl in tensor_lists]
     tptr = (C.POINTER(_vp) * n)(*[C.cast(k, C.POINTER(_vp)) for k in keep])
     nt = (_i * n)(*[len(tl) for tl in tensor_lists])
+    if levels is not None:
+        lv = (_i * n)(*[int(v) for v in levels])
+        _check(lib.dvm_launch_stacked_levels(n, cptr, csz, tptr, nt, lv, _stream(stream)), "dvm_launch_stacked_levels")
+        return
     fn = lib.dvm_launch_stacked_noalloc if noalloc else lib.dvm_launch_stacked
     _check(fn(n, cptr, csz, tptr, nt, _stream(stream)), fn.__name__)
 
@@ -383,9 +393,10 @@ class Fuser:
     are fused as they arrive and run at flush().  `alloc(shape, dtype)` returns the device tensor for a result
     (default: torch.empty on cuda); pass alloc=None ... address pairs for CPU-only planning tests."""
 
-    def __init__(self, stream=None, alloc=None):
+    def __init__(self, stream=None, alloc=None, temporal_stacking: bool = True):
         self._h = _vp()
         _check(lib.dvm_fuser_create(C.byref(self._h), _stream(stream)), "dvm_fuser_create")
+        _check(lib.dvm_fuser_set_temporal_stacking(self._h, int(temporal_stacking)), "dvm_fuser_set_temporal_stacking")
         self._alloc = alloc
         self.tensors = {}   # value id -> tensor (keeps result buffers alive)
 

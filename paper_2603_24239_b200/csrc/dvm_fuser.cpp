@@ -49,9 +49,13 @@ struct dvm_fuser {
   std::vector<FOp> ops;
   std::vector<FGroup> groups;
   int64_t n_ops = 0, n_groups = 0, n_launches = 0, n_elided = 0;
+  bool temporal = true;  // dependent groups share one launch (dvm_launch_stacked_levels)
 };
 
 namespace {
+
+// Levels of more tiles than this run as launches of their own (a tile is 256 threads x 16 elements here).
+constexpr int64_t kTemporalMaxTilesPerLevel = 1024;
 
 bool value_ok(const dvm_fuser* f, int v) { return v >= 0 && v < (int)f->values.size() && f->values[v].valid; }
 
@@ -297,6 +301,12 @@ extern "C" int dvm_fuser_stats(const dvm_fuser* f, int64_t* n_ops, int64_t* n_gr
   return DVM_OK;
 }
 
+extern "C" int dvm_fuser_set_temporal_stacking(dvm_fuser* f, int enabled) {
+  if (!f) return DVM_ERR_INVALID_ARG;
+  f->temporal = enabled != 0;
+  return DVM_OK;
+}
+
 extern "C" int dvm_fuser_flush(dvm_fuser* f) {
   if (!f) return DVM_ERR_INVALID_ARG;
   int status = DVM_OK;
@@ -319,73 +329,108 @@ extern "C" int dvm_fuser_flush(dvm_fuser* f) {
   int max_level = -1;
   for (const FGroup& g : f->groups)
     if (g.alive) max_level = std::max(max_level, g.level);
-  const int saved_v = dvm_get_elems_per_thread();
-  for (int level = 0; level <= max_level && status == DVM_OK; ++level) {
-    // the groups of one level do not depend on one another: spatial stacking (Sec. 5.1)
-    std::vector<int> at;
+  // Encode every live group, in level order.  More than one group means a stacked launch, whose programs
+  // share one elements-per-thread setting.
+  struct Ready {
+    std::vector<uint64_t> code;
+    size_t size;
+    std::vector<void*> tensors;
+    int level;
+    int64_t tiles;
+  };
+  std::vector<Ready> ready;
+  std::vector<int> order;
+  for (int level = 0; level <= max_level; ++level)
     for (int g = 0; g < (int)f->groups.size(); ++g)
-      if (f->groups[g].alive && f->groups[g].level == level) at.push_back(g);
-    struct Ready {
-      std::vector<uint64_t> code;
-      size_t size;
-      std::vector<void*> tensors;
-    };
-    std::vector<Ready> ready;
-    const bool stacked = at.size() > 1;
-    if (stacked) dvm_set_elems_per_thread(16);  // the programs of one stacked launch share the setting
-    for (int g : at) {
-      Built b;
-      int st = build(f, f->groups[g].ops, nullptr, g, false, &b);
-      if (st == DVM_ERR_INVALID_ARG && !b.prog) {
-        // nothing of this group is needed any more (every result released and unread): dead code
-        bool none = true;
-        for (int k : f->groups[g].ops)
-          if (!f->values[f->ops[k].out].released || read_elsewhere(f, f->ops[k].out, g)) none = false;
-        if (none) {
-          f->n_elided += (int64_t)f->groups[g].ops.size();
-          continue;
-        }
+      if (f->groups[g].alive && f->groups[g].level == level) order.push_back(g);
+  const int saved_v = dvm_get_elems_per_thread();
+  const bool stacked = order.size() > 1;
+  if (stacked) dvm_set_elems_per_thread(16);
+  for (int g : order) {
+    Built b;
+    int st = build(f, f->groups[g].ops, nullptr, g, false, &b);
+    if (st == DVM_ERR_INVALID_ARG && !b.prog) {
+      // nothing of this group is needed any more (every result released and unread): dead code
+      bool none = true;
+      for (int k : f->groups[g].ops)
+        if (!f->values[f->ops[k].out].released || read_elsewhere(f, f->ops[k].out, g)) none = false;
+      if (none) {
+        f->n_elided += (int64_t)f->groups[g].ops.size();
+        continue;
       }
-      if (st != DVM_OK) { status = st; break; }
-      Ready r;
-      st = encode(f, b, &r.code, &r.size, nullptr);
-      if (st == DVM_OK) {
-        for (int v : b.inputs) r.tensors.push_back(f->values[v].ptr);
-        for (int v : b.outputs) r.tensors.push_back(f->values[v].ptr);
-        f->n_elided += (int64_t)f->groups[g].ops.size() - (int64_t)b.outputs.size();
-        f->n_groups++;
-        ready.push_back(std::move(r));
-      }
-      dvm_program_destroy(b.prog);
-      if (st != DVM_OK) { status = st; break; }
     }
-    if (stacked) dvm_set_elems_per_thread(saved_v);
-    if (status != DVM_OK) break;
-    int st = DVM_OK;
-    if (ready.size() > 1) {
-      std::vector<const void*> codes;
-      std::vector<size_t> sizes;
-      std::vector<void* const*> tls;
-      std::vector<int> nts;
-      for (Ready& r : ready) {
-        codes.push_back(r.code.data());
-        sizes.push_back(r.size);
-        tls.push_back(r.tensors.data());
-        nts.push_back((int)r.tensors.size());
-      }
-      st = dvm_launch_stacked((int)ready.size(), codes.data(), sizes.data(), tls.data(), nts.data(), f->stream);
+    if (st != DVM_OK) { status = st; break; }
+    Ready r;
+    r.level = f->groups[g].level;
+    r.tiles = 0;
+    st = encode(f, b, &r.code, &r.size, nullptr);
+    if (st == DVM_OK) st = dvm_code_info(r.code.data(), r.size, nullptr, &r.tiles, nullptr, nullptr, nullptr, nullptr);
+    if (st == DVM_OK) {
+      for (int v : b.inputs) r.tensors.push_back(f->values[v].ptr);
+      for (int v : b.outputs) r.tensors.push_back(f->values[v].ptr);
+      f->n_elided += (int64_t)f->groups[g].ops.size() - (int64_t)b.outputs.size();
+      f->n_groups++;
+      ready.push_back(std::move(r));
+    }
+    dvm_program_destroy(b.prog);
+    if (st != DVM_OK) { status = st; break; }
+  }
+  if (stacked) dvm_set_elems_per_thread(saved_v);
+
+  // Launch programs [lo, hi) of `ready`: one stacked kernel (with in-kernel level waits when they span
+  // several levels), or one launch each when they do not fit one parameter block.
+  auto launch_range = [&](size_t lo, size_t hi) -> int {
+    if (hi - lo == 1) {
+      int st = dvm_launch(ready[lo].code.data(), ready[lo].size, ready[lo].tensors.data(), (int)ready[lo].tensors.size(), f->stream);
       if (st == DVM_OK) f->n_launches++;
-      else if (st == DVM_ERR_TOO_LARGE || st == DVM_ERR_UNSUPPORTED) {
-        st = DVM_OK;  // too many / too large for one parameter block: one launch each
-        for (Ready& r : ready) {
-          st = dvm_launch(r.code.data(), r.size, r.tensors.data(), (int)r.tensors.size(), f->stream);
-          if (st != DVM_OK) break;
-          f->n_launches++;
+      return st;
+    }
+    std::vector<const void*> codes;
+    std::vector<size_t> sizes;
+    std::vector<void* const*> tls;
+    std::vector<int> nts, levels;
+    for (size_t k = lo; k < hi; ++k) {
+      codes.push_back(ready[k].code.data());
+      sizes.push_back(ready[k].size);
+      tls.push_back(ready[k].tensors.data());
+      nts.push_back((int)ready[k].tensors.size());
+      levels.push_back(ready[k].level);
+    }
+    int st;
+    if (levels.front() != levels.back())  // temporal stacking of dependent groups (Sec. 5.1)
+      st = dvm_launch_stacked_levels((int)(hi - lo), codes.data(), sizes.data(), tls.data(), nts.data(), levels.data(), f->stream);
+    else  // the groups of one level do not depend on one another: spatial stacking (Sec. 5.1)
+      st = dvm_launch_stacked((int)(hi - lo), codes.data(), sizes.data(), tls.data(), nts.data(), f->stream);
+    if (st == DVM_OK) f->n_launches++;
+    return st;
+  };
+  // One kernel for all levels pays while the levels are short: an in-kernel level change costs a few
+  // microseconds of drained pipeline, about what a kernel boundary costs on the device, but it saves the host
+  // one launch per level; with long levels the host is far ahead of the device anyway, and a level that is
+  // alone in its launch runs the one-program interpreter variant, which is the faster one per tile.
+  bool short_levels = true;
+  for (size_t lo = 0; lo < ready.size();) {
+    size_t hi = lo;
+    int64_t tiles = 0;
+    for (; hi < ready.size() && ready[hi].level == ready[lo].level; ++hi) tiles += ready[hi].tiles;
+    if (tiles > kTemporalMaxTilesPerLevel) short_levels = false;
+    lo = hi;
+  }
+  if (status == DVM_OK && !ready.empty()) {
+    int st = (f->temporal && short_levels) ? launch_range(0, ready.size()) : DVM_ERR_TOO_LARGE;
+    if (st == DVM_ERR_TOO_LARGE || st == DVM_ERR_UNSUPPORTED) {
+      // one launch per level, in order on the stream
+      st = DVM_OK;
+      for (size_t lo = 0; lo < ready.size() && st == DVM_OK;) {
+        size_t hi = lo;
+        while (hi < ready.size() && ready[hi].level == ready[lo].level) ++hi;
+        st = launch_range(lo, hi);
+        if (st == DVM_ERR_TOO_LARGE || st == DVM_ERR_UNSUPPORTED) {
+          st = DVM_OK;  // too many / too large for one parameter block: one launch each
+          for (size_t k = lo; k < hi && st == DVM_OK; ++k) st = launch_range(k, k + 1);
         }
+        lo = hi;
       }
-    } else if (ready.size() == 1) {
-      st = dvm_launch(ready[0].code.data(), ready[0].size, ready[0].tensors.data(), (int)ready[0].tensors.size(), f->stream);
-      if (st == DVM_OK) f->n_launches++;
     }
     status = st;
   }

@@ -17,14 +17,16 @@ namespace {
 constexpr int PW_SMALL = 496;    // words of code in a 2 KB parameter block
 constexpr int PW_LARGE = 8000;   // ... in a 32 KB parameter block (the sm_70+ limit is 32764 bytes)
 constexpr int QUEUE_SLOTS = 504;
+constexpr size_t SCRATCH_BYTES = (8 + 4 * QUEUE_SLOTS) * sizeof(unsigned int);
 constexpr int MAX_DEVICES = 64;
 constexpr size_t kMaxDynSmem = 227 * 1024 - 9 * 1024;  // dynamic shared memory a CTA may ask for (8.3 KB static part excluded)
 
 struct DeviceState {
   bool ready = false;
-  unsigned int* scratch = nullptr;  // [0] status word, [8 + 2*slot] work-queue counter pairs
+  unsigned int* scratch = nullptr;  // [0] status word, [8 + 4*slot] work-queue counters (next tile, CTAs finished, tiles completed)
   int sm_count = 0;
   int occ[2][2][DVM_MAX_LOCAL_UNITS + 1];  // resident CTAs per SM for [V == 32][large parameter block][local units], 0 = not yet asked
+  int occ_levels[2][2][DVM_MAX_LOCAL_UNITS + 1];  // the same for the variants with level waits
   unsigned queue_slot = 0;
 };
 
@@ -46,6 +48,21 @@ int occupancy(int* out, size_t smem) {
   return DVM_OK;
 }
 
+// The variant with level waits: its grid must not exceed what the device keeps resident, so it is asked itself.
+template <int V, int PW>
+int occupancy_levels(int* out, size_t smem) {
+  int n = 0;
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  int a = 0, b = 0;
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, dvm::dvm_vm_kernel<V, PW, false, false, true>, dvm::THREADS, smem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dvm::dvm_vm_kernel<V, PW, false, true, true>, dvm::THREADS, smem));
+  n = a < b ? a : b;
+  if (n <= 0) return DVM_ERR_TOO_LARGE;  // not even one CTA fits: no launch
+  *out = n;
+  return DVM_OK;
+}
+
 }  // namespace
 
 int dvm_device_state(DvmDeviceInfo* info) {
@@ -56,9 +73,10 @@ int dvm_device_state(DvmDeviceInfo* info) {
   DeviceState& d = g_dev[dev];
   if (!d.ready) {
     DVM_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
-    DVM_CUDA(cudaMalloc(&d.scratch, 4096));
-    DVM_CUDA(cudaMemset(d.scratch, 0, 4096));
+    DVM_CUDA(cudaMalloc(&d.scratch, SCRATCH_BYTES));
+    DVM_CUDA(cudaMemset(d.scratch, 0, SCRATCH_BYTES));
     memset(d.occ, 0, sizeof d.occ);
+    memset(d.occ_levels, 0, sizeof d.occ_levels);
     d.ready = true;
   }
   info->scratch = d.scratch;
@@ -69,11 +87,22 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // Resident CTAs per SM of the interpreter for a launch with `units` local-memory units (cached per device).
-static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out) {
+static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out, bool levels = false) {
   int dev = 0;
   DVM_CUDA(cudaGetDevice(&dev));
   std::lock_guard<std::mutex> lk(g_mu);
   DeviceState& d = g_dev[dev];
+  if (levels) {
+    int& lslot = d.occ_levels[V == 32 ? 1 : 0][large ? 1 : 0][units];
+    if (lslot == 0) {
+      int st;
+      if (V == 32) st = large ? occupancy_levels<32, PW_LARGE>(&lslot, smem) : occupancy_levels<32, PW_SMALL>(&lslot, smem);
+      else st = large ? occupancy_levels<16, PW_LARGE>(&lslot, smem) : occupancy_levels<16, PW_SMALL>(&lslot, smem);
+      if (st != DVM_OK) return st;
+    }
+    *out = lslot;
+    return DVM_OK;
+  }
   int& slot = d.occ[V == 32 ? 1 : 0][large ? 1 : 0][units];
   if (slot == 0) {
     int st;
@@ -158,12 +187,28 @@ int launch_variant(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size
   return DVM_OK;
 }
 
+// The variants with level waits.
+template <int PW>
+int launch_variant_levels(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+  if (V == 32) {
+    if (ext) dvm::dvm_vm_kernel<32, PW, false, true, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<32, PW, false, false, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  } else {
+    if (ext) dvm::dvm_vm_kernel<16, PW, false, true, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<16, PW, false, false, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  }
+  DVM_CUDA(cudaGetLastError());
+  dvm_count_launch();
+  return DVM_OK;
+}
+
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
 
+// `level` (may be NULL): level[i] of program i, non-decreasing; a program reads what programs of lower levels store.
 int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
-               bool use_queue, cudaStream_t stream) {
-  // directory: [program word offsets (n)][tile prefix sums (n+1)]
-  uint32_t dir = 2 * (uint32_t)n_programs + 1;
+               bool use_queue, const int* level, cudaStream_t stream) {
+  // directory: [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, with levels)]
+  uint32_t dir = (level ? 3 : 2) * (uint32_t)n_programs + 1;
   uint64_t need = dir;
   uint64_t total_tiles = 0;
   uint32_t units = 0;
@@ -187,11 +232,15 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (st != DVM_OK) return st;
 
   dvm::VMParams<PW_LARGE>& P = t_large;
-  uint32_t pos = dir, tb = 0;
+  uint32_t pos = dir, tb = 0, level_start = 0;
   for (int i = 0; i < n_programs; ++i) {
     const uint32_t* c = (const uint32_t*)codes[i];
     P.words[i] = pos;
     P.words[n_programs + i] = tb;
+    if (level) {
+      if (i > 0 && level[i] != level[i - 1]) level_start = tb;  // every tile before this one belongs to a lower level
+      P.words[2 * n_programs + 1 + i] = level_start;
+    }
     st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
     if (st != DVM_OK) return st;
     pos += c[DVM_H_TOTAL_WORDS];
@@ -202,23 +251,26 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.total_tiles = (uint32_t)total_tiles;
   P.n_words = pos;
   P.use_queue = use_queue ? 1u : 0u;
+  P.levels = level ? 1u : 0u;
   P.status = dev.scratch;
-  P.queue = dev.scratch + 8 + 2 * dev.queue_slot;
+  P.queue = dev.scratch + 8 + 4 * dev.queue_slot;
 
   const bool large = pos > PW_SMALL;
   const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;  // one spare unit, two tile slots
   P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   int occ = 0;
-  st = dvm_occupancy(V, large, (int)units, smem, &occ);
+  st = dvm_occupancy(V, large, (int)units, smem, &occ, level != nullptr);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
   int grid = (int)(total_tiles < slots ? total_tiles : slots);
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
+    if (level) return launch_variant_levels<PW_SMALL>(V, ext, S, grid, smem, stream);
     return launch_variant<PW_SMALL>(V, ext, S, grid, smem, stream);
   }
+  if (level) return launch_variant_levels<PW_LARGE>(V, ext, P, grid, smem, stream);
   return launch_variant<PW_LARGE>(V, ext, P, grid, smem, stream);
 }
 
@@ -234,7 +286,7 @@ extern "C" int dvm_launch(const void* code, size_t code_size, void* const* tenso
     return dvm_launch_matmul(w, code_size / 4, tensors, n_tensors, (cudaStream_t)cuda_stream);
   const void* codes[1] = {code};
   void* const* tl[1] = {tensors};
-  return launch_vec(1, codes, tl, &n_tensors, false, (cudaStream_t)cuda_stream);
+  return launch_vec(1, codes, tl, &n_tensors, false, nullptr, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
@@ -250,7 +302,24 @@ extern "C" int dvm_launch_stacked(int n_programs, const void* const* codes, cons
     // only vector meta-kernels stack (Sec. 5.1: stacking of meta-kernels on the Vector units)
     if (((const uint32_t*)codes[i])[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_UNSUPPORTED;
   }
-  return launch_vec(n_programs, codes, tensors, n_tensors, true, (cudaStream_t)cuda_stream);
+  return launch_vec(n_programs, codes, tensors, n_tensors, true, nullptr, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int dvm_launch_stacked_levels(int n_programs, const void* const* codes, const size_t* code_sizes,
+                                         void* const* const* tensors, const int* n_tensors, const int* level,
+                                         void* cuda_stream) {
+  if (n_programs < 0 || (n_programs > 0 && (!codes || !code_sizes || !tensors || !n_tensors || !level)))
+    return DVM_ERR_INVALID_ARG;
+  if (n_programs == 0) return DVM_OK;
+  if (n_programs > DVM_MAX_STACK) return DVM_ERR_TOO_LARGE;
+  for (int i = 0; i < n_programs; ++i) {
+    if (!codes[i] || !tensors[i]) return DVM_ERR_INVALID_ARG;
+    if (i > 0 && level[i] < level[i - 1]) return DVM_ERR_INVALID_ARG;  // the work queue hands tiles out in level order
+    int st = dvm_verify(codes[i], code_sizes[i]);
+    if (st != DVM_OK) return st;
+    if (((const uint32_t*)codes[i])[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC) return DVM_ERR_UNSUPPORTED;
+  }
+  return launch_vec(n_programs, codes, tensors, n_tensors, true, level, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int dvm_run_host(const void* code, size_t code_size, void* const* host_tensors,
@@ -294,6 +363,11 @@ __global__ void dvm_selftest_vm_wait_kernel(unsigned int* status) {
   __syncthreads();
   if (!dvm::vm_mbar_wait(b, 0) && threadIdx.x == 0) atomicMax(status, (unsigned int)dvm::ST_TIMEOUT);
 }
+// The level wait of dvm_launch_stacked_levels on a counter nobody advances (the status word's neighbour,
+// which stays zero): it gives up after its limit.
+__global__ void dvm_selftest_level_wait_kernel(unsigned int* status) {
+  if (threadIdx.x == 0 && !dvm::vm_wait_tiles_done(status + 1, 1u)) atomicMax(status, (unsigned int)dvm::ST_TIMEOUT);
+}
 }  // namespace
 
 int dvm_selftest_mm_wait(unsigned int* status, cudaStream_t stream);
@@ -309,6 +383,12 @@ extern "C" int dvm_selftest_bounded_wait(int which, void* cuda_stream) {
     return DVM_OK;
   }
   if (which == 1) return dvm_selftest_mm_wait(dev.scratch, (cudaStream_t)cuda_stream);
+  if (which == 2) {
+    dvm_selftest_level_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(dev.scratch);
+    DVM_CUDA(cudaGetLastError());
+    dvm_count_launch();
+    return DVM_OK;
+  }
   return DVM_ERR_INVALID_ARG;
 }
 
@@ -337,7 +417,7 @@ extern "C" int dvm_last_device_status(void* cuda_stream, int* status) {
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-constexpr int NOALLOC_WORDS = 64;                 // 256 bytes: [0] status word, [2..3] work-queue counters
+constexpr int NOALLOC_WORDS = 64;                 // 256 bytes: [0] status word, [2..4] work-queue counters
 static __device__ __align__(256) unsigned int dvm_noalloc_scratch[NOALLOC_WORDS];
 
 struct NoAllocDevice {
@@ -416,6 +496,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.total_tiles = (uint32_t)total_tiles;
   P.n_words = pos;
   P.use_queue = 1u;
+  P.levels = 0u;
   P.status = dev.scratch;
   P.queue = dev.scratch + 2;
   const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;

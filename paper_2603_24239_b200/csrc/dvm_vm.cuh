@@ -60,10 +60,10 @@ struct VMParams {
   uint32_t n_words;      // words used in `words`
   uint32_t use_queue;    // 1: tiles beyond the first are claimed from the work queue
   uint32_t slot_bytes;   // bytes of one tile slot in local memory (the largest program's)
-  uint32_t pad_;
+  uint32_t levels;       // 1: the directory has a third table, and tiles wait for the tiles of earlier levels
   unsigned int* status;  // device status word
-  unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished (both zero between launches)
-  uint32_t words[PW];    // [program word offsets][tile prefix sums (n+1)][programs ...]
+  unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished, [2] tiles completed (all zero between launches)
+  uint32_t words[PW];    // [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, if levels)][programs ...]
 };
 
 struct TileCtx {
@@ -123,6 +123,21 @@ __device__ __forceinline__ bool vm_mbar_wait(uint32_t bar, uint32_t parity) {
   if (vm_mbar_try(bar, parity)) return true;
   return vm_mbar_wait_slow(bar, parity);
 }
+// Bounded wait until the grid-wide counter of completed tiles has reached `need` (acquire: what those tiles
+// stored is visible afterwards).  Same limits as the barrier wait; false when it ran out.
+__device__ __noinline__ bool vm_wait_tiles_done(const unsigned int* counter, uint32_t need) {
+  unsigned long long t0, t1;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (uint32_t spin = 0; spin < (1u << 27); ++spin) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= need) return true;
+    if ((spin & 15u) != 15u) continue;  // each poll is an L2 round trip: look at the clock now and then
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    if (t1 - t0 > 2000000000ull) break;
+  }
+  return false;
+}
 // global -> shared bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned), completion on `bar`
 __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
@@ -134,7 +149,8 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
 // EXT: the variant that also decodes Cmp / Select (launched when a program uses them: DVM_F_EXT_ISA); the
 // basic variant stays as compact as it is without them.
-template <int V, int PW, bool SINGLE, bool EXT>
+// LEVELS: the stacked variant with in-kernel waits between dependent levels (dvm_launch_stacked_levels).
+template <int V, int PW, bool SINGLE, bool EXT, bool LEVELS = false>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
@@ -155,6 +171,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   const uint32_t bar0 = static_cast<uint32_t>(__cvta_generic_to_shared(s_bar));
   const uint32_t n_prog = SINGLE ? 1u : prm.n_programs;
   const bool use_queue = SINGLE ? false : prm.use_queue != 0;
+  // dependent stacking: a tile of directory entry i reads what the tiles [0, CW(2n + 1 + i)) of the launch
+  // store, so its loads start only after that many tiles are complete (the tiles of the earlier levels)
+  constexpr bool levels = LEVELS && !SINGLE;
 #define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
 
   if (tid == 0) {
@@ -476,21 +495,64 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   c.nvalid = 0;
   c.ov = 0;
   uint32_t slot_prog[2] = {0xffffffffu, 0xffffffffu};  // program whose row-vector inputs each slot holds
+  uint32_t published = 0;  // tiles of this CTA already counted in the grid-wide completion counter (of `iter` done)
+  bool held = false;  // the current tile's loads are held back until the tiles of the earlier levels are complete
   if (tile < prm.total_tiles) {
     if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
-    TileCtx cl;
-    ctx_rows(cl, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
-    issue_loads(cl, buf, true);
-    slot_prog[0] = prog_idx;
-    cp_async_commit();
+    if (!SINGLE && levels && CW(2 * n_prog + 1 + prog_idx) > 0) {
+      held = true;
+    } else {
+      TileCtx cl;
+      ctx_rows(cl, SINGLE ? kSingleProg : CW(prog_idx), SINGLE ? tile : tile - CW(n_prog + prog_idx));
+      issue_loads(cl, buf, true);
+      slot_prog[0] = prog_idx;
+      cp_async_commit();
+    }
   }
 
   while (tile < prm.total_tiles) {
     // ---- Algorithm 2, outer loop.  Every thread must be done with the previous tile before the other slot
     // is overwritten with the next tile's loads, which start now, ahead of the wait for this tile's bytes. ----
+    if constexpr (levels) {
+      if (held) {
+        // This CTA moves on to a later level.  Behind the barrier the stores of its earlier tiles are all
+        // issued: thread 0 publishes them (the fence is cumulative over what the barrier ordered before it)
+        // and counts those tiles -- only here, and when the CTA ends: tiles of the level a CTA is still
+        // working on are nobody's business yet, and a fence per tile would hold up thread 0, which issues the
+        // next tile's copies.  Then it waits, before it claims anything further: a waiting CTA sits on one
+        // tile only, the rest of the queue stays open to CTAs that are free.
+        // All earlier tiles were claimed before this one, by CTAs that are resident (the grid never exceeds
+        // the resident capacity) and that wait only for still earlier levels: the count gets there.
+        __syncthreads();
+        if (tid == 0) {
+          if (iter > published) {
+            __threadfence();
+            atomicAdd(&prm.queue[2], iter - published);
+          }
+          if (!vm_wait_tiles_done(&prm.queue[2], CW(2 * n_prog + 1 + prog_idx))) {
+            err = ST_TIMEOUT;
+            s_abort = 1;
+          }
+        }
+        published = iter;
+      }
+    }
     if (use_queue && tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
     __syncthreads();
     if (s_abort) break;  // a wait ran out in some thread during the previous tile
+    if constexpr (levels) {
+      {
+        if (held) {
+          asm volatile("fence.proxy.async;" ::: "memory");  // the bulk copies below read what generic stores wrote
+          TileCtx cl;
+          ctx_rows(cl, CW(prog_idx), tile - CW(n_prog + prog_idx));
+          issue_loads(cl, buf, true);  // a held tile is this CTA's first of its program: earlier tiles were of earlier levels
+          if (buf) slot_prog[1] = prog_idx; else slot_prog[0] = prog_idx;
+          cp_async_commit();
+          held = false;
+        }
+      }
+    }
     const uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
     ++iter;
     const bool have_next = next < prm.total_tiles;
@@ -499,7 +561,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       if (!SINGLE) while (next_prog_idx + 1 < n_prog && next >= CW(n_prog + next_prog_idx + 1)) ++next_prog_idx;
       const uint32_t nprog = SINGLE ? kSingleProg : CW(next_prog_idx);
       const bool first = buf ? slot_prog[0] != next_prog_idx : slot_prog[1] != next_prog_idx;
-      if (((CW(nprog + DVM_H_GEOM) >> 24) & DVM_F_LOADS_BY_ROW) || warp == 0) {
+      // the next tile belongs to a later level than this one: it also waits for this tile, so its loads
+      // cannot start ahead (a tile of this tile's own level has nothing left to wait for)
+      if (!SINGLE && levels && CW(2 * n_prog + 1 + next_prog_idx) > tile) {
+        held = true;
+      } else if (((CW(nprog + DVM_H_GEOM) >> 24) & DVM_F_LOADS_BY_ROW) || warp == 0) {
         TileCtx cl;  // rows of the next tile, for the threads that may issue its copies
         ctx_rows(cl, nprog, SINGLE ? next : next - CW(n_prog + next_prog_idx));
         issue_loads(cl, buf ^ 1, first);
@@ -881,14 +947,16 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
   if (err && tid == 0) atomicMax(prm.status, err);
   if (use_queue) {
-    // the last CTA to finish returns the queue to its resting state (both counters zero)
+    // the last CTA to finish returns the queue to its resting state (all counters zero)
     __syncthreads();
     if (tid == 0) {
       __threadfence();
+      if (levels && iter > published) atomicAdd(&prm.queue[2], iter - published);  // this CTA's remaining tiles are complete
       const unsigned done = atomicAdd(&prm.queue[1], 1u);
       if (done == gridDim.x - 1) {
         prm.queue[0] = 0u;
         prm.queue[1] = 0u;
+        prm.queue[2] = 0u;
         __threadfence();
       }
     }

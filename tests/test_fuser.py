@@ -92,11 +92,12 @@ def test_softmax_like_stream_matches_oracle_and_elides_intermediates():
 
 
 @pytest.mark.gpu
-def test_independent_groups_run_as_one_stacked_launch_and_dependents_later():
+@pytest.mark.parametrize("temporal", [True, False])
+def test_independent_groups_run_as_one_stacked_launch_and_dependents_later(temporal):
     a = wl.randn((100, 333), torch.float32, 1).cuda(); b = wl.randn((100, 333), torch.float32, 2).cuda()
     x = wl.randn((7, 4000), torch.float32, 3).cuda()
     w = wl.randn((100, 64), torch.float32, 4).cuda()
-    f = dvm.Fuser()
+    f = dvm.Fuser(temporal_stacking=temporal)
     va, vb, vx, vw = f.tensor(a), f.tensor(b), f.tensor(x), f.tensor(w)
     c = f.unary("sqrt", f.unary("abs", f.binary("add", va, vb, (100, 333)), (100, 333)), (100, 333))   # group 1
     z = f.scalar("muls", f.unary("sigmoid", vx, (7, 4000)), 3.0, (7, 4000))                                # group 2
@@ -106,7 +107,9 @@ def test_independent_groups_run_as_one_stacked_launch_and_dependents_later():
     n0 = dvm.launch_count()
     f.flush()
     torch.cuda.synchronize()
-    assert dvm.launch_count() - n0 == 2      # level 0: groups 1 and 2 stacked into one launch; level 1: the dependent
+    # level 0: groups 1 and 2, stacked; level 1: the dependent group -- in the same launch behind an in-kernel
+    # wait (temporal stacking), or in a second launch on the stream
+    assert dvm.launch_count() - n0 == (1 if temporal else 2)
     assert dvm.last_device_status() == 0
     cc = torch.sqrt((a + b).abs())
     assert torch.allclose(f.tensors[c], cc, rtol=1e-6, atol=0)
@@ -127,3 +130,23 @@ def test_values_survive_a_flush_and_feed_later_operators():
     torch.cuda.synchronize()
     assert torch.allclose(f.tensors[d], (a + 1.5) * a, rtol=1e-6, atol=0)
     assert f.stats()["launches"] == 2
+
+
+@pytest.mark.gpu
+def test_long_levels_keep_their_own_launches():
+    """Dependent groups whose levels exceed 1024 tiles are not stacked temporally: one launch per level."""
+    R, C = 3000, 4096                      # 3000 tiles of 256 x 16 elements per level
+    a = wl.randn((R, C), torch.float32, 6).cuda()
+    w = wl.randn((R, 64), torch.float32, 7).cuda()
+    f = dvm.Fuser()
+    va, vw = f.tensor(a), f.tensor(w)
+    m = f.reduce("max", f.unary("abs", va, (R, C)), (R, 1))
+    r = f.binary("mul", vw, m, (R, 64))    # rows of 64 against [R,1]: a second group, one level up
+    n0 = dvm.launch_count()
+    f.flush()
+    torch.cuda.synchronize()
+    assert dvm.launch_count() - n0 == 2
+    assert dvm.last_device_status() == 0
+    mm = a.abs().max(dim=1, keepdim=True).values
+    assert torch.equal(f.tensors[m], mm)
+    assert torch.allclose(f.tensors[r], w * mm, rtol=1e-6, atol=0)

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 DVM_ERR_DEVICE_TIMEOUT = -7
 
 
-@pytest.mark.parametrize("which", [0, 1])  # 0: the interpreter's wait routine, 1: the matmul kernel's
+@pytest.mark.parametrize("which", [0, 1, 2])  # the interpreter's barrier wait, the matmul kernel's, the level wait
 def test_wait_runs_out_and_reports(which):
     assert dvm.last_device_status() == 0
     t0 = time.perf_counter()

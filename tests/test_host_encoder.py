@@ -203,3 +203,17 @@ def test_encode_batch_matches_single_encodes():
         assert "instance 2" in str(ei.value)
     finally:
         dvm.set_elems_per_thread(0)
+
+
+def test_stacked_levels_rejects_decreasing_levels_before_any_launch():
+    """dvm_launch_stacked_levels: levels must be non-decreasing (the work queue hands tiles out in that
+    order); the check is on the host, ahead of every CUDA call."""
+    p = wl.OpProgram("add")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.binary("add", a, b), "f32")
+    hp = dvm.program_from_nodes(p.nodes)
+    codes = [dvm.encode(hp, [(4, 8), (4, 8)]) for _ in range(2)]
+    fake = [[0x1000, 0x2000, 0x3000], [0x3000, 0x2000, 0x4000]]   # never dereferenced: the call fails first
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.launch_stacked(codes, fake, levels=[1, 0])
+    assert ei.value.status == -1   # DVM_ERR_INVALID_ARG
