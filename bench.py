@@ -367,6 +367,7 @@ class C4Workload:
         self.dvm = dvm
         if not dvm.binding.lib.dvm_get_elems_per_thread():
             dvm.set_elems_per_thread(16)   # programs of one stacked launch share the setting; 16 fits every program
+        dvm.set_min_resident_ctas(2)       # the CTAs of a stacked launch are sized by its largest program
         self.launches = wl.shapes_c4(n_launches)
         self.progs = {k: wl.stack_program(k) for k in wl.STACK_KINDS}
         self.ps = {k: dvm.program_from_nodes(p.nodes) for k, p in self.progs.items()}

@@ -151,6 +151,14 @@ int dvm_get_num_cores(void);
  * dvm_launch_stacked fix it before encoding.  Process-wide; not thread-safe against encode. */
 void dvm_set_elems_per_thread(int v);
 int dvm_get_elems_per_thread(void);
+/* Resident CTAs per SM every encoded geometry has to leave room for: 2, or 0 (default) for no constraint.
+ * A stacked launch sizes every CTA's local memory for its largest program, so ONE program whose tile slots
+ * exceed half an SM's shared memory leaves the whole launch with one CTA per SM.  With 2, the encoder
+ * takes the best geometry among those whose slots fit twice per SM (e.g. two column blocks per row, whose
+ * row-vector operands are then half as long); a program no geometry of which fits keeps its unconstrained
+ * best.  Callers of dvm_launch_stacked set it before encoding.  Process-wide; not thread-safe against encode. */
+void dvm_set_min_resident_ctas(int n);
+int dvm_get_min_resident_ctas(void);
 
 /* The paper's tile-size rule for a flat vector operator (Sec. 4.2,
  * hardware_align_div): among tile sizes t in [1, min(total, t_max)] take the

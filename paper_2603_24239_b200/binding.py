@@ -73,6 +73,8 @@ _sig = {
     "dvm_get_num_cores": ([], _i),
     "dvm_set_elems_per_thread": ([_i], None),
     "dvm_get_elems_per_thread": ([], _i),
+    "dvm_set_min_resident_ctas": ([_i], None),
+    "dvm_get_min_resident_ctas": ([], _i),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -498,3 +500,8 @@ def get_num_cores() -> int:
 
 def set_elems_per_thread(v: int):
     lib.dvm_set_elems_per_thread(v)
+
+
+def set_min_resident_ctas(n: int):
+    """2: encode only geometries whose tile slots fit twice per SM (programs of a stacked launch); 0: no constraint."""
+    lib.dvm_set_min_resident_ctas(n)

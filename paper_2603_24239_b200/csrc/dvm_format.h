@@ -70,7 +70,8 @@ enum {
   DVM_LM_PRIVATE = 0,  // temporary: thread-private fp32 vectors, vector q of thread tid at (q * 256 + tid) * 16
   DVM_LM_BLOCK = 1,    // input whose tile is one contiguous byte range of global memory: one bulk copy per tile
   DVM_LM_ROWS = 2,     // input copied row by row (one bulk copy per row): row images DVM_ROW_PITCH(...) apart
-  DVM_LM_BCAST = 3     // row-vector input, the same for every row and tile: one row image per slot
+  DVM_LM_BCAST = 3     // row-vector input, the same for every row: one row image per slot (of the tile's column block;
+                       // with one column block it is loaded once per slot and program, else with every tile)
 };
 // bytes between the row images of a ROWS register (room for the 16-byte alignment slack on both sides)
 #define DVM_ROW_PITCH(G, V, es) ((uint32_t)(G) * (uint32_t)(V) * (uint32_t)(es) + 32u)

@@ -345,7 +345,11 @@ extern "C" int dvm_fuser_flush(dvm_fuser* f) {
       if (f->groups[g].alive && f->groups[g].level == level) order.push_back(g);
   const int saved_v = dvm_get_elems_per_thread();
   const bool stacked = order.size() > 1;
-  if (stacked) dvm_set_elems_per_thread(16);
+  const int saved_ctas = dvm_get_min_resident_ctas();
+  if (stacked) {
+    dvm_set_elems_per_thread(16);
+    dvm_set_min_resident_ctas(2);  // the launch's CTAs are sized by its largest program
+  }
   for (int g : order) {
     Built b;
     int st = build(f, f->groups[g].ops, nullptr, g, false, &b);
@@ -375,7 +379,10 @@ extern "C" int dvm_fuser_flush(dvm_fuser* f) {
     dvm_program_destroy(b.prog);
     if (st != DVM_OK) { status = st; break; }
   }
-  if (stacked) dvm_set_elems_per_thread(saved_v);
+  if (stacked) {
+    dvm_set_elems_per_thread(saved_v);
+    dvm_set_min_resident_ctas(saved_ctas);
+  }
 
   // Launch programs [lo, hi) of `ready`: one stacked kernel (with in-kernel level waits when they span
   // several levels), or one launch each when they do not fit one parameter block.

@@ -21,6 +21,9 @@ static const int kDefaultCores = 148 * 3;
 static int g_elems_per_thread = 0;
 extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 32) ? v : 0; }
 extern "C" int dvm_get_elems_per_thread(void) { return g_elems_per_thread; }
+static int g_min_resident_ctas = 0;
+extern "C" void dvm_set_min_resident_ctas(int n) { g_min_resident_ctas = (n == 2) ? 2 : 0; }
+extern "C" int dvm_get_min_resident_ctas(void) { return g_min_resident_ctas; }
 extern "C" void dvm_set_num_cores(int n) { g_num_cores = n > 0 ? n : 0; }
 extern "C" int dvm_get_num_cores(void) { return g_num_cores > 0 ? g_num_cores : kDefaultCores; }
 
@@ -909,117 +912,118 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
     int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
     uint32_t flags, inv_mask;
     uint32_t lreg_table[DVM_MAX_LREGS];
-  } best;
+  } best, tight;  // `tight`: the best geometry among those that leave room for g_min_resident_ctas CTAs per SM
   best.cost = -1;
+  tight.cost = -1;
+  // Local-memory layout of ONE tile slot, in 256-byte units, for a candidate geometry; returns the CTAs per SM
+  // it leaves room for (0: it does not fit at all).  An input register is an image of the tile's rows as they
+  // lie in global memory (a dense operand: one contiguous range; otherwise one image per row, DVM_ROW_PITCH
+  // apart; a row vector shared by every row: one row image, of the tile's column block); a temporary is
+  // thread-private (V fp32 per thread); per-row scalar slots are thread-private.  A CTA holds two slots:
+  // while it computes the tile in one, the next tile (of this or of another stacked program) loads into the
+  // other.
+  auto layout = [&](Geo& g) -> int {
+    g.inv_mask = 0;
+    g.units = 0;
+    const int64_t Gthreads = 1ll << g.log2G;
+    for (int k = 0; k < e.n_in_regs; ++k) {
+      const Operand& od = e.opd[in_opd[k]];
+      const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
+      const bool inv = !flat && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
+      bool dense = od.col_stride == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
+      if (!flat) {
+        if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+        if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+      }
+      const int mode = inv ? DVM_LM_BCAST : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
+      if (inv) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
+      const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
+      const int64_t bytes = inv ? pitch : pitch * (T / Gthreads);
+      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
+      g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
+    }
+    for (int k = e.n_in_regs; k < nreg; ++k) {
+      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)DVM_LM_PRIVATE << 16);
+      g.units += g.V * 4 * T / DVM_LOCAL_UNIT;
+    }
+    g.scalar_unit = g.units;
+    if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
+    if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
+    int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
+    return ctas > 2 ? 2 : ctas;  // the interpreter is compiled for two resident CTAs per SM
+  };
+  // cores the tiles spread over when `ctas` CTAs are resident per SM (the core count is quoted at 3 CTAs per SM)
+  auto cores = [&](int ctas) -> int64_t { return (int64_t)dvm_get_num_cores() * ctas / 3; };
   const int W0 = W;
   for (int vi = 0; vi < 2; ++vi) {
     Geo g;
     g.V = 32 >> vi;
     if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
-    int ctas_guess = 2;
-    bool ok = false;
-    for (int attempt = 0; attempt < 3 && !ok; ++attempt) {
-      const int64_t N = (int64_t)dvm_get_num_cores() * ctas_guess / 3;  // the core count is quoted at 3 CTAs per SM
+    g.W = W0;
+    if (flat) {
+      g.log2G = 8;
+      g.CB = 1;
+      g.Ctile = (int64_t)T * W0;  // the layout of a flat program does not depend on the chunk
+      g.flags = DVM_F_FLAT | DVM_F_ALIGNED;
+      const int ctas = layout(g);
+      if (ctas < 1) continue;
+      const int64_t N = cores(ctas);
+      int64_t total = empty ? 0 : C;  // everything merged into one dim
+      int64_t best_chunk = (int64_t)T * W0;
       g.cost = -1;
-      g.W = W0;
-      if (flat) {
-        int64_t total = empty ? 0 : C;  // everything merged into one dim
-        int64_t best_chunk = (int64_t)T * W0;
-        for (int k = 1; k <= g.V / W0; ++k) {
-          int64_t chunk = (int64_t)T * W0 * k;
-          int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
-          if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
-        }
-        g.Ctile = best_chunk;
-        g.rowsR = cdiv(total, g.Ctile);
-        g.lastRowCols = g.rowsR > 0 ? total - (g.rowsR - 1) * g.Ctile : g.Ctile;
-        g.CB = 1;
-        g.log2G = 8;
-        g.n_tiles = g.rowsR;
-        g.flags = DVM_F_FLAT | DVM_F_ALIGNED;
-      } else {
-        // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
-        bool aligned = primary >= 0;
-        if (primary >= 0)
-          for (int q = 0; q < 3; ++q)
-            if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
-        {
-          const int w = W0;
-          const bool al = aligned;
-          // a misaligned row segment starts up to w - 1 slots into its first chunk: keep that much spare capacity
-          const int64_t pad = al ? 0 : w - 1;
-          for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
-            int64_t G = 1 << lg, cap = G * g.V;
-            int64_t ct;
-            if (has_reduce) {
-              // a whole row per thread group; at the widest group a row may use the full capacity: its last
-              // columns then wrap around into the head slots of a misaligned row
-              if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
-              ct = C;
-            } else {
-              ct = ((cap - pad) / w) * w;
-              if (ct <= 0) continue;
-              if (ct > C) ct = C;
-            }
-            int64_t cb = cdiv(C, ct);
-            int64_t tiles = cdiv(R, T / G) * cb;
-            int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
-            int64_t cost = cdiv(tiles, N) * (u + beta);
-            if (g.cost < 0 || cost < g.cost) {
-              g.cost = cost; g.log2G = lg; g.Ctile = ct; g.CB = cb; g.n_tiles = tiles; g.W = w;
-              g.flags = al ? DVM_F_ALIGNED : 0;
-            }
-          }
-        }
-        if (g.cost < 0) break;  // a reduced row does not fit V elements per thread
-        if (outer[1] > 1 || outer[2] > 1) g.flags |= DVM_F_OUTER_DIMS;
-        g.rowsR = R;
-        g.lastRowCols = C;
-        if (empty) g.n_tiles = 0;
+      for (int k = 1; k <= g.V / W0; ++k) {
+        int64_t chunk = (int64_t)T * W0 * k;
+        int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
+        if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
       }
-      // Local-memory layout of ONE tile slot, in 256-byte units.  An input register is an image of the
-      // tile's rows as they lie in global memory (a dense operand: one contiguous range; otherwise one
-      // image per row, DVM_ROW_PITCH apart; a row vector shared by every row: one row image); a
-      // temporary is thread-private (V fp32 per thread); per-row scalar slots are thread-private.
-      // A CTA holds two slots: while it computes the tile in one, the next tile (of this or of another
-      // stacked program) loads into the other.
-      g.inv_mask = 0;
-      g.units = 0;
-      const int64_t Gthreads = 1ll << g.log2G;
-      for (int k = 0; k < e.n_in_regs; ++k) {
-        const Operand& od = e.opd[in_opd[k]];
-        const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
-        const bool inv = !flat && g.CB == 1 && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
-        bool dense = od.col_stride == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
-        if (!flat) {
-          if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
-          if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
-        }
-        const int mode = inv ? DVM_LM_BCAST : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
-        if (inv) g.inv_mask |= 1u << k;  // the same for every tile: loaded once per slot
-        const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
-        const int64_t bytes = inv ? pitch : pitch * (T / Gthreads);
-        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
-        g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
-      }
-      for (int k = e.n_in_regs; k < nreg; ++k) {
-        g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)DVM_LM_PRIVATE << 16);
-        g.units += g.V * 4 * T / DVM_LOCAL_UNIT;
-      }
-      g.scalar_unit = g.units;
-      if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
-      if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) break;
-      int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
-      if (ctas > 2) ctas = 2;  // the interpreter is compiled for two resident CTAs per SM
-      if (ctas < 1) break;
-      // the geometry was costed for ctas_guess resident CTAs per SM: at least that many must fit
-      // (more is harmless; fewer: cost it again for the smaller number)
-      if (ctas >= ctas_guess) ok = true;
-      else ctas_guess = ctas;
+      g.Ctile = best_chunk;
+      g.rowsR = cdiv(total, g.Ctile);
+      g.lastRowCols = g.rowsR > 0 ? total - (g.rowsR - 1) * g.Ctile : g.Ctile;
+      g.n_tiles = g.rowsR;
+      layout(g);  // dense operands are recognised by the final chunk
+      if (best.cost < 0 || g.cost < best.cost) best = g;
+      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
+      continue;
     }
-    if (!ok) continue;
-    if (best.cost < 0 || g.cost < best.cost) best = g;
+    // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
+    bool aligned = primary >= 0;
+    if (primary >= 0)
+      for (int q = 0; q < 3; ++q)
+        if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
+    const int w = W0;
+    // a misaligned row segment starts up to w - 1 slots into its first chunk: keep that much spare capacity
+    const int64_t pad = aligned ? 0 : w - 1;
+    g.flags = (aligned ? DVM_F_ALIGNED : 0) | ((outer[1] > 1 || outer[2] > 1) ? DVM_F_OUTER_DIMS : 0);
+    g.rowsR = R;
+    g.lastRowCols = C;
+    for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
+      int64_t G = 1 << lg, cap = G * g.V;
+      int64_t ct;
+      if (has_reduce) {
+        // a whole row per thread group; at the widest group a row may use the full capacity: its last
+        // columns then wrap around into the head slots of a misaligned row
+        if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
+        ct = C;
+      } else {
+        ct = ((cap - pad) / w) * w;
+        if (ct <= 0) continue;
+        if (ct > C) ct = C;
+      }
+      g.log2G = lg;
+      g.Ctile = ct;
+      g.CB = cdiv(C, ct);
+      g.n_tiles = cdiv(R, T / G) * g.CB;
+      // the local-memory need of this geometry decides how many CTAs are resident at once
+      const int ctas = layout(g);
+      if (ctas < 1) continue;
+      int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
+      g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta);
+      if (empty) g.n_tiles = 0;
+      if (best.cost < 0 || g.cost < best.cost) best = g;
+      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
+    }
   }
+  if (tight.cost >= 0) best = tight;  // otherwise no geometry leaves that room: the unconstrained best stands
   if (best.cost < 0) return DVM_ERR_UNSUPPORTED;  // row longer than the register budget, or too much local memory
   const int log2G = best.log2G;
   W = best.W;

@@ -328,8 +328,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             n_el = (unsigned long long)c.ncols;
             dst += (uint32_t)(tid >> c.lgG) * DVM_ROW_PITCH(1 << c.lgG, V, 1u << lg_es);
           }
-        } else {  // DVM_LM_BCAST: the same row for every tile of the program
-          if (first_of_program && tid == 0) {
+        } else {  // DVM_LM_BCAST: the same row for every tile of the program's column block
+          if ((first_of_program || CW(prog + DVM_H_COL_BLOCKS) > 1) && tid == 0) {
             mine = true;
             a = c.col0;
             n_el = min(CW(prog + DVM_H_COLS) - c.col0, CW(prog + DVM_H_COL_TILE));

@@ -108,3 +108,29 @@ def test_stacked_equals_separate_launches():
     torch.cuda.synchronize()
     for a, t in zip(stacked, tls):
         assert torch.equal(a, t[-1])
+
+
+@pytest.mark.parametrize("v", [16, 32])
+def test_stacked_with_two_resident_ctas_per_sm(v):
+    """dvm_set_min_resident_ctas(2): every program's tile slots fit twice per SM; wide rows with row-vector
+    operands then run in two or more column blocks, whose slice of the row vector is loaded with every tile."""
+    dvm.set_elems_per_thread(v)
+    dvm.set_min_resident_ctas(2)
+    try:
+        items = [("gelu_affine", 337, 3249), ("gelu_affine", 148, 2893), ("gelu_affine", 5, 4096), ("layernorm", 64, 4096),
+                 ("sigmoid_mul", 511, 4095), ("gelu_affine", 40, 2049), ("gelu_affine", 3, 65), ("layernorm", 17, 100)]
+        codes, tls, meta = _stack(items, 321)
+        for c in codes:
+            words = torch.frombuffer(bytearray(c.bytes()), dtype=torch.int32)
+            units = (int(words[19]) >> 16) & 0xffff          # local-memory units of one tile slot
+            assert units <= 225 or v == 32                   # (at 32 elements per thread not every program can)
+        dvm.launch_stacked(codes, tls)
+        assert dvm.last_device_status() == 0
+        _check_all(meta)
+        for c, t in zip(codes, tls):                         # and each program on its own
+            t[-1].fill_(float("nan"))
+            dvm.launch(c, t)
+        assert dvm.last_device_status() == 0
+        _check_all(meta)
+    finally:
+        dvm.set_min_resident_ctas(0)

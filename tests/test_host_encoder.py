@@ -217,3 +217,20 @@ def test_stacked_levels_rejects_decreasing_levels_before_any_launch():
     with pytest.raises(dvm.DvmError) as ei:
         dvm.launch_stacked(codes, fake, levels=[1, 0])
     assert ei.value.status == -1   # DVM_ERR_INVALID_ARG
+
+
+def test_min_resident_ctas_picks_a_geometry_that_fits_twice_per_sm():
+    """A wide GELU(x*w+b) row at 16 elements per thread: unconstrained, one row per tile with whole-row images
+    of w and b (259 units per slot: one CTA per SM); with dvm_set_min_resident_ctas(2), two column blocks."""
+    p = dvm.program_from_nodes(wl.stack_program("gelu_affine").nodes)
+    shapes = [(148, 2893), (1, 2893), (1, 2893)]
+    dvm.set_elems_per_thread(16)
+    try:
+        free = dvm.disassemble(dvm.encode(p, shapes))
+        dvm.set_min_resident_ctas(2)
+        tight = dvm.disassemble(dvm.encode(p, shapes))
+    finally:
+        dvm.set_min_resident_ctas(0)
+        dvm.set_elems_per_thread(0)
+    assert "local_units=259" in free and "col_blocks=1 " in free
+    assert "local_units=195" in tight and "col_blocks=2 " in tight and "threads_per_row=128" in tight
