@@ -25,6 +25,9 @@ Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
   Broadcast                implicit in numpy-style broadcasting (Table 1, Broadcast)
   Cmp                      1.0 where the relation holds, else 0.0  (Table 1, Cmp)
   Select                   cond != 0 ? x : y                       (Table 1, Select)
+  ViewLoad / ViewStore     element (i_0..i_{d-1}) of a view lies at          (Table 1, ViewLoad / ViewStore:
+                           base + sum_k i_k * stride_k of its storage        non-contiguous tiles, per-dim strides)
+                           (view_load / view_store below; evaluate() itself sees logical arrays only)
 Extensions that the benchmark programs need and Table 1 lacks (stated as such
 in DESIGN.md): erf, sigmoid(x) = 1/(1+exp(-x)), rsqrt(x) = 1/sqrt(x),
 recip, neg, tanh, and matmul C[i,j] = sum_k A[i,k] B[k,j] (the paper's cube
@@ -173,3 +176,39 @@ def evaluate(nodes, inputs, params=()):
             else:
                 raise ValueError(f"unknown node kind {kind}")
     return outs
+
+
+def _view_index(offset, shape, strides):
+    """Flat storage index of every element of a view: offset + sum_k i_k * stride_k (Table 1, ViewLoad)."""
+    shape = tuple(int(d) for d in shape)
+    strides = tuple(int(t) for t in strides)
+    if len(shape) != len(strides):
+        raise ValueError("one stride per dim")
+    idx = np.full(shape, int(offset), dtype=np.int64)
+    for k, (d, t) in enumerate(zip(shape, strides)):
+        ik = np.arange(d, dtype=np.int64).reshape([d if j == k else 1 for j in range(len(shape))])
+        idx = idx + ik * t
+    return idx
+
+
+def view_load(storage: np.ndarray, offset: int, shape, strides) -> np.ndarray:
+    """ViewLoad (Table 1): the logical array a strided view denotes.  `storage` is the flat buffer, `offset`
+    and `strides` are in elements; a stride of 0 repeats the element (broadcast)."""
+    flat = np.asarray(storage).reshape(-1)
+    idx = _view_index(offset, shape, strides)
+    if idx.size and (idx.min() < 0 or idx.max() >= flat.size):
+        raise IndexError("view reaches outside its storage")
+    return flat[idx]
+
+
+def view_store(storage: np.ndarray, offset: int, shape, strides, values: np.ndarray) -> np.ndarray:
+    """ViewStore (Table 1): a copy of `storage` with the view's elements replaced by `values`; every other
+    element keeps its value.  The view must not alias itself (two index tuples, one address)."""
+    flat = np.array(storage, copy=True).reshape(-1)
+    idx = _view_index(offset, shape, strides)
+    if idx.size and (idx.min() < 0 or idx.max() >= flat.size):
+        raise IndexError("view reaches outside its storage")
+    if np.unique(idx).size != idx.size:
+        raise ValueError("a stored view must address every element once")
+    flat[idx.reshape(-1)] = np.asarray(values).reshape(-1)
+    return flat.reshape(np.asarray(storage).shape)

@@ -423,3 +423,41 @@ def test_if_else_add_closed_form():
     want = np.where(a > b, 2.0 * x, 4.0 * x) + y
     assert np.array_equal(got, want)
     assert np.array_equal(got[0, 0, :3], 4.0 * x[0, 0, :3] + y[0, 0, :3])
+
+
+# ---------------------------------------------------------------- views (Table 1, ViewLoad / ViewStore)
+def test_view_load_against_library_views_and_brute_force():
+    """view_load is pinned by numpy's own transposes, slices and broadcasts (another mechanism: numpy's
+    stride machinery) and by an explicit loop over index tuples on a tiny case."""
+    base = RNG.standard_normal((4, 6, 10))
+    flat = base.reshape(-1)
+    es = base.itemsize
+    for v in (base.transpose(1, 0, 2), base[:, 1:5, 2:9], base[::2, :, ::3], base.transpose(2, 0, 1)[3:, 1:],
+              np.broadcast_to(base[:, :1, :], (4, 6, 10)), base[1]):
+        off = (v.__array_interface__["data"][0] - base.__array_interface__["data"][0]) // es
+        got = orc.view_load(flat, off, v.shape, [t // es for t in v.strides])
+        assert np.array_equal(got, v)
+    shape, strides, off = (2, 3, 2), (7, 2, 30), 5
+    got = orc.view_load(flat, off, shape, strides)
+    for i in range(2):
+        for j in range(3):
+            for k in range(2):
+                assert got[i, j, k] == flat[off + 7 * i + 2 * j + 30 * k]
+    with pytest.raises(IndexError):
+        orc.view_load(flat, 0, (5, 100), (60, 1))
+
+
+def test_view_store_writes_the_view_and_nothing_else():
+    storage = np.arange(240, dtype=np.float64).reshape(4, 60)
+    vals = -1.0 - RNG.random((3, 5, 2))
+    out = orc.view_store(storage, 7, (3, 5, 2), (60, 4, 1), vals)
+    want = storage.copy().reshape(-1)
+    for i in range(3):
+        for j in range(5):
+            for k in range(2):
+                want[7 + 60 * i + 4 * j + k] = vals[i, j, k]
+    assert np.array_equal(out.reshape(-1), want) and out.shape == storage.shape
+    assert np.array_equal(storage, np.arange(240, dtype=np.float64).reshape(4, 60))  # the input is not modified
+    assert np.array_equal(orc.view_load(out, 7, (3, 5, 2), (60, 4, 1)), vals)       # load after store returns the values
+    with pytest.raises(ValueError):
+        orc.view_store(storage, 0, (3, 4), (2, 1), np.zeros((3, 4)))                # rows overlap: aliasing
