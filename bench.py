@@ -686,8 +686,79 @@ class IfElseWorkload:
         return k * 20 * n / t_all / 1e9, t_all, f"{k} evaluations of a [1,512,8192] instance, numpy float64"
 
 
-WORKLOADS = {"ifelse": IfElseWorkload, "addmm": AddmmWorkload, "c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
-for _W in (C1Workload, C2Workload, C3Workload, C4Workload, IfElseWorkload):   # the memory-bound sweeps: work = algorithmic bytes
+class ViewsWorkload:
+    """Views (Table 1, ViewLoad): out = 0.5 * x + y on bf16 [B,32,S,128], x read through a head-transpose view of
+    storage laid out [B,S,32,128], dynamic (B, S) instances."""
+    name = "views"
+    H, D = 32, 128
+
+    def __init__(self, dvm, n_instances=60, device="cuda"):
+        self.dvm = dvm
+        self.prog = wl.program_head_transpose_add()
+        self.p = dvm.program_from_nodes(self.prog.nodes)
+        self.enc = dvm.binding.Encoder(self.p)
+        self.shapes = wl.shapes_views(n_instances, self.H, self.D)
+        self.elems = [b * s_ * self.H * self.D for b, s_ in self.shapes]
+        self.pool = max(self.elems)
+        seed = wl.data_seed("views", 0)
+        self.ins = [wl.randn((self.pool,), torch.bfloat16, seed + i, device) for i in range(2)]
+        self.out = torch.empty((self.pool,), dtype=torch.bfloat16, device=device)
+        self.bytes_per_instance = [6 * n for n in self.elems]   # two bf16 reads, one bf16 write per element
+        self.total_bytes = sum(self.bytes_per_instance)
+        self.description = ("views: out = 0.5*x + y, bf16 [B,32,S,128], x a head-transpose VIEW of [B,S,32,128] storage "
+                            f"(rows of 128 elements, 256 B apart in groups), B 1..32, S 1..8192, {n_instances} dynamic "
+                            "instances, each re-encoded per launch (dvm_encode_strided)")
+        self.l2_policy = "mean instance 0.7 GB over three tensors, far above L2"
+
+    def _strides(self, b, s_):
+        H, D = self.H, self.D
+        return [[s_ * H * D, D, H * D, 1], None]   # element (b,h,s,d) of x lies at ((b*S + s)*H + h)*D + d
+
+    def run_step(self, stream, events=None, enc_ns=None):
+        import ctypes as C
+        lib_launch = self.dvm.binding.lib.dvm_launch
+        arr = (C.c_void_p * 3)(*[t.data_ptr() for t in self.ins], self.out.data_ptr())
+        for b, s_ in self.shapes:
+            shp = (b, self.H, s_, self.D)
+            t0 = time.perf_counter_ns()
+            size = self.enc.encode((shp, shp), (), self._strides(b, s_))
+            t1 = time.perf_counter_ns()
+            if enc_ns is not None:
+                enc_ns.append(t1 - t0)
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st = lib_launch(self.enc.buf, size, arr, 3, stream.cuda_stream)
+            if st != 0:
+                raise self.dvm.DvmError(st, "dvm_launch")
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+        return len(self.shapes)
+
+    def setup_e2e(self):
+        self.staging = None
+
+    def run_step_e2e(self, stream):
+        return None
+
+    def oracle_sample(self, budget_s=12.0):
+        from oracle import dvm_oracle as orc
+        B, S = 2, 512
+        n = B * S * self.H * self.D
+        x = wl.to_f64(self.ins[0][:n])
+        y = wl.to_f64(self.ins[1][:n]).reshape(B, self.H, S, self.D)
+        t_all, k = 0.0, 0
+        while t_all < budget_s:
+            t0 = time.perf_counter()
+            xv = orc.view_load(x, 0, (B, self.H, S, self.D), (S * self.H * self.D, self.D, self.H * self.D, 1))
+            orc.evaluate(self.prog.nodes, [xv, y])
+            t_all += time.perf_counter() - t0; k += 1
+        return k * 6 * n / t_all / 1e9, t_all, f"{k} evaluations of a [2,32,512,128] instance (view_load + program), numpy float64"
+
+
+WORKLOADS = {"views": ViewsWorkload, "ifelse": IfElseWorkload, "addmm": AddmmWorkload, "c1": C1Workload, "c2": C2Workload, "c3": C3Workload, "c4": C4Workload, "c5": C5Workload}
+for _W in (C1Workload, C2Workload, C3Workload, C4Workload, IfElseWorkload, ViewsWorkload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
 
@@ -727,6 +798,15 @@ def run_reference(args):
         nbytes = 20 * 512 * 8192
         sample = "one [1,512,8192] instance per step, numpy float64"
         desc = IfElseWorkload.__doc__
+        params = ()
+    elif args.workload == "views":
+        prog = wl.program_head_transpose_add()
+        B, S, H, D = 2, 512, 32, 128
+        xs = wl.to_f64(wl.randn((B * S * H * D,), torch.bfloat16, 1))
+        ins = [orc.view_load(xs, 0, (B, H, S, D), (S * H * D, D, H * D, 1)), wl.to_f64(wl.randn((B, H, S, D), torch.bfloat16, 2))]
+        nbytes = 6 * B * S * H * D
+        sample = "one [2,32,512,128] instance per step (program on the loaded view), numpy float64"
+        desc = ViewsWorkload.__doc__
         params = ()
     elif args.workload == "addmm":
         prog = wl.program_addmm()
@@ -788,6 +868,15 @@ def run_reference(args):
 
 def encode_latency(W, reps):
     """Host encode latency over `reps` repeats of each of (up to) 20 instances of the sweep: pure dvm_encode calls."""
+    if W.name == "views":
+        ns = []
+        for b, s_ in W.shapes[:20]:
+            shp = (b, W.H, s_, W.D)
+            for _ in range(reps):
+                t0 = time.perf_counter_ns(); W.enc.encode((shp, shp), (), W._strides(b, s_)); ns.append(time.perf_counter_ns() - t0)
+        us = sorted(x / 1e3 for x in ns)
+        return {"mean": sum(us) / len(us), "p50": us[len(us) // 2], "p99": us[int(0.99 * len(us))], "max": us[-1],
+                "n": len(us), "note": f"{reps} repeats of each of 20 instances, perf_counter around the binding's dvm_encode_strided call"}
     if W.name == "ifelse":
         shapes = [(shp,) * 4 for shp in W.shapes[:20]]
     elif W.name == "addmm":

@@ -207,6 +207,27 @@ def program_if_else_add() -> OpProgram:
     return p
 
 
+def program_head_transpose_add() -> OpProgram:
+    """out[b,h,s,:] = 0.5 * x[b,h,s,:] + y[b,h,s,:], bf16 rank 4: the elementwise consumer of an attention head
+    transpose.  x is given as a VIEW (stored [B,S,H,D], read as [B,H,S,D]: Table 1, ViewLoad); y, out dense."""
+    p = OpProgram("head_transpose_add")
+    x, y = p.input("bf16", 4), p.input("bf16", 4)
+    p.output(p.binary("add", p.scalar("muls", x, 0.5), y), "bf16")
+    return p
+
+
+def shapes_views(n: int = 60, H: int = 32, D: int = 128, max_tokens: int = 1 << 17) -> List[Tuple[int, int]]:
+    """(B, S) per instance: B ~ U{1..32}, S ~ U{1..8192}, redrawn while B*S exceeds max_tokens (the tensors are
+    [B,32,S,128] bf16: 8 KB per token)."""
+    rng = np.random.default_rng(CFG_SEED["views"])
+    out = []
+    while len(out) < n:
+        b, s_ = int(rng.integers(1, 32, endpoint=True)), int(rng.integers(1, 8192, endpoint=True))
+        if b * s_ <= max_tokens:
+            out.append((b, s_))
+    return out
+
+
 def program_matmul() -> OpProgram:
     """out = A @ B, bf16 in, fp32 accumulate, bf16 out (Table 2, matmul)."""
     p = OpProgram("matmul")
@@ -244,7 +265,7 @@ def stack_program(kind: str) -> OpProgram:
 # --------------------------------------------------------------------------
 # Seeds, shape samplers
 # --------------------------------------------------------------------------
-CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "addmm": 5, "ifelse": 6}
+CFG_SEED = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "addmm": 5, "ifelse": 6, "views": 7}
 
 # (n, k) pairs "extracted from common LLMs" of the paper's matmul / addmm experiments (Table 2)
 LLM_NK = ((4096, 4096), (11008, 4096), (4096, 11008), (5120, 5120), (13696, 5120), (5120, 13696),

@@ -127,6 +127,26 @@ int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
                const float* scalars, int n_scalars,
                void* code, size_t code_capacity, size_t* code_size,
                dvm_shape* out_shapes, int n_out);
+/* dvm_encode on VIEWS (Table 1, ViewLoad / ViewStore: non-contiguous tiles described by per-dim strides).
+ * in_strides[i] (one per input, or in_strides == NULL: all dense) gives the element stride of every dim of
+ * in_shapes[i]: element (i_0 .. i_{r-1}) of input i lies at tensors[i] + sum_k i_k * stride[k] elements, so
+ * the tensor pointer passed at launch is the address of the view's first element.  out_strides[o] (one per
+ * output, or NULL) does the same for output o over the dims out_shapes[o] reports.  Strides of dims of size
+ * 1 are ignored; a stride of 0 on an input dim repeats the element (an expanded view).
+ *  - DVM_ERR_INVALID_ARG: a negative stride; an output view that addresses an element twice (a zero stride,
+ *    or dims that overlap).
+ *  - DVM_ERR_UNSUPPORTED: a view whose last dim is not adjacent in memory (stride of the last dim != 1:
+ *    rows, and every outer dim, may lie anywhere -- slices, permuted outer dims, padded rows -- but a row's
+ *    elements are copied as one byte range); more than three outer dims left after adjacent dims that are
+ *    dense in every operand were merged; a program with a matmul.
+ * Everything else as dvm_encode. */
+typedef struct {
+  int64_t stride[DVM_MAX_RANK]; /* elements; entry k belongs to dim k of the shape */
+} dvm_strides;
+int dvm_encode_strided(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                       const float* scalars, int n_scalars, const dvm_strides* out_strides,
+                       void* code, size_t code_capacity, size_t* code_size,
+                       dvm_shape* out_shapes, int n_out);
 /* dvm_encode for n independent instances in one call -- the stacked-fusion case (Sec. 5.1), where every
  * program of a launch is re-encoded per launch.  All arrays are host memory of length n, except
  * in_shapes / scalars, which concatenate the instances' arguments (instance i consumes n_in[i] shapes and

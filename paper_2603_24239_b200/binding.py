@@ -35,6 +35,10 @@ class Shape(C.Structure):
     _fields_ = [("rank", C.c_int32), ("dims", C.c_int64 * DVM_MAX_RANK)]
 
 
+class Strides(C.Structure):
+    _fields_ = [("stride", C.c_int64 * DVM_MAX_RANK)]
+
+
 class DvmError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -66,6 +70,8 @@ _sig = {
     "dvm_program_num_outputs": ([_vp], _i),
     "dvm_encode": ([_vp, C.POINTER(Shape), _i, C.POINTER(C.c_float), _i, _vp, _sz, C.POINTER(_sz),
                     C.POINTER(Shape), _i], _i),
+    "dvm_encode_strided": ([_vp, C.POINTER(Shape), C.POINTER(Strides), _i, C.POINTER(C.c_float), _i, C.POINTER(Strides),
+                            _vp, _sz, C.POINTER(_sz), C.POINTER(Shape), _i], _i),
     "dvm_encode_batch": ([_i, C.POINTER(_vp), C.POINTER(Shape), _pi, C.POINTER(C.c_float), _pi, C.POINTER(_vp),
                           C.POINTER(_sz), C.POINTER(_sz), _pi], _i),
     "dvm_code_max_size": ([_vp], _sz),
@@ -240,17 +246,45 @@ class Encoder:
         self.size = _sz(0)
         self.scalars = (C.c_float * 16)()
 
-    def encode(self, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = ()) -> int:
+    def encode(self, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = (),
+               in_strides: Optional[Sequence[Optional[Sequence[int]]]] = None,
+               out_strides: Optional[Sequence[Optional[Sequence[int]]]] = None) -> int:
+        """in_strides / out_strides (element strides per dim, None = dense) select dvm_encode_strided."""
         for s, shp in zip(self.shapes, shapes):
             s.rank = len(shp)
             for k, d in enumerate(shp):
                 s.dims[k] = d
         for k, v in enumerate(scalars):
             self.scalars[k] = v
-        st = lib.dvm_encode(self.program._h, self.shapes, self.n_in, self.scalars, len(scalars),
-                            self.buf, self.cap, C.byref(self.size), self.out_shapes, self.n_out)
+        if in_strides is None and out_strides is None:
+            st = lib.dvm_encode(self.program._h, self.shapes, self.n_in, self.scalars, len(scalars),
+                                self.buf, self.cap, C.byref(self.size), self.out_shapes, self.n_out)
+            if st != 0:
+                raise DvmError(st, "dvm_encode")
+            return self.size.value
+        if out_strides is not None and any(t is None for t in out_strides):
+            # a dense output among views: its strides follow from the output shape, which a plain encode reports
+            st = lib.dvm_encode(self.program._h, self.shapes, self.n_in, self.scalars, len(scalars),
+                                self.buf, self.cap, C.byref(self.size), self.out_shapes, self.n_out)
+            if st != 0:
+                raise DvmError(st, "dvm_encode")
+            out_strides = [t if t is not None else _dense_strides(shp) for t, shp in zip(out_strides, self.output_shapes())]
+        ins = None
+        if in_strides is not None:
+            ins = (Strides * self.n_in)()
+            for a, t, shp in zip(ins, in_strides, shapes):
+                for k, v in enumerate(t if t is not None else _dense_strides(shp)):
+                    a.stride[k] = v
+        outs = None
+        if out_strides is not None:
+            outs = (Strides * max(self.n_out, 1))()
+            for a, t in zip(outs, out_strides):
+                for k, v in enumerate(t):
+                    a.stride[k] = v
+        st = lib.dvm_encode_strided(self.program._h, self.shapes, ins, self.n_in, self.scalars, len(scalars), outs,
+                                    self.buf, self.cap, C.byref(self.size), self.out_shapes, self.n_out)
         if st != 0:
-            raise DvmError(st, "dvm_encode")
+            raise DvmError(st, "dvm_encode_strided")
         return self.size.value
 
     def output_shapes(self) -> List[tuple]:
@@ -305,10 +339,20 @@ class BatchEncoder:
             raise DvmError(st, f"dvm_encode_batch (instance {self.failed.value})")
 
 
-def encode(program: Program, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = ()) -> Code:
-    """dvm_encode: one dynamic-shape instance -> bytecode."""
+def _dense_strides(shape: Sequence[int]) -> List[int]:
+    out, st = [], 1
+    for d in reversed(list(shape)):
+        out.append(st)
+        st *= max(int(d), 1)
+    return out[::-1]
+
+
+def encode(program: Program, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = (),
+           in_strides=None, out_strides=None) -> Code:
+    """dvm_encode: one dynamic-shape instance -> bytecode.  With in_strides / out_strides (element strides per
+    dim of each input / output view; None entries are dense): dvm_encode_strided."""
     enc = Encoder(program)
-    size = enc.encode(shapes, scalars)
+    size = enc.encode(shapes, scalars, in_strides, out_strides)
     return Code(enc.buf, size, enc.output_shapes())
 
 

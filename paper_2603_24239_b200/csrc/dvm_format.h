@@ -59,7 +59,7 @@ enum {
   DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
   DVM_F_FLAT = 4,       // pure elementwise program laid out as a flat range
   DVM_F_PRIMARY_DENSE = 8, // the primary operand is dense: row r starts at element r * C of its tensor
-  DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select: it needs the extended interpreter variant
+  DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select or stores a tile into a strided view: it needs the extended interpreter variant
   DVM_F_LOADS_BY_ROW = 16  // some load is issued per row (row-by-row images, per-row scalars); otherwise
                            // thread 0 alone issues every copy of a tile
 };
@@ -70,8 +70,9 @@ enum {
   DVM_LM_PRIVATE = 0,  // temporary: thread-private fp32 vectors, vector q of thread tid at (q * 256 + tid) * 16
   DVM_LM_BLOCK = 1,    // input whose tile is one contiguous byte range of global memory: one bulk copy per tile
   DVM_LM_ROWS = 2,     // input copied row by row (one bulk copy per row): row images DVM_ROW_PITCH(...) apart
-  DVM_LM_BCAST = 3     // row-vector input, the same for every row: one row image per slot (of the tile's column block;
-                       // with one column block it is loaded once per slot and program, else with every tile)
+  DVM_LM_BCAST = 3,    // row-vector input, the same for every row and tile: one row image per slot, loaded once per
+                       // slot and program
+  DVM_LM_BCAST_TILE = 4  // the same with several column blocks: the image holds the tile's column block, loaded with every tile
 };
 // bytes between the row images of a ROWS register (room for the 16-byte alignment slack on both sides)
 #define DVM_ROW_PITCH(G, V, es) ((uint32_t)(G) * (uint32_t)(V) * (uint32_t)(es) + 32u)

@@ -7,6 +7,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <utility>
+
 #include "../../include/dvm.h"
 #include "dvm_format.h"
 #include "dvm_internal.h"
@@ -713,18 +715,22 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
                       int n_scalars, void* code, size_t code_capacity, size_t* code_size,
                       dvm_shape* out_shapes, int n_out);
 
-extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
-                          const float* scalars, int n_scalars, void* code, size_t code_capacity,
-                          size_t* code_size, dvm_shape* out_shapes, int n_out) {
+// in_strides / out_strides (each may be NULL: dense row-major): element strides of the views (ViewLoad /
+// ViewStore, Table 1), one entry per input / output.
+static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                        const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
+                        size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out) {
   if (!p || !in_shapes || !code_size) return DVM_ERR_INVALID_ARG;
   if (!p->finalized) return DVM_ERR_NOT_FINALIZED;
   if (n_in != p->n_inputs) return DVM_ERR_INVALID_ARG;
   if (n_scalars < p->n_params || (p->n_params > 0 && !scalars)) return DVM_ERR_INVALID_ARG;
   if (out_shapes && n_out < p->n_outputs) return DVM_ERR_INVALID_ARG;
   if (((uintptr_t)code & 7) != 0) return DVM_ERR_INVALID_ARG;
-  if (p->n_matmul > 0)
+  if (p->n_matmul > 0) {
+    if (in_strides || out_strides) return DVM_ERR_UNSUPPORTED;  // the matmul's tensor maps describe dense matrices
     return dvm_encode_matmul(p, in_shapes, n_in, scalars, n_scalars, code, code_capacity, code_size,
                              out_shapes, n_out);
+  }
 
   Enc e;
   e.p = p;
@@ -828,6 +834,33 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
       st *= dk;
     }
     od.col_stride = (e.dims[v][Dt - 1] == 1 && Ccols > 1) ? 0 : 1;
+    const dvm_strides* us = i < n_in ? (in_strides ? &in_strides[i] : nullptr) : (out_strides ? &out_strides[i - n_in] : nullptr);
+    if (us) {
+      // a view: the caller's element strides replace the dense ones (dims of size 1 carry no stride)
+      const int r = i < n_in ? in_shapes[i].rank : D;  // an output has the dominant rank
+      for (int k = 0; k < D; ++k) {
+        const int64_t dk = e.dims[v][k];
+        const int uk = k - (D - r);
+        if (dk == 1 || uk < 0) continue;
+        const int64_t t = us->stride[uk];
+        if (t < 0) return DVM_ERR_INVALID_ARG;
+        if (i >= n_in && t == 0) return DVM_ERR_INVALID_ARG;  // a stored view addresses every element once
+        od.stride[k] = t;
+      }
+      if (e.dims[v][Dt - 1] != 1 && od.stride[Dt - 1] != 1)
+        return DVM_ERR_UNSUPPORTED;  // elements of a row must be adjacent in memory (rows and outer dims may lie anywhere)
+      if (i >= n_in) {
+        // no two index tuples at one address: sorted by stride, each dim must step over the one before it
+        int64_t sz[DVM_MAX_RANK], sd[DVM_MAX_RANK];
+        int m = 0;
+        for (int k = 0; k < D; ++k)
+          if (e.dims[v][k] > 1) { sz[m] = e.dims[v][k]; sd[m] = od.stride[k]; ++m; }
+        for (int a = 1; a < m; ++a)
+          for (int b = a; b > 0 && sd[b] < sd[b - 1]; --b) { std::swap(sd[b], sd[b - 1]); std::swap(sz[b], sz[b - 1]); }
+        for (int a = 1; a < m; ++a)
+          if (sd[a] < sd[a - 1] * sz[a - 1]) return DVM_ERR_INVALID_ARG;
+      }
+    }
     if (i >= n_in) {
       // an output must cover the dominant shape (or be one value per row); otherwise several
       // tiles would write the same element
@@ -935,7 +968,7 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
         if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
         if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
       }
-      const int mode = inv ? DVM_LM_BCAST : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
+      const int mode = inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
       if (inv) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
       const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
       const int64_t bytes = inv ? pitch : pitch * (T / Gthreads);
@@ -1055,6 +1088,8 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
   if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
   for (int i = 0; i < NN; ++i)
     if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;
+  for (int o = 0; o < p->n_outputs; ++o)  // a tile stored into a view whose rows are not one dense range: ViewStore
+    if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_EXT_ISA;
   for (int k = 0; k < e.n_in_regs; ++k)
     if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
 
@@ -1111,6 +1146,21 @@ extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int 
     for (int q = 0; q < 3; ++q)
       if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
   return DVM_OK;
+}
+
+extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
+                          const float* scalars, int n_scalars, void* code, size_t code_capacity,
+                          size_t* code_size, dvm_shape* out_shapes, int n_out) {
+  return encode_views(p, in_shapes, nullptr, n_in, scalars, n_scalars, nullptr, code, code_capacity, code_size,
+                      out_shapes, n_out);
+}
+
+extern "C" int dvm_encode_strided(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides,
+                                  int n_in, const float* scalars, int n_scalars, const dvm_strides* out_strides,
+                                  void* code, size_t code_capacity, size_t* code_size, dvm_shape* out_shapes,
+                                  int n_out) {
+  return encode_views(p, in_shapes, in_strides, n_in, scalars, n_scalars, out_strides, code, code_capacity,
+                      code_size, out_shapes, n_out);
 }
 
 extern "C" int dvm_encode_batch(int n, const dvm_program* const* programs, const dvm_shape* in_shapes, const int* n_in,
@@ -1195,10 +1245,11 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       if (mode != DVM_LM_PRIVATE || dt != DVM_DT_F32) return false;
       need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
     } else {
-      if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST || od >= n_opd) return false;
+      if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST_TILE || od >= n_opd) return false;
+      if (mode == DVM_LM_BCAST && w[DVM_H_COL_BLOCKS] > 1) return false;  // a once-per-program image holds whole rows
       if (((otab[od * DVM_OPD_WORDS] >> 8) & 0xff) != dt) return false;
       const uint64_t pitch = DVM_ROW_PITCH(1u << lg, Vv, dt == DVM_DT_BF16 ? 2 : 4);
-      const uint64_t bytes = mode == DVM_LM_BCAST ? pitch : pitch * (DVM_VM_THREADS >> lg);
+      const uint64_t bytes = mode >= DVM_LM_BCAST ? pitch : pitch * (DVM_VM_THREADS >> lg);
       need = (bytes + DVM_LOCAL_UNIT - 1) / DVM_LOCAL_UNIT;
     }
     return unit + need <= units;

@@ -147,8 +147,8 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
 
 // SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
-// EXT: the variant that also decodes Cmp / Select (launched when a program uses them: DVM_F_EXT_ISA); the
-// basic variant stays as compact as it is without them.
+// EXT: the variant that also decodes Cmp / Select and stores tiles into strided views (launched when a program
+// uses them: DVM_F_EXT_ISA); the basic variant stays as compact as it is without them.
 // LEVELS: the stacked variant with in-kernel waits between dependent levels (dvm_launch_stacked_levels).
 template <int V, int PW, bool SINGLE, bool EXT, bool LEVELS = false>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
@@ -328,8 +328,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             n_el = (unsigned long long)c.ncols;
             dst += (uint32_t)(tid >> c.lgG) * DVM_ROW_PITCH(1 << c.lgG, V, 1u << lg_es);
           }
-        } else {  // DVM_LM_BCAST: the same row for every tile of the program's column block
-          if ((first_of_program || CW(prog + DVM_H_COL_BLOCKS) > 1) && tid == 0) {
+        } else {  // DVM_LM_BCAST: the same row for every tile of the program; DVM_LM_BCAST_TILE: of its column block
+          if ((first_of_program || mode == DVM_LM_BCAST_TILE) && tid == 0) {
             mine = true;
             a = c.col0;
             n_el = min(CW(prog + DVM_H_COLS) - c.col0, CW(prog + DVM_H_COL_TILE));
@@ -776,12 +776,17 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                                (w >> 2) * PSTRIDE + (w & 3) * 4));
             s_S[ia][tid] = c.ncols > 0 ? v : 0.f;
           } else if (op == DVM_OP_STG) {
-            // an output covers the dominant shape: element (row, col) lies at row * C + col
+            // an output covers the dominant shape: element (row, col) of a dense one lies at row * C + col,
+            // the rows of a view (Table 1, ViewStore) lie where its strides put them
             const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
-            const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
+            const uint32_t info = CW(d + DVM_OPD_INFO);
+            const int dt = (info >> 8) & 0xff;
             const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
-            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) +
-                                              (((unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0) << lg_es));
+            unsigned long long el0 = (unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0;
+            if constexpr (EXT) {  // programs with a strided output run the extended variant (DVM_F_EXT_ISA)
+              if (!((info >> 25) & 1u)) el0 = row_offset(d, c);
+            }
+            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (el0 << lg_es));
             char* q0 = p + ((long long)c.cbase << lg_es);
             const long long qstep = (long long)((G << c.lgW) << lg_es);
             const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;

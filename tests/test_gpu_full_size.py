@@ -66,3 +66,29 @@ def test_masked_softmax_max_size_sampled(B, S):
         q = int(idx[r] % S)
         assert np.all(got[r][q + 1:] == 0)           # masked entries exactly zero
     assert not torch.isnan(out.float().sum())
+
+
+@pytest.mark.parametrize("B,S", [(16, 7640), (31, 3943)])
+def test_head_transpose_view_full_size_sampled(B, S):
+    """The views sweep at its largest instances (about 0.5 G elements per tensor): x read through the head
+    transpose view; sampled (b, h, s) rows against the oracle's ViewLoad + program, one by one."""
+    H, D = 32, 128
+    n = B * S * H * D
+    xs = wl.randn((n,), torch.bfloat16, 21, "cuda")
+    y = wl.randn((n,), torch.bfloat16, 22, "cuda")
+    out = torch.full((n,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    prog = wl.program_head_transpose_add()
+    shp = (B, H, S, D)
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [shp, shp], in_strides=[[S * H * D, D, H * D, 1], None])
+    dvm.launch(code, [xs, y, out])
+    assert dvm.last_device_status() == 0
+    rows = _sample_rows(B * H * S, 200, 3, extra=[S - 1, S, H * S - 1, H * S])
+    for r in rows:
+        b, h, s_ = int(r // (H * S)), int((r // S) % H), int(r % S)
+        src = ((b * S + s_) * H + h) * D
+        xrow = orc.view_load(wl.to_f64(xs[src:src + D]), 0, (1, 1, 1, D), (0, 0, 0, 1))
+        yrow = wl.to_f64(y[r * D:(r + 1) * D]).reshape(1, 1, 1, D)
+        want = orc.evaluate(prog.nodes, [xrow, yrow])[0]
+        g1, g2 = gate_errors(wl.to_f64(out[r * D:(r + 1) * D]).reshape(1, D), want.reshape(1, D))
+        assert g2 <= 2e-2, (r, g1, g2)
+    assert not torch.isnan(out.float().sum())   # every element was written

@@ -234,3 +234,31 @@ def test_min_resident_ctas_picks_a_geometry_that_fits_twice_per_sm():
         dvm.set_elems_per_thread(0)
     assert "local_units=259" in free and "col_blocks=1 " in free
     assert "local_units=195" in tight and "col_blocks=2 " in tight and "threads_per_row=128" in tight
+
+
+def test_encode_strided_views_geometry_and_errors():
+    """dvm_encode_strided: the caller's element strides reach the operand descriptors; rows must be adjacent
+    in memory; a stored view must address every element once."""
+    p = wl.OpProgram("axpy")
+    x, y = p.input("f32", 4), p.input("f32", 4)
+    p.output(p.binary("add", p.scalar("muls", x, 2.0), y), "f32")
+    hp = dvm.program_from_nodes(p.nodes)
+    B, S, H, D = 2, 100, 8, 64
+    shape = (B, H, S, D)
+    text = dvm.disassemble(dvm.encode(hp, [shape, shape], in_strides=[[S * H * D, D, H * D, 1], None]))
+    assert "in0 f32 col_stride=1 strides=[512,64,51200]" in text      # S, H, B over storage [B,S,H,D]
+    assert "in1 f32 col_stride=1 strides=[64,6400,51200]" in text     # dense [B,H,S,D]
+    # all-dense strides give the bytes of the plain encode
+    dense = [H * S * D, S * D, D, 1]
+    assert dvm.encode(hp, [shape, shape], in_strides=[dense, dense], out_strides=[dense]).bytes() == \
+        dvm.encode(hp, [shape, shape]).bytes()
+    for kwargs, status in [(dict(in_strides=[[S * H * D, D, 1, H], None]), -3),      # last dim not adjacent
+                           (dict(in_strides=[[-1, 1, 1, 1], None]), -1),               # negative stride
+                           (dict(out_strides=[[S * H * D, D, D, 1]]), -1),             # two rows at one address
+                           (dict(out_strides=[[H * S * D, S * D, 0, 1]]), -1)]:        # zero stride in an output
+        with pytest.raises(dvm.DvmError) as ei:
+            dvm.encode(hp, [shape, shape], **kwargs)
+        assert ei.value.status == status, kwargs
+    # an expanded input (stride 0) is a broadcast
+    text = dvm.disassemble(dvm.encode(hp, [shape, shape], in_strides=[[0, 0, 0, 1], None]))
+    assert "in0 f32 col_stride=1 strides=[0,0,0]" in text
