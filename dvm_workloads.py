@@ -35,8 +35,8 @@ import numpy as np
 import torch
 
 UNARY_OPS = ("exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
-             "recip", "floor", "round", "tanh")
-BINARY_OPS = ("add", "sub", "mul", "div", "min", "max")
+             "recip", "floor", "round", "tanh", "isfinite")
+BINARY_OPS = ("add", "sub", "mul", "div", "min", "max", "pow")
 SCALAR_OPS = ("adds", "muls")
 REDUCE_OPS = ("sum", "max", "min")
 COMPARE_OPS = ("gt", "ge", "lt", "le", "eq", "ne")

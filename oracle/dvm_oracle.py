@@ -104,6 +104,7 @@ _UNARY = {
     "neg": lambda x: -x,                             # extension
     "recip": lambda x: 1.0 / x,                      # extension
     "tanh": np.tanh,                                 # extension
+    "isfinite": lambda x: np.isfinite(x).astype(np.float64),   # Table 1, IsFinite: 1 for a finite value, else 0
 }
 
 _BINARY = {
@@ -113,6 +114,8 @@ _BINARY = {
     "div": lambda a, b: a / b,                       # Table 1, Div
     "max": lambda a, b: np.where(a > b, a, b),       # Table 1, Max
     "min": lambda a, b: np.where(a < b, a, b),       # Table 1, Min
+    "pow": lambda a, b: np.power(a, b),              # Table 1, Pow: a ** b (IEEE pow: NaN for a negative base
+                                                     # with a non-integer exponent)
 }
 
 _COMPARE = {                                         # Table 1, Cmp: 1 where the relation holds, else 0

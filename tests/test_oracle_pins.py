@@ -461,3 +461,36 @@ def test_view_store_writes_the_view_and_nothing_else():
     assert np.array_equal(orc.view_load(out, 7, (3, 5, 2), (60, 4, 1)), vals)       # load after store returns the values
     with pytest.raises(ValueError):
         orc.view_store(storage, 0, (3, 4), (2, 1), np.zeros((3, 4)))                # rows overlap: aliasing
+
+
+# ---------------------------------------------------------------- Pow, IsFinite (Table 1)
+def test_pow_against_math_pow_and_closed_forms():
+    """Pow is pinned by the C library's pow through math.pow, element by element, and by the identities
+    x^2 = x*x, x^0.5 = sqrt(x), x^0 = 1, x^-1 = 1/x, 2^k exact."""
+    p = wl.OpProgram("pow")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.binary("pow", a, b), "f32")
+    x = np.abs(RNG.standard_normal((5, 7))) + 0.1
+    y = RNG.standard_normal((5, 7)) * 3
+    got = orc.evaluate(p.nodes, [x, y])[0]
+    for i in range(5):
+        for j in range(7):
+            assert got[i, j] == pytest.approx(math.pow(x[i, j], y[i, j]), rel=1e-15)
+    ev = lambda xx, yy: orc.evaluate(p.nodes, [np.asarray(xx, dtype=np.float64).reshape(1, -1), np.asarray(yy, dtype=np.float64).reshape(1, -1)])[0][0]
+    assert np.allclose(ev(x[0], np.full(7, 2.0)), x[0] * x[0], rtol=1e-15)
+    assert np.allclose(ev(x[0], np.full(7, 0.5)), np.sqrt(x[0]), rtol=1e-15)
+    assert np.array_equal(ev(x[0], np.zeros(7)), np.ones(7))
+    assert np.allclose(ev(x[0], np.full(7, -1.0)), 1.0 / x[0], rtol=1e-15)
+    assert np.array_equal(ev([2.0, 2.0, 2.0, -2.0, -2.0], [10.0, -3.0, 0.0, 3.0, 2.0]), [1024.0, 0.125, 1.0, -8.0, 4.0])
+    with np.errstate(invalid="ignore"):
+        assert np.isnan(ev([-2.0], [0.5])[0])          # negative base, non-integer exponent
+
+
+def test_isfinite_flags():
+    p = wl.OpProgram("isfinite")
+    a = p.input("f32", 2)
+    p.output(p.unary("isfinite", a), "f32")
+    x = np.array([[0.0, -0.0, 1.5, -3e38, np.inf, -np.inf, np.nan, 1e-45]])
+    got = orc.evaluate(p.nodes, [x])[0]
+    assert np.array_equal(got, [[1, 1, 1, 1, 0, 0, 0, 1]])
+    assert np.array_equal(got[0], [1.0 if math.isfinite(v) else 0.0 for v in x[0]])
