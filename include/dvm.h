@@ -52,14 +52,16 @@ enum {
 
 enum { DVM_F32 = 0, DVM_BF16 = 1 };
 
-/* Unary operators.  EXP SQRT ABS LOG FLOOR ROUND are Table 1's; the others are
+/* Unary operators.  EXP SQRT ABS LOG FLOOR ROUND ISFINITE are Table 1's; the others are
  * extensions the LLM programs need (Table 1 has no erf / sigmoid / rsqrt). */
 enum {
   DVM_EXP = 0, DVM_SQRT = 1, DVM_RSQRT = 2, DVM_ABS = 3, DVM_LOG = 4, DVM_ERF = 5,
-  DVM_SIGMOID = 6, DVM_NEG = 7, DVM_RECIP = 8, DVM_FLOOR = 9, DVM_ROUND = 10, DVM_TANH = 11
+  DVM_SIGMOID = 6, DVM_NEG = 7, DVM_RECIP = 8, DVM_FLOOR = 9, DVM_ROUND = 10, DVM_TANH = 11,
+  DVM_ISFINITE = 12 /* Table 1, IsFinite: the value is 1.0 where x is finite, else 0.0 */
 };
-/* Binary operators (Table 1: Add Sub Mul Div Min Max). */
-enum { DVM_ADD = 0, DVM_SUB = 1, DVM_MUL = 2, DVM_DIV = 3, DVM_MIN = 4, DVM_MAX = 5 };
+/* Binary operators (Table 1: Add Sub Mul Div Min Max Pow).  Pow takes tile operands, like Cmp: an operand
+ * that is one value per row makes dvm_encode return DVM_ERR_UNSUPPORTED. */
+enum { DVM_ADD = 0, DVM_SUB = 1, DVM_MUL = 2, DVM_DIV = 3, DVM_MIN = 4, DVM_MAX = 5, DVM_POW = 6 };
 /* Tensor-scalar operators (Table 1: Adds, Muls). */
 enum { DVM_ADDS = 0, DVM_MULS = 1 };
 /* Comparisons (Table 1: Cmp): the value is 1.0 where the relation holds, else 0.0. */

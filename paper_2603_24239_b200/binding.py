@@ -24,8 +24,8 @@ DVM_MAX_RANK = 6
 F32, BF16 = 0, 1
 DTYPES = {"f32": F32, "bf16": BF16}
 UNARY = {"exp": 0, "sqrt": 1, "rsqrt": 2, "abs": 3, "log": 4, "erf": 5, "sigmoid": 6, "neg": 7,
-         "recip": 8, "floor": 9, "round": 10, "tanh": 11}
-BINARY = {"add": 0, "sub": 1, "mul": 2, "div": 3, "min": 4, "max": 5}
+         "recip": 8, "floor": 9, "round": 10, "tanh": 11, "isfinite": 12}
+BINARY = {"add": 0, "sub": 1, "mul": 2, "div": 3, "min": 4, "max": 5, "pow": 6}
 SCALAR = {"adds": 0, "muls": 1}
 REDUCE = {"sum": 0, "max": 1, "min": 2}
 COMPARE = {"gt": 0, "ge": 1, "lt": 2, "le": 3, "eq": 4, "ne": 5}

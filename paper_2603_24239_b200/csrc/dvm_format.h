@@ -120,9 +120,15 @@ enum {
 enum {
   DVM_U_EXP = 0, DVM_U_SQRT = 1, DVM_U_RSQRT = 2, DVM_U_ABS = 3, DVM_U_LOG = 4,
   DVM_U_ERF = 5, DVM_U_SIGMOID = 6, DVM_U_NEG = 7, DVM_U_RECIP = 8, DVM_U_FLOOR = 9,
-  DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12, DVM_U_NUN = 13
+  DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12,
+  DVM_U_ISFINITE = 13,  // Table 1, IsFinite: 1.0 for a finite value, else 0.0 (tile class: extended variant only)
+  DVM_U_NUN = 14
 };
-enum { DVM_C_GT = 0, DVM_C_GE = 1, DVM_C_LT = 2, DVM_C_LE = 3, DVM_C_EQ = 4, DVM_C_NE = 5, DVM_C_NCMP = 6 };
+// the two-tile-operand class of the extended variant: the comparisons (Table 1, Cmp) and Pow (Table 1)
+enum { DVM_C_GT = 0, DVM_C_GE = 1, DVM_C_LT = 2, DVM_C_LE = 3, DVM_C_EQ = 4, DVM_C_NE = 5,
+       DVM_C_POW = 6,   // ACC = ACC ^ L[a]
+       DVM_C_RPOW = 7,  // ACC = L[a] ^ ACC
+       DVM_C_NCMP = 8 };
 // SUMSQ (sum of squares of R0, R0 kept) is what the encoder emits for reduce_sum(x * x).
 enum { DVM_R_SUM = 0, DVM_R_MAX = 1, DVM_R_MIN = 2, DVM_R_SUMSQ = 3, DVM_R_NRED = 4 };
 
@@ -153,6 +159,7 @@ enum {
   DVM_OP_LD2 = 0x40,   // 0x40 + arith; a = local register x, b = local register y | dtype(x) << 6 | dtype(y) << 7
                        //                                             : ACC = L[x] op L[y]   (fused copy + arithmetic)
   DVM_OP_CMP = 0x50,   // 0x50 + comparison; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC cmp L[a] ? 1 : 0
+                       //   (0x56 / 0x57: Pow, ACC = ACC ^ L[a] / L[a] ^ ACC)
   DVM_OP_SEL = 0x58,   // Table 1, Select; a = local register p, b = local register q | dtype(p) << 6 | dtype(q) << 7
                        //   0x58: ACC = ACC != 0 ? L[p] : L[q]     (the condition is in the accumulator)
                        //   0x59: ACC = L[p] != 0 ? L[q] : ACC     (the else-value is in the accumulator)

@@ -66,7 +66,7 @@ extern "C" int dvm_program_input(dvm_program* p, int dtype, int rank, int* value
 }
 
 extern "C" int dvm_program_unary(dvm_program* p, int op, int x, int* value_id) {
-  if (!valid_value(p, x) || op < 0 || op > DVM_TANH) return DVM_ERR_INVALID_ARG;
+  if (!valid_value(p, x) || op < 0 || op > DVM_ISFINITE) return DVM_ERR_INVALID_ARG;
   Node n = {};
   n.kind = NK_UNARY;
   n.op = (uint8_t)op;
@@ -76,10 +76,11 @@ extern "C" int dvm_program_unary(dvm_program* p, int op, int x, int* value_id) {
 }
 
 extern "C" int dvm_program_binary(dvm_program* p, int op, int x, int y, int* value_id) {
-  if (!valid_value(p, x) || !valid_value(p, y) || op < 0 || op > DVM_MAX) return DVM_ERR_INVALID_ARG;
+  if (!valid_value(p, x) || !valid_value(p, y) || op < 0 || op > DVM_POW) return DVM_ERR_INVALID_ARG;
   Node n = {};
-  n.kind = NK_BINARY;
-  n.op = (uint8_t)op;
+  // Pow shares the two-tile-operand instruction class of the comparisons (extended interpreter variant)
+  n.kind = op == DVM_POW ? NK_COMPARE : NK_BINARY;
+  n.op = (uint8_t)(op == DVM_POW ? DVM_C_POW : op);
   n.x = (int16_t)x;
   n.y = (int16_t)y;
   n.param = -1;
@@ -198,6 +199,7 @@ extern "C" int dvm_program_finalize(dvm_program* p) {
         if (p->nodes[n.x].dtype != DVM_BF16 || p->nodes[n.y].dtype != DVM_BF16) return DVM_ERR_UNSUPPORTED;
       }
       if (n.kind == NK_REDUCE || n.kind == NK_COMPARE || n.kind == NK_SELECT) return DVM_ERR_UNSUPPORTED;  // epilogues: plain elementwise arithmetic only
+      if (n.kind == NK_UNARY && n.op == DVM_ISFINITE) return DVM_ERR_UNSUPPORTED;
     }
   }
   p->finalized = true;
@@ -411,8 +413,9 @@ static inline uint8_t reversed(uint8_t a) {
   if (a == DVM_A_DIV) return DVM_A_RDIV;
   return a;
 }
-static const uint8_t kUnMap[12] = {DVM_U_EXP, DVM_U_SQRT, DVM_U_RSQRT, DVM_U_ABS, DVM_U_LOG, DVM_U_ERF,
-                                   DVM_U_SIGMOID, DVM_U_NEG, DVM_U_RECIP, DVM_U_FLOOR, DVM_U_ROUND, DVM_U_TANH};
+static const uint8_t kUnMap[13] = {DVM_U_EXP, DVM_U_SQRT, DVM_U_RSQRT, DVM_U_ABS, DVM_U_LOG, DVM_U_ERF,
+                                   DVM_U_SIGMOID, DVM_U_NEG, DVM_U_RECIP, DVM_U_FLOOR, DVM_U_ROUND, DVM_U_TANH,
+                                   DVM_U_ISFINITE};
 
 // Generates the load section (every global load of a tile, issued asynchronously into local
 // registers before the tile is computed) and the compute section (accumulator code).
@@ -590,7 +593,7 @@ static bool gen_body(Enc& e) {
     // ---- tile-class result in the accumulator ----
     if (n.kind == NK_COMPARE) {
       // ACC = ACC cmp L[b]; with the right operand in the accumulator the relation is mirrored
-      static const uint8_t kMirror[6] = {DVM_C_LT, DVM_C_LE, DVM_C_GT, DVM_C_GE, DVM_C_EQ, DVM_C_NE};
+      static const uint8_t kMirror[8] = {DVM_C_LT, DVM_C_LE, DVM_C_GT, DVM_C_GE, DVM_C_EQ, DVM_C_NE, DVM_C_RPOW, DVM_C_POW};
       const int y = root(e, n.y);
       if (e.cls[i] != CLS_TILE || e.cls[x] != CLS_TILE || e.cls[y] != CLS_TILE) { e.fail = true; break; }
       int a = x, b = y;
@@ -1088,6 +1091,8 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
   for (int i = 0; i < NN; ++i)
     if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;
+  for (int i = 0; i < NN; ++i)
+    if (p->nodes[i].kind == NK_UNARY && p->nodes[i].op == DVM_ISFINITE && e.cls[i] == CLS_TILE) flags |= DVM_F_EXT_ISA;
   for (int o = 0; o < p->n_outputs; ++o)  // a tile stored into a view whose rows are not one dense range: ViewStore
     if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_EXT_ISA;
   for (int k = 0; k < e.n_in_regs; ++k)
@@ -1361,7 +1366,7 @@ static void outf(Out& o, const char* fmt, ...) {
 }
 static const char* kArith[8] = {"add", "sub", "rsub", "mul", "div", "rdiv", "min", "max"};
 static const char* kUn[DVM_U_NUN] = {"exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
-                                     "recip", "floor", "round", "tanh", "rnd_bf16"};
+                                     "recip", "floor", "round", "tanh", "rnd_bf16", "isfinite"};
 static const char* kRed[DVM_R_NRED] = {"sum", "max", "min", "sumsq"};
 }  // namespace
 
@@ -1425,7 +1430,7 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + 8)
       outf(o, "%-9s acc, l%u%s, l%u%s\n", kArith[op - DVM_OP_LD2], a, ((bb >> 6) & 1) ? ".bf16" : "", bb & 0x3f, (bb >> 7) ? ".bf16" : "");
     else if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) {
-      static const char* kCmp[6] = {"cmp.gt", "cmp.ge", "cmp.lt", "cmp.le", "cmp.eq", "cmp.ne"};
+      static const char* kCmp[DVM_C_NCMP] = {"cmp.gt", "cmp.ge", "cmp.lt", "cmp.le", "cmp.eq", "cmp.ne", "pow", "rpow"};
       if (a == DVM_REG_ACC) outf(o, "%-9s acc, acc, acc\n", kCmp[op - DVM_OP_CMP]);
       else outf(o, "%-9s acc, acc, l%u%s\n", kCmp[op - DVM_OP_CMP], a, dts);
     }

@@ -60,6 +60,7 @@ __device__ __forceinline__ float scalar_unary(int op, float x) {
     case DVM_U_FLOOR: return floorf(x);
     case DVM_U_ROUND: return rintf(x);
     case DVM_U_TANH: return tanhf(x);
+    case DVM_U_ISFINITE: return fabsf(x) < __int_as_float(0x7f800000) ? 1.0f : 0.0f;  // false for NaN, too
     default: return round_bf16(x);
   }
 }

@@ -422,7 +422,7 @@ int dvm_verify_matmul(const uint32_t* w, size_t n_words) {
     }
     else if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) want = 2;
     else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) { if (!mm_reg_ok(v, a, true, false)) return DVM_ERR_BAD_CODE; }
-    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {}
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_RND_BF16 + 1) {}
     else return DVM_ERR_BAD_CODE;
     if (len != want) return DVM_ERR_BAD_CODE;
     pc += len;
@@ -490,7 +490,7 @@ int dvm_disassemble_matmul(const uint32_t* w, size_t n_words, char* buf, size_t 
       memcpy(&f, &v.body[pc + 1], 4);
       mm_printf(o, "  %3u: BINI  ACC = ACC %s %g\n", pc, kMmArith[op & 7], f);
     } else if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) mm_printf(o, "  %3u: BIN   ACC = ACC %s %s\n", pc, kMmArith[op & 7], r);
-    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) mm_printf(o, "  %3u: UN    ACC = %s(ACC)\n", pc, kMmUn[op - DVM_OP_UN]);
+    else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_RND_BF16 + 1) mm_printf(o, "  %3u: UN    ACC = %s(ACC)\n", pc, kMmUn[op - DVM_OP_UN]);
     else return DVM_ERR_BAD_CODE;
     pc += len;
   }
@@ -829,7 +829,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                   for (int i = 0; i < CHUNK; ++i) acc[i] = mm_arith(sub, acc[i], v[i]);
               }
             }
-          } else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
+          } else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_RND_BF16 + 1) {
             const int u = op - DVM_OP_UN;
             if (u == DVM_U_SIGMOID) {
 #pragma unroll

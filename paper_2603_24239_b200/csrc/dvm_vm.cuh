@@ -145,6 +145,10 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
                : "memory");
 }
 
+// Table 1, Pow: the library's powf (special cases as IEEE pow), kept out of line: the extended interpreter
+// variant calls it once per element instead of carrying V copies of it.
+static __device__ __noinline__ float vm_pow(float a, float b) { return powf(a, b); }
+
 // SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
 // EXT: the variant that also decodes Cmp / Select and stores tiles into strided views (launched when a program
@@ -690,6 +694,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             DVM_UN_CASE(DVM_U_ROUND, rintf(x))
             DVM_UN_CASE(DVM_U_TANH, tanhf(x))
             default:
+              if constexpr (EXT) {  // Table 1, IsFinite (programs that use it on a tile run the extended variant)
+                if (op - DVM_OP_UN == DVM_U_ISFINITE) {
+                  DVM_EACH_PAIR A[i] = make_float2(scalar_unary(DVM_U_ISFINITE, A[i].x), scalar_unary(DVM_U_ISFINITE, A[i].y));
+                  break;
+                }
+              }
               DVM_EACH_PAIR A[i] = make_float2(round_bf16(A[i].x), round_bf16(A[i].y));
               break;
           }
@@ -913,6 +923,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             DVM_CMP_CASE(DVM_C_LT, <)
             DVM_CMP_CASE(DVM_C_LE, <=)
             DVM_CMP_CASE(DVM_C_EQ, ==)
+            // Table 1, Pow (unrolled calls of the out-of-line routine: ACC stays in registers)
+            case DVM_C_POW: DVM_EACH_PAIR A[i] = make_float2(vm_pow(A[i].x, Y[i].x), vm_pow(A[i].y, Y[i].y)); break;
+            case DVM_C_RPOW: DVM_EACH_PAIR A[i] = make_float2(vm_pow(Y[i].x, A[i].x), vm_pow(Y[i].y, A[i].y)); break;
             default: DVM_EACH_PAIR A[i] = make_float2(A[i].x != Y[i].x ? 1.f : 0.f, A[i].y != Y[i].y ? 1.f : 0.f); break;
           }
 #undef DVM_CMP_CASE

@@ -64,3 +64,64 @@ def test_compare_on_row_scalars_is_rejected():
     with pytest.raises(dvm.DvmError) as ei:
         dvm.encode(pp, [(4, 100), (4, 100)])
     assert ei.value.status == -3
+
+
+# ---------------------------------------------------------------- Pow, IsFinite (Table 1)
+def _rel_err(got, want):
+    got, want = np.asarray(got, dtype=np.float64), np.asarray(want, dtype=np.float64)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    fin = np.isfinite(want)
+    assert np.array_equal(got[~fin & ~np.isnan(want)], want[~fin & ~np.isnan(want)])
+    return float(np.max(np.abs(got[fin] - want[fin]) / np.maximum(np.abs(want[fin]), 1e-300))) if fin.any() else 0.0
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(3, 1000), (7, 1531), (2, 5, 4096), (1, 37)])
+def test_pow_elementwise(dt, shape):
+    """a ^ b with a > 0: every element within 1e-5 (fp32) / 2e-2 (bf16 output) of the oracle, relative."""
+    p = wl.OpProgram("pow")
+    a, b = p.input(dt, len(shape)), p.input(dt, len(shape))
+    p.output(p.binary("pow", a, b), dt)
+    tdt = torch.bfloat16 if dt == "bf16" else torch.float32
+    x = (wl.randn(shape, torch.float32, 1).abs() + 0.05).to(tdt)
+    y = (wl.randn(shape, torch.float32, 2) * 2).to(tdt)
+    outs, code = gpu_run(p, [x, y])
+    assert "pow" in dvm.disassemble(code)
+    assert _rel_err(wl.to_f64(outs[0]), oracle_run(p, [x, y])[0]) <= (2e-2 if dt == "bf16" else 1e-5)
+
+
+def test_pow_special_cases_and_mirrored_form():
+    """IEEE cases (negative base with integer / non-integer exponent, zero exponents, infinities), and the
+    form with the exponent in the accumulator: c ^ (a + b)."""
+    p = wl.OpProgram("pow")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.binary("pow", a, b), "f32")
+    inf = float("inf")
+    x = torch.tensor([[2.0, 2.0, -2.0, -2.0, -2.0, 0.0, 0.0, 5.0, inf, 0.5, 1.0, -1.0]])
+    y = torch.tensor([[10.0, -3.0, 3.0, 2.0, 0.5, 0.0, 2.0, 0.0, -1.0, inf, float("nan"), inf]])
+    outs, _ = gpu_run(p, [x, y])
+    with np.errstate(invalid="ignore"):
+        want = oracle_run(p, [x, y])[0]
+    assert _rel_err(wl.to_f64(outs[0]), want) <= 1e-6
+    q = wl.OpProgram("rpow")
+    a, b, c = q.input("f32", 2), q.input("f32", 2), q.input("f32", 2)
+    q.output(q.binary("pow", c, q.binary("add", a, b)), "f32")
+    ins = [wl.randn((5, 700), torch.float32, 3), wl.randn((5, 700), torch.float32, 4), wl.randn((5, 700), torch.float32, 5).abs() + 0.1]
+    outs, code = gpu_run(q, ins)
+    assert "rpow" in dvm.disassemble(code)
+    assert _rel_err(wl.to_f64(outs[0]), oracle_run(q, ins)[0]) <= 1e-5
+
+
+def test_isfinite_is_exact_on_tiles_and_on_row_scalars():
+    p = wl.OpProgram("isfinite")
+    a = p.input("f32", 2)
+    p.output(p.unary("isfinite", a), "f32")
+    p.output(p.unary("isfinite", p.reduce("sum", a)), "f32")     # one value per row
+    x = wl.randn((6, 333), torch.float32, 6)
+    x[0, 5], x[1, 7], x[2, 0], x[3, 332] = float("inf"), float("-inf"), float("nan"), 3.0e38
+    x[4] = 3.0e38                                                 # the row sum overflows: not finite
+    outs, _ = gpu_run(p, [x])
+    want = oracle_run(p, [x])
+    assert np.array_equal(wl.to_f64(outs[0]), want[0])
+    row = wl.to_f64(outs[1]).reshape(-1)
+    assert list(row) == [0.0, 0.0, 0.0, 1.0, 0.0, 1.0]           # fp32 row sums: inf, -inf, nan, finite, overflow, finite

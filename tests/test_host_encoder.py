@@ -262,3 +262,18 @@ def test_encode_strided_views_geometry_and_errors():
     # an expanded input (stride 0) is a broadcast
     text = dvm.disassemble(dvm.encode(hp, [shape, shape], in_strides=[[0, 0, 0, 1], None]))
     assert "in0 f32 col_stride=1 strides=[0,0,0]" in text
+
+
+def test_pow_and_isfinite_encode_for_the_extended_variant():
+    p = wl.OpProgram("pow")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.unary("isfinite", p.binary("pow", a, b)), "f32")
+    text = dvm.disassemble(dvm.encode(dvm.program_from_nodes(p.nodes), [(5, 100), (5, 100)]))
+    assert "pow " in text and "isfinite" in text
+    # Pow takes tile operands: a per-row value as exponent is refused
+    q = wl.OpProgram("pow_row")
+    a = q.input("f32", 2)
+    q.output(q.binary("pow", a, q.reduce("max", a)), "f32")
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.encode(dvm.program_from_nodes(q.nodes), [(5, 100)])
+    assert ei.value.status == -3
