@@ -137,10 +137,12 @@ int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,
  * 1 are ignored; a stride of 0 on an input dim repeats the element (an expanded view).
  *  - DVM_ERR_INVALID_ARG: a negative stride; an output view that addresses an element twice (a zero stride,
  *    or dims that overlap).
- *  - DVM_ERR_UNSUPPORTED: a view whose last dim is not adjacent in memory (stride of the last dim != 1:
- *    rows, and every outer dim, may lie anywhere -- slices, permuted outer dims, padded rows -- but a row's
- *    elements are copied as one byte range); more than three outer dims left after adjacent dims that are
- *    dense in every operand were merged; a program with a matmul.
+ *  - DVM_ERR_UNSUPPORTED: more than three outer dims left after adjacent dims that are dense in every
+ *    operand were merged; a program with a matmul.
+ * Cost: a view whose last dim is adjacent in memory (stride 1: slices, permuted outer dims, padded rows) is
+ * copied row by row as byte ranges, like a dense tensor.  A view whose last dim is strided (a transpose that
+ * moves the last dim, a column slice with a step, a last dim expanded with stride 0) is gathered / scattered
+ * element by element: correct, but every element costs a 32-byte memory sector.
  * Everything else as dvm_encode. */
 typedef struct {
   int64_t stride[DVM_MAX_RANK]; /* elements; entry k belongs to dim k of the shape */

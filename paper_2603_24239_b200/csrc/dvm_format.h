@@ -72,7 +72,9 @@ enum {
   DVM_LM_ROWS = 2,     // input copied row by row (one bulk copy per row): row images DVM_ROW_PITCH(...) apart
   DVM_LM_BCAST = 3,    // row-vector input, the same for every row and tile: one row image per slot, loaded once per
                        // slot and program
-  DVM_LM_BCAST_TILE = 4  // the same with several column blocks: the image holds the tile's column block, loaded with every tile
+  DVM_LM_BCAST_TILE = 4, // the same with several column blocks: the image holds the tile's column block, loaded with every tile
+  DVM_LM_GATHER = 5    // input whose columns are not adjacent in memory (Table 1, ViewLoad): every thread fetches its own
+                       // elements, widened to fp32, into the thread-private layout of a temporary (extended variant)
 };
 // bytes between the row images of a ROWS register (room for the 16-byte alignment slack on both sides)
 #define DVM_ROW_PITCH(G, V, es) ((uint32_t)(G) * (uint32_t)(V) * (uint32_t)(es) + 32u)
@@ -81,7 +83,7 @@ enum {
 enum {
   DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24 | dense << 25
                          // (dense: element (row, col) sits at flat offset row * C + col)
-  DVM_OPD_RSVD = 1,
+  DVM_OPD_COLSTRIDE = 1, // element stride between the columns of a tile-class operand: 1, or a view's (then gathered / scattered)
   DVM_OPD_STRIDE0 = 2,   // int64 element stride of outer dim 0 (lo, hi)
   DVM_OPD_STRIDE1 = 4,
   DVM_OPD_STRIDE2 = 6,

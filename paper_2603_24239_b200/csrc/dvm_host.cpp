@@ -267,7 +267,8 @@ enum { CLS_TILE = 0, CLS_SCAL = 1 };
 struct Operand {       // one global-memory access
   int slot;            // tensor slot
   int dtype;
-  int col_stride;      // 1 or 0
+  int col_stride;      // 1: a tile-class access (it has columns), 0: one value per row
+  int64_t cs;          // element stride between the columns of a tile-class access: 1, or what a view gives (ViewLoad / ViewStore)
   int64_t stride[DVM_MAX_RANK];  // element strides over the dominant dims (before merging)
   int64_t ostride[3];            // after merging: outer dims, innermost first
   bool primary;
@@ -478,7 +479,7 @@ static bool gen_body(Enc& e) {
       const int k = e.n_in_regs++;
       e.loads[e.n_loads++] = DVM_INSN(DVM_OP_LDG, 1, k, od);
       e.lreg_of[v] = (int8_t)k;
-      e.ldt_of[v] = (int8_t)e.opd[od].dtype;
+      e.ldt_of[v] = (int8_t)(e.opd[od].cs != 1 ? DVM_DT_F32 : e.opd[od].dtype);  // gathered elements are widened on the way in
     } else {
       if (e.n_sslots >= DVM_MAX_SSLOTS) return false;
       const int k = e.n_sslots++;
@@ -837,6 +838,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
       st *= dk;
     }
     od.col_stride = (e.dims[v][Dt - 1] == 1 && Ccols > 1) ? 0 : 1;
+    od.cs = 1;
     const dvm_strides* us = i < n_in ? (in_strides ? &in_strides[i] : nullptr) : (out_strides ? &out_strides[i - n_in] : nullptr);
     if (us) {
       // a view: the caller's element strides replace the dense ones (dims of size 1 carry no stride)
@@ -850,8 +852,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
         if (i >= n_in && t == 0) return DVM_ERR_INVALID_ARG;  // a stored view addresses every element once
         od.stride[k] = t;
       }
-      if (e.dims[v][Dt - 1] != 1 && od.stride[Dt - 1] != 1)
-        return DVM_ERR_UNSUPPORTED;  // elements of a row must be adjacent in memory (rows and outer dims may lie anywhere)
+      if (e.dims[v][Dt - 1] != 1) od.cs = od.stride[Dt - 1];  // != 1: the row's elements are gathered / scattered one by one
       if (i >= n_in) {
         // no two index tuples at one address: sorted by stride, each dim must step over the one before it
         int64_t sz[DVM_MAX_RANK], sd[DVM_MAX_RANK];
@@ -873,7 +874,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
     } else {
       e.in_operand[v] = (int8_t)e.n_opd;
     }
-    if (od.col_stride == 1 && od.dtype == DVM_DT_BF16) W = 8;
+    if (od.col_stride == 1 && od.cs == 1 && od.dtype == DVM_DT_BF16) W = 8;
     e.n_opd++;
   }
 
@@ -893,7 +894,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
       gsize[ng - 1] *= e.Sd[k];
     } else {
       gsize[ng] = e.Sd[k];
-      for (int o = 0; o < e.n_opd; ++o) gstride[o][ng] = (k == Dt - 1) ? e.opd[o].col_stride : e.opd[o].stride[k];
+      for (int o = 0; o < e.n_opd; ++o) gstride[o][ng] = (k == Dt - 1) ? (e.opd[o].col_stride ? e.opd[o].cs : 0) : e.opd[o].stride[k];
       ng++;
     }
   }
@@ -911,13 +912,13 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   int primary = -1;
   for (int o = 0; o < e.n_opd && primary < 0; ++o) {
     const Operand& od = e.opd[o];
-    if (od.col_stride != 1) continue;
+    if (od.col_stride != 1 || od.cs != 1) continue;
     bool full = true;
     for (int g = 0; g < 3; ++g) if (outer[g] > 1 && od.ostride[g] == 0) full = false;
     if (full) primary = o;
   }
   if (primary < 0) {
-    for (int o = 0; o < e.n_opd && primary < 0; ++o) if (e.opd[o].col_stride == 1) primary = o;
+    for (int o = 0; o < e.n_opd && primary < 0; ++o) if (e.opd[o].col_stride == 1 && e.opd[o].cs == 1) primary = o;
   }
   if (primary >= 0) e.opd[primary].primary = true;
 
@@ -966,15 +967,18 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
       const Operand& od = e.opd[in_opd[k]];
       const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
       const bool inv = !flat && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
-      bool dense = od.col_stride == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
+      const bool gather = od.col_stride == 1 && od.cs != 1;
+      bool dense = od.col_stride == 1 && od.cs == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
       if (!flat) {
         if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
         if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
       }
-      const int mode = inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS);
-      if (inv) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
+      const int mode = gather ? DVM_LM_GATHER
+                              : (inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS));
+      if (inv && !gather) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
       const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
-      const int64_t bytes = inv ? pitch : pitch * (T / Gthreads);
+      // a gathered register holds fp32 values in the thread-private layout of a temporary
+      const int64_t bytes = gather ? (int64_t)g.V * 4 * T : (inv ? pitch : pitch * (T / Gthreads));
       g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
       g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
     }
@@ -1070,7 +1074,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   if (flat) {
     C = Ctile;
     for (int o = 0; o < e.n_opd; ++o) {
-      e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile : 0;
+      e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile * e.opd[o].cs : 0;
       e.opd[o].ostride[1] = e.opd[o].ostride[2] = 0;
     }
     outer[0] = rowsR; outer[1] = outer[2] = 1;
@@ -1081,7 +1085,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   bool dense_of[DVM_MAX_OPERANDS];
   for (int o = 0; o < e.n_opd; ++o) {
     const Operand& od = e.opd[o];
-    bool dense = od.col_stride == 1 && od.ostride[0] == C;
+    bool dense = od.col_stride == 1 && od.cs == 1 && od.ostride[0] == C;
     if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
     if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
     dense_of[o] = dense;
@@ -1097,6 +1101,8 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
     if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_EXT_ISA;
   for (int k = 0; k < e.n_in_regs; ++k)
     if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
+  for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the extended variant
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER) flags |= DVM_F_LOADS_BY_ROW | DVM_F_EXT_ISA;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
@@ -1134,6 +1140,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
     const bool dense = dense_of[o];
     d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
                       ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25);
+    d[DVM_OPD_COLSTRIDE] = (uint32_t)(uint64_t)od.cs;
     for (int g = 0; g < 3; ++g) {
       d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
       d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
@@ -1150,6 +1157,8 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   for (int o = 0; o < e.n_opd; ++o)
     for (int q = 0; q < 3; ++q)
       if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
+  for (int o = 0; o < e.n_opd; ++o)
+    if ((uint64_t)e.opd[o].cs > 0xffffffffull) return DVM_ERR_TOO_LARGE;
   return DVM_OK;
 }
 
@@ -1249,6 +1258,9 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if (k >= n_inr) {
       if (mode != DVM_LM_PRIVATE || dt != DVM_DT_F32) return false;
       need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
+    } else if (mode == DVM_LM_GATHER) {
+      if (od >= n_opd || dt != DVM_DT_F32 || !((w[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA)) return false;
+      need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
     } else {
       if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST_TILE || od >= n_opd) return false;
       if (mode == DVM_LM_BCAST && w[DVM_H_COL_BLOCKS] > 1) return false;  // a once-per-program image holds whole rows
@@ -1303,7 +1315,12 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if (op == DVM_OP_LDG || op == DVM_OP_STG) {
       if (bb >= n_opd) return DVM_ERR_BAD_CODE;
       uint32_t info = ot[bb * DVM_OPD_WORDS];
-      if (op == DVM_OP_LDG && ((a & 0x7f) >= n_inr || !lreg_ok(a & 0x7f, ((info >> 8) & 0xff) == DVM_DT_BF16 ? u_bf16 : u_f32))) return DVM_ERR_BAD_CODE;
+      if (op == DVM_OP_LDG) {
+        if ((a & 0x7f) >= n_inr) return DVM_ERR_BAD_CODE;
+        const bool gathered = ((lt[a & 0x7f] >> 16) & 0xff) == DVM_LM_GATHER;  // widened to fp32 on the way in
+        if (!lreg_ok(a & 0x7f, (!gathered && ((info >> 8) & 0xff) == DVM_DT_BF16) ? u_bf16 : u_f32)) return DVM_ERR_BAD_CODE;
+        if (gathered != (ot[bb * DVM_OPD_WORDS + DVM_OPD_COLSTRIDE] != 1)) return DVM_ERR_BAD_CODE;
+      }
       bool is_out = (info & 0xff) >= n_in;
       if ((op == DVM_OP_STG) != is_out) return DVM_ERR_BAD_CODE;  // never store to an input, never load an output
       if (((info >> 16) & 0xff) != 1) return DVM_ERR_BAD_CODE;
@@ -1399,7 +1416,7 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     uint32_t info = d[0];
     outf(o, "  operand m%u: %s%u %s col_stride=%u strides=[%lld,%lld,%lld]%s\n", k,
          (info & 0xff) < n_in ? "in" : "out", (info & 0xff) < n_in ? (info & 0xff) : (info & 0xff) - n_in,
-         ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", (info >> 16) & 0xff,
+         ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", ((info >> 16) & 0xff) ? d[DVM_OPD_COLSTRIDE] : 0u,
          (long long)((uint64_t)d[2] | ((uint64_t)d[3] << 32)), (long long)((uint64_t)d[4] | ((uint64_t)d[5] << 32)),
          (long long)((uint64_t)d[6] | ((uint64_t)d[7] << 32)), (info >> 24) & 1 ? " primary" : "");
   }

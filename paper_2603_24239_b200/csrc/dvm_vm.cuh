@@ -145,6 +145,29 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
                : "memory");
 }
 
+// Table 1, ViewLoad with a strided column dim, one thread's part: slot sl of the thread holds column
+// cbase + (sl >> lgW << (lgG + lgW)) + (sl & (W - 1)) of the row (+ wrap when negative: the wrap-around slots
+// of a misaligned row's first thread); valid columns are fetched from row + col * cstep_bytes, widened to
+// fp32, into the thread-private layout (vector q of the thread at dst + q * 256 * 16).  fp32 elements travel
+// as 4-byte asynchronous copies, bf16 elements through a register.  Out of line: the extended variants call it.
+static __device__ __noinline__ void vm_gather(const char* row, unsigned long long cstep_bytes, int lg_es, uint32_t dst,
+                                              int cbase, int lgW, int lgG, int wrap, int ncols, int V) {
+#pragma unroll 1
+  for (int sl = 0; sl < V; ++sl) {
+    int col = cbase + ((sl >> lgW) << (lgG + lgW)) + (sl & ((1 << lgW) - 1));
+    if (col < 0) col += wrap;
+    if (col < 0 || col >= ncols) continue;
+    const char* src = row + (unsigned long long)col * cstep_bytes;
+    const uint32_t da = dst + (uint32_t)(sl >> 2) * (uint32_t)(DVM_VM_THREADS * 16) + (uint32_t)(sl & 3) * 4;
+    if (lg_es == 1) {
+      const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(src));
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(da), "f"(v) : "memory");
+    } else {
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(da), "l"(src) : "memory");
+    }
+  }
+}
+
 // Table 1, Pow: the library's powf (special cases as IEEE pow), kept out of line: the extended interpreter
 // variant calls it once per element instead of carrying V copies of it.
 static __device__ __noinline__ float vm_pow(float a, float b) { return powf(a, b); }
@@ -240,23 +263,25 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   };
   // The rest of the geometry: the row's shift and this thread's slot masks.  `c` still holds the previous
   // tile's masks on entry (prev_*: its program, segment length and shift): they are kept when nothing changed.
+  // misalignment (in elements) of the row segment start of the primary operand: the tile's chunks follow it
+  auto row_shift = [&](const TileCtx& c) -> int {
+    if (c.flags & DVM_F_ALIGNED) return 0;
+    const uint32_t prog = c.prog;
+    const uint32_t d = opd_base(prog) + CW(prog + DVM_H_PRIMARY) * DVM_OPD_WORDS;
+    const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
+    const uint32_t base_el = (uint32_t)tensor_ptr(prog, d) >> lg_es;
+    uint32_t off;
+    if (c.flags & DVM_F_PRIMARY_DENSE) off = c.row * CW(prog + DVM_H_COLS) + c.col0;  // low bits are all that matter
+    else off = (uint32_t)row_offset(d, c);
+    return (int)((base_el + off) & (uint32_t)((1 << c.lgW) - 1));
+  };
   auto ctx_masks = [&](TileCtx& c, uint32_t prev_prog, int prev_ncols, int prev_shift) {
     const uint32_t prog = c.prog;
     const int W = 1 << c.lgW;
     const int G = 1 << c.lgG;
     const int t = tid & (G - 1);
     const int nc = c.ncols;
-    int shift = 0;
-    if (!(c.flags & DVM_F_ALIGNED)) {
-      // misalignment (in elements) of the row segment start of the primary operand
-      const uint32_t d = opd_base(prog) + CW(prog + DVM_H_PRIMARY) * DVM_OPD_WORDS;
-      const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
-      const uint32_t base_el = (uint32_t)tensor_ptr(prog, d) >> lg_es;
-      uint32_t off;
-      if (c.flags & DVM_F_PRIMARY_DENSE) off = c.row * CW(prog + DVM_H_COLS) + c.col0;  // low bits are all that matter
-      else off = (uint32_t)row_offset(d, c);
-      shift = (int)((base_el + off) & (uint32_t)(W - 1));
-    }
+    const int shift = row_shift(c);
     c.cbase = (t << c.lgW) - shift;
     c.shift = shift;
     if (prev_prog == prog && nc == prev_ncols && shift == prev_shift) return;  // same masks as the previous tile
@@ -315,7 +340,18 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
         unsigned long long a = 0, n_el = 0;
         bool mine = false;
-        if (mode == DVM_LM_BLOCK) {
+        if (EXT && mode == DVM_LM_GATHER) {
+          // Table 1, ViewLoad with a strided column dim: this thread fetches the elements of its own slots
+          // (column of slot s as in the compute section), widened to fp32, into the private layout
+          // (vector q of the thread at (q * 256 + tid) * 16).  fp32 elements travel as 4-byte async copies.
+          const int shift = row_shift(c);
+          const unsigned long long cs = CW(d + DVM_OPD_COLSTRIDE);
+          const unsigned long long r0 = row_offset(d, c) - c.col0 + (unsigned long long)c.col0 * cs;
+          // wrap-around slots of a misaligned row's first thread (see ctx_masks)
+          const int ov = (shift > 0 && t == 0) ? c.ncols + shift - (V << c.lgG) : 0;
+          vm_gather(reinterpret_cast<const char*>(tensor_ptr(prog, d)) + (r0 << lg_es), cs << lg_es, (int)lg_es,
+                    dst + (uint32_t)tid * 16, (t << c.lgW) - shift, c.lgW, c.lgG, ov > 0 ? (V << c.lgG) : 0, c.ncols, V);
+        } else if (mode == DVM_LM_BLOCK) {
           if (tid == 0) {  // thread 0's row is the tile's first row: the whole tile is one byte range from there
             mine = true;
             const uint32_t rows = CW(prog + DVM_H_ROWS_LO), C = CW(prog + DVM_H_COLS);
@@ -378,7 +414,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t lw = CW(lreg0 + k);
     const uint32_t mode = (lw >> 16) & 0xf;
     uint32_t a = slot_base(buf) + (lw & 0xffffu) * DVM_LOCAL_UNIT;
-    if (mode == DVM_LM_PRIVATE) {
+    if (mode == DVM_LM_PRIVATE || (EXT && mode == DVM_LM_GATHER)) {
       r.a = a + (uint32_t)tid * 16;
       r.a1 = r.a + PSTRIDE;
       r.vA = 2 * PSTRIDE;
@@ -793,13 +829,17 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             const int dt = (info >> 8) & 0xff;
             const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
             unsigned long long el0 = (unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0;
+            long long cstep = 1;  // elements between two columns of the output
             if constexpr (EXT) {  // programs with a strided output run the extended variant (DVM_F_EXT_ISA)
-              if (!((info >> 25) & 1u)) el0 = row_offset(d, c);
+              if (!((info >> 25) & 1u)) {
+                cstep = (long long)CW(d + DVM_OPD_COLSTRIDE);
+                el0 = row_offset(d, c) - c.col0 + (unsigned long long)c.col0 * (unsigned long long)cstep;
+              }
             }
             char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (el0 << lg_es));
             char* q0 = p + ((long long)c.cbase << lg_es);
             const long long qstep = (long long)((G << c.lgW) << lg_es);
-            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
+            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0 && (!EXT || cstep == 1);
             const uint32_t fast = al ? c.fullmask : 0u;
             const uint32_t slow = c.partmask | (c.fullmask & ~fast);
             constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
@@ -863,8 +903,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                     if (col < 0 && c.ov > 0) col += V << c.lgG;  // wrap-around slots of the row's first thread
                     const float val = (el & 1) ? tp[el >> 1].y : tp[el >> 1].x;
                     if (col >= 0 && col < c.ncols) {
-                      if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
-                      else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
+                      const long long ce = EXT ? (long long)col * cstep : (long long)col;  // scattered columns (Table 1, ViewStore)
+                      if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + ce * 2) = __float2bfloat16_rn(val);
+                      else *reinterpret_cast<float*>(p + ce * 4) = val;
                     }
                   }
                 }

@@ -124,3 +124,61 @@ def test_view_of_four_outer_dims_that_merge_to_three():
     shape = (Cc, D, A, B, E)                       # storage [A,B,Cc,D,E] read as [Cc,D,A,B,E]
     xs = (D * E, E, B * Cc * D * E, Cc * D * E, 1)
     _run(_axpy("f32", 5), [(x, 0, shape, xs), (y, 0, shape, _dense(shape))], [(A * B * Cc * D * E, 0, _dense(shape), "f32")])
+
+
+# ---------------------------------------------------------------- views whose LAST dim is strided (gather / scatter)
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("R,C", [(5, 7), (64, 100), (257, 333), (3, 4096), (1000, 33)])
+def test_transposed_input(dt, R, C):
+    """x stored [C,R] read as its transpose [R,C] (column stride R, row stride 1); y and the output dense."""
+    x = wl.randn((C * R,), TORCH_DT[dt], 12)
+    y = wl.randn((R * C,), TORCH_DT[dt], 13)
+    _run(_axpy(dt, 2), [(x, 0, (R, C), (1, R)), (y, 0, (R, C), (C, 1))], [(R * C, 0, (C, 1), dt)])
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("R,C", [(5, 7), (130, 257), (33, 1000)])
+def test_transposed_output(dt, R, C):
+    """The result written as the transpose: logical [R,C] into storage laid out [C,R]; inputs dense."""
+    x = wl.randn((R * C,), TORCH_DT[dt], 14)
+    y = wl.randn((R * C,), TORCH_DT[dt], 15)
+    _run(_axpy(dt, 2), [(x, 0, (R, C), (C, 1)), (y, 0, (R, C), (C, 1))], [(C * R, 0, (1, R), dt)])
+
+
+def test_everything_transposed_no_aligned_operand():
+    """Both inputs and the output are transposed views: no operand has adjacent columns to align tiles to."""
+    R, C = 77, 130
+    x = wl.randn((R * C,), torch.float32, 16)
+    y = wl.randn((R * C,), torch.float32, 17)
+    _run(_axpy("f32", 2), [(x, 0, (R, C), (1, R)), (y, 0, (R, C), (1, R))], [(C * R, 0, (1, R), "f32")])
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+def test_column_slice_with_a_step_and_expanded_last_dim(dt):
+    """x[:, 1::3] (column stride 3) and a column vector expanded along the last dim with stride 0."""
+    R, C = 100, 200
+    x = wl.randn((R * (3 * C + 5),), TORCH_DT[dt], 18)
+    v = wl.randn((R,), TORCH_DT[dt], 19)
+    _run(_axpy(dt, 2), [(x, 1, (R, C), (3 * C + 5, 3)), (v, 0, (R, C), (1, 0))], [(R * C, 0, (C, 1), dt)])
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+def test_softmax_over_a_transposed_view(dt):
+    """Row reductions over a gathered operand: softmax along the columns of a [C,R] matrix, written back transposed."""
+    R, C = 50, 300
+    p = wl.OpProgram("softmax")
+    x = p.input(dt, 2)
+    m = p.reduce("max", x)
+    e = p.unary("exp", p.binary("sub", x, m))
+    p.output(p.binary("div", e, p.reduce("sum", e)), dt)
+    s = wl.randn((C * R,), TORCH_DT[dt], 20)
+    _run(p, [(s, 0, (R, C), (1, R))], [(C * R, 0, (1, R), dt)])
+
+
+def test_last_two_dims_swapped_in_a_4d_view():
+    """[B,H,S,D] read from storage [B,H,D,S] (K^T-style), with a dense second operand."""
+    B, H, S, D = 2, 3, 40, 64
+    x = wl.randn((B * H * D * S,), torch.float32, 21)
+    y = wl.randn((B * H * S * D,), torch.float32, 22)
+    shape = (B, H, S, D)
+    _run(_axpy("f32", 4), [(x, 0, shape, (H * D * S, D * S, 1, S)), (y, 0, shape, _dense(shape))], [(B * H * S * D, 0, _dense(shape), "f32")])
