@@ -16,7 +16,8 @@ Program node tuples (value ids are positions in ``nodes``):
     ("scalar", op, x, s)              op in SCALAR_OPS; s is a float immediate or
                                       ("param", k): k-th runtime scalar argument
     ("cast",   x, dtype)
-    ("reduce", op, x)                 op in REDUCE_OPS, over the last axis, keepdim
+    ("reduce", op, x[, axis])         op in REDUCE_OPS, keepdim; axis counts from the end (default -1: the last
+                                      axis; -2: the penultimate one, Table 1's [M,size,N] -> [M,1,N])
     ("matmul", a, b)                  [M,K] x [K,N]
     ("output", x, dtype)              marks value x as an output stored as dtype
 
@@ -77,9 +78,9 @@ class OpProgram:
         assert dtype in DTYPES
         return self._push(("cast", x, dtype))
 
-    def reduce(self, op: str, x: int) -> int:
-        assert op in REDUCE_OPS
-        return self._push(("reduce", op, x))
+    def reduce(self, op: str, x: int, axis: int = -1) -> int:
+        assert op in REDUCE_OPS and axis <= -1
+        return self._push(("reduce", op, x) if axis == -1 else ("reduce", op, x, axis))
 
     def matmul(self, a: int, b: int) -> int:
         return self._push(("matmul", a, b))

@@ -21,7 +21,8 @@ Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
   Adds/Muls                x op scalar                        (Table 1, Adds/Muls)
   Sqrt/Abs/Log/Exp/Round/Floor                                (Table 1, unary rows)
   Cast                     (dst_dtype)(x)                     (Table 1, Cast)
-  Sum/Max/Min reduce       [M,size,N] -> [M,1,N], here N = 1  (Table 1, Sum/Max/Min)
+  Sum/Max/Min reduce       [M,size,N] -> [M,1,N]; N = 1 unless a  (Table 1, Sum/Max/Min)
+                           reduce node names another axis
   Broadcast                implicit in numpy-style broadcasting (Table 1, Broadcast)
   Cmp                      1.0 where the relation holds, else 0.0  (Table 1, Cmp)
   Select                   cond != 0 ? x : y                       (Table 1, Select)
@@ -128,9 +129,11 @@ _COMPARE = {                                         # Table 1, Cmp: 1 where the
 }
 
 _REDUCE = {
-    "sum": lambda x: np.sum(x, axis=-1, keepdims=True),   # Table 1, Sum with N = 1
-    "max": lambda x: np.max(x, axis=-1, keepdims=True),   # Table 1, Max (reduce)
-    "min": lambda x: np.min(x, axis=-1, keepdims=True),   # Table 1, Min (reduce)
+    # Table 1, Sum / Max / Min: [M, size, N] -> [M, 1, N]; the reduced dim is `axis`, counted from the end
+    # (-1: the last dim, N = 1; -2: the paper's penultimate dim), and stays with size 1
+    "sum": lambda x, axis=-1: np.sum(x, axis=axis, keepdims=True),
+    "max": lambda x, axis=-1: np.max(x, axis=axis, keepdims=True),
+    "min": lambda x, axis=-1: np.min(x, axis=axis, keepdims=True),
 }
 
 
@@ -166,7 +169,10 @@ def evaluate(nodes, inputs, params=()):
             elif kind == "cast":
                 vals[i] = _round_to(vals[n[1]], n[2])
             elif kind == "reduce":
-                vals[i] = _REDUCE[n[1]](vals[n[2]])
+                axis = n[3] if len(n) > 3 else -1
+                if not (-vals[n[2]].ndim <= axis <= -1):
+                    raise ValueError("reduce axis counts from the end: -1 .. -rank")
+                vals[i] = _REDUCE[n[1]](vals[n[2]], axis)
             elif kind == "matmul":
                 vals[i] = np.matmul(vals[n[1]], vals[n[2]])
             elif kind == "compare":

@@ -68,10 +68,11 @@ def brute(nodes, inputs, params=()):
                        for idx in np.ndindex(so)}
         elif k == "reduce":
             s = shapes[n[2]]
-            so = s[:-1] + (1,)
+            ax = len(s) + (n[3] if len(n) > 3 else -1)
+            so = s[:ax] + (1,) + s[ax + 1:]
             shapes[i] = so
             red = {"sum": sum, "max": max, "min": min}[n[1]]
-            vals[i] = {idx: red(vals[n[2]][idx[:-1] + (j,)] for j in range(s[-1]))
+            vals[i] = {idx: red(vals[n[2]][idx[:ax] + (j,) + idx[ax + 1:]] for j in range(s[ax]))
                        for idx in np.ndindex(so)}
         elif k == "matmul":
             (M, K), (K2, N) = shapes[n[1]], shapes[n[2]]
@@ -496,3 +497,39 @@ def test_isfinite_flags():
     got = orc.evaluate(p.nodes, [x])[0]
     assert np.array_equal(got, [[1, 1, 1, 1, 0, 0, 0, 1]])
     assert np.array_equal(got[0], [1.0 if math.isfinite(v) else 0.0 for v in x[0]])
+
+
+# ---------------------------------------------------------------- reductions over another axis (Table 1, [M,size,N] -> [M,1,N])
+def test_reduce_over_the_penultimate_and_outer_axes():
+    """Pinned by closed forms (sums of index patterns), by the last-axis reduction of the swapped array
+    (numpy's swapaxes: another mechanism) and by brute force over index tuples."""
+    M, S, N = 3, 5, 4
+    x = RNG.standard_normal((M, S, N))
+    for op, ref in (("sum", np.sum), ("max", np.max), ("min", np.min)):
+        for axis in (-1, -2, -3):
+            p = wl.OpProgram()
+            a = p.input("f32", 3)
+            p.output(p.reduce(op, a, axis), "f32")
+            got = orc.evaluate(p.nodes, [x])[0]
+            want_shape = list(x.shape); want_shape[axis] = 1
+            assert list(got.shape) == want_shape
+            swapped = ref(np.swapaxes(x, axis, -1), axis=-1, keepdims=True)
+            assert np.array_equal(got, np.swapaxes(swapped, axis, -1))
+            np.testing.assert_allclose(got, brute(p.nodes, [x])[0], rtol=1e-14)
+    # closed form: x[m, s, n] = 100 m + 10 s + n  ->  sum over s = S (100 m + n) + 10 S (S - 1) / 2, max over s at s = S - 1
+    idx = np.indices((M, S, N)).astype(np.float64)
+    y = 100 * idx[0] + 10 * idx[1] + idx[2]
+    p = wl.OpProgram()
+    a = p.input("f32", 3)
+    p.output(p.reduce("sum", a, -2), "f32")
+    p.output(p.reduce("max", a, -2), "f32")
+    s_, m_ = orc.evaluate(p.nodes, [y])
+    mm, nn = np.meshgrid(np.arange(M), np.arange(N), indexing="ij")
+    assert np.array_equal(s_[:, 0, :], S * (100 * mm + nn) + 10 * S * (S - 1) / 2)
+    assert np.array_equal(m_[:, 0, :], 100 * mm + 10 * (S - 1) + nn)
+    # a column normalisation: x / sum over rows; every column of the result sums to 1
+    q = wl.OpProgram()
+    a = q.input("f32", 2)
+    q.output(q.binary("div", a, q.reduce("sum", a, -2)), "f32")
+    z = np.abs(RNG.standard_normal((7, 6))) + 0.1
+    assert np.allclose(orc.evaluate(q.nodes, [z])[0].sum(axis=0), 1.0, rtol=1e-14)
