@@ -103,7 +103,15 @@ int dvm_program_compare(dvm_program* p, int op, int x, int y, int* value_id);
 int dvm_program_select(dvm_program* p, int cond, int x, int y, int* value_id);
 /* Table 1 Cast: rounds the value to `dtype` (nearest even); values stay fp32 in registers. */
 int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
-/* Table 1 Sum / Max / Min over the last axis (axis must be -1), size-1 axis kept. */
+/* Table 1 Sum / Max / Min of [M, size, N] over `size` -> [M, 1, N] (the reduced axis stays with size 1).
+ * `axis` counts from the end of x's (right-aligned) shape: -1 the last axis (N = 1: threads of a row combine
+ * their partial results), -2 the penultimate one (the table's general form), ... down to -DVM_MAX_RANK;
+ * a non-negative axis is DVM_ERR_INVALID_ARG.  A reduction over another axis than the last is encoded over
+ * views: dvm_encode moves that axis to the end for every operand of the program (shapes and strides alike),
+ * so its elements are gathered with the stride the axis has in memory -- correct for every shape, fast only
+ * when that stride is small.  All reductions of one program must name the same axis
+ * (dvm_encode: DVM_ERR_UNSUPPORTED otherwise), and the reduced axis must fit the register budget
+ * (8192 elements), as a row does. */
 int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id);
 /* The cube operation (Sec. 4.2, matrix operations): a [M,K] x b [K,N], bf16 inputs, fp32 value.
  * Both operands must be program inputs; every matmul of a program shares `a`. */

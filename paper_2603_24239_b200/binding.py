@@ -208,7 +208,7 @@ def program_from_nodes(nodes: Iterable[tuple]) -> Program:
         elif k == "cast":
             ids[i] = p.cast(ids[n[1]], n[2])
         elif k == "reduce":
-            ids[i] = p.reduce(n[1], ids[n[2]])
+            ids[i] = p.reduce(n[1], ids[n[2]], n[3] if len(n) > 3 else -1)
         elif k == "matmul":
             ids[i] = p.matmul(ids[n[1]], ids[n[2]])
         elif k == "compare":

@@ -124,12 +124,13 @@ extern "C" int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id)
 
 extern "C" int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id) {
   if (!valid_value(p, x) || op < 0 || op > DVM_RMIN) return DVM_ERR_INVALID_ARG;
-  if (axis != -1) return DVM_ERR_UNSUPPORTED;
+  if (axis > -1 || axis < -DVM_MAX_RANK) return DVM_ERR_INVALID_ARG;  // the axis counts from the end: -1 .. -DVM_MAX_RANK
   Node n = {};
   n.kind = NK_REDUCE;
   n.op = (uint8_t)op;
   n.x = (int16_t)x;
-  n.y = n.param = -1;
+  n.y = -1;
+  n.param = (int16_t)axis;
   return push_node(p, n, value_id);
 }
 
@@ -721,9 +722,11 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
 
 // in_strides / out_strides (each may be NULL: dense row-major): element strides of the views (ViewLoad /
 // ViewStore, Table 1), one entry per input / output.
-static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
-                        const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
-                        size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out) {
+// `lowered`: the shapes are those of encode_views' axis permutation (rank of the dominant shape, not the
+// inputs' declared ranks); every reduction then runs over the last dim.
+static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                       const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
+                       size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out, bool lowered) {
   if (!p || !in_shapes || !code_size) return DVM_ERR_INVALID_ARG;
   if (!p->finalized) return DVM_ERR_NOT_FINALIZED;
   if (n_in != p->n_inputs) return DVM_ERR_INVALID_ARG;
@@ -745,7 +748,7 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   // ---- 1. shape inference (numpy-style right-aligned broadcasting) ----
   int D = 1;
   for (int i = 0; i < n_in; ++i) {
-    if (in_shapes[i].rank != p->nodes[p->inputs[i]].rank) return DVM_ERR_INVALID_ARG;
+    if (!lowered && in_shapes[i].rank != p->nodes[p->inputs[i]].rank) return DVM_ERR_INVALID_ARG;
     if (in_shapes[i].rank > D) D = in_shapes[i].rank;
   }
   {
@@ -1160,6 +1163,79 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
   for (int o = 0; o < e.n_opd; ++o)
     if ((uint64_t)e.opd[o].cs > 0xffffffffull) return DVM_ERR_TOO_LARGE;
   return DVM_OK;
+}
+
+// Reductions over another axis than the last (Table 1, Sum / Max / Min of [M, size, N] over `size`) are lowered
+// to views: elementwise operators do not care in which order the dims are walked, so the reduced axis is moved
+// to the end for EVERY operand (shapes and element strides permuted alike), the program is encoded as a
+// last-axis reduction over those views (ViewLoad / ViewStore), and the reported output shapes are permuted back.
+static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                        const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
+                        size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out) {
+  if (!p || !in_shapes || !code_size) return DVM_ERR_INVALID_ARG;
+  if (!p->finalized) return DVM_ERR_NOT_FINALIZED;
+  int ax = -1;
+  bool last_too = false;
+  for (int i = 0; i < p->n_nodes; ++i) {
+    if (p->nodes[i].kind != NK_REDUCE) continue;
+    const int a = p->nodes[i].param;
+    if (a == -1) { last_too = true; continue; }
+    if (ax != -1 && ax != a) return DVM_ERR_UNSUPPORTED;  // one reduced axis per program
+    ax = a;
+  }
+  if (ax == -1)
+    return encode_core(p, in_shapes, in_strides, n_in, scalars, n_scalars, out_strides, code, code_capacity, code_size,
+                       out_shapes, n_out, false);
+  if (last_too || p->n_matmul > 0) return DVM_ERR_UNSUPPORTED;
+  if (n_in != p->n_inputs || n_in > DVM_MAX_TENSORS || p->n_outputs > DVM_MAX_TENSORS) return DVM_ERR_INVALID_ARG;
+  int D = 1;
+  for (int i = 0; i < n_in; ++i) {
+    if (in_shapes[i].rank != p->nodes[p->inputs[i]].rank || in_shapes[i].rank > DVM_MAX_RANK) return DVM_ERR_INVALID_ARG;
+    if (in_shapes[i].rank > D) D = in_shapes[i].rank;
+  }
+  if (-ax > D) return DVM_ERR_INVALID_ARG;  // no such axis
+  const int q = D + ax;                      // the reduced dim of the right-aligned dominant shape
+  int perm[DVM_MAX_RANK];                    // dim k of the permuted shape is dim perm[k] of the original
+  for (int k = 0, m = 0; k < D; ++k)
+    if (k != q) perm[m++] = k;
+  perm[D - 1] = q;
+  dvm_shape ps[DVM_MAX_TENSORS];
+  dvm_strides pst[DVM_MAX_TENSORS];
+  for (int i = 0; i < n_in; ++i) {
+    const int r = in_shapes[i].rank;
+    int64_t d[DVM_MAX_RANK], t[DVM_MAX_RANK];
+    int64_t st = 1;
+    for (int k = D - 1; k >= 0; --k) {
+      const int uk = k - (D - r);
+      d[k] = uk >= 0 ? in_shapes[i].dims[uk] : 1;
+      t[k] = uk >= 0 ? (in_strides ? in_strides[i].stride[uk] : st) : 0;
+      if (d[k] < 0) return DVM_ERR_INVALID_ARG;
+      st *= d[k] > 0 ? d[k] : 1;
+    }
+    ps[i].rank = D;
+    for (int k = 0; k < DVM_MAX_RANK; ++k) { ps[i].dims[k] = k < D ? d[perm[k]] : 0; pst[i].stride[k] = k < D ? t[perm[k]] : 0; }
+  }
+  // pass 1: the output shapes (in permuted order); pass 2: with the outputs' strides permuted as well
+  dvm_shape pos[DVM_MAX_TENSORS];
+  int st = encode_core(p, ps, pst, n_in, scalars, n_scalars, nullptr, code, code_capacity, code_size, pos, p->n_outputs, true);
+  if (st != DVM_OK) return st;
+  dvm_strides post[DVM_MAX_TENSORS];
+  for (int o = 0; o < p->n_outputs; ++o) {
+    int64_t d[DVM_MAX_RANK], t[DVM_MAX_RANK];
+    for (int k = 0; k < D; ++k) d[perm[k]] = pos[o].dims[k];  // back to the caller's order
+    int64_t s2 = 1;
+    for (int k = D - 1; k >= 0; --k) {
+      t[k] = out_strides ? out_strides[o].stride[k] : s2;
+      s2 *= d[k] > 0 ? d[k] : 1;
+    }
+    for (int k = 0; k < DVM_MAX_RANK; ++k) post[o].stride[k] = k < D ? t[perm[k]] : 0;
+    if (out_shapes && o < n_out) {
+      out_shapes[o].rank = D;
+      for (int k = 0; k < DVM_MAX_RANK; ++k) out_shapes[o].dims[k] = k < D ? d[k] : 0;
+    }
+  }
+  if (out_shapes && n_out < p->n_outputs) return DVM_ERR_INVALID_ARG;
+  return encode_core(p, ps, pst, n_in, scalars, n_scalars, post, code, code_capacity, code_size, nullptr, 0, true);
 }
 
 extern "C" int dvm_encode(const dvm_program* p, const dvm_shape* in_shapes, int n_in,

@@ -279,3 +279,29 @@ def test_pow_and_isfinite_encode_for_the_extended_variant():
     with pytest.raises(dvm.DvmError) as ei:
         dvm.encode(dvm.program_from_nodes(q.nodes), [(5, 100)])
     assert ei.value.status == -3
+
+
+def test_reduce_over_another_axis_is_lowered_to_views():
+    """Sum over axis -2 of [M, S, N]: encoded as a last-axis reduction over the permuted view (the reduced axis
+    becomes the column dim with its memory stride N); output shape reported in the caller's order."""
+    p = wl.OpProgram("r")
+    a = p.input("f32", 3)
+    p.output(p.reduce("sum", a, -2), "f32")
+    hp = dvm.program_from_nodes(p.nodes)
+    code = dvm.encode(hp, [(4, 50, 8)])
+    assert code.out_shapes[0] == (4, 1, 8)
+    text = dvm.disassemble(code)
+    assert "cols=50 " in text and "in0 f32 col_stride=8" in text and "rowsum" in text
+    # two different reduced axes in one program, or a last-axis reduce next to another axis: refused
+    q = wl.OpProgram("rr")
+    a = q.input("f32", 3)
+    q.output(q.binary("add", q.reduce("sum", a, -2), q.reduce("sum", a, -3)), "f32")
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.encode(dvm.program_from_nodes(q.nodes), [(4, 5, 8)])
+    assert ei.value.status == -3
+    r1 = wl.OpProgram("r1")                      # axis -2 of a rank-1 value: no such axis
+    a = r1.input("f32", 1)
+    r1.output(r1.reduce("sum", a, -2), "f32")
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.encode(dvm.program_from_nodes(r1.nodes), [(9,)])
+    assert ei.value.status == -1
