@@ -1061,6 +1061,26 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       if (ctas < 1) continue;
       int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
       g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta);
+      // Gathered / scattered operands whose ROWS are adjacent in memory (a transposed matrix): a warp's 32
+      // lanes cover min(32, G) columns x 32 / min(32, G) consecutive rows, and only the rows share 32-byte
+      // sectors -- few threads per row keep the traffic near the algorithmic bytes, many multiply it.
+      {
+        int64_t num = 0, den = 0;
+        for (int o = 0; o < e.n_opd; ++o) {
+          const Operand& od = e.opd[o];
+          if (od.col_stride != 1) continue;
+          const int64_t es = od.dtype == DVM_DT_BF16 ? 2 : 4;
+          int64_t amp = 4;  // in quarters: 4 = no amplification
+          if (od.cs > 1 && od.ostride[0] == 1) {
+            const int64_t nT = G < 32 ? G : 32, nR = 32 / nT;
+            amp = 4 * nT * cdiv(nR * es, 32) * 32 / (32 * es);
+            if (amp < 4) amp = 4;
+          }
+          num += amp * es;
+          den += 4 * es;
+        }
+        if (den > 0) g.cost = g.cost * num / den;
+      }
       if (empty) g.n_tiles = 0;
       if (best.cost < 0 || g.cost < best.cost) best = g;
       if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;

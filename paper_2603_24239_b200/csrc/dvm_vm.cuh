@@ -152,18 +152,36 @@ __device__ __forceinline__ void vm_bulk_load(uint32_t dst, const void* src, uint
 // as 4-byte asynchronous copies, bf16 elements through a register.  Out of line: the extended variants call it.
 static __device__ __noinline__ void vm_gather(const char* row, unsigned long long cstep_bytes, int lg_es, uint32_t dst,
                                               int cbase, int lgW, int lgG, int wrap, int ncols, int V) {
-#pragma unroll 1
-  for (int sl = 0; sl < V; ++sl) {
+  auto column = [&](int sl) -> int {
     int col = cbase + ((sl >> lgW) << (lgG + lgW)) + (sl & ((1 << lgW) - 1));
     if (col < 0) col += wrap;
-    if (col < 0 || col >= ncols) continue;
-    const char* src = row + (unsigned long long)col * cstep_bytes;
-    const uint32_t da = dst + (uint32_t)(sl >> 2) * (uint32_t)(DVM_VM_THREADS * 16) + (uint32_t)(sl & 3) * 4;
-    if (lg_es == 1) {
-      const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(src));
-      asm volatile("st.shared.f32 [%0], %1;" ::"r"(da), "f"(v) : "memory");
-    } else {
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(da), "l"(src) : "memory");
+    return (col < 0 || col >= ncols) ? -1 : col;
+  };
+  auto slot_addr = [&](int sl) -> uint32_t {
+    return dst + (uint32_t)(sl >> 2) * (uint32_t)(DVM_VM_THREADS * 16) + (uint32_t)(sl & 3) * 4;
+  };
+  if (lg_es == 1) {
+    // bf16 goes through registers: eight loads in flight at a time, then their stores
+#pragma unroll 1
+    for (int s0 = 0; s0 < V; s0 += 8) {
+      unsigned short raw[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int col = column(s0 + k);
+        raw[k] = col >= 0 ? *reinterpret_cast<const unsigned short*>(row + (unsigned long long)col * cstep_bytes) : (unsigned short)0;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float v = __uint_as_float((uint32_t)raw[k] << 16);
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(slot_addr(s0 + k)), "f"(v) : "memory");
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int sl = 0; sl < V; ++sl) {
+      const int col = column(sl);
+      if (col < 0) continue;
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot_addr(sl)), "l"(row + (unsigned long long)col * cstep_bytes) : "memory");
     }
   }
 }
