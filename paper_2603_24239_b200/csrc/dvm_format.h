@@ -59,7 +59,8 @@ enum {
   DVM_F_OUTER_DIMS = 2, // row index must be decomposed over OUTER0..2 for some operand
   DVM_F_FLAT = 4,       // pure elementwise program laid out as a flat range
   DVM_F_PRIMARY_DENSE = 8, // the primary operand is dense: row r starts at element r * C of its tensor
-  DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select or stores a tile into a strided view: it needs the extended interpreter variant
+  DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select / Pow / IsFinite: it needs the extended interpreter variant
+  DVM_F_VIEWS = 64,        // a gathered input or a tile stored into a strided view: it needs the views variant
   DVM_F_LOADS_BY_ROW = 16  // some load is issued per row (row-by-row images, per-row scalars); otherwise
                            // thread 0 alone issues every copy of a tile
 };

@@ -1121,11 +1121,11 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   for (int i = 0; i < NN; ++i)
     if (p->nodes[i].kind == NK_UNARY && p->nodes[i].op == DVM_ISFINITE && e.cls[i] == CLS_TILE) flags |= DVM_F_EXT_ISA;
   for (int o = 0; o < p->n_outputs; ++o)  // a tile stored into a view whose rows are not one dense range: ViewStore
-    if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_EXT_ISA;
+    if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_VIEWS;
   for (int k = 0; k < e.n_in_regs; ++k)
     if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
-  for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the extended variant
-    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER) flags |= DVM_F_LOADS_BY_ROW | DVM_F_EXT_ISA;
+  for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the views variant
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER) flags |= DVM_F_LOADS_BY_ROW | DVM_F_VIEWS;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
@@ -1355,7 +1355,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       if (mode != DVM_LM_PRIVATE || dt != DVM_DT_F32) return false;
       need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
     } else if (mode == DVM_LM_GATHER) {
-      if (od >= n_opd || dt != DVM_DT_F32 || !((w[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA)) return false;
+      if (od >= n_opd || dt != DVM_DT_F32 || !((w[DVM_H_GEOM] >> 24) & DVM_F_VIEWS)) return false;
       need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
     } else {
       if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST_TILE || od >= n_opd) return false;

@@ -39,11 +39,13 @@ long long g_launches = 0;
 template <int V, int PW>
 int occupancy(int* out, size_t smem) {
   int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false, true>, dvm::THREADS, smem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false, 2>, dvm::THREADS, smem));
   *out = n > 0 ? n : 1;
   return DVM_OK;
 }
@@ -52,12 +54,15 @@ int occupancy(int* out, size_t smem) {
 template <int V, int PW>
 int occupancy_levels(int* out, size_t smem) {
   int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  int a = 0, b = 0;
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, dvm::dvm_vm_kernel<V, PW, false, false, true>, dvm::THREADS, smem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dvm::dvm_vm_kernel<V, PW, false, true, true>, dvm::THREADS, smem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  int a = 0, b = 0, c = 0;
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, dvm::dvm_vm_kernel<V, PW, false, 0, true>, dvm::THREADS, smem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dvm::dvm_vm_kernel<V, PW, false, 1, true>, dvm::THREADS, smem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c, dvm::dvm_vm_kernel<V, PW, false, 2, true>, dvm::THREADS, smem));
   n = a < b ? a : b;
+  n = n < c ? n : c;
   if (n <= 0) return DVM_ERR_TOO_LARGE;  // not even one CTA fits: no launch
   *out = n;
   return DVM_OK;
@@ -165,8 +170,8 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   return DVM_OK;
 }
 
-// One kernel variant per (elements per thread, parameter-block size, single program, extended ISA).
-template <int PW, bool EXT>
+// One kernel variant per (elements per thread, parameter-block size, single program, extension level).
+template <int PW, int EXT>
 void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
   if (V == 32) {
     if (single) dvm::dvm_vm_kernel<32, PW, true, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
@@ -178,10 +183,11 @@ void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int gr
 }
 
 template <int PW>
-int launch_variant(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+int launch_variant(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
   const bool single = prm.n_programs == 1 && !prm.use_queue;
-  if (ext) launch_variant_ext<PW, true>(V, single, prm, grid, smem, stream);
-  else launch_variant_ext<PW, false>(V, single, prm, grid, smem, stream);
+  if (ext >= 2) launch_variant_ext<PW, 2>(V, single, prm, grid, smem, stream);
+  else if (ext == 1) launch_variant_ext<PW, 1>(V, single, prm, grid, smem, stream);
+  else launch_variant_ext<PW, 0>(V, single, prm, grid, smem, stream);
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;
@@ -189,13 +195,15 @@ int launch_variant(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size
 
 // The variants with level waits.
 template <int PW>
-int launch_variant_levels(int V, bool ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+int launch_variant_levels(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
   if (V == 32) {
-    if (ext) dvm::dvm_vm_kernel<32, PW, false, true, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<32, PW, false, false, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    if (ext >= 2) dvm::dvm_vm_kernel<32, PW, false, 2, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else if (ext == 1) dvm::dvm_vm_kernel<32, PW, false, 1, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<32, PW, false, 0, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
   } else {
-    if (ext) dvm::dvm_vm_kernel<16, PW, false, true, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<16, PW, false, false, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    if (ext >= 2) dvm::dvm_vm_kernel<16, PW, false, 2, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else if (ext == 1) dvm::dvm_vm_kernel<16, PW, false, 1, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
+    else dvm::dvm_vm_kernel<16, PW, false, 0, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
   }
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
@@ -213,14 +221,15 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   uint64_t total_tiles = 0;
   uint32_t units = 0;
   int V = 0;
-  bool ext = false;  // some program uses Cmp / Select: the extended interpreter variant runs the launch
+  int ext = 0;  // the extension level the launch needs: 1 Cmp / Select / Pow / IsFinite, 2 also views
   for (int i = 0; i < n_programs; ++i) {
     const uint32_t* c = (const uint32_t*)codes[i];
     need += c[DVM_H_TOTAL_WORDS];
     total_tiles += c[DVM_H_N_TILES];
     if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
-    if ((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) ext = true;
+    if (((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) && ext < 1) ext = 1;
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) ext = 2;
     if (V && v != V) return DVM_ERR_INVALID_ARG;  // one kernel variant per launch: same elements per thread
     V = v;
   }
@@ -457,7 +466,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   uint64_t need = dir, total_tiles = 0;
   uint32_t units = 0;
   int V = 0;
-  bool ext = false;  // some program uses Cmp / Select: the extended interpreter variant runs the launch
+  int ext = 0;  // the extension level the launch needs: 1 Cmp / Select / Pow / IsFinite, 2 also views
   for (int i = 0; i < n_programs; ++i) {
     if (!codes[i] || !tensors[i]) return DVM_ERR_INVALID_ARG;
     int st = dvm_verify(codes[i], code_sizes[i]);
@@ -468,7 +477,8 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     total_tiles += c[DVM_H_N_TILES];
     if ((c[DVM_H_LOCAL2] >> 16) > units) units = c[DVM_H_LOCAL2] >> 16;
     const int v = (int)(c[DVM_H_LOCAL] >> 24);
-    if ((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) ext = true;
+    if (((c[DVM_H_GEOM] >> 24) & DVM_F_EXT_ISA) && ext < 1) ext = 1;
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) ext = 2;
     if (V && v != V) return DVM_ERR_INVALID_ARG;
     V = v;
   }

@@ -192,11 +192,13 @@ static __device__ __noinline__ float vm_pow(float a, float b) { return powf(a, b
 
 // SINGLE: one program per launch (dvm_launch).  Its word offset in the parameter block is a compile-time
 // constant, so header fields become direct constant-bank operands, and the work queue is compiled out.
-// EXT: the variant that also decodes Cmp / Select and stores tiles into strided views (launched when a program
-// uses them: DVM_F_EXT_ISA); the basic variant stays as compact as it is without them.
+// EXT: 1: the variant that also decodes Cmp / Select / Pow / IsFinite (launched when a program uses them:
+// DVM_F_EXT_ISA); 2: that, plus gathered inputs and tile stores into strided views (DVM_F_VIEWS).  The basic
+// variant (0) stays as compact as it is without them, and variant 1 without the view code.
 // LEVELS: the stacked variant with in-kernel waits between dependent levels (dvm_launch_stacked_levels).
-template <int V, int PW, bool SINGLE, bool EXT, bool LEVELS = false>
+template <int V, int PW, bool SINGLE, int EXT, bool LEVELS = false>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
+  constexpr bool VIEWS = EXT >= 2;
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
   constexpr int NST = V / 16;          // 16-element steps of a local-register operand
@@ -358,7 +360,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
         unsigned long long a = 0, n_el = 0;
         bool mine = false;
-        if (EXT && mode == DVM_LM_GATHER) {
+        if (VIEWS && mode == DVM_LM_GATHER) {
           // Table 1, ViewLoad with a strided column dim: this thread fetches the elements of its own slots
           // (column of slot s as in the compute section), widened to fp32, into the private layout
           // (vector q of the thread at (q * 256 + tid) * 16).  fp32 elements travel as 4-byte async copies.
@@ -432,7 +434,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t lw = CW(lreg0 + k);
     const uint32_t mode = (lw >> 16) & 0xf;
     uint32_t a = slot_base(buf) + (lw & 0xffffu) * DVM_LOCAL_UNIT;
-    if (mode == DVM_LM_PRIVATE || (EXT && mode == DVM_LM_GATHER)) {
+    if (mode == DVM_LM_PRIVATE || (VIEWS && mode == DVM_LM_GATHER)) {
       r.a = a + (uint32_t)tid * 16;
       r.a1 = r.a + PSTRIDE;
       r.vA = 2 * PSTRIDE;
@@ -748,7 +750,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             DVM_UN_CASE(DVM_U_ROUND, rintf(x))
             DVM_UN_CASE(DVM_U_TANH, tanhf(x))
             default:
-              if constexpr (EXT) {  // Table 1, IsFinite (programs that use it on a tile run the extended variant)
+              if constexpr (EXT >= 1) {  // Table 1, IsFinite (programs that use it on a tile run the extended variant)
                 if (op - DVM_OP_UN == DVM_U_ISFINITE) {
                   DVM_EACH_PAIR A[i] = make_float2(scalar_unary(DVM_U_ISFINITE, A[i].x), scalar_unary(DVM_U_ISFINITE, A[i].y));
                   break;
@@ -848,7 +850,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
             unsigned long long el0 = (unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0;
             long long cstep = 1;  // elements between two columns of the output
-            if constexpr (EXT) {  // programs with a strided output run the extended variant (DVM_F_EXT_ISA)
+            if constexpr (VIEWS) {  // programs with a strided output run the views variant (DVM_F_VIEWS)
               if (!((info >> 25) & 1u)) {
                 cstep = (long long)CW(d + DVM_OPD_COLSTRIDE);
                 el0 = row_offset(d, c) - c.col0 + (unsigned long long)c.col0 * (unsigned long long)cstep;
@@ -857,7 +859,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (el0 << lg_es));
             char* q0 = p + ((long long)c.cbase << lg_es);
             const long long qstep = (long long)((G << c.lgW) << lg_es);
-            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0 && (!EXT || cstep == 1);
+            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0 && (!VIEWS || cstep == 1);
             const uint32_t fast = al ? c.fullmask : 0u;
             const uint32_t slow = c.partmask | (c.fullmask & ~fast);
             constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
@@ -921,7 +923,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                     if (col < 0 && c.ov > 0) col += V << c.lgG;  // wrap-around slots of the row's first thread
                     const float val = (el & 1) ? tp[el >> 1].y : tp[el >> 1].x;
                     if (col >= 0 && col < c.ncols) {
-                      const long long ce = EXT ? (long long)col * cstep : (long long)col;  // scattered columns (Table 1, ViewStore)
+                      const long long ce = VIEWS ? (long long)col * cstep : (long long)col;  // scattered columns (Table 1, ViewStore)
                       if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + ce * 2) = __float2bfloat16_rn(val);
                       else *reinterpret_cast<float*>(p + ce * 4) = val;
                     }
@@ -967,7 +969,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             pc = pc_end;
           }
         } break;
-        case DVM_OP_CMP >> 3: if constexpr (!EXT) { err = ST_BAD_CODE; pc = pc_end; } else {
+        case DVM_OP_CMP >> 3: if constexpr (EXT == 0) { err = ST_BAD_CODE; pc = pc_end; } else {
           // ---- ACC = ACC cmp L[y] ? 1 : 0   (Table 1, Cmp) ----
           pc += 1;
           const int ky = DVM_INSN_A(w0);
@@ -989,7 +991,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           }
 #undef DVM_CMP_CASE
         } break;
-        case DVM_OP_SEL >> 3: if constexpr (!EXT) { err = ST_BAD_CODE; pc = pc_end; } else {
+        case DVM_OP_SEL >> 3: if constexpr (EXT == 0) { err = ST_BAD_CODE; pc = pc_end; } else {
           // ---- Table 1, Select: the condition shrinks to one bit per slot; the value not in ACC streams in ----
           pc += 1;
           const int ib = DVM_INSN_B(w0);
