@@ -61,6 +61,8 @@ enum {
   DVM_F_PRIMARY_DENSE = 8, // the primary operand is dense: row r starts at element r * C of its tensor
   DVM_F_EXT_ISA = 32,      // the program uses Cmp / Select / Pow / IsFinite: it needs the extended interpreter variant
   DVM_F_VIEWS = 64,        // a gathered input or a tile stored into a strided view: it needs the views variant
+  DVM_F_ONE_SLOT = 128,    // hint to dvm_launch: two tile slots leave room for one CTA per SM, one slot for two -- run the
+                           // program with a single slot (no prefetch inside a CTA; the SM's other CTA covers the loads)
   DVM_F_LOADS_BY_ROW = 16  // some load is issued per row (row-by-row images, per-row scalars); otherwise
                            // thread 0 alone issues every copy of a tile
 };

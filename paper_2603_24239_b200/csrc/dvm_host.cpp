@@ -949,6 +949,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
   struct Geo {
     int V, log2G, W, units, scalar_unit;
+    bool one_slot;  // costed for two CTAs per SM that hold ONE tile slot each (see DVM_F_ONE_SLOT)
     int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
     uint32_t flags, inv_mask;
     uint32_t lreg_table[DVM_MAX_LREGS];
@@ -991,8 +992,16 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     }
     g.scalar_unit = g.units;
     if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
+    g.one_slot = false;
     if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
     int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
+    if (ctas == 1 && g_min_resident_ctas < 2 && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
+      // Two slots fit once per SM, one slot fits twice: eight more warps per SM are worth more than the
+      // prefetch inside a CTA (the other CTA computes while this one waits for its tile).  Only a launch of
+      // the program on its own can honour this; the programs of a stacked launch share two slots.
+      g.one_slot = true;
+      return 2;
+    }
     return ctas > 2 ? 2 : ctas;  // the interpreter is compiled for two resident CTAs per SM
   };
   // cores the tiles spread over when `ctas` CTAs are resident per SM (the core count is quoted at 3 CTAs per SM)
@@ -1115,6 +1124,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   }
   if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
   if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
+  if (best.one_slot) flags |= DVM_F_ONE_SLOT;
   if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
   for (int i = 0; i < NN; ++i)
     if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;

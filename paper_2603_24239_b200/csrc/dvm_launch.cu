@@ -215,6 +215,12 @@ thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch 
 // `level` (may be NULL): level[i] of program i, non-decreasing; a program reads what programs of lower levels store.
 int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
                bool use_queue, const int* level, cudaStream_t stream) {
+  // A program that asks for a single tile slot (DVM_F_ONE_SLOT), launched on its own: the variant with level
+  // waits runs it, every tile held back until the CTA's previous tile is done, nothing waited for.
+  const bool one_slot = n_programs == 1 && !level &&
+                        ((((const uint32_t*)codes[0])[DVM_H_GEOM] >> 24) & DVM_F_ONE_SLOT) != 0;
+  static const int kOneLevel[1] = {0};
+  if (one_slot) { level = kOneLevel; use_queue = true; }
   // directory: [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, with levels)]
   uint32_t dir = (level ? 3 : 2) * (uint32_t)n_programs + 1;
   uint64_t need = dir;
@@ -260,16 +266,17 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.total_tiles = (uint32_t)total_tiles;
   P.n_words = pos;
   P.use_queue = use_queue ? 1u : 0u;
-  P.levels = level ? 1u : 0u;
+  P.levels = one_slot ? 2u : (level ? 1u : 0u);
   P.status = dev.scratch;
   P.queue = dev.scratch + 8 + 4 * dev.queue_slot;
 
   const bool large = pos > PW_SMALL;
-  const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;  // one spare unit, two tile slots
-  P.slot_bytes = units * DVM_LOCAL_UNIT;
+  const size_t smem = ((one_slot ? 1 : 2) * (size_t)units + 1) * DVM_LOCAL_UNIT;  // one spare unit, two tile slots (or one)
+  P.slot_bytes = one_slot ? 0u : units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   int occ = 0;
-  st = dvm_occupancy(V, large, (int)units, smem, &occ, level != nullptr);
+  // (the occupancy cache is keyed by the units of two slots: a one-slot launch asks under half its units)
+  st = dvm_occupancy(V, large, one_slot ? ((int)units + 1) / 2 : (int)units, smem, &occ, level != nullptr);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
   int grid = (int)(total_tiles < slots ? total_tiles : slots);

@@ -60,7 +60,8 @@ struct VMParams {
   uint32_t n_words;      // words used in `words`
   uint32_t use_queue;    // 1: tiles beyond the first are claimed from the work queue
   uint32_t slot_bytes;   // bytes of one tile slot in local memory (the largest program's)
-  uint32_t levels;       // 1: the directory has a third table, and tiles wait for the tiles of earlier levels
+  uint32_t levels;       // 1: the directory has a third table, and tiles wait for the tiles of earlier levels;
+                         // 2: one tile slot per CTA (slot_bytes = 0): no tile is loaded ahead, nothing is waited for
   unsigned int* status;  // device status word
   unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished, [2] tiles completed (all zero between launches)
   uint32_t words[PW];    // [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, if levels)][programs ...]
@@ -221,6 +222,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   // dependent stacking: a tile of directory entry i reads what the tiles [0, CW(2n + 1 + i)) of the launch
   // store, so its loads start only after that many tiles are complete (the tiles of the earlier levels)
   constexpr bool levels = LEVELS && !SINGLE;
+  // one tile slot (DVM_F_ONE_SLOT): both slots are the same memory, so a tile's loads start only when the
+  // previous tile is done -- the hold-back of a level change, without its wait
+  const bool one_slot = levels && prm.levels == 2;
 #define CW(i) (prm.words[(i)])  /* one word of the parameter block: a constant-bank load at a warp-uniform index */
 
   if (tid == 0) {
@@ -559,7 +563,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   bool held = false;  // the current tile's loads are held back until the tiles of the earlier levels are complete
   if (tile < prm.total_tiles) {
     if (!SINGLE) while (prog_idx + 1 < n_prog && tile >= CW(n_prog + prog_idx + 1)) ++prog_idx;
-    if (!SINGLE && levels && CW(2 * n_prog + 1 + prog_idx) > 0) {
+    if (!SINGLE && levels && (one_slot || CW(2 * n_prog + 1 + prog_idx) > 0)) {
       held = true;
     } else {
       TileCtx cl;
@@ -584,7 +588,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         // All earlier tiles were claimed before this one, by CTAs that are resident (the grid never exceeds
         // the resident capacity) and that wait only for still earlier levels: the count gets there.
         __syncthreads();
-        if (tid == 0) {
+        if (tid == 0 && !one_slot) {
           if (iter > published) {
             __threadfence();
             atomicAdd(&prm.queue[2], iter - published);
@@ -594,7 +598,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             s_abort = 1;
           }
         }
-        published = iter;
+        if (!one_slot) published = iter;
       }
     }
     if (use_queue && tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
@@ -623,7 +627,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
       const bool first = buf ? slot_prog[0] != next_prog_idx : slot_prog[1] != next_prog_idx;
       // the next tile belongs to a later level than this one: it also waits for this tile, so its loads
       // cannot start ahead (a tile of this tile's own level has nothing left to wait for)
-      if (!SINGLE && levels && CW(2 * n_prog + 1 + next_prog_idx) > tile) {
+      if (!SINGLE && levels && (one_slot || CW(2 * n_prog + 1 + next_prog_idx) > tile)) {
         held = true;
       } else if (((CW(nprog + DVM_H_GEOM) >> 24) & DVM_F_LOADS_BY_ROW) || warp == 0) {
         TileCtx cl;  // rows of the next tile, for the threads that may issue its copies

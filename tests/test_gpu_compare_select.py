@@ -125,3 +125,25 @@ def test_isfinite_is_exact_on_tiles_and_on_row_scalars():
     assert np.array_equal(wl.to_f64(outs[0]), want[0])
     row = wl.to_f64(outs[1]).reshape(-1)
     assert list(row) == [0.0, 0.0, 0.0, 1.0, 0.0, 1.0]           # fp32 row sums: inf, -inf, nan, finite, overflow, finite
+
+
+def test_if_else_add_many_tiles_single_slot_launch():
+    """An instance of thousands of tiles: the program's four fp32 inputs and two temporaries leave room for one
+    CTA per SM with two tile slots, so it is encoded for ONE slot per CTA (two CTAs per SM, no prefetch inside a
+    CTA).  The result is fixed bit for bit (2x, 4x and the add are exact or correctly rounded)."""
+    shape = (61, 67, 4099)
+    prog = wl.program_if_else_add()
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [shape] * 4)
+    words = np.frombuffer(code.bytes(), dtype=np.uint32)
+    assert (int(words[6]) >> 24) & 128          # header word 6 (geometry), flag 128: the single-slot hint
+    ins = [wl.randn(shape, torch.float32, 30 + i, "cuda") for i in range(4)]
+    out = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
+    dvm.launch(code, ins + [out])
+    assert dvm.last_device_status() == 0
+    ref = (torch.where(ins[0] > ins[1], 2 * ins[2], 4 * ins[2]).double() + ins[3].double()).float()
+    assert torch.equal(out, ref)
+    rows = [0, 1, 66, 61 * 67 - 1, 1234]
+    sub = [t.reshape(-1, shape[2])[rows].cpu() for t in ins]
+    want = oracle_run(prog, [s.reshape(1, len(rows), shape[2]) for s in sub])[0]
+    got = wl.to_f64(out.reshape(-1, shape[2])[rows])
+    assert float(np.max(np.abs(got - want[0]) / np.maximum(np.abs(want[0]), 1e-30))) <= 1e-6   # the oracle does not round to fp32

@@ -4,6 +4,8 @@ import ctypes
 import os
 import re
 
+import numpy as np
+
 import pytest
 
 import dvm_workloads as wl
@@ -305,3 +307,19 @@ def test_reduce_over_another_axis_is_lowered_to_views():
     with pytest.raises(dvm.DvmError) as ei:
         dvm.encode(dvm.program_from_nodes(r1.nodes), [(9,)])
     assert ei.value.status == -1
+
+
+def test_single_slot_hint_only_where_it_buys_a_second_cta():
+    """if-else-add at 16 elements per thread: 388 units per slot -- two slots fit once per SM, one slot twice:
+    the header carries the single-slot hint.  A program that fits twice with two slots does not, and neither
+    does any program encoded for a stacked launch (dvm_set_min_resident_ctas(2): its CTAs keep two slots)."""
+    flag = lambda code: (int(np.frombuffer(code.bytes(), dtype=np.uint32)[6]) >> 24) & 128
+    ifelse = dvm.program_from_nodes(wl.program_if_else_add().nodes)
+    assert flag(dvm.encode(ifelse, [(8, 64, 4096)] * 4))
+    norm = dvm.program_from_nodes(wl.program_add_rmsnorm().nodes)
+    assert not flag(dvm.encode(norm, [(300, 4096), (300, 4096), (4096,)]))
+    dvm.set_min_resident_ctas(2)
+    try:
+        assert not flag(dvm.encode(ifelse, [(8, 64, 4096)] * 4))
+    finally:
+        dvm.set_min_resident_ctas(0)
