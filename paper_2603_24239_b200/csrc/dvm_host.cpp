@@ -1070,6 +1070,13 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       if (ctas < 1) continue;
       int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
       g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta);
+      if (g_min_resident_ctas == 2) {
+        // A program of a stacked launch shares the machine with the launch's other programs: there are no
+        // waves of its own to fill, what counts is its total work -- tiles x (elements per thread + overhead).
+        // (A term for the row copies a tile issues was measured and did not pay: narrower tiles that waste
+        // fewer slots win even at 64 copies of 256 bytes per tile.)
+        g.cost = g.n_tiles * (u + beta);
+      }
       // Gathered / scattered operands whose ROWS are adjacent in memory (a transposed matrix): a warp's 32
       // lanes cover min(32, G) columns x 32 / min(32, G) consecutive rows, and only the rows share 32-byte
       // sectors -- few threads per row keep the traffic near the algorithmic bytes, many multiply it.

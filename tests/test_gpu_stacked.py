@@ -45,11 +45,17 @@ def test_stacked_small_mix():
     _check_all(meta)
 
 
-def test_stacked_config4_first_launch():
-    """The first seeded launch of config 4: 64 programs, one kernel."""
-    items = wl.shapes_c4(1)[0]
+@pytest.mark.parametrize("min_ctas,launch", [(0, 0), (2, 0), (2, 1), (2, 7)])
+def test_stacked_config4_launches(min_ctas, launch):
+    """Seeded launches of config 4: 64 programs, one kernel; with dvm_set_min_resident_ctas(2) in the
+    configuration bench.py times (geometries costed by total work, two CTAs per SM)."""
+    items = wl.shapes_c4(launch + 1)[launch]
     assert len(items) == 64
-    codes, tls, meta = _stack(items, wl.data_seed("c4", 0))
+    dvm.set_min_resident_ctas(min_ctas)
+    try:
+        codes, tls, meta = _stack(items, wl.data_seed("c4", 0) + launch)
+    finally:
+        dvm.set_min_resident_ctas(0)
     n0 = dvm.launch_count()
     dvm.launch_stacked(codes, tls)
     assert dvm.last_device_status() == 0
