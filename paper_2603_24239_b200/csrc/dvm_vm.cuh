@@ -808,8 +808,10 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           }
           if (G > 32) {
             if (lane == 0) s_red[red_par][warp] = v;
-            __syncthreads();
             const int wpg = G >> 5;  // warps per row group: 2, 4 or 8
+            // only the warps of this row exchange partial results: a named barrier of their own (1 + row group)
+            if (wpg == 8) __syncthreads();
+            else asm volatile("bar.sync %0, %1;" ::"r"(1 + (warp >> (c.lgG - 5))), "r"(G) : "memory");
             const float* pr = &s_red[red_par][warp & ~(wpg - 1)];
             float x[8];
             x[0] = pr[0]; x[1] = pr[1];
