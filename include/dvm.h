@@ -178,7 +178,9 @@ size_t dvm_code_max_size(const dvm_program* p);
 void dvm_set_num_cores(int n);
 int dvm_get_num_cores(void);
 /* Elements of a tile register that one thread holds (the analogue of the paper's tile size
- * limit T_max = M / n_max): 16 or 32.  0 (default) lets the cost model choose per instance.
+ * limit T_max = M / n_max): 16, 24 or 32.  0 (default) lets the cost model choose per instance (24 only for
+ * programs of the basic instruction set on dense tensors: it exists for dvm_launch alone, a stacked launch of
+ * a 24-element program returns DVM_ERR_UNSUPPORTED).
  * Programs stacked into one launch must all use the same value, so callers of
  * dvm_launch_stacked fix it before encoding.  Process-wide; not thread-safe against encode. */
 void dvm_set_elems_per_thread(int v);

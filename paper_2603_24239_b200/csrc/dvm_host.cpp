@@ -21,7 +21,7 @@ static int g_num_cores = 0;
 static const int kDefaultCores = 148 * 3;
 
 static int g_elems_per_thread = 0;
-extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 32) ? v : 0; }
+extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 24 || v == 32) ? v : 0; }
 extern "C" int dvm_get_elems_per_thread(void) { return g_elems_per_thread; }
 static int g_min_resident_ctas = 0;
 extern "C" void dvm_set_min_resident_ctas(int n) { g_min_resident_ctas = (n == 2) ? 2 : 0; }
@@ -995,7 +995,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     g.one_slot = false;
     if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
     int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
-    if (ctas == 1 && g_min_resident_ctas < 2 && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
+    if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
       // Two slots fit once per SM, one slot fits twice: eight more warps per SM are worth more than the
       // prefetch inside a CTA (the other CTA computes while this one waits for its tile).  Only a launch of
       // the program on its own can honour this; the programs of a stacked launch share two slots.
@@ -1007,10 +1007,27 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   // cores the tiles spread over when `ctas` CTAs are resident per SM (the core count is quoted at 3 CTAs per SM)
   auto cores = [&](int ctas) -> int64_t { return (int64_t)dvm_get_num_cores() * ctas / 3; };
   const int W0 = W;
-  for (int vi = 0; vi < 2; ++vi) {
+  // 24 elements per thread (rows that fill three quarters of a 32-element tile) exist as the one-program
+  // basic interpreter variant only: not for programs of stacked launches, not with Cmp / Select / views
+  bool plain = g_min_resident_ctas == 0;
+  for (int i = 0; i < NN; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_COMPARE || n.kind == NK_SELECT || (n.kind == NK_UNARY && n.op == DVM_ISFINITE)) plain = false;
+  }
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    if (od.col_stride != 1) continue;
+    bool dense = od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);
+    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+    if (od.cs != 1 || (o >= e.n_opd - p->n_outputs && !dense && !flat)) plain = false;
+  }
+  static const int kVs[3] = {32, 24, 16};
+  for (int vi = 0; vi < 3; ++vi) {
     Geo g;
-    g.V = 32 >> vi;
+    g.V = kVs[vi];
     if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
+    if (g.V == 24 && !plain && g_elems_per_thread != 24) continue;
     g.W = W0;
     if (flat) {
       g.log2G = 8;
@@ -1068,7 +1085,9 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       // the local-memory need of this geometry decides how many CTAs are resident at once
       const int ctas = layout(g);
       if (ctas < 1) continue;
-      int64_t u = w * cdiv(ct + pad, G * w);  // elements one thread holds
+      // elements one thread processes per tile: the interpreter walks all V slots of a tile register, used or
+      // not (a row that fills three quarters of 32 slots costs what a full one costs: hence the 24-slot variant)
+      int64_t u = g.V;
       g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta);
       if (g_min_resident_ctas == 2) {
         // A program of a stacked launch shares the machine with the launch's other programs: there are no
@@ -1124,7 +1143,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   bool dense_of[DVM_MAX_OPERANDS];
   for (int o = 0; o < e.n_opd; ++o) {
     const Operand& od = e.opd[o];
-    bool dense = od.col_stride == 1 && od.cs == 1 && od.ostride[0] == C;
+    bool dense = od.col_stride == 1 && od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);  // (a single row has no stride)
     if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
     if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
     dense_of[o] = dense;
@@ -1353,7 +1372,7 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   uint32_t lg = geom & 0xff, W = (geom >> 8) & 0xff, nreg = (geom >> 16) & 0xff;
   const uint32_t local = w[DVM_H_LOCAL];
   const uint32_t n_inr = local & 0xff, n_tmpr = (local >> 8) & 0xff, n_ss = (local >> 16) & 0xff, Vv = local >> 24;
-  if (Vv != 16 && Vv != 32) return DVM_ERR_BAD_CODE;
+  if (Vv != 16 && Vv != 24 && Vv != 32) return DVM_ERR_BAD_CODE;
   const uint32_t u_bf16 = DVM_DT_BF16, u_f32 = DVM_DT_F32;  // element type an instruction expects in a register
   if (lg > 8 || !(W == 4 || W == 8) || nreg != n_inr + n_tmpr) return DVM_ERR_BAD_CODE;
   const uint32_t local2 = w[DVM_H_LOCAL2];

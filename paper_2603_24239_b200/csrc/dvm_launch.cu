@@ -25,7 +25,7 @@ struct DeviceState {
   bool ready = false;
   unsigned int* scratch = nullptr;  // [0] status word, [8 + 4*slot] work-queue counters (next tile, CTAs finished, tiles completed)
   int sm_count = 0;
-  int occ[2][2][DVM_MAX_LOCAL_UNITS + 1];  // resident CTAs per SM for [V == 32][large parameter block][local units], 0 = not yet asked
+  int occ[3][2][DVM_MAX_LOCAL_UNITS + 1];  // resident CTAs per SM for [V: 16, 32, 24][large parameter block][local units], 0 = not yet asked
   int occ_levels[2][2][DVM_MAX_LOCAL_UNITS + 1];  // the same for the variants with level waits
   unsigned queue_slot = 0;
 };
@@ -46,6 +46,17 @@ int occupancy(int* out, size_t smem) {
   DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
   DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
   DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false, 2>, dvm::THREADS, smem));
+  *out = n > 0 ? n : 1;
+  return DVM_OK;
+}
+
+// 24 elements per thread exist as the one-program basic variant only (rows that fill three quarters of a
+// 32-element tile).
+template <int PW>
+int occupancy24(int* out, size_t smem) {
+  int n = 0;
+  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<24, PW, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
+  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<24, PW, true, 0>, dvm::THREADS, smem));
   *out = n > 0 ? n : 1;
   return DVM_OK;
 }
@@ -108,10 +119,11 @@ static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out, bo
     *out = lslot;
     return DVM_OK;
   }
-  int& slot = d.occ[V == 32 ? 1 : 0][large ? 1 : 0][units];
+  int& slot = d.occ[V == 32 ? 1 : (V == 24 ? 2 : 0)][large ? 1 : 0][units];
   if (slot == 0) {
     int st;
-    if (V == 32) st = large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem);
+    if (V == 24) st = large ? occupancy24<PW_LARGE>(&slot, smem) : occupancy24<PW_SMALL>(&slot, smem);
+    else if (V == 32) st = large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem);
     else st = large ? occupancy<16, PW_LARGE>(&slot, smem) : occupancy<16, PW_SMALL>(&slot, smem);
     if (st != DVM_OK) return st;
   }
@@ -185,7 +197,10 @@ void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int gr
 template <int PW>
 int launch_variant(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
   const bool single = prm.n_programs == 1 && !prm.use_queue;
-  if (ext >= 2) launch_variant_ext<PW, 2>(V, single, prm, grid, smem, stream);
+  if (V == 24) {
+    if (!single || ext != 0) return DVM_ERR_UNSUPPORTED;  // encoded for a launch of its own on the basic variant
+    dvm::dvm_vm_kernel<24, PW, true, 0><<<grid, dvm::THREADS, smem, stream>>>(prm);
+  } else if (ext >= 2) launch_variant_ext<PW, 2>(V, single, prm, grid, smem, stream);
   else if (ext == 1) launch_variant_ext<PW, 1>(V, single, prm, grid, smem, stream);
   else launch_variant_ext<PW, 0>(V, single, prm, grid, smem, stream);
   DVM_CUDA(cudaGetLastError());
@@ -196,6 +211,7 @@ int launch_variant(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_
 // The variants with level waits.
 template <int PW>
 int launch_variant_levels(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
+  if (V == 24) return DVM_ERR_UNSUPPORTED;
   if (V == 32) {
     if (ext >= 2) dvm::dvm_vm_kernel<32, PW, false, 2, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
     else if (ext == 1) dvm::dvm_vm_kernel<32, PW, false, 1, true><<<grid, dvm::THREADS, smem, stream>>>(prm);

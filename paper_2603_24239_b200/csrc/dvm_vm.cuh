@@ -525,7 +525,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     if (slow && c.ov > 0 && r.image) {
       // wrap-around: the first `ov` slots are the columns one chunk past this thread's last chunk
       float2 e[4];
-      const uint32_t wa = r.a + (uint32_t)(V >> (dt == DVM_DT_BF16 ? 4 : 3)) * r.vA;  // vector index V * es / 16
+      const uint32_t wv = (uint32_t)(V >> (dt == DVM_DT_BF16 ? 3 : 2));  // vector index V * es / 16: one past the thread's last
+      const uint32_t wa = ((wv & 1u) ? r.a1 : r.a) + (wv >> 1) * r.vA;
       const uint4 v0 = lds128_realign(wa, r.mis);
       if (dt == DVM_DT_BF16) {
         widen_bf16(v0, e);
