@@ -174,7 +174,7 @@ size_t dvm_code_max_size(const dvm_program* p);
 /* Number of parallel units N the tiling cost model balances for (Sec. 4.2: cost
  * = ceil(#tiles / N) * (tile + overhead)).  Default 444 (148 SMs x 3); the encoder scales it to the
  * CTAs that are actually resident per SM for the instance (at most 2).
- * n <= 0 restores the default.  Process-wide; not thread-safe against encode. */
+ * n <= 0 restores the default.  Per calling thread (the setting of one thread does not reach the encodes of another). */
 void dvm_set_num_cores(int n);
 int dvm_get_num_cores(void);
 /* Elements of a tile register that one thread holds (the analogue of the paper's tile size
@@ -182,7 +182,7 @@ int dvm_get_num_cores(void);
  * programs of the basic instruction set on dense tensors: it exists for dvm_launch alone, a stacked launch of
  * a 24-element program returns DVM_ERR_UNSUPPORTED).
  * Programs stacked into one launch must all use the same value, so callers of
- * dvm_launch_stacked fix it before encoding.  Process-wide; not thread-safe against encode. */
+ * dvm_launch_stacked fix it before encoding.  Per calling thread (the setting of one thread does not reach the encodes of another). */
 void dvm_set_elems_per_thread(int v);
 int dvm_get_elems_per_thread(void);
 /* Resident CTAs per SM every encoded geometry has to leave room for: 2, or 0 (default) for no constraint.
@@ -190,7 +190,7 @@ int dvm_get_elems_per_thread(void);
  * exceed half an SM's shared memory leaves the whole launch with one CTA per SM.  With 2, the encoder
  * takes the best geometry among those whose slots fit twice per SM (e.g. two column blocks per row, whose
  * row-vector operands are then half as long); a program no geometry of which fits keeps its unconstrained
- * best.  Callers of dvm_launch_stacked set it before encoding.  Process-wide; not thread-safe against encode. */
+ * best.  Callers of dvm_launch_stacked set it before encoding.  Per calling thread (the setting of one thread does not reach the encodes of another). */
 void dvm_set_min_resident_ctas(int n);
 int dvm_get_min_resident_ctas(void);
 

@@ -17,13 +17,13 @@
 // ---------------------------------------------------------------------------
 // Program description
 // ---------------------------------------------------------------------------
-static int g_num_cores = 0;
+static thread_local int g_num_cores = 0;
 static const int kDefaultCores = 148 * 3;
 
-static int g_elems_per_thread = 0;
+static thread_local int g_elems_per_thread = 0;
 extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 24 || v == 32) ? v : 0; }
 extern "C" int dvm_get_elems_per_thread(void) { return g_elems_per_thread; }
-static int g_min_resident_ctas = 0;
+static thread_local int g_min_resident_ctas = 0;
 extern "C" void dvm_set_min_resident_ctas(int n) { g_min_resident_ctas = (n == 2) ? 2 : 0; }
 extern "C" int dvm_get_min_resident_ctas(void) { return g_min_resident_ctas; }
 extern "C" void dvm_set_num_cores(int n) { g_num_cores = n > 0 ? n : 0; }

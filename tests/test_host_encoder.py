@@ -325,3 +325,22 @@ def test_single_slot_hint_only_where_it_buys_a_second_cta():
         assert not flag(dvm.encode(ifelse, [(8, 64, 4096)] * 4))
     finally:
         dvm.set_min_resident_ctas(0)
+
+
+def test_encoder_knobs_are_per_thread():
+    """dvm_set_elems_per_thread / dvm_set_min_resident_ctas / dvm_set_num_cores act on the calling thread only."""
+    import threading
+    lib = dvm.binding.lib
+    seen = {}
+
+    def worker():
+        lib.dvm_set_elems_per_thread(16)
+        lib.dvm_set_min_resident_ctas(2)
+        lib.dvm_set_num_cores(10)
+        seen["inside"] = (lib.dvm_get_elems_per_thread(), lib.dvm_get_min_resident_ctas(), lib.dvm_get_num_cores())
+
+    t = threading.Thread(target=worker)
+    t.start()
+    t.join()
+    assert seen["inside"] == (16, 2, 10)
+    assert (lib.dvm_get_elems_per_thread(), lib.dvm_get_min_resident_ctas(), lib.dvm_get_num_cores()) == (0, 0, 444)
