@@ -84,12 +84,16 @@ enum {
 
 // ---- operand descriptor ----
 enum {
-  DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24 | dense << 25
+  DVM_OPD_INFO = 0,      // tensor slot | dtype << 8 | col_stride << 16 | primary << 24 | dense << 25 | combine << 26
+                         // (combine, outputs only: 0 plain store; 1 sum, 2 max, 3 min: every tile combines its rows into
+                         //  the fp32 result with atomic operations -- a reduction over an axis the tiles walk along)
                          // (dense: element (row, col) sits at flat offset row * C + col)
   DVM_OPD_COLSTRIDE = 1, // element stride between the columns of a tile-class operand: 1, or a view's (then gathered / scattered)
   DVM_OPD_STRIDE0 = 2,   // int64 element stride of outer dim 0 (lo, hi)
   DVM_OPD_STRIDE1 = 4,
   DVM_OPD_STRIDE2 = 6,
+  DVM_OPD_FILL = 7,      // combined output: its element count (the launch pre-fills it with the operation's identity);
+                         // the word is the high half of stride 2, always 0 otherwise (strides stay below 2^32)
   DVM_OPD_WORDS = 8
 };
 

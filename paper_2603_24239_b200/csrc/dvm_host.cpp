@@ -270,6 +270,8 @@ struct Operand {       // one global-memory access
   int dtype;
   int col_stride;      // 1: a tile-class access (it has columns), 0: one value per row
   int64_t cs;          // element stride between the columns of a tile-class access: 1, or what a view gives (ViewLoad / ViewStore)
+  int combine;         // output only: 0 plain store, 1 + DVM_SUM / DVM_RMAX / DVM_RMIN: atomic combination (see combine_axis)
+  int64_t numel;       // combined output: its elements (the launch pre-fills them with the operation's identity)
   int64_t stride[DVM_MAX_RANK];  // element strides over the dominant dims (before merging)
   int64_t ostride[3];            // after merging: outer dims, innermost first
   bool primary;
@@ -722,11 +724,15 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
 
 // in_strides / out_strides (each may be NULL: dense row-major): element strides of the views (ViewLoad /
 // ViewStore, Table 1), one entry per input / output.
+// `combine_axis` (0: none; else the reduced axis, counted from the end): the program's reductions are results
+// only -- they become plain tile values that every tile combines into the result with atomic operations
+// (the stored view has stride 0 along the reduced axis: all its rows land on one address).
 // `lowered`: the shapes are those of encode_views' axis permutation (rank of the dominant shape, not the
 // inputs' declared ranks); every reduction then runs over the last dim.
 static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
                        const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
-                       size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out, bool lowered) {
+                       size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out, bool lowered,
+                       int combine_axis = 0) {
   if (!p || !in_shapes || !code_size) return DVM_ERR_INVALID_ARG;
   if (!p->finalized) return DVM_ERR_NOT_FINALIZED;
   if (n_in != p->n_inputs) return DVM_ERR_INVALID_ARG;
@@ -783,7 +789,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
         }
       } else {
         for (int k = 0; k < D; ++k) d[k] = e.dims[n.x][k];
-        if (n.kind == NK_REDUCE) d[D - 1] = 1;
+        if (n.kind == NK_REDUCE && !combine_axis) d[D - 1] = 1;
       }
     }
   }
@@ -804,6 +810,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       // the rank of an output is the rank the dominant shape has (leading 1s kept)
       out_shapes[o].rank = D;
       for (int k = 0; k < DVM_MAX_RANK; ++k) out_shapes[o].dims[k] = k < D ? e.dims[p->outputs[o].value][k] : 0;
+      if (combine_axis && p->nodes[p->outputs[o].value].kind == NK_REDUCE) out_shapes[o].dims[D + combine_axis] = 1;
     }
   }
   bool empty = false;
@@ -819,7 +826,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     int64_t last = e.dims[i][Dt - 1];
     e.cls[i] = (last == 1 && Ccols > 1) ? CLS_SCAL : CLS_TILE;
     if (n.kind == NK_REDUCE) {
-      if (Dt < D || e.dims[n.x][Dt - 1] == 1) e.alias[i] = n.x;  // reducing a size-1 axis: identity
+      if (combine_axis || Dt < D || e.dims[n.x][Dt - 1] == 1) e.alias[i] = n.x;  // reducing a size-1 axis: identity
       else has_reduce = true;
     }
     if (n.kind == NK_CAST && n.dtype == DVM_F32) e.alias[i] = n.x;  // registers are fp32 already
@@ -842,6 +849,22 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     }
     od.col_stride = (e.dims[v][Dt - 1] == 1 && Ccols > 1) ? 0 : 1;
     od.cs = 1;
+    od.combine = 0;
+    od.numel = 0;
+    if (combine_axis && i >= n_in && p->nodes[v].kind == NK_REDUCE) {
+      // the result of a reduction: dense over the reduced shape, stride 0 along the reduced axis
+      if (out_strides || od.dtype != DVM_DT_F32) return DVM_ERR_UNSUPPORTED;
+      const int q = D + combine_axis;
+      int64_t s2 = 1;
+      for (int k = D - 1; k >= 0; --k) {
+        const int64_t dk = k == q ? 1 : e.dims[v][k];
+        od.stride[k] = (k == q || (dk == 1 && e.Sd[k] != 1)) ? 0 : s2;
+        s2 *= dk;
+      }
+      od.combine = 1 + p->nodes[v].op;
+      od.numel = s2;
+      if (q == Dt - 1) return DVM_ERR_UNSUPPORTED;  // (the reduced axis is never the column dim here)
+    }
     const dvm_strides* us = i < n_in ? (in_strides ? &in_strides[i] : nullptr) : (out_strides ? &out_strides[i - n_in] : nullptr);
     if (us) {
       // a view: the caller's element strides replace the dense ones (dims of size 1 carry no stride)
@@ -923,6 +946,9 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   if (primary < 0) {
     for (int o = 0; o < e.n_opd && primary < 0; ++o) if (e.opd[o].col_stride == 1 && e.opd[o].cs == 1) primary = o;
   }
+  // combined results: the rows a warp holds are combined slot by slot, so every row must map its columns to
+  // the same slots -- no operand to align the chunks to, every operand is read at its own phase
+  if (combine_axis) primary = -1;
   if (primary >= 0) e.opd[primary].primary = true;
 
   // ---- 5. code: load section + compute section (independent of the tile geometry) ----
@@ -1009,7 +1035,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   const int W0 = W;
   // 24 elements per thread (rows that fill three quarters of a 32-element tile) exist as the one-program
   // basic interpreter variant only: not for programs of stacked launches, not with Cmp / Select / views
-  bool plain = g_min_resident_ctas == 0;
+  bool plain = g_min_resident_ctas == 0 && !combine_axis;
   for (int i = 0; i < NN; ++i) {
     const Node& n = p->nodes[i];
     if (n.kind == NK_COMPARE || n.kind == NK_SELECT || (n.kind == NK_UNARY && n.op == DVM_ISFINITE)) plain = false;
@@ -1066,7 +1092,11 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     g.rowsR = R;
     g.lastRowCols = C;
     for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
+      // combined results: the rows a warp holds (32 / G of them) are combined by shuffles before the atomics
+      if (combine_axis && lg > 5) continue;
       int64_t G = 1 << lg, cap = G * g.V;
+      // ... but not so few threads per row that a row copy shrinks below 256 bytes while the rows are wider
+      if (combine_axis && cap * 4 < 256 && C * 4 >= 256) continue;
       int64_t ct;
       if (has_reduce) {
         // a whole row per thread group; at the widest group a row may use the full capacity: its last
@@ -1088,7 +1118,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       // elements one thread processes per tile: the interpreter walks all V slots of a tile register, used or
       // not (a row that fills three quarters of 32 slots costs what a full one costs: hence the 24-slot variant)
       int64_t u = g.V;
-      g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta);
+      g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta + (combine_axis ? 2 * g.V * G / 32 : 0));  // + the atomics a thread issues
       if (g_min_resident_ctas == 2) {
         // A program of a stacked launch shares the machine with the launch's other programs: there are no
         // waves of its own to fill, what counts is its total work -- tiles x (elements per thread + overhead).
@@ -1198,12 +1228,14 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     uint32_t* d = ot + o * DVM_OPD_WORDS;
     const bool dense = dense_of[o];
     d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
-                      ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25);
+                      ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25) |
+                      ((uint32_t)od.combine << 26);
     d[DVM_OPD_COLSTRIDE] = (uint32_t)(uint64_t)od.cs;
     for (int g = 0; g < 3; ++g) {
       d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
       d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
     }
+    if (od.combine) d[DVM_OPD_FILL] = (uint32_t)od.numel;  // (strides stay below 2^32: the word is free)
   }
   uint32_t* lt = ot + e.n_opd * DVM_OPD_WORDS;
   memcpy(lt, lreg_table, (size_t)nreg * 4);
@@ -1217,7 +1249,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     for (int q = 0; q < 3; ++q)
       if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
   for (int o = 0; o < e.n_opd; ++o)
-    if ((uint64_t)e.opd[o].cs > 0xffffffffull) return DVM_ERR_TOO_LARGE;
+    if ((uint64_t)e.opd[o].cs > 0xffffffffull || (uint64_t)e.opd[o].numel > 0xffffffffull) return DVM_ERR_TOO_LARGE;
   return DVM_OK;
 }
 
@@ -1243,6 +1275,36 @@ static int encode_views(const dvm_program* p, const dvm_shape* in_shapes, const 
     return encode_core(p, in_shapes, in_strides, n_in, scalars, n_scalars, out_strides, code, code_capacity, code_size,
                        out_shapes, n_out, false);
   if (last_too || p->n_matmul > 0) return DVM_ERR_UNSUPPORTED;
+  if (n_in != p->n_inputs) return DVM_ERR_INVALID_ARG;
+  {
+    int rank = 1;
+    for (int i = 0; i < n_in; ++i) {
+      if (in_shapes[i].rank != p->nodes[p->inputs[i]].rank || in_shapes[i].rank > DVM_MAX_RANK) return DVM_ERR_INVALID_ARG;
+      if (in_shapes[i].rank > rank) rank = in_shapes[i].rank;
+    }
+    if (-ax > rank) return DVM_ERR_INVALID_ARG;  // no such axis
+  }
+  // Reductions that are results only (nothing in the program reads them), stored as fp32, dense: no view, no
+  // gather -- the program runs over its natural tiles (columns adjacent in memory) and every tile combines
+  // its rows into the result with atomic operations.
+  {
+    bool results_only = !out_strides;
+    for (int i = 0; i < p->n_nodes && results_only; ++i) {
+      const Node& n = p->nodes[i];
+      const int ops[3] = {n.kind == NK_INPUT ? -1 : n.x,
+                          (n.kind == NK_BINARY || n.kind == NK_COMPARE || n.kind == NK_SELECT) ? n.y : -1,
+                          n.kind == NK_SELECT ? n.param : -1};
+      for (int k = 0; k < 3; ++k)
+        if (ops[k] >= 0 && p->nodes[ops[k]].kind == NK_REDUCE) results_only = false;
+    }
+    for (int o = 0; o < p->n_outputs && results_only; ++o)
+      if (p->nodes[p->outputs[o].value].kind == NK_REDUCE && p->outputs[o].dtype != DVM_F32) results_only = false;
+    if (results_only) {
+      int st = encode_core(p, in_shapes, in_strides, n_in, scalars, n_scalars, nullptr, code, code_capacity, code_size,
+                           out_shapes, n_out, false, ax);
+      if (st != DVM_ERR_UNSUPPORTED) return st;  // otherwise (e.g. the reduced axis ends up as the column dim): the view lowering
+    }
+  }
   if (n_in != p->n_inputs || n_in > DVM_MAX_TENSORS || p->n_outputs > DVM_MAX_TENSORS) return DVM_ERR_INVALID_ARG;
   int D = 1;
   for (int i = 0; i < n_in; ++i) {
@@ -1426,9 +1488,17 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if ((info & 0xff) >= n_tensors) return DVM_ERR_BAD_CODE;
     if (((info >> 8) & 0xff) > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
     if (((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
-    if (ot[o * DVM_OPD_WORDS + 3] | ot[o * DVM_OPD_WORDS + 5] | ot[o * DVM_OPD_WORDS + 7]) return DVM_ERR_BAD_CODE;  // 32-bit strides
+    const uint32_t combine = (info >> 26) & 3;
+    if (ot[o * DVM_OPD_WORDS + 3] | ot[o * DVM_OPD_WORDS + 5]) return DVM_ERR_BAD_CODE;  // 32-bit strides
+    if (!combine && ot[o * DVM_OPD_WORDS + DVM_OPD_FILL]) return DVM_ERR_BAD_CODE;
     n_primary += (info >> 24) & 1;
-    if (info >> 26) return DVM_ERR_BAD_CODE;
+    if (info >> 28) return DVM_ERR_BAD_CODE;
+    if (combine) {
+      // an fp32 result that tiles combine atomically: an output, run by the views variant, never "dense"
+      if ((info & 0xff) < n_in || ((info >> 8) & 0xff) != DVM_DT_F32 || ((info >> 25) & 1) || ((info >> 24) & 1) ||
+          !((w[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) || (w[DVM_H_GEOM] & 0xff) > 5)
+        return DVM_ERR_BAD_CODE;
+    }
   }
   if (n_primary > 1) return DVM_ERR_BAD_CODE;
   if (w[DVM_H_PRIMARY] != 0xffffffffu) {
@@ -1549,8 +1619,8 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     outf(o, "  operand m%u: %s%u %s col_stride=%u strides=[%lld,%lld,%lld]%s\n", k,
          (info & 0xff) < n_in ? "in" : "out", (info & 0xff) < n_in ? (info & 0xff) : (info & 0xff) - n_in,
          ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", ((info >> 16) & 0xff) ? d[DVM_OPD_COLSTRIDE] : 0u,
-         (long long)((uint64_t)d[2] | ((uint64_t)d[3] << 32)), (long long)((uint64_t)d[4] | ((uint64_t)d[5] << 32)),
-         (long long)((uint64_t)d[6] | ((uint64_t)d[7] << 32)), (info >> 24) & 1 ? " primary" : "");
+         (long long)d[2], (long long)d[4], (long long)d[6],
+         (info >> 24) & 1 ? " primary" : (((info >> 26) & 3) == 1 ? " combine=sum" : ((info >> 26) & 3) == 2 ? " combine=max" : ((info >> 26) & 3) == 3 ? " combine=min" : ""));
   }
   const uint32_t* b = ot + n_opd * DVM_OPD_WORDS + ((geom >> 16) & 0xff);
   uint32_t body = w[DVM_H_CODE_WORDS], pc = 0;

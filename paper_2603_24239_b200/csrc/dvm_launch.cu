@@ -182,6 +182,29 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   return DVM_OK;
 }
 
+// Results that tiles combine atomically start from the operation's identity.
+__global__ void dvm_fill_kernel(uint32_t* p, uint32_t n, uint32_t bits) {
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = bits;
+}
+
+int prefill_combined(const uint32_t* code, void* const* tensors, cudaStream_t stream) {
+  const uint32_t counts = code[DVM_H_COUNTS];
+  const uint32_t nt = counts & 0xff, n_opd = (counts >> 16) & 0xff;
+  const uint32_t* ot = code + DVM_HDR_WORDS + 2 * nt;
+  for (uint32_t o = 0; o < n_opd; ++o) {
+    const uint32_t info = ot[o * DVM_OPD_WORDS + DVM_OPD_INFO], comb = (info >> 26) & 3u;
+    if (!comb) continue;
+    const uint32_t n = ot[o * DVM_OPD_WORDS + DVM_OPD_FILL];
+    if (n == 0) continue;
+    const uint32_t bits = comb == 1 ? 0u : (comb == 2 ? 0xff800000u : 0x7f800000u);  // 0, -inf, +inf
+    const int blocks = (int)((n + 255u) / 256u < 1184u ? (n + 255u) / 256u : 1184u);
+    dvm_fill_kernel<<<blocks, 256, 0, stream>>>(static_cast<uint32_t*>(tensors[info & 0xff]), n, bits);
+    DVM_CUDA(cudaGetLastError());
+    dvm_count_launch();
+  }
+  return DVM_OK;
+}
+
 // One kernel variant per (elements per thread, parameter-block size, single program, extension level).
 template <int PW, int EXT>
 void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
@@ -274,6 +297,10 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     }
     st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
     if (st != DVM_OK) return st;
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) {
+      st = prefill_combined(c, tensors[i], stream);
+      if (st != DVM_OK) return st;
+    }
     pos += c[DVM_H_TOTAL_WORDS];
     tb += c[DVM_H_N_TILES];
   }
@@ -521,6 +548,10 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     P.words[n_programs + i] = tb;
     st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
     if (st != DVM_OK) return st;
+    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) {
+      st = prefill_combined(c, tensors[i], stream);
+      if (st != DVM_OK) return st;
+    }
     pos += c[DVM_H_TOTAL_WORDS];
     tb += c[DVM_H_N_TILES];
   }

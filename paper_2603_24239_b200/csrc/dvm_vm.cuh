@@ -187,6 +187,47 @@ static __device__ __noinline__ void vm_gather(const char* row, unsigned long lon
   }
 }
 
+// One value into an fp32 result that many tiles combine: comb 1 sum, 2 max, 3 min (the result was pre-filled
+// with the operation's identity).  Max / min order floats through their bit patterns: non-negative values as
+// signed integers, negative ones as unsigned integers in reverse.
+static __device__ __forceinline__ void vm_atomic_combine(float* a, float v, uint32_t comb) {
+  if (comb == 1) {
+    atomicAdd(a, v);
+  } else if (comb == 2) {
+    v += 0.0f;  // -0 -> +0
+    if (v >= 0.f) atomicMax(reinterpret_cast<int*>(a), __float_as_int(v));
+    else atomicMin(reinterpret_cast<unsigned int*>(a), __float_as_uint(v));
+  } else {
+    v += 0.0f;
+    if (v >= 0.f) atomicMin(reinterpret_cast<int*>(a), __float_as_int(v));
+    else atomicMax(reinterpret_cast<unsigned int*>(a), __float_as_uint(v));
+  }
+}
+
+// The rows a warp holds (32 / G row groups of G threads, G <= 32, all landing on one result row) combined by a
+// reduce-scatter: at the step with lane distance sh a lane keeps the lower or upper half of its slots (by its
+// bit sh) and receives its partner's values for that half.  Afterwards the lane owns n_own = V * G / 32 combined
+// slots, R[0 .. n_own), which are the tile slots first_slot + i.
+template <int V, int COMB>
+static __device__ __forceinline__ void vm_combine_rows(float (&R)[V], int lane, int G, int& first_slot, int& n_own) {
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) {
+    const int half = V * sh / 32;  // the steps run from lane distance 16 down to G: the slots left halve each time
+    if (sh >= G && half >= 1) {
+      const bool up = (lane & sh) != 0;
+#pragma unroll
+      for (int i = 0; i < half; ++i) {
+        const float keep = up ? R[i + half] : R[i];
+        const float send = up ? R[i] : R[i + half];
+        const float got = __shfl_xor_sync(0xffffffffu, send, sh);
+        R[i] = COMB == 1 ? keep + got : (COMB == 2 ? fmaxf(keep, got) : fminf(keep, got));
+      }
+      if (up) first_slot += half;
+      n_own = half;
+    }
+  }
+}
+
 // Table 1, Pow: the library's powf (special cases as IEEE pow), kept out of line: the extended interpreter
 // variant calls it once per element instead of carrying V copies of it.
 static __device__ __noinline__ float vm_pow(float a, float b) { return powf(a, b); }
@@ -864,6 +905,55 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
               }
             }
             char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (el0 << lg_es));
+            if constexpr (VIEWS) {
+              const uint32_t comb = (info >> 26) & 3u;
+              if (comb) {
+                // A result that the tiles combine (a reduction over an axis the tiles walk along): the stored
+                // view has stride 0 along that axis, so the rows of a tile land on one fp32 row of the result.
+                // The rows a warp holds are combined by shuffles first when they share that row (32 / G row
+                // groups per warp, G <= 32), then the warp's first row group issues the atomics.
+                const bool row_ok = c.ncols > 0;
+                bool uni = false;
+                int colmax = c.ncols;
+                unsigned long long el_out = el0;  // the result row this lane's atomics go to
+                if (G <= 32) {
+                  const unsigned long long first = __shfl_sync(0xffffffffu, el0, lane & (G - 1));
+                  uni = __all_sync(0xffffffffu, !row_ok || el0 == first);
+                  if (uni) {
+                    // every lane writes combined slots, also lanes whose own row lies past the end: they all
+                    // write to the row of the warp's first row group (rows ascend: it is valid if any is)
+                    colmax = __shfl_sync(0xffffffffu, c.ncols, lane & (G - 1));
+                    el_out = first;
+                  }
+                }
+                const float ident = comb == 1 ? 0.f : (comb == 2 ? -INFINITY : INFINITY);
+                float R[V];
+#pragma unroll
+                for (int sl = 0; sl < V; ++sl) {
+                  const int col = c.cbase + ((sl >> c.lgW) << (c.lgG + c.lgW)) + (sl & (W - 1));
+                  const float a = (sl & 1) ? A[sl >> 1].y : A[sl >> 1].x;
+                  R[sl] = (row_ok && col >= 0 && col < c.ncols) ? a : ident;
+                }
+                // reduce-scatter over the warp's row groups: at each step a lane keeps one half of its slots and
+                // hands the other half to its partner, so every slot is combined once per step, not once per lane
+                int first_slot = 0, n_own = V;
+                if (uni) {
+                  if (comb == 1) vm_combine_rows<V, 1>(R, lane, G, first_slot, n_own);
+                  else if (comb == 2) vm_combine_rows<V, 2>(R, lane, G, first_slot, n_own);
+                  else vm_combine_rows<V, 3>(R, lane, G, first_slot, n_own);
+                }
+                float* prow = reinterpret_cast<float*>(tensor_ptr(prog, d)) + el_out;
+#pragma unroll
+                for (int i = 0; i < V; ++i) {
+                  if (i < n_own) {
+                    const int sl = first_slot + i;
+                    const int col = c.cbase + ((sl >> c.lgW) << (c.lgG + c.lgW)) + (sl & (W - 1));
+                    if (col >= 0 && col < colmax && (uni || row_ok)) vm_atomic_combine(prow + (long long)col * cstep, R[i], comb);
+                  }
+                }
+                break;
+              }
+            }
             char* q0 = p + ((long long)c.cbase << lg_es);
             const long long qstep = (long long)((G << c.lgW) << lg_es);
             const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0 && (!VIEWS || cstep == 1);

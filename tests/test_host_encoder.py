@@ -290,12 +290,27 @@ def test_reduce_over_another_axis_is_lowered_to_views():
     becomes the column dim with its memory stride N); output shape reported in the caller's order."""
     p = wl.OpProgram("r")
     a = p.input("f32", 3)
-    p.output(p.reduce("sum", a, -2), "f32")
+    s1 = p.reduce("sum", a, -2)
+    p.output(p.binary("sub", a, s1), "f32")         # the reduced value is used: the view lowering
     hp = dvm.program_from_nodes(p.nodes)
     code = dvm.encode(hp, [(4, 50, 8)])
-    assert code.out_shapes[0] == (4, 1, 8)
+    assert code.out_shapes[0] == (4, 50, 8)
     text = dvm.disassemble(code)
     assert "cols=50 " in text and "in0 f32 col_stride=8" in text and "rowsum" in text
+    # a reduction that is a result only: the tiles keep their natural shape (columns adjacent in memory) and
+    # combine their rows into the fp32 result atomically -- the stored view has stride 0 along the reduced axis
+    r = wl.OpProgram("r2")
+    a = r.input("f32", 3)
+    r.output(r.reduce("max", r.unary("abs", a), -2), "f32")
+    code = dvm.encode(dvm.program_from_nodes(r.nodes), [(4, 50, 256)])
+    assert code.out_shapes[0] == (4, 1, 256)
+    text = dvm.disassemble(code)
+    assert "cols=256 " in text and "strides=[0,256,0] combine=max" in text and "rowmax" not in text
+    # ... but not into a bf16 result (the view lowering again)
+    r = wl.OpProgram("r3")
+    a = r.input("bf16", 3)
+    r.output(r.reduce("sum", a, -2), "bf16")
+    assert "combine" not in dvm.disassemble(dvm.encode(dvm.program_from_nodes(r.nodes), [(4, 50, 256)]))
     # two different reduced axes in one program, or a last-axis reduce next to another axis: refused
     q = wl.OpProgram("rr")
     a = q.input("f32", 3)
