@@ -1095,8 +1095,9 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       // combined results: the rows a warp holds (32 / G of them) are combined by shuffles before the atomics
       if (combine_axis && lg > 5) continue;
       int64_t G = 1 << lg, cap = G * g.V;
-      // ... but not so few threads per row that a row copy shrinks below 256 bytes while the rows are wider
-      if (combine_axis && cap * 4 < 256 && C * 4 >= 256) continue;
+      // ... but not so few threads per row that a row copy shrinks below 512 bytes while the rows are wider
+      // (measured on column sums: 256-byte copies 1560 GB/s, 512 bytes 1640, 1 KB and more lose to the atomics)
+      if (combine_axis && cap * 4 < 512 && C * 4 >= 512) continue;
       int64_t ct;
       if (has_reduce) {
         // a whole row per thread group; at the widest group a row may use the full capacity: its last

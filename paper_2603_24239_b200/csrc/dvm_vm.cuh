@@ -930,9 +930,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                 float R[V];
 #pragma unroll
                 for (int sl = 0; sl < V; ++sl) {
-                  const int col = c.cbase + ((sl >> c.lgW) << (c.lgG + c.lgW)) + (sl & (W - 1));
                   const float a = (sl & 1) ? A[sl >> 1].y : A[sl >> 1].x;
-                  R[sl] = (row_ok && col >= 0 && col < c.ncols) ? a : ident;
+                  R[sl] = slot_valid(c, sl) ? a : ident;  // (the slot masks of a row past the end are empty)
                 }
                 // reduce-scatter over the warp's row groups: at each step a lane keeps one half of its slots and
                 // hands the other half to its partner, so every slot is combined once per step, not once per lane
