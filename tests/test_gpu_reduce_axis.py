@@ -82,3 +82,40 @@ def test_reduce_axis_on_a_view():
     assert dvm.last_device_status() == 0
     want = buf.view(R, pitch)[:, 3:3 + C].double().sum(dim=0)
     assert torch.allclose(out.cpu().double(), want, rtol=1e-5, atol=1e-5)
+
+
+@pytest.mark.parametrize("op", ["max", "min"])
+def test_combined_max_min_signs_and_zeros(op):
+    """Results-only max / min over axis -2 go through atomics on the floats' bit patterns: all-negative,
+    all-positive, mixed and all-zero columns (with -0.0), many tiles per result element."""
+    S, N = 3000, 260
+    x = wl.randn((S, N), torch.float32, 77)
+    x[:, 0:64] = -x[:, 0:64].abs() - 0.5        # all negative
+    x[:, 64:128] = x[:, 64:128].abs() + 0.5     # all positive
+    x[:, 128:130] = 0.0
+    x[::2, 129] = -0.0
+    p = wl.OpProgram("colext")
+    a = p.input("f32", 2)
+    p.output(p.reduce(op, a, -2), "f32")
+    outs, code = gpu_run(p, [x])
+    assert "combine=" + op in dvm.disassemble(code)
+    want = oracle_run(p, [x])[0]
+    assert np.array_equal(wl.to_f64(outs[0]), want)
+
+
+def test_combined_sum_next_to_a_plain_output():
+    """A results-only column sum of squares and the elementwise result itself, from one program."""
+    M, S, N = 3, 700, 96
+    p = wl.OpProgram("sq_and_colsum")
+    a = p.input("bf16", 3)
+    sq = p.binary("mul", a, a)
+    p.output(sq, "bf16")
+    p.output(p.reduce("sum", sq, -2), "f32")
+    x = wl.randn((M, S, N), torch.bfloat16, 5)
+    outs, code = gpu_run(p, [x])
+    assert "combine=sum" in dvm.disassemble(code)
+    want = oracle_run(p, [x])
+    g1, _ = gate_errors(wl.to_f64(outs[0]).reshape(1, -1), want[0].reshape(1, -1))
+    assert g1 <= 2e-2
+    g1, _ = gate_errors(wl.to_f64(outs[1]).reshape(1, -1), want[1].reshape(1, -1))
+    assert g1 <= 1e-5
