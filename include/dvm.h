@@ -109,7 +109,11 @@ int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
  * a non-negative axis is DVM_ERR_INVALID_ARG.  A reduction over another axis than the last is encoded over
  * views: dvm_encode moves that axis to the end for every operand of the program (shapes and strides alike),
  * so its elements are gathered with the stride the axis has in memory -- correct for every shape, fast only
- * when that stride is small.  All reductions of one program must name the same axis
+ * when that stride is small.  A reduction over such an axis that is a RESULT ONLY (nothing in the program reads
+ * it, stored as fp32 into a dense output) is encoded differently: the tiles keep their natural shape and
+ * combine their rows into the result with atomic operations; dvm_launch first fills that output with the
+ * operation's identity (one more small kernel on the stream), and a sum's order of additions is not fixed
+ * from run to run (the fp32 result varies in its last bits).  All reductions of one program must name the same axis
  * (dvm_encode: DVM_ERR_UNSUPPORTED otherwise), and the reduced axis must fit the register budget
  * (8192 elements), as a row does. */
 int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id);
