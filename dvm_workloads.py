@@ -107,8 +107,9 @@ class OpProgram:
 
 # --------------------------------------------------------------------------
 # The op programs of the five configurations (definitions: standard ones;
-# the readings chosen where the configuration is silent are listed in
-# DESIGN.md under "Readings").
+# where a configuration is silent the reading taken is stated in the program's
+# docstring: norm on the un-rounded fp32 sum, exact-erf GELU, LayerNorm without
+# affine parameters and with biased variance, mask added before the scale).
 # --------------------------------------------------------------------------
 
 def program_c1() -> OpProgram:

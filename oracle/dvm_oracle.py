@@ -29,8 +29,7 @@ Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
   ViewLoad / ViewStore     element (i_0..i_{d-1}) of a view lies at          (Table 1, ViewLoad / ViewStore:
                            base + sum_k i_k * stride_k of its storage        non-contiguous tiles, per-dim strides)
                            (view_load / view_store below; evaluate() itself sees logical arrays only)
-Extensions that the benchmark programs need and Table 1 lacks (stated as such
-in DESIGN.md): erf, sigmoid(x) = 1/(1+exp(-x)), rsqrt(x) = 1/sqrt(x),
+Extensions that the benchmark programs need and Table 1 lacks: erf, sigmoid(x) = 1/(1+exp(-x)), rsqrt(x) = 1/sqrt(x),
 recip, neg, tanh, and matmul C[i,j] = sum_k A[i,k] B[k,j] (the paper's cube
 operation, Sec. 4.2, described in prose only).
 
@@ -137,7 +136,7 @@ _REDUCE = {
 }
 
 
-def evaluate(nodes, inputs, params=()):
+def evaluate(nodes, inputs, params=(), diagnostic_fp32=False):
     """Evaluate an op program node by node on whole tensors.
 
     nodes  : list of node tuples (see the workload module's docstring).
@@ -145,7 +144,20 @@ def evaluate(nodes, inputs, params=()):
              broadcast against each other numpy-style (right-aligned).
     params : runtime scalar arguments referenced by ("param", k).
     Returns the list of outputs (float64, unrounded), in "output"-node order.
+
+    diagnostic_fp32=True runs the same steps with every value held in float32
+    instead of float64.  That is NOT the reference: it only labels the elements
+    on which a faithful fp32 evaluation already agrees with the float64 result
+    ("well conditioned"), for the statistics the parity tests report beside
+    their gates.
     """
+    if diagnostic_fp32:
+        outs32 = _evaluate(nodes, inputs, params, np.float32)
+        return [o.astype(np.float64) for o in outs32]
+    return _evaluate(nodes, inputs, params, np.float64)
+
+
+def _evaluate(nodes, inputs, params, ft):
     vals = [None] * len(nodes)
     outs = []
     it = iter(inputs)
@@ -153,7 +165,7 @@ def evaluate(nodes, inputs, params=()):
         for i, n in enumerate(nodes):
             kind = n[0]
             if kind == "input":
-                a = np.asarray(next(it), dtype=np.float64)
+                a = np.asarray(next(it), dtype=ft)
                 if a.ndim != n[2]:
                     raise ValueError(f"input node {i}: rank {a.ndim} != declared {n[2]}")
                 vals[i] = a
@@ -164,10 +176,10 @@ def evaluate(nodes, inputs, params=()):
             elif kind == "scalar":
                 s = n[3]
                 # the scalar is an fp32 immediate widened exactly (Table 1, Adds/Muls)
-                s = float(np.float32(params[s[1]] if isinstance(s, tuple) else s))
+                s = ft(np.float32(params[s[1]] if isinstance(s, tuple) else s))
                 vals[i] = vals[n[2]] + s if n[1] == "adds" else vals[n[2]] * s
             elif kind == "cast":
-                vals[i] = _round_to(vals[n[1]], n[2])
+                vals[i] = _round_to(vals[n[1]], n[2]).astype(ft)
             elif kind == "reduce":
                 axis = n[3] if len(n) > 3 else -1
                 if not (-vals[n[2]].ndim <= axis <= -1):
@@ -176,12 +188,12 @@ def evaluate(nodes, inputs, params=()):
             elif kind == "matmul":
                 vals[i] = np.matmul(vals[n[1]], vals[n[2]])
             elif kind == "compare":
-                vals[i] = _COMPARE[n[1]](*np.broadcast_arrays(vals[n[2]], vals[n[3]]))
+                vals[i] = _COMPARE[n[1]](*np.broadcast_arrays(vals[n[2]], vals[n[3]])).astype(ft)
             elif kind == "select":                   # Table 1, Select: cond ? x : y, cond = (value != 0)
                 c, x, y = np.broadcast_arrays(vals[n[1]], vals[n[2]], vals[n[3]])
                 vals[i] = np.where(c != 0, x, y)
             elif kind == "output":
-                outs.append(np.array(vals[n[1]], dtype=np.float64))
+                outs.append(np.array(vals[n[1]], dtype=ft))
             else:
                 raise ValueError(f"unknown node kind {kind}")
     return outs

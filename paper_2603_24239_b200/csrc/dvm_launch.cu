@@ -5,17 +5,19 @@
 #include <string.h>
 
 #include <mutex>
+#include <unordered_map>
 
 #include "../../include/dvm.h"
 #include "dvm_format.h"
 #include "dvm_internal.h"
 #include "dvm_launch.h"
 #include "dvm_vm.cuh"
+#include "dvm_vm_variants.h"
 
 namespace {
 
-constexpr int PW_SMALL = 496;    // words of code in a 2 KB parameter block
-constexpr int PW_LARGE = 8000;   // ... in a 32 KB parameter block (the sm_70+ limit is 32764 bytes)
+constexpr int PW_SMALL = DVM_PW_SMALL;
+constexpr int PW_LARGE = DVM_PW_LARGE;
 constexpr int QUEUE_SLOTS = 504;
 constexpr size_t SCRATCH_BYTES = (8 + 4 * QUEUE_SLOTS) * sizeof(unsigned int);
 constexpr int MAX_DEVICES = 64;
@@ -25,8 +27,9 @@ struct DeviceState {
   bool ready = false;
   unsigned int* scratch = nullptr;  // [0] status word, [8 + 4*slot] work-queue counters (next tile, CTAs finished, tiles completed)
   int sm_count = 0;
-  int occ[3][2][DVM_MAX_LOCAL_UNITS + 1];  // resident CTAs per SM for [V: 16, 32, 24][large parameter block][local units], 0 = not yet asked
-  int occ_levels[2][2][DVM_MAX_LOCAL_UNITS + 1];  // the same for the variants with level waits
+  // resident CTAs per SM, per (kernel variant, bytes of dynamic shared memory / DVM_LOCAL_UNIT): occupancy depends
+  // on exactly these two, so a one-slot and a two-slot launch of the same program never share an entry
+  std::unordered_map<uint64_t, int> occ;
   unsigned queue_slot = 0;
 };
 
@@ -34,50 +37,6 @@ DeviceState g_dev[MAX_DEVICES];
 std::mutex g_mu;
 thread_local int t_last_cuda_error = 0;
 long long g_launches = 0;
-
-
-template <int V, int PW>
-int occupancy(int* out, size_t smem) {
-  int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<V, PW, false, 2>, dvm::THREADS, smem));
-  *out = n > 0 ? n : 1;
-  return DVM_OK;
-}
-
-// 24 elements per thread exist as the one-program basic variant only (rows that fill three quarters of a
-// 32-element tile).
-template <int PW>
-int occupancy24(int* out, size_t smem) {
-  int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<24, PW, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dvm::dvm_vm_kernel<24, PW, true, 0>, dvm::THREADS, smem));
-  *out = n > 0 ? n : 1;
-  return DVM_OK;
-}
-
-// The variant with level waits: its grid must not exceed what the device keeps resident, so it is asked itself.
-template <int V, int PW>
-int occupancy_levels(int* out, size_t smem) {
-  int n = 0;
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  DVM_CUDA(cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, false, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem));
-  int a = 0, b = 0, c = 0;
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, dvm::dvm_vm_kernel<V, PW, false, 0, true>, dvm::THREADS, smem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, dvm::dvm_vm_kernel<V, PW, false, 1, true>, dvm::THREADS, smem));
-  DVM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c, dvm::dvm_vm_kernel<V, PW, false, 2, true>, dvm::THREADS, smem));
-  n = a < b ? a : b;
-  n = n < c ? n : c;
-  if (n <= 0) return DVM_ERR_TOO_LARGE;  // not even one CTA fits: no launch
-  *out = n;
-  return DVM_OK;
-}
 
 }  // namespace
 
@@ -91,8 +50,6 @@ int dvm_device_state(DvmDeviceInfo* info) {
     DVM_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
     DVM_CUDA(cudaMalloc(&d.scratch, SCRATCH_BYTES));
     DVM_CUDA(cudaMemset(d.scratch, 0, SCRATCH_BYTES));
-    memset(d.occ, 0, sizeof d.occ);
-    memset(d.occ_levels, 0, sizeof d.occ_levels);
     d.ready = true;
   }
   info->scratch = d.scratch;
@@ -102,32 +59,53 @@ int dvm_device_state(DvmDeviceInfo* info) {
   return DVM_OK;
 }
 
-// Resident CTAs per SM of the interpreter for a launch with `units` local-memory units (cached per device).
-static int dvm_occupancy(int V, bool large, int units, size_t smem, int* out, bool levels = false) {
+// The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
+DVM_GROUPS(DVM_DECL_GROUP)
+#undef DVM_DECL_GROUP
+
+const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels) {
+  typedef const DvmVmVariant* (*GroupFn)(int*);
+#define DVM_GROUP_FN(g) &dvm_vm_group_##g,
+  static const GroupFn groups[] = {DVM_GROUPS(DVM_GROUP_FN)};
+#undef DVM_GROUP_FN
+  for (GroupFn g : groups) {
+    int n = 0;
+    const DvmVmVariant* v = g(&n);
+    for (int i = 0; i < n; ++i)
+      if (v[i].V == V && v[i].large == (int)large && v[i].single == (int)single && v[i].ext == ext && v[i].levels == (int)levels)
+        return &v[i];
+  }
+  return nullptr;
+}
+
+// Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
+uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
+  const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
+                      ((uint64_t)v->levels << 12);
+  return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
+}
+
+// Resident CTAs per SM of one interpreter variant for a launch with `smem` bytes of dynamic shared memory
+// (cached per device).  The variants with level waits rely on the whole grid being resident: no CTA fits -> no launch.
+static int dvm_occupancy(const DvmVmVariant* v, size_t smem, int* out) {
   int dev = 0;
   DVM_CUDA(cudaGetDevice(&dev));
   std::lock_guard<std::mutex> lk(g_mu);
   DeviceState& d = g_dev[dev];
-  if (levels) {
-    int& lslot = d.occ_levels[V == 32 ? 1 : 0][large ? 1 : 0][units];
-    if (lslot == 0) {
-      int st;
-      if (V == 32) st = large ? occupancy_levels<32, PW_LARGE>(&lslot, smem) : occupancy_levels<32, PW_SMALL>(&lslot, smem);
-      else st = large ? occupancy_levels<16, PW_LARGE>(&lslot, smem) : occupancy_levels<16, PW_SMALL>(&lslot, smem);
-      if (st != DVM_OK) return st;
+  const uint64_t key = dvm_occupancy_key(v, smem);
+  auto it = d.occ.find(key);
+  if (it == d.occ.end()) {
+    int n = 0;
+    DVM_CUDA(v->occupancy(smem, kMaxDynSmem, &n));
+    if (n <= 0) {
+      if (v->levels) return DVM_ERR_TOO_LARGE;
+      n = 1;
     }
-    *out = lslot;
-    return DVM_OK;
+    it = d.occ.emplace(key, n).first;
   }
-  int& slot = d.occ[V == 32 ? 1 : (V == 24 ? 2 : 0)][large ? 1 : 0][units];
-  if (slot == 0) {
-    int st;
-    if (V == 24) st = large ? occupancy24<PW_LARGE>(&slot, smem) : occupancy24<PW_SMALL>(&slot, smem);
-    else if (V == 32) st = large ? occupancy<32, PW_LARGE>(&slot, smem) : occupancy<32, PW_SMALL>(&slot, smem);
-    else st = large ? occupancy<16, PW_LARGE>(&slot, smem) : occupancy<16, PW_SMALL>(&slot, smem);
-    if (st != DVM_OK) return st;
-  }
-  *out = slot;
+  *out = it->second;
   return DVM_OK;
 }
 
@@ -205,48 +183,27 @@ int prefill_combined(const uint32_t* code, void* const* tensors, cudaStream_t st
   return DVM_OK;
 }
 
-// One kernel variant per (elements per thread, parameter-block size, single program, extension level).
-template <int PW, int EXT>
-void launch_variant_ext(int V, bool single, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
-  if (V == 32) {
-    if (single) dvm::dvm_vm_kernel<32, PW, true, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<32, PW, false, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
-  } else {
-    if (single) dvm::dvm_vm_kernel<16, PW, true, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<16, PW, false, EXT><<<grid, dvm::THREADS, smem, stream>>>(prm);
+int prefill_all(int n_programs, const void* const* codes, void* const* const* tensors, cudaStream_t stream) {
+  for (int i = 0; i < n_programs; ++i) {
+    const uint32_t* c = (const uint32_t*)codes[i];
+    if (!((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS)) continue;
+    int st = prefill_combined(c, tensors[i], stream);
+    if (st != DVM_OK) return st;
   }
+  return DVM_OK;
 }
 
-template <int PW>
-int launch_variant(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
-  const bool single = prm.n_programs == 1 && !prm.use_queue;
-  if (V == 24) {
-    if (!single || ext != 0) return DVM_ERR_UNSUPPORTED;  // encoded for a launch of its own on the basic variant
-    dvm::dvm_vm_kernel<24, PW, true, 0><<<grid, dvm::THREADS, smem, stream>>>(prm);
-  } else if (ext >= 2) launch_variant_ext<PW, 2>(V, single, prm, grid, smem, stream);
-  else if (ext == 1) launch_variant_ext<PW, 1>(V, single, prm, grid, smem, stream);
-  else launch_variant_ext<PW, 0>(V, single, prm, grid, smem, stream);
-  DVM_CUDA(cudaGetLastError());
+// Starts one interpreter variant on `grid` CTAs.
+int launch_variant(const DvmVmVariant* v, const void* params, int grid, size_t smem, cudaStream_t stream) {
+  DVM_CUDA(v->launch(params, grid, smem, stream));
   dvm_count_launch();
   return DVM_OK;
 }
 
-// The variants with level waits.
-template <int PW>
-int launch_variant_levels(int V, int ext, const dvm::VMParams<PW>& prm, int grid, size_t smem, cudaStream_t stream) {
-  if (V == 24) return DVM_ERR_UNSUPPORTED;
-  if (V == 32) {
-    if (ext >= 2) dvm::dvm_vm_kernel<32, PW, false, 2, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else if (ext == 1) dvm::dvm_vm_kernel<32, PW, false, 1, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<32, PW, false, 0, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-  } else {
-    if (ext >= 2) dvm::dvm_vm_kernel<16, PW, false, 2, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else if (ext == 1) dvm::dvm_vm_kernel<16, PW, false, 1, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-    else dvm::dvm_vm_kernel<16, PW, false, 0, true><<<grid, dvm::THREADS, smem, stream>>>(prm);
-  }
-  DVM_CUDA(cudaGetLastError());
-  dvm_count_launch();
-  return DVM_OK;
+// The variant a launch needs: 24 elements per thread exist as the one-program basic variant only.
+const DvmVmVariant* pick_variant(int V, bool large, bool single, int ext, bool levels) {
+  if (levels) single = false;
+  return dvm_vm_find_variant(V, large, single, ext, levels);
 }
 
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
@@ -297,10 +254,6 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     }
     st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
     if (st != DVM_OK) return st;
-    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) {
-      st = prefill_combined(c, tensors[i], stream);
-      if (st != DVM_OK) return st;
-    }
     pos += c[DVM_H_TOTAL_WORDS];
     tb += c[DVM_H_N_TILES];
   }
@@ -317,20 +270,24 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   const size_t smem = ((one_slot ? 1 : 2) * (size_t)units + 1) * DVM_LOCAL_UNIT;  // one spare unit, two tile slots (or one)
   P.slot_bytes = one_slot ? 0u : units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
+  const bool single = n_programs == 1 && !use_queue;
+  const DvmVmVariant* variant = pick_variant(V, large, single, ext, level != nullptr);
+  if (!variant) return DVM_ERR_UNSUPPORTED;  // (24 elements per thread: encoded for a launch of its own on the basic variant)
   int occ = 0;
-  // (the occupancy cache is keyed by the units of two slots: a one-slot launch asks under half its units)
-  st = dvm_occupancy(V, large, one_slot ? ((int)units + 1) / 2 : (int)units, smem, &occ, level != nullptr);
+  st = dvm_occupancy(variant, smem, &occ);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
   int grid = (int)(total_tiles < slots ? total_tiles : slots);
+  // Everything is placed and checked: only now touch the caller's memory.  Results that tiles combine
+  // atomically are filled with their identity (one small kernel per such output), then the interpreter starts.
+  st = prefill_all(n_programs, codes, tensors, stream);
+  if (st != DVM_OK) return st;
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
-    if (level) return launch_variant_levels<PW_SMALL>(V, ext, S, grid, smem, stream);
-    return launch_variant<PW_SMALL>(V, ext, S, grid, smem, stream);
+    return launch_variant(variant, &S, grid, smem, stream);
   }
-  if (level) return launch_variant_levels<PW_LARGE>(V, ext, P, grid, smem, stream);
-  return launch_variant<PW_LARGE>(V, ext, P, grid, smem, stream);
+  return launch_variant(variant, &P, grid, smem, stream);
 }
 
 }  // namespace
@@ -548,10 +505,6 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     P.words[n_programs + i] = tb;
     st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
     if (st != DVM_OK) return st;
-    if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) {
-      st = prefill_combined(c, tensors[i], stream);
-      if (st != DVM_OK) return st;
-    }
     pos += c[DVM_H_TOTAL_WORDS];
     tb += c[DVM_H_N_TILES];
   }
@@ -567,17 +520,21 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool large = pos > PW_SMALL;
+  const DvmVmVariant* variant = pick_variant(V, large, false, ext, false);
+  if (!variant) return DVM_ERR_UNSUPPORTED;
   int occ = 0;
-  st = dvm_occupancy(V, large, (int)units, smem, &occ);
+  st = dvm_occupancy(variant, smem, &occ);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
   int grid = (int)(total_tiles < slots ? total_tiles : slots);
   // every call shares the array and it keeps the last call's contents: the queue counters must start at zero
   DVM_CUDA(cudaMemsetAsync(dev.scratch, 0, NOALLOC_WORDS * sizeof(unsigned int), stream));
+  st = prefill_all(n_programs, codes, tensors, stream);
+  if (st != DVM_OK) return st;
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
-    return launch_variant<PW_SMALL>(V, ext, S, grid, smem, stream);
+    return launch_variant(variant, &S, grid, smem, stream);
   }
-  return launch_variant<PW_LARGE>(V, ext, P, grid, smem, stream);
+  return launch_variant(variant, &P, grid, smem, stream);
 }

@@ -110,7 +110,7 @@ __device__ __forceinline__ bool vm_mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait (2 s of %globaltimer, and a poll cap): false when it ran out.
-__device__ __noinline__ bool vm_mbar_wait_slow(uint32_t bar, uint32_t parity) {
+static __device__ __noinline__ bool vm_mbar_wait_slow(uint32_t bar, uint32_t parity) {
   unsigned long long t0, t1;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
   for (uint32_t spin = 0; spin < (1u << 27); ++spin) {
@@ -126,7 +126,7 @@ __device__ __forceinline__ bool vm_mbar_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait until the grid-wide counter of completed tiles has reached `need` (acquire: what those tiles
 // stored is visible afterwards).  Same limits as the barrier wait; false when it ran out.
-__device__ __noinline__ bool vm_wait_tiles_done(const unsigned int* counter, uint32_t need) {
+static __device__ __noinline__ bool vm_wait_tiles_done(const unsigned int* counter, uint32_t need) {
   unsigned long long t0, t1;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
   for (uint32_t spin = 0; spin < (1u << 27); ++spin) {

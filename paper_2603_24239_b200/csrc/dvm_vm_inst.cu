@@ -1,0 +1,52 @@
+// Instantiations of the interpreter kernel, one group per compilation of this file (-DDVM_INST_GROUP=g):
+// group g < 12: V = 16 (g < 6) or 32, parameter block small (g % 6 < 3) or large, extension level g % 3,
+// each with the one-program, the stacked and the level-wait variant; group 12: the 24-element one-program
+// basic variants.
+#include "dvm_vm.cuh"
+#include "dvm_vm_variants.h"
+
+#ifndef DVM_INST_GROUP
+#error "compile with -DDVM_INST_GROUP=<0..12>"
+#endif
+
+namespace {
+
+template <int V, int PW, bool SINGLE, int EXT, bool LEVELS>
+struct Ops {
+  static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
+    dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>
+        <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
+    return cudaGetLastError();
+  }
+  static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>,
+                                                         dvm::THREADS, smem);
+  }
+};
+
+#define DVM_ENTRY(V, LARGE, SINGLE, EXT, LEVELS)                                       \
+  {V, LARGE, SINGLE, EXT, LEVELS,                                                     \
+   &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::launch, \
+   &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::occupancy}
+
+#if DVM_INST_GROUP < 12
+constexpr int GV = DVM_INST_GROUP < 6 ? 16 : 32;
+constexpr int GL = (DVM_INST_GROUP % 6) < 3 ? 0 : 1;
+constexpr int GE = DVM_INST_GROUP % 3;
+const DvmVmVariant kGroup[] = {DVM_ENTRY(GV, GL, 1, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 1)};
+#else
+const DvmVmVariant kGroup[] = {DVM_ENTRY(24, 0, 1, 0, 0), DVM_ENTRY(24, 1, 1, 0, 0)};
+#endif
+
+}  // namespace
+
+#define DVM_CAT_(a, b) a##b
+#define DVM_CAT(a, b) DVM_CAT_(a, b)
+// each group exports its table under a name of its own: dvm_vm_group_<g>(&count)
+const DvmVmVariant* DVM_CAT(dvm_vm_group_, DVM_INST_GROUP)(int* count) {
+  *count = (int)(sizeof(kGroup) / sizeof(kGroup[0]));
+  return kGroup;
+}

@@ -25,3 +25,19 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """Strict elementwise statistics of the programs gated by the row-scaled error only (reported, not gated)."""
+    try:
+        from tests.parity_util import STRICT_REPORT
+    except Exception:
+        return
+    if not STRICT_REPORT:
+        return
+    tr = terminalreporter
+    tr.section("strict elementwise error vs the fp64 oracle (reported, not gated)")
+    tr.write_line("label                               n        R     strict max  n > R   well-cond.  of them > R  max there")
+    for st in STRICT_REPORT:
+        tr.write_line(f"{st['label'][:34]:34s} {st['n']:9d} {st['r']:.0e}  {st['strict_max']:10.3e} {st['n_over']:7d} "
+                      f"{st['n_well']:10d} {st['n_over_well']:11d}  {st['well_max']:.3e}")

@@ -1,7 +1,8 @@
 """Helpers shared by the parity tests: run a program through the C-ABI on the GPU,
 evaluate the same inputs with the CPU oracle, and apply the tolerance gates.
 
-Gates (derivation in DESIGN.md, "Tolerances"):
+Gates (strict elementwise relative error is out of reach of any fp32 evaluation where a program cancels --
+exp(ab+c)-a, x-mean, x*w+b -- so the first gate scales by the row maximum):
   G1  |g - o| <= R * max(|o|, max_j |o_row_j|)   every program, every element
   G2  |g - o| <= R * |o|                          programs without subtractive cancellation
   G3  exact                                       structural zeros / integer outputs
@@ -67,6 +68,46 @@ def gate_errors(got: np.ndarray, want: np.ndarray):
         g1 = np.where(diff == 0, 0.0, diff / den1)
         g2 = np.where(diff == 0, 0.0, diff / absw)
     return float(np.max(g1)), float(np.max(g2))
+
+
+# Statistics reported beside the gates for the programs whose strict elementwise error no fp32 evaluation can
+# bound (C1, C4 GELU, C4 LayerNorm, C5): filled by the tests, printed in pytest's terminal summary.
+STRICT_REPORT = []
+
+
+def strict_stats(got, want, want_fp32, r):
+    """Strict elementwise relative error of `got` against the float64 oracle `want`: its maximum, how many
+    elements exceed r, and how many of those lie among the elements a faithful fp32 evaluation already gets
+    right (|o32 - o64| <= 1e-6 |o64|: "well conditioned").  Reported, not gated: the row-scaled gate cannot see
+    a small output that was zeroed, this count can."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    want = np.asarray(want, dtype=np.float64).reshape(-1)
+    w32 = np.asarray(want_fp32, dtype=np.float64).reshape(-1)
+    fin = np.isfinite(want) & (want != 0)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        rel = np.where(fin, np.abs(got - want) / np.abs(want), 0.0)
+        well = fin & (np.abs(w32 - want) <= 1e-6 * np.abs(want))
+    over = rel > r
+    return {"n": int(want.size), "strict_max": float(rel.max()) if want.size else 0.0, "n_over": int(over.sum()),
+            "n_well": int(well.sum()), "n_over_well": int((over & well).sum()),
+            "well_max": float(rel[well].max()) if well.any() else 0.0}
+
+
+def record_strict(label, prog, got_list, inputs, params=(), want_list=None):
+    """Computes strict_stats for every output of a program run and appends them to STRICT_REPORT."""
+    r = R_TOL[program_dtype(prog)]
+    ins64 = [wl.to_f64(t) for t in inputs]
+    if want_list is None:
+        want_list = orc.evaluate(prog.nodes, ins64, params)
+    want32 = orc.evaluate(prog.nodes, ins64, params, diagnostic_fp32=True)
+    out = []
+    for g, w, w32 in zip(got_list, want_list, want32):
+        st = strict_stats(wl.to_f64(g) if isinstance(g, torch.Tensor) else g, w, w32, r)
+        st["label"] = label
+        st["r"] = r
+        STRICT_REPORT.append(st)
+        out.append(st)
+    return out
 
 
 def check(prog, got_list, want_list, strict=False, tol=None):

@@ -6,7 +6,7 @@ import torch
 
 import dvm_workloads as wl
 import paper_2603_24239_b200 as dvm
-from tests.parity_util import check, gpu_run, oracle_run
+from tests.parity_util import check, gpu_run, oracle_run, record_strict
 
 pytestmark = pytest.mark.gpu
 
@@ -19,7 +19,11 @@ def _run(prog, inputs, params=(), strict=False):
 
 def test_c1_exact_config():
     """Config 1: out = exp(a*b + c) - a, fp32 [7, 1531], seed 0."""
-    _run(wl.program_c1(), wl.inputs_c1())
+    ins = wl.inputs_c1()
+    _, outs, want = _run(wl.program_c1(), ins)
+    st = record_strict("c1 exp(a*b+c)-a [7,1531]", wl.program_c1(), outs, ins, want_list=want)[0]
+    # where fp32 evaluation is well conditioned the device must be right as well: nothing small is zeroed or lost
+    assert st["n_well"] > 0.9 * st["n"] and st["well_max"] <= 1e-4
 
 
 @pytest.mark.parametrize("shape", [(1, 1), (1, 3), (3, 1), (5, 1023), (5, 1024), (5, 1025), (2, 4097),

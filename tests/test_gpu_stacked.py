@@ -4,7 +4,7 @@ import torch
 
 import dvm_workloads as wl
 import paper_2603_24239_b200 as dvm
-from tests.parity_util import check, oracle_run
+from tests.parity_util import record_strict, check, oracle_run
 
 pytestmark = pytest.mark.gpu
 
@@ -31,9 +31,15 @@ def _stack(items, seed0):
     return codes, tls, meta
 
 
-def _check_all(meta):
-    for prog, ins, params, out, kind in meta:
-        check(prog, [out], oracle_run(prog, ins, params), strict=(kind == "sigmoid_mul"))
+def _check_all(meta, report=None):
+    for j, (prog, ins, params, out, kind) in enumerate(meta):
+        want = oracle_run(prog, ins, params)
+        check(prog, [out], want, strict=(kind == "sigmoid_mul"))
+        if report and kind != "sigmoid_mul":
+            st = record_strict(f"{report} #{j} {kind} {tuple(out.shape)}", prog, [out], ins, params, want_list=want)[0]
+            # elements a faithful fp32 evaluation gets right must not be lost by the device (the row-scaled gate
+            # alone would not notice a small output that was zeroed)
+            assert st["well_max"] <= 1e-3, st
 
 
 def test_stacked_small_mix():
@@ -60,7 +66,7 @@ def test_stacked_config4_launches(min_ctas, launch):
     dvm.launch_stacked(codes, tls)
     assert dvm.last_device_status() == 0
     assert dvm.launch_count() - n0 == 1
-    _check_all(meta)
+    _check_all(meta, report=f"c4 launch {launch}" if (min_ctas, launch) == (2, 0) else None)
 
 
 def test_stacked_repeated_launches_reuse_queue():
