@@ -924,6 +924,8 @@ def main():
     ap.add_argument("--max-rows", type=int, default=0, help="cap rows per instance (small profiling case)")
     ap.add_argument("--elems-per-thread", type=int, default=0, help="fix the encoder's elements per thread (16/32/64; 0 = cost model)")
     ap.add_argument("--encode-reps", type=int, default=1000, help="repeats per instance of the host-encode latency measurement")
+    ap.add_argument("--general-interpreter", action="store_true",
+                    help="run every launch on the general interpreter instead of the lean one (for comparisons)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--detail", default="", help="write per-instance timings to this JSON file")
@@ -950,6 +952,8 @@ def main():
     kw = {}
     if args.elems_per_thread:
         dvm.set_elems_per_thread(args.elems_per_thread)
+    if args.general_interpreter:
+        dvm.set_lean_kernel(False)
     if args.instances:
         kw = {"n_launches": args.instances} if args.workload == "c4" else {"n_instances": args.instances}
     if args.max_rows and args.workload in ("c2", "c5", "addmm"):

@@ -81,6 +81,7 @@ _sig = {
     "dvm_get_elems_per_thread": ([], _i),
     "dvm_set_min_resident_ctas": ([_i], None),
     "dvm_get_min_resident_ctas": ([], _i),
+    "dvm_set_lean_kernel": ([_i], None),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -544,6 +545,12 @@ def get_num_cores() -> int:
 
 def set_elems_per_thread(v: int):
     lib.dvm_set_elems_per_thread(v)
+
+
+def set_lean_kernel(on: bool):
+    """False: every launch runs on the general interpreter (for comparisons); True (default): programs of the
+    basic instruction set run on the lean variant."""
+    lib.dvm_set_lean_kernel(int(on))
 
 
 def set_min_resident_ctas(n: int):

@@ -13,6 +13,7 @@
 #include "dvm_launch.h"
 #include "dvm_vm.cuh"
 #include "dvm_vm_variants.h"
+#include "dvm_link.h"
 
 namespace {
 
@@ -37,6 +38,7 @@ DeviceState g_dev[MAX_DEVICES];
 std::mutex g_mu;
 thread_local int t_last_cuda_error = 0;
 long long g_launches = 0;
+int g_use_lean = 1;  // dvm_set_lean_kernel(0): every launch runs on the general interpreter (for comparisons)
 
 }  // namespace
 
@@ -60,12 +62,12 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
 
-const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels) {
+const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy) {
   typedef const DvmVmVariant* (*GroupFn)(int*);
 #define DVM_GROUP_FN(g) &dvm_vm_group_##g,
   static const GroupFn groups[] = {DVM_GROUPS(DVM_GROUP_FN)};
@@ -74,7 +76,8 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
     int n = 0;
     const DvmVmVariant* v = g(&n);
     for (int i = 0; i < n; ++i)
-      if (v[i].V == V && v[i].large == (int)large && v[i].single == (int)single && v[i].ext == ext && v[i].levels == (int)levels)
+      if (v[i].V == V && v[i].large == (int)large && v[i].single == (int)single && v[i].ext == ext &&
+          v[i].levels == (int)levels && v[i].lean == lean && (!lean || v[i].heavy == (int)heavy))
         return &v[i];
   }
   return nullptr;
@@ -83,7 +86,7 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
 // Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
 uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
   const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
-                      ((uint64_t)v->levels << 12);
+                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 14);
   return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
 }
 
@@ -112,6 +115,7 @@ static int dvm_occupancy(const DvmVmVariant* v, size_t smem, int* out) {
 void dvm_note_cuda_error(int e) { t_last_cuda_error = e; }
 void dvm_count_launch() { __atomic_add_fetch(&g_launches, 1, __ATOMIC_RELAXED); }
 
+extern "C" void dvm_set_lean_kernel(int on) { g_use_lean = on; }
 extern "C" int dvm_last_cuda_error(void) { return t_last_cuda_error; }
 extern "C" int64_t dvm_launch_count(void) { return (int64_t)__atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
 
@@ -160,6 +164,198 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   return DVM_OK;
 }
 
+
+// ---- the linker of the lean interpreter (see dvm_link.h) ----
+// Turns the placed copy of one verified vector program at dst (word index `at` of the parameter block) into its
+// linked form: header, tables and load section stay, the compute section is replaced by records (which start at
+// a word index = 2 mod 4 of the block: 16-byte aligned in the kernel's parameter space).  `src` is the encoded
+// program, `tensors` its device pointers, `max_words` the room at dst.  Returns the words the linked program
+// takes, or 0 when it cannot be linked (no room, or an instruction only the general interpreter has).
+uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const uint32_t* src, void* const* tensors) {
+  const uint32_t counts = src[DVM_H_COUNTS], geom = src[DVM_H_GEOM];
+  const uint32_t nt = counts & 0xff, n_opd = (counts >> 16) & 0xff, nreg = (geom >> 16) & 0xff;
+  const uint32_t tables = DVM_HDR_WORDS + 2 * nt + n_opd * DVM_OPD_WORDS + nreg;
+  const uint32_t load_words = src[DVM_H_LOAD_WORDS], code_words = src[DVM_H_CODE_WORDS];
+  const uint32_t head = tables + load_words;  // header, tables and load section: copied as they are
+  if (n_opd > 63) return 0;
+  const uint32_t* ot = src + DVM_HDR_WORDS + 2 * nt;
+  const uint32_t* lt = dst + DVM_HDR_WORDS + 2 * nt + n_opd * DVM_OPD_WORDS;  // (the placed table: address phases patched in)
+  const uint32_t* body = src + tables;
+  const uint32_t scalar_unit = src[DVM_H_LOCAL2] & 0xffffu;
+  struct Rec { uint32_t w[4]; };
+  Rec rec[8 * DVM_MAX_NODES + 72];
+  uint32_t n = 0;
+  auto push = [&](uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+    rec[n].w[0] = w0; rec[n].w[1] = w1; rec[n].w[2] = w2; rec[n].w[3] = w3;
+    ++n;
+  };
+  auto f2u = [](float f) { uint32_t u; memcpy(&u, &f, 4); return u; };
+  auto u2f = [](uint32_t u) { float f; memcpy(&f, &u, 4); return f; };
+  // every output of the program is bf16: the one-piece exponential is accurate enough
+  bool fast = true;
+  for (uint32_t o = n_opd - (counts >> 24); o < n_opd; ++o)
+    if (((ot[o * DVM_OPD_WORDS + DVM_OPD_INFO] >> 8) & 0xff) != DVM_DT_BF16) fast = false;
+  // operand word of local register k holding elements of type dt
+  auto opw = [&](uint32_t k, uint32_t dt, int* kind) -> uint32_t {
+    const uint32_t lw = lt[k];
+    const uint32_t mode = (lw >> 16) & 0xf;
+    *kind = mode == DVM_LM_PRIVATE ? 2 : (dt == DVM_DT_BF16 ? 0 : 1);
+    return DVM_LK_OPW((lw & 0xffffu) * DVM_LOCAL_UNIT, mode, dt == DVM_DT_BF16 ? 0 : 1, (lw >> 20) & 0xfu, lw >> 24);
+  };
+  const float one = 1.0f, neg_one = -1.0f, neg_zero = -0.0f;
+  for (uint32_t pc = load_words; pc < code_words;) {
+    if (n + 4 > sizeof rec / sizeof rec[0]) return 0;
+    const uint32_t w0 = body[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0) ? DVM_INSN_LEN(w0) : 1;
+    const uint32_t ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
+    const uint32_t cls = op >> 3;
+    int kind = 0;
+    if (op == DVM_OP_LDA) {
+      const uint32_t ow = opw(ia, ib, &kind);
+      push(DVM_LK_W0(DVM_LK_LDA_BF16 + kind, 0, 0, 0), ow, 0, 0);
+    } else if (cls == (DVM_OP_LD2 >> 3)) {
+      const uint32_t ox = opw(ia, (ib >> 6) & 1, &kind);
+      push(DVM_LK_W0(DVM_LK_LDA_BF16 + kind, 0, 0, 0), ox, 0, 0);
+      const uint32_t oy = opw(ib & 0x3f, (ib >> 7) & 1, &kind);
+      push(DVM_LK_W0(DVM_LK_BIN_BF16 + kind, op & 7, 0, 0), oy, 0, 0);
+    } else if (cls == (DVM_OP_BIN >> 3)) {
+      if (ia == DVM_REG_ACC) {
+        push(DVM_LK_W0(DVM_LK_BIN_ACC, op & 7, 0, 0), 0, 0, 0);
+      } else {
+        const uint32_t oy = opw(ia, ib, &kind);
+        push(DVM_LK_W0(DVM_LK_BIN_BF16 + kind, op & 7, 0, 0), oy, 0, 0);
+      }
+    } else if (cls == (DVM_OP_BINI >> 3)) {
+      const float y = u2f(body[pc + 1]);
+      switch (op & 7) {  // ACC * m + c (a product plus -0 is the product, sign of zero included)
+        case DVM_A_ADD: push(DVM_LK_W0(DVM_LK_FMA, 0, 0, 0), f2u(one), f2u(y), 0); break;
+        case DVM_A_SUB: push(DVM_LK_W0(DVM_LK_FMA, 0, 0, 0), f2u(one), f2u(-y), 0); break;
+        case DVM_A_RSUB: push(DVM_LK_W0(DVM_LK_FMA, 0, 0, 0), f2u(neg_one), f2u(y), 0); break;
+        case DVM_A_MUL: push(DVM_LK_W0(DVM_LK_FMA, 0, 0, 0), f2u(y), f2u(neg_zero), 0); break;
+        case DVM_A_DIV: push(DVM_LK_W0(DVM_LK_FMA, 4, 0, 0), f2u(y), f2u(neg_zero), 0); break;  // the device's reciprocal, as for S[a]
+        default: push(DVM_LK_W0(DVM_LK_BINI, op & 7, 0, 0), body[pc + 1], 0, 0); break;
+      }
+    } else if (cls == (DVM_OP_BINS >> 3)) {
+      // ACC = ACC - S[a] ; exp  ->  EXPS
+      const uint32_t nx = pc + len < code_words ? body[pc + len] : 0;
+      if ((op & 7) == DVM_A_SUB && pc + len < code_words && DVM_INSN_OP(nx) == DVM_OP_UN + DVM_U_EXP) {
+        push(DVM_LK_W0(DVM_LK_EXPS, fast ? 1 : 0, ia, 0), 0, 0, 0);
+        pc += 1;  // (the unary has one word)
+      } else {
+        switch (op & 7) {
+          case DVM_A_ADD: push(DVM_LK_W0(DVM_LK_FMA, 2, 0, ia), f2u(one), 0, 0); break;
+          case DVM_A_SUB: push(DVM_LK_W0(DVM_LK_FMA, 2 | 8, 0, ia), f2u(one), 0, 0); break;
+          case DVM_A_RSUB: push(DVM_LK_W0(DVM_LK_FMA, 2, 0, ia), f2u(neg_one), 0, 0); break;
+          case DVM_A_MUL: push(DVM_LK_W0(DVM_LK_FMA, 1, ia, 0), 0, f2u(neg_zero), 0); break;
+          case DVM_A_DIV: push(DVM_LK_W0(DVM_LK_FMA, 1 | 4, ia, 0), 0, f2u(neg_zero), 0); break;
+          default: push(DVM_LK_W0(DVM_LK_BINS, op & 7, ia, 0), 0, 0, 0); break;
+        }
+      }
+    } else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
+      const uint32_t u = op - DVM_OP_UN;
+      if (u == DVM_U_ISFINITE) return 0;
+      push(DVM_LK_W0(DVM_LK_UN, u | ((fast && (u == DVM_U_EXP || u == DVM_U_SIGMOID)) ? 0x80u : 0u), 0, 0), 0, 0, 0);
+    } else if (cls == (DVM_OP_RED >> 3)) {
+      // RED ; SOP fma(-unary) that reads the result and overwrites it  ->  one reduction with a post-operation
+      const uint32_t nx = pc + len < code_words ? body[pc + len] : 0;
+      bool fused = false;
+      if (pc + len < code_words && DVM_INSN_OP(nx) == DVM_OP_SOP && DVM_INSN_B(nx) == DVM_SK_FMAU) {
+        const uint32_t w1 = body[pc + len + 1];
+        if (((w1 >> 8) & 0xff) == ia && DVM_INSN_A(nx) == ia) {
+          push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, 1), w1 & 0xff, body[pc + len + 2], body[pc + len + 3]);
+          pc += DVM_INSN_LEN(nx);
+          fused = true;
+        }
+      }
+      if (!fused) push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, 0), 0, 0, 0);
+    } else if (op == DVM_OP_STG) {
+      const uint32_t info = ot[ib * DVM_OPD_WORDS + DVM_OPD_INFO];
+      if (!((info >> 25) & 1u) || ((info >> 26) & 3u)) return 0;  // a stored view / a combined result: general interpreter
+      const unsigned long long a = (unsigned long long)(uintptr_t)tensors[info & 0xff];
+      push(DVM_LK_W0(DVM_LK_STG, 0, ((info >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2, 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
+    } else if (op == DVM_OP_STA) {
+      push(DVM_LK_W0(DVM_LK_STA, 0, 0, 0), (lt[ia] & 0xffffu) * DVM_LOCAL_UNIT, 0, 0);
+    } else if (op == DVM_OP_LSS) {
+      push(DVM_LK_W0(DVM_LK_LSS, 0, ia, 0), scalar_unit * DVM_LOCAL_UNIT + (ib >> 2) * (DVM_VM_THREADS * 16) + (ib & 3) * 4, 0, 0);
+    } else if (op == DVM_OP_STS) {
+      push(DVM_LK_W0(DVM_LK_STS, 0, ia, 0), DVM_HDR_WORDS + 2 * nt + ib * DVM_OPD_WORDS, 0, 0);
+    } else if (op == DVM_OP_BCS) {
+      push(DVM_LK_W0(DVM_LK_BCS, 0, ia, 0), 0, 0, 0);
+    } else if (op == DVM_OP_SOP) {
+      push(DVM_LK_W0(DVM_LK_SOP, ib, ia, 0), body[pc + 1], len > 2 ? body[pc + 2] : 0, len > 3 ? body[pc + 3] : 0);
+    } else if (op == DVM_OP_NOP) {
+    } else {
+      return 0;  // Cmp / Select / Pow ...: not the lean interpreter's
+    }
+    pc += len;
+  }
+  // ---- fusions over neighbouring records ----
+  auto hid = [&](uint32_t i) { return rec[i].w[0] & 0xffu; };
+  auto sub = [&](uint32_t i) { return (rec[i].w[0] >> 8) & 0xffu; };
+  uint32_t m = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    Rec r = rec[i];
+    const uint32_t h = r.w[0] & 0xffu;
+    if (i + 1 < n) {
+      const uint32_t h2 = hid(i + 1), s2 = sub(i + 1);
+      // ACC = L[x] ; ACC = ACC op L[y], both bf16 images  ->  LD2 (fp32 pairs stay two records: their raw words fill the registers)
+      if (h == DVM_LK_LDA_BF16 && h2 == DVM_LK_BIN_BF16) {
+        if ((s2 == DVM_A_ADD || s2 == DVM_A_SUB || s2 == DVM_A_RSUB || s2 == DVM_A_MUL) && !(rec[i + 1].w[0] >> 24)) {
+          r.w[0] = DVM_LK_W0(DVM_LK_LD2_BF16, s2, 0, 0);
+          r.w[2] = rec[i + 1].w[1];
+          ++i;
+          // ... followed by a multiplication by an immediate
+          if (i + 1 < n && hid(i + 1) == DVM_LK_FMA && sub(i + 1) == 0 && rec[i + 1].w[2] == f2u(neg_zero)) {
+            r.w[0] |= 1u << 24;
+            r.w[3] = rec[i + 1].w[1];
+            ++i;
+          }
+          rec[m++] = r;
+          continue;
+        }
+      }
+      // multiply by an immediate, then add an immediate  ->  one multiply-add
+      if (h == DVM_LK_FMA && sub(i) == 0 && r.w[2] == f2u(neg_zero) && h2 == DVM_LK_FMA && s2 == 0 && rec[i + 1].w[1] == f2u(one)) {
+        r.w[2] = rec[i + 1].w[2];
+        ++i;
+        rec[m++] = r;
+        continue;
+      }
+      // ACC = ACC * S[a] ; ACC = ACC * L[y]  ->  BIN with a pre-multiplier
+      if (h == DVM_LK_FMA && sub(i) == 1 && r.w[2] == f2u(neg_zero) && (h2 == DVM_LK_BIN_BF16 || h2 == DVM_LK_BIN_F32) &&
+          s2 == DVM_A_MUL && !(rec[i + 1].w[0] >> 24)) {
+        Rec q = rec[i + 1];
+        q.w[0] |= (1u + ((r.w[0] >> 16) & 0xffu)) << 24;
+        ++i;
+        rec[m++] = q;
+        continue;
+      }
+    }
+    rec[m++] = r;
+  }
+  n = m;
+  // the records start at a word index = 2 mod 4 of the parameter block (16-byte aligned in the kernel's parameter space)
+  uint32_t rec0 = head;
+  while ((at + rec0) % 4 != 2) ++rec0;
+  if (rec0 + 4 * (n + 1) > max_words) return 0;
+  for (uint32_t i = head; i < rec0; ++i) dst[i] = 0;
+  for (uint32_t i = 0; i < n; ++i) memcpy(dst + rec0 + 4 * i, rec[i].w, 16);
+  uint32_t* end = dst + rec0 + 4 * n;
+  end[0] = DVM_LK_W0(DVM_LK_END, 0, 0, 0); end[1] = end[2] = end[3] = 0;
+  ++n;
+  // Header words the device never reads carry what the lean interpreter wants ready: the offset of the records
+  // (magic word) and the multipliers that divide a row index by the two inner outer-dim sizes.
+  auto magic = [](uint32_t d, uint32_t* mult, uint32_t* l) {
+    uint32_t lg = 0;
+    while (lg < 32 && ((uint64_t)1 << lg) < d) ++lg;
+    *l = lg;
+    *mult = d ? (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << lg) - d)) / d + 1) : 0;
+  };
+  dst[DVM_H_MAGIC] = rec0;
+  magic(src[DVM_H_OUTER0], &dst[DVM_H_KERNEL_TYPE], &dst[DVM_H_CODE_WORDS]);
+  magic(src[DVM_H_OUTER1], &dst[DVM_H_N_TILES], &dst[DVM_H_TOTAL_WORDS]);
+  return rec0 + 4 * n;
+}
+
 // Results that tiles combine atomically start from the operation's identity.
 __global__ void dvm_fill_kernel(uint32_t* p, uint32_t n, uint32_t bits) {
   for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = bits;
@@ -201,22 +397,80 @@ int launch_variant(const DvmVmVariant* v, const void* params, int grid, size_t s
 }
 
 // The variant a launch needs: 24 elements per thread exist as the one-program basic variant only.
-const DvmVmVariant* pick_variant(int V, bool large, bool single, int ext, bool levels) {
+const DvmVmVariant* pick_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy) {
   if (levels) single = false;
-  return dvm_vm_find_variant(V, large, single, ext, levels);
+  return dvm_vm_find_variant(V, large, single, ext, levels, lean, heavy);
+}
+
+// What decides between the lean kernel and the general one, read off a placed program (tensor addresses known):
+//   wrap  -- a row may fill the tile's whole capacity while its chunks are shifted by a misaligned row start, so
+//            that its last columns wrap around into the head slots: only the general kernel does that;
+//   heavy -- a tile-class unary function that only the HEAVY variants of the lean kernel carry.
+void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* heavy) {
+  const uint32_t geom = w[DVM_H_GEOM];
+  uint32_t flags = geom >> 24;
+  const uint32_t lgG = geom & 0xff, W = (geom >> 8) & 0xff, V = w[DVM_H_LOCAL] >> 24;
+  const uint32_t counts = w[DVM_H_COUNTS];
+  const uint32_t* ot = w + DVM_HDR_WORDS + 2 * (counts & 0xff);
+  if ((flags & DVM_F_ALIGNED) && w[DVM_H_PRIMARY] != 0xffffffffu &&
+      (((uintptr_t)tensors[ot[w[DVM_H_PRIMARY] * DVM_OPD_WORDS] & 0xff]) & 15))
+    flags &= ~(uint32_t)DVM_F_ALIGNED;  // (what place_program does to the placed copy)
+  if (!(flags & DVM_F_ALIGNED) && (uint64_t)w[DVM_H_COL_TILE] + W - 1 > ((uint64_t)V << lgG)) *wrap = true;
+  const uint32_t* body = ot + ((counts >> 16) & 0xff) * DVM_OPD_WORDS + ((geom >> 16) & 0xff);
+  const uint32_t end = w[DVM_H_CODE_WORDS];
+  for (uint32_t pc = w[DVM_H_LOAD_WORDS]; pc < end;) {
+    const uint32_t op = DVM_INSN_OP(body[pc]), len = DVM_INSN_LEN(body[pc]);
+    if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
+      const uint32_t u = op - DVM_OP_UN;
+      if (u == DVM_U_SQRT || u == DVM_U_LOG || u == DVM_U_ERF || u == DVM_U_FLOOR || u == DVM_U_ROUND || u == DVM_U_TANH) *heavy = true;
+    }
+    pc += len ? len : 1;
+  }
 }
 
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
 
+// Writes the directory and the programs of a launch into the parameter block P.  `linked`: in the linked form
+// of the lean interpreter; returns DVM_ERR_UNSUPPORTED when some program cannot be linked or the linked forms
+// do not fit (the caller then places the plain forms for the general interpreter).
+int place_all(dvm::VMParams<PW_LARGE>& P, int n_programs, const void* const* codes, void* const* const* tensors,
+              const int* n_tensors, const int* level, bool linked, uint32_t* words_used) {
+  const uint32_t dir = (level ? 3 : 2) * (uint32_t)n_programs + 1;
+  uint32_t pos = dir, tb = 0, level_start = 0;
+  for (int i = 0; i < n_programs; ++i) {
+    const uint32_t* c = (const uint32_t*)codes[i];
+    if (pos + c[DVM_H_TOTAL_WORDS] > (uint32_t)PW_LARGE) return linked ? DVM_ERR_UNSUPPORTED : DVM_ERR_TOO_LARGE;
+    P.words[i] = pos;
+    P.words[n_programs + i] = tb;
+    if (level) {
+      if (i > 0 && level[i] != level[i - 1]) level_start = tb;  // every tile before this one belongs to a lower level
+      P.words[2 * n_programs + 1 + i] = level_start;
+    }
+    int st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
+    if (st != DVM_OK) return st;
+    uint32_t used = c[DVM_H_TOTAL_WORDS];
+    if (linked) {
+      used = dvm_link_program(P.words + pos, pos, (uint32_t)PW_LARGE - pos, c, tensors[i]);
+      if (used == 0) return DVM_ERR_UNSUPPORTED;
+    }
+    pos += used;
+    tb += c[DVM_H_N_TILES];
+  }
+  P.words[2 * n_programs] = tb;
+  *words_used = pos;
+  return DVM_OK;
+}
+
 // `level` (may be NULL): level[i] of program i, non-decreasing; a program reads what programs of lower levels store.
 int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
                bool use_queue, const int* level, cudaStream_t stream) {
-  // A program that asks for a single tile slot (DVM_F_ONE_SLOT), launched on its own: the variant with level
-  // waits runs it, every tile held back until the CTA's previous tile is done, nothing waited for.
-  const bool one_slot = n_programs == 1 && !level &&
-                        ((((const uint32_t*)codes[0])[DVM_H_GEOM] >> 24) & DVM_F_ONE_SLOT) != 0;
+  // A program that asks for a single tile slot (DVM_F_ONE_SLOT), launched on its own: the lean interpreter runs
+  // it with one slot; on the general interpreter the variant with level waits does (every tile held back until
+  // the CTA's previous tile is done, nothing waited for).
+  bool one_slot = n_programs == 1 && !level &&
+                  ((((const uint32_t*)codes[0])[DVM_H_GEOM] >> 24) & DVM_F_ONE_SLOT) != 0;
   static const int kOneLevel[1] = {0};
-  if (one_slot) { level = kOneLevel; use_queue = true; }
+  const bool queue_asked = use_queue;
   // directory: [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, with levels)]
   uint32_t dir = (level ? 3 : 2) * (uint32_t)n_programs + 1;
   uint64_t need = dir;
@@ -243,21 +497,22 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (st != DVM_OK) return st;
 
   dvm::VMParams<PW_LARGE>& P = t_large;
-  uint32_t pos = dir, tb = 0, level_start = 0;
+  bool wrap = false, heavy = false;
   for (int i = 0; i < n_programs; ++i) {
-    const uint32_t* c = (const uint32_t*)codes[i];
-    P.words[i] = pos;
-    P.words[n_programs + i] = tb;
-    if (level) {
-      if (i > 0 && level[i] != level[i - 1]) level_start = tb;  // every tile before this one belongs to a lower level
-      P.words[2 * n_programs + 1 + i] = level_start;
-    }
-    st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
-    if (st != DVM_OK) return st;
-    pos += c[DVM_H_TOTAL_WORDS];
-    tb += c[DVM_H_N_TILES];
+    const uint32_t nt = ((const uint32_t*)codes[i])[DVM_H_COUNTS] & 0xff;
+    if ((uint32_t)n_tensors[i] != nt) return DVM_ERR_INVALID_ARG;
+    for (uint32_t q = 0; q < nt; ++q) if (!tensors[i][q]) return DVM_ERR_INVALID_ARG;
+    program_traits((const uint32_t*)codes[i], tensors[i], &wrap, &heavy);
   }
-  P.words[2 * n_programs] = tb;
+  int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked)) ? g_use_lean : 0;
+  uint32_t pos = 0;
+  st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, level, true, &pos) : DVM_ERR_UNSUPPORTED;
+  if (st == DVM_ERR_UNSUPPORTED) {
+    lean = 0;
+    if (one_slot) { level = kOneLevel; use_queue = true; }
+    st = place_all(P, n_programs, codes, tensors, n_tensors, level, false, &pos);
+  }
+  if (st != DVM_OK) return st;
   P.n_programs = (uint32_t)n_programs;
   P.total_tiles = (uint32_t)total_tiles;
   P.n_words = pos;
@@ -271,7 +526,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.slot_bytes = one_slot ? 0u : units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool single = n_programs == 1 && !use_queue;
-  const DvmVmVariant* variant = pick_variant(V, large, single, ext, level != nullptr);
+  const DvmVmVariant* variant = pick_variant(V, large, single, ext, level != nullptr, lean, heavy);
   if (!variant) return DVM_ERR_UNSUPPORTED;  // (24 elements per thread: encoded for a launch of its own on the basic variant)
   int occ = 0;
   st = dvm_occupancy(variant, smem, &occ);
@@ -498,17 +753,21 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   cudaStream_t stream = (cudaStream_t)cuda_stream;
 
   dvm::VMParams<PW_LARGE>& P = t_large;
-  uint32_t pos = dir, tb = 0;
+  bool wrap = false, heavy = false;
   for (int i = 0; i < n_programs; ++i) {
-    const uint32_t* c = (const uint32_t*)codes[i];
-    P.words[i] = pos;
-    P.words[n_programs + i] = tb;
-    st = place_program(P.words + pos, c, tensors[i], n_tensors[i]);
-    if (st != DVM_OK) return st;
-    pos += c[DVM_H_TOTAL_WORDS];
-    tb += c[DVM_H_N_TILES];
+    const uint32_t nt = ((const uint32_t*)codes[i])[DVM_H_COUNTS] & 0xff;
+    if ((uint32_t)n_tensors[i] != nt) return DVM_ERR_INVALID_ARG;
+    for (uint32_t q = 0; q < nt; ++q) if (!tensors[i][q]) return DVM_ERR_INVALID_ARG;
+    program_traits((const uint32_t*)codes[i], tensors[i], &wrap, &heavy);
   }
-  P.words[2 * n_programs] = tb;
+  int lean = (ext == 0 && !wrap) ? g_use_lean : 0;
+  uint32_t pos = 0;
+  st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, nullptr, true, &pos) : DVM_ERR_UNSUPPORTED;
+  if (st == DVM_ERR_UNSUPPORTED) {
+    lean = 0;
+    st = place_all(P, n_programs, codes, tensors, n_tensors, nullptr, false, &pos);
+  }
+  if (st != DVM_OK) return st;
   P.n_programs = (uint32_t)n_programs;
   P.total_tiles = (uint32_t)total_tiles;
   P.n_words = pos;
@@ -520,7 +779,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.slot_bytes = units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool large = pos > PW_SMALL;
-  const DvmVmVariant* variant = pick_variant(V, large, false, ext, false);
+  const DvmVmVariant* variant = pick_variant(V, large, false, ext, false, lean, heavy);
   if (!variant) return DVM_ERR_UNSUPPORTED;
   int occ = 0;
   st = dvm_occupancy(variant, smem, &occ);

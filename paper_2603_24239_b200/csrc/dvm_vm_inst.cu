@@ -1,12 +1,15 @@
 // Instantiations of the interpreter kernel, one group per compilation of this file (-DDVM_INST_GROUP=g):
 // group g < 12: V = 16 (g < 6) or 32, parameter block small (g % 6 < 3) or large, extension level g % 3,
 // each with the one-program, the stacked and the level-wait variant; group 12: the 24-element one-program
-// basic variants.
+// basic variants; groups 13..16: the lean kernel for V = 16 (13, 14) or 32, parameter block small (13, 15) or
+// large, each one-program / stacked, with and without the heavy unary functions; group 17: the lean kernel with
+// 24 elements per thread (one program).
 #include "dvm_vm.cuh"
+#include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..12>"
+#error "compile with -DDVM_INST_GROUP=<0..17>"
 #endif
 
 namespace {
@@ -27,8 +30,29 @@ struct Ops {
   }
 };
 
+template <int V, int PW, bool SINGLE, bool HEAVY>
+struct LeanOps {
+  static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>
+        <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
+    return cudaGetLastError();
+  }
+  static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>,
+                                                         dvm::THREADS, smem);
+  }
+};
+
+#define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
+  {V, LARGE, SINGLE, 0, 0, 1, HEAVY,                                                        \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::launch, \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::occupancy}
+
 #define DVM_ENTRY(V, LARGE, SINGLE, EXT, LEVELS)                                       \
-  {V, LARGE, SINGLE, EXT, LEVELS,                                                     \
+  {V, LARGE, SINGLE, EXT, LEVELS, 0, 1,                                               \
    &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::launch, \
    &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::occupancy}
 
@@ -37,8 +61,14 @@ constexpr int GV = DVM_INST_GROUP < 6 ? 16 : 32;
 constexpr int GL = (DVM_INST_GROUP % 6) < 3 ? 0 : 1;
 constexpr int GE = DVM_INST_GROUP % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY(GV, GL, 1, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 1)};
-#else
+#elif DVM_INST_GROUP == 12
 const DvmVmVariant kGroup[] = {DVM_ENTRY(24, 0, 1, 0, 0), DVM_ENTRY(24, 1, 1, 0, 0)};
+#elif DVM_INST_GROUP < 17
+constexpr int GV = DVM_INST_GROUP < 15 ? 16 : 32;
+constexpr int GL = (DVM_INST_GROUP - 13) % 2;
+const DvmVmVariant kGroup[] = {DVM_LEAN(GV, GL, 1, 0), DVM_LEAN(GV, GL, 1, 1), DVM_LEAN(GV, GL, 0, 0), DVM_LEAN(GV, GL, 0, 1)};
+#else
+const DvmVmVariant kGroup[] = {DVM_LEAN(24, 0, 1, 0), DVM_LEAN(24, 0, 1, 1), DVM_LEAN(24, 1, 1, 0), DVM_LEAN(24, 1, 1, 1)};
 #endif
 
 }  // namespace

@@ -15,6 +15,8 @@ struct DvmVmVariant {
   int single;   // 1: one program per launch (dvm_launch)
   int ext;      // 0 basic, 1 + Cmp / Select / Pow / IsFinite, 2 + views
   int levels;   // 1: stacked launch with waits between dependent levels
+  int lean;     // 1: the lean kernel for the basic instruction set (no level waits, no wrap-around rows)
+  int heavy;    // unary functions log / erf / tanh / sqrt / floor / round on tiles: 1 present, 0 absent (lean only)
   // launches the kernel; `params` points at a dvm::VMParams<PW> of the variant's block size
   cudaError_t (*launch)(const void* params, int grid, size_t smem, cudaStream_t stream);
   // lifts the dynamic shared memory limit of the kernel and asks how many CTAs of it an SM holds
@@ -22,4 +24,4 @@ struct DvmVmVariant {
 };
 
 // NULL when the library has no such variant.
-const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels);
+const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy);
