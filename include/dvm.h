@@ -197,9 +197,10 @@ int dvm_get_elems_per_thread(void);
  * best.  Callers of dvm_launch_stacked set it before encoding.  Per calling thread (the setting of one thread does not reach the encodes of another). */
 void dvm_set_min_resident_ctas(int n);
 int dvm_get_min_resident_ctas(void);
-/* Programs of the basic instruction set run on a lean variant of the interpreter (Algorithm 2 with a shorter
- * instruction stream per tile); 0 sends every launch of the process to the general interpreter instead, for
- * comparisons.  Default 1.  Both run the same bytecode and give results inside the same tolerances. */
+/* One-program launches of the basic instruction set run on a lean variant of the interpreter (Algorithm 2 from
+ * linked code: a shorter instruction stream per tile).  0 sends every launch of the process to the general
+ * interpreter instead, 2 also sends stacked launches to the lean one (for comparisons; measured slower).
+ * Default 1.  Both interpreters run the same bytecode and give results inside the same tolerances. */
 void dvm_set_lean_kernel(int on);
 
 /* The paper's tile-size rule for a flat vector operator (Sec. 4.2,

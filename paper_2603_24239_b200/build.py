@@ -20,7 +20,7 @@ HEADERS = ["dvm_format.h", "dvm_internal.h", "dvm_launch.h", "dvm_vm.cuh", "dvm_
            "dvm_vm_variants.h", "dvm_vm_lean.cuh", "dvm_link.h", os.path.join("..", "..", "include", "dvm.h"),
            os.path.join("..", "..", "include", "dvm_fuser.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC"]
+              "-Xcompiler", "-fPIC"] + os.environ.get("DVM_EXTRA_NVCC_FLAGS", "").split()
 
 
 def _nvcc() -> str:

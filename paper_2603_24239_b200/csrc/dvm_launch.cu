@@ -504,7 +504,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     for (uint32_t q = 0; q < nt; ++q) if (!tensors[i][q]) return DVM_ERR_INVALID_ARG;
     program_traits((const uint32_t*)codes[i], tensors[i], &wrap, &heavy);
   }
-  int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked)) ? g_use_lean : 0;
+  // (launches with a work queue run on the general interpreter unless asked otherwise: measured faster there)
+  int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked) && (!queue_asked || g_use_lean >= 2)) ? (g_use_lean ? 1 : 0) : 0;
   uint32_t pos = 0;
   st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, level, true, &pos) : DVM_ERR_UNSUPPORTED;
   if (st == DVM_ERR_UNSUPPORTED) {
@@ -760,7 +761,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     for (uint32_t q = 0; q < nt; ++q) if (!tensors[i][q]) return DVM_ERR_INVALID_ARG;
     program_traits((const uint32_t*)codes[i], tensors[i], &wrap, &heavy);
   }
-  int lean = (ext == 0 && !wrap) ? g_use_lean : 0;
+  int lean = (ext == 0 && !wrap && g_use_lean >= 2) ? 1 : 0;
   uint32_t pos = 0;
   st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, nullptr, true, &pos) : DVM_ERR_UNSUPPORTED;
   if (st == DVM_ERR_UNSUPPORTED) {

