@@ -776,6 +776,192 @@ def oracle_threads(workload: str) -> int:
         return 1
 
 
+
+# ----------------------------------------------------------------------------- oracle spot checks (cpu_baseline leg)
+def _check_cases(name):
+    """Small seeded cases of a workload's program(s): (program, cpu inputs, runtime scalars, input strides or None)."""
+    bf = torch.bfloat16
+    if name == "c1":
+        return [(wl.program_c1(), wl.inputs_c1(), (), None)]
+    if name == "c2":
+        return [(wl.program_add_rmsnorm(4096), wl.inputs_add_rmsnorm(333, 4096, 1), (), None)]
+    if name == "c3":
+        return [(wl.program_masked_softmax(), wl.inputs_masked_softmax(1, 2, 333, 2), (), None),
+                (wl.program_masked_softmax(), wl.inputs_masked_softmax(1, 1, 1024, 3), (), None)]
+    if name == "c4":
+        out = []
+        for j, (kind, r, c) in enumerate([("gelu_affine", 200, 333), ("layernorm", 17, 1000), ("sigmoid_mul", 64, 4095)]):
+            ins, params = wl.inputs_stack(kind, r, c, 40 + 4 * j)
+            out.append((wl.stack_program(kind), ins, params, None))
+        return out
+    if name == "c5":
+        return [(wl.program_mlp_gate(), [wl.randn((96, 512), bf, 3), wl.randn((512, 1024), bf, 4, std=0.05),
+                                         wl.randn((512, 1024), bf, 5, std=0.05)], (), None)]
+    if name == "addmm":
+        return [(wl.program_addmm(), [wl.randn((130, 512), bf, 6), wl.randn((512, 520), bf, 7, std=0.05),
+                                      wl.randn((130, 520), bf, 8)], (), None)]
+    if name == "ifelse":
+        return [(wl.program_if_else_add(), [wl.randn((3, 50, 333), torch.float32, 10 + i) for i in range(4)], (), None)]
+    if name == "views":
+        B, H, S, D = 2, 32, 100, 128
+        xs = wl.randn((B * S * H * D,), bf, 20)
+        y = wl.randn((B, H, S, D), bf, 21)
+        return [(wl.program_head_transpose_add(), [xs, y], (), [[S * H * D, D, H * D, 1], None], (B, H, S, D))]
+    return []
+
+
+def oracle_check(dvm, name):
+    """Runs the workload's small cases through the C ABI on the GPU and through the CPU oracle, element by element:
+    worst row-scaled error |g - o| / max(|o|, row max |o|) against the gate (1e-5 fp32 programs, 2e-2 programs with a
+    bf16 tensor), and the strict elementwise statistics for the programs that only the row-scaled gate can hold."""
+    import numpy as np
+    from oracle import dvm_oracle as orc
+    worst, n_el, ok = 0.0, 0, True
+    strict = {"max": 0.0, "n_over": 0, "n_well": 0, "n_over_well": 0, "n": 0}
+    gate = 1e-5
+    stacked = name == "c4"
+    codes, tls, wants, progs_seen = [], [], [], []
+    if stacked:
+        dvm.set_elems_per_thread(16)
+    try:
+        for case in _check_cases(name):
+            prog, ins, params, strides = case[:4]
+            kinds = [n[1] for n in prog.nodes if n[0] == "input"] + [n[2] for n in prog.nodes if n[0] == "output"]
+            r = 2e-2 if "bf16" in kinds else 1e-5
+            gate = max(gate, r) if r == 2e-2 else gate
+            dev = [t.cuda() for t in ins]
+            shapes = [tuple(t.shape) for t in ins]
+            ins64 = [wl.to_f64(t) for t in ins]
+            if strides is not None:   # the first input is storage seen through a view
+                shapes[0] = case[4]
+                ins64[0] = orc.view_load(ins64[0], 0, case[4], strides[0])
+                code = dvm.encode(dvm.program_from_nodes(prog.nodes), shapes, params, in_strides=strides)
+            else:
+                code = dvm.encode(dvm.program_from_nodes(prog.nodes), shapes, params)
+            dt = {"f32": torch.float32, "bf16": torch.bfloat16}
+            outs = [torch.full(sh, float("nan"), dtype=dt[nd[2]], device="cuda") for sh, nd in zip(code.out_shapes, prog.output_nodes)]
+            want = orc.evaluate(prog.nodes, ins64, params)
+            want32 = orc.evaluate(prog.nodes, ins64, params, diagnostic_fp32=True)
+            if stacked:
+                codes.append(code); tls.append(dev + outs)
+            else:
+                dvm.launch(code, dev + outs)
+            wants.append((outs, want, want32, r))
+        if stacked:
+            dvm.launch_stacked(codes, tls)
+        assert dvm.last_device_status() == 0
+        for outs, want, want32, r in wants:
+            for g, w, w32 in zip(outs, want, want32):
+                g = wl.to_f64(g)
+                den = np.maximum(np.abs(w), np.max(np.abs(w), axis=-1, keepdims=True))
+                err = np.abs(g - w)
+                bad = ~(err <= r * den)
+                ok = ok and not bool(bad.any())
+                with np.errstate(divide="ignore", invalid="ignore"):
+                    g1 = np.where(err == 0, 0.0, err / den)
+                    rel = np.where((w != 0) & np.isfinite(w), err / np.abs(w), 0.0)
+                worst = max(worst, float(np.nanmax(g1)) if g1.size else 0.0)
+                well = (w != 0) & (np.abs(w32 - w) <= 1e-6 * np.abs(w))
+                over = rel > r
+                strict["max"] = max(strict["max"], float(rel.max()) if rel.size else 0.0)
+                strict["n_over"] += int(over.sum()); strict["n_well"] += int(well.sum())
+                strict["n_over_well"] += int((over & well).sum()); strict["n"] += int(w.size)
+                n_el += int(w.size)
+    finally:
+        if stacked:
+            dvm.set_elems_per_thread(0)
+    return {"pass": bool(ok), "worst_g1": worst, "gate": gate, "elements": n_el,
+            "strict": {"max": strict["max"], "n_over_gate": strict["n_over"], "n_well_conditioned": strict["n_well"],
+                       "n_over_gate_well_conditioned": strict["n_over_well"], "n": strict["n"],
+                       "note": "strict |g-o|/|o| (reported, not gated); well conditioned = a faithful fp32 evaluation is within 1e-6 of the fp64 oracle"}}
+
+
+def native_encode_us(W, reps):
+    """Host encode latency measured inside the library (steady clock around the encoder, no binding): `reps` repeats of
+    each of up to 20 instances of the sweep."""
+    import numpy as np
+    if not hasattr(W, "enc"):
+        return None
+    if W.name == "views":
+        cases = [(((b, W.H, s_, W.D),) * 2, (), W._strides(b, s_)) for b, s_ in W.shapes[:20]]
+    elif W.name == "ifelse":
+        cases = [((shp,) * 4, (), None) for shp in W.shapes[:20]]
+    elif W.name == "addmm":
+        cases = [(((m, k), (k, n), (m, n)), (), None) for m, n, k in W.shapes[:20]]
+    elif W.name == "c1":
+        cases = [(((7, 1531),) * 3, (), None)]
+    elif W.name == "c2":
+        cases = [(((t, 4096), (t, 4096), (4096,)), (), None) for t in W.rows[:20]]
+    elif W.name == "c3":
+        cases = [(((b, 32, s_, s_), (1, 1, s_, s_)), (), None) for b, s_ in W.shapes[:20]]
+    elif W.name == "c5":
+        cases = [(((m, 4096), (4096, 11008), (4096, 11008)), (), None) for m in W.Ms[:20]]
+    else:
+        return None
+    ns = []
+    for shp, sc, strides in cases:
+        ns += W.enc.time_encode(shp, sc, reps, strides)
+    a = np.sort(np.asarray(ns, dtype=np.float64)) / 1e3
+    return {"mean": float(a.mean()), "p50": float(a[len(a) // 2]), "p99": float(a[int(0.99 * len(a))]),
+            "p999": float(a[int(0.999 * len(a))]), "max": float(a[-1]), "n": int(len(a)),
+            "note": f"steady clock inside the library around the encoder, {reps} repeats of each of {len(cases)} instances"}
+
+
+def run_config(dvm, name, peaks, peak_kind, steps, warmup=3, check=True, baseline_s=1.5):
+    """One sweep of another workload for the `configs` object of the default line: kernel-only throughput over `steps`
+    timed steps after `warmup`, roofline fraction, host encode latency, and the oracle beside it (throughput on a
+    bounded sample, spot check of small cases)."""
+    import gc
+    kw = {}
+    W = WORKLOADS[name](dvm, **kw)
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        W.run_step(stream)
+    torch.cuda.synchronize()
+    events, enc_ns = [], []
+    gc_was = gc.isenabled()
+    gc.disable()
+    try:
+        l0 = dvm.launch_count()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            W.run_step(stream, events=events, enc_ns=enc_ns)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        launches = dvm.launch_count() - l0
+    finally:
+        if gc_was:
+            gc.enable()
+    assert dvm.last_device_status() == 0
+    ms = e0.elapsed_time(e1) / steps
+    work_each = getattr(W, "work_per_instance", W.bytes_per_instance)
+    value = sum(work_each) / (ms * 1e-3) / W.scale
+    kern_ms = [a.elapsed_time(b) for a, b in events]
+    achieved = sum(work_each) * steps / (sum(kern_ms) * 1e-3) / W.scale
+    peak = peaks[W.peak_key]
+    enc_us = sorted(x / 1e3 for x in enc_ns)
+    out = {"workload": W.description, "value": value, "unit": W.unit, "ms_per_step": ms, "steps": steps, "warmup": warmup,
+           "roofline": {"bound": W.bound, "achieved": achieved, "peak": peak, "frac": achieved / peak,
+                        "peak_kind": f"of {peak_kind} ({W.peak_key})",
+                        "frac_of_nominal": achieved / (2250.0 if W.bound == "tensor" else 8000.0)},
+           "launches_timed": len(kern_ms), "gpu_launches": launches,
+           "encode_us": {"mean": sum(enc_us) / len(enc_us), "p99": enc_us[min(len(enc_us) - 1, int(0.99 * len(enc_us)))],
+                         "max": enc_us[-1], "n": len(enc_us),
+                         "note": ("per program, one dvm_encode_batch call of 64 programs" if name == "c4" else
+                                  "perf_counter around the binding's encode call, garbage collector off")},
+           "encode_us_native": native_encode_us(W, 200)}
+    if name == "c1":
+        out["latency_us"] = {"kernel_event_mean": 1e3 * sum(kern_ms) / max(len(kern_ms), 1)}
+    if check:
+        v, dt, sample = W.oracle_sample(budget_s=baseline_s)
+        out["cpu_baseline"] = {"value": v, "unit": W.unit, "cores": oracle_threads(name), "kind": "oracle", "sample": sample,
+                               "seconds": dt, "check": oracle_check(dvm, name)}
+    del W
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------- reference arm
 def run_reference(args):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload per step."""
@@ -928,6 +1114,8 @@ def main():
                     help="run every launch on the general interpreter instead of the lean one (for comparisons)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the sweeps of the other workloads that the default line reports under `configs`")
     ap.add_argument("--detail", default="", help="write per-instance timings to this JSON file")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -981,11 +1169,15 @@ def main():
     step_ms = []
     barrier()
     e_start = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+    import gc
+    gc.collect()
+    gc.disable()   # a collection inside the sweep would show up as a host-encode outlier of a millisecond
     e_start.record(stream)
     n_inst = 0
     for k in range(args.steps):
         n_inst = W.run_step(stream, events=events, enc_ns=enc_ns)
     e_end.record(stream)
+    gc.enable()
     barrier()
     total_ms = e_start.elapsed_time(e_end)
     launches = dvm.launch_count() - launches0
@@ -1028,6 +1220,8 @@ def main():
         if mt:
             # measured DRAM bytes per algorithmic byte on an ncu-captured instance, scaled to the mean launch
             traffic = float(mt.group(1)) * sum(per_launch_bytes) / len(per_launch_bytes)
+    traffic_source = (f"ratio DRAM bytes / algorithmic bytes of the ncu capture summarised in profiles/{W.kernel}_{args.workload}.md "
+                      "(a committed measurement of a smaller instance, not taken in this run), scaled to the mean launch") if traffic else None
 
     line = {
         "metric": W.metric, "value": value, "unit": W.unit, "n_gpus": world,
@@ -1045,7 +1239,7 @@ def main():
                                if W.name == "c4" else "perf_counter around the ctypes call to dvm_encode")},
         "roofline": {"bound": W.bound, "kernel": W.kernel, "achieved": achieved, "peak": peak,
                      "unit": W.unit, "frac": achieved / peak, "peak_kind": f"of {peak_kind} ({W.peak_key})",
-                     "traffic": traffic, "large_instances": large_gbs,
+                     "traffic": traffic, "traffic_source": traffic_source, "large_instances": large_gbs,
                      "large_instances_frac": (large_gbs / peak) if large_gbs else None,
                      "roofline_time_frac": roofline_time_frac,
                      "per_launch": {"min": gbs_each[0], "p10": pct(gbs_each, 0.1), "p50": pct(gbs_each, 0.5),
@@ -1065,6 +1259,7 @@ def main():
                               "kernel_event_mean": 1e3 * kernel_total_ms / max(len(kern_ms), 1)}
     if rank == 0 and hasattr(W, "enc") and args.encode_reps > 0:
         line["encode_us_repeated"] = encode_latency(W, args.encode_reps)
+        line["encode_us_native"] = native_encode_us(W, args.encode_reps)
     if args.detail and rank == 0:
         with open(args.detail, "w") as f:
             json.dump({"bytes": per_launch_bytes, "ms": kern_ms, "enc_us": [x / 1e3 for x in enc_ns]}, f)
@@ -1091,7 +1286,23 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, dt, sample = W.oracle_sample()
         line["cpu_baseline"] = {"value": v, "unit": W.unit, "cores": oracle_threads(W.name), "kind": "oracle",
-                                "sample": sample, "seconds": dt, "host_cores_available": os.cpu_count()}
+                                "sample": sample, "seconds": dt, "host_cores_available": os.cpu_count(),
+                                "check": oracle_check(dvm, W.name)}
+    if rank == 0 and world == 1 and args.workload == "c2" and not args.no_configs and not args.instances and not args.max_rows:
+        # the other sweeps, fewer steps each, so that every configuration is measured by the default command
+        name_main = W.name
+        del W
+        torch.cuda.empty_cache()
+        cfgs = {}
+        for name, steps in (("c1", 50), ("c3", 2), ("c4", 2), ("c5", 2), ("addmm", 1), ("ifelse", 1), ("views", 1)):
+            if name == name_main:
+                continue
+            try:
+                cfgs[name] = run_config(dvm, name, peaks, peak_kind, steps, check=not args.no_cpu_baseline)
+            except Exception as e:   # one failing sweep must not take the headline line with it
+                cfgs[name] = {"error": f"{type(e).__name__}: {e}"}
+                torch.cuda.empty_cache()
+        line["configs"] = cfgs
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:

@@ -163,6 +163,12 @@ int dvm_encode_strided(const dvm_program* p, const dvm_shape* in_shapes, const d
                        const float* scalars, int n_scalars, const dvm_strides* out_strides,
                        void* code, size_t code_capacity, size_t* code_size,
                        dvm_shape* out_shapes, int n_out);
+/* Measurement helper: calls the encoder `reps` times on one instance (in_strides may be NULL: dense inputs) and
+ * writes the duration of every call, in nanoseconds of the steady clock, to ns_out[0 .. reps).  The clock is read
+ * inside the library, so the figures hold the encoder alone -- no binding, no interpreter of the caller's
+ * language.  `code` / `code_capacity`: a caller-owned buffer as for dvm_encode.  Host pointers throughout. */
+int dvm_time_encode(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                    const float* scalars, int n_scalars, void* code, size_t code_capacity, int reps, int64_t* ns_out);
 /* dvm_encode for n independent instances in one call -- the stacked-fusion case (Sec. 5.1), where every
  * program of a launch is re-encoded per launch.  All arrays are host memory of length n, except
  * in_shapes / scalars, which concatenate the instances' arguments (instance i consumes n_in[i] shapes and

@@ -74,6 +74,7 @@ _sig = {
                             _vp, _sz, C.POINTER(_sz), C.POINTER(Shape), _i], _i),
     "dvm_encode_batch": ([_i, C.POINTER(_vp), C.POINTER(Shape), _pi, C.POINTER(C.c_float), _pi, C.POINTER(_vp),
                           C.POINTER(_sz), C.POINTER(_sz), _pi], _i),
+    "dvm_time_encode": ([_vp, C.POINTER(Shape), _vp, _i, C.POINTER(C.c_float), _i, _vp, _sz, _i, _p64], _i),
     "dvm_code_max_size": ([_vp], _sz),
     "dvm_set_num_cores": ([_i], None),
     "dvm_get_num_cores": ([], _i),
@@ -246,6 +247,29 @@ class Encoder:
         self.buf = (C.c_uint64 * ((self.cap + 7) // 8))()
         self.size = _sz(0)
         self.scalars = (C.c_float * 16)()
+
+    def time_encode(self, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = (), reps: int = 1000,
+                    in_strides: Optional[Sequence[Optional[Sequence[int]]]] = None) -> List[int]:
+        """Durations (ns, steady clock read inside the library) of `reps` encodes of one instance: the encoder
+        alone, without the binding."""
+        for s, shp in zip(self.shapes, shapes):
+            s.rank = len(shp)
+            for k, d in enumerate(shp):
+                s.dims[k] = d
+        for k, v in enumerate(scalars):
+            self.scalars[k] = v
+        ins = None
+        if in_strides is not None:
+            ins = (Strides * self.n_in)()
+            for a, t, shp in zip(ins, in_strides, shapes):
+                for k, v in enumerate(t if t is not None else _dense_strides(shp)):
+                    a.stride[k] = v
+        out = (C.c_int64 * reps)()
+        st = lib.dvm_time_encode(self.program._h, self.shapes, ins, self.n_in, self.scalars, len(scalars),
+                                 self.buf, self.cap, reps, out)
+        if st != 0:
+            raise DvmError(st, "dvm_time_encode")
+        return list(out)
 
     def encode(self, shapes: Sequence[Sequence[int]], scalars: Sequence[float] = (),
                in_strides: Optional[Sequence[Optional[Sequence[int]]]] = None,

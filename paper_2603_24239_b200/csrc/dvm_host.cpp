@@ -7,6 +7,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <chrono>
+
 #include <utility>
 
 #include "../../include/dvm.h"
@@ -1370,6 +1372,22 @@ extern "C" int dvm_encode_strided(const dvm_program* p, const dvm_shape* in_shap
                                   int n_out) {
   return encode_views(p, in_shapes, in_strides, n_in, scalars, n_scalars, out_strides, code, code_capacity,
                       code_size, out_shapes, n_out);
+}
+
+extern "C" int dvm_time_encode(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
+                               const float* scalars, int n_scalars, void* code, size_t code_capacity, int reps,
+                               int64_t* ns_out) {
+  if (reps < 0 || (reps > 0 && !ns_out)) return DVM_ERR_INVALID_ARG;
+  for (int r = 0; r < reps; ++r) {
+    size_t size = 0;
+    const auto t0 = std::chrono::steady_clock::now();
+    const int st = encode_views(p, in_shapes, in_strides, n_in, scalars, n_scalars, nullptr, code, code_capacity, &size,
+                                nullptr, 0);
+    const auto t1 = std::chrono::steady_clock::now();
+    if (st != DVM_OK) return st;
+    ns_out[r] = (int64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(t1 - t0).count();
+  }
+  return DVM_OK;
 }
 
 extern "C" int dvm_encode_batch(int n, const dvm_program* const* programs, const dvm_shape* in_shapes, const int* n_in,
