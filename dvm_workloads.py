@@ -42,6 +42,7 @@ SCALAR_OPS = ("adds", "muls")
 REDUCE_OPS = ("sum", "max", "min")
 COMPARE_OPS = ("gt", "ge", "lt", "le", "eq", "ne")
 DTYPES = ("f32", "bf16")
+INT_DTYPES = ("u8", "i32")   # outputs and casts only (Table 1: Cast; Cmp / IsFinite results stored as 0 / 1)
 
 
 @dataclass
@@ -75,7 +76,7 @@ class OpProgram:
         return self._push(("scalar", op, x, s))
 
     def cast(self, x: int, dtype: str) -> int:
-        assert dtype in DTYPES
+        assert dtype in DTYPES + INT_DTYPES
         return self._push(("cast", x, dtype))
 
     def reduce(self, op: str, x: int, axis: int = -1) -> int:
@@ -93,7 +94,7 @@ class OpProgram:
         return self._push(("select", cond, x, y))
 
     def output(self, x: int, dtype: str) -> int:
-        assert dtype in DTYPES
+        assert dtype in DTYPES + INT_DTYPES
         return self._push(("output", x, dtype))
 
     @property

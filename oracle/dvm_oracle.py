@@ -20,7 +20,8 @@ Per-node definitions follow Table 1 ("Tile-level Virtual Instructions"):
   Add/Sub/Mul/Div/Min/Max  elementwise                       (Table 1, binary rows)
   Adds/Muls                x op scalar                        (Table 1, Adds/Muls)
   Sqrt/Abs/Log/Exp/Round/Floor                                (Table 1, unary rows)
-  Cast                     (dst_dtype)(x)                     (Table 1, Cast)
+  Cast                     (dst_dtype)(x); to an integer type   (Table 1, Cast)
+                           the fraction is dropped (toward zero)
   Sum/Max/Min reduce       [M,size,N] -> [M,1,N]; N = 1 unless a  (Table 1, Sum/Max/Min)
                            reduce node names another axis
   Broadcast                implicit in numpy-style broadcasting (Table 1, Broadcast)
@@ -45,7 +46,7 @@ from __future__ import annotations
 import numpy as np
 from scipy import special as _special
 
-__all__ = ["evaluate", "round_to_bf16", "round_to_f32"]
+__all__ = ["evaluate", "round_to_bf16", "round_to_f32", "cast_to_int"]
 
 
 def round_to_f32(x: np.ndarray) -> np.ndarray:
@@ -83,11 +84,28 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     return out.reshape(x.shape)
 
 
+_INT_RANGE = {"i32": (-2147483648.0, 2147483647.0), "u8": (0.0, 255.0)}
+
+
+def cast_to_int(x: np.ndarray, dtype: str) -> np.ndarray:
+    """Table 1, Cast to an integer type: the fraction is dropped (rounding toward zero, the conversion C defines);
+    the result is returned as float64 holding the integer.  Values outside the type's range take the nearest
+    bound and NaN becomes 0 -- the paper fixes neither ("parity unpinned"; the sweeps stay inside the range)."""
+    lo, hi = _INT_RANGE[dtype]
+    x = np.asarray(x, dtype=np.float64)
+    with np.errstate(invalid="ignore"):
+        t = np.where(x < 0, np.ceil(x), np.floor(x))          # toward zero, written out
+        t = np.where(np.isnan(x), 0.0, np.minimum(np.maximum(t, lo), hi))
+    return t + 0.0                                            # (-0 -> +0: an integer has one zero)
+
+
 def _round_to(x, dtype):
     if dtype == "f32":
         return round_to_f32(x)
     if dtype == "bf16":
         return round_to_bf16(x)
+    if dtype in _INT_RANGE:
+        return cast_to_int(x, dtype)
     raise ValueError(f"unknown dtype {dtype}")
 
 
@@ -193,7 +211,10 @@ def _evaluate(nodes, inputs, params, ft):
                 c, x, y = np.broadcast_arrays(vals[n[1]], vals[n[2]], vals[n[3]])
                 vals[i] = np.where(c != 0, x, y)
             elif kind == "output":
-                outs.append(np.array(vals[n[1]], dtype=ft))
+                # an output stored as an integer type holds the integer the cast gives (Table 1, Cast; Cmp and
+                # IsFinite values are 0 / 1 already); floating outputs are returned unrounded
+                v = vals[n[1]]
+                outs.append(np.array(cast_to_int(v, n[2]) if n[2] in _INT_RANGE else v, dtype=ft))
             else:
                 raise ValueError(f"unknown node kind {kind}")
     return outs

@@ -533,3 +533,39 @@ def test_reduce_over_the_penultimate_and_outer_axes():
     q.output(q.binary("div", a, q.reduce("sum", a, -2)), "f32")
     z = np.abs(RNG.standard_normal((7, 6))) + 0.1
     assert np.allclose(orc.evaluate(q.nodes, [z])[0].sum(axis=0), 1.0, rtol=1e-14)
+
+
+# ---------------------------------------------------------------- integer types (Table 1: Cast, Cmp, IsFinite)
+def test_cast_to_int_drops_the_fraction_toward_zero():
+    """Hand table, and numpy's own trunc and C-style astype on values inside the range."""
+    x = np.array([0.0, 0.5, 0.999, 1.0, 1.5, 2.5, -0.5, -0.999, -1.0, -1.5, -2.5, 254.9, 255.0, 1e6 + 0.75, -1e6 - 0.75])
+    want_i32 = np.array([0, 0, 0, 1, 1, 2, 0, 0, -1, -1, -2, 254, 255, 1000000, -1000000], dtype=np.float64)
+    assert np.array_equal(orc.cast_to_int(x, "i32"), want_i32)
+    assert np.array_equal(orc.cast_to_int(x, "i32"), np.trunc(x))
+    assert np.array_equal(orc.cast_to_int(x, "i32"), x.astype(np.int32).astype(np.float64))
+    # u8: the same inside 0..255; outside, the nearest bound
+    assert np.array_equal(orc.cast_to_int(np.array([0.2, 7.9, 255.0, 255.9, 300.0, -3.0]), "u8"), np.array([0, 7, 255, 255, 255, 0.0]))
+    assert not np.any(np.signbit(orc.cast_to_int(np.array([-0.5, -0.0]), "i32")))    # one zero
+    rng = np.random.default_rng(3)
+    r = rng.uniform(-1e5, 1e5, 10000)
+    assert np.array_equal(orc.cast_to_int(r, "i32"), np.trunc(r))
+
+
+def test_integer_outputs_of_cast_compare_and_isfinite():
+    p = wl.OpProgram("ints")
+    a, b = p.input("f32", 2), p.input("f32", 2)
+    p.output(p.cast(p.scalar("muls", a, 10.0), "i32"), "i32")       # (int)(10 a)
+    p.output(p.compare("gt", a, b), "u8")                              # a > b as 0 / 1
+    p.output(p.unary("isfinite", p.binary("div", a, b)), "u8")
+    p.output(p.scalar("muls", a, 10.0), "i32")                         # the store itself casts
+    av = np.array([[0.26, -0.26, 1.0, -7.77]]); bv = np.array([[0.25, 0.0, 1.0, 0.0]])
+    o = orc.evaluate(p.nodes, [av, bv])
+    assert np.array_equal(o[0], [[2, -2, 10, -77]])
+    assert np.array_equal(o[1], [[1, 0, 0, 0]])
+    assert np.array_equal(o[2], [[1, 0, 1, 0]])                        # -0.26 / 0 and -7.77 / 0 are infinite
+    assert np.array_equal(o[3], o[0])
+    # a cast in the middle of a program is a rounding point: (int)(2.7) + 0.5 = 2.5
+    q = wl.OpProgram("mid")
+    x = q.input("f32", 1)
+    q.output(q.scalar("adds", q.cast(x, "i32"), 0.5), "f32")
+    assert np.array_equal(orc.evaluate(q.nodes, [np.array([2.7, -2.7])])[0], [2.5, -1.5])
