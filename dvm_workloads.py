@@ -210,6 +210,29 @@ def program_if_else_add() -> OpProgram:
     return p
 
 
+def program_if_else_add_mask() -> OpProgram:
+    """The same, with the comparison's 0 / 1 also stored, as u8 (Table 1, Cmp: integer output, bit-exact)."""
+    p = OpProgram("if_else_add_mask")
+    a, b, x, y = (p.input("f32", 3) for _ in range(4))
+    c = p.compare("gt", a, b)
+    s = p.select(c, p.scalar("muls", x, 2.0), p.scalar("muls", x, 4.0))
+    p.output(p.binary("add", s, y), "f32")
+    p.output(c, "u8")
+    return p
+
+
+def program_quantise(in_dtype: str = "f32", scale: float = 10.0) -> OpProgram:
+    """Table 1, Cast: (int)(scale * x) stored as i32, the same clipped into a byte stored as u8, and the cast value
+    used again in fp32 arithmetic ((int)(scale * x) * 0.5)."""
+    p = OpProgram("quantise_" + in_dtype)
+    x = p.input(in_dtype, 2)
+    q = p.cast(p.scalar("muls", x, scale), "i32")
+    p.output(q, "i32")
+    p.output(p.scalar("adds", p.scalar("muls", x, scale), 128.0), "u8")
+    p.output(p.scalar("muls", q, 0.5), "f32")
+    return p
+
+
 def program_head_transpose_add() -> OpProgram:
     """out[b,h,s,:] = 0.5 * x[b,h,s,:] + y[b,h,s,:], bf16 rank 4: the elementwise consumer of an attention head
     transpose.  x is given as a VIEW (stored [B,S,H,D], read as [B,H,S,D]: Table 1, ViewLoad); y, out dense."""

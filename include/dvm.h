@@ -50,7 +50,10 @@ enum {
   DVM_ERR_TOO_LARGE = -10        /* program / stack exceeds a fixed library limit */
 };
 
-enum { DVM_F32 = 0, DVM_BF16 = 1 };
+/* Element types.  U8 and I32 are for outputs and for dvm_program_cast (Table 1, Cast; a Cmp / IsFinite result is
+ * stored as 0 / 1): the fp32 value is converted toward zero, values outside the type's range take the nearest
+ * bound, NaN gives 0.  Inputs are F32 or BF16. */
+enum { DVM_F32 = 0, DVM_BF16 = 1, DVM_U8 = 2, DVM_I32 = 3 };
 
 /* Unary operators.  EXP SQRT ABS LOG FLOOR ROUND ISFINITE are Table 1's; the others are
  * extensions the LLM programs need (Table 1 has no erf / sigmoid / rsqrt). */
@@ -101,7 +104,8 @@ int dvm_program_compare(dvm_program* p, int op, int x, int y, int* value_id);
 /* Table 1 Select: cond != 0 ? x : y elementwise (operands broadcast).  Cmp and Select take tile operands:
  * an operand that is one value per row makes dvm_encode return DVM_ERR_UNSUPPORTED. */
 int dvm_program_select(dvm_program* p, int cond, int x, int y, int* value_id);
-/* Table 1 Cast: rounds the value to `dtype` (nearest even); values stay fp32 in registers. */
+/* Table 1 Cast: rounds the value to `dtype` (BF16 / F32: nearest even; U8 / I32: toward zero, kept inside the
+ * type's range); values stay fp32 in registers. */
 int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
 /* Table 1 Sum / Max / Min of [M, size, N] over `size` -> [M, 1, N] (the reduced axis stays with size 1).
  * `axis` counts from the end of x's (right-aligned) shape: -1 the last axis (N = 1: threads of a row combine

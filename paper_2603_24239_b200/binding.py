@@ -21,8 +21,8 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 DVM_MAX_RANK = 6
-F32, BF16 = 0, 1
-DTYPES = {"f32": F32, "bf16": BF16}
+F32, BF16, U8, I32 = 0, 1, 2, 3
+DTYPES = {"f32": F32, "bf16": BF16, "u8": U8, "i32": I32}   # u8 / i32: outputs and casts (Table 1, Cast)
 UNARY = {"exp": 0, "sqrt": 1, "rsqrt": 2, "abs": 3, "log": 4, "erf": 5, "sigmoid": 6, "neg": 7,
          "recip": 8, "floor": 9, "round": 10, "tanh": 11, "isfinite": 12}
 BINARY = {"add": 0, "sub": 1, "mul": 2, "div": 3, "min": 4, "max": 5, "pow": 6}

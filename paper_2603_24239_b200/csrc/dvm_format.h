@@ -97,7 +97,10 @@ enum {
   DVM_OPD_WORDS = 8
 };
 
-enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1 };
+enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1,
+       DVM_DT_U8 = 2, DVM_DT_I32 = 3 };  // outputs only: the stored value is the fp32 register converted toward zero (Table 1, Cast)
+// log2 of an element's bytes: bf16 1, fp32 / i32 2, u8 0
+#define DVM_DT_LG_ES(dt) ((dt) == DVM_DT_BF16 ? 1 : ((dt) == DVM_DT_U8 ? 0 : 2))
 
 // ---- limits ----
 #define DVM_VM_THREADS 256       // threads per CTA of the interpreter
@@ -131,7 +134,9 @@ enum {
   DVM_U_ERF = 5, DVM_U_SIGMOID = 6, DVM_U_NEG = 7, DVM_U_RECIP = 8, DVM_U_FLOOR = 9,
   DVM_U_ROUND = 10, DVM_U_TANH = 11, DVM_U_RND_BF16 = 12,
   DVM_U_ISFINITE = 13,  // Table 1, IsFinite: 1.0 for a finite value, else 0.0 (tile class: extended variant only)
-  DVM_U_NUN = 14
+  DVM_U_TRUNC_I32 = 14, // Table 1, Cast to i32: the fraction dropped toward zero, the value kept inside the type's range (fp32 register)
+  DVM_U_TRUNC_U8 = 15,  // ... to u8
+  DVM_U_NUN = 16
 };
 // the two-tile-operand class of the extended variant: the comparisons (Table 1, Cmp) and Pow (Table 1)
 enum { DVM_C_GT = 0, DVM_C_GE = 1, DVM_C_LT = 2, DVM_C_LE = 3, DVM_C_EQ = 4, DVM_C_NE = 5,
@@ -163,7 +168,7 @@ enum {
   DVM_OP_BINI = 0x10,  // 0x10 + arith; len 2, word1 = fp32 immediate  : ACC = ACC op imm     (Adds / Muls)
   DVM_OP_BIN = 0x18,   // 0x18 + arith; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC op L[a]
   DVM_OP_BINS = 0x20,  // 0x20 + arith; a = scalar register            : ACC = ACC op S[a]    (row broadcast)
-  DVM_OP_UN = 0x28,    // 0x28 + unary (13)                            : ACC = f(ACC)
+  DVM_OP_UN = 0x28,    // 0x28 + unary (16)                            : ACC = f(ACC)
   DVM_OP_RED = 0x38,   // 0x38 + reduce (4); a = dst scalar register   : S[a] = reduce(ACC) over the row
   DVM_OP_LD2 = 0x40,   // 0x40 + arith; a = local register x, b = local register y | dtype(x) << 6 | dtype(y) << 7
                        //                                             : ACC = L[x] op L[y]   (fused copy + arithmetic)

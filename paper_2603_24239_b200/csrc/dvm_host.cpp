@@ -115,7 +115,7 @@ extern "C" int dvm_program_scalar_param(dvm_program* p, int op, int x, int param
 }
 
 extern "C" int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id) {
-  if (!valid_value(p, x) || (dtype != DVM_F32 && dtype != DVM_BF16)) return DVM_ERR_INVALID_ARG;
+  if (!valid_value(p, x) || dtype < DVM_F32 || dtype > DVM_I32) return DVM_ERR_INVALID_ARG;
   Node n = {};
   n.kind = NK_CAST;
   n.dtype = (uint8_t)dtype;
@@ -171,7 +171,7 @@ extern "C" int dvm_program_matmul(dvm_program* p, int a, int b, int* value_id) {
 }
 
 extern "C" int dvm_program_output(dvm_program* p, int x, int dtype) {
-  if (!valid_value(p, x) || (dtype != DVM_F32 && dtype != DVM_BF16)) return DVM_ERR_INVALID_ARG;
+  if (!valid_value(p, x) || dtype < DVM_F32 || dtype > DVM_I32) return DVM_ERR_INVALID_ARG;
   if (p->finalized) return DVM_ERR_INVALID_ARG;
   if (p->n_outputs >= DVM_MAX_TENSORS) return DVM_ERR_TOO_LARGE;
   p->outputs[p->n_outputs].value = (int16_t)x;
@@ -569,7 +569,8 @@ static bool gen_body(Enc& e) {
         emit(e, (uint32_t)(n.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL) | ((uint32_t)sx << 8));
         emit(e, f2u(s));
       } else {  // unary or rounding cast
-        uint32_t u = n.kind == NK_CAST ? (uint32_t)DVM_U_RND_BF16 : (uint32_t)kUnMap[n.op];
+        uint32_t u = n.kind == NK_CAST ? (uint32_t)(n.dtype == DVM_I32 ? DVM_U_TRUNC_I32 : n.dtype == DVM_U8 ? DVM_U_TRUNC_U8 : DVM_U_RND_BF16)
+                                       : (uint32_t)kUnMap[n.op];
         emit(e, DVM_INSN(DVM_OP_SOP, 2, d, DVM_SK_UN));
         emit(e, u | ((uint32_t)sx << 8));
       }
@@ -702,8 +703,8 @@ static bool gen_body(Enc& e) {
         float s = n.param >= 0 ? e.scalars[n.param] : n.imm;
         emit(e, DVM_INSN(DVM_OP_BINI + (n.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL), 2, 0, 0));
         emit(e, f2u(s));
-      } else {  // NK_CAST to bf16 (casts to f32 are aliases)
-        emit(e, DVM_INSN(DVM_OP_UN + DVM_U_RND_BF16, 1, 0, 0));
+      } else {  // NK_CAST to bf16 or to an integer type (casts to f32 are aliases)
+        emit(e, DVM_INSN(DVM_OP_UN + (n.dtype == DVM_I32 ? DVM_U_TRUNC_I32 : n.dtype == DVM_U8 ? DVM_U_TRUNC_U8 : DVM_U_RND_BF16), 1, 0, 0));
       }
       e.acc = (int16_t)i;
       release(e, x);
@@ -940,13 +941,14 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   int primary = -1;
   for (int o = 0; o < e.n_opd && primary < 0; ++o) {
     const Operand& od = e.opd[o];
-    if (od.col_stride != 1 || od.cs != 1) continue;
+    if (od.col_stride != 1 || od.cs != 1 || od.dtype > DVM_DT_BF16) continue;  // (never an integer output: the chunks follow 2- or 4-byte elements)
     bool full = true;
     for (int g = 0; g < 3; ++g) if (outer[g] > 1 && od.ostride[g] == 0) full = false;
     if (full) primary = o;
   }
   if (primary < 0) {
-    for (int o = 0; o < e.n_opd && primary < 0; ++o) if (e.opd[o].col_stride == 1 && e.opd[o].cs == 1) primary = o;
+    for (int o = 0; o < e.n_opd && primary < 0; ++o)
+      if (e.opd[o].col_stride == 1 && e.opd[o].cs == 1 && e.opd[o].dtype <= DVM_DT_BF16) primary = o;
   }
   // combined results: the rows a warp holds are combined slot by slot, so every row must map its columns to
   // the same slots -- no operand to align the chunks to, every operand is read at its own phase
@@ -1137,7 +1139,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
         for (int o = 0; o < e.n_opd; ++o) {
           const Operand& od = e.opd[o];
           if (od.col_stride != 1) continue;
-          const int64_t es = od.dtype == DVM_DT_BF16 ? 2 : 4;
+          const int64_t es = (int64_t)1 << DVM_DT_LG_ES(od.dtype);
           int64_t amp = 4;  // in quarters: 4 = no amplification
           if (od.cs > 1 && od.ostride[0] == 1) {
             const int64_t nT = G < 32 ? G : 32, nR = 32 / nT;
@@ -1505,7 +1507,8 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   for (uint32_t o = 0; o < n_opd; ++o) {
     uint32_t info = ot[o * DVM_OPD_WORDS + DVM_OPD_INFO];
     if ((info & 0xff) >= n_tensors) return DVM_ERR_BAD_CODE;
-    if (((info >> 8) & 0xff) > DVM_DT_BF16) return DVM_ERR_BAD_CODE;
+    if (((info >> 8) & 0xff) > (uint32_t)((info & 0xff) < n_in ? DVM_DT_BF16 : DVM_DT_I32)) return DVM_ERR_BAD_CODE;  // integer types: outputs only
+    if (((info >> 24) & 1) && ((info >> 8) & 0xff) > DVM_DT_BF16) return DVM_ERR_BAD_CODE;                            // ... and never the primary operand
     if (((info >> 16) & 0xff) > 1) return DVM_ERR_BAD_CODE;
     const uint32_t combine = (info >> 26) & 3;
     if (ot[o * DVM_OPD_WORDS + 3] | ot[o * DVM_OPD_WORDS + 5]) return DVM_ERR_BAD_CODE;  // 32-bit strides
@@ -1604,7 +1607,7 @@ static void outf(Out& o, const char* fmt, ...) {
 }
 static const char* kArith[8] = {"add", "sub", "rsub", "mul", "div", "rdiv", "min", "max"};
 static const char* kUn[DVM_U_NUN] = {"exp", "sqrt", "rsqrt", "abs", "log", "erf", "sigmoid", "neg",
-                                     "recip", "floor", "round", "tanh", "rnd_bf16", "isfinite"};
+                                     "recip", "floor", "round", "tanh", "rnd_bf16", "isfinite", "trunc_i32", "trunc_u8"};
 static const char* kRed[DVM_R_NRED] = {"sum", "max", "min", "sumsq"};
 }  // namespace
 
@@ -1637,7 +1640,8 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     uint32_t info = d[0];
     outf(o, "  operand m%u: %s%u %s col_stride=%u strides=[%lld,%lld,%lld]%s\n", k,
          (info & 0xff) < n_in ? "in" : "out", (info & 0xff) < n_in ? (info & 0xff) : (info & 0xff) - n_in,
-         ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : "f32", ((info >> 16) & 0xff) ? d[DVM_OPD_COLSTRIDE] : 0u,
+         ((info >> 8) & 0xff) == DVM_DT_BF16 ? "bf16" : ((info >> 8) & 0xff) == DVM_DT_U8 ? "u8" : ((info >> 8) & 0xff) == DVM_DT_I32 ? "i32" : "f32",
+         ((info >> 16) & 0xff) ? d[DVM_OPD_COLSTRIDE] : 0u,
          (long long)d[2], (long long)d[4], (long long)d[6],
          (info >> 24) & 1 ? " primary" : (((info >> 26) & 3) == 1 ? " combine=sum" : ((info >> 26) & 3) == 2 ? " combine=max" : ((info >> 26) & 3) == 3 ? " combine=min" : ""));
   }

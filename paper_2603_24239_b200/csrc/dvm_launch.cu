@@ -140,7 +140,7 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
   for (uint32_t o = 0; o < n_opd; ++o) {
     uint32_t info = ot[o * DVM_OPD_WORDS];
     uintptr_t a = (uintptr_t)tensors[info & 0xff];
-    uintptr_t es = ((info >> 8) & 0xff) == DVM_DT_BF16 ? 2 : 4;
+    uintptr_t es = (uintptr_t)1 << DVM_DT_LG_ES((info >> 8) & 0xff);
     if (a % es) return DVM_ERR_INVALID_ARG;
   }
   // every input register learns its tensor's address modulo 16 (the images keep that phase)
@@ -271,7 +271,8 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       const uint32_t info = ot[ib * DVM_OPD_WORDS + DVM_OPD_INFO];
       if (!((info >> 25) & 1u) || ((info >> 26) & 3u)) return 0;  // a stored view / a combined result: general interpreter
       const unsigned long long a = (unsigned long long)(uintptr_t)tensors[info & 0xff];
-      push(DVM_LK_W0(DVM_LK_STG, 0, ((info >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2, 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
+      const uint32_t sdt = (info >> 8) & 0xff;   // sub: 0 fp32 / bf16 as they are, 1: converted to i32, 2: to u8
+      push(DVM_LK_W0(DVM_LK_STG, sdt == DVM_DT_I32 ? 1 : sdt == DVM_DT_U8 ? 2 : 0, DVM_DT_LG_ES(sdt), 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
     } else if (op == DVM_OP_STA) {
       push(DVM_LK_W0(DVM_LK_STA, 0, 0, 0), (lt[ia] & 0xffffu) * DVM_LOCAL_UNIT, 0, 0);
     } else if (op == DVM_OP_LSS) {

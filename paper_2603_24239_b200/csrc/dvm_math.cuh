@@ -68,6 +68,17 @@ __device__ __forceinline__ float2 packed_erf(float2 x) {
   return make_float2(ax.x >= 1.0f ? copysignf(big.x, x.x) : small.x, ax.y >= 1.0f ? copysignf(big.y, x.y) : small.y);  // (a NaN takes the product's way)
 }
 
+// Table 1, Cast to an integer type, as an fp32 value: the fraction dropped toward zero (+ 0: one zero), then kept
+// inside the type's range (2^31 stands for the largest i32: the store's conversion saturates); NaN gives 0.
+// the stored forms: an i32 word, a byte (conversions toward zero that saturate; NaN gives 0)
+__device__ __forceinline__ uint32_t store_i32(float x) { return (uint32_t)__float2int_rz(x); }
+__device__ __forceinline__ uint32_t store_u8(float x) { return min(__float2uint_rz(x), 255u); }
+__device__ __forceinline__ uint32_t pack_u8x4(float a, float b, float c, float d) {
+  return store_u8(a) | (store_u8(b) << 8) | (store_u8(c) << 16) | (store_u8(d) << 24);
+}
+__device__ __forceinline__ float trunc_i32(float x) { return x != x ? 0.0f : fminf(fmaxf(truncf(x) + 0.0f, -2147483648.0f), 2147483648.0f); }
+__device__ __forceinline__ float trunc_u8(float x) { return x != x ? 0.0f : fminf(fmaxf(truncf(x) + 0.0f, 0.0f), 255.0f); }
+
 __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
   switch (op) {
     case DVM_A_ADD: return a + b;
@@ -96,6 +107,8 @@ __device__ __forceinline__ float scalar_unary(int op, float x) {
     case DVM_U_ROUND: return rintf(x);
     case DVM_U_TANH: return tanhf(x);
     case DVM_U_ISFINITE: return fabsf(x) < __int_as_float(0x7f800000) ? 1.0f : 0.0f;  // false for NaN, too
+    case DVM_U_TRUNC_I32: return trunc_i32(x);
+    case DVM_U_TRUNC_U8: return trunc_u8(x);
     default: return round_bf16(x);
   }
 }

@@ -230,6 +230,8 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
       nb++;
     } else if (n.kind == NK_CAST && n.dtype == DVM_F32) {
       e.alias[i] = n.x;  // values are fp32 already
+    } else if (n.kind == NK_CAST && n.dtype > DVM_BF16) {
+      return DVM_ERR_UNSUPPORTED;  // integer types exist in vector programs only
     } else if (n.kind == NK_REDUCE) {
       return DVM_ERR_UNSUPPORTED;
     }
@@ -292,6 +294,7 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
     if (e.n_opd >= DVM_MAX_OPERANDS) return DVM_ERR_TOO_LARGE;
     MmOperand& od = e.opd[e.n_opd];
     od.slot = n_in + o;
+    if (p->outputs[o].dtype > DVM_BF16) return DVM_ERR_UNSUPPORTED;  // integer outputs exist in vector programs only
     od.dtype = p->outputs[o].dtype == DVM_BF16 ? DVM_DT_BF16 : DVM_DT_F32;
     od.col_stride = 1;
     od.row_stride = N;

@@ -795,6 +795,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
             DVM_UN_CASE(DVM_U_ROUND, rintf(x))
             DVM_UN_CASE(DVM_U_TANH, tanhf(x))
+            DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
+            DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
             default:
               if constexpr (EXT >= 1) {  // Table 1, IsFinite (programs that use it on a tile run the extended variant)
                 if (op - DVM_OP_UN == DVM_U_ISFINITE) {
@@ -895,7 +897,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
             const uint32_t info = CW(d + DVM_OPD_INFO);
             const int dt = (info >> 8) & 0xff;
-            const int lg_es = dt == DVM_DT_BF16 ? 1 : 2;
+            const int lg_es = DVM_DT_LG_ES(dt);
             unsigned long long el0 = (unsigned long long)c.row * CW(prog + DVM_H_COLS) + c.col0;
             long long cstep = 1;  // elements between two columns of the output
             if constexpr (VIEWS) {  // programs with a strided output run the views variant (DVM_F_VIEWS)
@@ -955,7 +957,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             }
             char* q0 = p + ((long long)c.cbase << lg_es);
             const long long qstep = (long long)((G << c.lgW) << lg_es);
-            const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0 && (!VIEWS || cstep == 1);
+            // (a chunk of u8 is W bytes: its vector store wants that alignment; everything else goes in 16-byte vectors)
+            const bool al = (reinterpret_cast<uintptr_t>(q0) & (dt == DVM_DT_U8 ? (uintptr_t)(W - 1) : (uintptr_t)15)) == 0 && (!VIEWS || cstep == 1);
             const uint32_t fast = al ? c.fullmask : 0u;
             const uint32_t slow = c.partmask | (c.fullmask & ~fast);
             constexpr uint32_t ALL8 = (V / 8 >= 32) ? 0xffffffffu : ((1u << (V / 8)) - 1u);
@@ -982,6 +985,33 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                   }
                   *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
+              }
+            } else if (dt == DVM_DT_U8) {  // Table 1, Cast: a chunk is W bytes
+              if (W == 8) {
+  #pragma unroll
+                for (int j = 0; j < V / 8; ++j)
+                  if ((fast >> j) & 1)
+                    *reinterpret_cast<uint2*>(q0 + j * qstep) = make_uint2(pack_u8x4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y),
+                                                                           pack_u8x4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y));
+              } else {
+  #pragma unroll
+                for (int j = 0; j < V / 4; ++j)
+                  if ((fast >> j) & 1)
+                    *reinterpret_cast<uint32_t*>(q0 + j * qstep) = pack_u8x4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
+              }
+            } else if (dt == DVM_DT_I32) {
+              if (W == 8) {
+  #pragma unroll
+                for (int j = 0; j < V / 8; ++j)
+                  if ((fast >> j) & 1) {
+                    *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[4 * j].x), store_i32(A[4 * j].y), store_i32(A[4 * j + 1].x), store_i32(A[4 * j + 1].y));
+                    *reinterpret_cast<uint4*>(q0 + j * qstep + 16) = make_uint4(store_i32(A[4 * j + 2].x), store_i32(A[4 * j + 2].y), store_i32(A[4 * j + 3].x), store_i32(A[4 * j + 3].y));
+                  }
+              } else {
+  #pragma unroll
+                for (int j = 0; j < V / 4; ++j)
+                  if ((fast >> j) & 1)
+                    *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[2 * j].x), store_i32(A[2 * j].y), store_i32(A[2 * j + 1].x), store_i32(A[2 * j + 1].y));
               }
             } else if (W == 8) {
   #pragma unroll
@@ -1021,7 +1051,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                     if (col >= 0 && col < c.ncols) {
                       const long long ce = VIEWS ? (long long)col * cstep : (long long)col;  // scattered columns (Table 1, ViewStore)
                       if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p + ce * 2) = __float2bfloat16_rn(val);
-                      else *reinterpret_cast<float*>(p + ce * 4) = val;
+                      else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p + ce * 4) = val;
+                      else if (dt == DVM_DT_I32) *reinterpret_cast<uint32_t*>(p + ce * 4) = store_i32(val);
+                      else *reinterpret_cast<unsigned char*>(p + ce) = (unsigned char)store_u8(val);
                     }
                   }
                 }
@@ -1030,11 +1062,13 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           } else if (op == DVM_OP_STS) {
             const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
             const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
-            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << (dt == DVM_DT_BF16 ? 1 : 2)));
+            char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << DVM_DT_LG_ES(dt)));
             const float v = s_S[ia][tid];
             if (c.ncols > 0 && (tid & (G - 1)) == 0 && c.col0 == 0) {
               if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
-              else *reinterpret_cast<float*>(p) = v;
+              else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p) = v;
+              else if (dt == DVM_DT_I32) *reinterpret_cast<uint32_t*>(p) = store_i32(v);
+              else *reinterpret_cast<unsigned char*>(p) = (unsigned char)store_u8(v);
             }
           } else if (op != DVM_OP_NOP) {
             err = ST_BAD_CODE;

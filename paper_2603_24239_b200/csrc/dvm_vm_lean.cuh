@@ -625,6 +625,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             DVM_UN_CASE(DVM_U_NEG, -x)
             DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
             DVM_UN_CASE(DVM_U_RND_BF16, round_bf16(x))
+            DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
+            DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
             default:
               if constexpr (HEAVY) {
                 switch (sub) {
@@ -708,10 +710,38 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           char* p = reinterpret_cast<char*>(base + (el0 << lg_es));
           char* q0 = p + ((long long)cbase << lg_es);
           const long long qstep = (long long)((G << lgW) << lg_es);
-          const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
+          // (a chunk of u8 is W bytes: its vector store wants that alignment; everything else goes in 16-byte vectors)
+          const bool al = (reinterpret_cast<uintptr_t>(q0) & (lg_es == 0 ? (uintptr_t)((1 << lgW) - 1) : (uintptr_t)15)) == 0;
           const uint32_t fast = al ? fullmask : 0u;
           const uint32_t slow = partmask | (fullmask & ~fast);
-          if (lg_es == 1) {  // bf16: chunks of 8, chunk j = group j
+          if (sub == 2) {  // Table 1, Cast: stored as u8, a chunk is W bytes
+            if (lgW == 3) {
+#pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint2*>(q0 + j * qstep) = make_uint2(pack_u8x4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y),
+                                                                         pack_u8x4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y));
+            } else {
+#pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint32_t*>(q0 + j * qstep) = pack_u8x4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
+            }
+          } else if (sub == 1) {  // stored as i32
+            if (lgW == 3) {
+#pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1) {
+                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[4 * j].x), store_i32(A[4 * j].y), store_i32(A[4 * j + 1].x), store_i32(A[4 * j + 1].y));
+                  *reinterpret_cast<uint4*>(q0 + j * qstep + 16) = make_uint4(store_i32(A[4 * j + 2].x), store_i32(A[4 * j + 2].y), store_i32(A[4 * j + 3].x), store_i32(A[4 * j + 3].y));
+                }
+            } else {
+#pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[2 * j].x), store_i32(A[2 * j].y), store_i32(A[2 * j + 1].x), store_i32(A[2 * j + 1].y));
+            }
+          } else if (lg_es == 1) {  // bf16: chunks of 8, chunk j = group j
 #pragma unroll
             for (int j = 0; j < V / 8; ++j)
               if ((fast >> j) & 1) {
@@ -750,7 +780,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
                   const bool in_slow = lgW == 3 ? true : ((gm >> (e >> 2)) & 1u) != 0;
                   const float val = (e & 1) ? A[4 * g + (e >> 1)].y : A[4 * g + (e >> 1)].x;
                   if (in_slow && col >= 0 && col < r.ncols) {
-                    if (lg_es == 1) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
+                    if (sub == 2) *reinterpret_cast<unsigned char*>(p + (long long)col) = (unsigned char)store_u8(val);
+                    else if (sub == 1) *reinterpret_cast<uint32_t*>(p + (long long)col * 4) = store_i32(val);
+                    else if (lg_es == 1) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
                     else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
                   }
                 }
@@ -774,11 +806,13 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
         case DVM_LK_STS: {
           const uint32_t d = prog + rec.y;
           const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
-          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(prog, d, r) << (dt == DVM_DT_BF16 ? 1 : 2)));
+          char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(prog, d, r) << DVM_DT_LG_ES(dt)));
           const float v = s_S[ra][tid];
           if (r.ncols > 0 && t == 0 && r.col0 == 0) {
             if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
-            else *reinterpret_cast<float*>(p) = v;
+            else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p) = v;
+            else if (dt == DVM_DT_I32) *reinterpret_cast<uint32_t*>(p) = store_i32(v);
+            else *reinterpret_cast<unsigned char*>(p) = (unsigned char)store_u8(v);
           }
         } break;
         case DVM_LK_BCS: {

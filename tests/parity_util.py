@@ -18,7 +18,7 @@ import dvm_workloads as wl
 import paper_2603_24239_b200 as dvm
 from oracle import dvm_oracle as orc
 
-TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16, "u8": torch.uint8, "i32": torch.int32}
 R_TOL = {"f32": 1e-5, "bf16": 2e-2}
 
 
@@ -37,7 +37,7 @@ def gpu_run(prog: wl.OpProgram, inputs, params=(), stream=None, poison=True):
     for shp, node in zip(code.out_shapes, prog.output_nodes):
         o = torch.empty(shp, dtype=TORCH_DT[node[2]], device="cuda")
         if poison:
-            o.fill_(float("nan"))
+            o.fill_(float("nan") if o.dtype.is_floating_point else 123)
         outs.append(o)
     torch.cuda.synchronize()
     dvm.launch(code, dev_in + outs, stream)
