@@ -288,7 +288,12 @@ int dvm_launch_stacked_noalloc(int n_programs, const void* const* codes, const s
  * memory the caller provides (`staging`, device pointer, staging_bytes >= sum of
  * all tensor sizes rounded up to 256 B each), launches, copies the outputs back
  * and synchronises the stream.  host_tensors[i] has tensor_bytes[i] bytes;
- * pinned host memory makes the copies asynchronous. */
+ * pinned host memory makes the copies asynchronous.
+ * When every tensor of a vector program either follows the tiles (a dense operand) or is a row vector, and the
+ * tensors total 64 MB or more, the call pipelines: the tiles run in chunks (Algorithm 2's tile ranges), each chunk
+ * copying its input rows in, executing and copying its output rows out on one of three library-owned streams, so
+ * that copies in both directions overlap execution.  The result is the same; the call still returns after everything
+ * has finished on `cuda_stream`. */
 int dvm_run_host(const void* code, size_t code_size, void* const* host_tensors,
                  const size_t* tensor_bytes, int n_tensors, void* staging, size_t staging_bytes,
                  void* cuda_stream);

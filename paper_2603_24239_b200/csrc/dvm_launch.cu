@@ -168,7 +168,7 @@ int place_program(uint32_t* dst, const uint32_t* code, void* const* tensors, int
 // ---- the linker of the lean interpreter (see dvm_link.h) ----
 // Turns the placed copy of one verified vector program at dst (word index `at` of the parameter block) into its
 // linked form: header, tables and load section stay, the compute section is replaced by records (which start at
-// a word index = 2 mod 4 of the block: 16-byte aligned in the kernel's parameter space).  `src` is the encoded
+// a word index = 0 mod 4 of the block: 16-byte aligned in the kernel's parameter space).  `src` is the encoded
 // program, `tensors` its device pointers, `max_words` the room at dst.  Returns the words the linked program
 // takes, or 0 when it cannot be linked (no room, or an instruction only the general interpreter has).
 uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const uint32_t* src, void* const* tensors) {
@@ -272,7 +272,7 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       if (!((info >> 25) & 1u) || ((info >> 26) & 3u)) return 0;  // a stored view / a combined result: general interpreter
       const unsigned long long a = (unsigned long long)(uintptr_t)tensors[info & 0xff];
       const uint32_t sdt = (info >> 8) & 0xff;   // sub: 0 fp32 / bf16 as they are, 1: converted to i32, 2: to u8
-      push(DVM_LK_W0(DVM_LK_STG, sdt == DVM_DT_I32 ? 1 : sdt == DVM_DT_U8 ? 2 : 0, DVM_DT_LG_ES(sdt), 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
+      push(DVM_LK_W0(sdt > DVM_DT_BF16 ? DVM_LK_STGI : DVM_LK_STG, sdt == DVM_DT_I32 ? 1 : sdt == DVM_DT_U8 ? 2 : 0, DVM_DT_LG_ES(sdt), 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
     } else if (op == DVM_OP_STA) {
       push(DVM_LK_W0(DVM_LK_STA, 0, 0, 0), (lt[ia] & 0xffffu) * DVM_LOCAL_UNIT, 0, 0);
     } else if (op == DVM_OP_LSS) {
@@ -334,9 +334,9 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
     rec[m++] = r;
   }
   n = m;
-  // the records start at a word index = 2 mod 4 of the parameter block (16-byte aligned in the kernel's parameter space)
+  // the records start at a word index = 0 mod 4 of the parameter block (16-byte aligned in the kernel's parameter space)
   uint32_t rec0 = head;
-  while ((at + rec0) % 4 != 2) ++rec0;
+  while ((at + rec0) % 4 != 0) ++rec0;
   if (rec0 + 4 * (n + 1) > max_words) return 0;
   for (uint32_t i = head; i < rec0; ++i) dst[i] = 0;
   for (uint32_t i = 0; i < n; ++i) memcpy(dst + rec0 + 4 * i, rec[i].w, 16);
@@ -423,12 +423,15 @@ void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* h
     const uint32_t op = DVM_INSN_OP(body[pc]), len = DVM_INSN_LEN(body[pc]);
     if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) {
       const uint32_t u = op - DVM_OP_UN;
-      if (u == DVM_U_SQRT || u == DVM_U_LOG || u == DVM_U_ERF || u == DVM_U_FLOOR || u == DVM_U_ROUND || u == DVM_U_TANH) *heavy = true;
+      if (u == DVM_U_SQRT || u == DVM_U_LOG || u == DVM_U_ERF || u == DVM_U_FLOOR || u == DVM_U_ROUND || u == DVM_U_TANH ||
+          u == DVM_U_TRUNC_I32 || u == DVM_U_TRUNC_U8) *heavy = true;
     }
     pc += len ? len : 1;
   }
 }
 
+static_assert(offsetof(dvm::VMParams<PW_SMALL>, words) % 16 == 0 && offsetof(dvm::VMParams<PW_LARGE>, words) % 16 == 0,
+              "linked records are loaded as 16-byte vectors of the parameter space");
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
 
 // Writes the directory and the programs of a launch into the parameter block P.  `linked`: in the linked form
@@ -463,8 +466,9 @@ int place_all(dvm::VMParams<PW_LARGE>& P, int n_programs, const void* const* cod
 }
 
 // `level` (may be NULL): level[i] of program i, non-decreasing; a program reads what programs of lower levels store.
+// `tile_begin`, `tile_end` (one-program launches without a queue; 0, 0 = all): the range of tiles to run.
 int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
-               bool use_queue, const int* level, cudaStream_t stream) {
+               bool use_queue, const int* level, cudaStream_t stream, uint32_t tile_begin = 0, uint32_t tile_end = 0) {
   // A program that asks for a single tile slot (DVM_F_ONE_SLOT), launched on its own: the lean interpreter runs
   // it with one slot; on the general interpreter the variant with level waits does (every tile held back until
   // the CTA's previous tile is done, nothing waited for).
@@ -491,7 +495,13 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     V = v;
   }
   if (need > PW_LARGE || total_tiles > 0xffffffffull) return DVM_ERR_TOO_LARGE;
-  if (total_tiles == 0) return DVM_OK;
+  if (tile_end) {  // a range of the program's tiles
+    if (n_programs != 1 || use_queue || level || tile_begin > tile_end || tile_end > total_tiles) return DVM_ERR_INVALID_ARG;
+    total_tiles = tile_end;
+  } else {
+    tile_begin = 0;
+  }
+  if (total_tiles == tile_begin) return DVM_OK;
 
   DvmDeviceInfo dev;
   int st = dvm_device_state(&dev);
@@ -512,6 +522,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (st == DVM_ERR_UNSUPPORTED) {
     lean = 0;
     if (one_slot) { level = kOneLevel; use_queue = true; }
+    if (tile_end && use_queue) return DVM_ERR_UNSUPPORTED;  // (tile ranges exist for launches without a work queue)
     st = place_all(P, n_programs, codes, tensors, n_tensors, level, false, &pos);
   }
   if (st != DVM_OK) return st;
@@ -520,6 +531,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.n_words = pos;
   P.use_queue = use_queue ? 1u : 0u;
   P.levels = one_slot ? 2u : (level ? 1u : 0u);
+  P.tile_begin = tile_begin;
+  P.reserved = 0;
   P.status = dev.scratch;
   P.queue = dev.scratch + 8 + 4 * dev.queue_slot;
 
@@ -534,7 +547,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   st = dvm_occupancy(variant, smem, &occ);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
-  int grid = (int)(total_tiles < slots ? total_tiles : slots);
+  const uint64_t run_tiles = total_tiles - tile_begin;
+  int grid = (int)(run_tiles < slots ? run_tiles : slots);
   // Everything is placed and checked: only now touch the caller's memory.  Results that tiles combine
   // atomically are filled with their identity (one small kernel per such output), then the interpreter starts.
   st = prefill_all(n_programs, codes, tensors, stream);
@@ -595,6 +609,48 @@ extern "C" int dvm_launch_stacked_levels(int n_programs, const void* const* code
   return launch_vec(n_programs, codes, tensors, n_tensors, true, level, (cudaStream_t)cuda_stream);
 }
 
+// dvm_run_host pipelines when the program allows it: every tensor either follows the tiles row block by row block
+// (a dense operand: the rows of tile t are one byte range) or is a row vector shared by all rows.  The tiles are then
+// cut into chunks; chunk k copies its input rows to the device, runs its tiles and copies its output rows back on
+// stream k mod 3 of three library-owned streams, so that the copies of one chunk (PCIe in both directions) overlap
+// the execution of another.
+namespace {
+constexpr int kPipeStreams = 3;
+struct PipeStreams { bool ready = false; cudaStream_t s[kPipeStreams]; cudaEvent_t done[kPipeStreams]; cudaEvent_t start; };
+PipeStreams g_pipe[MAX_DEVICES];
+
+int pipe_streams(PipeStreams** out) {
+  int dev = 0;
+  DVM_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return DVM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_mu);
+  PipeStreams& p = g_pipe[dev];
+  if (!p.ready) {
+    for (int i = 0; i < kPipeStreams; ++i) {
+      DVM_CUDA(cudaStreamCreateWithFlags(&p.s[i], cudaStreamNonBlocking));
+      DVM_CUDA(cudaEventCreateWithFlags(&p.done[i], cudaEventDisableTiming));
+    }
+    DVM_CUDA(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+    p.ready = true;
+  }
+  *out = &p;
+  return DVM_OK;
+}
+
+// 0: the tensor follows the tiles (rows of `row_bytes` bytes), 1: a row vector copied whole, -1: neither
+int pipe_class(const uint32_t* w, const uint32_t* od, bool is_input, uint64_t* row_bytes) {
+  const uint32_t info = od[DVM_OPD_INFO];
+  const uint32_t es = 1u << DVM_DT_LG_ES((info >> 8) & 0xff);
+  if (((info >> 16) & 0xff) != 1 || od[DVM_OPD_COLSTRIDE] != 1 || ((info >> 26) & 3u)) return -1;
+  if ((info >> 25) & 1u) {  // dense: row r starts at element r * C
+    *row_bytes = (uint64_t)w[DVM_H_COLS] * es;
+    return 0;
+  }
+  if (is_input && od[DVM_OPD_STRIDE0] == 0 && od[DVM_OPD_STRIDE1] == 0 && od[DVM_OPD_STRIDE2] == 0) return 1;
+  return -1;
+}
+}  // namespace
+
 extern "C" int dvm_run_host(const void* code, size_t code_size, void* const* host_tensors,
                             const size_t* tensor_bytes, int n_tensors, void* staging, size_t staging_bytes,
                             void* cuda_stream) {
@@ -613,6 +669,78 @@ extern "C" int dvm_run_host(const void* code, size_t code_size, void* const* hos
     off += (tensor_bytes[i] + 255) & ~(size_t)255;
   }
   if (off > staging_bytes) return DVM_ERR_BUFFER_TOO_SMALL;
+
+  // ---- can the program be pipelined? ----
+  bool pipe = w[DVM_H_KERNEL_TYPE] == DVM_KERNEL_VEC && w[DVM_H_COL_BLOCKS] == 1 && w[DVM_H_N_TILES] >= 8;
+  int cls[DVM_MAX_TENSORS];
+  uint64_t row_bytes[DVM_MAX_TENSORS];
+  if (pipe) {
+    const uint32_t n_opd = (counts >> 16) & 0xff;
+    const uint32_t* ot = w + DVM_HDR_WORDS + 2 * nt;
+    for (int i = 0; i < nt; ++i) cls[i] = -2;  // (a tensor no operand names is not touched)
+    for (uint32_t o = 0; o < n_opd && pipe; ++o) {
+      const uint32_t* od = ot + o * DVM_OPD_WORDS;
+      const int slot = od[DVM_OPD_INFO] & 0xff;
+      uint64_t rb = 0;
+      const int c = pipe_class(w, od, slot < n_in, &rb);
+      if (c < 0 || (cls[slot] != -2 && cls[slot] != c)) pipe = false;
+      cls[slot] = c;
+      row_bytes[slot] = rb;
+    }
+    for (int i = 0; i < nt && pipe; ++i) if (cls[i] == -2) pipe = false;
+  }
+  const uint64_t total_bytes = off;
+  if (pipe && total_bytes >= (64u << 20)) {
+    PipeStreams* ps = nullptr;
+    st = pipe_streams(&ps);
+    if (st != DVM_OK) return st;
+    const uint32_t n_tiles = w[DVM_H_N_TILES];
+    const uint32_t R = (uint32_t)DVM_VM_THREADS >> (w[DVM_H_GEOM] & 0xff);   // rows per tile
+    // chunks of about 48 MB over all tensors, at least one tile, at most 256 chunks
+    uint64_t per_tile = 0;
+    for (int i = 0; i < nt; ++i) if (cls[i] == 0) per_tile += row_bytes[i] * R;
+    uint32_t chunk_tiles = per_tile ? (uint32_t)((48ull << 20) / per_tile) : n_tiles;
+    if (chunk_tiles < 1) chunk_tiles = 1;
+    if ((n_tiles + chunk_tiles - 1) / chunk_tiles > 256) chunk_tiles = (n_tiles + 255) / 256;
+    // row vectors first, on the caller's stream; the chunk streams start behind them
+    for (int i = 0; i < n_in; ++i)
+      if (cls[i] == 1 && tensor_bytes[i]) DVM_CUDA(cudaMemcpyAsync(dev[i], host_tensors[i], tensor_bytes[i], cudaMemcpyHostToDevice, stream));
+    DVM_CUDA(cudaEventRecord(ps->start, stream));
+    for (int k = 0; k < kPipeStreams; ++k) DVM_CUDA(cudaStreamWaitEvent(ps->s[k], ps->start, 0));
+    const void* codes[1] = {code};
+    void* const* tl[1] = {dev};
+    int launched = DVM_OK;
+    uint32_t k = 0;
+    for (uint32_t t0 = 0; t0 < n_tiles; t0 += chunk_tiles, ++k) {
+      const uint32_t t1 = t0 + chunk_tiles < n_tiles ? t0 + chunk_tiles : n_tiles;
+      cudaStream_t cs = ps->s[k % kPipeStreams];
+      for (int i = 0; i < nt; ++i) {
+        if (cls[i] != 0 || i >= n_in) continue;
+        const uint64_t b0 = (uint64_t)t0 * R * row_bytes[i];
+        uint64_t b1 = (uint64_t)t1 * R * row_bytes[i];
+        if (b1 > tensor_bytes[i]) b1 = tensor_bytes[i];
+        if (b1 > b0) DVM_CUDA(cudaMemcpyAsync((char*)dev[i] + b0, (const char*)host_tensors[i] + b0, b1 - b0, cudaMemcpyHostToDevice, cs));
+      }
+      launched = launch_vec(1, codes, tl, &n_tensors, false, nullptr, cs, t0, t1);
+      if (launched != DVM_OK) break;
+      for (int i = n_in; i < nt; ++i) {
+        if (cls[i] != 0) continue;
+        const uint64_t b0 = (uint64_t)t0 * R * row_bytes[i];
+        uint64_t b1 = (uint64_t)t1 * R * row_bytes[i];
+        if (b1 > tensor_bytes[i]) b1 = tensor_bytes[i];
+        if (b1 > b0) DVM_CUDA(cudaMemcpyAsync((char*)host_tensors[i] + b0, (const char*)dev[i] + b0, b1 - b0, cudaMemcpyDeviceToHost, cs));
+      }
+    }
+    for (int q = 0; q < kPipeStreams; ++q) {
+      DVM_CUDA(cudaEventRecord(ps->done[q], ps->s[q]));
+      DVM_CUDA(cudaStreamWaitEvent(stream, ps->done[q], 0));
+    }
+    DVM_CUDA(cudaStreamSynchronize(stream));
+    if (launched == DVM_OK) return DVM_OK;
+    if (launched != DVM_ERR_UNSUPPORTED || k != 0) return launched;
+    // (the first chunk could not be launched as a range of tiles: nothing ran yet, take the plain way)
+  }
+
   for (int i = 0; i < n_in; ++i)
     if (tensor_bytes[i]) DVM_CUDA(cudaMemcpyAsync(dev[i], host_tensors[i], tensor_bytes[i], cudaMemcpyHostToDevice, stream));
   st = dvm_launch(code, code_size, dev, nt, cuda_stream);
@@ -775,6 +903,8 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.n_words = pos;
   P.use_queue = 1u;
   P.levels = 0u;
+  P.tile_begin = 0u;
+  P.reserved = 0u;
   P.status = dev.scratch;
   P.queue = dev.scratch + 2;
   const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;

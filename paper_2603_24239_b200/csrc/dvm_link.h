@@ -35,6 +35,7 @@ enum {
   DVM_LK_EXPS,                                           // ACC = exp(ACC - S[a])      sub = 1: one-piece exponential
   DVM_LK_RED,                                            // S[a] = reduce(ACC); b = 1: S[a] = unary(S[a] * w2 + w3), w1 = unary or 0xff
   DVM_LK_STG,                                            // store ACC: a = log2(element size), w1 | w2 << 32 = tensor address
+  DVM_LK_STGI,                                           // store ACC converted to i32 (sub 1) or u8 (sub 2): the same fields
   DVM_LK_STA,                                            // L[tmp] = ACC               w1 = byte offset of the temporary in a tile slot
   DVM_LK_LSS,                                            // S[a] = loaded row scalar   w1 = byte offset of its word in a tile slot (thread 0's)
   DVM_LK_STS,                                            // store S[a] per row         w1 = operand descriptor (word offset from the program)

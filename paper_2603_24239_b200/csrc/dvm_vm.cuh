@@ -62,6 +62,9 @@ struct VMParams {
   uint32_t slot_bytes;   // bytes of one tile slot in local memory (the largest program's)
   uint32_t levels;       // 1: the directory has a third table, and tiles wait for the tiles of earlier levels;
                          // 2: one tile slot per CTA (slot_bytes = 0): no tile is loaded ahead, nothing is waited for
+  uint32_t tile_begin;   // one-program launches: the first tile of the launch (tiles [tile_begin, total_tiles) run; a
+                         // caller that pipelines host copies with execution launches a program in ranges of tiles)
+  uint32_t reserved;     // (keeps `words` on a 16-byte boundary of the parameter space: linked records are loaded as vectors)
   unsigned int* status;  // device status word
   unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished, [2] tiles completed (all zero between launches)
   uint32_t words[PW];    // [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, if levels)][programs ...]
@@ -587,7 +590,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   };
 
   uint32_t prog_idx = 0;
-  uint32_t tile = blockIdx.x;
+  uint32_t tile = blockIdx.x + (SINGLE ? prm.tile_begin : 0u);
   uint32_t iter = 0;
   int red_par = 0;
   int buf = 0;

@@ -29,6 +29,16 @@ __device__ __forceinline__ uint4 lean_lds128(uint32_t addr) {
   return v;
 }
 
+// A value the compiler must take as it is at this point of this handler.  Several handlers start with the same
+// computation on a record's fields (the address of the operand a word names, the load of a per-row scalar); left
+// alone, the compiler hoists such common code in front of the dispatch, where EVERY record pays for it (measured:
+// a fifth more instructions per tile).  ID makes each use distinct, so nothing can be merged across handlers.
+template <int ID>
+__device__ __forceinline__ uint32_t lean_opaque(uint32_t v) {
+  asm volatile("// handler %1" : "+r"(v) : "n"(ID));
+  return v;
+}
+
 // bf16 pair in a word -> two floats
 __device__ __forceinline__ float2 lean_widen(uint32_t w) {
   return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
@@ -322,7 +332,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
   }
 
   uint32_t prog_idx = 0;
-  uint32_t tile = blockIdx.x;
+  uint32_t tile = blockIdx.x + (SINGLE ? prm.tile_begin : 0u);
   uint32_t iter = 0;
   int red_par = 0;
   int buf = 0;
@@ -475,14 +485,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
       switch (h) {
         case DVM_LK_LDA_BF16: {
           uint32_t R[V / 2];
-          lean_raw_bf16<V>(R, opw_addr(rec.y), (uint32_t)(G << 4));
+          lean_raw_bf16<V>(R, opw_addr(lean_opaque<1>(rec.y)), (uint32_t)(G << 4));
           DVM_EACH_PAIR A[i] = lean_widen(R[i]);
         } break;
         case DVM_LK_LD2_BF16: {  // ACC = L[x] op L[y] (* imm): add / sub / rsub / mul
           uint32_t R[V / 2];
-          lean_raw_bf16<V>(R, opw_addr(rec.y), (uint32_t)(G << 4));
+          lean_raw_bf16<V>(R, opw_addr(lean_opaque<2>(rec.y)), (uint32_t)(G << 4));
           DVM_EACH_PAIR A[i] = lean_widen(R[i]);
-          lean_raw_bf16<V>(R, opw_addr(rec.z), (uint32_t)(G << 4));
+          lean_raw_bf16<V>(R, opw_addr(lean_opaque<42>(rec.z)), (uint32_t)(G << 4));
           if (sub == DVM_A_ADD) { DVM_EACH_PAIR A[i] = __fadd2_rn(A[i], lean_widen(R[i])); }
           else if (sub == DVM_A_MUL) { DVM_EACH_PAIR A[i] = __fmul2_rn(A[i], lean_widen(R[i])); }
           else if (sub == DVM_A_SUB) { DVM_EACH_PAIR A[i] = __ffma2_rn(lean_widen(R[i]), make_float2(-1.f, -1.f), A[i]); }
@@ -494,7 +504,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
         } break;
         case DVM_LK_BIN_BF16: {
           uint32_t R[V / 2];
-          lean_raw_bf16<V>(R, opw_addr(rec.y), (uint32_t)(G << 4));
+          lean_raw_bf16<V>(R, opw_addr(lean_opaque<3>(rec.y)), (uint32_t)(G << 4));
           if (rec.x >> 24) {  // ACC = ACC * S[.] * L[y]
             const float m = s_S[(rec.x >> 24) - 1][tid];
             DVM_EACH_PAIR A[i] = __fmul2_rn(__fmul2_rn(A[i], make_float2(m, m)), lean_widen(R[i]));
@@ -503,7 +513,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           }
         } break;
         case DVM_LK_LDA_F32: {  // (in two halves: the raw words of a whole fp32 tile register would crowd the registers)
-          const uint32_t a = opw_addr(rec.y);
+          const uint32_t a = opw_addr(lean_opaque<4>(rec.y));
 #define DVM_LDA_F32_HALF(H)                                                                               \
           {                                                                                               \
             uint32_t R[V / 2];                                                                            \
@@ -517,7 +527,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
 #undef DVM_LDA_F32_HALF
         } break;
         case DVM_LK_BIN_F32: {
-          const uint32_t a = opw_addr(rec.y);
+          const uint32_t a = opw_addr(lean_opaque<5>(rec.y));
           const bool pre = (rec.x >> 24) != 0;  // ACC = ACC * S[.] * L[y]
           const float m = pre ? s_S[(rec.x >> 24) - 1][tid] : 1.0f;
 #define DVM_BIN_F32_HALF(H)                                                                               \
@@ -550,7 +560,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
 #undef DVM_BIN_F32_HALF
         } break;
         case DVM_LK_LDA_PRIV: {
-          const uint32_t a = sb + (rec.y & 0x3ffffu) + (uint32_t)tid * 16;
+          const uint32_t a = sb + (lean_opaque<6>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
 #pragma unroll
           for (int q = 0; q < V / 4; ++q) {
             const uint4 v = lean_lds128(a + q * PSTRIDE);
@@ -559,7 +569,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           }
         } break;
         case DVM_LK_BIN_PRIV: {
-          const uint32_t a = sb + (rec.y & 0x3ffffu) + (uint32_t)tid * 16;
+          const uint32_t a = sb + (lean_opaque<7>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
           uint32_t R[V];
 #pragma unroll
           for (int q = 0; q < V / 4; ++q) {
@@ -574,7 +584,8 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           DVM_ARITH(sub, Y[i].x, Y[i].y)
         } break;
         case DVM_LK_FMA: {  // ACC = ACC * m + c, m and c immediates or per-row scalars: add / sub / rsub / mul / div by a scalar
-          float m = (sub & 1u) ? s_S[ra][tid] : __uint_as_float(rec.y);
+          const uint32_t ra_ = lean_opaque<9>(ra);
+          float m = (sub & 1u) ? s_S[ra_][tid] : __uint_as_float(rec.y);
           float c = (sub & 2u) ? s_S[rec.x >> 24][tid] : __uint_as_float(rec.z);
           if (sub & 4u) m = fast_rcp(m);
           if (sub & 8u) c = -c;
@@ -582,13 +593,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
         } break;
         case DVM_LK_BINI:
         case DVM_LK_BINS: {  // (what the multiply-add form does not cover: rdiv, min, max)
-          const float y = h == DVM_LK_BINS ? s_S[ra][tid] : __uint_as_float(rec.y);
+          const uint32_t ra_ = lean_opaque<10>(ra);
+          const float y = h == DVM_LK_BINS ? s_S[ra_][tid] : __uint_as_float(rec.y);
           if (sub == DVM_A_RDIV) { DVM_EACH_PAIR A[i] = make_float2(fast_div(y, A[i].x), fast_div(y, A[i].y)); }
           else if (sub == DVM_A_MIN) { DVM_EACH_PAIR A[i] = make_float2(A[i].x < y ? A[i].x : y, A[i].y < y ? A[i].y : y); }
           else { DVM_EACH_PAIR A[i] = make_float2(A[i].x > y ? A[i].x : y, A[i].y > y ? A[i].y : y); }
         } break;
         case DVM_LK_EXPS: {
-          const float m = -s_S[ra][tid];
+          const float m = -s_S[lean_opaque<11>(ra)][tid];
           if (sub) {  // every output of the program is bf16: the one-piece exponential
             const float nc = m * 1.44269502162933349609375f;
             DVM_EACH_PAIR A[i] = lean_exp2_fast(A[i], nc);
@@ -625,11 +637,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             DVM_UN_CASE(DVM_U_NEG, -x)
             DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
             DVM_UN_CASE(DVM_U_RND_BF16, round_bf16(x))
-            DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
-            DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
             default:
               if constexpr (HEAVY) {
                 switch (sub) {
+                  DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
+                  DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
                   DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
                   DVM_UN_CASE(DVM_U_LOG, logf(x))
                   case DVM_U_ERF: DVM_EACH_PAIR A[i] = packed_erf(A[i]); break;
@@ -701,47 +713,19 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             v = __fadd_rn(__fmul_rn(v, __uint_as_float(rec.z)), __uint_as_float(rec.w));
             if (rec.y != 0xffu) v = scalar_unary((int)rec.y, v);
           }
-          s_S[ra][tid] = v;
+          s_S[lean_opaque<13>(ra)][tid] = v;
         } break;
         case DVM_LK_STG: {
-          const int lg_es = (int)ra;
-          const unsigned long long base = (unsigned long long)rec.y | ((unsigned long long)rec.z << 32);
+          const int lg_es = (int)lean_opaque<54>(ra);
+          const unsigned long long base = (unsigned long long)lean_opaque<14>(rec.y) | ((unsigned long long)rec.z << 32);
           const unsigned long long el0 = (unsigned long long)r.row * C + r.col0;
           char* p = reinterpret_cast<char*>(base + (el0 << lg_es));
           char* q0 = p + ((long long)cbase << lg_es);
           const long long qstep = (long long)((G << lgW) << lg_es);
-          // (a chunk of u8 is W bytes: its vector store wants that alignment; everything else goes in 16-byte vectors)
-          const bool al = (reinterpret_cast<uintptr_t>(q0) & (lg_es == 0 ? (uintptr_t)((1 << lgW) - 1) : (uintptr_t)15)) == 0;
+          const bool al = (reinterpret_cast<uintptr_t>(q0) & 15) == 0;
           const uint32_t fast = al ? fullmask : 0u;
           const uint32_t slow = partmask | (fullmask & ~fast);
-          if (sub == 2) {  // Table 1, Cast: stored as u8, a chunk is W bytes
-            if (lgW == 3) {
-#pragma unroll
-              for (int j = 0; j < V / 8; ++j)
-                if ((fast >> j) & 1)
-                  *reinterpret_cast<uint2*>(q0 + j * qstep) = make_uint2(pack_u8x4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y),
-                                                                         pack_u8x4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y));
-            } else {
-#pragma unroll
-              for (int j = 0; j < V / 4; ++j)
-                if ((fast >> j) & 1)
-                  *reinterpret_cast<uint32_t*>(q0 + j * qstep) = pack_u8x4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
-            }
-          } else if (sub == 1) {  // stored as i32
-            if (lgW == 3) {
-#pragma unroll
-              for (int j = 0; j < V / 8; ++j)
-                if ((fast >> j) & 1) {
-                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[4 * j].x), store_i32(A[4 * j].y), store_i32(A[4 * j + 1].x), store_i32(A[4 * j + 1].y));
-                  *reinterpret_cast<uint4*>(q0 + j * qstep + 16) = make_uint4(store_i32(A[4 * j + 2].x), store_i32(A[4 * j + 2].y), store_i32(A[4 * j + 3].x), store_i32(A[4 * j + 3].y));
-                }
-            } else {
-#pragma unroll
-              for (int j = 0; j < V / 4; ++j)
-                if ((fast >> j) & 1)
-                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[2 * j].x), store_i32(A[2 * j].y), store_i32(A[2 * j + 1].x), store_i32(A[2 * j + 1].y));
-            }
-          } else if (lg_es == 1) {  // bf16: chunks of 8, chunk j = group j
+          if (lg_es == 1) {  // bf16: chunks of 8, chunk j = group j
 #pragma unroll
             for (int j = 0; j < V / 8; ++j)
               if ((fast >> j) & 1) {
@@ -768,21 +752,24 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           }
           if (slow) {
             // chunks cut by the row's head or tail (or stored at another alignment than the tile's chunks):
-            // element stores, one 8-slot group at a time
+            // element stores, one 8-slot group at a time.  (The column arithmetic hangs on an opaque copy of the
+            // chunk base: it is the same for every record of a tile, and the compiler would otherwise compute all
+            // of it at the top of every tile, for a path few threads take.)
+            const int cb = (int)lean_opaque<90>((uint32_t)cbase);
 #pragma unroll
             for (int g = 0; g < NG; ++g) {
               const uint32_t gm = lgW == 3 ? ((slow >> g) & 1u) : ((slow >> (2 * g)) & 3u);
               if (gm) {
+                // first column of the group's first (and, with chunks of 4, second) chunk
+                const int c0 = cb + ((lgW == 3 ? g : 2 * g) << (lgG + lgW));
+                const int c1 = lgW == 3 ? c0 + 4 : c0 + (1 << (lgG + 2));
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                  const int s = 8 * g + e;
-                  const int col = cbase + ((s >> lgW) << (lgG + lgW)) + (s & ((1 << lgW) - 1));
+                  const int col = e < 4 ? c0 + e : c1 + (e - 4);
                   const bool in_slow = lgW == 3 ? true : ((gm >> (e >> 2)) & 1u) != 0;
                   const float val = (e & 1) ? A[4 * g + (e >> 1)].y : A[4 * g + (e >> 1)].x;
                   if (in_slow && col >= 0 && col < r.ncols) {
-                    if (sub == 2) *reinterpret_cast<unsigned char*>(p + (long long)col) = (unsigned char)store_u8(val);
-                    else if (sub == 1) *reinterpret_cast<uint32_t*>(p + (long long)col * 4) = store_i32(val);
-                    else if (lg_es == 1) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
+                    if (lg_es == 1) *reinterpret_cast<__nv_bfloat16*>(p + (long long)col * 2) = __float2bfloat16_rn(val);
                     else *reinterpret_cast<float*>(p + (long long)col * 4) = val;
                   }
                 }
@@ -790,8 +777,69 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             }
           }
         } break;
+        case DVM_LK_STGI: {  // Table 1, Cast: ACC stored as i32 (sub 1) or u8 (sub 2), converted toward zero
+          const int lg_es = (int)lean_opaque<55>(ra);
+          const unsigned long long base = (unsigned long long)lean_opaque<15>(rec.y) | ((unsigned long long)rec.z << 32);
+          const unsigned long long el0 = (unsigned long long)r.row * C + r.col0;
+          char* p = reinterpret_cast<char*>(base + (el0 << lg_es));
+          char* q0 = p + ((long long)cbase << lg_es);
+          const long long qstep = (long long)((G << lgW) << lg_es);
+          // (a chunk of u8 is W bytes: its vector store wants that alignment; i32 goes in 16-byte vectors)
+          const bool al = (reinterpret_cast<uintptr_t>(q0) & (lg_es == 0 ? (uintptr_t)((1 << lgW) - 1) : (uintptr_t)15)) == 0;
+          const uint32_t fast = al ? fullmask : 0u;
+          const uint32_t slow = partmask | (fullmask & ~fast);
+          if (sub == 2) {  // Table 1, Cast: stored as u8, a chunk is W bytes
+            if (lgW == 3) {
+#pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint2*>(q0 + j * qstep) = make_uint2(pack_u8x4(A[4 * j].x, A[4 * j].y, A[4 * j + 1].x, A[4 * j + 1].y),
+                                                                         pack_u8x4(A[4 * j + 2].x, A[4 * j + 2].y, A[4 * j + 3].x, A[4 * j + 3].y));
+            } else {
+#pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint32_t*>(q0 + j * qstep) = pack_u8x4(A[2 * j].x, A[2 * j].y, A[2 * j + 1].x, A[2 * j + 1].y);
+            }
+          } else {  // stored as i32
+            if (lgW == 3) {
+#pragma unroll
+              for (int j = 0; j < V / 8; ++j)
+                if ((fast >> j) & 1) {
+                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[4 * j].x), store_i32(A[4 * j].y), store_i32(A[4 * j + 1].x), store_i32(A[4 * j + 1].y));
+                  *reinterpret_cast<uint4*>(q0 + j * qstep + 16) = make_uint4(store_i32(A[4 * j + 2].x), store_i32(A[4 * j + 2].y), store_i32(A[4 * j + 3].x), store_i32(A[4 * j + 3].y));
+                }
+            } else {
+#pragma unroll
+              for (int j = 0; j < V / 4; ++j)
+                if ((fast >> j) & 1)
+                  *reinterpret_cast<uint4*>(q0 + j * qstep) = make_uint4(store_i32(A[2 * j].x), store_i32(A[2 * j].y), store_i32(A[2 * j + 1].x), store_i32(A[2 * j + 1].y));
+            }
+          }
+          if (slow) {
+            const int cb = (int)lean_opaque<91>((uint32_t)cbase);
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+              const uint32_t gm = lgW == 3 ? ((slow >> g) & 1u) : ((slow >> (2 * g)) & 3u);
+              if (gm) {
+                const int c0 = cb + ((lgW == 3 ? g : 2 * g) << (lgG + lgW));
+                const int c1 = lgW == 3 ? c0 + 4 : c0 + (1 << (lgG + 2));
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const int col = e < 4 ? c0 + e : c1 + (e - 4);
+                  const bool in_slow = lgW == 3 ? true : ((gm >> (e >> 2)) & 1u) != 0;
+                  const float val = (e & 1) ? A[4 * g + (e >> 1)].y : A[4 * g + (e >> 1)].x;
+                  if (in_slow && col >= 0 && col < r.ncols) {
+                    if (sub == 2) *reinterpret_cast<unsigned char*>(p + (long long)col) = (unsigned char)store_u8(val);
+                    else *reinterpret_cast<uint32_t*>(p + (long long)col * 4) = store_i32(val);
+                  }
+                }
+              }
+            }
+          }
+        } break;
         case DVM_LK_STA: {
-          const uint32_t a0 = sb + rec.y + (uint32_t)tid * 16;
+          const uint32_t a0 = sb + lean_opaque<16>(rec.y) + (uint32_t)tid * 16;
 #pragma unroll
           for (int q = 0; q < V / 4; ++q)
             asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a0 + q * PSTRIDE), "f"(A[2 * q].x), "f"(A[2 * q].y),
@@ -800,14 +848,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
         } break;
         case DVM_LK_LSS: {
           float v;
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(sb + rec.y + (uint32_t)tid * 16));
-          s_S[ra][tid] = r.ncols > 0 ? v : 0.f;
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(sb + lean_opaque<17>(rec.y) + (uint32_t)tid * 16));
+          s_S[lean_opaque<57>(ra)][tid] = r.ncols > 0 ? v : 0.f;
         } break;
         case DVM_LK_STS: {
-          const uint32_t d = prog + rec.y;
+          const uint32_t d = prog + lean_opaque<18>(rec.y);
           const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
           char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(prog, d, r) << DVM_DT_LG_ES(dt)));
-          const float v = s_S[ra][tid];
+          const float v = s_S[lean_opaque<58>(ra)][tid];
           if (r.ncols > 0 && t == 0 && r.col0 == 0) {
             if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
             else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p) = v;
@@ -816,11 +864,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
           }
         } break;
         case DVM_LK_BCS: {
-          const float v = s_S[ra][tid];
+          const float v = s_S[lean_opaque<19>(ra)][tid];
           DVM_EACH_PAIR A[i] = make_float2(v, v);
         } break;
         case DVM_LK_SOP: {
-          const int s1 = (rec.y >> 8) & 0xff, s2 = (rec.y >> 16) & 0xff, sop = rec.y & 0xff;
+          const uint32_t ry = lean_opaque<20>(rec.y);
+          const int s1 = (ry >> 8) & 0xff, s2 = (ry >> 16) & 0xff, sop = ry & 0xff;
           const float x = s_S[s1][tid];
           float rv;
           if (sub == DVM_SK_FMAU) {
@@ -828,7 +877,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             if (sop != 0xff) rv = scalar_unary(sop, rv);
           } else if (sub == DVM_SK_UN) rv = scalar_unary(sop, x);
           else rv = scalar_arith(sop, x, sub == DVM_SK_BIN ? s_S[s2][tid] : __uint_as_float(rec.z));
-          s_S[ra][tid] = rv;
+          s_S[lean_opaque<60>(ra)][tid] = rv;
         } break;
         default:
           err = ST_BAD_CODE;
