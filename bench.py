@@ -1127,6 +1127,8 @@ def main():
     ap.add_argument("--encode-reps", type=int, default=1000, help="repeats per instance of the host-encode latency measurement")
     ap.add_argument("--general-interpreter", action="store_true",
                     help="run every launch on the general interpreter instead of the lean one (for comparisons)")
+    ap.add_argument("--lean-stacked", action="store_true",
+                    help="run stacked launches on the lean interpreter too (default: the general one; for comparisons)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
@@ -1157,6 +1159,8 @@ def main():
         dvm.set_elems_per_thread(args.elems_per_thread)
     if args.general_interpreter:
         dvm.set_lean_kernel(False)
+    if args.lean_stacked:
+        dvm.set_lean_kernel(2)
     if args.instances:
         kw = {"n_launches": args.instances} if args.workload == "c4" else {"n_instances": args.instances}
     if args.max_rows and args.workload in ("c2", "c5", "addmm"):

@@ -138,6 +138,7 @@ enum {
   DVM_U_TRUNC_U8 = 15,  // ... to u8
   DVM_U_NUN = 16
 };
+enum { DVM_ACT_GELU = 0, DVM_ACT_SILU = 1, DVM_ACT_N = 2 };
 // the two-tile-operand class of the extended variant: the comparisons (Table 1, Cmp) and Pow (Table 1)
 enum { DVM_C_GT = 0, DVM_C_GE = 1, DVM_C_LT = 2, DVM_C_LE = 3, DVM_C_EQ = 4, DVM_C_NE = 5,
        DVM_C_POW = 6,   // ACC = ACC ^ L[a]
@@ -172,6 +173,9 @@ enum {
   DVM_OP_RED = 0x38,   // 0x38 + reduce (4); a = dst scalar register   : S[a] = reduce(ACC) over the row
   DVM_OP_LD2 = 0x40,   // 0x40 + arith; a = local register x, b = local register y | dtype(x) << 6 | dtype(y) << 7
                        //                                             : ACC = L[x] op L[y]   (fused copy + arithmetic)
+  DVM_OP_ACT = 0x48,   // 0x48 + activation: ACC = act(ACC), a self-gating chain of Table 1 operations fused by the encoder
+                       //   (pattern-based fusion, Sec. 5.1): 0 GELU  0.5 t (1 + erf(t / sqrt 2)),  1 SiLU  t sigmoid(t);
+                       //   fused, the chain needs no temporary for t
   DVM_OP_CMP = 0x50,   // 0x50 + comparison; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC cmp L[a] ? 1 : 0
                        //   (0x56 / 0x57: Pow, ACC = ACC ^ L[a] / L[a] ^ ACC)
   DVM_OP_SEL = 0x58,   // Table 1, Select; a = local register p, b = local register q | dtype(p) << 6 | dtype(q) << 7

@@ -303,6 +303,9 @@ struct Enc {
   int n_in_regs, n_tmp_regs, n_sslots;
   bool fused_sq[DVM_MAX_NODES];   // x*x whose only consumer is a row sum: folded into that reduction
   bool fused_sc[DVM_MAX_NODES];   // per-row scalar muls/adds folded into a later multiply-add(-unary) instruction
+  int8_t act_of[DVM_MAX_NODES];   // -1, or the fused activation (DVM_ACT_*) this node is the result of
+  int16_t act_src[DVM_MAX_NODES]; // ... applied to this value
+  bool act_part[DVM_MAX_NODES];   // an inner node of a fused activation chain: never materialises
   int16_t n_cons[DVM_MAX_NODES];  // number of consuming nodes / outputs of a value
   int16_t one_cons[DVM_MAX_NODES];// the consuming node when there is exactly one (and it is a node)
   int lda_pos;                    // body position of the LDA just emitted by ensure_acc, or -1
@@ -461,12 +464,57 @@ static bool gen_body(Enc& e) {
     }
   }
 
+  // Self-gating activations (pattern-based fusion, Sec. 5.1): the chains  0.5 * (t * (1 + erf(t / sqrt 2)))  and
+  // t * sigmoid(t)  of single-consumer tile values become ONE instruction on t: no temporary has to keep t alive.
+  for (int i = 0; i < p->n_nodes; ++i) { e.act_of[i] = -1; e.act_src[i] = -1; e.act_part[i] = false; }
+  {
+    auto is_imm = [&](const Node& n, int op, float v) {
+      return n.kind == NK_SCALAR && n.op == op && n.param < 0 && fabsf(n.imm - v) <= 1e-6f * fabsf(v);
+    };
+    auto inner_ok = [&](int v) { return e.uses[v] == 1 && e.cls[v] == CLS_TILE && e.alias[v] < 0; };
+    for (int i = 0; i < p->n_nodes; ++i) {
+      const Node& n = p->nodes[i];
+      if (e.alias[i] >= 0 || e.cls[i] != CLS_TILE) continue;
+      if (is_imm(n, DVM_MULS, 0.5f)) {                          // 0.5 * m
+        const int m = root(e, n.x);
+        const Node& mn = p->nodes[m];
+        if (mn.kind != NK_BINARY || mn.op != DVM_MUL || !inner_ok(m)) continue;
+        for (int side = 0; side < 2; ++side) {                    // m = t * u3 or u3 * t
+          const int t = root(e, side ? mn.y : mn.x), u3 = root(e, side ? mn.x : mn.y);
+          if (t == u3 || e.cls[t] != CLS_TILE || !inner_ok(u3) || !is_imm(p->nodes[u3], DVM_ADDS, 1.0f)) continue;
+          const int u2 = root(e, p->nodes[u3].x);
+          if (!inner_ok(u2) || p->nodes[u2].kind != NK_UNARY || p->nodes[u2].op != DVM_ERF) continue;
+          const int u1 = root(e, p->nodes[u2].x);
+          if (!inner_ok(u1) || !is_imm(p->nodes[u1], DVM_MULS, 0.70710678f) || root(e, p->nodes[u1].x) != t) continue;
+          e.act_of[i] = DVM_ACT_GELU; e.act_src[i] = (int16_t)t;
+          e.act_part[m] = e.act_part[u3] = e.act_part[u2] = e.act_part[u1] = true;
+          e.uses[m] = e.uses[u3] = e.uses[u2] = e.uses[u1] = 0;
+          e.uses[t] -= 1;                                         // t fed u1 and m: the fused instruction reads it once
+          break;
+        }
+      } else if (n.kind == NK_BINARY && n.op == DVM_MUL) {        // t * sigmoid(t)
+        for (int side = 0; side < 2; ++side) {
+          const int t = root(e, side ? n.y : n.x), s = root(e, side ? n.x : n.y);
+          if (t == s || e.cls[t] != CLS_TILE || !inner_ok(s) || e.act_part[s] || p->nodes[s].kind != NK_UNARY ||
+              p->nodes[s].op != DVM_SIGMOID || root(e, p->nodes[s].x) != t)
+            continue;
+          e.act_of[i] = DVM_ACT_SILU; e.act_src[i] = (int16_t)t;
+          e.act_part[s] = true;
+          e.uses[s] = 0;
+          e.uses[t] -= 1;
+          break;
+        }
+      }
+    }
+  }
+
   // consumers of every value (for the scalar multiply-add fusion below)
   for (int i = 0; i < p->n_nodes; ++i) { e.n_cons[i] = 0; e.one_cons[i] = -1; e.fused_sc[i] = false; }
   for (int i = 0; i < p->n_nodes; ++i) {
     const Node& n = p->nodes[i];
-    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i]) continue;
+    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i] || e.act_part[i]) continue;
     int x = root(e, n.x);
+    if (e.act_of[i] >= 0) { e.n_cons[e.act_src[i]]++; e.one_cons[e.act_src[i]] = (int16_t)i; continue; }
     if (n.kind == NK_REDUCE && e.fused_sq[x]) x = root(e, p->nodes[x].x);
     e.n_cons[x]++; e.one_cons[x] = (int16_t)i;
     if (n.kind == NK_BINARY || n.kind == NK_COMPARE || n.kind == NK_SELECT) { int y = root(e, n.y); e.n_cons[y]++; e.one_cons[y] = (int16_t)i; }
@@ -496,8 +544,22 @@ static bool gen_body(Enc& e) {
   // ---- compute section ----
   for (int i = 0; i < p->n_nodes && !e.fail; ++i) {
     const Node& n = p->nodes[i];
-    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i]) continue;
+    if (n.kind == NK_INPUT || e.alias[i] >= 0 || e.fused_sq[i] || e.act_part[i]) continue;
     int x = root(e, n.x);
+    if (e.act_of[i] >= 0) {  // a fused activation of the value act_src: one instruction on the accumulator
+      const int t = e.act_src[i];
+      ensure_acc(e, t);
+      if (e.fail) break;
+      e.uses[t]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      emit(e, DVM_INSN(DVM_OP_ACT + e.act_of[i], 1, 0, 0));
+      e.acc = (int16_t)i;
+      release(e, t);
+      store_outputs_of(e, i);
+      if (e.acc == i && e.uses[i] == 0) e.acc = -1;
+      continue;
+    }
     if (e.cls[i] == CLS_SCAL && (n.kind == NK_COMPARE || n.kind == NK_SELECT)) { e.fail = true; break; }
     if (e.cls[i] == CLS_SCAL && n.kind != NK_REDUCE) {
       // ---- per-row scalar arithmetic ----
@@ -1428,6 +1490,7 @@ static int insn_expected_len(uint32_t op, uint32_t w0) {
   if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) return 1;
+  if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) return 1;
   if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) return 1;
   if (op == DVM_OP_SOP) return DVM_INSN_B(w0) == DVM_SK_BINI ? 3 : 2;
   return -1;
@@ -1684,6 +1747,7 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
       else outf(o, "select    acc, l%u%s ? acc : l%u%s\n", a, s1, bb & 0x3f, s2);
     }
     else if (op >= DVM_OP_UN && op < DVM_OP_UN + DVM_U_NUN) outf(o, "%-9s acc, acc\n", kUn[op - DVM_OP_UN]);
+    else if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) outf(o, "%-9s acc, acc\n", op == DVM_OP_ACT + DVM_ACT_GELU ? "gelu" : "silu");
     else if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) outf(o, "row%-6s s%u, acc\n", kRed[op - DVM_OP_RED], a);
     else if (op == DVM_OP_SOP) {
       uint32_t w1 = b[pc + 1], sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;

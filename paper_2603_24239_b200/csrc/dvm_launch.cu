@@ -254,6 +254,8 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       const uint32_t u = op - DVM_OP_UN;
       if (u == DVM_U_ISFINITE) return 0;
       push(DVM_LK_W0(DVM_LK_UN, u | ((fast && (u == DVM_U_EXP || u == DVM_U_SIGMOID)) ? 0x80u : 0u), 0, 0), 0, 0, 0);
+    } else if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) {
+      push(DVM_LK_W0(DVM_LK_ACT, op - DVM_OP_ACT, 0, 0), 0, 0, 0);
     } else if (cls == (DVM_OP_RED >> 3)) {
       // RED ; SOP fma(-unary) that reads the result and overwrites it  ->  one reduction with a post-operation
       const uint32_t nx = pc + len < code_words ? body[pc + len] : 0;
@@ -426,6 +428,7 @@ void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* h
       if (u == DVM_U_SQRT || u == DVM_U_LOG || u == DVM_U_ERF || u == DVM_U_FLOOR || u == DVM_U_ROUND || u == DVM_U_TANH ||
           u == DVM_U_TRUNC_I32 || u == DVM_U_TRUNC_U8) *heavy = true;
     }
+    if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) *heavy = true;
     pc += len ? len : 1;
   }
 }

@@ -31,6 +31,7 @@ enum {
                                                          //                            c = sub & 2 ? S[b] : w2 (sub & 8: negated)
   DVM_LK_BINI,                                           // ACC = ACC op imm           sub = rdiv / min / max, w1 = imm
   DVM_LK_BINS,                                           // ACC = ACC op S[a]          sub = rdiv / min / max
+  DVM_LK_ACT,                                            // ACC = act(ACC)             sub = DVM_ACT_* (HEAVY variants)
   DVM_LK_UN,                                             // ACC = f(ACC)               sub = unary (| 0x80: one-piece exponential)
   DVM_LK_EXPS,                                           // ACC = exp(ACC - S[a])      sub = 1: one-piece exponential
   DVM_LK_RED,                                            // S[a] = reduce(ACC); b = 1: S[a] = unary(S[a] * w2 + w3), w1 = unary or 0xff

@@ -79,6 +79,16 @@ __device__ __forceinline__ uint32_t pack_u8x4(float a, float b, float c, float d
 __device__ __forceinline__ float trunc_i32(float x) { return x != x ? 0.0f : fminf(fmaxf(truncf(x) + 0.0f, -2147483648.0f), 2147483648.0f); }
 __device__ __forceinline__ float trunc_u8(float x) { return x != x ? 0.0f : fminf(fmaxf(truncf(x) + 0.0f, 0.0f), 255.0f); }
 
+// The fused activations (DVM_OP_ACT), on pairs.  Every step rounds as the separate instructions would.
+__device__ __forceinline__ float2 packed_gelu(float2 t) {
+  const float2 e = packed_erf(__fmul2_rn(t, make_float2(0.707106769084930419921875f, 0.707106769084930419921875f)));
+  const float2 u = __fadd2_rn(e, make_float2(1.0f, 1.0f));
+  return __fmul2_rn(__fmul2_rn(t, u), make_float2(0.5f, 0.5f));
+}
+__device__ __forceinline__ float2 packed_silu(float2 t) {
+  return make_float2(t.x * fast_rcp(1.0f + fast_exp(-t.x)), t.y * fast_rcp(1.0f + fast_exp(-t.y)));
+}
+
 __device__ __forceinline__ float scalar_arith(int op, float a, float b) {
   switch (op) {
     case DVM_A_ADD: return a + b;

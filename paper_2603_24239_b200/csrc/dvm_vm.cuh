@@ -812,6 +812,11 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           }
 #undef DVM_UN_CASE
         } break;
+        case DVM_OP_ACT >> 3: {  // fused activations (pattern-based fusion, Sec. 5.1)
+          pc += 1;
+          if (op == DVM_OP_ACT + DVM_ACT_GELU) { DVM_EACH_PAIR A[i] = packed_gelu(A[i]); }
+          else { DVM_EACH_PAIR A[i] = packed_silu(A[i]); }
+        } break;
         case DVM_OP_RED >> 3: {
           // ---- row reduction (Table 1, Sum / Max / Min with N = 1): thread-local over valid slots, shuffles
           // inside the warp, shared memory across the warps of a row group ----

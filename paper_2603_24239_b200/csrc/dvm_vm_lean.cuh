@@ -608,6 +608,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(c
             DVM_EACH_PAIR A[i] = lean_exp2(__fadd2_rn(A[i], make_float2(m, m)));
           }
         } break;
+        case DVM_LK_ACT: {
+          if constexpr (HEAVY) {
+            if (sub == DVM_ACT_GELU) { DVM_EACH_PAIR A[i] = packed_gelu(A[i]); }
+            else { DVM_EACH_PAIR A[i] = packed_silu(A[i]); }
+          } else {
+            err = ST_BAD_CODE;
+          }
+        } break;
         case DVM_LK_UN: {
 #define DVM_UN_CASE(U, EXPR)                                                          \
   case U:                                                                             \

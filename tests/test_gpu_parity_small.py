@@ -216,3 +216,37 @@ def test_outer_broadcast_3d():
     cs = wl.randn((5, 1, 130), torch.float32, 3)
     outs, _ = gpu_run(p, [xs, bs, cs])
     check(p, outs, oracle_run(p, [xs, bs, cs]))
+
+
+def _gelu_prog(order=0, scale=1.0 / 2 ** 0.5, reuse_t=False):
+    p = wl.OpProgram("gelu_variant")
+    x, w = p.input("f32", 2), p.input("f32", 2)
+    t = p.binary("mul", x, w)
+    u = p.scalar("adds", p.unary("erf", p.scalar("muls", t, scale)), 1.0)
+    m = p.binary("mul", t, u) if order == 0 else p.binary("mul", u, t)
+    p.output(p.scalar("muls", m, 0.5), "f32")
+    if reuse_t:
+        p.output(p.scalar("adds", t, 3.0), "f32")
+    return p
+
+
+@pytest.mark.parametrize("order,scale,reuse_t", [(0, 1.0 / 2 ** 0.5, False), (1, 1.0 / 2 ** 0.5, False), (0, 1.0 / 2 ** 0.5, True),
+                                                 (0, 0.7, False)])
+def test_fused_gelu_matches_the_chain_it_replaces(order, scale, reuse_t):
+    """The encoder turns 0.5 * (t * (1 + erf(t / sqrt 2))) into one activation instruction (pattern-based fusion,
+    Sec. 5.1); a chain with another constant stays as it is.  Either way the result is the oracle's."""
+    prog = _gelu_prog(order, scale, reuse_t)
+    ins = [wl.randn((37, 1001), torch.float32, 5), wl.randn((1, 1001), torch.float32, 6)]
+    (g1, _), outs, want = _run(prog, ins)
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [tuple(t.shape) for t in ins])
+    assert ("gelu" in dvm.disassemble(code)) == (abs(scale - 1.0 / 2 ** 0.5) < 1e-6)
+
+
+def test_fused_silu():
+    p = wl.OpProgram("silu")
+    x, y = p.input("bf16", 2), p.input("bf16", 2)
+    p.output(p.binary("mul", p.binary("mul", p.unary("sigmoid", x), x), y), "bf16")
+    ins = [wl.randn((129, 513), torch.bfloat16, 1), wl.randn((129, 513), torch.bfloat16, 2)]
+    _run(p, ins)
+    code = dvm.encode(dvm.program_from_nodes(p.nodes), [tuple(t.shape) for t in ins])
+    assert "silu" in dvm.disassemble(code)

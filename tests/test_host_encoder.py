@@ -223,8 +223,9 @@ def test_stacked_levels_rejects_decreasing_levels_before_any_launch():
 
 def test_min_resident_ctas_picks_a_geometry_that_fits_twice_per_sm():
     """A wide GELU(x*w+b) row at 16 elements per thread: unconstrained, one row per tile with whole-row images
-    of w and b (259 units per slot: one CTA per SM); with dvm_set_min_resident_ctas(2), column blocks that fit
-    twice per SM, chosen by total work (the program shares its launch: no waves of its own to fill)."""
+    of w and b (195 units per slot: one CTA per SM; the fused activation needs no temporary); with
+    dvm_set_min_resident_ctas(2), column blocks that fit twice per SM, chosen by total work (the program shares
+    its launch: no waves of its own to fill)."""
     p = dvm.program_from_nodes(wl.stack_program("gelu_affine").nodes)
     shapes = [(148, 2893), (1, 2893), (1, 2893)]
     dvm.set_elems_per_thread(16)
@@ -235,9 +236,9 @@ def test_min_resident_ctas_picks_a_geometry_that_fits_twice_per_sm():
     finally:
         dvm.set_min_resident_ctas(0)
         dvm.set_elems_per_thread(0)
-    assert "local_units=259" in free and "col_blocks=1 " in free
+    assert "local_units=195" in free and "col_blocks=1 " in free and "gelu" in free
     # costed by total work: 3 column blocks of 1020 columns waste fewer slots than 2 of 2044 (2893 = 2 x 1020 + 853)
-    assert "local_units=163" in tight and "col_blocks=3 " in tight and "threads_per_row=64" in tight
+    assert "local_units=99" in tight and "col_blocks=3 " in tight and "threads_per_row=64" in tight
 
 
 def test_encode_strided_views_geometry_and_errors():
