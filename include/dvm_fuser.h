@@ -52,6 +52,15 @@ int dvm_fuser_unary(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, d
 int dvm_fuser_binary(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 int dvm_fuser_scalar(dvm_fuser* f, int op, int x, float s, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 int dvm_fuser_reduce(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
+/* Table 1 Cmp, Select (cond != 0 ? x : y), Cast (the value rounded to `dtype`), and the cube operation a [M,K] x b [K,N]
+ * (Sec. 4.2; bf16 operands that lie in memory).  A matmul starts a group of its own; the vector operators that
+ * arrive behind it join that group as its epilogue while the group still encodes as one matmul meta-kernel --
+ * cube-vector fusion (Sec. 5.1) on arrival.  out_dtype may be DVM_U8 / DVM_I32 (a comparison stored as 0 / 1, a cast);
+ * a value of an integer type can be read by later operators of its own group only (tensors in memory are F32 / BF16). */
+int dvm_fuser_compare(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
+int dvm_fuser_select(dvm_fuser* f, int cond, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
+int dvm_fuser_cast(dvm_fuser* f, int x, int dtype, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
+int dvm_fuser_matmul(dvm_fuser* f, int a, int b, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 
 /* The framework dropped its last reference to `value`: if it is still pending and only its own group reads
  * it, it will not be stored. */

@@ -108,6 +108,10 @@ _sig.update({
     "dvm_fuser_binary": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_scalar": ([_vp, _i, _i, C.c_float, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_reduce": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_compare": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_select": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_cast": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_matmul": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_release": ([_vp, _i], _i),
     "dvm_fuser_flush": ([_vp], _i),
     "dvm_fuser_pending": ([_vp, _pi, _pi], _i),
@@ -496,7 +500,8 @@ class Fuser:
         import torch
         if self._alloc is not None:
             return self._alloc(shape_guess, dtype)
-        return torch.empty(shape_guess, dtype=torch.bfloat16 if dtype == "bf16" else torch.float32, device="cuda")
+        tdt = {"bf16": torch.bfloat16, "f32": torch.float32, "u8": torch.uint8, "i32": torch.int32}[dtype]
+        return torch.empty(shape_guess, dtype=tdt, device="cuda")
 
     def _op(self, fn, args, out_shape, dtype):
         buf = self._result(out_shape, dtype)
@@ -519,6 +524,19 @@ class Fuser:
 
     def reduce(self, op, x, out_shape, dtype="f32"):
         return self._op(lib.dvm_fuser_reduce, (REDUCE.get(op, op), x), out_shape, dtype)
+
+    def compare(self, op, x, y, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_compare, (COMPARE.get(op, op), x, y), out_shape, dtype)
+
+    def select(self, cond, x, y, out_shape, dtype="f32"):
+        return self._op(lib.dvm_fuser_select, (cond, x, y), out_shape, dtype)
+
+    def cast(self, x, to, out_shape, dtype=None):
+        """x rounded to type `to`; stored as `dtype` (default: `to`)."""
+        return self._op(lib.dvm_fuser_cast, (x, DTYPES[to]), out_shape, dtype or to)
+
+    def matmul(self, a, b, out_shape, dtype="bf16"):
+        return self._op(lib.dvm_fuser_matmul, (a, b), out_shape, dtype)
 
     def release(self, value):
         _check(lib.dvm_fuser_release(self._h, value), "dvm_fuser_release")

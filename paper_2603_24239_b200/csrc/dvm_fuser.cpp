@@ -11,7 +11,7 @@
 
 namespace {
 
-enum OpKind { OP_UNARY, OP_BINARY, OP_SCALAR, OP_REDUCE };
+enum OpKind { OP_UNARY, OP_BINARY, OP_SCALAR, OP_REDUCE, OP_COMPARE, OP_SELECT, OP_CAST, OP_MATMUL };
 
 struct FValue {
   int dtype;
@@ -23,11 +23,19 @@ struct FValue {
 };
 
 struct FOp {
-  int kind, op, x, y;
+  int kind, op, x, y;  // (OP_SELECT: x the condition, y the then-value; OP_CAST: op the target type)
   float s;
   int out;    // value id of the result
   int group;  // index into `groups`
+  int z;      // OP_SELECT: the else-value, otherwise -1
 };
+
+// the value operands of an operator: x, then y and z where the kind has them (-1 otherwise)
+inline void operands_of(const FOp& o, int v[3]) {
+  v[0] = o.x;
+  v[1] = (o.kind == OP_BINARY || o.kind == OP_COMPARE || o.kind == OP_SELECT || o.kind == OP_MATMUL) ? o.y : -1;
+  v[2] = o.kind == OP_SELECT ? o.z : -1;
+}
 
 struct FGroup {
   std::vector<int> ops;  // pending operator indices, in arrival order
@@ -61,8 +69,12 @@ bool value_ok(const dvm_fuser* f, int v) { return v >= 0 && v < (int)f->values.s
 
 // Does another group than `g` read value v (among the pending operators)?
 bool read_elsewhere(const dvm_fuser* f, int v, int g) {
-  for (const FOp& o : f->ops)
-    if (o.group != g && (o.x == v || (o.kind == OP_BINARY && o.y == v))) return true;
+  for (const FOp& o : f->ops) {
+    if (o.group == g) continue;
+    int xs[3];
+    operands_of(o, xs);
+    if (xs[0] == v || xs[1] == v || xs[2] == v) return true;
+  }
   return false;
 }
 
@@ -95,14 +107,21 @@ int build(const dvm_fuser* f, const std::vector<int>& op_list, const FOp* extra,
   if (extra) seq.push_back(extra);
   for (size_t k = 0; k < n && st == DVM_OK; ++k) {
     const FOp& o = *seq[k];
-    int px = -1, py = -1, pid = -1;
-    st = operand(o.x, &px);
-    if (st == DVM_OK && o.kind == OP_BINARY) st = operand(o.y, &py);
+    int px = -1, py = -1, pz = -1, pid = -1;
+    int xs[3];
+    operands_of(o, xs);
+    st = operand(xs[0], &px);
+    if (st == DVM_OK && xs[1] >= 0) st = operand(xs[1], &py);
+    if (st == DVM_OK && xs[2] >= 0) st = operand(xs[2], &pz);
     if (st != DVM_OK) break;
     switch (o.kind) {
       case OP_UNARY: st = dvm_program_unary(b->prog, o.op, px, &pid); break;
       case OP_BINARY: st = dvm_program_binary(b->prog, o.op, px, py, &pid); break;
       case OP_SCALAR: st = dvm_program_scalar(b->prog, o.op, px, o.s, &pid); break;
+      case OP_COMPARE: st = dvm_program_compare(b->prog, o.op, px, py, &pid); break;
+      case OP_SELECT: st = dvm_program_select(b->prog, px, py, pz, &pid); break;
+      case OP_CAST: st = dvm_program_cast(b->prog, px, o.op, &pid); break;
+      case OP_MATMUL: st = dvm_program_matmul(b->prog, px, py, &pid); break;
       default: st = dvm_program_reduce(b->prog, o.op, px, -1, &pid); break;
     }
     if (st == DVM_OK) ids.push_back({o.out, pid});
@@ -138,8 +157,11 @@ int encode(const dvm_fuser* f, const Built& b, std::vector<uint64_t>* code, size
 }
 
 int add_op(dvm_fuser* f, FOp o, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
-  if (!f || !value || !out_ptr || (out_dtype != DVM_F32 && out_dtype != DVM_BF16)) return DVM_ERR_INVALID_ARG;
-  if (!value_ok(f, o.x) || (o.kind == OP_BINARY && !value_ok(f, o.y))) return DVM_ERR_INVALID_ARG;
+  if (!f || !value || !out_ptr || out_dtype < DVM_F32 || out_dtype > DVM_I32) return DVM_ERR_INVALID_ARG;
+  int xs[3];
+  operands_of(o, xs);
+  for (int k = 0; k < 3; ++k)
+    if ((k == 0 || xs[k] >= 0) && !value_ok(f, xs[k])) return DVM_ERR_INVALID_ARG;
   if ((int)f->ops.size() >= DVM_FUSER_MAX_OPS) {  // flush condition: the operator buffer is full
     int st = dvm_fuser_flush(f);
     if (st != DVM_OK) return st;
@@ -155,25 +177,28 @@ int add_op(dvm_fuser* f, FOp o, int out_dtype, void* out_ptr, dvm_shape* out_sha
   o.out = (int)f->values.size() - 1;
 
   // producer groups of the operands
-  int prod[2] = {-1, -1}, np = 0;
-  const int xs[2] = {o.x, o.kind == OP_BINARY ? o.y : -1};
-  for (int k = 0; k < 2; ++k)
+  int prod[3] = {-1, -1, -1}, np = 0;
+  for (int k = 0; k < 3; ++k)
     if (xs[k] >= 0 && f->values[xs[k]].op >= 0) {
       const int g = f->ops[f->values[xs[k]].op].group;
-      if (np == 0 || prod[0] != g) prod[np++] = g;
+      bool seen = false;
+      for (int q = 0; q < np; ++q) seen = seen || prod[q] == g;
+      if (!seen) prod[np++] = g;
     }
   // candidate: the operator joins the producers' group (two producer groups: they merge around it)
   int joined = -1, st = DVM_OK;
   std::vector<dvm_shape> shapes;
   // two producer groups merge around the operator only when both read nothing but tensors in memory:
   // then no third group can sit between them, and the merged group cannot end up depending on itself
-  const bool can_join = np == 1 || (np == 2 && f->groups[prod[0]].level == 0 && f->groups[prod[1]].level == 0);
+  bool can_join = np == 1;
+  if (np >= 2) {
+    can_join = true;
+    for (int q = 0; q < np; ++q) can_join = can_join && f->groups[prod[q]].level == 0;
+  }
   if (can_join) {
     std::vector<int> cand = f->groups[prod[0]].ops;
-    if (np == 2) {
-      cand.insert(cand.end(), f->groups[prod[1]].ops.begin(), f->groups[prod[1]].ops.end());
-      std::sort(cand.begin(), cand.end());
-    }
+    for (int q = 1; q < np; ++q) cand.insert(cand.end(), f->groups[prod[q]].ops.begin(), f->groups[prod[q]].ops.end());
+    if (np >= 2) std::sort(cand.begin(), cand.end());
     Built b;
     st = build(f, cand, &o, prod[0], true, &b);
     if (st == DVM_OK) {
@@ -189,9 +214,9 @@ int add_op(dvm_fuser* f, FOp o, int out_dtype, void* out_ptr, dvm_shape* out_sha
     }
   }
   if (joined >= 0) {
-    if (np == 2) {  // merge the second producer group into the first
+    for (int q = 1; q < np; ++q) {  // merge the other producer groups into the first
       FGroup& a = f->groups[prod[0]];
-      FGroup& c = f->groups[prod[1]];
+      FGroup& c = f->groups[prod[q]];
       for (int k : c.ops) f->ops[k].group = prod[0];
       a.ops.insert(a.ops.end(), c.ops.begin(), c.ops.end());
       std::sort(a.ops.begin(), a.ops.end());
@@ -259,19 +284,35 @@ extern "C" int dvm_fuser_tensor(dvm_fuser* f, int dtype, const dvm_shape* shape,
 }
 
 extern "C" int dvm_fuser_unary(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
-  FOp o = {OP_UNARY, op, x, -1, 0.f, -1, -1};
+  FOp o = {OP_UNARY, op, x, -1, 0.f, -1, -1, -1};
   return add_op(f, o, out_dtype, out_ptr, out_shape, value);
 }
 extern "C" int dvm_fuser_binary(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
-  FOp o = {OP_BINARY, op, x, y, 0.f, -1, -1};
+  FOp o = {OP_BINARY, op, x, y, 0.f, -1, -1, -1};
   return add_op(f, o, out_dtype, out_ptr, out_shape, value);
 }
 extern "C" int dvm_fuser_scalar(dvm_fuser* f, int op, int x, float s, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
-  FOp o = {OP_SCALAR, op, x, -1, s, -1, -1};
+  FOp o = {OP_SCALAR, op, x, -1, s, -1, -1, -1};
   return add_op(f, o, out_dtype, out_ptr, out_shape, value);
 }
 extern "C" int dvm_fuser_reduce(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
-  FOp o = {OP_REDUCE, op, x, -1, 0.f, -1, -1};
+  FOp o = {OP_REDUCE, op, x, -1, 0.f, -1, -1, -1};
+  return add_op(f, o, out_dtype, out_ptr, out_shape, value);
+}
+extern "C" int dvm_fuser_compare(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
+  FOp o = {OP_COMPARE, op, x, y, 0.f, -1, -1, -1};
+  return add_op(f, o, out_dtype, out_ptr, out_shape, value);
+}
+extern "C" int dvm_fuser_select(dvm_fuser* f, int cond, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
+  FOp o = {OP_SELECT, 0, cond, x, 0.f, -1, -1, y};
+  return add_op(f, o, out_dtype, out_ptr, out_shape, value);
+}
+extern "C" int dvm_fuser_cast(dvm_fuser* f, int x, int dtype, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
+  FOp o = {OP_CAST, dtype, x, -1, 0.f, -1, -1, -1};
+  return add_op(f, o, out_dtype, out_ptr, out_shape, value);
+}
+extern "C" int dvm_fuser_matmul(dvm_fuser* f, int a, int b, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
+  FOp o = {OP_MATMUL, 0, a, b, 0.f, -1, -1, -1};
   return add_op(f, o, out_dtype, out_ptr, out_shape, value);
 }
 
@@ -315,8 +356,9 @@ extern "C" int dvm_fuser_flush(dvm_fuser* f) {
   for (bool changed = true; changed;) {
     changed = false;
     for (const FOp& o : f->ops) {
-      const int xs[2] = {o.x, o.kind == OP_BINARY ? o.y : -1};
-      for (int k = 0; k < 2; ++k) {
+      int xs[3];
+      operands_of(o, xs);
+      for (int k = 0; k < 3; ++k) {
         if (xs[k] < 0 || f->values[xs[k]].op < 0) continue;
         const int h = f->ops[f->values[xs[k]].op].group;
         if (h != o.group && f->groups[o.group].level < f->groups[h].level + 1) {

@@ -58,13 +58,41 @@ def test_shape_errors_are_reported_and_leave_the_buffer_intact():
     assert f.pending() == (0, 0)
 
 
+def test_matmul_takes_its_epilogue_on_arrival():
+    """Cube-vector fusion (Sec. 5.1) in the stream: a matmul opens a group, the vector operators that arrive behind
+    it become its epilogue, and an operator the matmul meta-kernel cannot hold (a second matmul) opens another."""
+    f = dvm.Fuser(alloc=_fake_alloc())
+    x = f.tensor(0x1000, "bf16", (100, 512)); w = f.tensor(0x100000, "bf16", (512, 256))
+    c = f.tensor(0x200000, "bf16", (100, 256))
+    mm = f.matmul(x, w, (100, 256))
+    assert f.pending() == (1, 1)
+    y = f.binary("add", mm, c, (100, 256), "bf16")
+    z = f.unary("sigmoid", y, (100, 256), "bf16")
+    assert f.pending() == (3, 1)
+    w2 = f.tensor(0x300000, "bf16", (256, 64))
+    f.matmul(z, w2, (100, 64))                 # its A operand is computed, not in memory: a group of its own
+    assert f.pending() == (4, 2)
+
+
+def test_compare_select_cast_fuse_with_their_producers():
+    f = dvm.Fuser(alloc=_fake_alloc())
+    a = f.tensor(0x1000, "f32", (9, 70)); b = f.tensor(0x2000, "f32", (9, 70))
+    m = f.compare("gt", a, b, (9, 70), "u8")
+    s = f.select(m, f.binary("add", a, b, (9, 70)), f.binary("sub", a, b, (9, 70)), (9, 70))
+    q = f.cast(f.scalar("muls", s, 10.0, (9, 70)), "i32", (9, 70))
+    assert f.pending() == (6, 1)
+    with pytest.raises(dvm.DvmError):
+        f.select(m, a, 99, (9, 70))            # unknown value id
+    assert f.pending() == (6, 1)
+
+
 # ------------------------------------------------------------------------------------------- on the GPU
-def _oracle_chain(nodes_fn, ins):
+def _oracle_chain(nodes_fn, ins, out_dtypes=None):
     p = wl.OpProgram("chain")
-    ids = [p.input("f32", t.dim()) for t in ins]
+    ids = [p.input("bf16" if t.dtype == torch.bfloat16 else "f32", t.dim()) for t in ins]
     outs = nodes_fn(p, ids)
-    for o in outs:
-        p.output(o, "f32")
+    for k, o in enumerate(outs):
+        p.output(o, out_dtypes[k] if out_dtypes else "f32")
     return orc.evaluate(p.nodes, [wl.to_f64(t) for t in ins])
 
 
@@ -173,3 +201,63 @@ def test_long_levels_keep_their_own_launches():
     # |x| and max are exact in any precision: the maxima equal the oracle's bit for bit
     assert np.array_equal(wl.to_f64(f.tensors[m]), want[0])
     _close(f.tensors[r], want[1])
+
+
+@pytest.mark.gpu
+def test_if_else_add_stream_with_mask_and_quantised_output():
+    """Table 1 Cmp / Select / Cast through the streaming fuser: one group, one launch; the u8 mask and the i32
+    codes bit-exact against the oracle (inputs on a grid of sixteenths, so every decision is exact in fp32)."""
+    a = (torch.round(wl.randn((77, 1500), torch.float32, 11) * 16) / 16).cuda()
+    b = (torch.round(wl.randn((77, 1500), torch.float32, 12) * 16) / 16).cuda()
+    f = dvm.Fuser()
+    va, vb = f.tensor(a), f.tensor(b)
+    m = f.compare("gt", va, vb, a.shape, "u8")
+    s = f.select(m, f.binary("add", va, vb, a.shape), f.binary("sub", va, vb, a.shape), a.shape)
+    q = f.cast(f.scalar("muls", s, 4.0, a.shape), "i32", a.shape)
+    assert f.pending() == (6, 1)
+    n0 = dvm.launch_count()
+    f.flush()
+    torch.cuda.synchronize()
+    assert dvm.launch_count() - n0 == 1 and dvm.last_device_status() == 0
+    def chain(p, i):
+        pm = p.compare("gt", i[0], i[1])
+        ps = p.select(pm, p.binary("add", i[0], i[1]), p.binary("sub", i[0], i[1]))
+        return [pm, ps, p.cast(p.scalar("muls", ps, 4.0), "i32")]
+    want = _oracle_chain(chain, [a, b], ["u8", "f32", "i32"])
+    assert f.tensors[m].dtype == torch.uint8 and f.tensors[q].dtype == torch.int32
+    assert np.array_equal(f.tensors[m].cpu().numpy().astype(np.float64), want[0])
+    assert np.array_equal(wl.to_f64(f.tensors[s]), want[1])
+    assert np.array_equal(f.tensors[q].cpu().numpy().astype(np.float64), want[2])
+
+
+@pytest.mark.gpu
+def test_matmul_with_streamed_epilogue_matches_oracle_in_one_launch():
+    M, K, N = 300, 512, 384
+    x = wl.randn((M, K), torch.bfloat16, 21).cuda()
+    w = wl.randn((K, N), torch.bfloat16, 22, std=K ** -0.5).cuda()
+    c = wl.randn((M, N), torch.bfloat16, 23).cuda()
+    f = dvm.Fuser()
+    vx, vw, vc = f.tensor(x), f.tensor(w), f.tensor(c)
+    mm = f.matmul(vx, vw, (M, N))
+    y = f.unary("sigmoid", f.binary("add", mm, vc, (M, N), "bf16"), (M, N), "f32")
+    f.release(mm)
+    assert f.pending() == (3, 1)
+    n0 = dvm.launch_count()
+    f.flush()
+    torch.cuda.synchronize()
+    assert dvm.launch_count() - n0 == 1 and dvm.last_device_status() == 0
+    want = _oracle_chain(lambda p, i: [p.unary("sigmoid", p.binary("add", p.matmul(i[0], i[1]), i[2]))], [x, w, c])[0]
+    # fp32 accumulation over K = 512 products of bf16 values, then sigmoid (slope <= 1/4)
+    assert np.max(np.abs(wl.to_f64(f.tensors[y]) - want)) <= 2e-5
+    # a matmul next to an independent vector group: the stacked launch refuses the mix, each runs by itself
+    f2 = dvm.Fuser()
+    vx, vw, vc = f2.tensor(x), f2.tensor(w), f2.tensor(c)
+    mm = f2.matmul(vx, vw, (M, N), "f32")
+    e = f2.unary("exp", vc, (M, N))
+    assert f2.pending() == (2, 2)
+    f2.flush()
+    torch.cuda.synchronize()
+    assert dvm.last_device_status() == 0
+    want = _oracle_chain(lambda p, i: [p.matmul(i[0], i[1]), p.unary("exp", i[2])], [x, w, c])
+    assert np.max(np.abs(wl.to_f64(f2.tensors[mm]) - want[0])) <= 1e-4 * np.max(np.abs(want[0]))
+    _close(f2.tensors[e], want[1])
