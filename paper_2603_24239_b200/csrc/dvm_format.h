@@ -119,7 +119,10 @@ enum { DVM_DT_F32 = 0, DVM_DT_BF16 = 1,
 #define DVM_INSN(op, len, a, b) \
   ((uint32_t)(op) | ((uint32_t)(len) << 8) | ((uint32_t)(a) << 16) | ((uint32_t)(b) << 24))
 #define DVM_INSN_OP(w) ((w) & 0xffu)
-#define DVM_INSN_LEN(w) (((w) >> 8) & 0xffu)
+#define DVM_INSN_LEN(w) (((w) >> 8) & 0xfu)
+// bits 12..15 of word 0: the phase tag of an instruction of a phased program (see DVM_OP_PHASE); 0 everywhere else
+#define DVM_INSN_TAG(w) (((w) >> 12) & 0xfu)
+#define DVM_INSN_SET_TAG(w, t) (((w) & ~0xf000u) | ((uint32_t)(t) << 12))
 #define DVM_INSN_A(w) (((w) >> 16) & 0xffu)
 #define DVM_INSN_B(w) (((w) >> 24) & 0xffu)
 
@@ -166,6 +169,16 @@ enum {
   DVM_OP_BCS = 0x08,   // a = scalar register                          : ACC = broadcast(S[a]) (Table 1, Broadcast)
   DVM_OP_SOP = 0x09,   // per-row scalar arithmetic; a = dst scalar register, b = kind;
                        // len 2: word1 = sub_op | src1 << 8 | src2 << 16 ; len 3: word2 = fp32 immediate
+  DVM_OP_PHASE = 0x0a, // Rows longer than a tile (Table 1, Sum / Max / Min over a long axis): the program runs in P phases over
+                       // the CB column blocks of a row -- a CTA takes a row through P * CB tiles in order, every tile walks
+                       // the same code, and the per-row scalars stay in place between them.  A reduction accumulates over
+                       // the blocks of its phase and is complete for the next one (a softmax: the maximum, then the sum of
+                       // the exponentials, then the quotient).
+                       //   a = 0xff, b = P : first compute instruction of a phased program, nothing at run time
+                       //   a = q           : the tiles of phases < q end here
+                       // Tag t > 0 (DVM_INSN_TAG) on RED / SOP / STS / STG: the instruction runs in phase t - 1 only;
+                       // RED in every block of it (combining with the blocks before), SOP and STS in its last block
+                       // (right behind the reductions that complete there), STG in every block.
   DVM_OP_BINI = 0x10,  // 0x10 + arith; len 2, word1 = fp32 immediate  : ACC = ACC op imm     (Adds / Muls)
   DVM_OP_BIN = 0x18,   // 0x18 + arith; a = local register or 0xff (ACC itself), b = dtype : ACC = ACC op L[a]
   DVM_OP_BINS = 0x20,  // 0x20 + arith; a = scalar register            : ACC = ACC op S[a]    (row broadcast)
@@ -185,6 +198,9 @@ enum {
   DVM_OP_LAST = 0x60   // every arithmetic class starts at a multiple of 8: the low 3 bits are the operation
 };
 #define DVM_REG_ACC 0xff
+#define DVM_MAX_PHASES 8
+// phases of a phased program, from the first word of its compute section; 0: the program is not phased
+#define DVM_PHASES_OF(w0) ((DVM_INSN_OP(w0) == DVM_OP_PHASE && DVM_INSN_A(w0) == 0xffu) ? DVM_INSN_B(w0) : 0u)
 // DVM_SK_FMAU: S[a] = unary(S[src] * imm0 + imm1); len 4: word1 = unary (0xff: none) | src << 8, word2 = imm0, word3 = imm1
 enum { DVM_SK_BIN = 0, DVM_SK_BINI = 1, DVM_SK_UN = 2, DVM_SK_FMAU = 3 };
 

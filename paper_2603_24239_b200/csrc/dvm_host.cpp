@@ -7,6 +7,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <chrono>
 
 #include <utility>
@@ -315,6 +316,8 @@ struct Enc {
   const float* scalars;
   int n_scalars;
   bool fail;
+  bool phased;                    // rows longer than a tile: the program runs in phases over column blocks (DVM_OP_PHASE)
+  int n_phases;
 };
 
 static inline int root(const Enc& e, int v) {
@@ -354,7 +357,7 @@ static void release(Enc& e, int v) {  // free the registers of a dead value
       e.tmp_val[e.lreg_of[v] - e.n_in_regs] = -1;
       e.lreg_of[v] = -1;
     }
-  } else if (e.sreg_of[v] >= 0) {
+  } else if (e.sreg_of[v] >= 0 && !e.phased) {  // (a phased program's scalars outlive the tile: never recycled)
     e.sreg_val[e.sreg_of[v]] = -1;
     e.sreg_of[v] = -1;
   }
@@ -781,6 +784,80 @@ static bool gen_body(Enc& e) {
   return !e.fail;
 }
 
+// Rows longer than a tile (DVM_OP_PHASE).  The compute section was generated for one tile; every tile of a row
+// walks it again, so what a tile computes must depend only on the tile's own loads and on per-row scalars that are
+// complete.  This pass follows the code once, notes in which phase each value becomes available -- a tile value
+// as early as its operands, a reduction one phase after the value it reduces -- tags the instructions that must
+// run once (RED in the phase of its operand; scalar arithmetic and scalar stores in the last block of the phase
+// that completes their operands; tile stores in the last phase), cuts every phase's walk off behind the last
+// instruction it needs, and puts the phase count in front.
+static bool tag_phases(Enc& e) {
+  int lreg_av[DVM_MAX_LREGS], s_ready[DVM_MAX_SREGS];
+  for (int k = 0; k < DVM_MAX_LREGS; ++k) lreg_av[k] = 0;
+  for (int k = 0; k < DVM_MAX_SREGS; ++k) s_ready[k] = -1;  // -1: ready from the first tile on (a loaded per-row value)
+  int acc_av = 0, P = 1;
+  auto after = [](int ready) { return ready + 1; };  // first phase that may read a scalar completed in phase `ready`
+  for (int pass = 0; pass < 2; ++pass) {
+    acc_av = 0;
+    for (int pc = 0; pc < e.n_body;) {
+      uint32_t w0 = e.body[pc];
+      const uint32_t op = DVM_INSN_OP(w0), a = DVM_INSN_A(w0), b = DVM_INSN_B(w0);
+      const int len = (int)DVM_INSN_LEN(w0);
+      int tag = 0;
+      if (op == DVM_OP_LDA) acc_av = lreg_av[a];
+      else if (op == DVM_OP_STA) lreg_av[a] = acc_av;
+      else if (op == DVM_OP_LSS) s_ready[a] = -1;
+      else if (op == DVM_OP_BCS) acc_av = after(s_ready[a]);
+      else if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) acc_av = std::max(lreg_av[a], lreg_av[b & 0x3f]);
+      else if ((op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) || (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP)) {
+        if (a != DVM_REG_ACC) acc_av = std::max(acc_av, lreg_av[a]);
+      } else if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) acc_av = std::max(acc_av, std::max(lreg_av[a], lreg_av[b & 0x3f]));
+      else if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) acc_av = std::max(acc_av, after(s_ready[a]));
+      else if (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) {
+        tag = acc_av + 1;
+        s_ready[a] = acc_av;
+        P = std::max(P, acc_av + 1);
+      } else if (op == DVM_OP_SOP) {
+        const uint32_t w1 = e.body[pc + 1];
+        int j = s_ready[(w1 >> 8) & 0xff];
+        if (b == DVM_SK_BIN) j = std::max(j, s_ready[(w1 >> 16) & 0xff]);
+        tag = j < 0 ? 0 : j + 1;  // from loaded values only: every tile may repeat it
+        s_ready[a] = j;
+      } else if (op == DVM_OP_STS) {
+        tag = std::max(s_ready[a], 0) + 1;
+      } else if (op == DVM_OP_STG) {
+        P = std::max(P, acc_av + 1);
+        tag = P;  // (final in the second pass)
+      }
+      if (pass == 1 && tag) e.body[pc] = DVM_INSN_SET_TAG(w0, tag);
+      pc += len;
+    }
+    if (P > DVM_MAX_PHASES) return false;
+  }
+  // the walk of phase k ends behind the last instruction tagged for a phase <= k
+  uint32_t out[sizeof(e.body) / sizeof(e.body[0])];
+  int n = 0, cut[DVM_MAX_PHASES];
+  for (int k = 0; k + 1 < P; ++k) cut[k] = 0;
+  for (int pc = 0; pc < e.n_body; pc += (int)DVM_INSN_LEN(e.body[pc])) {
+    const int t = (int)DVM_INSN_TAG(e.body[pc]);
+    for (int k = 0; k + 1 < P; ++k)
+      if (t && t - 1 <= k) cut[k] = pc + (int)DVM_INSN_LEN(e.body[pc]);
+  }
+  if (e.n_body + P + 1 > (int)(sizeof(e.body) / sizeof(e.body[0]))) return false;
+  out[n++] = DVM_INSN(DVM_OP_PHASE, 1, 0xff, P);
+  for (int pc = 0; pc < e.n_body;) {
+    const int len = (int)DVM_INSN_LEN(e.body[pc]);
+    for (int q = 0; q < len; ++q) out[n++] = e.body[pc + q];
+    pc += len;
+    for (int k = 0; k + 1 < P; ++k)
+      if (cut[k] == pc) out[n++] = DVM_INSN(DVM_OP_PHASE, 1, k + 1, 0);
+  }
+  memcpy(e.body, out, (size_t)n * 4);
+  e.n_body = n;
+  e.n_phases = P;
+  return true;
+}
+
 }  // namespace
 
 int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in, const float* scalars,
@@ -1018,7 +1095,11 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   if (primary >= 0) e.opd[primary].primary = true;
 
   // ---- 5. code: load section + compute section (independent of the tile geometry) ----
+  // a reduced row longer than the widest tile (256 threads x 32 elements) is walked in column blocks, in phases
+  e.phased = has_reduce && !combine_axis && !empty && C > (int64_t)DVM_VM_THREADS * DVM_VM_VMAX;
+  e.n_phases = 1;
   if (!gen_body(e)) return DVM_ERR_UNSUPPORTED;  // more live tile values than local registers
+  if (e.phased && !tag_phases(e)) return DVM_ERR_UNSUPPORTED;  // more phases, or per-row scalars, than the machine holds
   const int nreg = e.n_in_regs + e.n_tmp_regs;
   int in_dtype[DVM_MAX_LREGS], in_opd[DVM_MAX_LREGS];
   for (int k = 0; k < e.n_in_regs; ++k) {
@@ -1087,7 +1168,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     g.one_slot = false;
     if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
     int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
-    if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
+    if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && !e.phased && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
       // Two slots fit once per SM, one slot fits twice: eight more warps per SM are worth more than the
       // prefetch inside a CTA (the other CTA computes while this one waits for its tile).  Only a launch of
       // the program on its own can honour this; the programs of a stacked launch share two slots.
@@ -1101,7 +1182,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   const int W0 = W;
   // 24 elements per thread (rows that fill three quarters of a 32-element tile) exist as the one-program
   // basic interpreter variant only: not for programs of stacked launches, not with Cmp / Select / views
-  bool plain = g_min_resident_ctas == 0 && !combine_axis;
+  bool plain = g_min_resident_ctas == 0 && !combine_axis && !e.phased;
   for (int i = 0; i < NN; ++i) {
     const Node& n = p->nodes[i];
     if (n.kind == NK_COMPARE || n.kind == NK_SELECT || (n.kind == NK_UNARY && n.op == DVM_ISFINITE)) plain = false;
@@ -1164,8 +1245,9 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       // ... but not so few threads per row that a row copy shrinks below 512 bytes while the rows are wider
       // (measured on column sums: 256-byte copies 1560 GB/s, 512 bytes 1640, 1 KB and more lose to the atomics)
       if (combine_axis && cap * 4 < 512 && C * 4 >= 512) continue;
+      if (e.phased && lg != 8) continue;  // one row per tile: the whole CTA on a column block
       int64_t ct;
-      if (has_reduce) {
+      if (has_reduce && !e.phased) {
         // a whole row per thread group; at the widest group a row may use the full capacity: its last
         // columns then wrap around into the head slots of a misaligned row
         if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
@@ -1178,7 +1260,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
       g.log2G = lg;
       g.Ctile = ct;
       g.CB = cdiv(C, ct);
-      g.n_tiles = cdiv(R, T / G) * g.CB;
+      g.n_tiles = cdiv(R, T / G) * g.CB * e.n_phases;
       // the local-memory need of this geometry decides how many CTAs are resident at once
       const int ctas = layout(g);
       if (ctas < 1) continue;
@@ -1481,7 +1563,7 @@ extern "C" int dvm_encode_batch(int n, const dvm_program* const* programs, const
 // Verification and the readable dump
 // ---------------------------------------------------------------------------
 static int insn_expected_len(uint32_t op, uint32_t w0) {
-  if (op <= DVM_OP_BCS) return 1;
+  if (op <= DVM_OP_BCS || op == DVM_OP_PHASE) return 1;
   if (op == DVM_OP_SOP) return DVM_INSN_B(w0) == DVM_SK_BINI ? 3 : (DVM_INSN_B(w0) == DVM_SK_FMAU ? 4 : 2);
   if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) return 1;
@@ -1556,12 +1638,16 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
   uint64_t R = (uint64_t)w[DVM_H_ROWS_LO] | ((uint64_t)w[DVM_H_ROWS_HI] << 32);
   uint32_t flags = geom >> 24;
   const uint64_t pad = 0;  // a misaligned row that fills the whole capacity wraps its last columns into the head slots
+  // a phased program (rows longer than a tile) says so in the first word of its compute section
+  const uint32_t n_phases = load_words < body ? DVM_PHASES_OF((lt + n_lregs)[load_words]) : 0u;  // 0: not phased
+  if (n_phases > DVM_MAX_PHASES) return DVM_ERR_BAD_CODE;
+  if (n_phases && (lg != 8 || (flags & DVM_F_FLAT))) return DVM_ERR_BAD_CODE;  // one row per tile
   if (!(flags & DVM_F_ALIGNED) && w[DVM_H_PRIMARY] == 0xffffffffu) return DVM_ERR_BAD_CODE;
   if (w[DVM_H_N_TILES] > 0) {
     if (ctile == 0 || cb == 0 || ctile + pad > G * Vv) return DVM_ERR_BAD_CODE;
     if (cb * ctile < C || (cb - 1) * ctile >= C) return DVM_ERR_BAD_CODE;
     uint64_t rpt = DVM_VM_THREADS / G;
-    if ((uint64_t)w[DVM_H_N_TILES] != ((R + rpt - 1) / rpt) * cb) return DVM_ERR_BAD_CODE;
+    if ((uint64_t)w[DVM_H_N_TILES] != ((R + rpt - 1) / rpt) * cb * (n_phases ? n_phases : 1u)) return DVM_ERR_BAD_CODE;
     if (w[DVM_H_LAST_ROW_COLS] == 0 || w[DVM_H_LAST_ROW_COLS] > C) return DVM_ERR_BAD_CODE;
     if ((uint64_t)w[DVM_H_OUTER0] * w[DVM_H_OUTER1] * w[DVM_H_OUTER2] != R) return DVM_ERR_BAD_CODE;
   }
@@ -1599,6 +1685,17 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     if (el < 0 || (uint32_t)el != len || pc + len > body) return DVM_ERR_BAD_CODE;
     const bool in_load = pc < load_words;
     if ((op == DVM_OP_LDG || op == DVM_OP_LDS) != in_load) return DVM_ERR_BAD_CODE;  // loads live in the load section only
+    {
+      // phase tags: on the run-once instructions of a phased program only
+      const uint32_t tag = DVM_INSN_TAG(w0);
+      const bool taggable = op == DVM_OP_STG || op == DVM_OP_STS || op == DVM_OP_SOP || (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED);
+      if (tag > (taggable ? n_phases : 0u)) return DVM_ERR_BAD_CODE;
+      if (n_phases && tag == 0 && (op == DVM_OP_STG || op == DVM_OP_STS || (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED)))
+        return DVM_ERR_BAD_CODE;
+      if (op == DVM_OP_PHASE) {
+        if (pc == load_words ? (a != 0xffu || bb < 1) : (a < 1 || a >= n_phases || bb != 0)) return DVM_ERR_BAD_CODE;
+      }
+    }
     if (op == DVM_OP_LDG || op == DVM_OP_STG) {
       if (bb >= n_opd) return DVM_ERR_BAD_CODE;
       uint32_t info = ot[bb * DVM_OPD_WORDS];
@@ -1714,10 +1811,12 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     uint32_t w0 = b[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), bb = DVM_INSN_B(w0);
     if (pc == w[DVM_H_LOAD_WORDS]) outf(o, "  ---- compute ----\n");
     outf(o, "  %04x: ", pc * 4);
+    if (DVM_INSN_TAG(w0)) outf(o, "@p%u ", DVM_INSN_TAG(w0) - 1);  // runs in this phase only
     float imm = 0.f;
     if (len >= 2) memcpy(&imm, &b[pc + len - 1], 4);
     const char* dts = bb == DVM_DT_BF16 ? ".bf16" : "";
     if (op == DVM_OP_NOP) outf(o, "nop\n");
+    else if (op == DVM_OP_PHASE) { if (a == 0xffu) outf(o, "phases    %u\n", bb); else outf(o, "end.below p%u\n", a); }
     else if (op == DVM_OP_LDG) outf(o, "load%s l%u, m%u\n", (a & 0x80) ? ".once" : "     ", a & 0x7f, bb);
     else if (op == DVM_OP_LDS) outf(o, "load.row  x%u, m%u\n", a, bb);
     else if (op == DVM_OP_LDA) outf(o, "copy      acc, l%u%s\n", a, dts);

@@ -433,6 +433,13 @@ void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* h
   }
 }
 
+// Phases of a phased program (rows longer than a tile run in phases over their column blocks: DVM_OP_PHASE), 0 for the rest.
+uint32_t program_phases(const uint32_t* w) {
+  const uint32_t counts = w[DVM_H_COUNTS], geom = w[DVM_H_GEOM];
+  const uint32_t* body = w + DVM_HDR_WORDS + 2 * (counts & 0xff) + ((counts >> 16) & 0xff) * DVM_OPD_WORDS + ((geom >> 16) & 0xff);
+  return w[DVM_H_LOAD_WORDS] < w[DVM_H_CODE_WORDS] ? DVM_PHASES_OF(body[w[DVM_H_LOAD_WORDS]]) : 0u;
+}
+
 static_assert(offsetof(dvm::VMParams<PW_SMALL>, words) % 16 == 0 && offsetof(dvm::VMParams<PW_LARGE>, words) % 16 == 0,
               "linked records are loaded as 16-byte vectors of the parameter space");
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
@@ -484,6 +491,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   uint64_t need = dir;
   uint64_t total_tiles = 0;
   uint32_t units = 0;
+  uint32_t row_tiles = 0;
   int V = 0;
   int ext = 0;  // the extension level the launch needs: 1 Cmp / Select / Pow / IsFinite, 2 also views
   for (int i = 0; i < n_programs; ++i) {
@@ -496,6 +504,15 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) ext = 2;
     if (V && v != V) return DVM_ERR_INVALID_ARG;  // one kernel variant per launch: same elements per thread
     V = v;
+    const uint32_t phases = program_phases(c);
+    if (phases) {
+      // a phased program: a CTA walks the tiles of a row in order -- a launch of its own, without a work queue;
+      // the views variant of the interpreter carries the phase logic
+      if (n_programs != 1 || use_queue || level || tile_end) return DVM_ERR_UNSUPPORTED;
+      if (total_tiles > 0x7fffffffull) return DVM_ERR_TOO_LARGE;
+      row_tiles = phases * c[DVM_H_COL_BLOCKS];
+      ext = 2;
+    }
   }
   if (need > PW_LARGE || total_tiles > 0xffffffffull) return DVM_ERR_TOO_LARGE;
   if (tile_end) {  // a range of the program's tiles
@@ -535,7 +552,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.use_queue = use_queue ? 1u : 0u;
   P.levels = one_slot ? 2u : (level ? 1u : 0u);
   P.tile_begin = tile_begin;
-  P.reserved = 0;
+  P.row_tiles = row_tiles;
   P.status = dev.scratch;
   P.queue = dev.scratch + 8 + 4 * dev.queue_slot;
 
@@ -550,7 +567,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   st = dvm_occupancy(variant, smem, &occ);
   if (st != DVM_OK) return st;
   uint64_t slots = (uint64_t)dev.sm_count * occ;
-  const uint64_t run_tiles = total_tiles - tile_begin;
+  const uint64_t run_tiles = row_tiles ? total_tiles / row_tiles : total_tiles - tile_begin;  // (phased: whole rows per CTA)
   int grid = (int)(run_tiles < slots ? run_tiles : slots);
   // Everything is placed and checked: only now touch the caller's memory.  Results that tiles combine
   // atomically are filled with their identity (one small kernel per such output), then the interpreter starts.
@@ -876,6 +893,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
     if ((c[DVM_H_GEOM] >> 24) & DVM_F_VIEWS) ext = 2;
     if (V && v != V) return DVM_ERR_INVALID_ARG;
     V = v;
+    if (program_phases(c)) return DVM_ERR_UNSUPPORTED;  // a phased program is launched on its own (dvm_launch)
   }
   if (need > PW_LARGE || total_tiles > DVM_NOALLOC_MAX_TILES) return DVM_ERR_TOO_LARGE;
   if (total_tiles == 0) return DVM_OK;
@@ -907,7 +925,7 @@ extern "C" int dvm_launch_stacked_noalloc(int n_programs, const void* const* cod
   P.use_queue = 1u;
   P.levels = 0u;
   P.tile_begin = 0u;
-  P.reserved = 0u;
+  P.row_tiles = 0u;
   P.status = dev.scratch;
   P.queue = dev.scratch + 2;
   const size_t smem = (2 * (size_t)units + 1) * DVM_LOCAL_UNIT;

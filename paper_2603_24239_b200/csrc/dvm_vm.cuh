@@ -64,7 +64,9 @@ struct VMParams {
                          // 2: one tile slot per CTA (slot_bytes = 0): no tile is loaded ahead, nothing is waited for
   uint32_t tile_begin;   // one-program launches: the first tile of the launch (tiles [tile_begin, total_tiles) run; a
                          // caller that pipelines host copies with execution launches a program in ranges of tiles)
-  uint32_t reserved;     // (keeps `words` on a 16-byte boundary of the parameter space: linked records are loaded as vectors)
+  uint32_t row_tiles;    // a phased program (DVM_OP_PHASE; one-program launches of the views variant): the P * CB tiles a CTA
+                         // takes a row through, in order, before it moves on to its next row; otherwise 0
+                         // (the field also keeps `words` on a 16-byte boundary: linked records are loaded as vectors)
   unsigned int* status;  // device status word
   unsigned int* queue;   // [0] next tile to claim, [1] CTAs finished, [2] tiles completed (all zero between launches)
   uint32_t words[PW];    // [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, if levels)][programs ...]
@@ -84,6 +86,8 @@ struct TileCtx {
   uint32_t row;      // row of the dominant (collapsed) shape (not clamped: rows past the end have ncols = 0)
   uint32_t col0;
   uint32_t flags;
+  uint32_t phase;    // phased programs: the tile's phase, and whether its column block is the row's last
+  bool last_block;
 };
 
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
@@ -319,6 +323,17 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     const uint32_t CB = CW(prog + DVM_H_COL_BLOCKS);
     uint32_t rb = local_tile, cb = 0;
     if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
+    if constexpr (VIEWS && SINGLE) {
+      c.phase = 0;
+      c.last_block = true;
+      if (prm.row_tiles) {  // tile -> (row, phase, column block): the row's tiles are consecutive, phase by phase
+        rb = local_tile / prm.row_tiles;
+        const uint32_t sub = local_tile - rb * prm.row_tiles;
+        c.phase = sub / CB;
+        cb = sub - c.phase * CB;
+        c.last_block = cb == CB - 1;
+      }
+    }
     const uint32_t rows = CW(prog + DVM_H_ROWS_LO);  // the host rejects more than 2^32 - 1 rows per program
     const uint32_t row = rb * (uint32_t)(THREADS >> c.lgG) + (uint32_t)(tid >> c.lgG);
     const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
@@ -591,6 +606,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
   uint32_t prog_idx = 0;
   uint32_t tile = blockIdx.x + (SINGLE ? prm.tile_begin : 0u);
+  if constexpr (VIEWS && SINGLE) if (prm.row_tiles) tile = blockIdx.x * prm.row_tiles;
   uint32_t iter = 0;
   int red_par = 0;
   int buf = 0;
@@ -662,7 +678,13 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
         }
       }
     }
-    const uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
+    uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
+    if constexpr (VIEWS && SINGLE) {
+      if (prm.row_tiles) {  // the next tile of this row, or the first tile of this CTA's next row
+        next = tile + 1;
+        if (next % prm.row_tiles == 0) next += (gridDim.x - 1) * prm.row_tiles;
+      }
+    }
     ++iter;
     const bool have_next = next < prm.total_tiles;
     uint32_t next_prog_idx = prog_idx;
@@ -822,6 +844,14 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           // inside the warp, shared memory across the warps of a row group ----
           pc += 1;
           const int rop = op & 7;
+          bool accumulate = false;
+          if constexpr (VIEWS && SINGLE) {
+            const uint32_t tag = DVM_INSN_TAG(w0);
+            if (tag) {  // a phased program: the reduction belongs to one phase and runs over that phase's blocks
+              if (tag - 1 != c.phase) break;
+              accumulate = c.col0 != 0;
+            }
+          }
           float v;
           if (rop == DVM_R_SUM || rop == DVM_R_SUMSQ) {
             float2 acc = make_float2(0.f, 0.f);
@@ -877,6 +907,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             else v = ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
             red_par ^= 1;
           }
+          if constexpr (VIEWS && SINGLE) {
+            if (accumulate) {
+              const float prev = s_S[DVM_INSN_A(w0)][tid];
+              v = rop == DVM_R_MAX ? fmaxf(prev, v) : (rop == DVM_R_MIN ? fminf(prev, v) : prev + v);
+            }
+          }
           s_S[DVM_INSN_A(w0)][tid] = v;
         } break;
         case 0: {  // NOP LDG LDS LDA STA LSS STG STS
@@ -900,6 +936,9 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
                                (w >> 2) * PSTRIDE + (w & 3) * 4));
             s_S[ia][tid] = c.ncols > 0 ? v : 0.f;
           } else if (op == DVM_OP_STG) {
+            if constexpr (VIEWS && SINGLE) {
+              if (DVM_INSN_TAG(w0) && DVM_INSN_TAG(w0) - 1 != c.phase) break;  // a phased program stores in its last phase
+            }
             // an output covers the dominant shape: element (row, col) of a dense one lies at row * C + col,
             // the rows of a view (Table 1, ViewStore) lie where its strides put them
             const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
@@ -1068,11 +1107,19 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
               }
             }
           } else if (op == DVM_OP_STS) {
+            bool first_block = c.col0 == 0;  // a row's value is stored once: by the tile of its first column block, or ...
+            if constexpr (VIEWS && SINGLE) {
+              const uint32_t tag = DVM_INSN_TAG(w0);
+              if (tag) {  // ... in a phased program by the last block of the phase that completes it
+                if (tag - 1 != c.phase || !c.last_block) break;
+                first_block = true;
+              }
+            }
             const uint32_t d = opd0 + ib * DVM_OPD_WORDS;
             const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
             char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(d, c) << DVM_DT_LG_ES(dt)));
             const float v = s_S[ia][tid];
-            if (c.ncols > 0 && (tid & (G - 1)) == 0 && c.col0 == 0) {
+            if (c.ncols > 0 && (tid & (G - 1)) == 0 && first_block) {
               if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
               else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p) = v;
               else if (dt == DVM_DT_I32) *reinterpret_cast<uint32_t*>(p) = store_i32(v);
@@ -1089,7 +1136,19 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             pc += 1;
             const float v = s_S[ia][tid];
             DVM_EACH_PAIR A[i] = make_float2(v, v);
+          } else if (op == DVM_OP_PHASE) {
+            pc += 1;
+            if constexpr (VIEWS && SINGLE) {
+              if (ia != 0xff && c.phase < (uint32_t)ia) pc = pc_end;  // the tiles of the earlier phases end here
+            }
           } else if (op == DVM_OP_SOP) {
+            if constexpr (VIEWS && SINGLE) {
+              const uint32_t tag = DVM_INSN_TAG(w0);
+              if (tag && (tag - 1 != c.phase || !c.last_block)) {  // phased: once, when its operands are complete
+                pc += DVM_INSN_LEN(w0);
+                break;
+              }
+            }
             const uint32_t w1 = CW(pc + 1);
             const int sub = w1 & 0xff, s1 = (w1 >> 8) & 0xff, s2 = (w1 >> 16) & 0xff;
             const float x = s_S[s1][tid];

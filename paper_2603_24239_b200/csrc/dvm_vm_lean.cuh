@@ -21,6 +21,10 @@
 #include "dvm_link.h"
 #include "dvm_vm.cuh"
 
+#ifndef DVM_LEAN_MIN_CTAS
+#define DVM_LEAN_MIN_CTAS 2
+#endif
+
 namespace dvm {
 
 __device__ __forceinline__ uint4 lean_lds128(uint32_t addr) {
@@ -150,7 +154,7 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
 }
 
 template <int V, int PW, bool SINGLE, bool HEAVY>
-__global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
+__global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
   constexpr int NG = V / 8;            // 8-slot groups of a tile register

@@ -1,4 +1,4 @@
-"""Edge cases of the interpreter: the longest reducible row, rows one element longer (rejected), long
+"""Edge cases of the interpreter: the longest reducible row, rows one element longer (run in phases), long
 non-reduced rows split into column blocks, one-element rows, and the largest stacked launch."""
 import pytest
 import torch
@@ -29,12 +29,13 @@ def test_longest_reducible_row(cols):
     assert dvm.code_info(code)["threads_per_row"] == 256
 
 
-def test_row_longer_than_capacity_is_rejected():
+def test_row_longer_than_capacity_runs_in_phases():
+    """One column more than a tile holds: the row is walked in column blocks, the mean first, then the difference."""
     prog = _layernorm_like()
-    p = dvm.program_from_nodes(prog.nodes)
-    with pytest.raises(dvm.DvmError) as ei:
-        dvm.encode(p, [(3, 8193)], [1.0 / 8193])
-    assert ei.value.status == -3   # DVM_ERR_UNSUPPORTED
+    x = wl.randn((3, 8193), torch.float32, 11)
+    outs, code = gpu_run(prog, [x], [1.0 / 8193])
+    assert "phases    2" in dvm.disassemble(code)
+    check(prog, outs, oracle_run(prog, [x], [1.0 / 8193]))
 
 
 @pytest.mark.parametrize("rows,cols", [(3, 20000), (2, 65537), (1, 100001)])

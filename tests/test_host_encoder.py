@@ -98,10 +98,18 @@ def test_encode_errors():
     with pytest.raises(dvm.DvmError) as e:
         dvm.encode(p, [(7, 5), (7, 5)])
     assert e.value.status == -1
-    # a reduced row longer than the register budget
+    # a reduced row longer than a tile runs in phases; nine reductions that each need the one before would
+    # need nine phases and nine per-row scalars that outlive their tiles: more than the machine holds
     q = dvm.program_from_nodes(wl.program_layernorm().nodes)
+    assert dvm.verify(dvm.encode(q, [(4, 17000)], (1 / 17000,))) == 0
+    deep = wl.OpProgram("deep")
+    v = deep.input("f32", 2)
+    for _ in range(9):
+        v = deep.binary("sub", v, deep.reduce("max", v))
+    deep.output(v, "f32")
+    assert dvm.verify(dvm.encode(dvm.program_from_nodes(deep.nodes), [(4, 8000)])) == 0
     with pytest.raises(dvm.DvmError) as e:
-        dvm.encode(q, [(4, 17000)], (1 / 17000,))
+        dvm.encode(dvm.program_from_nodes(deep.nodes), [(4, 17000)])
     assert e.value.status == -3
     # missing runtime scalar
     with pytest.raises(dvm.DvmError):
