@@ -1201,6 +1201,9 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
     g.V = kVs[vi];
     if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
     if (g.V == 24 && !plain && g_elems_per_thread != 24) continue;
+    // a phased program walks a row P times: the fewest, largest column blocks keep the per-tile overhead and the
+    // ragged last block small (8200 columns: 2 blocks of 4104 instead of 3 of 4096 / 4096 / 8)
+    if (e.phased && g.V != 32 && !g_elems_per_thread) continue;
     g.W = W0;
     if (flat) {
       g.log2G = 8;
@@ -1256,6 +1259,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
         ct = ((cap - pad) / w) * w;
         if (ct <= 0) continue;
         if (ct > C) ct = C;
+        if (e.phased) ct = cdiv(cdiv(C, cdiv(C, ct)), w) * w;  // column blocks of even length
       }
       g.log2G = lg;
       g.Ctile = ct;
