@@ -118,8 +118,13 @@ int dvm_program_cast(dvm_program* p, int x, int dtype, int* value_id);
  * combine their rows into the result with atomic operations; dvm_launch first fills that output with the
  * operation's identity (one more small kernel on the stream), and a sum's order of additions is not fixed
  * from run to run (the fp32 result varies in its last bits).  All reductions of one program must name the same axis
- * (dvm_encode: DVM_ERR_UNSUPPORTED otherwise), and the reduced axis must fit the register budget
- * (8192 elements), as a row does. */
+ * (dvm_encode: DVM_ERR_UNSUPPORTED otherwise; the streaming fuser, dvm_fuser_reduce_axis, splits such a chain into
+ * two meta-kernels on consecutive levels).
+ * Length of the reduced axis: up to 8192 elements a row is one tile.  A longer LAST axis is walked in column
+ * blocks, in as many passes as the program has reductions that depend on one another (a softmax: maximum, sum
+ * of exponentials, quotient; at most 8 passes and 8 per-row values, DVM_ERR_UNSUPPORTED beyond): such a program
+ * runs through dvm_launch only, not in a stacked launch.  Another axis than the last that is read back by the
+ * program must fit 8192 elements. */
 int dvm_program_reduce(dvm_program* p, int op, int x, int axis, int* value_id);
 /* The cube operation (Sec. 4.2, matrix operations): a [M,K] x b [K,N], bf16 inputs, fp32 value.
  * Both operands must be program inputs; every matmul of a program shares `a`. */

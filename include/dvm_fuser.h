@@ -52,6 +52,10 @@ int dvm_fuser_unary(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, d
 int dvm_fuser_binary(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 int dvm_fuser_scalar(dvm_fuser* f, int op, int x, float s, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 int dvm_fuser_reduce(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
+/* The same over another axis (axis < 0, counted from the end; -1 is dvm_fuser_reduce).  One meta-kernel reduces over
+ * one axis: an operator that reduces over a second axis, or that reads across the first one's result in another
+ * direction, opens the next group, one level up -- a chain with two reduced axes runs as two stacked levels. */
+int dvm_fuser_reduce_axis(dvm_fuser* f, int op, int x, int axis, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value);
 /* Table 1 Cmp, Select (cond != 0 ? x : y), Cast (the value rounded to `dtype`), and the cube operation a [M,K] x b [K,N]
  * (Sec. 4.2; bf16 operands that lie in memory).  A matmul starts a group of its own; the vector operators that
  * arrive behind it join that group as its epilogue while the group still encodes as one matmul meta-kernel --

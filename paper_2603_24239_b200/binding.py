@@ -108,6 +108,7 @@ _sig.update({
     "dvm_fuser_binary": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_scalar": ([_vp, _i, _i, C.c_float, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_reduce": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_fuser_reduce_axis": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_compare": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_select": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_cast": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
@@ -522,7 +523,9 @@ class Fuser:
     def scalar(self, op, x, s, out_shape, dtype="f32"):
         return self._op(lib.dvm_fuser_scalar, (SCALAR.get(op, op), x, float(s)), out_shape, dtype)
 
-    def reduce(self, op, x, out_shape, dtype="f32"):
+    def reduce(self, op, x, out_shape, dtype="f32", axis=-1):
+        if axis != -1:
+            return self._op(lib.dvm_fuser_reduce_axis, (REDUCE.get(op, op), x, axis), out_shape, dtype)
         return self._op(lib.dvm_fuser_reduce, (REDUCE.get(op, op), x), out_shape, dtype)
 
     def compare(self, op, x, y, out_shape, dtype="f32"):

@@ -122,7 +122,7 @@ int build(const dvm_fuser* f, const std::vector<int>& op_list, const FOp* extra,
       case OP_SELECT: st = dvm_program_select(b->prog, px, py, pz, &pid); break;
       case OP_CAST: st = dvm_program_cast(b->prog, px, o.op, &pid); break;
       case OP_MATMUL: st = dvm_program_matmul(b->prog, px, py, &pid); break;
-      default: st = dvm_program_reduce(b->prog, o.op, px, -1, &pid); break;
+      default: st = dvm_program_reduce(b->prog, o.op, px, o.y, &pid); break;  // (OP_REDUCE: y is the axis)
     }
     if (st == DVM_OK) ids.push_back({o.out, pid});
   }
@@ -297,6 +297,11 @@ extern "C" int dvm_fuser_scalar(dvm_fuser* f, int op, int x, float s, int out_dt
 }
 extern "C" int dvm_fuser_reduce(dvm_fuser* f, int op, int x, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
   FOp o = {OP_REDUCE, op, x, -1, 0.f, -1, -1, -1};
+  return add_op(f, o, out_dtype, out_ptr, out_shape, value);
+}
+extern "C" int dvm_fuser_reduce_axis(dvm_fuser* f, int op, int x, int axis, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {
+  if (axis >= 0) return DVM_ERR_INVALID_ARG;  // counted from the end, like dvm_program_reduce
+  FOp o = {OP_REDUCE, op, x, axis, 0.f, -1, -1, -1};
   return add_op(f, o, out_dtype, out_ptr, out_shape, value);
 }
 extern "C" int dvm_fuser_compare(dvm_fuser* f, int op, int x, int y, int out_dtype, void* out_ptr, dvm_shape* out_shape, int* value) {

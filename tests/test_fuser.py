@@ -261,3 +261,29 @@ def test_matmul_with_streamed_epilogue_matches_oracle_in_one_launch():
     want = _oracle_chain(lambda p, i: [p.matmul(i[0], i[1]), p.unary("exp", i[2])], [x, w, c])
     assert np.max(np.abs(wl.to_f64(f2.tensors[mm]) - want[0])) <= 1e-4 * np.max(np.abs(want[0]))
     _close(f2.tensors[e], want[1])
+
+
+@pytest.mark.gpu
+def test_two_reduced_axes_split_into_two_levels():
+    """A column statistic followed by a row normalisation: one meta-kernel reduces over one axis, so the chain
+    becomes two groups on consecutive levels; both results against the oracle."""
+    a = wl.randn((300, 257), torch.float32, 31).cuda()
+    f = dvm.Fuser()
+    va = f.tensor(a)
+    cm = f.reduce("max", f.unary("abs", va, a.shape), (1, 257), axis=-2)      # column maxima of |a|
+    sc = f.binary("div", va, cm, a.shape)                                     # a scaled column by column
+    rs = f.reduce("sum", f.binary("mul", sc, sc, a.shape), (300, 1))          # row sums of squares
+    out = f.binary("div", sc, f.unary("sqrt", rs, (300, 1)), a.shape)
+    ops, groups = f.pending()
+    assert ops == 7 and groups >= 2
+    f.flush()
+    torch.cuda.synchronize()
+    assert dvm.last_device_status() == 0
+    def chain(p, i):
+        pc = p.reduce("max", p.unary("abs", i[0]), axis=-2)
+        ps = p.binary("div", i[0], pc)
+        pr = p.reduce("sum", p.binary("mul", ps, ps))
+        return [pc, p.binary("div", ps, p.unary("sqrt", pr))]
+    want = _oracle_chain(chain, [a])
+    assert np.array_equal(wl.to_f64(f.tensors[cm]), want[0])                  # |x| and max are exact
+    _close(f.tensors[out], want[1])
