@@ -844,7 +844,15 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     break;
               switch (u) {
                 DVM_MM_UN(DVM_U_EXP) DVM_MM_UN(DVM_U_SQRT) DVM_MM_UN(DVM_U_RSQRT) DVM_MM_UN(DVM_U_ABS)
-                DVM_MM_UN(DVM_U_LOG) DVM_MM_UN(DVM_U_ERF) DVM_MM_UN(DVM_U_NEG) DVM_MM_UN(DVM_U_RECIP)
+                DVM_MM_UN(DVM_U_LOG) DVM_MM_UN(DVM_U_NEG) DVM_MM_UN(DVM_U_RECIP)
+                case DVM_U_ERF:  // on pairs: half as many polynomial chains as element by element
+#pragma unroll
+                  for (int i = 0; i < CHUNK; i += 2) {
+                    const float2 r = packed_erf(make_float2(acc[i], acc[i + 1]));
+                    acc[i] = r.x;
+                    acc[i + 1] = r.y;
+                  }
+                  break;
                 DVM_MM_UN(DVM_U_FLOOR) DVM_MM_UN(DVM_U_ROUND) DVM_MM_UN(DVM_U_TANH)
                 default:
 #pragma unroll
