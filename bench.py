@@ -7,9 +7,10 @@ dvm_launch_stacked); nothing is cached between instances.  The default
 workload is the fused residual-add + RMSNorm sweep (200 instances, bf16
 [B*S, 4096], B in 1..32, S in 1..8192).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5|addmm|ifelse] [--impl dvm|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5|addmm|ifelse|views] [--impl dvm|reference]
 
-Prints one JSON line (rank 0).  `value` is algorithmic GB/s of the whole job
+Prints one JSON line (rank 0).  The default run (c2) also measures every other workload briefly and reports
+them under `configs` (throughput, roofline fraction, launches; --no-configs leaves that out).  `value` is algorithmic GB/s of the whole job
 with inputs resident in HBM; `e2e` is the same metric through dvm_run_host
 with pinned HOST buffers (copies inside the timed region); `roofline` is the
 interpreter kernel's algorithmic bytes over its CUDA-event time against the
@@ -761,6 +762,8 @@ WORKLOADS = {"views": ViewsWorkload, "ifelse": IfElseWorkload, "addmm": AddmmWor
 for _W in (C1Workload, C2Workload, C3Workload, C4Workload, IfElseWorkload, ViewsWorkload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
+for _W in (C1Workload, C2Workload, C3Workload):   # one basic program per launch: the lean interpreter runs it
+    _W.kernel = "dvm_vm_lean_kernel"
 
 
 def oracle_threads(workload: str) -> int:
@@ -1313,7 +1316,7 @@ def main():
         del W
         torch.cuda.empty_cache()
         cfgs = {}
-        for name, steps in (("c1", 50), ("c3", 2), ("c4", 2), ("c5", 2), ("addmm", 1), ("ifelse", 1), ("views", 1)):
+        for name, steps in (("c1", 50), ("c3", 2), ("c4", 2), ("c5", 2), ("addmm", 2), ("ifelse", 2), ("views", 2)):
             if name == name_main:
                 continue
             try:
