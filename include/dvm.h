@@ -253,8 +253,8 @@ int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_t
 int dvm_launch_stacked(int n_programs, const void* const* codes, const size_t* code_sizes,
                        void* const* const* tensors, const int* n_tensors, void* cuda_stream);
 
-/* Temporal stacking of DEPENDENT meta-kernels (Sec. 5.1: tiles of different operators run one after the
- * other on the same core, which "does not require operators to be independent").  As dvm_launch_stacked,
+/* Temporal stacking of DEPENDENT meta-kernels (Sec. 5.1: stacking in time puts tiles of different operators
+ * one after the other on a core, so it also covers operators that depend on one another).  As dvm_launch_stacked,
  * plus level[n_programs] (host): a program may read tensors that programs of LOWER levels of the same call
  * write; programs of one level must be independent of one another.  Levels must be non-decreasing in i
  * (DVM_ERR_INVALID_ARG otherwise): the work queue hands tiles out in that order.  Inside the kernel a tile
