@@ -76,9 +76,15 @@ enum {
   DVM_LM_BCAST = 3,    // row-vector input, the same for every row and tile: one row image per slot, loaded once per
                        // slot and program
   DVM_LM_BCAST_TILE = 4, // the same with several column blocks: the image holds the tile's column block, loaded with every tile
-  DVM_LM_GATHER = 5    // input whose columns are not adjacent in memory (Table 1, ViewLoad): every thread fetches its own
+  DVM_LM_GATHER = 5,   // input whose columns are not adjacent in memory (Table 1, ViewLoad): every thread fetches its own
                        // elements, widened to fp32, into the thread-private layout of a temporary (extended variant)
+  DVM_LM_TRANSPOSED = 6 // such an input whose ROWS are adjacent in memory (a transposed matrix): the tile's part of every column
+                       // is one contiguous strip -- one bulk copy per column into strip images DVM_STRIP_PITCH apart; a thread
+                       // reads its row's element of each of its columns from the strips (raw element type; the instructions
+                       // that read the register say fp32, as for a gathered one)
 };
+// bytes between the strip images of a TRANSPOSED register (R rows of the tile; alignment slack on both sides)
+#define DVM_STRIP_PITCH(R, es) ((uint32_t)(R) * (uint32_t)(es) + 32u)
 // bytes between the row images of a ROWS register (room for the 16-byte alignment slack on both sides)
 #define DVM_ROW_PITCH(G, V, es) ((uint32_t)(G) * (uint32_t)(V) * (uint32_t)(es) + 32u)
 

@@ -1150,12 +1150,19 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
         if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
         if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
       }
-      const int mode = gather ? DVM_LM_GATHER
+      // a gathered operand whose rows are adjacent in memory (a transposed matrix): with few threads per row the
+      // tile's part of a column is a contiguous strip of 256 / G elements -- copied in bulk, one strip per column
+      bool transposed = gather && !flat && !e.phased && od.ostride[0] == 1 && (od.cs * es) % 16 == 0 &&
+                        Gthreads * g.V <= T && ((T / Gthreads) * es) % 16 == 0;
+      for (int q = 1; q < 3 && transposed; ++q)
+        if (outer[q] > 1 && ((od.ostride[q] * es) % 16 != 0 || outer[0] % (T / Gthreads) != 0)) transposed = false;
+      const int mode = transposed ? DVM_LM_TRANSPOSED : gather ? DVM_LM_GATHER
                               : (inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS));
       if (inv && !gather) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
       const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
       // a gathered register holds fp32 values in the thread-private layout of a temporary
-      const int64_t bytes = gather ? (int64_t)g.V * 4 * T : (inv ? pitch : pitch * (T / Gthreads));
+      const int64_t bytes = transposed ? g.Ctile * (int64_t)DVM_STRIP_PITCH(T / Gthreads, es)
+                                       : gather ? (int64_t)g.V * 4 * T : (inv ? pitch : pitch * (T / Gthreads));
       g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
       g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
     }
@@ -1344,7 +1351,8 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   for (int k = 0; k < e.n_in_regs; ++k)
     if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
   for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the views variant
-    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER) flags |= DVM_F_LOADS_BY_ROW | DVM_F_VIEWS;
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER || ((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_TRANSPOSED)
+      flags |= DVM_F_LOADS_BY_ROW | DVM_F_VIEWS;
 
   // ---- 7. assemble ----
   const int n_tensors = n_in + p->n_outputs;
@@ -1625,6 +1633,19 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
     } else if (mode == DVM_LM_GATHER) {
       if (od >= n_opd || dt != DVM_DT_F32 || !((w[DVM_H_GEOM] >> 24) & DVM_F_VIEWS)) return false;
       need = (uint64_t)Vv * 4 * DVM_VM_THREADS / DVM_LOCAL_UNIT;
+    } else if (mode == DVM_LM_TRANSPOSED) {
+      // one strip per column of the column block, each holding the tile's rows: at most one strip per thread,
+      // strips and column stride in whole 16-byte units, rows adjacent in memory
+      if (od >= n_opd || dt != DVM_DT_F32 || !((w[DVM_H_GEOM] >> 24) & DVM_F_VIEWS)) return false;
+      const uint32_t* d = otab + od * DVM_OPD_WORDS;
+      const uint64_t es = 1ull << DVM_DT_LG_ES((d[0] >> 8) & 0xff), Rt = DVM_VM_THREADS >> lg;
+      if (((uint64_t)Vv << lg) > DVM_VM_THREADS || (Rt * es) % 16 || ((uint64_t)d[DVM_OPD_COLSTRIDE] * es) % 16 || d[DVM_OPD_STRIDE0] != 1 ||
+          (w[DVM_H_GEOM] >> 24) & DVM_F_FLAT)
+        return false;
+      if ((w[DVM_H_OUTER1] > 1 || w[DVM_H_OUTER2] > 1) &&
+          (((uint64_t)d[DVM_OPD_STRIDE1] * es) % 16 || ((uint64_t)d[DVM_OPD_STRIDE2] * es) % 16 || w[DVM_H_OUTER0] % Rt))
+        return false;
+      need = ((uint64_t)w[DVM_H_COL_TILE] * DVM_STRIP_PITCH(Rt, es) + DVM_LOCAL_UNIT - 1) / DVM_LOCAL_UNIT;
     } else {
       if (mode < DVM_LM_BLOCK || mode > DVM_LM_BCAST_TILE || od >= n_opd) return false;
       if (mode == DVM_LM_BCAST && w[DVM_H_COL_BLOCKS] > 1) return false;  // a once-per-program image holds whole rows
@@ -1705,7 +1726,8 @@ extern "C" int dvm_verify(const void* code, size_t code_size) {
       uint32_t info = ot[bb * DVM_OPD_WORDS];
       if (op == DVM_OP_LDG) {
         if ((a & 0x7f) >= n_inr) return DVM_ERR_BAD_CODE;
-        const bool gathered = ((lt[a & 0x7f] >> 16) & 0xff) == DVM_LM_GATHER;  // widened to fp32 on the way in
+        const uint32_t lmode = (lt[a & 0x7f] >> 16) & 0xff;
+        const bool gathered = lmode == DVM_LM_GATHER || lmode == DVM_LM_TRANSPOSED;  // read as fp32 by the instructions
         if (!lreg_ok(a & 0x7f, (!gathered && ((info >> 8) & 0xff) == DVM_DT_BF16) ? u_bf16 : u_f32)) return DVM_ERR_BAD_CODE;
         if (gathered != (ot[bb * DVM_OPD_WORDS + DVM_OPD_COLSTRIDE] != 1)) return DVM_ERR_BAD_CODE;
       }

@@ -434,6 +434,21 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           const int ov = (shift > 0 && t == 0) ? c.ncols + shift - (V << c.lgG) : 0;
           vm_gather(reinterpret_cast<const char*>(tensor_ptr(prog, d)) + (r0 << lg_es), cs << lg_es, (int)lg_es,
                     dst + (uint32_t)tid * 16, (t << c.lgW) - shift, c.lgW, c.lgG, ov > 0 ? (V << c.lgG) : 0, c.ncols, V);
+        } else if (VIEWS && mode == DVM_LM_TRANSPOSED) {
+          // a transposed operand: thread j copies column j of the tile's column block -- the tile's rows of that
+          // column are adjacent in memory (row stride 1), one strip of up to 256 / G elements
+          const uint32_t rows = CW(prog + DVM_H_ROWS_LO);
+          const uint32_t R = (uint32_t)(THREADS >> c.lgG);
+          const uint32_t row0 = c.row - (uint32_t)(tid >> c.lgG);  // the tile's first row
+          const uint32_t ncol_t = min(CW(prog + DVM_H_COLS) - c.col0, CW(prog + DVM_H_COL_TILE));
+          if ((uint32_t)tid < ncol_t && row0 < rows) {
+            mine = true;
+            TileCtx c0 = c;
+            c0.row = row0;
+            a = row_offset(d, c0) - c.col0 + (unsigned long long)(c.col0 + (uint32_t)tid) * CW(d + DVM_OPD_COLSTRIDE);
+            n_el = min(R, rows - row0);
+            dst += (uint32_t)tid * DVM_STRIP_PITCH(R, 1u << lg_es);
+          }
         } else if (mode == DVM_LM_BLOCK) {
           if (tid == 0) {  // thread 0's row is the tile's first row: the whole tile is one byte range from there
             mine = true;
@@ -491,12 +506,31 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
 
   // Where this thread's part of local register k (element type dt) lies in tile slot `buf`:
   // 16-byte vector u is at  (u & 1 ? a1 : a) + (u >> 1) * vA ;  mis != 0: the vectors are not 16-byte aligned.
-  struct RegView { uint32_t a, a1, vA, mis; bool image; };
+  // tr_pitch != 0: a TRANSPOSED register -- the element of column col lies at a + col * tr_pitch (raw type: tr_bf16).
+  struct RegView { uint32_t a, a1, vA, mis; bool image; uint32_t tr_pitch; bool tr_bf16; };
   auto reg_view = [&](const TileCtx& c, uint32_t prog, uint32_t opd0, uint32_t lreg0, int k, int dt, int buf) -> RegView {
     RegView r;
     const uint32_t lw = CW(lreg0 + k);
     const uint32_t mode = (lw >> 16) & 0xf;
     uint32_t a = slot_base(buf) + (lw & 0xffffu) * DVM_LOCAL_UNIT;
+    r.tr_pitch = 0;
+    r.tr_bf16 = false;
+    if constexpr (VIEWS) {
+      if (mode == DVM_LM_TRANSPOSED) {
+        const uint32_t raw_dt = (CW(opd0 + (lw >> 24) * DVM_OPD_WORDS + DVM_OPD_INFO) >> 8) & 0xff;
+        const uint32_t lg_raw = raw_dt == DVM_DT_BF16 ? 1u : 2u;
+        // every strip starts on the same phase of a 16-byte word as the tensor itself (column stride, strip length
+        // and outer strides are whole 16-byte units): the address modulo 16 patched in at launch
+        r.a = a + ((lw >> 20) & 0xfu) + ((uint32_t)(tid >> c.lgG) << lg_raw);
+        r.a1 = r.a;
+        r.vA = 0;
+        r.mis = 0;
+        r.image = false;
+        r.tr_pitch = DVM_STRIP_PITCH(THREADS >> c.lgG, 1u << lg_raw);
+        r.tr_bf16 = raw_dt == DVM_DT_BF16;
+        return r;
+      }
+    }
     if (mode == DVM_LM_PRIVATE || (VIEWS && mode == DVM_LM_GATHER)) {
       r.a = a + (uint32_t)tid * 16;
       r.a1 = r.a + PSTRIDE;
@@ -554,6 +588,31 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
   // D = L[k] widened to fp32: the whole tile register of this thread.  One warp-uniform branch picks the
   // variant (element type; aligned vectors or realigned ones); each variant is straight-line code.
   auto load_reg = [&](float2 (&D)[VP], const TileCtx& c, const RegView& r, int dt) {
+    if constexpr (VIEWS) {
+      if (r.tr_pitch) {
+        // transposed strips: slot s holds column cbase + chunk offset (wrapped / clamped like a gathered slot:
+        // slots outside the row read some strip of the image and are masked by their consumers)
+        const int wrapcap = c.ov > 0 ? (V << c.lgG) : 0;
+        const int last = max((int)CW((SINGLE ? kSingleProg : c.prog) + DVM_H_COL_TILE) - 1, 0);
+#pragma unroll
+        for (int sl = 0; sl < V; ++sl) {
+          int col = c.cbase + ((sl >> c.lgW) << (c.lgG + c.lgW)) + (sl & ((1 << c.lgW) - 1));
+          if (col < 0) col += wrapcap;
+          col = min(max(col, 0), last);
+          const uint32_t addr = r.a + (uint32_t)col * r.tr_pitch;
+          float v;
+          if (r.tr_bf16) {
+            unsigned short h;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+            v = __uint_as_float((uint32_t)h << 16);
+          } else {
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+          }
+          if (sl & 1) D[sl >> 1].y = v; else D[sl >> 1].x = v;
+        }
+        return;
+      }
+    }
     const bool slow = __any_sync(0xffffffffu, r.mis != 0 || (c.ov > 0 && r.image));
     if (dt == DVM_DT_BF16) {
       if (!slow) {

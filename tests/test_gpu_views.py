@@ -182,3 +182,50 @@ def test_last_two_dims_swapped_in_a_4d_view():
     y = wl.randn((B * H * S * D,), torch.float32, 22)
     shape = (B, H, S, D)
     _run(_axpy("f32", 4), [(x, 0, shape, (H * D * S, D * S, 1, S)), (y, 0, shape, _dense(shape))], [(B * H * S * D, 0, _dense(shape), "f32")])
+
+
+def _mode_of(code, reg):
+    """Layout mode of input register `reg` (local register table of the encoded program)."""
+    w = np.frombuffer(code.bytes(), dtype=np.uint32)
+    counts = int(w[5])
+    lt = 20 + 2 * (counts & 0xff) + 8 * ((counts >> 16) & 0xff)
+    return (int(w[lt + reg]) >> 16) & 0xf
+
+
+@pytest.mark.parametrize("dt,rows,cols,ld,offset", [
+    ("bf16", 1000, 777, 1000, 0),      # ragged last row block and column block
+    ("bf16", 4096, 512, 4104, 0),      # padded leading dimension (a multiple of 8 elements)
+    ("bf16", 640, 300, 640, 3),        # view starts 6 bytes into a 16-byte word: the strips keep that phase
+    ("f32", 513, 129, 516, 0),
+    ("f32", 2048, 64, 2048, 1),
+])
+def test_transposed_input_goes_through_strips(dt, rows, cols, ld, offset):
+    """x given as the transpose of a [cols, ld] storage (rows adjacent in memory, column stride ld): the tile's
+    part of every column is copied as one strip (layout mode 6), not gathered element by element."""
+    prog = _axpy(dt, 2)
+    tdt = TORCH_DT[dt]
+    xs = wl.randn((cols * ld + offset + 8,), tdt, 41)
+    ys = wl.randn((rows * cols,), tdt, 42)
+    hp = dvm.program_from_nodes(prog.nodes)
+    code = dvm.encode(hp, [(rows, cols), (rows, cols)], in_strides=[[1, ld], [cols, 1]], out_strides=[[cols, 1]])
+    assert _mode_of(code, 0) == 6
+    _run(prog, [(xs, offset, (rows, cols), (1, ld)), (ys, 0, (rows, cols), (cols, 1))], [(rows * cols, 0, (cols, 1), dt)])
+
+
+def test_transposed_batched_and_odd_strides_fall_back():
+    """Batched transposes [B, rows, cols] of [B, cols, rows] storage take the strips when the rows per tile divide
+    the row count; a column stride that is not a whole number of 16-byte units takes the element gather."""
+    prog = _axpy("bf16", 3)
+    B, rows, cols = 3, 256, 200
+    xs = wl.randn((B * cols * rows,), torch.bfloat16, 43)
+    ys = wl.randn((B * rows * cols,), torch.bfloat16, 44)
+    _run(prog, [(xs, 0, (B, rows, cols), (cols * rows, 1, rows)), (ys, 0, (B, rows, cols), (rows * cols, cols, 1))],
+         [(B * rows * cols, 0, (rows * cols, cols, 1), "bf16")])
+    prog2 = _axpy("bf16", 2)
+    rows, cols, ld = 300, 100, 301                      # 602 bytes between columns
+    xs = wl.randn((cols * ld,), torch.bfloat16, 45)
+    ys = wl.randn((rows * cols,), torch.bfloat16, 46)
+    hp = dvm.program_from_nodes(prog2.nodes)
+    code = dvm.encode(hp, [(rows, cols), (rows, cols)], in_strides=[[1, ld], [cols, 1]], out_strides=[[cols, 1]])
+    assert _mode_of(code, 0) == 5
+    _run(prog2, [(xs, 0, (rows, cols), (1, ld)), (ys, 0, (rows, cols), (cols, 1))], [(rows * cols, 0, (cols, 1), "bf16")])
