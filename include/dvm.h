@@ -316,6 +316,19 @@ int dvm_disassemble(const void* code, size_t code_size, char* buf, size_t cap);
 /* Header fields of an encoded program (each output may be NULL). */
 int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t* n_tiles,
                   int* code_body_bytes, int* threads_per_row, int* vector_width, int* n_tile_regs);
+/* The bytes of every tensor slot that a launch of `code` reads or writes, counted from the pointer given at launch
+ * (inputs first, then outputs): bytes_needed[i] = 1 + the largest byte offset the program addresses in slot i, 0 for
+ * a slot nothing addresses or an empty program.  Host only.  (Tile loads fetch whole 16-byte units: a launch may
+ * READ up to 15 bytes on either side of an input's range, inside the same 16-byte aligned units.) */
+int dvm_tensor_extents(const void* code, size_t code_size, int64_t* bytes_needed, int n_tensors);
+/* dvm_launch behind a bounds check: DVM_ERR_BUFFER_TOO_SMALL when some tensor_bytes[i] (host array) is below what
+ * dvm_tensor_extents reports, before anything is launched.
+ * Debug mode: with the environment variable DVM_DEBUG=1 every launch of this library (checked or not) runs on the
+ * general interpreter with its device-side checks on (register, operand and tensor-slot indices and instruction
+ * lengths of every decoded instruction; a failed check sets the status word instead of touching memory),
+ * synchronises the stream and returns the device status (DVM_ERR_DEVICE_*) as its own. */
+int dvm_launch_checked(const void* code, size_t code_size, void* const* tensors, const size_t* tensor_bytes,
+                       int n_tensors, void* cuda_stream);
 /* Self-test of the bounded device-side waits (no counterpart in the paper): launches one CTA that waits on
  * an mbarrier nobody completes, with the very wait routine of the interpreter (which = 0) or of the matmul
  * kernel (which = 1), or on a tile counter nobody advances with the level wait of dvm_launch_stacked_levels

@@ -108,6 +108,8 @@ _sig.update({
     "dvm_fuser_binary": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_scalar": ([_vp, _i, _i, C.c_float, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_reduce": ([_vp, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
+    "dvm_tensor_extents": ([_vp, C.c_size_t, C.POINTER(C.c_int64), _i], _i),
+    "dvm_launch_checked": ([_vp, C.c_size_t, C.POINTER(_vp), C.POINTER(C.c_size_t), _i, _vp], _i),
     "dvm_fuser_reduce_axis": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_compare": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
     "dvm_fuser_select": ([_vp, _i, _i, _i, _i, _vp, C.POINTER(Shape), _pi], _i),
@@ -400,6 +402,26 @@ def launch(code: Code, tensors: Sequence, stream=None):
     """dvm_launch: tensors are device tensors (or raw device addresses), inputs then outputs."""
     arr = (_vp * len(tensors))(*[_ptr(t) for t in tensors])
     _check(lib.dvm_launch(code.buf, code.size, arr, len(tensors), _stream(stream)), "dvm_launch")
+
+
+def tensor_extents(code: Code) -> List[int]:
+    """dvm_tensor_extents: bytes of every tensor slot (inputs, then outputs) a launch of `code` addresses."""
+    n = 0
+    out = (C.c_int64 * 16)()
+    for n in range(17):   # the slot count is part of the code: ask until it matches
+        st = lib.dvm_tensor_extents(code.buf, code.size, out, n)
+        if st == 0:
+            return [int(out[i]) for i in range(n)]
+        if st != -1:
+            _check(st, "dvm_tensor_extents")
+    raise DvmError(-1, "dvm_tensor_extents")
+
+
+def launch_checked(code: Code, tensors: Sequence, tensor_bytes: Sequence[int], stream=None):
+    """dvm_launch_checked: dvm_launch behind a bounds check of every tensor against the bytes the program addresses."""
+    arr = (_vp * len(tensors))(*[_ptr(t) for t in tensors])
+    sizes = (C.c_size_t * len(tensor_bytes))(*[int(b) for b in tensor_bytes])
+    _check(lib.dvm_launch_checked(code.buf, code.size, arr, sizes, len(tensors), _stream(stream)), "dvm_launch_checked")
 
 
 def launch_stacked(codes: Sequence[Code], tensor_lists: Sequence[Sequence], stream=None, noalloc: bool = False,

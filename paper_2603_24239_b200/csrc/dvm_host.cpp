@@ -961,7 +961,7 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
   // ---- 2. classes: a value whose last dim is 1 while the dominant last dim is not is a per-row scalar ----
   int Dt = D;  // trailing size-1 dominant dims carry no extent: drop them
   while (Dt > 1 && e.Sd[Dt - 1] == 1) --Dt;
-  const int64_t Ccols = empty ? 1 : e.Sd[Dt - 1];
+  const int64_t Ccols = e.Sd[Dt - 1] == 0 ? 1 : e.Sd[Dt - 1];  // (an instance without rows keeps its row length: classes as usual)
   bool has_reduce = false;
   for (int i = 0; i < NN; ++i) {
     const Node& n = p->nodes[i];
@@ -1888,6 +1888,55 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
     pc += len;
   }
   return o.overflow ? DVM_ERR_BUFFER_TOO_SMALL : DVM_OK;
+}
+
+extern "C" int dvm_tensor_extents(const void* code, size_t code_size, int64_t* bytes_needed, int n_tensors) {
+  if (!bytes_needed) return DVM_ERR_INVALID_ARG;
+  int st = dvm_verify(code, code_size);
+  if (st != DVM_OK) return st;
+  const uint32_t* w = (const uint32_t*)code;
+  const uint32_t counts = w[DVM_H_COUNTS];
+  const uint32_t nt = counts & 0xff, n_opd = (counts >> 16) & 0xff;
+  if ((uint32_t)n_tensors != nt) return DVM_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < nt; ++i) bytes_needed[i] = 0;
+  if (w[DVM_H_N_TILES] == 0) return DVM_OK;
+  auto need = [&](uint32_t slot, uint64_t last_element, uint32_t dt) {
+    const int64_t b = (int64_t)((last_element + 1) << DVM_DT_LG_ES(dt));
+    if (slot < nt && b > bytes_needed[slot]) bytes_needed[slot] = b;
+  };
+  if (w[DVM_H_KERNEL_TYPE] == DVM_KERNEL_MATMUL) {
+    // A [M,K] and the B matrices [K,N] are dense bf16; epilogue operands are [M,N], [1,N] or [M,1] with a row stride
+    const uint32_t* x = w + DVM_HDR_WORDS + 2 * nt;
+    const uint64_t M = x[DVM_MM_M], N = x[DVM_MM_N], K = x[DVM_MM_K];
+    need(x[DVM_MM_SLOTS] & 0xff, M * K - 1, DVM_DT_BF16);
+    need((x[DVM_MM_SLOTS] >> 8) & 0xff, K * N - 1, DVM_DT_BF16);
+    need((x[DVM_MM_SLOTS] >> 16) & 0xff, K * N - 1, DVM_DT_BF16);
+    const uint32_t* ot = x + DVM_MM_WORDS;
+    for (uint32_t o = 0; o < n_opd; ++o) {
+      const uint32_t* d = ot + o * DVM_OPD_WORDS;
+      const uint64_t rs = d[DVM_OPD_STRIDE0], cs = (d[DVM_OPD_INFO] >> 16) & 0xff;
+      need(d[DVM_OPD_INFO] & 0xff, (M - 1) * rs + (N - 1) * cs, (d[DVM_OPD_INFO] >> 8) & 0xff);
+    }
+    return DVM_OK;
+  }
+  // vector programs: element (i2, i1, i0, col) of an operand lies at the sum of index x stride; the last row of a
+  // flat program is shorter
+  const uint32_t* ot = w + DVM_HDR_WORDS + 2 * nt;
+  const uint64_t outer[3] = {w[DVM_H_OUTER0], w[DVM_H_OUTER1], w[DVM_H_OUTER2]};
+  const uint64_t last_cols = w[DVM_H_LAST_ROW_COLS];
+  for (uint32_t o = 0; o < n_opd; ++o) {
+    const uint32_t* d = ot + o * DVM_OPD_WORDS;
+    const uint32_t info = d[DVM_OPD_INFO];
+    if ((info >> 26) & 3) {  // a combined result: dense, its element count in the descriptor
+      need(info & 0xff, (uint64_t)d[DVM_OPD_FILL] - 1, DVM_DT_F32);
+      continue;
+    }
+    uint64_t last = 0;
+    for (int q = 0; q < 3; ++q) last += (outer[q] ? outer[q] - 1 : 0) * (uint64_t)d[DVM_OPD_STRIDE0 + 2 * q];
+    if ((info >> 16) & 0xff) last += (last_cols - 1) * (uint64_t)d[DVM_OPD_COLSTRIDE];
+    need(info & 0xff, last, (info >> 8) & 0xff);
+  }
+  return DVM_OK;
 }
 
 extern "C" int dvm_code_info(const void* code, size_t code_size, int* kernel_type, int64_t* n_tiles,

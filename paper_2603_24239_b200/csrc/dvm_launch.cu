@@ -441,6 +441,78 @@ uint32_t program_phases(const uint32_t* w) {
   return w[DVM_H_LOAD_WORDS] < w[DVM_H_CODE_WORDS] ? DVM_PHASES_OF(body[w[DVM_H_LOAD_WORDS]]) : 0u;
 }
 
+// ---- debug mode (environment variable DVM_DEBUG=1) ----
+// Before the interpreter starts, one thread on the DEVICE walks the parameter block as it arrived there: the
+// directory, every program's header, tables and instructions -- tensor pointers present and aligned to their
+// element type, register / operand / tensor-slot indices inside their tables, instruction lengths inside the
+// code body.  A failed check sets the status word (the launch is then not made); nothing is dereferenced.
+bool debug_mode() {
+  static const bool on = getenv("DVM_DEBUG") && atoi(getenv("DVM_DEBUG")) != 0;
+  return on;
+}
+template <int PW>
+__global__ void dvm_debug_check_kernel(const __grid_constant__ dvm::VMParams<PW> prm) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  bool ok = prm.n_programs >= 1 && prm.n_words <= (uint32_t)PW;
+  const uint32_t n = prm.n_programs;
+  for (uint32_t i = 0; ok && i < n; ++i) {
+    const uint32_t at = prm.words[i];
+    if (at + DVM_HDR_WORDS > prm.n_words) { ok = false; break; }
+    const uint32_t* w = prm.words + at;
+    const uint32_t counts = w[DVM_H_COUNTS], geom = w[DVM_H_GEOM];
+    const uint32_t nt = counts & 0xff, n_opd = (counts >> 16) & 0xff, n_lregs = (geom >> 16) & 0xff;
+    const uint32_t body = w[DVM_H_CODE_WORDS], load_words = w[DVM_H_LOAD_WORDS];
+    const uint32_t total = DVM_HDR_WORDS + 2 * nt + DVM_OPD_WORDS * n_opd + n_lregs + body;
+    if (w[DVM_H_MAGIC] != DVM_MAGIC || w[DVM_H_KERNEL_TYPE] != DVM_KERNEL_VEC || total != w[DVM_H_TOTAL_WORDS] ||
+        at + total > prm.n_words || nt > DVM_MAX_TENSORS || n_opd > DVM_MAX_OPERANDS || n_lregs > DVM_MAX_LREGS || load_words > body) {
+      ok = false;
+      break;
+    }
+    const uint32_t* ot = w + DVM_HDR_WORDS + 2 * nt;
+    const uint32_t* lt = ot + n_opd * DVM_OPD_WORDS;
+    const uint32_t* code = lt + n_lregs;
+    for (uint32_t o = 0; ok && o < n_opd; ++o) {
+      const uint32_t info = ot[o * DVM_OPD_WORDS], slot = info & 0xff, dt = (info >> 8) & 0xff;
+      if (slot >= nt || dt > DVM_DT_I32) { ok = false; break; }
+      const unsigned long long p = ((unsigned long long)w[DVM_HDR_WORDS + 2 * slot + 1] << 32) | w[DVM_HDR_WORDS + 2 * slot];
+      if (p == 0 || (p & ((1ull << DVM_DT_LG_ES(dt)) - 1))) ok = false;
+    }
+    for (uint32_t k = 0; ok && k < (w[DVM_H_LOCAL] & 0xff); ++k)
+      if (k >= n_lregs || (lt[k] >> 24) >= n_opd) ok = false;
+    for (uint32_t pc = 0; ok && pc < body;) {
+      const uint32_t w0 = code[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0), a = DVM_INSN_A(w0), b = DVM_INSN_B(w0);
+      if (len == 0 || pc + len > body || op >= DVM_OP_LAST) { ok = false; break; }
+      if (op == DVM_OP_LDG && ((a & 0x7f) >= n_lregs || b >= n_opd)) ok = false;
+      if ((op == DVM_OP_STG || op == DVM_OP_LDS || op == DVM_OP_STS) && b >= n_opd) ok = false;
+      if ((op == DVM_OP_LDA || op == DVM_OP_STA) && a >= n_lregs) ok = false;
+      if (((op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) || (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP)) &&
+          a != DVM_REG_ACC && a >= n_lregs)
+        ok = false;
+      if (((op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) || (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3)) &&
+          (a >= n_lregs || (b & 0x3f) >= n_lregs))
+        ok = false;
+      if (((op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) || (op >= DVM_OP_RED && op < DVM_OP_RED + DVM_R_NRED) ||
+           op == DVM_OP_BCS || op == DVM_OP_LSS || op == DVM_OP_SOP) && a >= DVM_MAX_SREGS)
+        ok = false;
+      if ((pc < load_words) != (op == DVM_OP_LDG || op == DVM_OP_LDS)) ok = false;
+      pc += len;
+    }
+  }
+  if (!ok) atomicMax(prm.status, (unsigned int)dvm::ST_BAD_CODE);
+}
+
+// Debug mode, before the interpreter launch: the device-side check of the placed block, then a synchronisation; returns
+// the status the device reported (and clears it).
+template <int PW>
+int debug_check(const dvm::VMParams<PW>& P, cudaStream_t stream) {
+  dvm_debug_check_kernel<PW><<<1, 32, 0, stream>>>(P);
+  DVM_CUDA(cudaGetLastError());
+  dvm_count_launch();
+  int status = DVM_OK;
+  const int st = dvm_last_device_status((void*)stream, &status);
+  return st != DVM_OK ? st : status;
+}
+
 static_assert(offsetof(dvm::VMParams<PW_SMALL>, words) % 16 == 0 && offsetof(dvm::VMParams<PW_LARGE>, words) % 16 == 0,
               "linked records are loaded as 16-byte vectors of the parameter space");
 thread_local dvm::VMParams<PW_LARGE> t_large;  // 32 KB, reused by every launch of the thread
@@ -538,6 +610,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   }
   // (launches with a work queue run on the general interpreter unless asked otherwise: measured faster there)
   int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked) && (!queue_asked || g_use_lean >= 2)) ? (g_use_lean ? 1 : 0) : 0;
+  if (debug_mode()) lean = 0;  // the bytecode itself travels to the device, where the check kernel reads it
   uint32_t pos = 0;
   st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, level, true, &pos) : DVM_ERR_UNSUPPORTED;
   if (st == DVM_ERR_UNSUPPORTED) {
@@ -577,12 +650,41 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (!large) {
     dvm::VMParams<PW_SMALL> S;
     memcpy(&S, &P, offsetof(dvm::VMParams<PW_SMALL>, words) + (size_t)pos * 4);
+    if (debug_mode()) {
+      st = debug_check(S, stream);
+      if (st != DVM_OK) return st;
+      st = launch_variant(variant, &S, grid, smem, stream);
+      if (st != DVM_OK) return st;
+      int status = DVM_OK;
+      st = dvm_last_device_status((void*)stream, &status);
+      return st != DVM_OK ? st : status;
+    }
     return launch_variant(variant, &S, grid, smem, stream);
+  }
+  if (debug_mode()) {
+    st = debug_check(P, stream);
+    if (st != DVM_OK) return st;
+    st = launch_variant(variant, &P, grid, smem, stream);
+    if (st != DVM_OK) return st;
+    int status = DVM_OK;
+    st = dvm_last_device_status((void*)stream, &status);
+    return st != DVM_OK ? st : status;
   }
   return launch_variant(variant, &P, grid, smem, stream);
 }
 
 }  // namespace
+
+extern "C" int dvm_launch_checked(const void* code, size_t code_size, void* const* tensors, const size_t* tensor_bytes,
+                                  int n_tensors, void* cuda_stream) {
+  if (!code || !tensors || !tensor_bytes || n_tensors < 0 || n_tensors > DVM_MAX_TENSORS) return DVM_ERR_INVALID_ARG;
+  int64_t need[DVM_MAX_TENSORS];
+  int st = dvm_tensor_extents(code, code_size, need, n_tensors);
+  if (st != DVM_OK) return st;
+  for (int i = 0; i < n_tensors; ++i)
+    if ((int64_t)tensor_bytes[i] < need[i]) return DVM_ERR_BUFFER_TOO_SMALL;
+  return dvm_launch(code, code_size, tensors, n_tensors, cuda_stream);
+}
 
 extern "C" int dvm_launch(const void* code, size_t code_size, void* const* tensors, int n_tensors,
                           void* cuda_stream) {

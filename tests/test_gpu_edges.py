@@ -87,3 +87,24 @@ def test_large_stacked_launch():
         assert ei.value.status == -10   # DVM_ERR_TOO_LARGE
     finally:
         dvm.set_elems_per_thread(0)
+
+
+def test_instance_without_rows_launches_nothing():
+    """[0, 300]: a softmax-like program with a reduction encodes (zero tiles), launches nothing and leaves the
+    (empty) outputs alone; reducing over an EMPTY axis ([300, 0]) is refused."""
+    p = wl.OpProgram("norm")
+    x = p.input("f32", 2)
+    m = p.reduce("max", x)
+    p.output(p.binary("sub", x, m), "f32")
+    p.output(m, "f32")
+    hp = dvm.program_from_nodes(p.nodes)
+    code = dvm.encode(hp, [(0, 300)])
+    assert code.out_shapes == [(0, 300), (0, 1)] and dvm.code_info(code)["n_tiles"] == 0
+    n0 = dvm.launch_count()
+    guard = torch.full((8,), 7.0, device="cuda")
+    dvm.launch(code, [guard, guard, guard])
+    torch.cuda.synchronize()
+    assert dvm.launch_count() == n0 and torch.all(guard == 7.0)
+    with pytest.raises(dvm.DvmError) as ei:
+        dvm.encode(hp, [(300, 0)])
+    assert ei.value.status == -3
