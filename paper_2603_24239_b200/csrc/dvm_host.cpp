@@ -871,6 +871,340 @@ int dvm_encode_matmul(const dvm_program* p, const dvm_shape* in_shapes, int n_in
 // (the stored view has stride 0 along the reduced axis: all its rows land on one address).
 // `lowered`: the shapes are those of encode_views' axis permutation (rank of the dominant shape, not the
 // inputs' declared ranks); every reduction then runs over the last dim.
+// What steps 1 - 5 of the encoder hand to the shape tiling and to the assembly: the collapsed iteration space and
+// the registers the generated code uses.
+struct Lowered {
+  int64_t C, R, outer[3];        // columns, rows and the (up to three) collapsed outer dims of the dominant shape
+  bool flat, empty, has_reduce;
+  int primary, combine_axis, W, nreg;
+  int in_dtype[DVM_MAX_LREGS], in_opd[DVM_MAX_LREGS];  // element type and operand of every input register
+};
+
+// One candidate of the shape tiling, with the local-memory layout of its tile slot.
+struct Geo {
+  int V, log2G, W, units, scalar_unit;
+  bool one_slot;  // costed for two CTAs per SM that hold ONE tile slot each (see DVM_F_ONE_SLOT)
+  int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
+  uint32_t flags, inv_mask;
+  uint32_t lreg_table[DVM_MAX_LREGS];
+};
+
+// Step 6 of the encoder: the shape tiling.  Leaves the cheapest geometry in `best`.
+static int choose_geometry(const Enc& e, const Lowered& L, Geo& best) {
+  const dvm_program* p = e.p;
+  const int NN = p->n_nodes;
+  const bool flat = L.flat, empty = L.empty, has_reduce = L.has_reduce;
+  const int64_t C = L.C, R = L.R;
+  const int64_t* outer = L.outer;
+  const int W = L.W, primary = L.primary, combine_axis = L.combine_axis, nreg = L.nreg;
+  const int* in_dtype = L.in_dtype;
+  const int* in_opd = L.in_opd;
+  // ---- 6. shape tiling (Sec. 4.2): elements per thread V, threads per row G, column tile, tile count.
+  // Candidates are compared with the paper's cost  ceil(#tiles / N) * (tile + overhead)  in per-thread
+  // element units; N is the number of CTAs resident at once, which the local-memory need decides.
+  const int T = DVM_VM_THREADS;
+  const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
+  Geo tight;  // the best geometry among those that leave room for g_min_resident_ctas CTAs per SM
+  best.cost = -1;
+  tight.cost = -1;
+  // Local-memory layout of ONE tile slot, in 256-byte units, for a candidate geometry; returns the CTAs per SM
+  // it leaves room for (0: it does not fit at all).  An input register is an image of the tile's rows as they
+  // lie in global memory (a dense operand: one contiguous range; otherwise one image per row, DVM_ROW_PITCH
+  // apart; a row vector shared by every row: one row image, of the tile's column block); a temporary is
+  // thread-private (V fp32 per thread); per-row scalar slots are thread-private.  A CTA holds two slots:
+  // while it computes the tile in one, the next tile (of this or of another stacked program) loads into the
+  // other.
+  auto layout = [&](Geo& g) -> int {
+    g.inv_mask = 0;
+    g.units = 0;
+    const int64_t Gthreads = 1ll << g.log2G;
+    for (int k = 0; k < e.n_in_regs; ++k) {
+      const Operand& od = e.opd[in_opd[k]];
+      const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
+      const bool inv = !flat && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
+      const bool gather = od.col_stride == 1 && od.cs != 1;
+      bool dense = od.col_stride == 1 && od.cs == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
+      if (!flat) {
+        if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+        if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+      }
+      // a gathered operand whose rows are adjacent in memory (a transposed matrix): with few threads per row the
+      // tile's part of a column is a contiguous strip of 256 / G elements -- copied in bulk, one strip per column
+      bool transposed = gather && !flat && !e.phased && od.ostride[0] == 1 && (od.cs * es) % 16 == 0 &&
+                        Gthreads * g.V <= T && ((T / Gthreads) * es) % 16 == 0;
+      for (int q = 1; q < 3 && transposed; ++q)
+        if (outer[q] > 1 && ((od.ostride[q] * es) % 16 != 0 || outer[0] % (T / Gthreads) != 0)) transposed = false;
+      const int mode = transposed ? DVM_LM_TRANSPOSED : gather ? DVM_LM_GATHER
+                              : (inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS));
+      if (inv && !gather) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
+      const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
+      // a gathered register holds fp32 values in the thread-private layout of a temporary
+      const int64_t bytes = transposed ? g.Ctile * (int64_t)DVM_STRIP_PITCH(T / Gthreads, es)
+                                       : gather ? (int64_t)g.V * 4 * T : (inv ? pitch : pitch * (T / Gthreads));
+      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
+      g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
+    }
+    for (int k = e.n_in_regs; k < nreg; ++k) {
+      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)DVM_LM_PRIVATE << 16);
+      g.units += g.V * 4 * T / DVM_LOCAL_UNIT;
+    }
+    g.scalar_unit = g.units;
+    if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
+    g.one_slot = false;
+    if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
+    int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
+    if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && !e.phased && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
+      // Two slots fit once per SM, one slot fits twice: eight more warps per SM are worth more than the
+      // prefetch inside a CTA (the other CTA computes while this one waits for its tile).  Only a launch of
+      // the program on its own can honour this; the programs of a stacked launch share two slots.
+      g.one_slot = true;
+      return 2;
+    }
+    return ctas > 2 ? 2 : ctas;  // the interpreter is compiled for two resident CTAs per SM
+  };
+  // cores the tiles spread over when `ctas` CTAs are resident per SM (the core count is quoted at 3 CTAs per SM)
+  auto cores = [&](int ctas) -> int64_t { return (int64_t)dvm_get_num_cores() * ctas / 3; };
+  const int W0 = W;
+  // 24 elements per thread (rows that fill three quarters of a 32-element tile) exist as the one-program
+  // basic interpreter variant only: not for programs of stacked launches, not with Cmp / Select / views
+  bool plain = g_min_resident_ctas == 0 && !combine_axis && !e.phased;
+  for (int i = 0; i < NN; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind == NK_COMPARE || n.kind == NK_SELECT || (n.kind == NK_UNARY && n.op == DVM_ISFINITE)) plain = false;
+  }
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    if (od.col_stride != 1) continue;
+    bool dense = od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);
+    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+    if (od.cs != 1 || (o >= e.n_opd - p->n_outputs && !dense && !flat)) plain = false;
+  }
+  static const int kVs[3] = {32, 24, 16};
+  for (int vi = 0; vi < 3; ++vi) {
+    Geo g;
+    g.V = kVs[vi];
+    if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
+    if (g.V == 24 && !plain && g_elems_per_thread != 24) continue;
+    // a phased program walks a row P times: the fewest, largest column blocks keep the per-tile overhead and the
+    // ragged last block small (8200 columns: 2 blocks of 4104 instead of 3 of 4096 / 4096 / 8)
+    if (e.phased && g.V != 32 && !g_elems_per_thread) continue;
+    g.W = W0;
+    if (flat) {
+      g.log2G = 8;
+      g.CB = 1;
+      g.Ctile = (int64_t)T * W0;  // the layout of a flat program does not depend on the chunk
+      g.flags = DVM_F_FLAT | DVM_F_ALIGNED;
+      const int ctas = layout(g);
+      if (ctas < 1) continue;
+      const int64_t N = cores(ctas);
+      int64_t total = empty ? 0 : C;  // everything merged into one dim
+      int64_t best_chunk = (int64_t)T * W0;
+      g.cost = -1;
+      for (int k = 1; k <= g.V / W0; ++k) {
+        int64_t chunk = (int64_t)T * W0 * k;
+        int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
+        if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
+      }
+      g.Ctile = best_chunk;
+      g.rowsR = cdiv(total, g.Ctile);
+      g.lastRowCols = g.rowsR > 0 ? total - (g.rowsR - 1) * g.Ctile : g.Ctile;
+      g.n_tiles = g.rowsR;
+      layout(g);  // dense operands are recognised by the final chunk
+      if (best.cost < 0 || g.cost < best.cost) best = g;
+      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
+      continue;
+    }
+    // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
+    bool aligned = primary >= 0;
+    if (primary >= 0)
+      for (int q = 0; q < 3; ++q)
+        if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
+    const int w = W0;
+    // a misaligned row segment starts up to w - 1 slots into its first chunk: keep that much spare capacity
+    const int64_t pad = aligned ? 0 : w - 1;
+    g.flags = (aligned ? DVM_F_ALIGNED : 0) | ((outer[1] > 1 || outer[2] > 1) ? DVM_F_OUTER_DIMS : 0);
+    g.rowsR = R;
+    g.lastRowCols = C;
+    for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
+      // combined results: the rows a warp holds (32 / G of them) are combined by shuffles before the atomics
+      if (combine_axis && lg > 5) continue;
+      int64_t G = 1 << lg, cap = G * g.V;
+      // ... but not so few threads per row that a row copy shrinks below 512 bytes while the rows are wider
+      // (measured on column sums: 256-byte copies 1560 GB/s, 512 bytes 1640, 1 KB and more lose to the atomics)
+      if (combine_axis && cap * 4 < 512 && C * 4 >= 512) continue;
+      if (e.phased && lg != 8) continue;  // one row per tile: the whole CTA on a column block
+      int64_t ct;
+      if (has_reduce && !e.phased) {
+        // a whole row per thread group; at the widest group a row may use the full capacity: its last
+        // columns then wrap around into the head slots of a misaligned row
+        if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
+        ct = C;
+      } else {
+        ct = ((cap - pad) / w) * w;
+        if (ct <= 0) continue;
+        if (ct > C) ct = C;
+        if (e.phased) ct = cdiv(cdiv(C, cdiv(C, ct)), w) * w;  // column blocks of even length
+      }
+      g.log2G = lg;
+      g.Ctile = ct;
+      g.CB = cdiv(C, ct);
+      g.n_tiles = cdiv(R, T / G) * g.CB * e.n_phases;
+      // the local-memory need of this geometry decides how many CTAs are resident at once
+      const int ctas = layout(g);
+      if (ctas < 1) continue;
+      // elements one thread processes per tile: the interpreter walks all V slots of a tile register, used or
+      // not (a row that fills three quarters of 32 slots costs what a full one costs: hence the 24-slot variant)
+      int64_t u = g.V;
+      g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta + (combine_axis ? 2 * g.V * G / 32 : 0));  // + the atomics a thread issues
+      if (g_min_resident_ctas == 2) {
+        // A program of a stacked launch shares the machine with the launch's other programs: there are no
+        // waves of its own to fill, what counts is its total work -- tiles x (elements per thread + overhead).
+        // (A term for the row copies a tile issues was measured and did not pay: narrower tiles that waste
+        // fewer slots win even at 64 copies of 256 bytes per tile.)
+        g.cost = g.n_tiles * (u + beta);
+      }
+      // Gathered / scattered operands whose ROWS are adjacent in memory (a transposed matrix): a warp's 32
+      // lanes cover min(32, G) columns x 32 / min(32, G) consecutive rows, and only the rows share 32-byte
+      // sectors -- few threads per row keep the traffic near the algorithmic bytes, many multiply it.
+      {
+        int64_t num = 0, den = 0;
+        for (int o = 0; o < e.n_opd; ++o) {
+          const Operand& od = e.opd[o];
+          if (od.col_stride != 1) continue;
+          const int64_t es = (int64_t)1 << DVM_DT_LG_ES(od.dtype);
+          int64_t amp = 4;  // in quarters: 4 = no amplification
+          if (od.cs > 1 && od.ostride[0] == 1) {
+            const int64_t nT = G < 32 ? G : 32, nR = 32 / nT;
+            amp = 4 * nT * cdiv(nR * es, 32) * 32 / (32 * es);
+            if (amp < 4) amp = 4;
+          }
+          num += amp * es;
+          den += 4 * es;
+        }
+        if (den > 0) g.cost = g.cost * num / den;
+      }
+      if (empty) g.n_tiles = 0;
+      if (best.cost < 0 || g.cost < best.cost) best = g;
+      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
+    }
+  }
+  if (tight.cost >= 0) best = tight;  // otherwise no geometry leaves that room: the unconstrained best stands
+  if (best.cost < 0) return DVM_ERR_UNSUPPORTED;  // row longer than the register budget, or too much local memory
+  return DVM_OK;
+}
+
+// Step 7 of the encoder: flags, header, tables and code of the chosen geometry into the caller's buffer.
+static int assemble_program(Enc& e, const Lowered& L, const Geo& best, int n_in, void* code, size_t code_capacity,
+                            size_t* code_size) {
+  const dvm_program* p = e.p;
+  const int NN = p->n_nodes;
+  const bool flat = L.flat;
+  const int primary = L.primary, nreg = L.nreg;
+  int W = L.W;
+  int64_t C = L.C;
+  int64_t outer[3] = {L.outer[0], L.outer[1], L.outer[2]};
+  const int log2G = best.log2G;
+  W = best.W;
+  const int64_t Ctile = best.Ctile, CB = best.CB, rowsR = best.rowsR, lastRowCols = best.lastRowCols, n_tiles = best.n_tiles;
+  uint32_t flags = best.flags;
+  const int units = best.units, scalar_unit = best.scalar_unit;
+  const uint32_t* lreg_table = best.lreg_table;
+  if (flat) {
+    C = Ctile;
+    for (int o = 0; o < e.n_opd; ++o) {
+      e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile * e.opd[o].cs : 0;
+      e.opd[o].ostride[1] = e.opd[o].ostride[2] = 0;
+    }
+    outer[0] = rowsR; outer[1] = outer[2] = 1;
+  }
+  if (n_tiles > 0xffffffffll || rowsR > 0xffffffffll) return DVM_ERR_TOO_LARGE;
+
+  // dense operands: the rows of a tile are one contiguous range (flat offset = row * C + col)
+  bool dense_of[DVM_MAX_OPERANDS];
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    bool dense = od.col_stride == 1 && od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);  // (a single row has no stride)
+    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
+    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
+    dense_of[o] = dense;
+  }
+  if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
+  if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
+  if (best.one_slot) flags |= DVM_F_ONE_SLOT;
+  if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
+  for (int i = 0; i < NN; ++i)
+    if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;
+  for (int i = 0; i < NN; ++i)
+    if (p->nodes[i].kind == NK_UNARY && p->nodes[i].op == DVM_ISFINITE && e.cls[i] == CLS_TILE) flags |= DVM_F_EXT_ISA;
+  for (int o = 0; o < p->n_outputs; ++o)  // a tile stored into a view whose rows are not one dense range: ViewStore
+    if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_VIEWS;
+  for (int k = 0; k < e.n_in_regs; ++k)
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
+  for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the views variant
+    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER || ((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_TRANSPOSED)
+      flags |= DVM_F_LOADS_BY_ROW | DVM_F_VIEWS;
+
+  // ---- 7. assemble ----
+  const int n_tensors = n_in + p->n_outputs;
+  const int code_words = e.n_loads + e.n_body;
+  size_t words = DVM_HDR_WORDS + 2 * (size_t)n_tensors + (size_t)DVM_OPD_WORDS * e.n_opd + nreg + code_words;
+  *code_size = words * 4;
+  if (!code || code_capacity < words * 4) return DVM_ERR_BUFFER_TOO_SMALL;
+  uint32_t* w = (uint32_t*)code;
+  memset(w, 0, words * 4);
+  w[DVM_H_MAGIC] = DVM_MAGIC;
+  w[DVM_H_KERNEL_TYPE] = DVM_KERNEL_VEC;
+  w[DVM_H_CODE_WORDS] = (uint32_t)code_words;
+  w[DVM_H_N_TILES] = (uint32_t)n_tiles;
+  w[DVM_H_TOTAL_WORDS] = (uint32_t)words;
+  w[DVM_H_COUNTS] = (uint32_t)n_tensors | ((uint32_t)n_in << 8) | ((uint32_t)e.n_opd << 16) |
+                    ((uint32_t)p->n_outputs << 24);
+  w[DVM_H_GEOM] = (uint32_t)log2G | ((uint32_t)W << 8) | ((uint32_t)nreg << 16) | (flags << 24);
+  w[DVM_H_COLS] = (uint32_t)C;
+  w[DVM_H_ROWS_LO] = (uint32_t)rowsR;
+  w[DVM_H_ROWS_HI] = (uint32_t)((uint64_t)rowsR >> 32);
+  w[DVM_H_COL_BLOCKS] = (uint32_t)CB;
+  w[DVM_H_COL_TILE] = (uint32_t)Ctile;
+  w[DVM_H_OUTER0] = (uint32_t)outer[0];
+  w[DVM_H_OUTER1] = (uint32_t)outer[1];
+  w[DVM_H_OUTER2] = (uint32_t)outer[2];
+  w[DVM_H_LAST_ROW_COLS] = (uint32_t)lastRowCols;
+  w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
+  w[DVM_H_LOCAL] = (uint32_t)e.n_in_regs | ((uint32_t)e.n_tmp_regs << 8) | ((uint32_t)e.n_sslots << 16) | ((uint32_t)best.V << 24);
+  w[DVM_H_LOAD_WORDS] = (uint32_t)e.n_loads;
+  w[DVM_H_LOCAL2] = (uint32_t)scalar_unit | ((uint32_t)units << 16);
+  uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
+  for (int o = 0; o < e.n_opd; ++o) {
+    const Operand& od = e.opd[o];
+    uint32_t* d = ot + o * DVM_OPD_WORDS;
+    const bool dense = dense_of[o];
+    d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
+                      ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25) |
+                      ((uint32_t)od.combine << 26);
+    d[DVM_OPD_COLSTRIDE] = (uint32_t)(uint64_t)od.cs;
+    for (int g = 0; g < 3; ++g) {
+      d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
+      d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
+    }
+    if (od.combine) d[DVM_OPD_FILL] = (uint32_t)od.numel;  // (strides stay below 2^32: the word is free)
+  }
+  uint32_t* lt = ot + e.n_opd * DVM_OPD_WORDS;
+  memcpy(lt, lreg_table, (size_t)nreg * 4);
+  for (int q = 0; q < e.n_loads; ++q)
+    if (DVM_INSN_OP(e.loads[q]) == DVM_OP_LDG && ((best.inv_mask >> DVM_INSN_A(e.loads[q])) & 1)) e.loads[q] |= 0x80u << 16;
+  memcpy(lt + nreg, e.loads, (size_t)e.n_loads * 4);
+  memcpy(lt + nreg + e.n_loads, e.body, (size_t)e.n_body * 4);
+  if (C > 0xffffffffll || outer[0] > 0xffffffffll || outer[1] > 0xffffffffll || outer[2] > 0xffffffffll)
+    return DVM_ERR_TOO_LARGE;
+  for (int o = 0; o < e.n_opd; ++o)
+    for (int q = 0; q < 3; ++q)
+      if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
+  for (int o = 0; o < e.n_opd; ++o)
+    if ((uint64_t)e.opd[o].cs > 0xffffffffull || (uint64_t)e.opd[o].numel > 0xffffffffull) return DVM_ERR_TOO_LARGE;
+  return DVM_OK;
+}
+
 static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const dvm_strides* in_strides, int n_in,
                        const float* scalars, int n_scalars, const dvm_strides* out_strides, void* code,
                        size_t code_capacity, size_t* code_size, dvm_shape* out_shapes, int n_out, bool lowered,
@@ -1111,307 +1445,18 @@ static int encode_core(const dvm_program* p, const dvm_shape* in_shapes, const d
         in_dtype[k] = e.opd[in_opd[k]].dtype;
       }
   }
-  int out_es = 2;
-  for (int o = 0; o < p->n_outputs; ++o)
-    if (p->outputs[o].dtype == DVM_F32 && e.cls[root(e, p->outputs[o].value)] == CLS_TILE) out_es = 4;
 
-  // ---- 6. shape tiling (Sec. 4.2): elements per thread V, threads per row G, column tile, tile count.
-  // Candidates are compared with the paper's cost  ceil(#tiles / N) * (tile + overhead)  in per-thread
-  // element units; N is the number of CTAs resident at once, which the local-memory need decides.
-  const int T = DVM_VM_THREADS;
-  const int64_t beta = 12;  // per-tile decode overhead in element units (the paper's "+2")
-  struct Geo {
-    int V, log2G, W, units, scalar_unit;
-    bool one_slot;  // costed for two CTAs per SM that hold ONE tile slot each (see DVM_F_ONE_SLOT)
-    int64_t Ctile, CB, rowsR, lastRowCols, n_tiles, cost;
-    uint32_t flags, inv_mask;
-    uint32_t lreg_table[DVM_MAX_LREGS];
-  } best, tight;  // `tight`: the best geometry among those that leave room for g_min_resident_ctas CTAs per SM
-  best.cost = -1;
-  tight.cost = -1;
-  // Local-memory layout of ONE tile slot, in 256-byte units, for a candidate geometry; returns the CTAs per SM
-  // it leaves room for (0: it does not fit at all).  An input register is an image of the tile's rows as they
-  // lie in global memory (a dense operand: one contiguous range; otherwise one image per row, DVM_ROW_PITCH
-  // apart; a row vector shared by every row: one row image, of the tile's column block); a temporary is
-  // thread-private (V fp32 per thread); per-row scalar slots are thread-private.  A CTA holds two slots:
-  // while it computes the tile in one, the next tile (of this or of another stacked program) loads into the
-  // other.
-  auto layout = [&](Geo& g) -> int {
-    g.inv_mask = 0;
-    g.units = 0;
-    const int64_t Gthreads = 1ll << g.log2G;
-    for (int k = 0; k < e.n_in_regs; ++k) {
-      const Operand& od = e.opd[in_opd[k]];
-      const int es = in_dtype[k] == DVM_DT_BF16 ? 2 : 4;
-      const bool inv = !flat && od.ostride[0] == 0 && od.ostride[1] == 0 && od.ostride[2] == 0;
-      const bool gather = od.col_stride == 1 && od.cs != 1;
-      bool dense = od.col_stride == 1 && od.cs == 1 && od.ostride[0] == (flat ? g.Ctile : C) && g.CB == 1;
-      if (!flat) {
-        if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
-        if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
-      }
-      // a gathered operand whose rows are adjacent in memory (a transposed matrix): with few threads per row the
-      // tile's part of a column is a contiguous strip of 256 / G elements -- copied in bulk, one strip per column
-      bool transposed = gather && !flat && !e.phased && od.ostride[0] == 1 && (od.cs * es) % 16 == 0 &&
-                        Gthreads * g.V <= T && ((T / Gthreads) * es) % 16 == 0;
-      for (int q = 1; q < 3 && transposed; ++q)
-        if (outer[q] > 1 && ((od.ostride[q] * es) % 16 != 0 || outer[0] % (T / Gthreads) != 0)) transposed = false;
-      const int mode = transposed ? DVM_LM_TRANSPOSED : gather ? DVM_LM_GATHER
-                              : (inv ? (g.CB == 1 ? DVM_LM_BCAST : DVM_LM_BCAST_TILE) : (dense ? DVM_LM_BLOCK : DVM_LM_ROWS));
-      if (inv && !gather) g.inv_mask |= 1u << k;  // one column block: the same for every tile, loaded once per slot
-      const int64_t pitch = DVM_ROW_PITCH(Gthreads, g.V, es);
-      // a gathered register holds fp32 values in the thread-private layout of a temporary
-      const int64_t bytes = transposed ? g.Ctile * (int64_t)DVM_STRIP_PITCH(T / Gthreads, es)
-                                       : gather ? (int64_t)g.V * 4 * T : (inv ? pitch : pitch * (T / Gthreads));
-      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)mode << 16) | ((uint32_t)in_opd[k] << 24);
-      g.units += (int)cdiv(bytes, DVM_LOCAL_UNIT);
-    }
-    for (int k = e.n_in_regs; k < nreg; ++k) {
-      g.lreg_table[k] = (uint32_t)g.units | ((uint32_t)DVM_LM_PRIVATE << 16);
-      g.units += g.V * 4 * T / DVM_LOCAL_UNIT;
-    }
-    g.scalar_unit = g.units;
-    if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
-    g.one_slot = false;
-    if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
-    int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
-    if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && !e.phased && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {
-      // Two slots fit once per SM, one slot fits twice: eight more warps per SM are worth more than the
-      // prefetch inside a CTA (the other CTA computes while this one waits for its tile).  Only a launch of
-      // the program on its own can honour this; the programs of a stacked launch share two slots.
-      g.one_slot = true;
-      return 2;
-    }
-    return ctas > 2 ? 2 : ctas;  // the interpreter is compiled for two resident CTAs per SM
-  };
-  // cores the tiles spread over when `ctas` CTAs are resident per SM (the core count is quoted at 3 CTAs per SM)
-  auto cores = [&](int ctas) -> int64_t { return (int64_t)dvm_get_num_cores() * ctas / 3; };
-  const int W0 = W;
-  // 24 elements per thread (rows that fill three quarters of a 32-element tile) exist as the one-program
-  // basic interpreter variant only: not for programs of stacked launches, not with Cmp / Select / views
-  bool plain = g_min_resident_ctas == 0 && !combine_axis && !e.phased;
-  for (int i = 0; i < NN; ++i) {
-    const Node& n = p->nodes[i];
-    if (n.kind == NK_COMPARE || n.kind == NK_SELECT || (n.kind == NK_UNARY && n.op == DVM_ISFINITE)) plain = false;
-  }
-  for (int o = 0; o < e.n_opd; ++o) {
-    const Operand& od = e.opd[o];
-    if (od.col_stride != 1) continue;
-    bool dense = od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);
-    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
-    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
-    if (od.cs != 1 || (o >= e.n_opd - p->n_outputs && !dense && !flat)) plain = false;
-  }
-  static const int kVs[3] = {32, 24, 16};
-  for (int vi = 0; vi < 3; ++vi) {
-    Geo g;
-    g.V = kVs[vi];
-    if (g_elems_per_thread && g.V != g_elems_per_thread) continue;
-    if (g.V == 24 && !plain && g_elems_per_thread != 24) continue;
-    // a phased program walks a row P times: the fewest, largest column blocks keep the per-tile overhead and the
-    // ragged last block small (8200 columns: 2 blocks of 4104 instead of 3 of 4096 / 4096 / 8)
-    if (e.phased && g.V != 32 && !g_elems_per_thread) continue;
-    g.W = W0;
-    if (flat) {
-      g.log2G = 8;
-      g.CB = 1;
-      g.Ctile = (int64_t)T * W0;  // the layout of a flat program does not depend on the chunk
-      g.flags = DVM_F_FLAT | DVM_F_ALIGNED;
-      const int ctas = layout(g);
-      if (ctas < 1) continue;
-      const int64_t N = cores(ctas);
-      int64_t total = empty ? 0 : C;  // everything merged into one dim
-      int64_t best_chunk = (int64_t)T * W0;
-      g.cost = -1;
-      for (int k = 1; k <= g.V / W0; ++k) {
-        int64_t chunk = (int64_t)T * W0 * k;
-        int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
-        if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
-      }
-      g.Ctile = best_chunk;
-      g.rowsR = cdiv(total, g.Ctile);
-      g.lastRowCols = g.rowsR > 0 ? total - (g.rowsR - 1) * g.Ctile : g.Ctile;
-      g.n_tiles = g.rowsR;
-      layout(g);  // dense operands are recognised by the final chunk
-      if (best.cost < 0 || g.cost < best.cost) best = g;
-      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
-      continue;
-    }
-    // rows of the primary operand start on W-element boundaries (given an aligned base pointer)?
-    bool aligned = primary >= 0;
-    if (primary >= 0)
-      for (int q = 0; q < 3; ++q)
-        if (outer[q] > 1 && (e.opd[primary].ostride[q] % W0) != 0) aligned = false;
-    const int w = W0;
-    // a misaligned row segment starts up to w - 1 slots into its first chunk: keep that much spare capacity
-    const int64_t pad = aligned ? 0 : w - 1;
-    g.flags = (aligned ? DVM_F_ALIGNED : 0) | ((outer[1] > 1 || outer[2] > 1) ? DVM_F_OUTER_DIMS : 0);
-    g.rowsR = R;
-    g.lastRowCols = C;
-    for (int lg = 8; lg >= 0; --lg) {  // ties go to more threads per row: wider coalesced accesses
-      // combined results: the rows a warp holds (32 / G of them) are combined by shuffles before the atomics
-      if (combine_axis && lg > 5) continue;
-      int64_t G = 1 << lg, cap = G * g.V;
-      // ... but not so few threads per row that a row copy shrinks below 512 bytes while the rows are wider
-      // (measured on column sums: 256-byte copies 1560 GB/s, 512 bytes 1640, 1 KB and more lose to the atomics)
-      if (combine_axis && cap * 4 < 512 && C * 4 >= 512) continue;
-      if (e.phased && lg != 8) continue;  // one row per tile: the whole CTA on a column block
-      int64_t ct;
-      if (has_reduce && !e.phased) {
-        // a whole row per thread group; at the widest group a row may use the full capacity: its last
-        // columns then wrap around into the head slots of a misaligned row
-        if (cap < C + pad && !(lg == 8 && cap >= C)) continue;
-        ct = C;
-      } else {
-        ct = ((cap - pad) / w) * w;
-        if (ct <= 0) continue;
-        if (ct > C) ct = C;
-        if (e.phased) ct = cdiv(cdiv(C, cdiv(C, ct)), w) * w;  // column blocks of even length
-      }
-      g.log2G = lg;
-      g.Ctile = ct;
-      g.CB = cdiv(C, ct);
-      g.n_tiles = cdiv(R, T / G) * g.CB * e.n_phases;
-      // the local-memory need of this geometry decides how many CTAs are resident at once
-      const int ctas = layout(g);
-      if (ctas < 1) continue;
-      // elements one thread processes per tile: the interpreter walks all V slots of a tile register, used or
-      // not (a row that fills three quarters of 32 slots costs what a full one costs: hence the 24-slot variant)
-      int64_t u = g.V;
-      g.cost = cdiv(g.n_tiles, cores(ctas)) * (u + beta + (combine_axis ? 2 * g.V * G / 32 : 0));  // + the atomics a thread issues
-      if (g_min_resident_ctas == 2) {
-        // A program of a stacked launch shares the machine with the launch's other programs: there are no
-        // waves of its own to fill, what counts is its total work -- tiles x (elements per thread + overhead).
-        // (A term for the row copies a tile issues was measured and did not pay: narrower tiles that waste
-        // fewer slots win even at 64 copies of 256 bytes per tile.)
-        g.cost = g.n_tiles * (u + beta);
-      }
-      // Gathered / scattered operands whose ROWS are adjacent in memory (a transposed matrix): a warp's 32
-      // lanes cover min(32, G) columns x 32 / min(32, G) consecutive rows, and only the rows share 32-byte
-      // sectors -- few threads per row keep the traffic near the algorithmic bytes, many multiply it.
-      {
-        int64_t num = 0, den = 0;
-        for (int o = 0; o < e.n_opd; ++o) {
-          const Operand& od = e.opd[o];
-          if (od.col_stride != 1) continue;
-          const int64_t es = (int64_t)1 << DVM_DT_LG_ES(od.dtype);
-          int64_t amp = 4;  // in quarters: 4 = no amplification
-          if (od.cs > 1 && od.ostride[0] == 1) {
-            const int64_t nT = G < 32 ? G : 32, nR = 32 / nT;
-            amp = 4 * nT * cdiv(nR * es, 32) * 32 / (32 * es);
-            if (amp < 4) amp = 4;
-          }
-          num += amp * es;
-          den += 4 * es;
-        }
-        if (den > 0) g.cost = g.cost * num / den;
-      }
-      if (empty) g.n_tiles = 0;
-      if (best.cost < 0 || g.cost < best.cost) best = g;
-      if (ctas >= g_min_resident_ctas && (tight.cost < 0 || g.cost < tight.cost)) tight = g;
-    }
-  }
-  if (tight.cost >= 0) best = tight;  // otherwise no geometry leaves that room: the unconstrained best stands
-  if (best.cost < 0) return DVM_ERR_UNSUPPORTED;  // row longer than the register budget, or too much local memory
-  const int log2G = best.log2G;
-  W = best.W;
-  const int64_t Ctile = best.Ctile, CB = best.CB, rowsR = best.rowsR, lastRowCols = best.lastRowCols, n_tiles = best.n_tiles;
-  uint32_t flags = best.flags;
-  const int units = best.units, scalar_unit = best.scalar_unit;
-  const uint32_t* lreg_table = best.lreg_table;
-  if (flat) {
-    C = Ctile;
-    for (int o = 0; o < e.n_opd; ++o) {
-      e.opd[o].ostride[0] = e.opd[o].col_stride ? Ctile * e.opd[o].cs : 0;
-      e.opd[o].ostride[1] = e.opd[o].ostride[2] = 0;
-    }
-    outer[0] = rowsR; outer[1] = outer[2] = 1;
-  }
-  if (n_tiles > 0xffffffffll || rowsR > 0xffffffffll) return DVM_ERR_TOO_LARGE;
-
-  // dense operands: the rows of a tile are one contiguous range (flat offset = row * C + col)
-  bool dense_of[DVM_MAX_OPERANDS];
-  for (int o = 0; o < e.n_opd; ++o) {
-    const Operand& od = e.opd[o];
-    bool dense = od.col_stride == 1 && od.cs == 1 && (od.ostride[0] == C || outer[0] == 1);  // (a single row has no stride)
-    if (outer[1] > 1 && od.ostride[1] != od.ostride[0] * outer[0]) dense = false;
-    if (outer[2] > 1 && od.ostride[2] != od.ostride[1] * outer[1]) dense = false;
-    dense_of[o] = dense;
-  }
-  if (primary >= 0 && dense_of[primary]) flags |= DVM_F_PRIMARY_DENSE;
-  if (primary < 0) flags |= DVM_F_ALIGNED;  // no tile-class memory operand: nothing to align to
-  if (best.one_slot) flags |= DVM_F_ONE_SLOT;
-  if (e.n_sslots > 0) flags |= DVM_F_LOADS_BY_ROW;
-  for (int i = 0; i < NN; ++i)
-    if (p->nodes[i].kind == NK_COMPARE || p->nodes[i].kind == NK_SELECT) flags |= DVM_F_EXT_ISA;
-  for (int i = 0; i < NN; ++i)
-    if (p->nodes[i].kind == NK_UNARY && p->nodes[i].op == DVM_ISFINITE && e.cls[i] == CLS_TILE) flags |= DVM_F_EXT_ISA;
-  for (int o = 0; o < p->n_outputs; ++o)  // a tile stored into a view whose rows are not one dense range: ViewStore
-    if (e.cls[root(e, p->outputs[o].value)] == CLS_TILE && !dense_of[e.out_operand[o]]) flags |= DVM_F_VIEWS;
-  for (int k = 0; k < e.n_in_regs; ++k)
-    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_ROWS) flags |= DVM_F_LOADS_BY_ROW;
-  for (int k = 0; k < e.n_in_regs; ++k)  // gathered rows: every thread fetches its own elements, in the views variant
-    if (((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_GATHER || ((best.lreg_table[k] >> 16) & 0xf) == DVM_LM_TRANSPOSED)
-      flags |= DVM_F_LOADS_BY_ROW | DVM_F_VIEWS;
-
-  // ---- 7. assemble ----
-  const int n_tensors = n_in + p->n_outputs;
-  const int code_words = e.n_loads + e.n_body;
-  size_t words = DVM_HDR_WORDS + 2 * (size_t)n_tensors + (size_t)DVM_OPD_WORDS * e.n_opd + nreg + code_words;
-  *code_size = words * 4;
-  if (!code || code_capacity < words * 4) return DVM_ERR_BUFFER_TOO_SMALL;
-  uint32_t* w = (uint32_t*)code;
-  memset(w, 0, words * 4);
-  w[DVM_H_MAGIC] = DVM_MAGIC;
-  w[DVM_H_KERNEL_TYPE] = DVM_KERNEL_VEC;
-  w[DVM_H_CODE_WORDS] = (uint32_t)code_words;
-  w[DVM_H_N_TILES] = (uint32_t)n_tiles;
-  w[DVM_H_TOTAL_WORDS] = (uint32_t)words;
-  w[DVM_H_COUNTS] = (uint32_t)n_tensors | ((uint32_t)n_in << 8) | ((uint32_t)e.n_opd << 16) |
-                    ((uint32_t)p->n_outputs << 24);
-  w[DVM_H_GEOM] = (uint32_t)log2G | ((uint32_t)W << 8) | ((uint32_t)nreg << 16) | (flags << 24);
-  w[DVM_H_COLS] = (uint32_t)C;
-  w[DVM_H_ROWS_LO] = (uint32_t)rowsR;
-  w[DVM_H_ROWS_HI] = (uint32_t)((uint64_t)rowsR >> 32);
-  w[DVM_H_COL_BLOCKS] = (uint32_t)CB;
-  w[DVM_H_COL_TILE] = (uint32_t)Ctile;
-  w[DVM_H_OUTER0] = (uint32_t)outer[0];
-  w[DVM_H_OUTER1] = (uint32_t)outer[1];
-  w[DVM_H_OUTER2] = (uint32_t)outer[2];
-  w[DVM_H_LAST_ROW_COLS] = (uint32_t)lastRowCols;
-  w[DVM_H_PRIMARY] = primary >= 0 ? (uint32_t)primary : 0xffffffffu;
-  w[DVM_H_LOCAL] = (uint32_t)e.n_in_regs | ((uint32_t)e.n_tmp_regs << 8) | ((uint32_t)e.n_sslots << 16) | ((uint32_t)best.V << 24);
-  w[DVM_H_LOAD_WORDS] = (uint32_t)e.n_loads;
-  w[DVM_H_LOCAL2] = (uint32_t)scalar_unit | ((uint32_t)units << 16);
-  uint32_t* ot = w + DVM_HDR_WORDS + 2 * n_tensors;
-  for (int o = 0; o < e.n_opd; ++o) {
-    const Operand& od = e.opd[o];
-    uint32_t* d = ot + o * DVM_OPD_WORDS;
-    const bool dense = dense_of[o];
-    d[DVM_OPD_INFO] = (uint32_t)od.slot | ((uint32_t)od.dtype << 8) | ((uint32_t)od.col_stride << 16) |
-                      ((uint32_t)(od.primary ? 1 : 0) << 24) | ((uint32_t)(dense ? 1 : 0) << 25) |
-                      ((uint32_t)od.combine << 26);
-    d[DVM_OPD_COLSTRIDE] = (uint32_t)(uint64_t)od.cs;
-    for (int g = 0; g < 3; ++g) {
-      d[DVM_OPD_STRIDE0 + 2 * g] = (uint32_t)(uint64_t)od.ostride[g];
-      d[DVM_OPD_STRIDE0 + 2 * g + 1] = (uint32_t)((uint64_t)od.ostride[g] >> 32);
-    }
-    if (od.combine) d[DVM_OPD_FILL] = (uint32_t)od.numel;  // (strides stay below 2^32: the word is free)
-  }
-  uint32_t* lt = ot + e.n_opd * DVM_OPD_WORDS;
-  memcpy(lt, lreg_table, (size_t)nreg * 4);
-  for (int q = 0; q < e.n_loads; ++q)
-    if (DVM_INSN_OP(e.loads[q]) == DVM_OP_LDG && ((best.inv_mask >> DVM_INSN_A(e.loads[q])) & 1)) e.loads[q] |= 0x80u << 16;
-  memcpy(lt + nreg, e.loads, (size_t)e.n_loads * 4);
-  memcpy(lt + nreg + e.n_loads, e.body, (size_t)e.n_body * 4);
-  if (C > 0xffffffffll || outer[0] > 0xffffffffll || outer[1] > 0xffffffffll || outer[2] > 0xffffffffll)
-    return DVM_ERR_TOO_LARGE;
-  for (int o = 0; o < e.n_opd; ++o)
-    for (int q = 0; q < 3; ++q)
-      if ((uint64_t)e.opd[o].ostride[q] > 0xffffffffull) return DVM_ERR_TOO_LARGE;  // the VM multiplies 32-bit strides
-  for (int o = 0; o < e.n_opd; ++o)
-    if ((uint64_t)e.opd[o].cs > 0xffffffffull || (uint64_t)e.opd[o].numel > 0xffffffffull) return DVM_ERR_TOO_LARGE;
-  return DVM_OK;
+  // ---- 6. shape tiling, 7. assembly ----
+  Lowered L;
+  L.C = C; L.R = R;
+  for (int q = 0; q < 3; ++q) L.outer[q] = outer[q];
+  L.flat = flat; L.empty = empty; L.has_reduce = has_reduce;
+  L.primary = primary; L.combine_axis = combine_axis; L.W = W; L.nreg = nreg;
+  for (int k = 0; k < DVM_MAX_LREGS; ++k) { L.in_dtype[k] = k < e.n_in_regs ? in_dtype[k] : 0; L.in_opd[k] = k < e.n_in_regs ? in_opd[k] : 0; }
+  Geo best;
+  const int gst = choose_geometry(e, L, best);
+  if (gst != DVM_OK) return gst;
+  return assemble_program(e, L, best, n_in, code, code_capacity, code_size);
 }
 
 // Reductions over another axis than the last (Table 1, Sum / Max / Min of [M, size, N] over `size`) are lowered
