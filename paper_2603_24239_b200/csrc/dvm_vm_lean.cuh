@@ -486,6 +486,9 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
       const uint32_t sub = (rec.x >> 8) & 0xffu;
       const uint32_t ra = (rec.x >> 16) & 0xffu;
       if (h == DVM_LK_END) break;
+      // two dispatch levels: the records of the bf16 sweeps (load, multiply-add, exponential, reduction, store) first
+      if (h == DVM_LK_LD2_BF16 || h == DVM_LK_BIN_BF16 || h == DVM_LK_STG || h == DVM_LK_RED || h == DVM_LK_FMA ||
+          h == DVM_LK_EXPS || h == DVM_LK_LDA_BF16) {
       switch (h) {
         case DVM_LK_LDA_BF16: {
           uint32_t R[V / 2];
@@ -516,77 +519,6 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
             DVM_ARITH(sub, __uint_as_float(R[i] << 16), __uint_as_float(R[i] & 0xffff0000u))
           }
         } break;
-        case DVM_LK_LDA_F32: {  // (in two halves: the raw words of a whole fp32 tile register would crowd the registers)
-          const uint32_t a = opw_addr(lean_opaque<4>(rec.y));
-#define DVM_LDA_F32_HALF(H)                                                                               \
-          {                                                                                               \
-            uint32_t R[V / 2];                                                                            \
-            if (lgW == 3) lean_raw_f32<2, (H) * (V / 16), ((H) + 1) * (V / 16)>(R, a, (uint32_t)(G << 5)); \
-            else lean_raw_f32<1, (H) * (V / 8), ((H) + 1) * (V / 8)>(R, a, (uint32_t)(G << 4));            \
-            _Pragma("unroll") for (int i = 0; i < VP / 2; ++i)                                            \
-              A[(H) * (VP / 2) + i] = make_float2(__uint_as_float(R[2 * i]), __uint_as_float(R[2 * i + 1])); \
-          }
-          DVM_LDA_F32_HALF(0)
-          DVM_LDA_F32_HALF(1)
-#undef DVM_LDA_F32_HALF
-        } break;
-        case DVM_LK_BIN_F32: {
-          const uint32_t a = opw_addr(lean_opaque<5>(rec.y));
-          const bool pre = (rec.x >> 24) != 0;  // ACC = ACC * S[.] * L[y]
-          const float m = pre ? s_S[(rec.x >> 24) - 1][tid] : 1.0f;
-#define DVM_BIN_F32_HALF(H)                                                                               \
-          {                                                                                               \
-            uint32_t R[V / 2];                                                                            \
-            if (lgW == 3) lean_raw_f32<2, (H) * (V / 16), ((H) + 1) * (V / 16)>(R, a, (uint32_t)(G << 5)); \
-            else lean_raw_f32<1, (H) * (V / 8), ((H) + 1) * (V / 8)>(R, a, (uint32_t)(G << 4));            \
-            if (pre) {                                                                                    \
-              _Pragma("unroll") for (int i = (H) * (VP / 2); i < ((H) + 1) * (VP / 2); ++i)               \
-                A[i] = __fmul2_rn(__fmul2_rn(A[i], make_float2(m, m)),                                    \
-                                  make_float2(__uint_as_float(R[2 * i - (H) * (V / 2)]), __uint_as_float(R[2 * i + 1 - (H) * (V / 2)]))); \
-            } else {                                                                                      \
-              DVM_ARITH(sub, __uint_as_float(R[2 * i - (H) * (V / 2)]), __uint_as_float(R[2 * i + 1 - (H) * (V / 2)])) \
-            }                                                                                             \
-          }
-#undef DVM_P0
-#undef DVM_P1
-#define DVM_P0 0
-#define DVM_P1 (VP / 2)
-          DVM_BIN_F32_HALF(0)
-#undef DVM_P0
-#undef DVM_P1
-#define DVM_P0 (VP / 2)
-#define DVM_P1 VP
-          DVM_BIN_F32_HALF(1)
-#undef DVM_P0
-#undef DVM_P1
-#define DVM_P0 0
-#define DVM_P1 VP
-#undef DVM_BIN_F32_HALF
-        } break;
-        case DVM_LK_LDA_PRIV: {
-          const uint32_t a = sb + (lean_opaque<6>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
-#pragma unroll
-          for (int q = 0; q < V / 4; ++q) {
-            const uint4 v = lean_lds128(a + q * PSTRIDE);
-            A[2 * q] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
-            A[2 * q + 1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
-          }
-        } break;
-        case DVM_LK_BIN_PRIV: {
-          const uint32_t a = sb + (lean_opaque<7>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
-          uint32_t R[V];
-#pragma unroll
-          for (int q = 0; q < V / 4; ++q) {
-            const uint4 v = lean_lds128(a + q * PSTRIDE);
-            R[4 * q] = v.x; R[4 * q + 1] = v.y; R[4 * q + 2] = v.z; R[4 * q + 3] = v.w;
-          }
-          DVM_ARITH(sub, __uint_as_float(R[2 * i]), __uint_as_float(R[2 * i + 1]))
-        } break;
-        case DVM_LK_BIN_ACC: {
-          float2 Y[VP];
-          DVM_EACH_PAIR Y[i] = A[i];
-          DVM_ARITH(sub, Y[i].x, Y[i].y)
-        } break;
         case DVM_LK_FMA: {  // ACC = ACC * m + c, m and c immediates or per-row scalars: add / sub / rsub / mul / div by a scalar
           const uint32_t ra_ = lean_opaque<9>(ra);
           float m = (sub & 1u) ? s_S[ra_][tid] : __uint_as_float(rec.y);
@@ -594,14 +526,6 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
           if (sub & 4u) m = fast_rcp(m);
           if (sub & 8u) c = -c;
           DVM_EACH_PAIR A[i] = __ffma2_rn(A[i], make_float2(m, m), make_float2(c, c));
-        } break;
-        case DVM_LK_BINI:
-        case DVM_LK_BINS: {  // (what the multiply-add form does not cover: rdiv, min, max)
-          const uint32_t ra_ = lean_opaque<10>(ra);
-          const float y = h == DVM_LK_BINS ? s_S[ra_][tid] : __uint_as_float(rec.y);
-          if (sub == DVM_A_RDIV) { DVM_EACH_PAIR A[i] = make_float2(fast_div(y, A[i].x), fast_div(y, A[i].y)); }
-          else if (sub == DVM_A_MIN) { DVM_EACH_PAIR A[i] = make_float2(A[i].x < y ? A[i].x : y, A[i].y < y ? A[i].y : y); }
-          else { DVM_EACH_PAIR A[i] = make_float2(A[i].x > y ? A[i].x : y, A[i].y > y ? A[i].y : y); }
         } break;
         case DVM_LK_EXPS: {
           const float m = -s_S[lean_opaque<11>(ra)][tid];
@@ -611,63 +535,6 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
           } else {
             DVM_EACH_PAIR A[i] = lean_exp2(__fadd2_rn(A[i], make_float2(m, m)));
           }
-        } break;
-        case DVM_LK_ACT: {
-          if constexpr (HEAVY) {
-            if (sub == DVM_ACT_GELU) { DVM_EACH_PAIR A[i] = packed_gelu(A[i]); }
-            else { DVM_EACH_PAIR A[i] = packed_silu(A[i]); }
-          } else {
-            err = ST_BAD_CODE;
-          }
-        } break;
-        case DVM_LK_UN: {
-#define DVM_UN_CASE(U, EXPR)                                                          \
-  case U:                                                                             \
-    DVM_EACH_PAIR {                                                                   \
-      float x = A[i].x; const float vx = (EXPR);                                      \
-      x = A[i].y; const float vy = (EXPR);                                            \
-      A[i] = make_float2(vx, vy);                                                     \
-    }                                                                                 \
-    break;
-          switch (sub) {
-            case DVM_U_EXP: DVM_EACH_PAIR A[i] = lean_exp2(A[i]); break;
-            case DVM_U_EXP | 0x80: DVM_EACH_PAIR A[i] = lean_exp2_fast(A[i], 0.f); break;
-            case DVM_U_SIGMOID | 0x80:
-              DVM_EACH_PAIR {
-                const float2 e = lean_exp2_fast(make_float2(-A[i].x, -A[i].y), 0.f);
-                A[i] = make_float2(fast_rcp(1.0f + e.x), fast_rcp(1.0f + e.y));
-              }
-              break;
-            DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
-            DVM_UN_CASE(DVM_U_ABS, fabsf(x))
-            case DVM_U_SIGMOID:
-              DVM_EACH_PAIR {
-                const float2 e = lean_exp2(make_float2(-A[i].x, -A[i].y));
-                A[i] = make_float2(fast_rcp(1.0f + e.x), fast_rcp(1.0f + e.y));
-              }
-              break;
-            DVM_UN_CASE(DVM_U_NEG, -x)
-            DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
-            DVM_UN_CASE(DVM_U_RND_BF16, round_bf16(x))
-            default:
-              if constexpr (HEAVY) {
-                switch (sub) {
-                  DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
-                  DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
-                  DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
-                  DVM_UN_CASE(DVM_U_LOG, logf(x))
-                  case DVM_U_ERF: DVM_EACH_PAIR A[i] = packed_erf(A[i]); break;
-                  DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
-                  DVM_UN_CASE(DVM_U_ROUND, rintf(x))
-                  DVM_UN_CASE(DVM_U_TANH, tanhf(x))
-                  default: err = ST_BAD_CODE; break;
-                }
-              } else {
-                err = ST_BAD_CODE;
-              }
-              break;
-          }
-#undef DVM_UN_CASE
         } break;
         case DVM_LK_RED: {
           // ---- row reduction (Table 1, Sum / Max / Min with N = 1) ----
@@ -789,6 +656,146 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
             }
           }
         } break;
+        default: break;
+      }
+      } else {
+      switch (h) {
+        case DVM_LK_LDA_F32: {  // (in two halves: the raw words of a whole fp32 tile register would crowd the registers)
+          const uint32_t a = opw_addr(lean_opaque<4>(rec.y));
+#define DVM_LDA_F32_HALF(H)                                                                               \
+          {                                                                                               \
+            uint32_t R[V / 2];                                                                            \
+            if (lgW == 3) lean_raw_f32<2, (H) * (V / 16), ((H) + 1) * (V / 16)>(R, a, (uint32_t)(G << 5)); \
+            else lean_raw_f32<1, (H) * (V / 8), ((H) + 1) * (V / 8)>(R, a, (uint32_t)(G << 4));            \
+            _Pragma("unroll") for (int i = 0; i < VP / 2; ++i)                                            \
+              A[(H) * (VP / 2) + i] = make_float2(__uint_as_float(R[2 * i]), __uint_as_float(R[2 * i + 1])); \
+          }
+          DVM_LDA_F32_HALF(0)
+          DVM_LDA_F32_HALF(1)
+#undef DVM_LDA_F32_HALF
+        } break;
+        case DVM_LK_BIN_F32: {
+          const uint32_t a = opw_addr(lean_opaque<5>(rec.y));
+          const bool pre = (rec.x >> 24) != 0;  // ACC = ACC * S[.] * L[y]
+          const float m = pre ? s_S[(rec.x >> 24) - 1][tid] : 1.0f;
+#define DVM_BIN_F32_HALF(H)                                                                               \
+          {                                                                                               \
+            uint32_t R[V / 2];                                                                            \
+            if (lgW == 3) lean_raw_f32<2, (H) * (V / 16), ((H) + 1) * (V / 16)>(R, a, (uint32_t)(G << 5)); \
+            else lean_raw_f32<1, (H) * (V / 8), ((H) + 1) * (V / 8)>(R, a, (uint32_t)(G << 4));            \
+            if (pre) {                                                                                    \
+              _Pragma("unroll") for (int i = (H) * (VP / 2); i < ((H) + 1) * (VP / 2); ++i)               \
+                A[i] = __fmul2_rn(__fmul2_rn(A[i], make_float2(m, m)),                                    \
+                                  make_float2(__uint_as_float(R[2 * i - (H) * (V / 2)]), __uint_as_float(R[2 * i + 1 - (H) * (V / 2)]))); \
+            } else {                                                                                      \
+              DVM_ARITH(sub, __uint_as_float(R[2 * i - (H) * (V / 2)]), __uint_as_float(R[2 * i + 1 - (H) * (V / 2)])) \
+            }                                                                                             \
+          }
+#undef DVM_P0
+#undef DVM_P1
+#define DVM_P0 0
+#define DVM_P1 (VP / 2)
+          DVM_BIN_F32_HALF(0)
+#undef DVM_P0
+#undef DVM_P1
+#define DVM_P0 (VP / 2)
+#define DVM_P1 VP
+          DVM_BIN_F32_HALF(1)
+#undef DVM_P0
+#undef DVM_P1
+#define DVM_P0 0
+#define DVM_P1 VP
+#undef DVM_BIN_F32_HALF
+        } break;
+        case DVM_LK_LDA_PRIV: {
+          const uint32_t a = sb + (lean_opaque<6>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
+#pragma unroll
+          for (int q = 0; q < V / 4; ++q) {
+            const uint4 v = lean_lds128(a + q * PSTRIDE);
+            A[2 * q] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+            A[2 * q + 1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+          }
+        } break;
+        case DVM_LK_BIN_PRIV: {
+          const uint32_t a = sb + (lean_opaque<7>(rec.y) & 0x3ffffu) + (uint32_t)tid * 16;
+          uint32_t R[V];
+#pragma unroll
+          for (int q = 0; q < V / 4; ++q) {
+            const uint4 v = lean_lds128(a + q * PSTRIDE);
+            R[4 * q] = v.x; R[4 * q + 1] = v.y; R[4 * q + 2] = v.z; R[4 * q + 3] = v.w;
+          }
+          DVM_ARITH(sub, __uint_as_float(R[2 * i]), __uint_as_float(R[2 * i + 1]))
+        } break;
+        case DVM_LK_BIN_ACC: {
+          float2 Y[VP];
+          DVM_EACH_PAIR Y[i] = A[i];
+          DVM_ARITH(sub, Y[i].x, Y[i].y)
+        } break;
+        case DVM_LK_BINI:
+        case DVM_LK_BINS: {  // (what the multiply-add form does not cover: rdiv, min, max)
+          const uint32_t ra_ = lean_opaque<10>(ra);
+          const float y = h == DVM_LK_BINS ? s_S[ra_][tid] : __uint_as_float(rec.y);
+          if (sub == DVM_A_RDIV) { DVM_EACH_PAIR A[i] = make_float2(fast_div(y, A[i].x), fast_div(y, A[i].y)); }
+          else if (sub == DVM_A_MIN) { DVM_EACH_PAIR A[i] = make_float2(A[i].x < y ? A[i].x : y, A[i].y < y ? A[i].y : y); }
+          else { DVM_EACH_PAIR A[i] = make_float2(A[i].x > y ? A[i].x : y, A[i].y > y ? A[i].y : y); }
+        } break;
+        case DVM_LK_ACT: {
+          if constexpr (HEAVY) {
+            if (sub == DVM_ACT_GELU) { DVM_EACH_PAIR A[i] = packed_gelu(A[i]); }
+            else { DVM_EACH_PAIR A[i] = packed_silu(A[i]); }
+          } else {
+            err = ST_BAD_CODE;
+          }
+        } break;
+        case DVM_LK_UN: {
+#define DVM_UN_CASE(U, EXPR)                                                          \
+  case U:                                                                             \
+    DVM_EACH_PAIR {                                                                   \
+      float x = A[i].x; const float vx = (EXPR);                                      \
+      x = A[i].y; const float vy = (EXPR);                                            \
+      A[i] = make_float2(vx, vy);                                                     \
+    }                                                                                 \
+    break;
+          switch (sub) {
+            case DVM_U_EXP: DVM_EACH_PAIR A[i] = lean_exp2(A[i]); break;
+            case DVM_U_EXP | 0x80: DVM_EACH_PAIR A[i] = lean_exp2_fast(A[i], 0.f); break;
+            case DVM_U_SIGMOID | 0x80:
+              DVM_EACH_PAIR {
+                const float2 e = lean_exp2_fast(make_float2(-A[i].x, -A[i].y), 0.f);
+                A[i] = make_float2(fast_rcp(1.0f + e.x), fast_rcp(1.0f + e.y));
+              }
+              break;
+            DVM_UN_CASE(DVM_U_RSQRT, rsqrtf(x))
+            DVM_UN_CASE(DVM_U_ABS, fabsf(x))
+            case DVM_U_SIGMOID:
+              DVM_EACH_PAIR {
+                const float2 e = lean_exp2(make_float2(-A[i].x, -A[i].y));
+                A[i] = make_float2(fast_rcp(1.0f + e.x), fast_rcp(1.0f + e.y));
+              }
+              break;
+            DVM_UN_CASE(DVM_U_NEG, -x)
+            DVM_UN_CASE(DVM_U_RECIP, fast_rcp(x))
+            DVM_UN_CASE(DVM_U_RND_BF16, round_bf16(x))
+            default:
+              if constexpr (HEAVY) {
+                switch (sub) {
+                  DVM_UN_CASE(DVM_U_TRUNC_I32, trunc_i32(x))
+                  DVM_UN_CASE(DVM_U_TRUNC_U8, trunc_u8(x))
+                  DVM_UN_CASE(DVM_U_SQRT, sqrtf(x))
+                  DVM_UN_CASE(DVM_U_LOG, logf(x))
+                  case DVM_U_ERF: DVM_EACH_PAIR A[i] = packed_erf(A[i]); break;
+                  DVM_UN_CASE(DVM_U_FLOOR, floorf(x))
+                  DVM_UN_CASE(DVM_U_ROUND, rintf(x))
+                  DVM_UN_CASE(DVM_U_TANH, tanhf(x))
+                  default: err = ST_BAD_CODE; break;
+                }
+              } else {
+                err = ST_BAD_CODE;
+              }
+              break;
+          }
+#undef DVM_UN_CASE
+        } break;
         case DVM_LK_STGI: {  // Table 1, Cast: ACC stored as i32 (sub 1) or u8 (sub 2), converted toward zero
           const int lg_es = (int)lean_opaque<55>(ra);
           const unsigned long long base = (unsigned long long)lean_opaque<15>(rec.y) | ((unsigned long long)rec.z << 32);
@@ -894,6 +901,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
         default:
           err = ST_BAD_CODE;
           break;
+      }
       }
       if (err == ST_BAD_CODE) break;
     }
