@@ -1004,6 +1004,10 @@ static int choose_geometry(const Enc& e, const Lowered& L, Geo& best) {
       for (int k = 1; k <= g.V / W0; ++k) {
         int64_t chunk = (int64_t)T * W0 * k;
         int64_t cost = cdiv(cdiv(total, chunk), N) * (W0 * k + beta);
+        // a program of a stacked launch has no waves of its own: its cost is its total work, and a tile costs its
+        // V slots whether the chunk fills them or not (half-filled chunks doubled sigmoid(x) * y: 117 -> instructions
+        // per element in the C4 mix)
+        if (g_min_resident_ctas == 2) cost = cdiv(total, chunk) * (g.V + beta);
         if (g.cost < 0 || cost <= g.cost) { g.cost = cost; best_chunk = chunk; }
       }
       g.Ctile = best_chunk;
