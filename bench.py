@@ -366,9 +366,14 @@ class C4Workload:
 
     def __init__(self, dvm, n_launches=50, device="cuda"):
         self.dvm = dvm
+        # Programs of one stacked launch share the elements-per-thread setting, and the launch's CTAs are sized by
+        # its largest program.  32 elements per thread halve the per-tile overhead per element; two tile slots of that
+        # size fit an SM once, so the launch runs with ONE slot per CTA, two CTAs per SM (measured on this sweep:
+        # 16 elements / two slots 2007 GB/s kernel-only, 32 / two slots 1809, 16 / one slot 1622, 32 / one slot 2268).
         if not dvm.binding.lib.dvm_get_elems_per_thread():
-            dvm.set_elems_per_thread(16)   # programs of one stacked launch share the setting; 16 fits every program
-        dvm.set_min_resident_ctas(2)       # the CTAs of a stacked launch are sized by its largest program
+            dvm.set_elems_per_thread(32)
+        dvm.set_min_resident_ctas(3)
+        dvm.set_stacked_one_slot(True)
         self.launches = wl.shapes_c4(n_launches)
         self.progs = {k: wl.stack_program(k) for k in wl.STACK_KINDS}
         self.ps = {k: dvm.program_from_nodes(p.nodes) for k, p in self.progs.items()}
@@ -825,7 +830,7 @@ def oracle_check(dvm, name):
     stacked = name == "c4"
     codes, tls, wants, progs_seen = [], [], [], []
     if stacked:
-        dvm.set_elems_per_thread(16)
+        dvm.set_elems_per_thread(32)
     try:
         for case in _check_cases(name):
             prog, ins, params, strides = case[:4]

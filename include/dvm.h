@@ -209,8 +209,16 @@ int dvm_get_elems_per_thread(void);
  * exceed half an SM's shared memory leaves the whole launch with one CTA per SM.  With 2, the encoder
  * takes the best geometry among those whose slots fit twice per SM (e.g. two column blocks per row, whose
  * row-vector operands are then half as long); a program no geometry of which fits keeps its unconstrained
- * best.  Callers of dvm_launch_stacked set it before encoding.  Per calling thread (the setting of one thread does not reach the encodes of another). */
+ * best.  Callers of dvm_launch_stacked set it before encoding.  Per calling thread (the setting of one thread does not reach the encodes of another).
+ * n = 3: as 2, for stacked launches that run with ONE tile slot per CTA (dvm_set_stacked_one_slot): a geometry has
+ * to leave room for two CTAs that hold one slot each, so tiles may be twice as large. */
 void dvm_set_min_resident_ctas(int n);
+/* Stacked launches of this process (dvm_launch_stacked, and the flushes of the streaming fuser) run with one tile
+ * slot per CTA when `on` != 0: a tile's loads start when the CTA's previous tile is done (no load-ahead inside a
+ * CTA; the SM's other CTA computes meanwhile), every program on one level of the variant with level waits.  For
+ * programs encoded with dvm_set_min_resident_ctas(3); programs whose single slot does not fit twice leave the launch
+ * with one CTA per SM.  Default off. */
+void dvm_set_stacked_one_slot(int on);
 int dvm_get_min_resident_ctas(void);
 /* One-program launches of the basic instruction set run on a lean variant of the interpreter (Algorithm 2 from
  * linked code: a shorter instruction stream per tile).  0 sends every launch of the process to the general

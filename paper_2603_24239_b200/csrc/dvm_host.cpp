@@ -27,8 +27,12 @@ static thread_local int g_elems_per_thread = 0;
 extern "C" void dvm_set_elems_per_thread(int v) { g_elems_per_thread = (v == 16 || v == 24 || v == 32) ? v : 0; }
 extern "C" int dvm_get_elems_per_thread(void) { return g_elems_per_thread; }
 static thread_local int g_min_resident_ctas = 0;
-extern "C" void dvm_set_min_resident_ctas(int n) { g_min_resident_ctas = (n == 2) ? 2 : 0; }
-extern "C" int dvm_get_min_resident_ctas(void) { return g_min_resident_ctas; }
+static thread_local bool g_stack_one_slot = false;  // (n = 3: two CTAs per SM that hold ONE tile slot each)
+extern "C" void dvm_set_min_resident_ctas(int n) {
+  g_min_resident_ctas = (n == 2 || n == 3) ? 2 : 0;
+  g_stack_one_slot = n == 3;
+}
+extern "C" int dvm_get_min_resident_ctas(void) { return g_stack_one_slot ? 3 : g_min_resident_ctas; }
 extern "C" void dvm_set_num_cores(int n) { g_num_cores = n > 0 ? n : 0; }
 extern "C" int dvm_get_num_cores(void) { return g_num_cores > 0 ? g_num_cores : kDefaultCores; }
 
@@ -951,6 +955,11 @@ static int choose_geometry(const Enc& e, const Lowered& L, Geo& best) {
     g.scalar_unit = g.units;
     if (e.n_sslots > 0) g.units += 2 * 16 * T / DVM_LOCAL_UNIT;  // 8 fp32 slots per thread
     g.one_slot = false;
+    if (g_stack_one_slot) {  // a stacked launch whose CTAs hold one tile slot: what has to fit twice is one slot
+      if (g.units + 1 > DVM_MAX_LOCAL_UNITS / 2) return g.units + 1 > DVM_MAX_LOCAL_UNITS ? 0 : 1;
+      const int one = 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600);
+      return one > 2 ? 2 : one;
+    }
     if (2 * g.units + 1 > DVM_MAX_LOCAL_UNITS) return 0;
     int ctas = 233472 / ((2 * g.units + 1) * DVM_LOCAL_UNIT + 9600);  // 228 KB per SM; per CTA: 1 KB reserved + 8.3 KB static
     if (ctas == 1 && g.V != 24 && g_min_resident_ctas < 2 && !e.phased && 233472 / ((g.units + 1) * DVM_LOCAL_UNIT + 9600) >= 2) {

@@ -117,6 +117,8 @@ void dvm_note_cuda_error(int e) { t_last_cuda_error = e; }
 void dvm_count_launch() { __atomic_add_fetch(&g_launches, 1, __ATOMIC_RELAXED); }
 
 extern "C" void dvm_set_lean_kernel(int on) { g_use_lean = on; }
+static int g_stacked_one_slot = 0;
+extern "C" void dvm_set_stacked_one_slot(int on) { g_stacked_one_slot = on != 0; }
 extern "C" int dvm_last_cuda_error(void) { return t_last_cuda_error; }
 extern "C" int64_t dvm_launch_count(void) { return (int64_t)__atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
 
@@ -558,6 +560,10 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   bool one_slot = n_programs == 1 && !level &&
                   ((((const uint32_t*)codes[0])[DVM_H_GEOM] >> 24) & DVM_F_ONE_SLOT) != 0;
   static const int kOneLevel[1] = {0};
+  static const int kNoLevels[DVM_MAX_STACK] = {0};
+  // stacked launches with one tile slot per CTA (dvm_set_stacked_one_slot): every program on level 0, every tile's
+  // loads held back until the CTA's previous tile is done -- twice the tile size fits two CTAs per SM
+  if (g_stacked_one_slot && use_queue && !level && n_programs >= 1) { one_slot = true; level = kNoLevels; }
   const bool queue_asked = use_queue;
   // directory: [program word offsets (n)][tile prefix sums (n+1)][tiles before the program's level (n, with levels)]
   uint32_t dir = (level ? 3 : 2) * (uint32_t)n_programs + 1;
@@ -615,7 +621,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, level, true, &pos) : DVM_ERR_UNSUPPORTED;
   if (st == DVM_ERR_UNSUPPORTED) {
     lean = 0;
-    if (one_slot) { level = kOneLevel; use_queue = true; }
+    if (one_slot && !level) { level = kOneLevel; use_queue = true; }
     if (tile_end && use_queue) return DVM_ERR_UNSUPPORTED;  // (tile ranges exist for launches without a work queue)
     st = place_all(P, n_programs, codes, tensors, n_tensors, level, false, &pos);
   }

@@ -69,6 +69,31 @@ def test_stacked_config4_launches(min_ctas, launch):
     _check_all(meta, report=f"c4 launch {launch}" if (min_ctas, launch) == (2, 0) else None)
 
 
+@pytest.mark.parametrize("launch", [0, 3])
+def test_stacked_config4_launches_one_slot_per_cta(launch):
+    """The configuration bench.py times for config 4: 32 elements per thread, geometries that fit two CTAs with
+    one tile slot each (dvm_set_min_resident_ctas(3)), launched with dvm_set_stacked_one_slot."""
+    items = wl.shapes_c4(launch + 1)[launch]
+    dvm.set_elems_per_thread(32)
+    dvm.set_min_resident_ctas(3)
+    dvm.set_stacked_one_slot(True)
+    try:
+        codes, tls, meta = _stack(items, wl.data_seed("c4", 0) + launch)
+        n0 = dvm.launch_count()
+        dvm.launch_stacked(codes, tls)
+        assert dvm.last_device_status() == 0
+        assert dvm.launch_count() - n0 == 1
+        # a second launch of the same programs finds the queue counters at rest
+        for t in tls:
+            t[-1].fill_(float("nan"))
+        dvm.launch_stacked(codes, tls)
+        assert dvm.last_device_status() == 0
+    finally:
+        dvm.set_min_resident_ctas(0)
+        dvm.set_stacked_one_slot(False)
+    _check_all(meta)
+
+
 def test_stacked_repeated_launches_reuse_queue():
     """The work queue returns to its resting state after every launch."""
     items = wl.shapes_c4(2)[1][:16]
