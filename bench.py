@@ -967,6 +967,10 @@ def run_config(dvm, name, peaks, peak_kind, steps, warmup=3, check=True, baselin
                                "seconds": dt, "check": oracle_check(dvm, name)}
     del W
     torch.cuda.empty_cache()
+    # a workload may have set the encoder's knobs for its own programs (c4): the next one starts from the defaults
+    dvm.set_elems_per_thread(0)
+    dvm.set_min_resident_ctas(0)
+    dvm.set_stacked_one_slot(False)
     return out
 
 
@@ -1321,7 +1325,8 @@ def main():
         del W
         torch.cuda.empty_cache()
         cfgs = {}
-        for name, steps in (("c1", 50), ("c3", 2), ("c4", 2), ("c5", 2), ("addmm", 2), ("ifelse", 2), ("views", 2)):
+        # (the tensor-core sweeps first, while the GPU is coolest; c4 last: it changes the encoder's knobs)
+        for name, steps in (("c5", 2), ("addmm", 2), ("ifelse", 2), ("views", 2), ("c1", 50), ("c3", 2), ("c4", 2)):
             if name == name_main:
                 continue
             try:
