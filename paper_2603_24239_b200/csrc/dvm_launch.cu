@@ -63,7 +63,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -87,13 +87,31 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
 // Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
 uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
   const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
-                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 14);
+                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 15);  // (lean: two bits)
   return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
 }
 
 // Resident CTAs per SM of one interpreter variant for a launch with `smem` bytes of dynamic shared memory
 // (cached per device).  The variants with level waits rely on the whole grid being resident: no CTA fits -> no launch.
+// Two variants never share a cache key (a shared key would also skip the second kernel's shared-memory attribute).
+static bool dvm_variant_keys_distinct() {
+  typedef const DvmVmVariant* (*GroupFn)(int*);
+#define DVM_GROUP_FN(g) &dvm_vm_group_##g,
+  static const GroupFn groups[] = {DVM_GROUPS(DVM_GROUP_FN)};
+#undef DVM_GROUP_FN
+  std::unordered_map<uint64_t, const DvmVmVariant*> seen;
+  for (GroupFn g : groups) {
+    int n = 0;
+    const DvmVmVariant* v = g(&n);
+    for (int i = 0; i < n; ++i)
+      if (!seen.emplace(dvm_occupancy_key(&v[i], 0), &v[i]).second) return false;
+  }
+  return true;
+}
+
 static int dvm_occupancy(const DvmVmVariant* v, size_t smem, int* out) {
+  static const bool keys_ok = dvm_variant_keys_distinct();
+  if (!keys_ok) return DVM_ERR_UNSUPPORTED;
   int dev = 0;
   DVM_CUDA(cudaGetDevice(&dev));
   std::lock_guard<std::mutex> lk(g_mu);
@@ -211,8 +229,11 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
     const uint32_t w0 = body[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0) ? DVM_INSN_LEN(w0) : 1;
     const uint32_t ia = DVM_INSN_A(w0), ib = DVM_INSN_B(w0);
     const uint32_t cls = op >> 3;
+    const uint32_t tag = DVM_INSN_TAG(w0);  // phased programs: the phase a run-once instruction belongs to
     int kind = 0;
-    if (op == DVM_OP_LDA) {
+    if (op == DVM_OP_PHASE) {
+      if (ia != 0xffu) push(DVM_LK_W0(DVM_LK_PHASE, 0, ia, 0), 0, 0, 0);
+    } else if (op == DVM_OP_LDA) {
       const uint32_t ow = opw(ia, ib, &kind);
       push(DVM_LK_W0(DVM_LK_LDA_BF16 + kind, 0, 0, 0), ow, 0, 0);
     } else if (cls == (DVM_OP_LD2 >> 3)) {
@@ -265,29 +286,29 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       bool fused = false;
       if (pc + len < code_words && DVM_INSN_OP(nx) == DVM_OP_SOP && DVM_INSN_B(nx) == DVM_SK_FMAU) {
         const uint32_t w1 = body[pc + len + 1];
-        if (((w1 >> 8) & 0xff) == ia && DVM_INSN_A(nx) == ia) {
-          push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, 1), w1 & 0xff, body[pc + len + 2], body[pc + len + 3]);
+        if (((w1 >> 8) & 0xff) == ia && DVM_INSN_A(nx) == ia && DVM_INSN_TAG(nx) == tag) {
+          push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, 1 | (tag << 4)), w1 & 0xff, body[pc + len + 2], body[pc + len + 3]);
           pc += DVM_INSN_LEN(nx);
           fused = true;
         }
       }
-      if (!fused) push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, 0), 0, 0, 0);
+      if (!fused) push(DVM_LK_W0(DVM_LK_RED, op & 7, ia, tag << 4), 0, 0, 0);
     } else if (op == DVM_OP_STG) {
       const uint32_t info = ot[ib * DVM_OPD_WORDS + DVM_OPD_INFO];
       if (!((info >> 25) & 1u) || ((info >> 26) & 3u)) return 0;  // a stored view / a combined result: general interpreter
       const unsigned long long a = (unsigned long long)(uintptr_t)tensors[info & 0xff];
       const uint32_t sdt = (info >> 8) & 0xff;   // sub: 0 fp32 / bf16 as they are, 1: converted to i32, 2: to u8
-      push(DVM_LK_W0(sdt > DVM_DT_BF16 ? DVM_LK_STGI : DVM_LK_STG, sdt == DVM_DT_I32 ? 1 : sdt == DVM_DT_U8 ? 2 : 0, DVM_DT_LG_ES(sdt), 0), (uint32_t)a, (uint32_t)(a >> 32), 0);
+      push(DVM_LK_W0(sdt > DVM_DT_BF16 ? DVM_LK_STGI : DVM_LK_STG, sdt == DVM_DT_I32 ? 1 : sdt == DVM_DT_U8 ? 2 : 0, DVM_DT_LG_ES(sdt), tag), (uint32_t)a, (uint32_t)(a >> 32), 0);
     } else if (op == DVM_OP_STA) {
       push(DVM_LK_W0(DVM_LK_STA, 0, 0, 0), (lt[ia] & 0xffffu) * DVM_LOCAL_UNIT, 0, 0);
     } else if (op == DVM_OP_LSS) {
       push(DVM_LK_W0(DVM_LK_LSS, 0, ia, 0), scalar_unit * DVM_LOCAL_UNIT + (ib >> 2) * (DVM_VM_THREADS * 16) + (ib & 3) * 4, 0, 0);
     } else if (op == DVM_OP_STS) {
-      push(DVM_LK_W0(DVM_LK_STS, 0, ia, 0), DVM_HDR_WORDS + 2 * nt + ib * DVM_OPD_WORDS, 0, 0);
+      push(DVM_LK_W0(DVM_LK_STS, 0, ia, tag), DVM_HDR_WORDS + 2 * nt + ib * DVM_OPD_WORDS, 0, 0);
     } else if (op == DVM_OP_BCS) {
       push(DVM_LK_W0(DVM_LK_BCS, 0, ia, 0), 0, 0, 0);
     } else if (op == DVM_OP_SOP) {
-      push(DVM_LK_W0(DVM_LK_SOP, ib, ia, 0), body[pc + 1], len > 2 ? body[pc + 2] : 0, len > 3 ? body[pc + 3] : 0);
+      push(DVM_LK_W0(DVM_LK_SOP, ib, ia, tag), body[pc + 1], len > 2 ? body[pc + 2] : 0, len > 3 ? body[pc + 3] : 0);
     } else if (op == DVM_OP_NOP) {
     } else {
       return 0;  // Cmp / Select / Pow ...: not the lean interpreter's
@@ -571,6 +592,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   uint64_t total_tiles = 0;
   uint32_t units = 0;
   uint32_t row_tiles = 0;
+  bool phased_basic = false;
   int V = 0;
   int ext = 0;  // the extension level the launch needs: 1 Cmp / Select / Pow / IsFinite, 2 also views
   for (int i = 0; i < n_programs; ++i) {
@@ -590,6 +612,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
       if (n_programs != 1 || use_queue || level || tile_end) return DVM_ERR_UNSUPPORTED;
       if (total_tiles > 0x7fffffffull) return DVM_ERR_TOO_LARGE;
       row_tiles = phases * c[DVM_H_COL_BLOCKS];
+      phased_basic = ext == 0;  // nothing else asks for the general interpreter: the lean one has a phased variant
       ext = 2;
     }
   }
@@ -616,6 +639,9 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   }
   // (launches with a work queue run on the general interpreter unless asked otherwise: measured faster there)
   int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked) && (!queue_asked || g_use_lean >= 2)) ? (g_use_lean ? 1 : 0) : 0;
+  // a phased program of the basic instruction set: the lean interpreter's phased variant (lean = 2), when the
+  // library has one for these elements per thread
+  if (phased_basic && !wrap && g_use_lean && dvm_vm_find_variant(V, false, true, 0, false, 2, heavy)) lean = 2;
   if (debug_mode()) lean = 0;  // the bytecode itself travels to the device, where the check kernel reads it
   uint32_t pos = 0;
   st = lean ? place_all(P, n_programs, codes, tensors, n_tensors, level, true, &pos) : DVM_ERR_UNSUPPORTED;
@@ -641,7 +667,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   P.slot_bytes = one_slot ? 0u : units * DVM_LOCAL_UNIT;
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool single = n_programs == 1 && !use_queue;
-  const DvmVmVariant* variant = pick_variant(V, large, single, ext, level != nullptr, lean, heavy);
+  const DvmVmVariant* variant = pick_variant(V, large, single, lean ? 0 : ext, level != nullptr, lean, heavy);
   if (!variant) return DVM_ERR_UNSUPPORTED;  // (24 elements per thread: encoded for a launch of its own on the basic variant)
   int occ = 0;
   st = dvm_occupancy(variant, smem, &occ);

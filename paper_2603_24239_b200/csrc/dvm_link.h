@@ -42,9 +42,12 @@ enum {
   DVM_LK_STS,                                            // store S[a] per row         w1 = operand descriptor (word offset from the program)
   DVM_LK_BCS,                                            // ACC = broadcast(S[a])
   DVM_LK_SOP,                                            // per-row scalar arithmetic  sub = kind, a = dst; w1, w2, w3 as in the bytecode
+  DVM_LK_PHASE,                                          // phased programs (DVM_OP_PHASE): the tiles of phases < a end here
   DVM_LK_N
 };
 
+// Phased programs (rows longer than a tile): the phase tag of the bytecode travels in the top four bits of record
+// word 0 (RED: bits 28..31, below them the post-operation flag; STG / STGI / STS / SOP: bits 24..27 = b).
 // record word 0
 #define DVM_LK_W0(h, sub, a, b) ((uint32_t)(h) | ((uint32_t)(sub) << 8) | ((uint32_t)(a) << 16) | ((uint32_t)(b) << 24))
 // operand word of a local register: byte offset in the slot | mode << 18 | (fp32 ? 1 : 0) << 21 | address phase << 22 | operand << 26

@@ -30,21 +30,26 @@ struct Ops {
   }
 };
 
-template <int V, int PW, bool SINGLE, bool HEAVY>
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>,
                                                          dvm::THREADS, smem);
   }
 };
+
+#define DVM_LEAN_PHASED(V, LARGE, HEAVY)                                                  \
+  {V, LARGE, 1, 0, 0, 2, HEAVY,                                                           \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY,                                                        \
@@ -67,8 +72,11 @@ const DvmVmVariant kGroup[] = {DVM_ENTRY(24, 0, 1, 0, 0), DVM_ENTRY(24, 1, 1, 0,
 constexpr int GV = DVM_INST_GROUP < 15 ? 16 : 32;
 constexpr int GL = (DVM_INST_GROUP - 13) % 2;
 const DvmVmVariant kGroup[] = {DVM_LEAN(GV, GL, 1, 0), DVM_LEAN(GV, GL, 1, 1), DVM_LEAN(GV, GL, 0, 0), DVM_LEAN(GV, GL, 0, 1)};
-#else
+#elif DVM_INST_GROUP == 17
 const DvmVmVariant kGroup[] = {DVM_LEAN(24, 0, 1, 0), DVM_LEAN(24, 0, 1, 1), DVM_LEAN(24, 1, 1, 0), DVM_LEAN(24, 1, 1, 1)};
+#else
+// phased programs (rows longer than a tile) are encoded with 32 elements per thread
+const DvmVmVariant kGroup[] = {DVM_LEAN_PHASED(32, 0, 0), DVM_LEAN_PHASED(32, 0, 1), DVM_LEAN_PHASED(32, 1, 0), DVM_LEAN_PHASED(32, 1, 1)};
 #endif
 
 }  // namespace

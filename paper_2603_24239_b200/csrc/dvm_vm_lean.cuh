@@ -153,7 +153,9 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
   return p;
 }
 
-template <int V, int PW, bool SINGLE, bool HEAVY>
+// PHASED: the variant for phased programs (rows longer than a tile, DVM_OP_PHASE; one program per launch): a CTA takes
+// a row through its phases x column blocks in order; everything it adds is behind `if constexpr (PHASED)`.
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false>
 __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
@@ -189,6 +191,8 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
   struct Rows {
     uint32_t row, col0;    // this thread's row of the dominant shape (may lie past the end), first column of the block
     int ncols;             // valid columns of that row inside the column block (0: nothing to do)
+    uint32_t phase;        // phased programs: the tile's phase, and whether its column block is the row's last
+    bool last_block;
   };
   struct Coord { uint32_t i0, i1, i2; };  // a row's coordinates over the collapsed outer dims
   auto tile_rows = [&](uint32_t prog, uint32_t local_tile) -> Rows {
@@ -198,6 +202,13 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
     const uint32_t CB = CW(prog + DVM_H_COL_BLOCKS);
     uint32_t rb = local_tile, cb = 0;
     if (CB > 1) { rb = local_tile / CB; cb = local_tile - rb * CB; }
+    if constexpr (PHASED) {  // tile -> (row, phase, column block): the row's tiles are consecutive, phase by phase
+      rb = local_tile / prm.row_tiles;
+      const uint32_t sub = local_tile - rb * prm.row_tiles;
+      r.phase = sub / CB;
+      cb = sub - r.phase * CB;
+      r.last_block = cb == CB - 1;
+    }
     const uint32_t rows = CW(prog + DVM_H_ROWS_LO);
     r.row = rb * (uint32_t)(THREADS >> lgG) + (uint32_t)(tid >> lgG);
     const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
@@ -337,6 +348,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
 
   uint32_t prog_idx = 0;
   uint32_t tile = blockIdx.x + (SINGLE ? prm.tile_begin : 0u);
+  if constexpr (PHASED) tile = blockIdx.x * prm.row_tiles;
   uint32_t iter = 0;
   int red_par = 0;
   int buf = 0;
@@ -363,7 +375,11 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
     if (use_queue && tid == 0) s_next[iter & 1] = atomicAdd(&prm.queue[0], 1u) + gridDim.x;
     __syncthreads();  // everybody is done with the previous tile: its slot may be refilled
     if (s_abort) break;
-    const uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
+    uint32_t next = use_queue ? s_next[iter & 1] : tile + gridDim.x;
+    if constexpr (PHASED) {  // the next tile of this row, or the first tile of this CTA's next row
+      next = tile + 1;
+      if (next % prm.row_tiles == 0) next += (gridDim.x - 1) * prm.row_tiles;
+    }
     ++iter;
     uint32_t next_prog_idx = prog_idx;
     if (SINGLE && one_slot) {
@@ -479,6 +495,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
 
     // ---- Algorithm 2, inner loop: the linked compute section, one record per step ----
     uint32_t rp = prog + CW(prog + DVM_H_MAGIC);  // (the launch put the records' offset where the magic word was)
+    bool stop = false;  // (phased programs: a phase marker ended this tile's walk)
     for (;;) {
       const uint4 rec = *reinterpret_cast<const uint4*>(&CW(rp));
       rp += 4;
@@ -539,6 +556,15 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
         case DVM_LK_RED: {
           // ---- row reduction (Table 1, Sum / Max / Min with N = 1) ----
           const int rop = (int)sub;
+          bool accumulate = false, finish = true;
+          if constexpr (PHASED) {
+            const uint32_t tag = rec.x >> 28;
+            if (tag) {  // the reduction belongs to one phase: it runs over that phase's blocks and completes in the last
+              if (tag - 1 != r.phase) break;
+              accumulate = r.col0 != 0;
+              finish = r.last_block;
+            }
+          }
           const bool is_sum = rop == DVM_R_SUM || rop == DVM_R_SUMSQ;
           const float ident = is_sum ? 0.f : (rop == DVM_R_MAX ? -INFINITY : INFINITY);
           if (!all_valid) sanitize(ident);
@@ -588,13 +614,22 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
             else v = ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
             red_par ^= 1;
           }
-          if (rec.x >> 24) {  // the scalar multiply-add(-unary) that followed the reduction, rounded like the separate steps
+          if constexpr (PHASED) {
+            if (accumulate) {
+              const float prev = s_S[ra][tid];
+              v = rop == DVM_R_MAX ? fmaxf(prev, v) : (rop == DVM_R_MIN ? fminf(prev, v) : prev + v);
+            }
+          }
+          if (PHASED ? (((rec.x >> 24) & 1u) != 0 && finish) : (rec.x >> 24) != 0) {  // the scalar multiply-add(-unary) that followed the reduction, rounded like the separate steps
             v = __fadd_rn(__fmul_rn(v, __uint_as_float(rec.z)), __uint_as_float(rec.w));
             if (rec.y != 0xffu) v = scalar_unary((int)rec.y, v);
           }
           s_S[lean_opaque<13>(ra)][tid] = v;
         } break;
         case DVM_LK_STG: {
+          if constexpr (PHASED) {
+            if ((rec.x >> 24) && (rec.x >> 24) - 1 != r.phase) break;  // a phased program stores in its last phase
+          }
           const int lg_es = (int)lean_opaque<54>(ra);
           const unsigned long long base = (unsigned long long)lean_opaque<14>(rec.y) | ((unsigned long long)rec.z << 32);
           const unsigned long long el0 = (unsigned long long)r.row * C + r.col0;
@@ -797,6 +832,9 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
 #undef DVM_UN_CASE
         } break;
         case DVM_LK_STGI: {  // Table 1, Cast: ACC stored as i32 (sub 1) or u8 (sub 2), converted toward zero
+          if constexpr (PHASED) {
+            if ((rec.x >> 24) && (rec.x >> 24) - 1 != r.phase) break;
+          }
           const int lg_es = (int)lean_opaque<55>(ra);
           const unsigned long long base = (unsigned long long)lean_opaque<15>(rec.y) | ((unsigned long long)rec.z << 32);
           const unsigned long long el0 = (unsigned long long)r.row * C + r.col0;
@@ -871,11 +909,19 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
           s_S[lean_opaque<57>(ra)][tid] = r.ncols > 0 ? v : 0.f;
         } break;
         case DVM_LK_STS: {
+          bool first_block = r.col0 == 0;  // a row's value is stored once: by the tile of its first column block, or ...
+          if constexpr (PHASED) {
+            const uint32_t tag = rec.x >> 24;
+            if (tag) {  // ... in a phased program by the last block of the phase that completes it
+              if (tag - 1 != r.phase || !r.last_block) break;
+              first_block = true;
+            }
+          }
           const uint32_t d = prog + lean_opaque<18>(rec.y);
           const int dt = (CW(d + DVM_OPD_INFO) >> 8) & 0xff;
           char* p = reinterpret_cast<char*>(tensor_ptr(prog, d) + (row_offset(prog, d, r) << DVM_DT_LG_ES(dt)));
           const float v = s_S[lean_opaque<58>(ra)][tid];
-          if (r.ncols > 0 && t == 0 && r.col0 == 0) {
+          if (r.ncols > 0 && t == 0 && first_block) {
             if (dt == DVM_DT_BF16) *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(v);
             else if (dt == DVM_DT_F32) *reinterpret_cast<float*>(p) = v;
             else if (dt == DVM_DT_I32) *reinterpret_cast<uint32_t*>(p) = store_i32(v);
@@ -886,7 +932,16 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
           const float v = s_S[lean_opaque<19>(ra)][tid];
           DVM_EACH_PAIR A[i] = make_float2(v, v);
         } break;
+        case DVM_LK_PHASE: {
+          if constexpr (PHASED) {
+            if (r.phase < ra) stop = true;  // the tiles of the earlier phases end here
+          }
+        } break;
         case DVM_LK_SOP: {
+          if constexpr (PHASED) {
+            const uint32_t tag = rec.x >> 24;
+            if (tag && (tag - 1 != r.phase || !r.last_block)) break;  // once, when its operands are complete
+          }
           const uint32_t ry = lean_opaque<20>(rec.y);
           const int s1 = (ry >> 8) & 0xff, s2 = (ry >> 16) & 0xff, sop = ry & 0xff;
           const float x = s_S[s1][tid];
@@ -901,6 +956,9 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
         default:
           err = ST_BAD_CODE;
           break;
+      }
+      if constexpr (PHASED) {
+        if (stop) break;
       }
       }
       if (err == ST_BAD_CODE) break;

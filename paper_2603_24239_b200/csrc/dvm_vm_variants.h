@@ -15,7 +15,8 @@ struct DvmVmVariant {
   int single;   // 1: one program per launch (dvm_launch)
   int ext;      // 0 basic, 1 + Cmp / Select / Pow / IsFinite, 2 + views
   int levels;   // 1: stacked launch with waits between dependent levels
-  int lean;     // 1: the lean kernel for the basic instruction set (no level waits, no wrap-around rows)
+  int lean;     // 1: the lean kernel for the basic instruction set (no level waits, no wrap-around rows); 2: its variant
+                // for phased programs (rows longer than a tile, DVM_OP_PHASE; one program per launch)
   int heavy;    // unary functions log / erf / tanh / sqrt / floor / round on tiles: 1 present, 0 absent (lean only)
   // launches the kernel; `params` points at a dvm::VMParams<PW> of the variant's block size
   cudaError_t (*launch)(const void* params, int grid, size_t smem, cudaStream_t stream);

@@ -19,6 +19,15 @@ def _softmax(dtype):
     return p
 
 
+@pytest.fixture(autouse=True, params=["lean", "general"])
+def interpreter(request):
+    """Phased programs of the basic instruction set run on the lean interpreter's phased variant; with the lean
+    kernel switched off, on the general interpreter: both against the oracle."""
+    dvm.set_lean_kernel(request.param == "lean")
+    yield request.param
+    dvm.set_lean_kernel(True)
+
+
 def _phases(code):
     for line in dvm.disassemble(code).splitlines():
         if " phases " in line:
