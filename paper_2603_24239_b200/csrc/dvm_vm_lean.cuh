@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
     bool last_block;
   };
   struct Coord { uint32_t i0, i1, i2; };  // a row's coordinates over the collapsed outer dims
-  auto tile_rows = [&](uint32_t prog, uint32_t local_tile) -> Rows {
+  auto tile_rows = [&](uint32_t prog, uint32_t local_tile, int as_tid) -> Rows {
     Rows r;
     const uint32_t geom = CW(prog + DVM_H_GEOM);
     const int lgG = geom & 0xff;
@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
       r.last_block = cb == CB - 1;
     }
     const uint32_t rows = CW(prog + DVM_H_ROWS_LO);
-    r.row = rb * (uint32_t)(THREADS >> lgG) + (uint32_t)(tid >> lgG);
+    r.row = rb * (uint32_t)(THREADS >> lgG) + (uint32_t)(as_tid >> lgG);
     const uint32_t ctile = CW(prog + DVM_H_COL_TILE);
     r.col0 = cb * ctile;
     const uint32_t cend = (r.row == rows - 1) ? CW(prog + DVM_H_LAST_ROW_COLS) : CW(prog + DVM_H_COLS);
@@ -263,13 +263,17 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
     const int t = tid & ((1 << lgG) - 1);
     const bool by_row = ((geom >> 24) & DVM_F_LOADS_BY_ROW) != 0;
     const bool scalars = ((CW(prog + DVM_H_LOCAL) >> 16) & 0xff) != 0;
-    if (tid == 0 || scalars || (by_row && t == 0)) {
-      const Rows r = tile_rows(prog, local_tile);
+    const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
+    // A program whose copies are all thread 0's (dense tiles, row vectors): the lanes of warp 0 take one load
+    // instruction each, as thread 0 would -- the warp walks the load section once, not once per instruction.
+    const bool by_lane = !scalars && !by_row;
+    if (by_lane ? (warp == 0 && (uint32_t)lane < load_words) : (tid == 0 || scalars || (by_row && t == 0))) {
+      const int me = by_lane ? 0 : tid;  // (the thread whose part of the tile this thread copies)
+      const Rows r = tile_rows(prog, local_tile, me);
       const uint32_t opd0 = opd_base(prog), lreg0 = lreg_base(prog), body0 = body_base(prog);
-      const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
       const uint32_t sb = slot_base(slot);
       const int Vv = V;
-      for (uint32_t pc = 0; pc < load_words; ++pc) {
+      for (uint32_t pc = by_lane ? (uint32_t)lane : 0u; pc < (by_lane ? (uint32_t)lane + 1u : load_words); ++pc) {
         const uint32_t w0 = CW(body0 + pc);
         const uint32_t d = opd0 + DVM_INSN_B(w0) * DVM_OPD_WORDS;
         const uint32_t lg_es = ((CW(d + DVM_OPD_INFO) >> 8) & 0xff) == DVM_DT_BF16 ? 1 : 2;
@@ -280,7 +284,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
           unsigned long long a = 0, n_el = 0;
           bool mine = false;
           if (mode == DVM_LM_BLOCK) {
-            if (tid == 0) {  // thread 0's row is the tile's first: the whole tile is one byte range from there
+            if (me == 0) {  // thread 0's row is the tile's first: the whole tile is one byte range from there
               mine = true;
               const uint32_t rows = CW(prog + DVM_H_ROWS_LO), C = CW(prog + DVM_H_COLS);
               const uint32_t rv = min((uint32_t)(THREADS >> lgG), rows - r.row);
@@ -296,7 +300,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
               dst += (uint32_t)(tid >> lgG) * DVM_ROW_PITCH(1 << lgG, Vv, 1u << lg_es);
             }
           } else {  // a row vector: the same for every tile (BCAST: loaded once per slot and program) or column block
-            if ((first_of_program || mode == DVM_LM_BCAST_TILE) && tid == 0) {
+            if ((first_of_program || mode == DVM_LM_BCAST_TILE) && me == 0) {
               mine = true;
               a = r.col0;
               n_el = min(CW(prog + DVM_H_COLS) - r.col0, CW(prog + DVM_H_COL_TILE));
@@ -410,7 +414,7 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
 
     // ---- this tile: rows, shift, slot masks, where this thread's chunks lie ----
     const uint32_t prog = SINGLE ? kSingleProg : CW(prog_idx);
-    const Rows r = tile_rows(prog, SINGLE ? tile : tile - CW(n_prog + prog_idx));
+    const Rows r = tile_rows(prog, SINGLE ? tile : tile - CW(n_prog + prog_idx), tid);
     const uint32_t geom = CW(prog + DVM_H_GEOM);
     const int lgG = geom & 0xff;
     const int lgW = ((geom >> 8) & 0xff) == 8 ? 3 : 2;
