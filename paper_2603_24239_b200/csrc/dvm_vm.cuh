@@ -413,7 +413,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
     }
     const uint32_t sb = slot_base(slot);
     const int t = tid & ((1 << c.lgG) - 1);
-    for (uint32_t pc = 0; pc < load_words; ++pc) {
+    // When every copy of the tile is thread 0's (dense tiles, row vectors), the lanes of warp 0 take one load
+    // instruction each, as thread 0 would: the warp walks the load section once, in parallel.  What the issuing warp
+    // spends here, the other warps wait for at the tile's next barrier.
+    const bool by_lane = !(c.flags & DVM_F_LOADS_BY_ROW);
+    const uint32_t row0 = c.row - (uint32_t)(tid >> c.lgG);  // the tile's first row
+    for (uint32_t pc = by_lane ? (uint32_t)lane : 0u; pc < (by_lane ? min((uint32_t)lane + 1u, load_words) : load_words); ++pc) {
       const uint32_t w0 = CW(body0 + pc);
       const uint32_t d = opd0 + DVM_INSN_B(w0) * DVM_OPD_WORDS;
       if (DVM_INSN_OP(w0) == DVM_OP_LDG) {
@@ -450,13 +455,13 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             dst += (uint32_t)tid * DVM_STRIP_PITCH(R, 1u << lg_es);
           }
         } else if (mode == DVM_LM_BLOCK) {
-          if (tid == 0) {  // thread 0's row is the tile's first row: the whole tile is one byte range from there
+          if (by_lane || tid == 0) {  // the tile's first row: the whole tile is one byte range from there
             mine = true;
             const uint32_t rows = CW(prog + DVM_H_ROWS_LO), C = CW(prog + DVM_H_COLS);
             const uint32_t R = (uint32_t)(THREADS >> c.lgG);
-            const uint32_t rv = min(R, rows - c.row);
-            const uint32_t last = (c.row + rv == rows) ? CW(prog + DVM_H_LAST_ROW_COLS) : C;
-            a = (unsigned long long)c.row * C;
+            const uint32_t rv = min(R, rows - row0);
+            const uint32_t last = (row0 + rv == rows) ? CW(prog + DVM_H_LAST_ROW_COLS) : C;
+            a = (unsigned long long)row0 * C;
             n_el = (unsigned long long)(rv - 1) * C + last;
           }
         } else if (mode == DVM_LM_ROWS) {
@@ -467,7 +472,7 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
             dst += (uint32_t)(tid >> c.lgG) * DVM_ROW_PITCH(1 << c.lgG, V, 1u << lg_es);
           }
         } else {  // DVM_LM_BCAST: the same row for every tile of the program; DVM_LM_BCAST_TILE: of its column block
-          if ((first_of_program || mode == DVM_LM_BCAST_TILE) && tid == 0) {
+          if ((first_of_program || mode == DVM_LM_BCAST_TILE) && (by_lane || tid == 0)) {
             mine = true;
             a = c.col0;
             n_el = min(CW(prog + DVM_H_COLS) - c.col0, CW(prog + DVM_H_COL_TILE));
