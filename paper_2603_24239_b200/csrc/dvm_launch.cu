@@ -309,9 +309,23 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       push(DVM_LK_W0(DVM_LK_BCS, 0, ia, 0), 0, 0, 0);
     } else if (op == DVM_OP_SOP) {
       push(DVM_LK_W0(DVM_LK_SOP, ib, ia, tag), body[pc + 1], len > 2 ? body[pc + 2] : 0, len > 3 ? body[pc + 3] : 0);
+    } else if (op >= DVM_OP_CMP && op <= DVM_OP_CMP + DVM_C_NE) {
+      // Table 1, Cmp against an fp32 image, a temporary or the accumulator itself (bf16 images, Pow: general interpreter)
+      if (ia == DVM_REG_ACC) {
+        push(DVM_LK_W0(DVM_LK_CMP, op - DVM_OP_CMP, 3, 0), 0, 0, 0);
+      } else {
+        const uint32_t oy = opw(ia, ib, &kind);
+        if (kind == 0) return 0;
+        push(DVM_LK_W0(DVM_LK_CMP, op - DVM_OP_CMP, kind, 0), oy, 0, 0);
+      }
+    } else if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) {
+      int kp = 0, kq = 0;
+      const uint32_t op_ = opw(ia, (ib >> 6) & 1, &kp), oq = opw(ib & 0x3f, (ib >> 7) & 1, &kq);
+      if (kp == 0 || kq == 0) return 0;
+      push(DVM_LK_W0(DVM_LK_SEL, op - DVM_OP_SEL, (uint32_t)kp | ((uint32_t)kq << 2), 0), op_, oq, 0);
     } else if (op == DVM_OP_NOP) {
     } else {
-      return 0;  // Cmp / Select / Pow ...: not the lean interpreter's
+      return 0;  // Pow, IsFinite, Cmp / Select on bf16 images: not the lean interpreter's
     }
     pc += len;
   }
@@ -453,6 +467,7 @@ void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* h
           u == DVM_U_TRUNC_I32 || u == DVM_U_TRUNC_U8) *heavy = true;
     }
     if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) *heavy = true;
+    if (op >= DVM_OP_CMP && op < DVM_OP_SEL + 3) *heavy = true;  // (Cmp / Select: in the HEAVY variants of the lean kernel)
     pc += len ? len : 1;
   }
 }
@@ -638,7 +653,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     program_traits((const uint32_t*)codes[i], tensors[i], &wrap, &heavy);
   }
   // (launches with a work queue run on the general interpreter unless asked otherwise: measured faster there)
-  int lean = (ext == 0 && !level && !wrap && !(one_slot && queue_asked) && (!queue_asked || g_use_lean >= 2)) ? (g_use_lean ? 1 : 0) : 0;
+  int lean = (ext <= 1 && !level && !wrap && !(one_slot && queue_asked) && (!queue_asked || g_use_lean >= 2)) ? (g_use_lean ? 1 : 0) : 0;
   // a phased program of the basic instruction set: the lean interpreter's phased variant (lean = 2), when the
   // library has one for these elements per thread
   if (phased_basic && !wrap && g_use_lean && dvm_vm_find_variant(V, false, true, 0, false, 2, heavy)) lean = 2;

@@ -43,6 +43,10 @@ enum {
   DVM_LK_BCS,                                            // ACC = broadcast(S[a])
   DVM_LK_SOP,                                            // per-row scalar arithmetic  sub = kind, a = dst; w1, w2, w3 as in the bytecode
   DVM_LK_PHASE,                                          // phased programs (DVM_OP_PHASE): the tiles of phases < a end here
+  DVM_LK_CMP,                                            // ACC = ACC cmp Y ? 1 : 0 (Table 1, Cmp)   sub = relation, a = kind of Y (1 fp32 image,
+                                                         //   2 private, 3 ACC itself), w1 = operand word                 (HEAVY variants)
+  DVM_LK_SEL,                                            // Table 1, Select         sub = form (as DVM_OP_SEL + form), a = kind(p) | kind(q) << 2,
+                                                         //   w1, w2 = operand words of p and q                          (HEAVY variants)
   DVM_LK_N
 };
 

@@ -18,6 +18,8 @@
 //   * the heavy unary functions (log, erf, tanh, sqrt, floor, round) exist only in the HEAVY variant, so the
 //     hot loop of the programs that do not use them stays small.
 #pragma once
+#include <type_traits>
+
 #include "dvm_link.h"
 #include "dvm_vm.cuh"
 
@@ -935,6 +937,74 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
         case DVM_LK_BCS: {
           const float v = s_S[lean_opaque<19>(ra)][tid];
           DVM_EACH_PAIR A[i] = make_float2(v, v);
+        } break;
+        case DVM_LK_CMP:
+        case DVM_LK_SEL: {
+          // Table 1, Cmp and Select (HEAVY variants): operands are fp32 images or temporaries, read in two halves
+          if constexpr (HEAVY) {
+            // half H of the register an operand word names (kind 1: fp32 image, 2: thread-private temporary) into pairs Y
+#define DVM_LOAD_HALF(H, OW, KIND, Y)                                                                           \
+            if ((KIND) == 2u) {                                                                                   \
+              const uint32_t a_ = sb + ((OW) & 0x3ffffu) + (uint32_t)tid * 16;                                    \
+              _Pragma("unroll") for (int q = 0; q < V / 8; ++q) {                                                 \
+                const uint4 v = lean_lds128(a_ + (uint32_t)((H) * (V / 8) + q) * PSTRIDE);                        \
+                Y[2 * q] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));                               \
+                Y[2 * q + 1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));                           \
+              }                                                                                                   \
+            } else {                                                                                              \
+              const uint32_t a_ = opw_addr(OW);                                                                   \
+              uint32_t R[V / 2];                                                                                  \
+              if (lgW == 3) lean_raw_f32<2, (H) * (V / 16), ((H) + 1) * (V / 16)>(R, a_, (uint32_t)(G << 5));     \
+              else lean_raw_f32<1, (H) * (V / 8), ((H) + 1) * (V / 8)>(R, a_, (uint32_t)(G << 4));                \
+              _Pragma("unroll") for (int i = 0; i < VP / 2; ++i)                                                  \
+                Y[i] = make_float2(__uint_as_float(R[2 * i]), __uint_as_float(R[2 * i + 1]));                     \
+            }
+            if (h == DVM_LK_CMP) {
+#define DVM_CMP_HALF(H)                                                                                          \
+              {                                                                                                   \
+                float2 Y[VP / 2];                                                                                 \
+                if (ra == 3u) { _Pragma("unroll") for (int i = 0; i < VP / 2; ++i) Y[i] = A[(H) * (VP / 2) + i]; } \
+                else { DVM_LOAD_HALF(H, rec.y, ra, Y) }                                                           \
+                _Pragma("unroll") for (int i = 0; i < VP / 2; ++i) {                                              \
+                  float2& a = A[(H) * (VP / 2) + i];                                                              \
+                  bool bx, by;                                                                                    \
+                  switch (sub) {                                                                                  \
+                    case DVM_C_GT: bx = a.x > Y[i].x; by = a.y > Y[i].y; break;                                   \
+                    case DVM_C_GE: bx = a.x >= Y[i].x; by = a.y >= Y[i].y; break;                                 \
+                    case DVM_C_LT: bx = a.x < Y[i].x; by = a.y < Y[i].y; break;                                   \
+                    case DVM_C_LE: bx = a.x <= Y[i].x; by = a.y <= Y[i].y; break;                                 \
+                    case DVM_C_EQ: bx = a.x == Y[i].x; by = a.y == Y[i].y; break;                                 \
+                    default: bx = a.x != Y[i].x; by = a.y != Y[i].y; break;                                       \
+                  }                                                                                               \
+                  a = make_float2(bx ? 1.f : 0.f, by ? 1.f : 0.f);                                                \
+                }                                                                                                 \
+              }
+              DVM_CMP_HALF(0)
+              DVM_CMP_HALF(1)
+#undef DVM_CMP_HALF
+            } else {
+              // sub 0: ACC = ACC != 0 ? L[p] : L[q];  1: ACC = L[p] != 0 ? L[q] : ACC;  2: ACC = L[p] != 0 ? ACC : L[q]
+              const uint32_t kp = ra & 3u, kq = (ra >> 2) & 3u;
+#define DVM_SEL_HALF(H)                                                                                          \
+              {                                                                                                   \
+                float2 P[VP / 2], Q[VP / 2];                                                                      \
+                DVM_LOAD_HALF(H, rec.y, kp, P)                                                                    \
+                DVM_LOAD_HALF(H, rec.z, kq, Q)                                                                    \
+                _Pragma("unroll") for (int i = 0; i < VP / 2; ++i) {                                              \
+                  float2& a = A[(H) * (VP / 2) + i];                                                              \
+                  if (sub == 0u) a = make_float2(a.x != 0.f ? P[i].x : Q[i].x, a.y != 0.f ? P[i].y : Q[i].y);     \
+                  else if (sub == 1u) a = make_float2(P[i].x != 0.f ? Q[i].x : a.x, P[i].y != 0.f ? Q[i].y : a.y); \
+                  else a = make_float2(P[i].x != 0.f ? a.x : Q[i].x, P[i].y != 0.f ? a.y : Q[i].y);               \
+                }                                                                                                 \
+              }
+              DVM_SEL_HALF(0)
+              DVM_SEL_HALF(1)
+#undef DVM_SEL_HALF
+            }
+#undef DVM_LOAD_HALF
+          } else {
+            err = ST_BAD_CODE;
+          }
         } break;
         case DVM_LK_PHASE: {
           if constexpr (PHASED) {
