@@ -201,6 +201,9 @@ enum {
                        //   0x58: ACC = ACC != 0 ? L[p] : L[q]     (the condition is in the accumulator)
                        //   0x59: ACC = L[p] != 0 ? L[q] : ACC     (the else-value is in the accumulator)
                        //   0x5a: ACC = L[p] != 0 ? ACC : L[q]     (the then-value is in the accumulator)
+                       //   0x5b: ACC = ACC != 0 ? imm1 : imm2     (len 3; pattern-based fusion, Sec. 5.1: a Select between two
+                       //         scalar multiples (or offsets) of ONE value x is x times (plus) the selected scalar --
+                       //         no temporaries for the two candidates, bit-identical results)
   DVM_OP_LAST = 0x60   // every arithmetic class starts at a multiple of 8: the low 3 bits are the operation
 };
 #define DVM_REG_ACC 0xff

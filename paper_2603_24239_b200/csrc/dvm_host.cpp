@@ -311,6 +311,9 @@ struct Enc {
   int8_t act_of[DVM_MAX_NODES];   // -1, or the fused activation (DVM_ACT_*) this node is the result of
   int16_t act_src[DVM_MAX_NODES]; // ... applied to this value
   bool act_part[DVM_MAX_NODES];   // an inner node of a fused activation chain: never materialises
+  int16_t sel_src[DVM_MAX_NODES]; // -1, or: this Select chooses between two scalar multiples / offsets of value sel_src
+  uint8_t sel_ar[DVM_MAX_NODES];  // ... DVM_A_MUL or DVM_A_ADD
+  float sel_imm[DVM_MAX_NODES][2];
   int16_t n_cons[DVM_MAX_NODES];  // number of consuming nodes / outputs of a value
   int16_t one_cons[DVM_MAX_NODES];// the consuming node when there is exactly one (and it is a node)
   int lda_pos;                    // body position of the LDA just emitted by ensure_acc, or -1
@@ -515,6 +518,28 @@ static bool gen_body(Enc& e) {
     }
   }
 
+  // Select(c, x * a, x * b) = x * Select(c, a, b), and the same with + : the two candidates never materialise
+  for (int i = 0; i < p->n_nodes; ++i) e.sel_src[i] = -1;
+  for (int i = 0; i < p->n_nodes; ++i) {
+    const Node& n = p->nodes[i];
+    if (n.kind != NK_SELECT || e.alias[i] >= 0 || e.cls[i] != CLS_TILE) continue;
+    const int c = root(e, n.x), u = root(e, n.y), v = root(e, n.param);
+    const Node& un = p->nodes[u];
+    const Node& vn = p->nodes[v];
+    if (u == v || un.kind != NK_SCALAR || vn.kind != NK_SCALAR || un.op != vn.op || e.uses[u] != 1 || e.uses[v] != 1 ||
+        e.act_part[u] || e.act_part[v] || e.alias[u] >= 0 || e.alias[v] >= 0 || e.cls[u] != CLS_TILE || e.cls[v] != CLS_TILE)
+      continue;
+    const int x = root(e, un.x);
+    if (x != root(e, vn.x) || x == c || e.cls[x] != CLS_TILE || e.cls[c] != CLS_TILE || p->nodes[x].kind != NK_INPUT) continue;
+    e.sel_src[i] = (int16_t)x;
+    e.sel_ar[i] = un.op == DVM_ADDS ? DVM_A_ADD : DVM_A_MUL;
+    e.sel_imm[i][0] = un.param >= 0 ? e.scalars[un.param] : un.imm;
+    e.sel_imm[i][1] = vn.param >= 0 ? e.scalars[vn.param] : vn.imm;
+    e.act_part[u] = e.act_part[v] = true;  // (skipped like the inner nodes of a fused activation)
+    e.uses[u] = e.uses[v] = 0;
+    e.uses[x] -= 1;                        // x fed both candidates: the fused form reads it once
+  }
+
   // consumers of every value (for the scalar multiply-add fusion below)
   for (int i = 0; i < p->n_nodes; ++i) { e.n_cons[i] = 0; e.one_cons[i] = -1; e.fused_sc[i] = false; }
   for (int i = 0; i < p->n_nodes; ++i) {
@@ -687,6 +712,23 @@ static bool gen_body(Enc& e) {
       e.acc = (int16_t)i;
       release(e, a);
       if (b != a) release(e, b);
+    } else if (n.kind == NK_SELECT && e.sel_src[i] >= 0) {
+      // the scalar is selected in the accumulator, then applied to x (an input: it has a local register)
+      const int xs = e.sel_src[i];
+      if (e.lreg_of[xs] < 0) { e.fail = true; break; }
+      ensure_acc(e, x);
+      if (e.fail) break;
+      e.uses[x]--;
+      spill_acc_if_live(e);
+      if (e.fail) break;
+      emit(e, DVM_INSN(DVM_OP_SEL + 3, 3, 0, 0));
+      emit(e, f2u(e.sel_imm[i][0]));
+      emit(e, f2u(e.sel_imm[i][1]));
+      emit(e, DVM_INSN(DVM_OP_BIN + e.sel_ar[i], 1, e.lreg_of[xs], e.ldt_of[xs]));
+      e.uses[xs]--;
+      e.acc = (int16_t)i;
+      release(e, x);
+      release(e, xs);
     } else if (n.kind == NK_SELECT) {
       // one of {condition, then-value, else-value} stays in (or moves to) the accumulator, the other two are
       // read from local registers
@@ -1638,6 +1680,7 @@ static int insn_expected_len(uint32_t op, uint32_t w0) {
   if (op >= DVM_OP_LD2 && op < DVM_OP_LD2 + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_CMP && op < DVM_OP_CMP + DVM_C_NCMP) return 1;
   if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) return 1;
+  if (op == DVM_OP_SEL + 3) return 3;
   if (op >= DVM_OP_BINI && op < DVM_OP_BINI + DVM_A_NBIN) return 2;
   if (op >= DVM_OP_BIN && op < DVM_OP_BIN + DVM_A_NBIN) return 1;
   if (op >= DVM_OP_BINS && op < DVM_OP_BINS + DVM_A_NBIN) return 1;
@@ -1921,6 +1964,12 @@ extern "C" int dvm_disassemble(const void* code, size_t code_size, char* buf, si
       static const char* kCmp[DVM_C_NCMP] = {"cmp.gt", "cmp.ge", "cmp.lt", "cmp.le", "cmp.eq", "cmp.ne", "pow", "rpow"};
       if (a == DVM_REG_ACC) outf(o, "%-9s acc, acc, acc\n", kCmp[op - DVM_OP_CMP]);
       else outf(o, "%-9s acc, acc, l%u%s\n", kCmp[op - DVM_OP_CMP], a, dts);
+    }
+    else if (op == DVM_OP_SEL + 3) {
+      float i1, i2;
+      memcpy(&i1, &b[pc + 1], 4);
+      memcpy(&i2, &b[pc + 2], 4);
+      outf(o, "select    acc, acc ? %.9g : %.9g\n", i1, i2);
     }
     else if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) {
       const char* s1 = ((bb >> 6) & 1) ? ".bf16" : "";

@@ -318,6 +318,8 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
         if (kind == 0) return 0;
         push(DVM_LK_W0(DVM_LK_CMP, op - DVM_OP_CMP, kind, 0), oy, 0, 0);
       }
+    } else if (op == DVM_OP_SEL + 3) {
+      push(DVM_LK_W0(DVM_LK_SEL, 3, 0, 0), body[pc + 1], body[pc + 2], 0);
     } else if (op >= DVM_OP_SEL && op < DVM_OP_SEL + 3) {
       int kp = 0, kq = 0;
       const uint32_t op_ = opw(ia, (ib >> 6) & 1, &kp), oq = opw(ib & 0x3f, (ib >> 7) & 1, &kq);
@@ -467,7 +469,7 @@ void program_traits(const uint32_t* w, void* const* tensors, bool* wrap, bool* h
           u == DVM_U_TRUNC_I32 || u == DVM_U_TRUNC_U8) *heavy = true;
     }
     if (op >= DVM_OP_ACT && op < DVM_OP_ACT + DVM_ACT_N) *heavy = true;
-    if (op >= DVM_OP_CMP && op < DVM_OP_SEL + 3) *heavy = true;  // (Cmp / Select: in the HEAVY variants of the lean kernel)
+    if (op >= DVM_OP_CMP && op <= DVM_OP_SEL + 3) *heavy = true;  // (Cmp / Select: in the HEAVY variants of the lean kernel)
     pc += len ? len : 1;
   }
 }

@@ -1258,6 +1258,12 @@ __global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const 
           const int ib = DVM_INSN_B(w0);
           const int dt1 = (ib >> 6) & 1, dt2 = (ib >> 7) & 1;
           const int form = op & 7;
+          if (form == 3) {  // ACC = ACC != 0 ? imm1 : imm2
+            const float i1 = __uint_as_float(CW(pc)), i2 = __uint_as_float(CW(pc + 1));
+            pc += 2;
+            DVM_EACH_PAIR A[i] = make_float2(A[i].x != 0.f ? i1 : i2, A[i].y != 0.f ? i1 : i2);
+            break;
+          }
           float2 Y[VP];
           unsigned long long m = 0;
           if (form == 0) {  // ACC = ACC != 0 ? L[p] : L[q]

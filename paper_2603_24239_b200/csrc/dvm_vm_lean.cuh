@@ -982,6 +982,9 @@ __global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel
               DVM_CMP_HALF(0)
               DVM_CMP_HALF(1)
 #undef DVM_CMP_HALF
+            } else if (sub == 3u) {  // ACC = ACC != 0 ? imm1 : imm2
+              const float i1 = __uint_as_float(rec.y), i2 = __uint_as_float(rec.z);
+              DVM_EACH_PAIR A[i] = make_float2(A[i].x != 0.f ? i1 : i2, A[i].y != 0.f ? i1 : i2);
             } else {
               // sub 0: ACC = ACC != 0 ? L[p] : L[q];  1: ACC = L[p] != 0 ? L[q] : ACC;  2: ACC = L[p] != 0 ? ACC : L[q]
               const uint32_t kp = ra & 3u, kq = (ra >> 2) & 3u;

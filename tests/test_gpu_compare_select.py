@@ -147,3 +147,26 @@ def test_if_else_add_many_tiles_single_slot_launch():
     want = oracle_run(prog, [s.reshape(1, len(rows), shape[2]) for s in sub])[0]
     got = wl.to_f64(out.reshape(-1, shape[2])[rows])
     assert float(np.max(np.abs(got - want[0]) / np.maximum(np.abs(want[0]), 1e-30))) <= 1e-6   # the oracle does not round to fp32
+
+
+@pytest.mark.parametrize("kind", ["muls", "adds", "mixed"])
+def test_select_between_scalar_multiples_of_one_value(kind):
+    """Select(c, x * a, x * b) is encoded as x * Select(c, a, b) (one instruction on the accumulator, no temporaries
+    for the candidates; the same with +); candidates of different kinds keep the general form.  Exact either way."""
+    p = wl.OpProgram("affine_select")
+    a, b, x = p.input("f32", 2), p.input("f32", 2), p.input("f32", 2)
+    c = p.compare("le", a, b)
+    if kind == "muls":
+        u, v = p.scalar("muls", x, 3.0), p.scalar("muls", x, -0.5)
+    elif kind == "adds":
+        u, v = p.scalar("adds", x, 3.0), p.scalar("adds", x, -0.5)
+    else:
+        u, v = p.scalar("muls", x, 3.0), p.scalar("adds", x, -0.5)
+    p.output(p.select(c, u, v), "f32")
+    ins = [wl.randn((37, 1001), torch.float32, 51), wl.randn((37, 1001), torch.float32, 52), wl.randn((37, 1001), torch.float32, 53)]
+    outs, code = gpu_run(p, ins)
+    text = dvm.disassemble(code)
+    assert ("acc ? 3 : -0.5" in text) == (kind != "mixed")
+    want = oracle_run(p, ins)
+    # one fp32 rounding per element on the device; the oracle's float64 product / sum is exact, rounded here
+    assert np.array_equal(wl.to_f64(outs[0]), want[0].astype(np.float32).astype(np.float64))
