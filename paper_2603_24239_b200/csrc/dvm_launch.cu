@@ -63,12 +63,12 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
 
-const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy) {
+const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy, int ctas) {
   typedef const DvmVmVariant* (*GroupFn)(int*);
 #define DVM_GROUP_FN(g) &dvm_vm_group_##g,
   static const GroupFn groups[] = {DVM_GROUPS(DVM_GROUP_FN)};
@@ -78,7 +78,7 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
     const DvmVmVariant* v = g(&n);
     for (int i = 0; i < n; ++i)
       if (v[i].V == V && v[i].large == (int)large && v[i].single == (int)single && v[i].ext == ext &&
-          v[i].levels == (int)levels && v[i].lean == lean && (!lean || v[i].heavy == (int)heavy))
+          v[i].levels == (int)levels && v[i].lean == lean && (!lean || v[i].heavy == (int)heavy) && v[i].ctas == ctas)
         return &v[i];
   }
   return nullptr;
@@ -87,7 +87,8 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
 // Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
 uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
   const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
-                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 15);  // (lean: two bits)
+                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 15) |  // (lean: two bits)
+                      ((uint64_t)v->ctas << 16);
   return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
 }
 
@@ -685,6 +686,12 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   if (smem > kMaxDynSmem) return DVM_ERR_TOO_LARGE;
   const bool single = n_programs == 1 && !use_queue;
   const DvmVmVariant* variant = pick_variant(V, large, single, lean ? 0 : ext, level != nullptr, lean, heavy);
+  if (one_slot && variant && 3 * (smem + 9600) <= 233472) {
+    // one tile slot per CTA, and three such CTAs fit an SM: the kernel compiled for three (where the library has it)
+    const DvmVmVariant* v3 = dvm_vm_find_variant(V, large, variant->single != 0, variant->ext, variant->levels != 0, variant->lean,
+                                                 variant->heavy != 0, 3);
+    if (v3) variant = v3;
+  }
   if (!variant) return DVM_ERR_UNSUPPORTED;  // (24 elements per thread: encoded for a launch of its own on the basic variant)
   int occ = 0;
   st = dvm_occupancy(variant, smem, &occ);

@@ -245,8 +245,10 @@ static __device__ __noinline__ float vm_pow(float a, float b) { return powf(a, b
 // DVM_F_EXT_ISA); 2: that, plus gathered inputs and tile stores into strided views (DVM_F_VIEWS).  The basic
 // variant (0) stays as compact as it is without them, and variant 1 without the view code.
 // LEVELS: the stacked variant with in-kernel waits between dependent levels (dvm_launch_stacked_levels).
-template <int V, int PW, bool SINGLE, int EXT, bool LEVELS = false>
-__global__ void __launch_bounds__(THREADS, DVM_VM_MIN_CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
+// CTAS: resident CTAs per SM the kernel is compiled for (2; 3 for the one-slot launches of the level-wait variant,
+// whose CTAs wait for their own tile: a third CTA is worth more there than the registers it costs).
+template <int V, int PW, bool SINGLE, int EXT, bool LEVELS = false, int CTAS = DVM_VM_MIN_CTAS>
+__global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr bool VIEWS = EXT >= 2;
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register

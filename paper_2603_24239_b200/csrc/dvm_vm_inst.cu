@@ -3,69 +3,90 @@
 // each with the one-program, the stacked and the level-wait variant; group 12: the 24-element one-program
 // basic variants; groups 13..16: the lean kernel for V = 16 (13, 14) or 32, parameter block small (13, 15) or
 // large, each one-program / stacked, with and without the heavy unary functions; group 17: the lean kernel with
-// 24 elements per thread (one program).
+// 24 elements per thread (one program); group 18: the lean kernel for phased programs; groups 19..30: the level-wait
+// variant of groups 0..11 compiled for three resident CTAs per SM; group 31: the one-program lean kernel, 16 elements
+// per thread, compiled for three.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..17>"
+#error "compile with -DDVM_INST_GROUP=<0..31>"
 #endif
 
 namespace {
 
-template <int V, int PW, bool SINGLE, int EXT, bool LEVELS>
+template <int V, int PW, bool SINGLE, int EXT, bool LEVELS, int CTAS = DVM_VM_MIN_CTAS>
 struct Ops {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>
+    dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS, CTAS>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS, CTAS>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_kernel<V, PW, SINGLE, EXT, LEVELS, CTAS>,
                                                          dvm::THREADS, smem);
   }
 };
 
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false>
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>,
                                                          dvm::THREADS, smem);
   }
 };
 
 #define DVM_LEAN_PHASED(V, LARGE, HEAVY)                                                  \
-  {V, LARGE, 1, 0, 0, 2, HEAVY,                                                           \
+  {V, LARGE, 1, 0, 0, 2, HEAVY, 2,                                                        \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
-  {V, LARGE, SINGLE, 0, 0, 1, HEAVY,                                                        \
+  {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::launch, \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::occupancy}
 
 #define DVM_ENTRY(V, LARGE, SINGLE, EXT, LEVELS)                                       \
-  {V, LARGE, SINGLE, EXT, LEVELS, 0, 1,                                               \
+  {V, LARGE, SINGLE, EXT, LEVELS, 0, 1, 2,                                            \
    &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::launch, \
    &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, EXT, (LEVELS) != 0>::occupancy}
+
+// the level-wait variant compiled for three resident CTAs (one-slot launches)
+#define DVM_ENTRY3(V, LARGE, EXT)                                                      \
+  {V, LARGE, 0, EXT, 1, 0, 1, 3,                                                      \
+   &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, false, EXT, true, 3>::launch,       \
+   &Ops<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, false, EXT, true, 3>::occupancy}
+// the one-program lean kernel compiled for three resident CTAs (one-slot programs)
+#define DVM_LEAN3(V, LARGE, HEAVY)                                                          \
+  {V, LARGE, 1, 0, 0, 1, HEAVY, 3,                                                          \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 3>::launch, \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 3>::occupancy}
 
 #if DVM_INST_GROUP < 12
 constexpr int GV = DVM_INST_GROUP < 6 ? 16 : 32;
 constexpr int GL = (DVM_INST_GROUP % 6) < 3 ? 0 : 1;
 constexpr int GE = DVM_INST_GROUP % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY(GV, GL, 1, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 0), DVM_ENTRY(GV, GL, 0, GE, 1)};
+#elif DVM_INST_GROUP >= 19 && DVM_INST_GROUP < 31
+constexpr int G3 = DVM_INST_GROUP - 19;
+constexpr int GV = G3 < 6 ? 16 : 32;
+constexpr int GL = (G3 % 6) < 3 ? 0 : 1;
+constexpr int GE = G3 % 3;
+const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
+#elif DVM_INST_GROUP == 31
+const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
 #elif DVM_INST_GROUP == 12
 const DvmVmVariant kGroup[] = {DVM_ENTRY(24, 0, 1, 0, 0), DVM_ENTRY(24, 1, 1, 0, 0)};
 #elif DVM_INST_GROUP < 17

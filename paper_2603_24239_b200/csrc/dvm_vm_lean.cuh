@@ -157,8 +157,9 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
 
 // PHASED: the variant for phased programs (rows longer than a tile, DVM_OP_PHASE; one program per launch): a CTA takes
 // a row through its phases x column blocks in order; everything it adds is behind `if constexpr (PHASED)`.
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false>
-__global__ void __launch_bounds__(THREADS, DVM_LEAN_MIN_CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
+// CTAS: resident CTAs per SM the kernel is compiled for (2; 3 for one-slot programs, see dvm_vm_kernel).
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS>
+__global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
   constexpr int NG = V / 8;            // 8-slot groups of a tile register

@@ -18,6 +18,7 @@ struct DvmVmVariant {
   int lean;     // 1: the lean kernel for the basic instruction set (no level waits, no wrap-around rows); 2: its variant
                 // for phased programs (rows longer than a tile, DVM_OP_PHASE; one program per launch)
   int heavy;    // unary functions log / erf / tanh / sqrt / floor / round on tiles: 1 present, 0 absent (lean only)
+  int ctas;     // resident CTAs per SM the kernel is compiled for: 2, or 3 (variants for one-slot launches)
   // launches the kernel; `params` points at a dvm::VMParams<PW> of the variant's block size
   cudaError_t (*launch)(const void* params, int grid, size_t smem, cudaStream_t stream);
   // lifts the dynamic shared memory limit of the kernel and asks how many CTAs of it an SM holds
@@ -25,4 +26,4 @@ struct DvmVmVariant {
 };
 
 // NULL when the library has no such variant.
-const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy);
+const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext, bool levels, int lean, bool heavy, int ctas = 2);
