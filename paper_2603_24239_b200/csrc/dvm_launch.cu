@@ -225,6 +225,9 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
     return DVM_LK_OPW((lw & 0xffffu) * DVM_LOCAL_UNIT, mode, dt == DVM_DT_BF16 ? 0 : 1, (lw >> 20) & 0xfu, lw >> 24);
   };
   const float one = 1.0f, neg_one = -1.0f, neg_zero = -0.0f;
+  // handlers by kind of operand (0 bf16 image, 1 fp32 image, 2 private temporary)
+  static const uint32_t kLda[3] = {DVM_LK_LDA_BF16, DVM_LK_LDA_F32, DVM_LK_LDA_PRIV};
+  static const uint32_t kBin[3] = {DVM_LK_BIN_BF16, DVM_LK_BIN_F32, DVM_LK_BIN_PRIV};
   for (uint32_t pc = load_words; pc < code_words;) {
     if (n + 4 > sizeof rec / sizeof rec[0]) return 0;
     const uint32_t w0 = body[pc], op = DVM_INSN_OP(w0), len = DVM_INSN_LEN(w0) ? DVM_INSN_LEN(w0) : 1;
@@ -236,18 +239,18 @@ uint32_t dvm_link_program(uint32_t* dst, uint32_t at, uint32_t max_words, const 
       if (ia != 0xffu) push(DVM_LK_W0(DVM_LK_PHASE, 0, ia, 0), 0, 0, 0);
     } else if (op == DVM_OP_LDA) {
       const uint32_t ow = opw(ia, ib, &kind);
-      push(DVM_LK_W0(DVM_LK_LDA_BF16 + kind, 0, 0, 0), ow, 0, 0);
+      push(DVM_LK_W0(kLda[kind], 0, 0, 0), ow, 0, 0);
     } else if (cls == (DVM_OP_LD2 >> 3)) {
       const uint32_t ox = opw(ia, (ib >> 6) & 1, &kind);
-      push(DVM_LK_W0(DVM_LK_LDA_BF16 + kind, 0, 0, 0), ox, 0, 0);
+      push(DVM_LK_W0(kLda[kind], 0, 0, 0), ox, 0, 0);
       const uint32_t oy = opw(ib & 0x3f, (ib >> 7) & 1, &kind);
-      push(DVM_LK_W0(DVM_LK_BIN_BF16 + kind, op & 7, 0, 0), oy, 0, 0);
+      push(DVM_LK_W0(kBin[kind], op & 7, 0, 0), oy, 0, 0);
     } else if (cls == (DVM_OP_BIN >> 3)) {
       if (ia == DVM_REG_ACC) {
         push(DVM_LK_W0(DVM_LK_BIN_ACC, op & 7, 0, 0), 0, 0, 0);
       } else {
         const uint32_t oy = opw(ia, ib, &kind);
-        push(DVM_LK_W0(DVM_LK_BIN_BF16 + kind, op & 7, 0, 0), oy, 0, 0);
+        push(DVM_LK_W0(kBin[kind], op & 7, 0, 0), oy, 0, 0);
       }
     } else if (cls == (DVM_OP_BINI >> 3)) {
       const float y = u2f(body[pc + 1]);

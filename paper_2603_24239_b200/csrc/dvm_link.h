@@ -23,19 +23,23 @@
 
 enum {
   DVM_LK_END = 0,
-  DVM_LK_LDA_BF16, DVM_LK_LDA_F32, DVM_LK_LDA_PRIV,      // ACC = L[x]                 w1 = operand word
-  DVM_LK_BIN_BF16, DVM_LK_BIN_F32, DVM_LK_BIN_PRIV,      // ACC = ACC op L[y]          sub = arith, w1 = operand word; b = 1 + s: ACC * S[s] * L[y]
+  // the records of the bf16 sweeps first (DVM_LK_HOT_LAST closes the set: the interpreter tests them as a range)
   DVM_LK_LD2_BF16,                                       // ACC = L[x] op L[y] (* w3 when b) sub = add / sub / rsub / mul, w1, w2 = operand words
-  DVM_LK_BIN_ACC,                                        // ACC = ACC op ACC           sub = arith
+  DVM_LK_BIN_BF16,                                       // ACC = ACC op L[y]          sub = arith, w1 = operand word; b = 1 + s: ACC * S[s] * L[y]
   DVM_LK_FMA,                                            // ACC = ACC * m + c          m = sub & 1 ? S[a] : w1 (sub & 4: its reciprocal),
                                                          //                            c = sub & 2 ? S[b] : w2 (sub & 8: negated)
+  DVM_LK_EXPS,                                           // ACC = exp(ACC - S[a])      sub = 1: one-piece exponential
+  DVM_LK_RED,                                            // S[a] = reduce(ACC); b = 1: S[a] = unary(S[a] * w2 + w3), w1 = unary or 0xff
+  DVM_LK_STG,                                            // store ACC: a = log2(element size), w1 | w2 << 32 = tensor address
+  DVM_LK_LDA_BF16,                                       // ACC = L[x]                 w1 = operand word
+  DVM_LK_HOT_LAST = DVM_LK_LDA_BF16,
+  DVM_LK_LDA_F32, DVM_LK_LDA_PRIV,                       // ACC = L[x] (fp32 image, private temporary)
+  DVM_LK_BIN_F32, DVM_LK_BIN_PRIV,                       // ACC = ACC op L[y] (as DVM_LK_BIN_BF16)
+  DVM_LK_BIN_ACC,                                        // ACC = ACC op ACC           sub = arith
   DVM_LK_BINI,                                           // ACC = ACC op imm           sub = rdiv / min / max, w1 = imm
   DVM_LK_BINS,                                           // ACC = ACC op S[a]          sub = rdiv / min / max
   DVM_LK_ACT,                                            // ACC = act(ACC)             sub = DVM_ACT_* (HEAVY variants)
   DVM_LK_UN,                                             // ACC = f(ACC)               sub = unary (| 0x80: one-piece exponential)
-  DVM_LK_EXPS,                                           // ACC = exp(ACC - S[a])      sub = 1: one-piece exponential
-  DVM_LK_RED,                                            // S[a] = reduce(ACC); b = 1: S[a] = unary(S[a] * w2 + w3), w1 = unary or 0xff
-  DVM_LK_STG,                                            // store ACC: a = log2(element size), w1 | w2 << 32 = tensor address
   DVM_LK_STGI,                                           // store ACC converted to i32 (sub 1) or u8 (sub 2): the same fields
   DVM_LK_STA,                                            // L[tmp] = ACC               w1 = byte offset of the temporary in a tile slot
   DVM_LK_LSS,                                            // S[a] = loaded row scalar   w1 = byte offset of its word in a tile slot (thread 0's)

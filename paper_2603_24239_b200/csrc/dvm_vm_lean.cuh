@@ -511,8 +511,7 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
       const uint32_t ra = (rec.x >> 16) & 0xffu;
       if (h == DVM_LK_END) break;
       // two dispatch levels: the records of the bf16 sweeps (load, multiply-add, exponential, reduction, store) first
-      if (h == DVM_LK_LD2_BF16 || h == DVM_LK_BIN_BF16 || h == DVM_LK_STG || h == DVM_LK_RED || h == DVM_LK_FMA ||
-          h == DVM_LK_EXPS || h == DVM_LK_LDA_BF16) {
+      if (h <= DVM_LK_HOT_LAST) {
       switch (h) {
         case DVM_LK_LDA_BF16: {
           uint32_t R[V / 2];
