@@ -920,17 +920,21 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_kernel(const __grid_cons
           }
           float v;
           if (rop == DVM_R_SUM || rop == DVM_R_SUMSQ) {
-            float2 acc = make_float2(0.f, 0.f);
+            // four partial sums per thread, pair i into sum i % 4 (as the lean interpreter: independent chains), then a tree
+            float2 acc[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.f, 0.f);
             if (all_valid) {
-              if (rop == DVM_R_SUM) { DVM_EACH_PAIR acc = __fadd2_rn(acc, A[i]); }
-              else { DVM_EACH_PAIR acc = __ffma2_rn(A[i], A[i], acc); }
+              if (rop == DVM_R_SUM) { DVM_EACH_PAIR acc[i & 3] = __fadd2_rn(acc[i & 3], A[i]); }
+              else { DVM_EACH_PAIR acc[i & 3] = __ffma2_rn(A[i], A[i], acc[i & 3]); }
             } else {
               DVM_EACH_PAIR {
                 const float2 x = make_float2(slot_valid(c, 2 * i) ? A[i].x : 0.f, slot_valid(c, 2 * i + 1) ? A[i].y : 0.f);
-                acc = rop == DVM_R_SUM ? __fadd2_rn(acc, x) : __ffma2_rn(x, x, acc);
+                acc[i & 3] = rop == DVM_R_SUM ? __fadd2_rn(acc[i & 3], x) : __ffma2_rn(x, x, acc[i & 3]);
               }
             }
-            v = acc.x + acc.y;
+            const float2 a2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
+            v = a2.x + a2.y;
 #pragma unroll
             for (int sh = 1; sh < 32; sh <<= 1)
               if (sh < G) v += __shfl_xor_sync(0xffffffffu, v, sh);
@@ -947,12 +951,19 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_kernel(const __grid_cons
                 v = mx ? fmaxf(v, fmaxf(x0, x1)) : fminf(v, fminf(x0, x1));
               }
             }
+            if (G >= 32) {  // the whole warp holds one row: the warp-wide fp32 max / min instruction of sm_100a
+              float w;
+              if (mx) asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(w) : "f"(v));
+              else asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(w) : "f"(v));
+              v = w;
+            } else {
 #pragma unroll
-            for (int sh = 1; sh < 32; sh <<= 1)
-              if (sh < G) {
-                const float x = __shfl_xor_sync(0xffffffffu, v, sh);
-                v = mx ? fmaxf(v, x) : fminf(v, x);
-              }
+              for (int sh = 1; sh < 32; sh <<= 1)
+                if (sh < G) {
+                  const float x = __shfl_xor_sync(0xffffffffu, v, sh);
+                  v = mx ? fmaxf(v, x) : fminf(v, x);
+                }
+            }
           }
           if (G > 32) {
             if (lane == 0) s_red[red_par][warp] = v;

@@ -576,32 +576,46 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
           if (!all_valid) sanitize(ident);
           float v;
           if (is_sum) {
-            float2 acc = make_float2(0.f, 0.f);
+            // four partial sums per thread, one per pair of an 8-slot group (independent chains), then a tree
+            float2 acc[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.f, 0.f);
 #pragma unroll
             for (int g = 0; g < NG; ++g)
               if (all_valid || group_on(g)) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) acc = rop == DVM_R_SUM ? __fadd2_rn(acc, A[4 * g + q]) : __ffma2_rn(A[4 * g + q], A[4 * g + q], acc);
+                for (int q = 0; q < 4; ++q) acc[q] = rop == DVM_R_SUM ? __fadd2_rn(acc[q], A[4 * g + q]) : __ffma2_rn(A[4 * g + q], A[4 * g + q], acc[q]);
               }
-            v = acc.x + acc.y;
+            const float2 a2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
+            v = a2.x + a2.y;
 #pragma unroll
             for (int sh = 1; sh < 32; sh <<= 1)
               if (sh < G) v += __shfl_xor_sync(0xffffffffu, v, sh);
           } else {
             const bool mx = rop == DVM_R_MAX;
-            v = ident;
+            float m4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) m4[q] = ident;
 #pragma unroll
             for (int g = 0; g < NG; ++g)
               if (all_valid || group_on(g)) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) v = mx ? fmaxf(v, fmaxf(A[4 * g + q].x, A[4 * g + q].y)) : fminf(v, fminf(A[4 * g + q].x, A[4 * g + q].y));
+                for (int q = 0; q < 4; ++q) m4[q] = mx ? fmaxf(m4[q], fmaxf(A[4 * g + q].x, A[4 * g + q].y)) : fminf(m4[q], fminf(A[4 * g + q].x, A[4 * g + q].y));
               }
+            v = mx ? fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) : fminf(fminf(m4[0], m4[1]), fminf(m4[2], m4[3]));
+            if (G >= 32) {  // the whole warp holds one row: the warp-wide fp32 max / min instruction of sm_100a
+              float w;
+              if (mx) asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(w) : "f"(v));
+              else asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(w) : "f"(v));
+              v = w;
+            } else {
 #pragma unroll
-            for (int sh = 1; sh < 32; sh <<= 1)
-              if (sh < G) {
-                const float x = __shfl_xor_sync(0xffffffffu, v, sh);
-                v = mx ? fmaxf(v, x) : fminf(v, x);
-              }
+              for (int sh = 1; sh < 32; sh <<= 1)
+                if (sh < G) {
+                  const float x = __shfl_xor_sync(0xffffffffu, v, sh);
+                  v = mx ? fmaxf(v, x) : fminf(v, x);
+                }
+            }
           }
           if (G > 32) {
             if (lane == 0) s_red[red_par][warp] = v;
