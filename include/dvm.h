@@ -226,6 +226,14 @@ int dvm_get_min_resident_ctas(void);
  * Default 1.  Both interpreters run the same bytecode and give results inside the same tolerances. */
 void dvm_set_lean_kernel(int on);
 
+/* Matmul launches (Sec. 4.2, matrix operations): when the last wave of output tiles would occupy at most half
+ * of the SMs, each of its tiles is computed by up to four CTAs, every one taking a share of the k blocks; the
+ * shares meet in a library-owned fp32 workspace (one per device and stream, 15 MB, allocated by the first launch
+ * that needs it; none is made while the stream is being captured -- such launches run unsplit) and are added in
+ * a fixed order, so results are deterministic.  They differ from the unsplit result by fp32 rounding of the
+ * partial sums.  on = 0 switches the split off.  Default 1. */
+void dvm_set_matmul_tail_split(int on);
+
 /* The paper's tile-size rule for a flat vector operator (Sec. 4.2,
  * hardware_align_div): among tile sizes t in [1, min(total, t_max)] take the
  * one minimising ceil(ceil(total / t) / n_cores) * (t + overhead) (ties: the

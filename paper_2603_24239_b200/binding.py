@@ -84,6 +84,7 @@ _sig = {
     "dvm_get_min_resident_ctas": ([], _i),
     "dvm_set_lean_kernel": ([_i], None),
     "dvm_set_stacked_one_slot": ([_i], None),
+    "dvm_set_matmul_tail_split": ([_i], None),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -619,6 +620,11 @@ def set_lean_kernel(on: bool):
     """False: every launch runs on the general interpreter (for comparisons); True (default): programs of the
     basic instruction set run on the lean variant."""
     lib.dvm_set_lean_kernel(int(on))
+
+
+def set_matmul_tail_split(on: bool):
+    """dvm_set_matmul_tail_split: split the tiles of a matmul launch's last, partial wave along k (default on)."""
+    lib.dvm_set_matmul_tail_split(int(bool(on)))
 
 
 def set_stacked_one_slot(on: bool):

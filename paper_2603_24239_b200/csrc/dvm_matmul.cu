@@ -520,12 +520,23 @@ constexpr unsigned long long WAIT_NS = 2000000000ull;   // limit of one wait: 2 
 constexpr unsigned long long DRAIN_NS = 200000000ull;   // limit of a wait for work in flight after an abort
 constexpr uint32_t WAIT_SPINS = 1u << 27;
 
+// Tail split (split_s >= 2): the tiles [split_first, split_first + split_r) -- the last, partial wave of the
+// launch -- are each computed by split_s CTAs, part p taking the k blocks [p * split_kb, (p + 1) * split_kb).
+// Parts 1.. write their accumulators to `ws` (partial index r * (split_s - 1) + p - 1, laid out
+// [column][row] fp32) and publish flags[4 r + p - 1] = epoch; part 0 (the tile's owner) waits
+// for them, adds them to its own accumulators in tensor memory in the order of p and runs the epilogue.
 struct MMParams {
   unsigned int* status;
+  float* ws;
+  uint32_t* flags;
+  uint32_t epoch;
+  uint32_t split_first, split_r, split_s, split_kb;
   uint32_t n_words;
   uint32_t n_stages;
   uint32_t words[DVM_MM_MAX_WORDS];
 };
+constexpr uint32_t MAX_SPLIT = 4;                    // CTAs per tail tile at most
+constexpr size_t PART_FLOATS = (size_t)BLOCK_M * ACC_COLS;  // one partial accumulator: 128 KB
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -605,6 +616,41 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[CHUNK]) {
   for (int i = 0; i < CHUNK; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// the same 32 columns written back (the caller waits with tmem_st_wait before it reads them again)
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[CHUNK]) {
+  uint32_t r[CHUNK];
+#pragma unroll
+  for (int i = 0; i < CHUNK; ++i) r[i] = __float_as_uint(v[i]);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+        "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Bounded wait of a tile's owner for the n flags of its other parts (each becomes `epoch` once that part's
+// accumulators are in the workspace); like mbar_wait_slow it raises the CTA's abort flag when it gives up.
+__device__ __noinline__ bool flags_wait(const uint32_t* f, uint32_t n, uint32_t epoch, volatile uint32_t* abort_flag) {
+  const unsigned long long t0 = gtimer();
+  uint32_t k = 0;
+  for (uint32_t spin = 0; spin < WAIT_SPINS && k < n; ++spin) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f + k) : "memory");
+    if (v == epoch) { ++k; continue; }
+    if (*abort_flag) return false;
+    if (gtimer() - t0 > WAIT_NS) break;
+  }
+  if (k == n) return true;
+  *abort_flag = 1;
+  return false;
+}
+
 // Shared-memory matrix descriptors (128-byte swizzle, sm_100 descriptor version 1).
 // A tile, K-major: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t desc_k_major(uint32_t addr) {
@@ -674,14 +720,36 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = *(volatile uint32_t*)tmem_slot;
 
+  // The i-th piece of work of this CTA: whole tiles blockIdx.x + i * gridDim.x below split_first, then (tail
+  // split) one part of one tail tile.
+  struct Work { uint32_t tile, kb0, kb1, part, r; };
+  const uint32_t split_first = prm.split_s >= 2 ? prm.split_first : n_tiles;
+  auto work_at = [&](uint32_t i, Work& w) -> bool {
+    const uint32_t t = blockIdx.x + i * gridDim.x;
+    w.part = 0; w.r = 0; w.kb0 = 0; w.kb1 = k_blocks;
+    if (t < split_first) { w.tile = t; return true; }
+    const uint32_t u = t - split_first;  // (split_first is a multiple of the grid size: u = blockIdx.x in the round after the whole tiles)
+    if (prm.split_s < 2 || u >= prm.split_r * prm.split_s) return false;
+    w.part = u / prm.split_r;
+    w.r = u - w.part * prm.split_r;
+    w.tile = split_first + w.r;
+    w.kb0 = w.part * prm.split_kb;
+    w.kb1 = min(k_blocks, w.kb0 + prm.split_kb);
+    return true;
+  };
+  const bool split = prm.split_s >= 2;
+  volatile uint32_t* const split_ok = tmem_slot + 2;
+
   uint32_t issued = 0, p_stage = 0, p_phase = 0;  // producer state, kept for the abort path
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      Work w;
+      for (uint32_t i = 0; ok && work_at(i, w); ++i) {
+        const uint32_t t = w.tile;
         const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
-        for (uint32_t kb = 0; kb < k_blocks; ++kb) {
+        for (uint32_t kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(bar_empty + 8 * p_stage, p_phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8 * p_stage;
           const uint32_t sa = base + p_stage * STAGE_BYTES;
@@ -708,19 +776,20 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, it = 0;
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
+      Work w;
+      for (; ok && work_at(it, w); ++it) {
         const uint32_t as = it & 1, aph = (it >> 1) & 1;
         if (!mbar_wait(bar_tempty + 8 * as, aph ^ 1, abort_flag)) break;  // the epilogue has drained this stage
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + as * ACC_COLS;
-        for (uint32_t kb = 0; kb < k_blocks; ++kb) {
+        for (uint32_t kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * STAGE_BYTES;
           const uint64_t adesc = desc_k_major(sa), bdesc = desc_n_major(sa + STAGE_A);
 #pragma unroll
           for (uint32_t j = 0; j < BLOCK_K / 16; ++j)  // K = 16 per instruction: 32 bytes along A's rows, two k groups of B
-            umma_bf16(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC, (kb | j) != 0);
+            umma_bf16(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC, ((kb - w.kb0) | j) != 0);
           umma_commit(bar_empty + 8 * stage);  // the stage is free once these MMAs have read it
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
@@ -735,11 +804,64 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     float* const tmp_mine = (float*)(sm + tmp_base) + erow * 4;
     uint32_t it = 0;
-    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+    Work w;
+    for (; work_at(it, w); ++it) {
+      const uint32_t t = w.tile;
       const uint32_t as = it & 1, aph = (it >> 1) & 1;
       const bool got = mbar_wait(bar_tfull + 8 * as, aph, abort_flag);
       if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
+      if (split && t >= split_first) {
+        // ---- a tail tile computed in parts (see MMParams) ----
+        const uint32_t used_chunks = (uint32_t)(nb == 2 ? ACC_COLS : tile_n) / CHUNK;
+        const uint32_t acc0 = lane_addr + as * ACC_COLS;
+        if (w.part > 0) {  // this CTA's accumulators go to the workspace; the owner is told; nothing else to do here
+          float* const dst0 = prm.ws + (size_t)(w.r * (prm.split_s - 1) + (w.part - 1)) * PART_FLOATS + erow;
+          for (uint32_t c = 0; c < used_chunks; ++c) {
+            float v[CHUNK];
+            tmem_ld32(acc0 + c * CHUNK, v);
+            float* dst = dst0 + (size_t)c * CHUNK * BLOCK_M;
+#pragma unroll
+            for (int k = 0; k < CHUNK; ++k) __stcg(dst + k * BLOCK_M, v[k]);  // (a warp's 32 rows of one column: one 128-byte line)
+          }
+          __threadfence();
+          tc_fence_before();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (threadIdx.x == 64) {
+            uint32_t* f = prm.flags + 4 * w.r + (w.part - 1);
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(f), "r"(prm.epoch) : "memory");
+          }
+          mbar_arrive(bar_tempty + 8 * as);
+          continue;
+        }
+        // the owner: every other part's accumulators, added in the order of the parts
+        if (threadIdx.x == 64) {
+          const bool ok = flags_wait(prm.flags + 4 * w.r, prm.split_s - 1, prm.epoch, abort_flag);
+          __threadfence();
+          *split_ok = ok ? 1u : 0u;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (!*split_ok) break;
+        for (uint32_t c = 0; c < used_chunks; ++c) {
+          float v[CHUNK];
+          tmem_ld32(acc0 + c * CHUNK, v);
+          // (all loads of the chunk are issued before the first sum: the parts' lines come from L2 together)
+          float x[MAX_SPLIT - 1][CHUNK];
+#pragma unroll
+          for (uint32_t p2 = 0; p2 < MAX_SPLIT - 1; ++p2) {
+            const float* src = prm.ws + (size_t)(w.r * (prm.split_s - 1) + p2) * PART_FLOATS + (size_t)c * CHUNK * BLOCK_M + erow;
+#pragma unroll
+            for (int k = 0; k < CHUNK; ++k) x[p2][k] = p2 + 1 < prm.split_s ? __ldcg(src + k * BLOCK_M) : 0.0f;
+          }
+#pragma unroll
+          for (uint32_t p2 = 0; p2 < MAX_SPLIT - 1; ++p2) {
+#pragma unroll
+            for (int k = 0; k < CHUNK; ++k) v[k] += x[p2][k];
+          }
+          tmem_st32(acc0 + c * CHUNK, v);
+        }
+        tmem_st_wait();
+      }
       const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
       const int row = m0 + erow;
       const bool row_ok = row < M;
@@ -966,6 +1088,49 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 std::mutex g_mm_mu;
 EncodeTiledFn g_encode_tiled = nullptr;
 bool g_attr_set[64] = {};
+int g_tail_split = 1;  // dvm_set_matmul_tail_split
+
+// Workspace of the tail split, one per (device, stream): launches of one stream run in order, so they may share
+// it; launches of different streams may overlap, so they do not.  Allocated at the first launch that splits.
+struct SplitSpace {
+  int device;
+  cudaStream_t stream;
+  float* ws;
+  uint32_t* flags;
+  uint32_t epoch;
+};
+constexpr int MAX_SPLIT_SPACES = 16;
+constexpr size_t SPLIT_WS_PARTS = 112;  // partial accumulators: max over r of r * (min(4, sms / r) - 1) for up to 148 SMs, rounded up
+constexpr size_t SPLIT_FLAG_WORDS = 4 * 160;
+SplitSpace g_split[MAX_SPLIT_SPACES];
+int g_n_split = 0;
+
+// The workspace of (device, stream), or NULL (then the launch does not split): none is made while the stream is
+// being captured (an allocation does not belong into a graph) or when every slot is taken.
+SplitSpace* split_space(int device, cudaStream_t stream) {
+  std::lock_guard<std::mutex> lk(g_mm_mu);
+  for (int i = 0; i < g_n_split; ++i)
+    if (g_split[i].device == device && g_split[i].stream == stream) return &g_split[i];
+  if (g_n_split == MAX_SPLIT_SPACES) return nullptr;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  SplitSpace sp = {device, stream, nullptr, nullptr, 0};
+  if (cudaMalloc(&sp.ws, SPLIT_WS_PARTS * dvm::mm::PART_FLOATS * sizeof(float)) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  if (cudaMalloc(&sp.flags, SPLIT_FLAG_WORDS * 4) != cudaSuccess || cudaMemset(sp.flags, 0, SPLIT_FLAG_WORDS * 4) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(sp.ws);
+    if (sp.flags) cudaFree(sp.flags);
+    return nullptr;
+  }
+  g_split[g_n_split] = sp;
+  return &g_split[g_n_split++];
+}
 
 int mm_encode_fn(EncodeTiledFn* out) {
   std::lock_guard<std::mutex> lk(g_mm_mu);
@@ -1057,12 +1222,38 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   P.n_words = (uint32_t)n_words;
   P.n_stages = n_stages;
   const uint32_t tiles = code[DVM_H_N_TILES];
-  const int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
+  int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
+  // Tail split: the last wave of r < sms / 2 tiles would leave most SMs idle for a whole tile time; instead
+  // s = min(4, sms / r) CTAs take each of its tiles, a share of the k blocks each (see MMParams).
+  P.split_s = P.split_r = P.split_first = P.split_kb = 0;
+  P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
+  const uint32_t sms = (uint32_t)dev.sm_count, kblocks = x[DVM_MM_KBLOCKS];
+  const uint32_t tail = tiles % sms;
+  if (g_tail_split && tail && 2 * tail <= sms && kblocks >= 16 && sms <= 148) {
+    uint32_t s_want = sms / tail;
+    if (s_want > dvm::mm::MAX_SPLIT) s_want = dvm::mm::MAX_SPLIT;
+    const uint32_t per = (kblocks + s_want - 1) / s_want;
+    const uint32_t s_eff = (kblocks + per - 1) / per;
+    SplitSpace* sp = (s_eff >= 2 && (size_t)tail * (s_eff - 1) <= SPLIT_WS_PARTS) ? split_space(devid, stream) : nullptr;
+    if (sp) {
+      P.split_first = tiles - tail;
+      P.split_r = tail;
+      P.split_s = s_eff;
+      P.split_kb = per;
+      P.ws = sp->ws;
+      P.flags = sp->flags;
+      if (++sp->epoch == 0) sp->epoch = 1;
+      P.epoch = sp->epoch;
+      if (tiles < sms) grid = (int)(tail * s_eff);
+    }
+  }
   dvm::mm::dvm_mm_kernel<<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;
 }
+
+extern "C" void dvm_set_matmul_tail_split(int on) { g_tail_split = on; }
 
 // ---- self-test of the matmul kernel's bounded wait (see dvm_selftest_bounded_wait) ----
 namespace dvm {

@@ -194,3 +194,59 @@ def test_addmm_largest_shapes_sampled_rows(m, n, k):
     g1, _ = gate_errors(wl.to_f64(out[ti]), want[0])
     assert g1 <= R_BF16, g1
     assert not torch.isnan(out.float().sum())
+
+
+# ---- tail split: the tiles of the last, partial wave computed by several CTAs, a share of the k blocks each ----
+
+def _tail_case(kind, M, K, N, seed):
+    if kind == "mlp":
+        return wl.program_mlp_gate(), _mlp_inputs(M, K, N, seed)
+    a = wl.randn((M, K), torch.bfloat16, seed)
+    b = wl.randn((K, N), torch.bfloat16, seed + 1, std=0.02)
+    c = wl.randn((M, N), torch.bfloat16, seed + 2)
+    return wl.program_addmm(), [a, b, c]
+
+
+@pytest.mark.parametrize("kind,M,K,N", [
+    ("addmm", 128, 1088, 2560),    # one wave of 10 tiles: four CTAs per tile, 17 k blocks shared 5 / 5 / 5 / 2
+    ("addmm", 1024, 1024, 4864),   # 152 tiles: a full wave, then 4 tiles by four CTAs each
+    ("mlp", 256, 1024, 12672),     # 198 tiles of both products: a full wave, then 50 tiles by two CTAs each
+    ("mlp", 100, 2048, 3200),      # one wave of 25 tiles, ragged M: four CTAs per tile (the cap)
+    ("addmm", 77, 1600, 9000),     # ragged M, N and a k tail: 36 tiles, four CTAs each
+])
+def test_tail_split_against_oracle_and_unsplit(kind, M, K, N):
+    prog, ins = _tail_case(kind, M, K, N, seed=M + N + K)
+    try:
+        dvm.set_matmul_tail_split(True)
+        outs, _ = gpu_run(prog, ins)
+        again, _ = gpu_run(prog, ins)
+        dvm.set_matmul_tail_split(False)
+        plain, _ = gpu_run(prog, ins)
+    finally:
+        dvm.set_matmul_tail_split(True)
+    want = oracle_run(prog, ins)
+    check(prog, outs, want)
+    check(prog, plain, want)
+    assert not torch.isnan(outs[0].float()).any()
+    # the shares are added in a fixed order: the same bits every time
+    assert torch.equal(outs[0], again[0])
+    # against the unsplit accumulation only the fp32 rounding of the partial sums differs: a bf16 step at most
+    a, b = outs[0].float(), plain[0].float()
+    scale = b.abs().max().item()
+    assert (a - b).abs().max().item() <= 2.0 ** -7 * scale
+    assert (a != b).float().mean().item() < 0.2
+
+
+def test_tail_split_on_two_streams():
+    """Every stream has a workspace of its own: launches of two streams may overlap."""
+    prog, ins = _tail_case("addmm", 128, 2048, 2560, seed=9)
+    want = oracle_run(prog, ins)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    res = []
+    for _ in range(3):
+        for s in (s1, s2):
+            res.append(gpu_run(prog, ins, stream=s)[0])
+    torch.cuda.synchronize()
+    for outs in res:
+        check(prog, outs, want)
+        assert torch.equal(outs[0], res[0][0])
