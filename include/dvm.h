@@ -234,6 +234,13 @@ void dvm_set_lean_kernel(int on);
  * partial sums.  on = 0 switches the split off.  Default 1. */
 void dvm_set_matmul_tail_split(int on);
 
+/* Matmul launches on CTA pairs: two CTAs of a cluster compute a tile of 256 output rows with one tcgen05
+ * cta_group::2 instruction stream, each loading its own rows of A and half of the B tile (a third less
+ * shared-memory traffic per flop).  mode = 0: never; 1 (default): where the launch's shape favours it; 2: wherever
+ * the output has at least two blocks of 128 rows.  Results are those of the single-CTA kernel bit for bit (the
+ * same instruction shape along k). */
+void dvm_set_matmul_cta_pairs(int mode);
+
 /* The paper's tile-size rule for a flat vector operator (Sec. 4.2,
  * hardware_align_div): among tile sizes t in [1, min(total, t_max)] take the
  * one minimising ceil(ceil(total / t) / n_cores) * (t + overhead) (ties: the

@@ -85,6 +85,7 @@ _sig = {
     "dvm_set_lean_kernel": ([_i], None),
     "dvm_set_stacked_one_slot": ([_i], None),
     "dvm_set_matmul_tail_split": ([_i], None),
+    "dvm_set_matmul_cta_pairs": ([_i], None),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -625,6 +626,11 @@ def set_lean_kernel(on: bool):
 def set_matmul_tail_split(on: bool):
     """dvm_set_matmul_tail_split: split the tiles of a matmul launch's last, partial wave along k (default on)."""
     lib.dvm_set_matmul_tail_split(int(bool(on)))
+
+
+def set_matmul_cta_pairs(mode: int):
+    """dvm_set_matmul_cta_pairs: matmul launches on CTA pairs (0 never, 1 default: by shape, 2 wherever possible)."""
+    lib.dvm_set_matmul_cta_pairs(int(mode))
 
 
 def set_stacked_one_slot(on: bool):

@@ -512,7 +512,10 @@ constexpr int ACC_COLS = 256;                       // accumulator columns of on
 constexpr uint32_t STAGE_A = BLOCK_M * BLOCK_K * 2; // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t BOX_B = 64 * BLOCK_K * 2;        // 8 KB: 64 k-rows of 64 columns
 constexpr uint32_t STAGE_BYTES = STAGE_A + 4 * BOX_B;  // 48 KB
-constexpr int MAX_STAGES = 4;
+constexpr int MAX_STAGES = 8;                       // barrier slots; 4 stages of 48 KB, or 6 of 32 KB for a CTA pair
+constexpr uint32_t STAGE_PAIR = STAGE_A + 2 * BOX_B;  // 32 KB: this CTA's A rows and its half of the B tile
+constexpr uint32_t STAGES_SINGLE = 4, STAGES_PAIR = 6;
+constexpr uint32_t BAR_BYTES = 256;                  // barriers and flags behind the epilogue temporaries
 constexpr uint32_t TMP_BYTES = 128 * CHUNK * 4;     // one epilogue temporary: 16 KB
 constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
@@ -527,6 +530,7 @@ constexpr uint32_t WAIT_SPINS = 1u << 27;
 // for them, adds them to its own accumulators in tensor memory in the order of p and runs the epilogue.
 struct MMParams {
   unsigned int* status;
+  uint32_t pair_tiles, pair_mblocks;  // CTA pairs: tiles of 256 rows, blocks of 256 rows
   float* ws;
   uint32_t* flags;
   uint32_t epoch;
@@ -598,6 +602,43 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- the CTA-pair forms (tcgen05 cta_group::2: two CTAs of a cluster, one MMA over both their shared memories) ----
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// the shared::cluster address of `addr` (a shared-memory address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t peer_addr(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// tile load of one CTA of a pair; the bytes are counted on `cluster_bar`, a barrier of the pair's first CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this address in BOTH CTAs of the pair once the MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 // 32 consecutive accumulator columns of this thread's tensor-memory lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[CHUNK]) {
   uint32_t r[CHUNK];
@@ -665,9 +706,17 @@ __device__ __forceinline__ uint64_t desc_n_major(uint32_t addr) {
 // kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = 256
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                            ((uint32_t)(ACC_COLS >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+// the same over a CTA pair: M = 256
+constexpr uint32_t IDESC_PAIR = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(ACC_COLS >> 3) << 17) | ((uint32_t)(2 * BLOCK_M >> 4) << 24);
 
 __device__ __forceinline__ float mm_arith(int op, float a, float b) { return scalar_arith(op, a, b); }
 
+// PAIR: two CTAs of a cluster work on one tile of 256 rows (128 each) with tcgen05 cta_group::2 -- each loads its
+// own A rows and HALF of the B tile (the first CTA the accumulator columns 0..127, the second 128..255), the first
+// CTA's MMA thread issues one instruction over both shared memories, both CTAs hold the accumulators of their own
+// rows: a stage is 32 KB per CTA instead of 48, a third less traffic from L2 per flop.
+template <bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ MMParams prm) {
@@ -689,13 +738,15 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   const uint32_t n_tiles = MW(DVM_H_N_TILES);
   const uint32_t n_stages = prm.n_stages;
 
-  const uint32_t tmp_base = n_stages * STAGE_BYTES;                 // byte offsets from `base`
+  constexpr uint32_t SB = PAIR ? STAGE_PAIR : STAGE_BYTES;          // bytes of one pipeline stage in this CTA
+  const uint32_t tmp_base = n_stages * SB;                          // byte offsets from `base`
   const uint32_t bar_base = base + tmp_base + (uint32_t)ntmp * TMP_BYTES;
-  // barriers: full[4] empty[4] tmem_full[2] tmem_empty[2] drain
-  const uint32_t bar_full = bar_base, bar_empty = bar_base + 32, bar_tfull = bar_base + 64, bar_tempty = bar_base + 80,
-                 bar_drain = bar_base + 96;
-  uint32_t* const tmem_slot = (uint32_t*)(sm + tmp_base + (uint32_t)ntmp * TMP_BYTES + 112);
+  // barriers: full[8] empty[8] tmem_full[2] tmem_empty[2] drain
+  const uint32_t bar_full = bar_base, bar_empty = bar_base + 64, bar_tfull = bar_base + 128, bar_tempty = bar_base + 144,
+                 bar_drain = bar_base + 160;
+  uint32_t* const tmem_slot = (uint32_t*)(sm + tmp_base + (uint32_t)ntmp * TMP_BYTES + 176);
   volatile uint32_t* const abort_flag = tmem_slot + 1;
+  const uint32_t rank = PAIR ? cluster_rank() : 0u;                 // 0: the pair's first CTA, which issues its MMAs
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -705,29 +756,36 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
     for (uint32_t a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 128);
+      mbar_init(bar_tempty + 8 * a, PAIR ? 8 : 128);  // (a pair: one arrival per epilogue warp of both CTAs)
     }
     mbar_init(bar_drain, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // tensor memory: both accumulator stages
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync();  // the other CTA's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *(volatile uint32_t*)tmem_slot;
 
   // The i-th piece of work of this CTA: whole tiles blockIdx.x + i * gridDim.x below split_first, then (tail
   // split) one part of one tail tile.
   struct Work { uint32_t tile, kb0, kb1, part, r; };
-  const uint32_t split_first = prm.split_s >= 2 ? prm.split_first : n_tiles;
+  const uint32_t split_first = PAIR ? prm.pair_tiles : (prm.split_s >= 2 ? prm.split_first : n_tiles);
   auto work_at = [&](uint32_t i, Work& w) -> bool {
-    const uint32_t t = blockIdx.x + i * gridDim.x;
+    const uint32_t t = PAIR ? (blockIdx.x >> 1) + i * (gridDim.x >> 1) : blockIdx.x + i * gridDim.x;
     w.part = 0; w.r = 0; w.kb0 = 0; w.kb1 = k_blocks;
     if (t < split_first) { w.tile = t; return true; }
+    if constexpr (PAIR) return false;
     const uint32_t u = t - split_first;  // (split_first is a multiple of the grid size: u = blockIdx.x in the round after the whole tiles)
     if (prm.split_s < 2 || u >= prm.split_r * prm.split_s) return false;
     w.part = u / prm.split_r;
@@ -737,7 +795,11 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     w.kb1 = min(k_blocks, w.kb0 + prm.split_kb);
     return true;
   };
-  const bool split = prm.split_s >= 2;
+  const bool split = !PAIR && prm.split_s >= 2;
+  // first row and column of a tile for this CTA (a pair: blocks of 256 rows, this CTA's half of them)
+  const uint32_t mbl = PAIR ? prm.pair_mblocks : m_blocks;
+  auto tile_m0 = [&](uint32_t t) -> int { return (int)(t % mbl) * (PAIR ? 2 * BLOCK_M : BLOCK_M) + (int)rank * BLOCK_M; };
+  auto tile_n0 = [&](uint32_t t) -> int { return (int)(t / mbl) * tile_n; };
   volatile uint32_t* const split_ok = tmem_slot + 2;
 
   uint32_t issued = 0, p_stage = 0, p_phase = 0;  // producer state, kept for the abort path
@@ -748,13 +810,26 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
       Work w;
       for (uint32_t i = 0; ok && work_at(i, w); ++i) {
         const uint32_t t = w.tile;
-        const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
+        const int m0 = tile_m0(t), n0 = tile_n0(t);
         for (uint32_t kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(bar_empty + 8 * p_stage, p_phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8 * p_stage;
-          const uint32_t sa = base + p_stage * STAGE_BYTES;
-          mbar_expect_tx(full, STAGE_BYTES);
+          const uint32_t sa = base + p_stage * SB;
           const int k0 = (int)kb * BLOCK_K;
+          if constexpr (PAIR) {
+            // both CTAs' bytes are counted on the first CTA's barrier, which alone expects them
+            const uint32_t full0 = peer_addr(full, 0);
+            if (rank == 0) mbar_expect_tx(full, 2 * SB);
+            tma_load_2d_pair(sa, &tmA, full0, k0, m0);
+            const CUtensorMap* mapb = (nb == 2 && rank == 1) ? &tmB1 : &tmB0;
+            const int nh = n0 + (nb == 2 ? 0 : (int)rank * 128);
+            tma_load_2d_pair(sa + STAGE_A, mapb, full0, nh, k0);
+            tma_load_2d_pair(sa + STAGE_A + BOX_B, mapb, full0, nh + 64, k0);
+            ++issued;
+            if (++p_stage == n_stages) { p_stage = 0; p_phase ^= 1; }
+            continue;
+          }
+          mbar_expect_tx(full, STAGE_BYTES);
           tma_load_2d(sa, &tmA, full, k0, m0);
           if (nb == 2) {
             tma_load_2d(sa + STAGE_A, &tmB0, full, n0, k0);
@@ -772,8 +847,8 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (a pair: the first CTA's) ----------------
+    if (lane == 0 && rank == 0) {
       uint32_t stage = 0, phase = 0, it = 0;
       bool ok = true;
       Work w;
@@ -785,15 +860,18 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         for (uint32_t kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint32_t sa = base + stage * SB;
           const uint64_t adesc = desc_k_major(sa), bdesc = desc_n_major(sa + STAGE_A);
 #pragma unroll
-          for (uint32_t j = 0; j < BLOCK_K / 16; ++j)  // K = 16 per instruction: 32 bytes along A's rows, two k groups of B
-            umma_bf16(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC, ((kb - w.kb0) | j) != 0);
-          umma_commit(bar_empty + 8 * stage);  // the stage is free once these MMAs have read it
+          for (uint32_t j = 0; j < BLOCK_K / 16; ++j) {  // K = 16 per instruction: 32 bytes along A's rows, two k groups of B
+            if constexpr (PAIR) umma_bf16_pair(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC_PAIR, ((kb - w.kb0) | j) != 0);
+            else umma_bf16(d_tmem, adesc + 2 * j, bdesc + (uint64_t)(2048 >> 4) * j, IDESC, ((kb - w.kb0) | j) != 0);
+          }
+          // the stage is free once these MMAs have read it (a pair: in both CTAs)
+          if constexpr (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
-        if (ok) umma_commit(bar_tfull + 8 * as);
+        if (ok) { if constexpr (PAIR) umma_commit_pair(bar_tfull + 8 * as); else umma_commit(bar_tfull + 8 * as); }
       }
     }
     __syncwarp();
@@ -862,7 +940,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
         tmem_st_wait();
       }
-      const int m0 = (int)(t % m_blocks) * BLOCK_M, n0 = (int)(t / m_blocks) * tile_n;
+      const int m0 = tile_m0(t), n0 = tile_n0(t);
       const int row = m0 + erow;
       const bool row_ok = row < M;
       const int n_chunks = tile_n / CHUNK;
@@ -1041,7 +1119,12 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
       }
       // this accumulator stage may be overwritten by the tile after next
       tc_fence_before();
-      mbar_arrive(bar_tempty + 8 * as);
+      if constexpr (PAIR) {  // (told to the first CTA, whose MMA thread writes both CTAs' accumulators)
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(peer_addr(bar_tempty + 8 * as, 0));
+      } else {
+        mbar_arrive(bar_tempty + 8 * as);
+      }
     }
   }
 
@@ -1049,8 +1132,9 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (warp == 0 && lane == 0) {
-      // wait (bounded) for the tile loads still in flight: the latest fill of every stage
+    if (warp == 0 && lane == 0 && rank == 0) {
+      // wait (bounded) for the tile loads still in flight: the latest fill of every stage (a pair: the first
+      // CTA's barriers count both CTAs' bytes)
       uint32_t s = p_stage, ph = p_phase;
       const uint32_t n = issued < n_stages ? issued : n_stages;
       for (uint32_t i = 0; i < n; ++i) {
@@ -1058,17 +1142,22 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (!mbar_try(bar_full + 8 * s, ph)) mbar_wait_slow(bar_full + 8 * s, ph, abort_flag, DRAIN_NS, false);
       }
     }
-    if (warp == 1 && lane == 0) {
+    if (warp == 1 && lane == 0 && rank == 0) {
       // wait (bounded) for every MMA issued so far
-      umma_commit(bar_drain);
+      if constexpr (PAIR) asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_drain) : "memory");
+      else umma_commit(bar_drain);
       if (!mbar_try(bar_drain, 0)) mbar_wait_slow(bar_drain, 0, abort_flag, DRAIN_NS, false);
     }
+    if (PAIR && rank == 1 && warp == 0) __nanosleep(50000);  // (this CTA's own last copies land meanwhile)
     if (threadIdx.x == 0) atomicMax(prm.status, (unsigned int)ST_TIMEOUT);
     __syncthreads();
   }
+  // a pair leaves together: the first CTA's MMAs read the second one's shared memory and write its tensor memory
+  if constexpr (PAIR) cluster_sync();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 #undef MW
 }
@@ -1089,6 +1178,8 @@ std::mutex g_mm_mu;
 EncodeTiledFn g_encode_tiled = nullptr;
 bool g_attr_set[64] = {};
 int g_tail_split = 1;  // dvm_set_matmul_tail_split
+int g_cta_pairs = 1;   // dvm_set_matmul_cta_pairs: 0 never, 1 where the cost estimate favours them, 2 wherever possible
+int g_pair_clusters[64] = {};  // CTA pairs the device runs at a time (0: not asked yet, -1: none)
 
 // Workspace of the tail split, one per (device, stream): launches of one stream run in order, so they may share
 // it; launches of different streams may overlap, so they do not.  Allocated at the first launch that splits.
@@ -1166,6 +1257,27 @@ int mm_make_map(EncodeTiledFn fn, CUtensorMap* map, void* ptr, uint64_t rows, ui
 
 }  // namespace
 
+// Whether a launch of mblocks x nblocks tiles (of 128 rows) should run on CTA pairs (tiles of 256 rows): the
+// estimated time of both ways in tile times.  One CTA per tile: the full waves, plus a last wave that costs a
+// whole tile time, or with the tail split 1 / s of it and the exchange of the parts (about 8 us, a tile time
+// being about 0.47 us per k block).  Pairs: whole waves of the tiles of 256 rows over the clusters the device
+// runs at a time, each 1.12 times faster (measured on the large launches of both sweeps: what a third less
+// shared-memory traffic buys).
+bool mm_prefers_pairs(uint32_t mblocks, uint32_t nblocks, uint32_t kblocks, uint32_t sms, uint32_t clusters) {
+  if (g_cta_pairs >= 2) return true;
+  const uint64_t t1 = (uint64_t)mblocks * nblocks;
+  const uint32_t r1 = (uint32_t)(t1 % sms);
+  double single = (double)(t1 / sms);
+  if (r1) {
+    const bool splits = g_tail_split && 2 * r1 <= sms && kblocks >= 16;
+    const uint32_t s = sms / r1 < 4 ? sms / r1 : 4;
+    single += splits ? 1.0 / s + 17.0 / kblocks : 1.0;
+  }
+  const uint64_t t2 = (uint64_t)((mblocks + 1) / 2) * nblocks;
+  const double pair = (double)((t2 + clusters - 1) / clusters) / 1.12;
+  return pair < single;
+}
+
 int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors, int n_tensors, cudaStream_t stream) {
   MmView v;
   if (!mm_view(code, n_words, &v)) return DVM_ERR_BAD_CODE;
@@ -1207,21 +1319,58 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   if ((st = mm_make_map(fn, &mb0, pb0, K, N, 64, DVM_MM_BLOCK_K)) != DVM_OK) return st;
   if ((st = mm_make_map(fn, &mb1, pb1, K, N, 64, DVM_MM_BLOCK_K)) != DVM_OK) return st;
 
-  const uint32_t n_stages = dvm::mm::MAX_STAGES;
-  const size_t smem = 1024 + (size_t)n_stages * dvm::mm::STAGE_BYTES + (size_t)v.ntmp * dvm::mm::TMP_BYTES + 128;
+  // (both variants hold 192 KB of stages: 4 x 48 KB, or 6 x 32 KB per CTA of a pair)
+  const size_t smem = 1024 + (size_t)dvm::mm::STAGES_SINGLE * dvm::mm::STAGE_BYTES + (size_t)v.ntmp * dvm::mm::TMP_BYTES +
+                      dvm::mm::BAR_BYTES;
+  static_assert(dvm::mm::STAGES_SINGLE * dvm::mm::STAGE_BYTES == dvm::mm::STAGES_PAIR * dvm::mm::STAGE_PAIR, "one shared-memory size");
   int devid = 0;
   DVM_CUDA(cudaGetDevice(&devid));
+  if (devid < 0 || devid >= 64) return DVM_ERR_INVALID_ARG;
+  int pair_clusters = 0;
   {
     std::lock_guard<std::mutex> lk(g_mm_mu);
-    if (devid >= 0 && devid < 64 && !g_attr_set[devid]) {
-      DVM_CUDA(cudaFuncSetAttribute(dvm::mm::dvm_mm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024));
+    if (!g_attr_set[devid]) {
+      DVM_CUDA(cudaFuncSetAttribute(dvm::mm::dvm_mm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024));
+      DVM_CUDA(cudaFuncSetAttribute(dvm::mm::dvm_mm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024));
       g_attr_set[devid] = true;
     }
+    if (g_pair_clusters[devid] == 0) {  // how many CTA pairs run at a time (with the largest shared-memory request)
+      cudaLaunchConfig_t cfg = {};
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.gridDim = dim3(2 * (unsigned)dev.sm_count); cfg.blockDim = dim3(dvm::mm::THREADS);
+      cfg.dynamicSmemBytes = 232448 - 1024; cfg.attrs = at; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, dvm::mm::dvm_mm_kernel<true>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+      g_pair_clusters[devid] = n > 0 ? n : -1;
+    }
+    pair_clusters = g_pair_clusters[devid] > 0 ? g_pair_clusters[devid] : 0;
   }
   P.status = dev.scratch;
   P.n_words = (uint32_t)n_words;
-  P.n_stages = n_stages;
+  P.n_stages = dvm::mm::STAGES_SINGLE;
+  P.pair_tiles = P.pair_mblocks = 0;
   const uint32_t tiles = code[DVM_H_N_TILES];
+  // CTA pairs (see dvm_mm_kernel): tiles of 256 rows
+  const uint32_t mblocks = x[DVM_MM_MBLOCKS], nblocks = x[DVM_MM_NBLOCKS];
+  if (g_cta_pairs && pair_clusters > 0 && mblocks >= 2 && mm_prefers_pairs(mblocks, nblocks, x[DVM_MM_KBLOCKS], (uint32_t)dev.sm_count, (uint32_t)pair_clusters)) {
+    P.split_s = P.split_r = P.split_first = P.split_kb = 0;
+    P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
+    P.n_stages = dvm::mm::STAGES_PAIR;
+    P.pair_mblocks = (mblocks + 1) / 2;
+    P.pair_tiles = P.pair_mblocks * nblocks;
+    const uint32_t pairs = P.pair_tiles < (uint32_t)pair_clusters ? P.pair_tiles : (uint32_t)pair_clusters;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(dvm::mm::THREADS);
+    cfg.dynamicSmemBytes = smem; cfg.stream = stream; cfg.attrs = at; cfg.numAttrs = 1;
+    DVM_CUDA(cudaLaunchKernelEx(&cfg, dvm::mm::dvm_mm_kernel<true>, ma, mb0, mb1, P));
+    dvm_count_launch();
+    return DVM_OK;
+  }
   int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
   // Tail split: the last wave of r < sms / 2 tiles would leave most SMs idle for a whole tile time; instead
   // s = min(4, sms / r) CTAs take each of its tiles, a share of the k blocks each (see MMParams).
@@ -1247,13 +1396,14 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
       if (tiles < sms) grid = (int)(tail * s_eff);
     }
   }
-  dvm::mm::dvm_mm_kernel<<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);
+  dvm::mm::dvm_mm_kernel<false><<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);
   DVM_CUDA(cudaGetLastError());
   dvm_count_launch();
   return DVM_OK;
 }
 
 extern "C" void dvm_set_matmul_tail_split(int on) { g_tail_split = on; }
+extern "C" void dvm_set_matmul_cta_pairs(int mode) { g_cta_pairs = mode; }
 
 // ---- self-test of the matmul kernel's bounded wait (see dvm_selftest_bounded_wait) ----
 namespace dvm {

@@ -250,3 +250,36 @@ def test_tail_split_on_two_streams():
     for outs in res:
         check(prog, outs, want)
         assert torch.equal(outs[0], res[0][0])
+
+
+# ---- CTA pairs: two CTAs of a cluster on one tile of 256 rows (tcgen05 cta_group::2) ----
+
+@pytest.mark.parametrize("kind,M,K,N", [
+    ("addmm", 256, 128, 256),      # one tile of a pair
+    ("addmm", 129, 200, 264),      # the second CTA's rows end after one; ragged k and n
+    ("mlp", 300, 512, 392),        # three blocks of 128 rows: the last pair's second half is empty
+    ("mlp", 1024, 4096, 1536),     # both products side by side in the accumulators, 64 k blocks through 6 stages
+    ("addmm", 1000, 2048, 5000),   # 80 tiles of 256 rows: more than the device runs pairs at a time
+])
+def test_cta_pairs_equal_single_cta_kernel(kind, M, K, N):
+    prog, ins = _tail_case(kind, M, K, N, seed=M + K)
+    try:
+        dvm.set_matmul_tail_split(False)
+        dvm.set_matmul_cta_pairs(0)
+        single, _ = gpu_run(prog, ins)
+        dvm.set_matmul_cta_pairs(2)
+        pairs, _ = gpu_run(prog, ins)
+    finally:
+        dvm.set_matmul_tail_split(True)
+        dvm.set_matmul_cta_pairs(1)
+    check(prog, pairs, oracle_run(prog, ins))
+    assert not torch.isnan(pairs[0].float()).any()
+    assert torch.equal(pairs[0], single[0])  # the same k order, the same instruction shape along k
+
+
+def test_cta_pairs_default_choice_keeps_parity():
+    """The default mode picks pairs or single CTAs per launch; both routes against the oracle at one shape each."""
+    for M, K, N in ((2048, 1024, 4096), (128, 1024, 4096)):
+        prog, ins = _tail_case("addmm", M, K, N, seed=3)
+        outs, _ = gpu_run(prog, ins)
+        check(prog, outs, oracle_run(prog, ins))
