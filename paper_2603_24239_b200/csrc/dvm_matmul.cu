@@ -526,7 +526,8 @@ constexpr uint32_t WAIT_SPINS = 1u << 27;
 // Tail split (split_s >= 2): the tiles [split_first, split_first + split_r) -- the last, partial wave of the
 // launch -- are each computed by split_s CTAs, part p taking the k blocks [p * split_kb, (p + 1) * split_kb).
 // Parts 1.. write their accumulators to `ws` (partial index r * (split_s - 1) + p - 1, laid out
-// [column][row] fp32) and publish flags[4 r + p - 1] = epoch; part 0 (the tile's owner) waits
+// [column][row] fp32) and publish flags[4 r + p - 1] = epoch (on a CTA pair
+// partial index and flag index are doubled, plus the CTA's rank: each CTA's 128 rows are a part of their own); part 0 (the tile's owner) waits
 // for them, adds them to its own accumulators in tensor memory in the order of p and runs the epilogue.
 struct MMParams {
   unsigned int* status;
@@ -675,14 +676,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[CHUNK
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Bounded wait of a tile's owner for the n flags of its other parts (each becomes `epoch` once that part's
+// Bounded wait of a tile's owner for the n flags (`stride` words apart) of its other parts (each becomes `epoch` once that part's
 // accumulators are in the workspace); like mbar_wait_slow it raises the CTA's abort flag when it gives up.
-__device__ __noinline__ bool flags_wait(const uint32_t* f, uint32_t n, uint32_t epoch, volatile uint32_t* abort_flag) {
+__device__ __noinline__ bool flags_wait(const uint32_t* f, uint32_t stride, uint32_t n, uint32_t epoch, volatile uint32_t* abort_flag) {
   const unsigned long long t0 = gtimer();
   uint32_t k = 0;
   for (uint32_t spin = 0; spin < WAIT_SPINS && k < n; ++spin) {
     uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f + k) : "memory");
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f + k * stride) : "memory");
     if (v == epoch) { ++k; continue; }
     if (*abort_flag) return false;
     if (gtimer() - t0 > WAIT_NS) break;
@@ -780,13 +781,13 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   // The i-th piece of work of this CTA: whole tiles blockIdx.x + i * gridDim.x below split_first, then (tail
   // split) one part of one tail tile.
   struct Work { uint32_t tile, kb0, kb1, part, r; };
-  const uint32_t split_first = PAIR ? prm.pair_tiles : (prm.split_s >= 2 ? prm.split_first : n_tiles);
+  // (a pair counts in clusters: its tiles, its grid)
+  const uint32_t split_first = prm.split_s >= 2 ? prm.split_first : (PAIR ? prm.pair_tiles : n_tiles);
   auto work_at = [&](uint32_t i, Work& w) -> bool {
     const uint32_t t = PAIR ? (blockIdx.x >> 1) + i * (gridDim.x >> 1) : blockIdx.x + i * gridDim.x;
     w.part = 0; w.r = 0; w.kb0 = 0; w.kb1 = k_blocks;
     if (t < split_first) { w.tile = t; return true; }
-    if constexpr (PAIR) return false;
-    const uint32_t u = t - split_first;  // (split_first is a multiple of the grid size: u = blockIdx.x in the round after the whole tiles)
+    const uint32_t u = t - split_first;  // (split_first is a multiple of the grid size: u = this CTA's or pair's index in the round after the whole tiles)
     if (prm.split_s < 2 || u >= prm.split_r * prm.split_s) return false;
     w.part = u / prm.split_r;
     w.r = u - w.part * prm.split_r;
@@ -795,7 +796,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     w.kb1 = min(k_blocks, w.kb0 + prm.split_kb);
     return true;
   };
-  const bool split = !PAIR && prm.split_s >= 2;
+  const bool split = prm.split_s >= 2;
   // first row and column of a tile for this CTA (a pair: blocks of 256 rows, this CTA's half of them)
   const uint32_t mbl = PAIR ? prm.pair_mblocks : m_blocks;
   auto tile_m0 = [&](uint32_t t) -> int { return (int)(t % mbl) * (PAIR ? 2 * BLOCK_M : BLOCK_M) + (int)rank * BLOCK_M; };
@@ -883,6 +884,16 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     float* const tmp_mine = (float*)(sm + tmp_base) + erow * 4;
     uint32_t it = 0;
     Work w;
+    // the epilogue is done with accumulator stage `as` (a pair: told to the first CTA, whose MMA thread writes both
+    // CTAs' accumulators, once per warp)
+    auto release_acc = [&](uint32_t as) {
+      if constexpr (PAIR) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(peer_addr(bar_tempty + 8 * as, 0));
+      } else {
+        mbar_arrive(bar_tempty + 8 * as);
+      }
+    };
     for (; work_at(it, w); ++it) {
       const uint32_t t = w.tile;
       const uint32_t as = it & 1, aph = (it >> 1) & 1;
@@ -890,11 +901,12 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
       if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       if (split && t >= split_first) {
-        // ---- a tail tile computed in parts (see MMParams) ----
+        // ---- a tail tile computed in parts (see MMParams; a pair: each CTA's rows are a part of their own) ----
+        constexpr uint32_t NR = PAIR ? 2 : 1;
         const uint32_t used_chunks = (uint32_t)(nb == 2 ? ACC_COLS : tile_n) / CHUNK;
         const uint32_t acc0 = lane_addr + as * ACC_COLS;
         if (w.part > 0) {  // this CTA's accumulators go to the workspace; the owner is told; nothing else to do here
-          float* const dst0 = prm.ws + (size_t)(w.r * (prm.split_s - 1) + (w.part - 1)) * PART_FLOATS + erow;
+          float* const dst0 = prm.ws + ((size_t)(w.r * (prm.split_s - 1) + (w.part - 1)) * NR + rank) * PART_FLOATS + erow;
           for (uint32_t c = 0; c < used_chunks; ++c) {
             float v[CHUNK];
             tmem_ld32(acc0 + c * CHUNK, v);
@@ -906,15 +918,15 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
           tc_fence_before();
           asm volatile("bar.sync 1, 128;" ::: "memory");
           if (threadIdx.x == 64) {
-            uint32_t* f = prm.flags + 4 * w.r + (w.part - 1);
+            uint32_t* f = prm.flags + (4 * w.r + (w.part - 1)) * NR + rank;
             asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(f), "r"(prm.epoch) : "memory");
           }
-          mbar_arrive(bar_tempty + 8 * as);
+          release_acc(as);
           continue;
         }
         // the owner: every other part's accumulators, added in the order of the parts
         if (threadIdx.x == 64) {
-          const bool ok = flags_wait(prm.flags + 4 * w.r, prm.split_s - 1, prm.epoch, abort_flag);
+          const bool ok = flags_wait(prm.flags + 4 * w.r * NR + rank, NR, prm.split_s - 1, prm.epoch, abort_flag);
           __threadfence();
           *split_ok = ok ? 1u : 0u;
         }
@@ -927,7 +939,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
           float x[MAX_SPLIT - 1][CHUNK];
 #pragma unroll
           for (uint32_t p2 = 0; p2 < MAX_SPLIT - 1; ++p2) {
-            const float* src = prm.ws + (size_t)(w.r * (prm.split_s - 1) + p2) * PART_FLOATS + (size_t)c * CHUNK * BLOCK_M + erow;
+            const float* src = prm.ws + ((size_t)(w.r * (prm.split_s - 1) + p2) * NR + rank) * PART_FLOATS + (size_t)c * CHUNK * BLOCK_M + erow;
 #pragma unroll
             for (int k = 0; k < CHUNK; ++k) x[p2][k] = p2 + 1 < prm.split_s ? __ldcg(src + k * BLOCK_M) : 0.0f;
           }
@@ -1119,12 +1131,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
       }
       // this accumulator stage may be overwritten by the tile after next
       tc_fence_before();
-      if constexpr (PAIR) {  // (told to the first CTA, whose MMA thread writes both CTAs' accumulators)
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(peer_addr(bar_tempty + 8 * as, 0));
-      } else {
-        mbar_arrive(bar_tempty + 8 * as);
-      }
+      release_acc(as);
     }
   }
 
@@ -1257,24 +1264,38 @@ int mm_make_map(EncodeTiledFn fn, CUtensorMap* map, void* ptr, uint64_t rows, ui
 
 }  // namespace
 
-// Whether a launch of mblocks x nblocks tiles (of 128 rows) should run on CTA pairs (tiles of 256 rows): the
-// estimated time of both ways in tile times.  One CTA per tile: the full waves, plus a last wave that costs a
-// whole tile time, or with the tail split 1 / s of it and the exchange of the parts (about 8 us, a tile time
-// being about 0.47 us per k block).  Pairs: whole waves of the tiles of 256 rows over the clusters the device
-// runs at a time, each 1.12 times faster (measured on the large launches of both sweeps: what a third less
-// shared-memory traffic buys).
+// Tail split of a launch of `tiles` tiles over `units` CTAs (or CTA pairs, nr = 2 CTAs each): the last wave, its
+// CTAs per tile and k blocks per part; false when the launch does not split.
+struct SplitPlan { uint32_t first, r, s, kb; };
+bool mm_plan_split(uint32_t tiles, uint32_t units, uint32_t kblocks, uint32_t nr, SplitPlan* sp) {
+  const uint32_t tail = tiles % units;
+  if (!g_tail_split || !tail || 2 * tail > units || kblocks < 16) return false;
+  uint32_t s_want = units / tail;
+  if (s_want > dvm::mm::MAX_SPLIT) s_want = dvm::mm::MAX_SPLIT;
+  const uint32_t per = (kblocks + s_want - 1) / s_want;
+  const uint32_t s_eff = (kblocks + per - 1) / per;
+  if (s_eff < 2 || (size_t)tail * (s_eff - 1) * nr > SPLIT_WS_PARTS || (4 * (size_t)tail + 4) * nr > SPLIT_FLAG_WORDS) return false;
+  sp->first = tiles - tail; sp->r = tail; sp->s = s_eff; sp->kb = per;
+  return true;
+}
+// Estimated time of such a launch in tile times: the full waves, plus a last wave that costs a whole tile time,
+// or with the tail split 1 / s of it and the exchange of the parts (about 8 us, a tile time being about 0.47 us
+// per k block).
+double mm_waves(uint32_t tiles, uint32_t units, uint32_t kblocks, uint32_t nr) {
+  double w = (double)(tiles / units);
+  if (tiles % units) {
+    SplitPlan sp;
+    w += mm_plan_split(tiles, units, kblocks, nr, &sp) ? 1.0 / sp.s + 17.0 / kblocks : 1.0;
+  }
+  return w;
+}
+// Whether a launch of mblocks x nblocks tiles (of 128 rows) should run on CTA pairs (tiles of 256 rows, over the
+// clusters the device runs at a time): pairs run a tile 1.12 times faster (measured on the large launches of both
+// sweeps: what a third less shared-memory traffic buys) but come in whole blocks of 256 rows and half as many units.
 bool mm_prefers_pairs(uint32_t mblocks, uint32_t nblocks, uint32_t kblocks, uint32_t sms, uint32_t clusters) {
   if (g_cta_pairs >= 2) return true;
-  const uint64_t t1 = (uint64_t)mblocks * nblocks;
-  const uint32_t r1 = (uint32_t)(t1 % sms);
-  double single = (double)(t1 / sms);
-  if (r1) {
-    const bool splits = g_tail_split && 2 * r1 <= sms && kblocks >= 16;
-    const uint32_t s = sms / r1 < 4 ? sms / r1 : 4;
-    single += splits ? 1.0 / s + 17.0 / kblocks : 1.0;
-  }
-  const uint64_t t2 = (uint64_t)((mblocks + 1) / 2) * nblocks;
-  const double pair = (double)((t2 + clusters - 1) / clusters) / 1.12;
+  const double single = mm_waves(mblocks * nblocks, sms, kblocks, 1);
+  const double pair = mm_waves(((mblocks + 1) / 2) * nblocks, clusters, kblocks, 2) / 1.12;
   return pair < single;
 }
 
@@ -1360,7 +1381,17 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
     P.n_stages = dvm::mm::STAGES_PAIR;
     P.pair_mblocks = (mblocks + 1) / 2;
     P.pair_tiles = P.pair_mblocks * nblocks;
-    const uint32_t pairs = P.pair_tiles < (uint32_t)pair_clusters ? P.pair_tiles : (uint32_t)pair_clusters;
+    uint32_t pairs = P.pair_tiles < (uint32_t)pair_clusters ? P.pair_tiles : (uint32_t)pair_clusters;
+    SplitPlan plan;
+    if (mm_plan_split(P.pair_tiles, (uint32_t)pair_clusters, x[DVM_MM_KBLOCKS], 2, &plan)) {
+      if (SplitSpace* sp = split_space(devid, stream)) {
+        P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb;
+        P.ws = sp->ws; P.flags = sp->flags;
+        if (++sp->epoch == 0) sp->epoch = 1;
+        P.epoch = sp->epoch;
+        if (P.pair_tiles < (uint32_t)pair_clusters) pairs = plan.r * plan.s;
+      }
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1372,28 +1403,19 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
     return DVM_OK;
   }
   int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
-  // Tail split: the last wave of r < sms / 2 tiles would leave most SMs idle for a whole tile time; instead
+  // Tail split: the last wave of r <= sms / 2 tiles would leave most SMs idle for a whole tile time; instead
   // s = min(4, sms / r) CTAs take each of its tiles, a share of the k blocks each (see MMParams).
   P.split_s = P.split_r = P.split_first = P.split_kb = 0;
   P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
-  const uint32_t sms = (uint32_t)dev.sm_count, kblocks = x[DVM_MM_KBLOCKS];
-  const uint32_t tail = tiles % sms;
-  if (g_tail_split && tail && 2 * tail <= sms && kblocks >= 16 && sms <= 148) {
-    uint32_t s_want = sms / tail;
-    if (s_want > dvm::mm::MAX_SPLIT) s_want = dvm::mm::MAX_SPLIT;
-    const uint32_t per = (kblocks + s_want - 1) / s_want;
-    const uint32_t s_eff = (kblocks + per - 1) / per;
-    SplitSpace* sp = (s_eff >= 2 && (size_t)tail * (s_eff - 1) <= SPLIT_WS_PARTS) ? split_space(devid, stream) : nullptr;
-    if (sp) {
-      P.split_first = tiles - tail;
-      P.split_r = tail;
-      P.split_s = s_eff;
-      P.split_kb = per;
-      P.ws = sp->ws;
-      P.flags = sp->flags;
+  const uint32_t sms = (uint32_t)dev.sm_count;
+  SplitPlan plan;
+  if (mm_plan_split(tiles, sms, x[DVM_MM_KBLOCKS], 1, &plan)) {
+    if (SplitSpace* sp = split_space(devid, stream)) {
+      P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb;
+      P.ws = sp->ws; P.flags = sp->flags;
       if (++sp->epoch == 0) sp->epoch = 1;
       P.epoch = sp->epoch;
-      if (tiles < sms) grid = (int)(tail * s_eff);
+      if (tiles < sms) grid = (int)(plan.r * plan.s);
     }
   }
   dvm::mm::dvm_mm_kernel<false><<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);

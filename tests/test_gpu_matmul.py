@@ -283,3 +283,29 @@ def test_cta_pairs_default_choice_keeps_parity():
         prog, ins = _tail_case("addmm", M, K, N, seed=3)
         outs, _ = gpu_run(prog, ins)
         check(prog, outs, oracle_run(prog, ins))
+
+
+@pytest.mark.parametrize("kind,M,K,N", [
+    ("addmm", 256, 1024, 512),     # two tiles of 256 rows: four pairs each, 16 k blocks shared 4 / 4 / 4 / 4
+    ("mlp", 512, 2048, 1280),      # 20 tiles: three pairs each
+    ("addmm", 4096, 1088, 4864),   # 304 tiles: four full waves of pairs, then 8 tiles by four pairs each, 17 k blocks
+    ("mlp", 300, 1024, 3000),      # the last pair's second CTA holds 44 rows; ragged n
+])
+def test_tail_split_on_cta_pairs(kind, M, K, N):
+    prog, ins = _tail_case(kind, M, K, N, seed=M + N)
+    try:
+        dvm.set_matmul_cta_pairs(2)
+        outs, _ = gpu_run(prog, ins)
+        again, _ = gpu_run(prog, ins)
+        dvm.set_matmul_tail_split(False)
+        plain, _ = gpu_run(prog, ins)
+    finally:
+        dvm.set_matmul_tail_split(True)
+        dvm.set_matmul_cta_pairs(1)
+    want = oracle_run(prog, ins)
+    check(prog, outs, want)
+    check(prog, plain, want)
+    assert not torch.isnan(outs[0].float()).any()
+    assert torch.equal(outs[0], again[0])
+    a, b = outs[0].float(), plain[0].float()
+    assert (a - b).abs().max().item() <= 2.0 ** -7 * b.abs().max().item()
