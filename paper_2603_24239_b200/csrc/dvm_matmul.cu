@@ -16,6 +16,10 @@
 //               32-column chunks of the accumulators out of tensor memory (tcgen05.ld), runs the
 //               epilogue code on them in registers and stores the narrowed result; it overlaps the
 //               next tile's MMAs (the other accumulator stage).
+// Two forms, chosen per launch (dvm_launch_matmul): single CTAs as above, or CTA pairs -- two CTAs of a cluster on
+// a tile of 256 rows with tcgen05 cta_group::2, each loading its own A rows and half of the B tile (see
+// dvm_mm_kernel).  In both, a last wave of tiles that would fill at most half of the device is split along k
+// among several CTAs (pairs) per tile (see MMParams).
 // Every wait on an mbarrier is bounded (time and iteration limit): when one runs out the CTA raises its
 // abort flag, every role leaves its loop, copies and MMAs in flight are awaited (bounded again), tensor
 // memory is released and the status word reports DVM_ERR_DEVICE_TIMEOUT.
