@@ -229,7 +229,7 @@ void dvm_set_lean_kernel(int on);
 /* Matmul launches (Sec. 4.2, matrix operations): when the last wave of output tiles would occupy at most half
  * of the SMs, each of its tiles is computed by up to four CTAs, every one taking a share of the k blocks; the
  * shares meet in a library-owned fp32 workspace (one per device and stream, 15 MB, allocated by the first launch
- * that needs it; none is made while the stream is being captured -- such launches run unsplit) and are added in
+ * that needs it; launches into a stream that is being captured run unsplit) and are added in
  * a fixed order, so results are deterministic.  They differ from the unsplit result by fp32 rounding of the
  * partial sums.  on = 0 switches the split off.  Default 1. */
 void dvm_set_matmul_tail_split(int on);

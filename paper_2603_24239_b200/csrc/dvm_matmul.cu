@@ -1207,18 +1207,20 @@ constexpr size_t SPLIT_FLAG_WORDS = 4 * 160;
 SplitSpace g_split[MAX_SPLIT_SPACES];
 int g_n_split = 0;
 
-// The workspace of (device, stream), or NULL (then the launch does not split): none is made while the stream is
-// being captured (an allocation does not belong into a graph) or when every slot is taken.
+// The workspace of (device, stream), or NULL (then the launch does not split): while the stream is being captured,
+// or when every slot is taken.
 SplitSpace* split_space(int device, cudaStream_t stream) {
-  std::lock_guard<std::mutex> lk(g_mm_mu);
-  for (int i = 0; i < g_n_split; ++i)
-    if (g_split[i].device == device && g_split[i].stream == stream) return &g_split[i];
-  if (g_n_split == MAX_SPLIT_SPACES) return nullptr;
+  // A captured launch would be replayed with the epoch number it was captured with, which its flags then already
+  // hold: launches into a capturing stream never split (nor would an allocation belong into a graph).
   cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
     cudaGetLastError();
     return nullptr;
   }
+  std::lock_guard<std::mutex> lk(g_mm_mu);
+  for (int i = 0; i < g_n_split; ++i)
+    if (g_split[i].device == device && g_split[i].stream == stream) return &g_split[i];
+  if (g_n_split == MAX_SPLIT_SPACES) return nullptr;
   SplitSpace sp = {device, stream, nullptr, nullptr, 0};
   if (cudaMalloc(&sp.ws, SPLIT_WS_PARTS * dvm::mm::PART_FLOATS * sizeof(float)) != cudaSuccess) {
     cudaGetLastError();

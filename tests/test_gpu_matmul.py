@@ -309,3 +309,30 @@ def test_tail_split_on_cta_pairs(kind, M, K, N):
     assert torch.equal(outs[0], again[0])
     a, b = outs[0].float(), plain[0].float()
     assert (a - b).abs().max().item() <= 2.0 ** -7 * b.abs().max().item()
+
+
+def test_matmul_launch_inside_a_cuda_graph():
+    """A captured matmul launch replays correctly on new data: launches into a capturing stream never use the
+    tail split (a replay would meet the flags of its own earlier run), pairs and single CTAs both replay."""
+    for M, K, N in ((128, 1024, 2560), (1024, 1024, 4864)):   # shapes that split when launched directly
+        prog, ins = _tail_case("addmm", M, K, N, seed=21)
+        p = dvm.program_from_nodes(prog.nodes)
+        dev = [t.cuda() for t in ins]
+        code = dvm.encode(p, [tuple(t.shape) for t in dev])
+        out = torch.empty(code.out_shapes[0], dtype=torch.bfloat16, device="cuda")
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            dvm.launch(code, dev + [out], s)   # set-up outside the capture
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            dvm.launch(code, dev + [out], s)
+        for rep in range(3):
+            dev[0].copy_(wl.randn((M, K), torch.bfloat16, 100 + rep).cuda())
+            out.fill_(float("nan"))
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            assert dvm.last_device_status() == 0
+            want = oracle_run(prog, [dev[0].cpu(), ins[1], ins[2]])
+            check(prog, [out], want)
