@@ -767,7 +767,7 @@ WORKLOADS = {"views": ViewsWorkload, "ifelse": IfElseWorkload, "addmm": AddmmWor
 for _W in (C1Workload, C2Workload, C3Workload, C4Workload, IfElseWorkload, ViewsWorkload):   # the memory-bound sweeps: work = algorithmic bytes
     _W.metric, _W.unit, _W.scale, _W.bound = "hbm_gbs_dynamic_shape_sweep", "GB/s", 1e9, "hbm"
     _W.kernel, _W.peak_key = "dvm_vm_kernel", "hbm_gbs"
-for _W in (C1Workload, C2Workload, C3Workload, IfElseWorkload):   # one program per launch that the lean interpreter runs
+for _W in (C1Workload, C2Workload, C3Workload, IfElseWorkload, ViewsWorkload):   # one program per launch that the lean interpreter runs
     _W.kernel = "dvm_vm_lean_kernel"
 
 
