@@ -226,9 +226,10 @@ int dvm_get_min_resident_ctas(void);
  * Default 1.  Both interpreters run the same bytecode and give results inside the same tolerances. */
 void dvm_set_lean_kernel(int on);
 
-/* Matmul launches (Sec. 4.2, matrix operations): when the last wave of output tiles would occupy at most half
- * of the SMs, each of its tiles is computed by up to four CTAs, every one taking a share of the k blocks; the
- * shares meet in a library-owned fp32 workspace (one per device and stream, 15 MB, allocated by the first launch
+/* Matmul launches (Sec. 4.2, matrix operations): the tiles of a last, partial wave are shared along k -- a small
+ * wave gives each tile up to four CTAs (or CTA pairs), a larger one is cut into equal ranges of its k blocks over
+ * all of them -- whenever the k blocks saved outweigh the exchange (decided per launch from its shape).  The
+ * shares meet in a library-owned fp32 workspace (one per device and stream, 26 MB, allocated by the first launch
  * that needs it; launches into a stream that is being captured run unsplit) and are added in
  * a fixed order, so results are deterministic.  They differ from the unsplit result by fp32 rounding of the
  * partial sums.  on = 0 switches the split off.  Default 1. */

@@ -528,18 +528,24 @@ constexpr unsigned long long DRAIN_NS = 200000000ull;   // limit of a wait for w
 constexpr uint32_t WAIT_SPINS = 1u << 27;
 
 // Tail split (split_s >= 2): the tiles [split_first, split_first + split_r) -- the last, partial wave of the
-// launch -- are each computed by split_s CTAs, part p taking the k blocks [p * split_kb, (p + 1) * split_kb).
-// Parts 1.. write their accumulators to `ws` (partial index r * (split_s - 1) + p - 1, laid out
-// [column][row] fp32) and publish flags[4 r + p - 1] = epoch (on a CTA pair
-// partial index and flag index are doubled, plus the CTA's rank: each CTA's 128 rows are a part of their own); part 0 (the tile's owner) waits
-// for them, adds them to its own accumulators in tensor memory in the order of p and runs the epilogue.
+// launch -- are shared along k.  Their k blocks form one line, tile a at [a * split_kbp, a * split_kbp + k_blocks);
+// unit c (a CTA, or a CTA pair) takes the blocks [c * split_kb, (c + 1) * split_kb) of that line, i.e. a part of
+// one tile, or the end of one tile and the start of the next.  Two layouts: a small last wave (at most half of
+// the units) gives every tile s units of its own (split_kbp = s * split_kb: the parts are aligned to the tiles);
+// a larger one is cut into equal ranges over all units (split_kbp = k_blocks: a tile has up to three parts).
+// The unit holding a tile's first block owns it.  The other parts p = 1.. write their accumulators to `ws` (partial
+// index a * (split_s - 1) + p - 1, laid out [column][row] fp32) and publish flags[4 a + p - 1] = epoch (on a CTA
+// pair partial index and flag index are doubled, plus the CTA's rank: each CTA's 128 rows are a part of their
+// own); the owner waits for them, adds them to its own accumulators in tensor memory in the order of p and runs
+// the epilogue.  A unit works through its range in order, so it dumps (the end of a tile) before it waits (as the
+// owner of the next): nobody waits for a unit that waits.  split_s is the largest number of parts of any tile.
 struct MMParams {
   unsigned int* status;
   uint32_t pair_tiles, pair_mblocks;  // CTA pairs: tiles of 256 rows, blocks of 256 rows
   float* ws;
   uint32_t* flags;
   uint32_t epoch;
-  uint32_t split_first, split_r, split_s, split_kb;
+  uint32_t split_first, split_r, split_s, split_kb, split_kbp;
   uint32_t n_words;
   uint32_t n_stages;
   uint32_t words[DVM_MM_MAX_WORDS];
@@ -784,20 +790,32 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
   // The i-th piece of work of this CTA: whole tiles blockIdx.x + i * gridDim.x below split_first, then (tail
   // split) one part of one tail tile.
-  struct Work { uint32_t tile, kb0, kb1, part, r; };
+  struct Work { uint32_t tile, kb0, kb1, part, parts, r; };
   // (a pair counts in clusters: its tiles, its grid)
   const uint32_t split_first = prm.split_s >= 2 ? prm.split_first : (PAIR ? prm.pair_tiles : n_tiles);
+  const uint32_t unit = PAIR ? blockIdx.x >> 1 : blockIdx.x, n_units = PAIR ? gridDim.x >> 1 : gridDim.x;
   auto work_at = [&](uint32_t i, Work& w) -> bool {
-    const uint32_t t = PAIR ? (blockIdx.x >> 1) + i * (gridDim.x >> 1) : blockIdx.x + i * gridDim.x;
-    w.part = 0; w.r = 0; w.kb0 = 0; w.kb1 = k_blocks;
+    const uint32_t t = unit + i * n_units;
+    w.part = 0; w.parts = 1; w.r = 0; w.kb0 = 0; w.kb1 = k_blocks;
     if (t < split_first) { w.tile = t; return true; }
-    const uint32_t u = t - split_first;  // (split_first is a multiple of the grid size: u = this CTA's or pair's index in the round after the whole tiles)
-    if (prm.split_s < 2 || u >= prm.split_r * prm.split_s) return false;
-    w.part = u / prm.split_r;
-    w.r = u - w.part * prm.split_r;
-    w.tile = split_first + w.r;
-    w.kb0 = w.part * prm.split_kb;
-    w.kb1 = min(k_blocks, w.kb0 + prm.split_kb);
+    if (prm.split_s < 2) return false;
+    // the q-th tile this unit's range of the tail's k blocks touches (split_first is a multiple of the units)
+    const uint32_t q = (t - split_first) / n_units;
+    const uint32_t W = prm.split_kb, kbp = prm.split_kbp;
+    const uint32_t g0 = unit * W, gend = (prm.split_r - 1) * kbp + k_blocks;
+    if (g0 >= gend) return false;
+    const uint32_t g1 = min(g0 + W, gend);
+    const uint32_t a = g0 / kbp + q;
+    if (a >= prm.split_r) return false;
+    const uint32_t s0 = max(g0, a * kbp), s1 = min(g1, a * kbp + k_blocks);
+    if (s0 >= s1) return false;
+    const uint32_t first_unit = (a * kbp) / W;  // the tile's owner
+    w.r = a;
+    w.tile = split_first + a;
+    w.kb0 = s0 - a * kbp;
+    w.kb1 = s1 - a * kbp;
+    w.part = unit - first_unit;
+    w.parts = (a * kbp + k_blocks - 1) / W - first_unit + 1;
     return true;
   };
   const bool split = prm.split_s >= 2;
@@ -904,7 +922,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
       const bool got = mbar_wait(bar_tfull + 8 * as, aph, abort_flag);
       if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
-      if (split && t >= split_first) {
+      if (split && t >= split_first && w.parts > 1) {
         // ---- a tail tile computed in parts (see MMParams; a pair: each CTA's rows are a part of their own) ----
         constexpr uint32_t NR = PAIR ? 2 : 1;
         const uint32_t used_chunks = (uint32_t)(nb == 2 ? ACC_COLS : tile_n) / CHUNK;
@@ -930,7 +948,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
         // the owner: every other part's accumulators, added in the order of the parts
         if (threadIdx.x == 64) {
-          const bool ok = flags_wait(prm.flags + 4 * w.r * NR + rank, NR, prm.split_s - 1, prm.epoch, abort_flag);
+          const bool ok = flags_wait(prm.flags + 4 * w.r * NR + rank, NR, w.parts - 1, prm.epoch, abort_flag);
           __threadfence();
           *split_ok = ok ? 1u : 0u;
         }
@@ -945,7 +963,7 @@ dvm_mm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
           for (uint32_t p2 = 0; p2 < MAX_SPLIT - 1; ++p2) {
             const float* src = prm.ws + ((size_t)(w.r * (prm.split_s - 1) + p2) * NR + rank) * PART_FLOATS + (size_t)c * CHUNK * BLOCK_M + erow;
 #pragma unroll
-            for (int k = 0; k < CHUNK; ++k) x[p2][k] = p2 + 1 < prm.split_s ? __ldcg(src + k * BLOCK_M) : 0.0f;
+            for (int k = 0; k < CHUNK; ++k) x[p2][k] = p2 + 1 < w.parts ? __ldcg(src + k * BLOCK_M) : 0.0f;
           }
 #pragma unroll
           for (uint32_t p2 = 0; p2 < MAX_SPLIT - 1; ++p2) {
@@ -1202,7 +1220,7 @@ struct SplitSpace {
   uint32_t epoch;
 };
 constexpr int MAX_SPLIT_SPACES = 16;
-constexpr size_t SPLIT_WS_PARTS = 112;  // partial accumulators: max over r of r * (min(4, sms / r) - 1) for up to 148 SMs, rounded up
+constexpr size_t SPLIT_WS_PARTS = 200;  // partial accumulators of 128 KB: a last wave of up to two thirds of 148 units with two exchanged parts per tile
 constexpr size_t SPLIT_FLAG_WORDS = 4 * 160;
 SplitSpace g_split[MAX_SPLIT_SPACES];
 int g_n_split = 0;
@@ -1270,28 +1288,61 @@ int mm_make_map(EncodeTiledFn fn, CUtensorMap* map, void* ptr, uint64_t rows, ui
 
 }  // namespace
 
-// Tail split of a launch of `tiles` tiles over `units` CTAs (or CTA pairs, nr = 2 CTAs each): the last wave, its
-// CTAs per tile and k blocks per part; false when the launch does not split.
-struct SplitPlan { uint32_t first, r, s, kb; };
+// Tail split of a launch of `tiles` tiles over `units` CTAs (or CTA pairs, nr = 2 CTAs each), see MMParams: the
+// first tile of the last wave, its tiles, the most parts of a tile, the k blocks per unit and the tile pitch of
+// the k line; false when the launch does not split.  A split saves the k blocks a unit no longer computes (0.47 us
+// each) and costs the exchange: about 8 us, plus 0.2 us per 128-KB part that crosses L2 at the same moment
+// (measured on both sweeps: two parts of 34 tiles on pairs cost 25 us, four parts of 2 tiles 10 us).
+struct SplitPlan { uint32_t first, r, s, kb, kbp, units_used; double cost_blocks; };
+constexpr double kUsPerKBlock = 0.47, kExchangeUs = 8.0, kUsPerPart = 0.2;
 bool mm_plan_split(uint32_t tiles, uint32_t units, uint32_t kblocks, uint32_t nr, SplitPlan* sp) {
   const uint32_t tail = tiles % units;
-  if (!g_tail_split || !tail || 2 * tail > units || kblocks < 16) return false;
-  uint32_t s_want = units / tail;
-  if (s_want > dvm::mm::MAX_SPLIT) s_want = dvm::mm::MAX_SPLIT;
-  const uint32_t per = (kblocks + s_want - 1) / s_want;
-  const uint32_t s_eff = (kblocks + per - 1) / per;
-  if (s_eff < 2 || (size_t)tail * (s_eff - 1) * nr > SPLIT_WS_PARTS || (4 * (size_t)tail + 4) * nr > SPLIT_FLAG_WORDS) return false;
-  sp->first = tiles - tail; sp->r = tail; sp->s = s_eff; sp->kb = per;
+  if (!g_tail_split || !tail || kblocks < 16) return false;
+  sp->first = tiles - tail;
+  sp->r = tail;
+  double best = 0.0;  // microseconds gained
+  if (2 * tail <= units) {  // every tile gets s units of its own, aligned parts: the best s
+    uint32_t s_max = units / tail;
+    if (s_max > dvm::mm::MAX_SPLIT) s_max = dvm::mm::MAX_SPLIT;
+    for (uint32_t s_want = s_max; s_want >= 2; --s_want) {
+      const uint32_t per = (kblocks + s_want - 1) / s_want;
+      const uint32_t s_eff = (kblocks + per - 1) / per;
+      if (s_eff < 2) continue;
+      const double cost = kExchangeUs + kUsPerPart * tail * (s_eff - 1) * nr;
+      const double gain = (kblocks - per) * kUsPerKBlock - cost;
+      if (gain > best) {
+        best = gain;
+        sp->s = s_eff; sp->kb = per; sp->kbp = s_eff * per; sp->units_used = tail * s_eff;
+        sp->cost_blocks = per + cost / kUsPerKBlock;
+      }
+    }
+  } else {  // equal ranges of the tail's k line over all units: every unit dumps a part and owns a tile
+    const uint32_t W = (uint32_t)(((uint64_t)tail * kblocks + units - 1) / units);
+    uint32_t smax = 1, n_parts = 0;
+    for (uint32_t a = 0; a < tail && W < kblocks; ++a) {
+      const uint32_t parts = (a * kblocks + kblocks - 1) / W - (a * kblocks) / W + 1;
+      if (parts > smax) smax = parts;
+      n_parts += parts - 1;
+    }
+    const double cost = kExchangeUs + kUsPerPart * n_parts * nr;
+    const double gain = W < kblocks ? (kblocks - W) * kUsPerKBlock - cost : 0.0;
+    if (smax >= 2 && smax <= dvm::mm::MAX_SPLIT && gain > best) {
+      best = gain;
+      sp->s = smax; sp->kb = W; sp->kbp = kblocks; sp->units_used = (uint32_t)(((uint64_t)tail * kblocks + W - 1) / W);
+      sp->cost_blocks = W + cost / kUsPerKBlock;
+    }
+  }
+  if (best <= 0.0) return false;
+  if ((size_t)tail * (sp->s - 1) * nr > SPLIT_WS_PARTS || (4 * (size_t)tail + 4) * nr > SPLIT_FLAG_WORDS) return false;
   return true;
 }
-// Estimated time of such a launch in tile times: the full waves, plus a last wave that costs a whole tile time,
-// or with the tail split 1 / s of it and the exchange of the parts (about 8 us, a tile time being about 0.47 us
-// per k block).
+// Estimated time of such a launch in tile times: the full waves, plus a last wave that costs a whole tile time, or
+// with the tail split its longest share and the exchange.
 double mm_waves(uint32_t tiles, uint32_t units, uint32_t kblocks, uint32_t nr) {
   double w = (double)(tiles / units);
   if (tiles % units) {
     SplitPlan sp;
-    w += mm_plan_split(tiles, units, kblocks, nr, &sp) ? 1.0 / sp.s + 17.0 / kblocks : 1.0;
+    w += mm_plan_split(tiles, units, kblocks, nr, &sp) ? sp.cost_blocks / kblocks : 1.0;
   }
   return w;
 }
@@ -1382,7 +1433,7 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   // CTA pairs (see dvm_mm_kernel): tiles of 256 rows
   const uint32_t mblocks = x[DVM_MM_MBLOCKS], nblocks = x[DVM_MM_NBLOCKS];
   if (g_cta_pairs && pair_clusters > 0 && mblocks >= 2 && mm_prefers_pairs(mblocks, nblocks, x[DVM_MM_KBLOCKS], (uint32_t)dev.sm_count, (uint32_t)pair_clusters)) {
-    P.split_s = P.split_r = P.split_first = P.split_kb = 0;
+    P.split_s = P.split_r = P.split_first = P.split_kb = P.split_kbp = 0;
     P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
     P.n_stages = dvm::mm::STAGES_PAIR;
     P.pair_mblocks = (mblocks + 1) / 2;
@@ -1391,11 +1442,11 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
     SplitPlan plan;
     if (mm_plan_split(P.pair_tiles, (uint32_t)pair_clusters, x[DVM_MM_KBLOCKS], 2, &plan)) {
       if (SplitSpace* sp = split_space(devid, stream)) {
-        P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb;
+        P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb; P.split_kbp = plan.kbp;
         P.ws = sp->ws; P.flags = sp->flags;
         if (++sp->epoch == 0) sp->epoch = 1;
         P.epoch = sp->epoch;
-        if (P.pair_tiles < (uint32_t)pair_clusters) pairs = plan.r * plan.s;
+        if (P.pair_tiles < (uint32_t)pair_clusters) pairs = plan.units_used;
       }
     }
     cudaLaunchConfig_t cfg = {};
@@ -1411,17 +1462,17 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   int grid = (int)(tiles < (uint32_t)dev.sm_count ? tiles : (uint32_t)dev.sm_count);
   // Tail split: the last wave of r <= sms / 2 tiles would leave most SMs idle for a whole tile time; instead
   // s = min(4, sms / r) CTAs take each of its tiles, a share of the k blocks each (see MMParams).
-  P.split_s = P.split_r = P.split_first = P.split_kb = 0;
+  P.split_s = P.split_r = P.split_first = P.split_kb = P.split_kbp = 0;
   P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
   const uint32_t sms = (uint32_t)dev.sm_count;
   SplitPlan plan;
   if (mm_plan_split(tiles, sms, x[DVM_MM_KBLOCKS], 1, &plan)) {
     if (SplitSpace* sp = split_space(devid, stream)) {
-      P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb;
+      P.split_first = plan.first; P.split_r = plan.r; P.split_s = plan.s; P.split_kb = plan.kb; P.split_kbp = plan.kbp;
       P.ws = sp->ws; P.flags = sp->flags;
       if (++sp->epoch == 0) sp->epoch = 1;
       P.epoch = sp->epoch;
-      if (tiles < sms) grid = (int)(plan.r * plan.s);
+      if (tiles < sms) grid = (int)plan.units_used;
     }
   }
   dvm::mm::dvm_mm_kernel<false><<<grid, dvm::mm::THREADS, smem, stream>>>(ma, mb0, mb1, P);

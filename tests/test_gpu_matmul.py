@@ -336,3 +336,32 @@ def test_matmul_launch_inside_a_cuda_graph():
             assert dvm.last_device_status() == 0
             want = oracle_run(prog, [dev[0].cpu(), ins[1], ins[2]])
             check(prog, [out], want)
+
+
+@pytest.mark.parametrize("pairs,kind,M,K,N", [
+    (0, "addmm", 128, 16384, 20480),   # one wave of 80 tiles on 148 CTAs: ranges of 139 of the 256 k blocks, tiles in two or three parts
+    (0, "addmm", 1024, 16384, 7424),   # 232 tiles: a full wave, then 84 tiles in ranges of 146 k blocks
+    (2, "addmm", 256, 16384, 10240),   # 40 tiles of 256 rows on 74 pairs: ranges of 139 k blocks
+    (2, "mlp", 512, 16384, 2560),      # both products: 40 tiles of 256 rows, 20 column blocks
+])
+def test_tail_split_of_a_large_last_wave(pairs, kind, M, K, N):
+    """A last wave above half of the units is cut into equal ranges of its k blocks: a unit ends one tile and starts
+    the next."""
+    prog, ins = _tail_case(kind, M, K, N, seed=M + N + pairs)
+    try:
+        dvm.set_matmul_cta_pairs(pairs)
+        outs, _ = gpu_run(prog, ins)
+        again, _ = gpu_run(prog, ins)
+        dvm.set_matmul_tail_split(False)
+        plain, _ = gpu_run(prog, ins)
+    finally:
+        dvm.set_matmul_tail_split(True)
+        dvm.set_matmul_cta_pairs(1)
+    want = oracle_run(prog, ins)
+    check(prog, outs, want)
+    check(prog, plain, want)
+    assert not torch.isnan(outs[0].float()).any()
+    assert torch.equal(outs[0], again[0])
+    a, b = outs[0].float(), plain[0].float()
+    assert (a - b).abs().max().item() <= 2.0 ** -7 * b.abs().max().item()
+    assert (a != b).any().item()   # (the launch did split: some sums rounded differently)
