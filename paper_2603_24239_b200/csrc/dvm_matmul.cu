@@ -1435,7 +1435,9 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
   if (g_cta_pairs && pair_clusters > 0 && mblocks >= 2 && mm_prefers_pairs(mblocks, nblocks, x[DVM_MM_KBLOCKS], (uint32_t)dev.sm_count, (uint32_t)pair_clusters)) {
     P.split_s = P.split_r = P.split_first = P.split_kb = P.split_kbp = 0;
     P.ws = nullptr; P.flags = nullptr; P.epoch = 0;
-    P.n_stages = dvm::mm::STAGES_PAIR;
+    // (an epilogue without temporaries leaves room for a seventh stage)
+    P.n_stages = v.ntmp == 0 ? dvm::mm::STAGES_PAIR + 1 : dvm::mm::STAGES_PAIR;
+    const size_t smem_pair = 1024 + (size_t)P.n_stages * dvm::mm::STAGE_PAIR + (size_t)v.ntmp * dvm::mm::TMP_BYTES + dvm::mm::BAR_BYTES;
     P.pair_mblocks = (mblocks + 1) / 2;
     P.pair_tiles = P.pair_mblocks * nblocks;
     uint32_t pairs = P.pair_tiles < (uint32_t)pair_clusters ? P.pair_tiles : (uint32_t)pair_clusters;
@@ -1454,7 +1456,7 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(dvm::mm::THREADS);
-    cfg.dynamicSmemBytes = smem; cfg.stream = stream; cfg.attrs = at; cfg.numAttrs = 1;
+    cfg.dynamicSmemBytes = smem_pair; cfg.stream = stream; cfg.attrs = at; cfg.numAttrs = 1;
     DVM_CUDA(cudaLaunchKernelEx(&cfg, dvm::mm::dvm_mm_kernel<true>, ma, mb0, mb1, P));
     dvm_count_launch();
     return DVM_OK;
