@@ -235,6 +235,14 @@ void dvm_set_lean_kernel(int on);
  * partial sums.  on = 0 switches the split off.  Default 1. */
 void dvm_set_matmul_tail_split(int on);
 
+/* The tail split a matmul launch of `tiles` output tiles with `k_blocks` blocks of 64 along k would use on `units`
+ * CTAs (ctas_per_unit = 1) or CTA pairs (2).  Returns 0 when such a launch does not split, 1 when it does, and then
+ * out = { first tile of the last wave, its tiles r, most parts of a tile, k blocks per unit W, pitch P of the tiles
+ * on the line of k blocks, units that take part }: tile a of the wave lies at blocks [a P, a P + k_blocks) of the
+ * line, unit c takes [c W, (c + 1) W), the unit holding a tile's first block owns it.  Host only (the arithmetic
+ * of dvm_launch, for tests and tools). */
+int dvm_matmul_tail_plan(int64_t tiles, int units, int k_blocks, int ctas_per_unit, int32_t out[6]);
+
 /* Matmul launches on CTA pairs: two CTAs of a cluster compute a tile of 256 output rows with one tcgen05
  * cta_group::2 instruction stream, each loading its own rows of A and half of the B tile (a third less
  * shared-memory traffic per flop).  mode = 0: never; 1 (default): where the launch's shape favours it; 2: wherever

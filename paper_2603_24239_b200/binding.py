@@ -86,6 +86,7 @@ _sig = {
     "dvm_set_stacked_one_slot": ([_i], None),
     "dvm_set_matmul_tail_split": ([_i], None),
     "dvm_set_matmul_cta_pairs": ([_i], None),
+    "dvm_matmul_tail_plan": ([C.c_int64, _i, _i, _i, C.POINTER(C.c_int32)], _i),
     "dvm_hardware_align_div": ([C.c_int64, _i, C.c_int64, C.c_int64, C.c_int64, _p64, _p64, _p64, _p64], _i),
     "dvm_vm_tile_range": ([C.c_int64, _i, _i, _p64, _p64], _i),
     "dvm_launch": ([_vp, _sz, C.POINTER(_vp), _i, _vp], _i),
@@ -626,6 +627,17 @@ def set_lean_kernel(on: bool):
 def set_matmul_tail_split(on: bool):
     """dvm_set_matmul_tail_split: split the tiles of a matmul launch's last, partial wave along k (default on)."""
     lib.dvm_set_matmul_tail_split(int(bool(on)))
+
+
+def matmul_tail_plan(tiles: int, units: int, k_blocks: int, ctas_per_unit: int = 1):
+    """dvm_matmul_tail_plan: None when such a launch does not split its last wave, else a dict of the plan."""
+    out = (C.c_int32 * 6)()
+    st = lib.dvm_matmul_tail_plan(tiles, units, k_blocks, ctas_per_unit, out)
+    if st < 0:
+        _check(st, "dvm_matmul_tail_plan")
+    if st == 0:
+        return None
+    return {"first": out[0], "r": out[1], "parts_max": out[2], "kb_per_unit": out[3], "tile_pitch": out[4], "units_used": out[5]}
 
 
 def set_matmul_cta_pairs(mode: int):

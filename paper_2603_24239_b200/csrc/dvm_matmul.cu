@@ -1484,6 +1484,16 @@ int dvm_launch_matmul(const uint32_t* code, size_t n_words, void* const* tensors
 }
 
 extern "C" void dvm_set_matmul_tail_split(int on) { g_tail_split = on; }
+
+extern "C" int dvm_matmul_tail_plan(int64_t tiles, int units, int k_blocks, int ctas_per_unit, int32_t out[6]) {
+  if (!out || tiles < 0 || tiles >= (1ll << 31) || units < 1 || k_blocks < 1 || ctas_per_unit < 1 || ctas_per_unit > 2)
+    return DVM_ERR_INVALID_ARG;
+  SplitPlan sp = {};
+  if (!mm_plan_split((uint32_t)tiles, (uint32_t)units, (uint32_t)k_blocks, (uint32_t)ctas_per_unit, &sp)) return 0;
+  out[0] = (int32_t)sp.first; out[1] = (int32_t)sp.r; out[2] = (int32_t)sp.s;
+  out[3] = (int32_t)sp.kb; out[4] = (int32_t)sp.kbp; out[5] = (int32_t)sp.units_used;
+  return 1;
+}
 extern "C" void dvm_set_matmul_cta_pairs(int mode) { g_cta_pairs = mode; }
 
 // ---- self-test of the matmul kernel's bounded wait (see dvm_selftest_bounded_wait) ----
