@@ -1129,7 +1129,9 @@ def whole_job_value(work_per_rank: float, world: int, ms_per_step: float, scale:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed passes over the sweep (default 5; 100 for the matmul workloads, about two seconds: their "
+                         "roofline is the SUSTAINED cuBLAS rate under the power cap, which a 0.1 s run does not meet)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="dvm", choices=["dvm", "reference"])
@@ -1148,6 +1150,8 @@ def main():
     ap.add_argument("--detail", default="", help="write per-instance timings to this JSON file")
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.steps is None:
+            args.steps = 5
         return run_reference(args)
 
     rank = int(os.environ.get("RANK", "0"))
@@ -1178,6 +1182,8 @@ def main():
     if args.max_rows and args.workload in ("c2", "c5", "addmm"):
         kw["max_rows"] = args.max_rows
     W = WORKLOADS[args.workload](dvm, **kw)
+    if args.steps is None:
+        args.steps = 100 if W.bound == "tensor" else 5
     stream = torch.cuda.current_stream()
     peaks, peak_kind = measured_peaks()
 
@@ -1326,7 +1332,7 @@ def main():
         torch.cuda.empty_cache()
         cfgs = {}
         # (the tensor-core sweeps first, while the GPU is coolest; c4 last: it changes the encoder's knobs)
-        for name, steps in (("c5", 2), ("addmm", 2), ("ifelse", 2), ("views", 2), ("c1", 50), ("c3", 2), ("c4", 2)):
+        for name, steps in (("c5", 40), ("addmm", 40), ("ifelse", 2), ("views", 2), ("c1", 50), ("c3", 2), ("c4", 2)):
             if name == name_main:
                 continue
             try:
