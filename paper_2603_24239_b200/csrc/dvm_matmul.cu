@@ -18,8 +18,8 @@
 //               next tile's MMAs (the other accumulator stage).
 // Two forms, chosen per launch (dvm_launch_matmul): single CTAs as above, or CTA pairs -- two CTAs of a cluster on
 // a tile of 256 rows with tcgen05 cta_group::2, each loading its own A rows and half of the B tile (see
-// dvm_mm_kernel).  In both, a last wave of tiles that would fill at most half of the device is split along k
-// among several CTAs (pairs) per tile (see MMParams).
+// dvm_mm_kernel).  In both, the tiles of a last, partial wave are shared along k among the CTAs (pairs) where
+// that saves more than the exchange of the partial sums costs (see MMParams, mm_plan_split).
 // Every wait on an mbarrier is bounded (time and iteration limit): when one runs out the CTA raises its
 // abort flag, every role leaves its loop, copies and MMAs in flight are awaited (bounded again), tensor
 // memory is released and the status word reports DVM_ERR_DEVICE_TIMEOUT.
@@ -516,7 +516,7 @@ constexpr int ACC_COLS = 256;                       // accumulator columns of on
 constexpr uint32_t STAGE_A = BLOCK_M * BLOCK_K * 2; // 16 KB: 128 rows of 128 bytes
 constexpr uint32_t BOX_B = 64 * BLOCK_K * 2;        // 8 KB: 64 k-rows of 64 columns
 constexpr uint32_t STAGE_BYTES = STAGE_A + 4 * BOX_B;  // 48 KB
-constexpr int MAX_STAGES = 8;                       // barrier slots; 4 stages of 48 KB, or 6 of 32 KB for a CTA pair
+constexpr int MAX_STAGES = 8;                       // barrier slots; 4 stages of 48 KB, or 6 to 7 of 32 KB for a CTA pair
 constexpr uint32_t STAGE_PAIR = STAGE_A + 2 * BOX_B;  // 32 KB: this CTA's A rows and its half of the B tile
 constexpr uint32_t STAGES_SINGLE = 4, STAGES_PAIR = 6;
 constexpr uint32_t BAR_BYTES = 256;                  // barriers and flags behind the epilogue temporaries
@@ -550,7 +550,7 @@ struct MMParams {
   uint32_t n_stages;
   uint32_t words[DVM_MM_MAX_WORDS];
 };
-constexpr uint32_t MAX_SPLIT = 4;                    // CTAs per tail tile at most
+constexpr uint32_t MAX_SPLIT = 4;                    // parts of a tail tile at most
 constexpr size_t PART_FLOATS = (size_t)BLOCK_M * ACC_COLS;  // one partial accumulator: 128 KB
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
