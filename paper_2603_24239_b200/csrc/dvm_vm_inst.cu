@@ -5,13 +5,14 @@
 // large, each one-program / stacked, with and without the heavy unary functions; group 17: the lean kernel with
 // 24 elements per thread (one program); group 18: the lean kernel for phased programs; groups 19..30: the level-wait
 // variant of groups 0..11 compiled for three resident CTAs per SM; group 31: the one-program lean kernel, 16 elements
-// per thread, compiled for three.
+// per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
+// for launches with two tile slots (its one-slot path compiled out).
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..31>"
+#error "compile with -DDVM_INST_GROUP=<0..34>"
 #endif
 
 namespace {
@@ -32,18 +33,18 @@ struct Ops {
   }
 };
 
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS>
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>,
                                                          dvm::THREADS, smem);
   }
 };
@@ -52,6 +53,12 @@ struct LeanOps {
   {V, LARGE, 1, 0, 0, 2, HEAVY, 2,                                                        \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, true>::occupancy}
+
+// the one-program lean kernel for launches with two tile slots (lean = 3: its one-slot path compiled out)
+#define DVM_LEAN_TWO(V, LARGE, HEAVY)                                                               \
+  {V, LARGE, 1, 0, 0, 3, HEAVY, 2,                                                                  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
@@ -87,6 +94,9 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 32
+constexpr int GV = DVM_INST_GROUP == 32 ? 16 : (DVM_INST_GROUP == 33 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO(GV, 0, 0), DVM_LEAN_TWO(GV, 0, 1), DVM_LEAN_TWO(GV, 1, 0), DVM_LEAN_TWO(GV, 1, 1)};
 #elif DVM_INST_GROUP == 12
 const DvmVmVariant kGroup[] = {DVM_ENTRY(24, 0, 1, 0, 0), DVM_ENTRY(24, 1, 1, 0, 0)};
 #elif DVM_INST_GROUP < 17
