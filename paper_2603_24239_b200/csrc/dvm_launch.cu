@@ -63,7 +63,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -87,8 +87,8 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
 // Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
 uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
   const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
-                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 15) |  // (lean: two bits)
-                      ((uint64_t)v->ctas << 16);
+                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 16) |  // (lean: three bits)
+                      ((uint64_t)v->ctas << 17);
   return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
 }
 
@@ -697,7 +697,10 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
   }
   if (lean == 1 && single && !one_slot && variant) {
     // one program with two tile slots: the build without the one-slot path
-    const DvmVmVariant* v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);
+    const uint32_t* c0 = (const uint32_t*)codes[0];
+    const bool dense = !((c0[DVM_H_GEOM] >> 24) & (DVM_F_LOADS_BY_ROW | DVM_F_OUTER_DIMS)) && ((c0[DVM_H_LOCAL] >> 16) & 0xff) == 0;
+    const DvmVmVariant* v2 = dense ? dvm_vm_find_variant(V, large, true, 0, false, 4, heavy) : nullptr;
+    if (!v2) v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);
     if (v2) variant = v2;
   }
   if (!variant) return DVM_ERR_UNSUPPORTED;  // (24 elements per thread: encoded for a launch of its own on the basic variant)

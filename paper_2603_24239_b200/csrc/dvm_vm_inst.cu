@@ -6,13 +6,14 @@
 // 24 elements per thread (one program); group 18: the lean kernel for phased programs; groups 19..30: the level-wait
 // variant of groups 0..11 compiled for three resident CTAs per SM; group 31: the one-program lean kernel, 16 elements
 // per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
-// for launches with two tile slots (its one-slot path compiled out).
+// for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
+// loads are all one thread's.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..34>"
+#error "compile with -DDVM_INST_GROUP=<0..37>"
 #endif
 
 namespace {
@@ -33,18 +34,18 @@ struct Ops {
   }
 };
 
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false>
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>,
                                                          dvm::THREADS, smem);
   }
 };
@@ -59,6 +60,12 @@ struct LeanOps {
   {V, LARGE, 1, 0, 0, 3, HEAVY, 2,                                                                  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true>::occupancy}
+
+// ... and for programs whose loads are all one thread's (lean = 4: also without row-by-row copies, per-row scalar inputs, outer dims)
+#define DVM_LEAN_TWO_DENSE(V, LARGE, HEAVY)                                                               \
+  {V, LARGE, 1, 0, 0, 4, HEAVY, 2,                                                                        \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
@@ -94,6 +101,9 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 35
+constexpr int GV = DVM_INST_GROUP == 35 ? 16 : (DVM_INST_GROUP == 36 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE(GV, 0, 0), DVM_LEAN_TWO_DENSE(GV, 0, 1), DVM_LEAN_TWO_DENSE(GV, 1, 0), DVM_LEAN_TWO_DENSE(GV, 1, 1)};
 #elif DVM_INST_GROUP >= 32
 constexpr int GV = DVM_INST_GROUP == 32 ? 16 : (DVM_INST_GROUP == 33 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO(GV, 0, 0), DVM_LEAN_TWO(GV, 0, 1), DVM_LEAN_TWO(GV, 1, 0), DVM_LEAN_TWO(GV, 1, 1)};

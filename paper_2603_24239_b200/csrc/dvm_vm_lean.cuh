@@ -160,7 +160,10 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
 // CTAS: resident CTAs per SM the kernel is compiled for (2; 3 for one-slot programs, see dvm_vm_kernel).
 // TWO: the build for launches that are known to run with two tile slots: the one-slot path is compiled out (the
 // tile loop is short enough that every branch in it shows: +1.6 % on C2).
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false>
+// DENSE: the build for programs whose loads are all one thread's (dense tiles and row vectors: no row-by-row copies, no
+// per-row scalar inputs, no outer dims to decompose): those paths are compiled out of the load issue and of the
+// operand addressing (+5 % on C2).
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false>
 __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
@@ -226,7 +229,7 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
     Coord c;
     c.i0 = row;
     c.i1 = c.i2 = 0;
-    if ((CW(prog + DVM_H_GEOM) >> 24) & DVM_F_OUTER_DIMS) {
+    if (!DENSE && ((CW(prog + DVM_H_GEOM) >> 24) & DVM_F_OUTER_DIMS)) {
       // row -> coordinates over the outer dims: two divisions by multiply-and-shift (the linker left the
       // multipliers where the kernel type, code size, tile count and total words were)
       const uint32_t n0 = CW(prog + DVM_H_OUTER0), n1 = CW(prog + DVM_H_OUTER1);
@@ -266,8 +269,8 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
     const uint32_t geom = CW(prog + DVM_H_GEOM);
     const int lgG = geom & 0xff;
     const int t = tid & ((1 << lgG) - 1);
-    const bool by_row = ((geom >> 24) & DVM_F_LOADS_BY_ROW) != 0;
-    const bool scalars = ((CW(prog + DVM_H_LOCAL) >> 16) & 0xff) != 0;
+    const bool by_row = DENSE ? false : ((geom >> 24) & DVM_F_LOADS_BY_ROW) != 0;
+    const bool scalars = DENSE ? false : ((CW(prog + DVM_H_LOCAL) >> 16) & 0xff) != 0;
     const uint32_t load_words = CW(prog + DVM_H_LOAD_WORDS);
     // A program whose copies are all thread 0's (dense tiles, row vectors): the lanes of warp 0 take one load
     // instruction each, as thread 0 would -- the warp walks the load section once, not once per instruction.
@@ -297,7 +300,7 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
               a = (unsigned long long)r.row * C;
               n_el = (unsigned long long)(rv - 1) * C + last;
             }
-          } else if (mode == DVM_LM_ROWS) {
+          } else if (!DENSE && mode == DVM_LM_ROWS) {
             if (t == 0 && r.ncols > 0) {
               mine = true;
               a = row_offset(prog, d, r);
@@ -473,7 +476,7 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
       uint32_t a = sb + (ow & 0x3ffffu);
       if (mode == DVM_LM_BLOCK) return a + (img << lg_es) + ((base_lo + (row0C << lg_es)) & 15u);
       uint32_t off;
-      if (mode == DVM_LM_ROWS) {
+      if (!DENSE && mode == DVM_LM_ROWS) {
         off = row_offset32(prog, opd_base(prog) + (ow >> 26) * DVM_OPD_WORDS, r);
         a += rr * (((uint32_t)V << (lgG + lg_es)) + 32u);
       } else {
