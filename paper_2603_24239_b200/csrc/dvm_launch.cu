@@ -63,7 +63,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -592,6 +592,33 @@ int place_all(dvm::VMParams<PW_LARGE>& P, int n_programs, const void* const* cod
   return DVM_OK;
 }
 
+// Whether every input of a program whose loads are all one thread's is aligned like the tile's chunks: the tensor
+// on a 16-byte boundary, its rows (and column blocks) a whole number of 16-byte units, a chunk of it 16 bytes or
+// more.  Then no read of an image needs realigning (the lean interpreter has a build without that code).
+bool program_all_aligned(const uint32_t* c, void* const* tensors) {
+  const uint32_t geom = c[DVM_H_GEOM];
+  if (!((geom >> 24) & DVM_F_ALIGNED)) return false;
+  const uint32_t counts = c[DVM_H_COUNTS], nt = counts & 0xff, n_opd = (counts >> 16) & 0xff;
+  const uint32_t* ot = c + DVM_HDR_WORDS + 2 * nt;
+  const uint32_t* lt = ot + n_opd * DVM_OPD_WORDS;
+  const uint32_t n_inr = c[DVM_H_LOCAL] & 0xff, W = (geom >> 8) & 0xff;
+  const uint64_t C = c[DVM_H_COLS], ctile = c[DVM_H_COL_TILE], cb = c[DVM_H_COL_BLOCKS];
+  for (uint32_t k = 0; k < n_inr; ++k) {
+    const uint32_t mode = (lt[k] >> 16) & 0xf, info = ot[(lt[k] >> 24) * DVM_OPD_WORDS];
+    const uint32_t dt = (info >> 8) & 0xff;
+    const uint64_t es = (uint64_t)1 << DVM_DT_LG_ES(dt);
+    if (((uintptr_t)tensors[info & 0xff]) & 15) return false;
+    if (W * es < 16) return false;  // (a chunk of 4 bf16 elements is 8 bytes)
+    if (cb > 1 && (ctile * es) % 16) return false;
+    if (mode == DVM_LM_BLOCK) {
+      if ((C * es) % 16) return false;
+    } else if (mode != DVM_LM_BCAST && mode != DVM_LM_BCAST_TILE) {
+      return false;
+    }
+  }
+  return true;
+}
+
 // `level` (may be NULL): level[i] of program i, non-decreasing; a program reads what programs of lower levels store.
 // `tile_begin`, `tile_end` (one-program launches without a queue; 0, 0 = all): the range of tiles to run.
 int launch_vec(int n_programs, const void* const* codes, void* const* const* tensors, const int* n_tensors,
@@ -699,7 +726,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     // one program with two tile slots: the build without the one-slot path
     const uint32_t* c0 = (const uint32_t*)codes[0];
     const bool dense = !((c0[DVM_H_GEOM] >> 24) & (DVM_F_LOADS_BY_ROW | DVM_F_OUTER_DIMS)) && ((c0[DVM_H_LOCAL] >> 16) & 0xff) == 0;
-    const DvmVmVariant* v2 = dense ? dvm_vm_find_variant(V, large, true, 0, false, 4, heavy) : nullptr;
+    const DvmVmVariant* v2 = (dense && program_all_aligned(c0, tensors[0])) ? dvm_vm_find_variant(V, large, true, 0, false, 5, heavy) : nullptr;
+    if (!v2 && dense) v2 = dvm_vm_find_variant(V, large, true, 0, false, 4, heavy);
     if (!v2) v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);
     if (v2) variant = v2;
   }

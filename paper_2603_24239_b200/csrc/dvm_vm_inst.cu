@@ -7,13 +7,13 @@
 // variant of groups 0..11 compiled for three resident CTAs per SM; group 31: the one-program lean kernel, 16 elements
 // per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
 // for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
-// loads are all one thread's.
+// loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..37>"
+#error "compile with -DDVM_INST_GROUP=<0..40>"
 #endif
 
 namespace {
@@ -34,18 +34,19 @@ struct Ops {
   }
 };
 
-template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false>
+template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false,
+          bool AL = false>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>,
                                                          dvm::THREADS, smem);
   }
 };
@@ -66,6 +67,12 @@ struct LeanOps {
   {V, LARGE, 1, 0, 0, 4, HEAVY, 2,                                                                        \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true>::occupancy}
+
+// ... all of whose operands are aligned like the tile's chunks (lean = 5: also without the realignment of reads)
+#define DVM_LEAN_TWO_DENSE_AL(V, LARGE, HEAVY)                                                                  \
+  {V, LARGE, 1, 0, 0, 5, HEAVY, 2,                                                                              \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
@@ -101,6 +108,9 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 38
+constexpr int GV = DVM_INST_GROUP == 38 ? 16 : (DVM_INST_GROUP == 39 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE_AL(GV, 0, 0), DVM_LEAN_TWO_DENSE_AL(GV, 0, 1), DVM_LEAN_TWO_DENSE_AL(GV, 1, 0), DVM_LEAN_TWO_DENSE_AL(GV, 1, 1)};
 #elif DVM_INST_GROUP >= 35
 constexpr int GV = DVM_INST_GROUP == 35 ? 16 : (DVM_INST_GROUP == 36 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE(GV, 0, 0), DVM_LEAN_TWO_DENSE(GV, 0, 1), DVM_LEAN_TWO_DENSE(GV, 1, 0), DVM_LEAN_TWO_DENSE(GV, 1, 1)};
