@@ -63,7 +63,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -592,9 +592,9 @@ int place_all(dvm::VMParams<PW_LARGE>& P, int n_programs, const void* const* cod
   return DVM_OK;
 }
 
-// Whether every input of a program whose loads are all one thread's is aligned like the tile's chunks: the tensor
-// on a 16-byte boundary, its rows (and column blocks) a whole number of 16-byte units, a chunk of it 16 bytes or
-// more.  Then no read of an image needs realigning (the lean interpreter has a build without that code).
+// Whether every input of a program is aligned like the tile's chunks: the tensor on a 16-byte boundary, its rows
+// (and column blocks; for a row-by-row copied input its outer strides) a whole number of 16-byte units, a chunk of
+// it 16 bytes or more.  Then no read of an image needs realigning (the lean interpreter has a build without that code).
 bool program_all_aligned(const uint32_t* c, void* const* tensors) {
   const uint32_t geom = c[DVM_H_GEOM];
   if (!((geom >> 24) & DVM_F_ALIGNED)) return false;
@@ -612,6 +612,10 @@ bool program_all_aligned(const uint32_t* c, void* const* tensors) {
     if (cb > 1 && (ctile * es) % 16) return false;
     if (mode == DVM_LM_BLOCK) {
       if ((C * es) % 16) return false;
+    } else if (mode == DVM_LM_ROWS) {  // a row copied on its own starts wherever the outer strides put it
+      const uint32_t* d = ot + (lt[k] >> 24) * DVM_OPD_WORDS;
+      for (int q = 0; q < 3; ++q)
+        if (((uint64_t)d[DVM_OPD_STRIDE0 + 2 * q] * es) % 16 || d[DVM_OPD_STRIDE0 + 2 * q + 1]) return false;
     } else if (mode != DVM_LM_BCAST && mode != DVM_LM_BCAST_TILE) {
       return false;
     }
@@ -726,7 +730,8 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     // one program with two tile slots: the build without the one-slot path
     const uint32_t* c0 = (const uint32_t*)codes[0];
     const bool dense = !((c0[DVM_H_GEOM] >> 24) & (DVM_F_LOADS_BY_ROW | DVM_F_OUTER_DIMS)) && ((c0[DVM_H_LOCAL] >> 16) & 0xff) == 0;
-    const DvmVmVariant* v2 = (dense && program_all_aligned(c0, tensors[0])) ? dvm_vm_find_variant(V, large, true, 0, false, 5, heavy) : nullptr;
+    const bool aligned = program_all_aligned(c0, tensors[0]);
+    const DvmVmVariant* v2 = aligned ? dvm_vm_find_variant(V, large, true, 0, false, dense ? 5 : 6, heavy) : nullptr;
     if (!v2 && dense) v2 = dvm_vm_find_variant(V, large, true, 0, false, 4, heavy);
     if (!v2) v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);
     if (v2) variant = v2;

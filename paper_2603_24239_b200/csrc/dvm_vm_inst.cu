@@ -7,13 +7,14 @@
 // variant of groups 0..11 compiled for three resident CTAs per SM; group 31: the one-program lean kernel, 16 elements
 // per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
 // for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
-// loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks.
+// loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks; groups 41..43: two slots, aligned rows,
+// row-by-row copies allowed.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..40>"
+#error "compile with -DDVM_INST_GROUP=<0..43>"
 #endif
 
 namespace {
@@ -74,6 +75,12 @@ struct LeanOps {
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true>::occupancy}
 
+// ... for programs with row-by-row copies whose rows are all aligned like the tile's chunks (lean = 6)
+#define DVM_LEAN_TWO_AL(V, LARGE, HEAVY)                                                                         \
+  {V, LARGE, 1, 0, 0, 6, HEAVY, 2,                                                                               \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true>::occupancy}
+
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::launch, \
@@ -108,6 +115,9 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 41
+constexpr int GV = DVM_INST_GROUP == 41 ? 16 : (DVM_INST_GROUP == 42 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_AL(GV, 0, 0), DVM_LEAN_TWO_AL(GV, 0, 1), DVM_LEAN_TWO_AL(GV, 1, 0), DVM_LEAN_TWO_AL(GV, 1, 1)};
 #elif DVM_INST_GROUP >= 38
 constexpr int GV = DVM_INST_GROUP == 38 ? 16 : (DVM_INST_GROUP == 39 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE_AL(GV, 0, 0), DVM_LEAN_TWO_DENSE_AL(GV, 0, 1), DVM_LEAN_TWO_DENSE_AL(GV, 1, 0), DVM_LEAN_TWO_DENSE_AL(GV, 1, 1)};
