@@ -226,6 +226,15 @@ int dvm_get_min_resident_ctas(void);
  * Default 1.  Both interpreters run the same bytecode and give results inside the same tolerances. */
 void dvm_set_lean_kernel(int on);
 
+/* Which build of the interpreter the calling thread's last vector launch ran on (for tests and tools): out =
+ * { elements per thread, 1 for the 32 KB parameter block, 1 for one program per launch, extension level, 1 with
+ *   level waits, lean, 1 with the heavy unary functions, resident CTAs per SM it is compiled for }.  lean: 0 the
+ * general interpreter; 1 the lean one with every path; 2 its build for phased programs; 3 for two tile slots;
+ * 4 ... and dense loads (no row-by-row copies, per-row scalar inputs, outer dims); 5 ... and aligned operands (no
+ * realignment of reads); 6 two slots and aligned operands with row-by-row copies; 7 as 5 for rows that fill the
+ * tile's slots exactly (no slot masks).  DVM_ERR_INVALID_ARG before the thread's first launch. */
+int dvm_last_launch_variant(int out[8]);
+
 /* Matmul launches (Sec. 4.2, matrix operations): the tiles of a last, partial wave are shared along k -- a small
  * wave gives each tile up to four CTAs (or CTA pairs), a larger one is cut into equal ranges of its k blocks over
  * all of them -- whenever the k blocks saved outweigh the exchange (decided per launch from its shape).  The

@@ -11,7 +11,7 @@ import importlib
 _BINDING_NAMES = (
     "DvmError", "Program", "Code", "Encoder", "encode", "launch", "launch_stacked", "run_host", "verify",
     "disassemble", "code_info", "last_device_status", "launch_count", "hardware_align_div",
-    "vm_tile_range", "set_num_cores", "get_num_cores", "set_elems_per_thread", "set_min_resident_ctas", "set_stacked_one_slot", "set_matmul_tail_split", "set_matmul_cta_pairs", "matmul_tail_plan", "set_lean_kernel", "program_from_nodes",
+    "vm_tile_range", "set_num_cores", "get_num_cores", "set_elems_per_thread", "set_min_resident_ctas", "set_stacked_one_slot", "set_matmul_tail_split", "set_matmul_cta_pairs", "matmul_tail_plan", "last_launch_variant", "set_lean_kernel", "program_from_nodes",
     "BatchEncoder", "selftest_bounded_wait", "Fuser", "tensor_extents", "launch_checked",
     "lib", "LIB_PATH",
 )

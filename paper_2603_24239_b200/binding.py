@@ -83,6 +83,7 @@ _sig = {
     "dvm_set_min_resident_ctas": ([_i], None),
     "dvm_get_min_resident_ctas": ([], _i),
     "dvm_set_lean_kernel": ([_i], None),
+    "dvm_last_launch_variant": ([C.POINTER(C.c_int)], _i),
     "dvm_set_stacked_one_slot": ([_i], None),
     "dvm_set_matmul_tail_split": ([_i], None),
     "dvm_set_matmul_cta_pairs": ([_i], None),
@@ -638,6 +639,13 @@ def matmul_tail_plan(tiles: int, units: int, k_blocks: int, ctas_per_unit: int =
     if st == 0:
         return None
     return {"first": out[0], "r": out[1], "parts_max": out[2], "kb_per_unit": out[3], "tile_pitch": out[4], "units_used": out[5]}
+
+
+def last_launch_variant() -> dict:
+    """dvm_last_launch_variant: the interpreter build the last vector launch of this thread ran on."""
+    out = (C.c_int * 8)()
+    _check(lib.dvm_last_launch_variant(out), "dvm_last_launch_variant")
+    return dict(zip(("V", "large", "single", "ext", "levels", "lean", "heavy", "ctas"), list(out)))
 
 
 def set_matmul_cta_pairs(mode: int):

@@ -39,6 +39,7 @@ DeviceState g_dev[MAX_DEVICES];
 std::mutex g_mu;
 thread_local int t_last_cuda_error = 0;
 long long g_launches = 0;
+thread_local const DvmVmVariant* t_last_variant = nullptr;  // dvm_last_launch_variant
 int g_use_lean = 1;  // dvm_set_lean_kernel(0): every launch runs on the general interpreter (for comparisons)
 
 }  // namespace
@@ -63,7 +64,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43) X(44) X(45) X(46)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -136,6 +137,15 @@ void dvm_note_cuda_error(int e) { t_last_cuda_error = e; }
 void dvm_count_launch() { __atomic_add_fetch(&g_launches, 1, __ATOMIC_RELAXED); }
 
 extern "C" void dvm_set_lean_kernel(int on) { g_use_lean = on; }
+
+extern "C" int dvm_last_launch_variant(int out[8]) {
+  if (!out) return DVM_ERR_INVALID_ARG;
+  const DvmVmVariant* v = t_last_variant;
+  if (!v) return DVM_ERR_INVALID_ARG;
+  out[0] = v->V; out[1] = v->large; out[2] = v->single; out[3] = v->ext;
+  out[4] = v->levels; out[5] = v->lean; out[6] = v->heavy; out[7] = v->ctas;
+  return DVM_OK;
+}
 static int g_stacked_one_slot = 0;
 extern "C" void dvm_set_stacked_one_slot(int on) { g_stacked_one_slot = on != 0; }
 extern "C" int dvm_last_cuda_error(void) { return t_last_cuda_error; }
@@ -438,6 +448,7 @@ int prefill_all(int n_programs, const void* const* codes, void* const* const* te
 
 // Starts one interpreter variant on `grid` CTAs.
 int launch_variant(const DvmVmVariant* v, const void* params, int grid, size_t smem, cudaStream_t stream) {
+  t_last_variant = v;
   DVM_CUDA(v->launch(params, grid, smem, stream));
   dvm_count_launch();
   return DVM_OK;
@@ -731,7 +742,11 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     const uint32_t* c0 = (const uint32_t*)codes[0];
     const bool dense = !((c0[DVM_H_GEOM] >> 24) & (DVM_F_LOADS_BY_ROW | DVM_F_OUTER_DIMS)) && ((c0[DVM_H_LOCAL] >> 16) & 0xff) == 0;
     const bool aligned = program_all_aligned(c0, tensors[0]);
-    const DvmVmVariant* v2 = aligned ? dvm_vm_find_variant(V, large, true, 0, false, dense ? 5 : 6, heavy) : nullptr;
+    // every row fills the slots of the threads that hold it: columns = threads per row x elements per thread
+    const bool full = c0[DVM_H_COL_BLOCKS] == 1 && c0[DVM_H_LAST_ROW_COLS] == c0[DVM_H_COLS] &&
+                      c0[DVM_H_COLS] == ((uint32_t)V << (c0[DVM_H_GEOM] & 0xff));
+    const DvmVmVariant* v2 = (aligned && dense && full) ? dvm_vm_find_variant(V, large, true, 0, false, 7, heavy) : nullptr;
+    if (!v2 && aligned) v2 = dvm_vm_find_variant(V, large, true, 0, false, dense ? 5 : 6, heavy);
     if (!v2 && dense) v2 = dvm_vm_find_variant(V, large, true, 0, false, 4, heavy);
     if (!v2) v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);
     if (v2) variant = v2;

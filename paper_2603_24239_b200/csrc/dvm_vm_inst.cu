@@ -8,13 +8,13 @@
 // per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
 // for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
 // loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks; groups 41..43: two slots, aligned rows,
-// row-by-row copies allowed.
+// row-by-row copies allowed; groups 44..46: groups 38..40 for programs whose rows fill the tile's slots exactly.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..43>"
+#error "compile with -DDVM_INST_GROUP=<0..46>"
 #endif
 
 namespace {
@@ -36,18 +36,18 @@ struct Ops {
 };
 
 template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false,
-          bool AL = false>
+          bool AL = false, bool FULL = false>
 struct LeanOps {
   static cudaError_t launch(const void* params, int grid, size_t smem, cudaStream_t stream) {
-    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>
+    dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL, FULL>
         <<<grid, dvm::THREADS, smem, stream>>>(*static_cast<const dvm::VMParams<PW>*>(params));
     return cudaGetLastError();
   }
   static cudaError_t occupancy(size_t smem, size_t max_smem, int* n) {
-    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>,
+    cudaError_t e = cudaFuncSetAttribute(dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL, FULL>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL>,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, dvm::dvm_vm_lean_kernel<V, PW, SINGLE, HEAVY, PHASED, CTAS, TWO, DENSE, AL, FULL>,
                                                          dvm::THREADS, smem);
   }
 };
@@ -80,6 +80,12 @@ struct LeanOps {
   {V, LARGE, 1, 0, 0, 6, HEAVY, 2,                                                                               \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true>::occupancy}
+
+// ... dense, aligned programs whose rows fill the tile's slots exactly (lean = 7: also without the slot masks)
+#define DVM_LEAN_TWO_DENSE_AL_FULL(V, LARGE, HEAVY)                                                                   \
+  {V, LARGE, 1, 0, 0, 7, HEAVY, 2,                                                                                    \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true, true>::occupancy}
 
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
@@ -115,6 +121,10 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 44
+constexpr int GV = DVM_INST_GROUP == 44 ? 16 : (DVM_INST_GROUP == 45 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE_AL_FULL(GV, 0, 0), DVM_LEAN_TWO_DENSE_AL_FULL(GV, 0, 1), DVM_LEAN_TWO_DENSE_AL_FULL(GV, 1, 0),
+                               DVM_LEAN_TWO_DENSE_AL_FULL(GV, 1, 1)};
 #elif DVM_INST_GROUP >= 41
 constexpr int GV = DVM_INST_GROUP == 41 ? 16 : (DVM_INST_GROUP == 42 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_AL(GV, 0, 0), DVM_LEAN_TWO_AL(GV, 0, 1), DVM_LEAN_TWO_AL(GV, 1, 0), DVM_LEAN_TWO_AL(GV, 1, 1)};

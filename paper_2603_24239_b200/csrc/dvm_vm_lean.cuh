@@ -170,8 +170,11 @@ __device__ __forceinline__ float2 lean_exp2_fast(float2 x, float nc) {
 // operand addressing (+5 % on C2).
 // AL: the build for programs all of whose operands are aligned like the tile's chunks (16-byte aligned tensors, rows a
 // whole number of 16-byte units): the realignment of reads and the row shift are compiled out (+3 % on C2).
+// FULL: the build for programs whose rows all fill the tile's slots exactly (columns = threads per row x elements per
+// thread, one column block, no shorter last row): a thread's slots are all valid or -- past the last row -- all
+// empty, so the slot masks, the sanitising of reductions and the element-wise store path are compiled out (+3 % on C2).
 template <int V, int PW, bool SINGLE, bool HEAVY, bool PHASED = false, int CTAS = DVM_LEAN_MIN_CTAS, bool TWO = false, bool DENSE = false,
-          bool AL = false>
+          bool AL = false, bool FULL = false>
 __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid_constant__ VMParams<PW> prm) {
   constexpr uint32_t kSingleProg = 3;  // directory of a one-program launch: [offset][0][n_tiles]
   constexpr int VP = V / 2;            // float2 pairs per tile register
@@ -452,7 +455,15 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
     const uint32_t img = rr * C + (uint32_t)cbase;   // element offset of this thread's first chunk in a dense tile image
     const uint32_t row0C = (r.row - rr) * C;         // element offset of the tile's first row in a dense tensor (low bits)
     // (the test is made warp-wide: the vote below needs every lane)
-    if (__any_sync(0xffffffffu, m_prog != prog || m_ncols != r.ncols || m_shift != shift)) {
+    if constexpr (FULL) {
+      const int nch = V >> lgW;
+      const bool ok = r.ncols > 0;
+      nvalid = ok ? V : 0;
+      hm = ok ? 0xffu : 0u;
+      partmask = 0u;
+      fullmask = ok ? ((nch >= 32) ? 0xffffffffu : ((1u << nch) - 1u)) : 0u;
+      all_valid = true;  // (a row past the end reduces whatever its slots hold: nobody reads the result)
+    } else if (__any_sync(0xffffffffu, m_prog != prog || m_ncols != r.ncols || m_shift != shift)) {
       m_prog = prog; m_ncols = r.ncols; m_shift = shift;
       // In mapping coordinates the row segment is [shift, shift + ncols); this thread owns chunks t, t + G, ...
       const int W = 1 << lgW;
