@@ -64,7 +64,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43) X(44) X(45) X(46)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43) X(44) X(45) X(46) X(47) X(48) X(49)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -88,8 +88,8 @@ const DvmVmVariant* dvm_vm_find_variant(int V, bool large, bool single, int ext,
 // Key of the occupancy cache: the variant and the dynamic shared memory in local-memory units.
 uint64_t dvm_occupancy_key(const DvmVmVariant* v, size_t smem) {
   const uint64_t id = (uint64_t)v->V | ((uint64_t)v->large << 8) | ((uint64_t)v->single << 9) | ((uint64_t)v->ext << 10) |
-                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 16) |  // (lean: three bits)
-                      ((uint64_t)v->ctas << 17);
+                      ((uint64_t)v->levels << 12) | ((uint64_t)v->lean << 13) | ((uint64_t)v->heavy << 17) |  // (lean: four bits)
+                      ((uint64_t)v->ctas << 18);
   return (id << 32) | (uint64_t)(smem / DVM_LOCAL_UNIT);
 }
 
@@ -745,7 +745,7 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     // every row fills the slots of the threads that hold it: columns = threads per row x elements per thread
     const bool full = c0[DVM_H_COL_BLOCKS] == 1 && c0[DVM_H_LAST_ROW_COLS] == c0[DVM_H_COLS] &&
                       c0[DVM_H_COLS] == ((uint32_t)V << (c0[DVM_H_GEOM] & 0xff));
-    const DvmVmVariant* v2 = (aligned && dense && full) ? dvm_vm_find_variant(V, large, true, 0, false, 7, heavy) : nullptr;
+    const DvmVmVariant* v2 = (aligned && full) ? dvm_vm_find_variant(V, large, true, 0, false, dense ? 7 : 8, heavy) : nullptr;
     if (!v2 && aligned) v2 = dvm_vm_find_variant(V, large, true, 0, false, dense ? 5 : 6, heavy);
     if (!v2 && dense) v2 = dvm_vm_find_variant(V, large, true, 0, false, 4, heavy);
     if (!v2) v2 = dvm_vm_find_variant(V, large, true, 0, false, 3, heavy);

@@ -8,13 +8,14 @@
 // per thread, compiled for three; groups 32..34: the one-program lean kernel with 16 / 32 / 24 elements per thread
 // for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
 // loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks; groups 41..43: two slots, aligned rows,
-// row-by-row copies allowed; groups 44..46: groups 38..40 for programs whose rows fill the tile's slots exactly.
+// row-by-row copies allowed; groups 44..46: groups 38..40 for programs whose rows fill the tile's slots exactly; groups 47..49: groups
+// 41..43 for such programs.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..46>"
+#error "compile with -DDVM_INST_GROUP=<0..49>"
 #endif
 
 namespace {
@@ -87,6 +88,12 @@ struct LeanOps {
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, true, true, true>::occupancy}
 
+// ... aligned programs with row-by-row copies whose rows fill the tile's slots exactly (lean = 8)
+#define DVM_LEAN_TWO_AL_FULL(V, LARGE, HEAVY)                                                                          \
+  {V, LARGE, 1, 0, 0, 8, HEAVY, 2,                                                                                     \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true, true>::launch,  \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true, true>::occupancy}
+
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::launch, \
@@ -121,6 +128,9 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP >= 47
+constexpr int GV = DVM_INST_GROUP == 47 ? 16 : (DVM_INST_GROUP == 48 ? 32 : 24);
+const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_AL_FULL(GV, 0, 0), DVM_LEAN_TWO_AL_FULL(GV, 0, 1), DVM_LEAN_TWO_AL_FULL(GV, 1, 0), DVM_LEAN_TWO_AL_FULL(GV, 1, 1)};
 #elif DVM_INST_GROUP >= 44
 constexpr int GV = DVM_INST_GROUP == 44 ? 16 : (DVM_INST_GROUP == 45 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_DENSE_AL_FULL(GV, 0, 0), DVM_LEAN_TWO_DENSE_AL_FULL(GV, 0, 1), DVM_LEAN_TWO_DENSE_AL_FULL(GV, 1, 0),

@@ -45,7 +45,8 @@ def test_dense_aligned_full_rows_and_what_moves_a_program_off_that_build():
 
 def test_row_by_row_copies_aligned_and_not():
     prog = wl.program_masked_softmax(128)
-    for S, want_lean in ((256, 6), (250, 3)):                       # the mask's rows are 512 / 500 bytes long
+    # the mask's rows are 512 bytes long and fill the slots exactly / 496 bytes: aligned, slots left empty / 500 bytes
+    for S, want_lean in ((256, 8), (248, 6), (250, 3)):
         sc = wl.randn((2, 32, S, S), torch.bfloat16, S).cuda()
         m = wl.causal_mask(S, "cuda")
         lean, _ = _run(prog, [sc, m])
