@@ -195,7 +195,8 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_lean_kernel(const __grid
   const bool use_queue = SINGLE ? false : prm.use_queue != 0;
   // one tile slot (DVM_F_ONE_SLOT, one-program launches): both slots are the same memory, a tile's loads start
   // when the previous tile is done; the SM's other CTA computes meanwhile
-  const bool one_slot = TWO ? false : (SINGLE && prm.levels == 2);
+  // (the builds for three resident CTAs only ever run one-slot launches: there the two-slot path folds away)
+  const bool one_slot = TWO ? false : (SINGLE && (CTAS == 3 || prm.levels == 2));
 #define CW(i) (prm.words[(i)])
 
   if (tid == 0) {
