@@ -232,7 +232,7 @@ void dvm_set_lean_kernel(int on);
  * general interpreter; 1 the lean one with every path; 2 its build for phased programs; 3 for two tile slots;
  * 4 ... and dense loads (no row-by-row copies, per-row scalar inputs, outer dims); 5 ... and aligned operands (no
  * realignment of reads); 6 two slots and aligned operands with row-by-row copies; 7 as 5 for rows that fill the
- * tile's slots exactly (no slot masks); 8 as 6 for such rows.  DVM_ERR_INVALID_ARG before the thread's first launch. */
+ * tile's slots exactly (no slot masks); 8 as 6 for such rows; 9 aligned programs with one tile slot.  DVM_ERR_INVALID_ARG before the thread's first launch. */
 int dvm_last_launch_variant(int out[8]);
 
 /* Matmul launches (Sec. 4.2, matrix operations): the tiles of a last, partial wave are shared along k -- a small

@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libdvm.so")
 SOURCES = ["dvm_host.cpp", "dvm_fuser.cpp", "dvm_launch.cu", "dvm_matmul.cu"]
-DVM_INST_GROUPS = 50
+DVM_INST_GROUPS = 51
 HEADERS = ["dvm_format.h", "dvm_internal.h", "dvm_launch.h", "dvm_vm.cuh", "dvm_math.cuh", "dvm_program.h",
            "dvm_vm_variants.h", "dvm_vm_lean.cuh", "dvm_link.h", os.path.join("..", "..", "include", "dvm.h"),
            os.path.join("..", "..", "include", "dvm_fuser.h")]

@@ -64,7 +64,7 @@ int dvm_device_state(DvmDeviceInfo* info) {
 }
 
 // The groups of interpreter variants (dvm_vm_inst.cu, compiled once per group).
-#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43) X(44) X(45) X(46) X(47) X(48) X(49)
+#define DVM_GROUPS(X) X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(33) X(34) X(35) X(36) X(37) X(38) X(39) X(40) X(41) X(42) X(43) X(44) X(45) X(46) X(47) X(48) X(49) X(50)
 #define DVM_DECL_GROUP(g) const DvmVmVariant* dvm_vm_group_##g(int* count);
 DVM_GROUPS(DVM_DECL_GROUP)
 #undef DVM_DECL_GROUP
@@ -736,6 +736,12 @@ int launch_vec(int n_programs, const void* const* codes, void* const* const* ten
     const DvmVmVariant* v3 = dvm_vm_find_variant(V, large, variant->single != 0, variant->ext, variant->levels != 0, variant->lean,
                                                  variant->heavy != 0, 3);
     if (v3) variant = v3;
+  }
+  if (lean == 1 && single && one_slot && variant && variant->ctas == 3) {
+    // one program with one tile slot on the build for three CTAs: its build for aligned programs
+    const uint32_t* c0 = (const uint32_t*)codes[0];
+    const DvmVmVariant* v9 = program_all_aligned(c0, tensors[0]) ? dvm_vm_find_variant(V, large, true, 0, false, 9, heavy, 3) : nullptr;
+    if (v9) variant = v9;
   }
   if (lean == 1 && single && !one_slot && variant) {
     // one program with two tile slots: the build without the one-slot path

@@ -9,13 +9,13 @@
 // for launches with two tile slots (its one-slot path compiled out); groups 35..37: the same for programs whose
 // loads are all one thread's; groups 38..40: ... and whose operands are all aligned like the tile's chunks; groups 41..43: two slots, aligned rows,
 // row-by-row copies allowed; groups 44..46: groups 38..40 for programs whose rows fill the tile's slots exactly; groups 47..49: groups
-// 41..43 for such programs.
+// 41..43 for such programs; group 50: group 31's kernel for aligned programs.
 #include "dvm_vm.cuh"
 #include "dvm_vm_lean.cuh"
 #include "dvm_vm_variants.h"
 
 #ifndef DVM_INST_GROUP
-#error "compile with -DDVM_INST_GROUP=<0..49>"
+#error "compile with -DDVM_INST_GROUP=<0..50>"
 #endif
 
 namespace {
@@ -94,6 +94,12 @@ struct LeanOps {
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true, true>::launch,  \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 2, true, false, true, true>::occupancy}
 
+// the one-program lean kernel compiled for three resident CTAs (one-slot programs) for aligned programs (lean = 9)
+#define DVM_LEAN3_AL(V, LARGE, HEAVY)                                                                       \
+  {V, LARGE, 1, 0, 0, 9, HEAVY, 3,                                                                                \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 3, false, false, true>::launch,   \
+   &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, true, (HEAVY) != 0, false, 3, false, false, true>::occupancy}
+
 #define DVM_LEAN(V, LARGE, SINGLE, HEAVY)                                                   \
   {V, LARGE, SINGLE, 0, 0, 1, HEAVY, 2,                                                     \
    &LeanOps<V, (LARGE) ? DVM_PW_LARGE : DVM_PW_SMALL, (SINGLE) != 0, (HEAVY) != 0>::launch, \
@@ -128,6 +134,8 @@ constexpr int GE = G3 % 3;
 const DvmVmVariant kGroup[] = {DVM_ENTRY3(GV, GL, GE)};
 #elif DVM_INST_GROUP == 31
 const DvmVmVariant kGroup[] = {DVM_LEAN3(16, 0, 0), DVM_LEAN3(16, 0, 1), DVM_LEAN3(16, 1, 0), DVM_LEAN3(16, 1, 1)};
+#elif DVM_INST_GROUP == 50
+const DvmVmVariant kGroup[] = {DVM_LEAN3_AL(16, 0, 0), DVM_LEAN3_AL(16, 0, 1), DVM_LEAN3_AL(16, 1, 0), DVM_LEAN3_AL(16, 1, 1)};
 #elif DVM_INST_GROUP >= 47
 constexpr int GV = DVM_INST_GROUP == 47 ? 16 : (DVM_INST_GROUP == 48 ? 32 : 24);
 const DvmVmVariant kGroup[] = {DVM_LEAN_TWO_AL_FULL(GV, 0, 0), DVM_LEAN_TWO_AL_FULL(GV, 0, 1), DVM_LEAN_TWO_AL_FULL(GV, 1, 0), DVM_LEAN_TWO_AL_FULL(GV, 1, 1)};

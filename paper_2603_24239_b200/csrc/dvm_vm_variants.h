@@ -21,7 +21,7 @@ struct DvmVmVariant {
                 // for programs whose loads are all one thread's (no row-by-row copies, per-row scalar inputs, outer dims);
                 // 5: that for programs all of whose operands are aligned like the tile's chunks (no realignment of reads);
                 // 6: two slots and aligned operands, row-by-row copies allowed; 7: as 5 for programs whose rows fill the
-                // tile's slots exactly (no slot masks); 8: as 6 for such programs
+                // tile's slots exactly (no slot masks); 8: as 6 for such programs; 9: aligned programs with one tile slot (three CTAs)
   int heavy;    // unary functions log / erf / tanh / sqrt / floor / round on tiles: 1 present, 0 absent (lean only)
   int ctas;     // resident CTAs per SM the kernel is compiled for: 2, or 3 (variants for one-slot launches)
   // launches the kernel; `params` points at a dvm::VMParams<PW> of the variant's block size

@@ -53,9 +53,16 @@ def test_row_by_row_copies_aligned_and_not():
         assert lean == want_lean
 
 
-def test_one_slot_program_keeps_the_general_lean_build():
+def test_one_slot_program_aligned_and_not():
     prog = wl.program_if_else_add()
     ins = [wl.randn((7, 33, 1000), torch.float32, 5 + i).cuda() for i in range(4)]
-    lean, _ = _run(prog, ins)
+    lean, _ = _run(prog, ins)                                       # one tile slot, three CTAs per SM, every tensor aligned
     v = dvm.last_launch_variant()
-    assert lean == 1 and v["single"] == 1
+    assert lean == 9 and v["single"] == 1 and v["ctas"] == 3
+    flat = [wl.randn((7 * 33 * 1000 + 8,), torch.float32, 15 + i).cuda() for i in range(4)]
+    ins = [flat[0][1:1 + 7 * 33 * 1000].view(7, 33, 1000)] + [t[:7 * 33 * 1000].view(7, 33, 1000) for t in flat[1:]]
+    lean, _ = _run(prog, ins)                                       # the first input starts 4 bytes off: reads are realigned
+    assert lean in (0, 1)
+    ins = [wl.randn((5, 31, 1001), torch.float32, 25 + i).cuda() for i in range(4)]
+    lean, _ = _run(prog, ins)                                       # an odd element count: whichever build, the oracle's result
+    assert lean in (0, 1, 9)
