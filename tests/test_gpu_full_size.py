@@ -116,3 +116,27 @@ def test_head_transpose_view_full_size_sampled(B, S):
         g1, g2 = gate_errors(wl.to_f64(out[r * D:(r + 1) * D]).reshape(1, D), want.reshape(1, D))
         assert g2 <= 2e-2, (r, g1, g2)
     assert not torch.isnan(out.float().sum())   # every element was written
+
+
+@pytest.mark.parametrize("shape", [(256, 512, 1024), (251, 509, 1049)])
+def test_if_else_add_full_size_sampled(shape):
+    """The if-else-add sweep at its size limit (2^27 elements per tensor; the second shape has an odd element
+    count): the one-slot launch on three CTAs per SM.  Sampled rows against the oracle one by one; 2x, 4x and
+    the add are exact or correctly rounded, so the whole output also equals its fp32 closed form bit for bit."""
+    b, s, f = shape
+    prog = wl.program_if_else_add()
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [shape] * 4)
+    ins = [wl.randn(shape, torch.float32, 70 + i, "cuda") for i in range(4)]
+    out = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
+    dvm.launch(code, ins + [out])
+    assert dvm.last_device_status() == 0
+    v = dvm.last_launch_variant()
+    assert v["single"] == 1 and v["ctas"] == 3 and v["lean"] == 9   # torch's allocations are 16-byte aligned
+    rows = _sample_rows(b * s, 150, 4, extra=[s - 1, s, b * s - 2])
+    sub = [t.reshape(-1, f)[torch.as_tensor(rows, device="cuda")].cpu() for t in ins]
+    want = orc.evaluate(prog.nodes, [wl.to_f64(x).reshape(1, len(rows), f) for x in sub])[0].reshape(len(rows), f)
+    got = wl.to_f64(out.reshape(-1, f)[torch.as_tensor(rows, device="cuda")])
+    assert float(np.max(np.abs(got - want) / np.maximum(np.abs(want), 1e-30))) <= 1e-6   # (the oracle does not round to fp32)
+    ref = torch.where(ins[0] > ins[1], 2 * ins[2], 4 * ins[2])
+    ref = (ref.double() + ins[3].double()).float()
+    assert torch.equal(out, ref)
