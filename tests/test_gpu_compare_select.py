@@ -170,3 +170,25 @@ def test_select_between_scalar_multiples_of_one_value(kind):
     want = oracle_run(p, ins)
     # one fp32 rounding per element on the device; the oracle's float64 product / sum is exact, rounded here
     assert np.array_equal(wl.to_f64(outs[0]), want[0].astype(np.float32).astype(np.float64))
+
+
+def test_if_else_add_misaligned_flat_tiles_wrap_around_on_one_slot():
+    """fp32 inputs that start 20, 16, 12 and 28 bytes into a 16-byte word, an output 24 bytes in: the flat tiles fill the
+    threads' whole capacity, so the first thread's head slots take the tile's last columns (wrap-around; the general
+    interpreter, one tile slot per CTA).  The wrapped columns are read one chunk past the thread's last -- and nothing
+    further: the last input's image ends the CTA's local memory.  960 tiles, results exact, storage around the
+    output untouched."""
+    shape, n = (24, 160, 1024), 24 * 160 * 1024
+    prog = wl.program_if_else_add()
+    code = dvm.encode(dvm.program_from_nodes(prog.nodes), [shape] * 4)
+    bases = [wl.randn((n + 16,), torch.float32, 90 + i, "cuda") for i in range(4)]
+    ins = [b[s:s + n].view(shape) for b, s in zip(bases, (5, 4, 3, 7))]
+    obase = torch.full((n + 16,), float("nan"), dtype=torch.float32, device="cuda")
+    out = obase[6:6 + n].view(shape)
+    dvm.launch(code, ins + [out])
+    assert dvm.last_device_status() == 0
+    v = dvm.last_launch_variant()
+    assert v["lean"] == 0 and v["ctas"] == 3        # wrap-around rows: the general interpreter, its build for one-slot launches
+    ref = (torch.where(ins[0] > ins[1], 2 * ins[2], 4 * ins[2]).double() + ins[3].double()).float()
+    assert torch.equal(out, ref)
+    assert torch.isnan(obase[:6]).all() and torch.isnan(obase[6 + n:]).all()
