@@ -658,7 +658,7 @@ __global__ void __launch_bounds__(THREADS, CTAS) dvm_vm_kernel(const __grid_cons
       } else {
         // second half of an 8-element chunk; with chunks of 4 the address would be the NEXT chunk's, a sixth chunk that no
         // image holds -- past the end of the CTA's local memory when the register is the slot's last
-        const uint4 v1 = c.lgW == 3 ? lds128_realign(wa + (r.a1 - r.a), r.mis) : make_uint4(0u, 0u, 0u, 0u);
+        const uint4 v1 = lds128_realign(wa + (c.lgW == 3 ? r.a1 - r.a : 0u), r.mis);  // (chunks of 4: the first half again, unused)
         e[0] = make_float2(__uint_as_float(v0.x), __uint_as_float(v0.y));
         e[1] = make_float2(__uint_as_float(v0.z), __uint_as_float(v0.w));
         e[2] = make_float2(__uint_as_float(v1.x), __uint_as_float(v1.y));
