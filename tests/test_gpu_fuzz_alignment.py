@@ -1,0 +1,92 @@
+"""Random shapes with every input and output starting a random number of elements into a 16-byte word: the four
+single-program sweeps' programs (if-else-add fp32, add + RMSNorm, masked softmax, the head-transpose view) against
+the oracle, on whichever interpreter build the launch picks -- small instances (one tile per CTA) and instances of
+hundreds to thousands of tiles (several tiles per CTA, both tile slots, wrap-around rows on the general interpreter).
+Storage around every output must stay untouched."""
+import collections
+
+import numpy as np
+import pytest
+import torch
+
+import dvm_workloads as wl
+import paper_2603_24239_b200 as dvm
+from tests.parity_util import TORCH_DT, check, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+def _shifted(shape, dtype, seed, sh):
+    n = int(np.prod(shape))
+    base = wl.randn((n + 16,), dtype, seed).cuda()
+    return base[sh:sh + n].view(*shape)
+
+
+def _guarded_out(shape, dtype, sh):
+    n = int(np.prod(shape))
+    base = torch.full((n + 16,), float("nan"), dtype=dtype, device="cuda")
+    return base, base[sh:sh + n].view(*shape)
+
+
+def _launch_and_check(prog, code, ins, outs, bases, shifts, want, seen):
+    dvm.launch(code, ins + outs)
+    assert dvm.last_device_status() == 0
+    v = dvm.last_launch_variant()
+    seen[(v["lean"], v["ctas"], v["V"])] += 1
+    check(prog, outs, want)
+    for base, out, sh in zip(bases, outs, shifts):
+        assert torch.isnan(base[:sh]).all() and torch.isnan(base[sh + out.numel():]).all()
+
+
+@pytest.mark.parametrize("seed,n_cases,big", [(1, 120, False), (2, 40, True)])
+def test_random_alignments_of_every_operand(seed, n_cases, big):
+    rng = np.random.default_rng(seed)
+    seen = collections.Counter()
+    for it in range(n_cases):
+        kind = int(rng.integers(0, 4))
+        aligned = rng.random() < 0.4     # a fair share of fully aligned cases
+
+        def sh():
+            return 0 if aligned else int(rng.integers(0, 8))
+        s0 = 1000 + 10 * it
+        if kind == 0:
+            shape = (int(rng.integers(1, 6)) * (8 if big else 1), int(rng.integers(1, 40)) * (8 if big else 1),
+                     int(rng.choice([8, 64, 1000, 1001, 1024, 4099, int(rng.integers(1, 3000))])))
+            prog = wl.program_if_else_add()
+            ins = [_shifted(shape, torch.float32, s0 + i, sh()) for i in range(4)]
+        elif kind == 1:
+            cols = int(rng.choice([4096, 4000, 4001, 2048, 1536, 1000, 264]))
+            rows = int(rng.integers(1, 70)) * (40 if big else 1)
+            prog = wl.program_add_rmsnorm(cols)
+            ins = [_shifted((rows, cols), torch.bfloat16, s0, sh()), _shifted((rows, cols), torch.bfloat16, s0 + 1, sh()),
+                   _shifted((cols,), torch.bfloat16, s0 + 2, sh())]
+        elif kind == 2:
+            S = int(rng.choice([256, 248, 250, 128, 512, 509, 384, int(rng.integers(17, 600))] + ([1024, 2048, 1236] if big else [])))
+            B, H = int(rng.integers(1, 3)), int(rng.integers(1, 5))
+            prog = wl.program_masked_softmax(128)
+            ins = [_shifted((B, H, S, S), torch.bfloat16, s0, sh()), wl.causal_mask(S, "cuda")]
+        else:
+            B, S, H, D = int(rng.integers(1, 3)), int(rng.integers(1, 300)) * (4 if big else 1), 32, 128
+            prog = wl.program_head_transpose_add()
+            n, shp = B * S * H * D, (B, H, S, D)
+            xs, y = _shifted((n,), torch.bfloat16, s0, sh()), _shifted((n,), torch.bfloat16, s0 + 1, sh())
+            code = dvm.encode(dvm.program_from_nodes(prog.nodes), [shp, shp], in_strides=[[S * H * D, D, H * D, 1], None])
+            so = sh()
+            base, out = _guarded_out((n,), torch.bfloat16, so)
+            want = oracle_run(prog, [xs.view(B, S, H, D).permute(0, 2, 1, 3).contiguous().cpu(), y.view(shp).cpu()])
+            try:
+                _launch_and_check(prog, code, [xs, y], [out], [base], [so], [w.reshape(-1) for w in want], seen)
+            except AssertionError as e:
+                raise AssertionError(f"case {it}: views {shp}: {e}") from e
+            continue
+        code = dvm.encode(dvm.program_from_nodes(prog.nodes), [tuple(t.shape) for t in ins])
+        shifts = [sh() for _ in prog.output_nodes]
+        pairs = [_guarded_out(shp, TORCH_DT[node[2]], s) for shp, node, s in zip(code.out_shapes, prog.output_nodes, shifts)]
+        want = oracle_run(prog, [t.cpu() for t in ins])
+        try:
+            _launch_and_check(prog, code, ins, [o for _, o in pairs], [b for b, _ in pairs], shifts, want, seen)
+        except AssertionError as e:
+            raise AssertionError(f"case {it}: {prog.name} {[tuple(t.shape) for t in ins]}: {e}") from e
+    # the sweep reached the lean builds and the general interpreter, on two and on three CTAs per SM
+    leans = {k[0] for k in seen}
+    assert {0, 1, 3, 4, 9} <= leans and any(k[1] == 3 for k in seen), dict(seen)
