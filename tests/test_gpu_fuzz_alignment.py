@@ -206,3 +206,30 @@ def test_random_alignments_of_long_rows_and_integer_outputs():
             else:
                 check(prog, [out], [w])
             assert _guards_ok(base, out, so), (it, prog.name)
+
+
+def test_random_alignments_of_matmul_epilogue_operands():
+    """addmm (Table 2) with its epilogue operand -- [m,n], [1,n] or [m,1] -- and its output at random element offsets
+    (the matrices A and B stay 16-byte aligned: the tile loads need that, and the launch refuses anything else)."""
+    from tests.parity_util import gate_errors
+    rng = np.random.default_rng(4)
+    prog = wl.program_addmm()
+    for it in range(50):
+        M = int(rng.choice([1, 7, 100, 128, 129, 300, 1000, int(rng.integers(1, 1500))]))
+        K, N = int(rng.choice([64, 256, 512, 1024])), int(rng.choice([64, 256, 264, 512, 1000, 1024]))
+        cshape = [(M, N), (1, N), (M, 1)][int(rng.integers(0, 3))]
+        sc, so = int(rng.integers(0, 8)), int(rng.integers(0, 8))
+        a = (wl.randn((M, K), torch.bfloat16, 100 + it) * 0.25).cuda()
+        b = (wl.randn((K, N), torch.bfloat16, 200 + it) * 0.25).cuda()
+        c = _shifted(cshape, torch.bfloat16, 300 + it, sc)
+        base, out = _guarded_out((M, N), torch.bfloat16, so)
+        code = dvm.encode(dvm.program_from_nodes(prog.nodes), [(M, K), (K, N), cshape])
+        dvm.launch(code, [a, b, c, out])
+        assert dvm.last_device_status() == 0
+        g1, _ = gate_errors(wl.to_f64(out), oracle_run(prog, [a.cpu(), b.cpu(), c.cpu()])[0])
+        assert g1 <= 2e-2, (it, M, K, N, cshape, sc, so, g1)
+        assert _guards_ok(base, out, so), (it, M, K, N, cshape, sc, so)
+    a = wl.randn((128 * 64 + 8,), torch.bfloat16, 1).cuda()[1:1 + 128 * 64].view(128, 64)   # A two bytes off: refused
+    with pytest.raises(dvm.DvmError):
+        dvm.launch(dvm.encode(dvm.program_from_nodes(wl.program_matmul().nodes), [(128, 64), (64, 64)]),
+                   [a, torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda"), torch.empty((128, 64), dtype=torch.bfloat16, device="cuda")])
